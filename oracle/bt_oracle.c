@@ -1,0 +1,197 @@
+/*
+ * bt_oracle.c -- TEST INFRASTRUCTURE ONLY (see bt_oracle.h).
+ *
+ * Every loop walks one element (one bit) at a time in the order the paper's
+ * Algorithms 1 and 2 state; there is no blocking, vectorisation or threading.
+ * Where the paper leaves a point open the reading taken is written beside it.
+ */
+#include "bt_oracle.h"
+#include <string.h>
+
+#define CHUNK_ELEMS 4096u
+
+int oracle_elem_size(int kind)
+{
+    switch (kind) {
+    case ORACLE_F32:  return 4;
+    case ORACLE_F16:  return 2;
+    case ORACLE_BF16: return 2;
+    case ORACLE_F64:  return 8;
+    default:          return 0;
+    }
+}
+
+/* "T[i] == 0" of Algorithm 1 is read as "every byte of the element is zero":
+ * -0.0, NaN, infinities and subnormals are non-zero and are stored verbatim,
+ * which is what makes the round trip bitwise lossless. */
+static int all_bytes_zero(const unsigned char *p, int elem_size)
+{
+    for (int b = 0; b < elem_size; ++b)
+        if (p[b] != 0) return 0;
+    return 1;
+}
+
+/* Algorithm 1: scan the flattened tensor; push a 0 bit for a zero, else push
+ * the element to the values vector and push a 1 bit. The chunk prefix entry is
+ * the count of values pushed so far, taken whenever i reaches a multiple of 4096. */
+uint64_t oracle_compress(const void *dense, uint64_t n, int elem_size,
+                         uint32_t *bitmap, void *values, uint64_t *prefix)
+{
+    const unsigned char *src = (const unsigned char *)dense;
+    unsigned char *val = (unsigned char *)values;
+    uint64_t words = (n + 31) / 32;
+    uint64_t j = 0;
+
+    for (uint64_t w = 0; w < words; ++w) bitmap[w] = 0;     /* padding bits stay 0 */
+
+    for (uint64_t i = 0; i < n; ++i) {                      /* half-open: 0 <= i < n */
+        if (i % CHUNK_ELEMS == 0) prefix[i / CHUNK_ELEMS] = j;
+        const unsigned char *e = src + i * (uint64_t)elem_size;
+        if (all_bytes_zero(e, elem_size)) {
+            /* push 0 bit: already 0 */
+        } else {
+            memcpy(val + j * (uint64_t)elem_size, e, (size_t)elem_size);   /* push T[i] */
+            j += 1;
+            bitmap[i >> 5] |= (uint32_t)1 << (i & 31);                     /* push 1 bit */
+        }
+    }
+    return j;
+}
+
+/* Algorithm 2: j = 0; for every bit, a set bit takes values[j] and advances j,
+ * a clear bit yields 0.0 (all-zero bytes in every precision). */
+void oracle_decompress(const uint32_t *bitmap, const void *values,
+                       uint64_t n, int elem_size, void *dense_out)
+{
+    const unsigned char *val = (const unsigned char *)values;
+    unsigned char *dst = (unsigned char *)dense_out;
+    uint64_t j = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        unsigned char *e = dst + i * (uint64_t)elem_size;
+        if ((bitmap[i >> 5] >> (i & 31)) & 1u) {
+            memcpy(e, val + j * (uint64_t)elem_size, (size_t)elem_size);
+            j += 1;
+        } else {
+            memset(e, 0, (size_t)elem_size);
+        }
+    }
+}
+
+void oracle_decompress_chunked(const uint32_t *bitmap, const void *values,
+                               const uint64_t *prefix, uint64_t n, int elem_size,
+                               void *dense_out)
+{
+    const unsigned char *val = (const unsigned char *)values;
+    unsigned char *dst = (unsigned char *)dense_out;
+    uint64_t chunks = (n + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
+    for (uint64_t c = 0; c < chunks; ++c) {
+        uint64_t j = prefix[c];                               /* restart the counter */
+        uint64_t lo = c * CHUNK_ELEMS;
+        uint64_t hi = lo + CHUNK_ELEMS < n ? lo + CHUNK_ELEMS : n;
+        for (uint64_t i = lo; i < hi; ++i) {
+            unsigned char *e = dst + i * (uint64_t)elem_size;
+            if ((bitmap[i >> 5] >> (i & 31)) & 1u) {
+                memcpy(e, val + j * (uint64_t)elem_size, (size_t)elem_size);
+                j += 1;
+            } else {
+                memset(e, 0, (size_t)elem_size);
+            }
+        }
+    }
+}
+
+/* binary16 -> binary32, exact (every half is representable as a float). */
+float oracle_half_to_float(uint16_t h)
+{
+    uint32_t sign = (uint32_t)(h >> 15) & 1u;
+    uint32_t expo = (uint32_t)(h >> 10) & 0x1Fu;
+    uint32_t mant = (uint32_t)h & 0x3FFu;
+    uint32_t out;
+    if (expo == 0x1Fu) {                       /* inf or NaN: keep the payload */
+        out = (sign << 31) | 0x7F800000u | (mant << 13);
+    } else if (expo != 0) {                    /* normal: rebias 15 -> 127 */
+        out = (sign << 31) | ((expo + 112u) << 23) | (mant << 13);
+    } else if (mant == 0) {                    /* signed zero */
+        out = sign << 31;
+    } else {                                   /* subnormal: value = mant * 2^-24 */
+        float f = (float)mant * (1.0f / 16777216.0f);
+        if (sign) f = -f;
+        return f;
+    }
+    float f;
+    memcpy(&f, &out, 4);
+    return f;
+}
+
+/* Is this element "<= 0" under IEEE comparison?  (false for NaN) */
+static int le_zero(const unsigned char *e, int kind)
+{
+    switch (kind) {
+    case ORACLE_F32: { float f; memcpy(&f, e, 4); return f <= 0.0f; }
+    case ORACLE_F64: { double d; memcpy(&d, e, 8); return d <= 0.0; }
+    case ORACLE_F16: { uint16_t h; memcpy(&h, e, 2); return oracle_half_to_float(h) <= 0.0f; }
+    case ORACLE_BF16: {                        /* bfloat16 is the top half of a binary32 */
+        uint16_t h; memcpy(&h, e, 2);
+        uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4);
+        return f <= 0.0f;
+    }
+    default: return 0;
+    }
+}
+
+/* ReLU is where the sparsity comes from (section 3.1); the activation is
+ * stashed in the forward pass (section 3.2).  y = (x <= 0) ? +0 : x, so -0,
+ * negatives and -inf become +0 (all-zero bytes), positives are raw copies and
+ * a NaN stays a NaN with its payload.  Then Algorithm 1 on y. */
+uint64_t oracle_relu_fwd_compress(const void *pre_act, uint64_t n, int kind,
+                                  void *y, uint32_t *bitmap, void *values,
+                                  uint64_t *prefix)
+{
+    int elem_size = oracle_elem_size(kind);
+    const unsigned char *src = (const unsigned char *)pre_act;
+    unsigned char *yo = (unsigned char *)y;
+    unsigned char *val = (unsigned char *)values;
+    uint64_t words = (n + 31) / 32;
+    uint64_t j = 0;
+    unsigned char act[8];
+
+    for (uint64_t w = 0; w < words; ++w) bitmap[w] = 0;
+
+    for (uint64_t i = 0; i < n; ++i) {
+        if (i % CHUNK_ELEMS == 0) prefix[i / CHUNK_ELEMS] = j;
+        const unsigned char *e = src + i * (uint64_t)elem_size;
+        if (le_zero(e, kind)) memset(act, 0, (size_t)elem_size);
+        else                  memcpy(act, e, (size_t)elem_size);
+        if (yo) memcpy(yo + i * (uint64_t)elem_size, act, (size_t)elem_size);
+        if (!all_bytes_zero(act, elem_size)) {
+            memcpy(val + j * (uint64_t)elem_size, act, (size_t)elem_size);
+            j += 1;
+            bitmap[i >> 5] |= (uint32_t)1 << (i & 31);
+        }
+    }
+    return j;
+}
+
+/* The ReLU gradient needs only the bitmap: a select, not a multiply, so that a
+ * masked lane is +0 whatever the upstream gradient holds (-x, inf, NaN). */
+void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
+                                 uint64_t n, int elem_size, void *grad_in)
+{
+    const unsigned char *g = (const unsigned char *)grad_out;
+    unsigned char *o = (unsigned char *)grad_in;
+    for (uint64_t i = 0; i < n; ++i) {
+        if ((bitmap[i >> 5] >> (i & 31)) & 1u)
+            memmove(o + i * (uint64_t)elem_size, g + i * (uint64_t)elem_size, (size_t)elem_size);
+        else
+            memset(o + i * (uint64_t)elem_size, 0, (size_t)elem_size);
+    }
+}
+
+/* M_b = elem_size * nnz + n/8 (section 3.2), with whole 32-bit bitmap words and
+ * the 8-byte-per-chunk prefix array this layout adds. */
+uint64_t oracle_compressed_bytes(uint64_t n, uint64_t nnz, int elem_size)
+{
+    uint64_t words  = (n + 31) / 32;
+    uint64_t chunks = (n + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
+    return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;
+}

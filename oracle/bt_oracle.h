@@ -1,0 +1,69 @@
+/*
+ * bt_oracle.h -- TEST INFRASTRUCTURE ONLY.
+ *
+ * Plain, slow, single-threaded CPU statement of the BitTrain sparse-bitmap
+ * codec (Algorithm 1 "Dense to Bitmap Matrix Compression" and Algorithm 2
+ * "Bitmap to Dense Matrix Decompression", section 3.3 of the paper) in the
+ * concrete layout this project fixes:
+ *
+ *   bitmap  : uint32 words, element i <-> word i>>5, bit i&31 (LSB first),
+ *             ceil(n/32) words, padding bits of the last word are 0
+ *   values  : the elements whose bit pattern is not all-zero, raw copies,
+ *             in flattened element order
+ *   prefix  : uint64, one entry per 4096-element chunk, prefix[c] = number of
+ *             non-zero elements in chunks 0..c-1 (exclusive, no trailing total)
+ *
+ * Nothing here shares code, headers or constants with the CUDA library; only
+ * tests, the smoke check and the CPU-baseline leg of the benchmark call it.
+ * All pointers are host pointers owned by the caller.
+ *
+ * Element kinds for the ReLU pair (the codec itself only needs the size):
+ */
+#ifndef BT_ORACLE_H
+#define BT_ORACLE_H
+#include <stdint.h>
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { ORACLE_F32 = 0, ORACLE_F16 = 1, ORACLE_BF16 = 2, ORACLE_F64 = 3 };
+
+/* bytes of one element of kind `kind`, 0 if the kind is unknown */
+int oracle_elem_size(int kind);
+
+/* Algorithm 1. elem_size in {2,4,8}. Returns nnz (also the number of values written). */
+uint64_t oracle_compress(const void *dense, uint64_t n, int elem_size,
+                         uint32_t *bitmap, void *values, uint64_t *prefix);
+
+/* Algorithm 2, literal: one running counter j over the whole bitmap. */
+void oracle_decompress(const uint32_t *bitmap, const void *values,
+                       uint64_t n, int elem_size, void *dense_out);
+
+/* Algorithm 2 restarted per chunk with j = prefix[c]: shows the prefix array
+ * alone is enough to decode chunks independently. */
+void oracle_decompress_chunked(const uint32_t *bitmap, const void *values,
+                               const uint64_t *prefix, uint64_t n, int elem_size,
+                               void *dense_out);
+
+/* y = (x <= 0) ? +0 : x with IEEE comparison (NaN kept with payload), then
+ * Algorithm 1 on y. y may be NULL. Returns nnz. */
+uint64_t oracle_relu_fwd_compress(const void *pre_act, uint64_t n, int kind,
+                                  void *y, uint32_t *bitmap, void *values,
+                                  uint64_t *prefix);
+
+/* grad_in[i] = bit i ? grad_out[i] (raw copy) : +0 */
+void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
+                                 uint64_t n, int elem_size, void *grad_in);
+
+/* M_b of section 3.2 generalised: bitmap words + values + prefix entries */
+uint64_t oracle_compressed_bytes(uint64_t n, uint64_t nnz, int elem_size);
+
+/* exact widening of one IEEE binary16 pattern to binary32 (used by the ReLU test) */
+float oracle_half_to_float(uint16_t h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif
