@@ -1,0 +1,140 @@
+/*
+ * bittrain.h -- C ABI of the sparse-bitmap activation codec for NVIDIA B200 (sm_100a).
+ *
+ * The method is BitTrain's stash format: in the forward pass a layer's (mostly
+ * zero, post-ReLU) activation is turned into a bitmap plus the vector of its
+ * non-zero elements, and in the backward pass it is turned back (paper,
+ * section 3.2 "Bitmap Format", Algorithm 1 and Algorithm 2).  The paper leaves
+ * the concrete layout open; this library fixes it as
+ *
+ *   bitmap       uint32 words; element i <-> word i>>5, bit i&31 (LSB first);
+ *                ceil(n/32) words; unused high bits of the last word are 0
+ *   values       the elements whose bit pattern is not all-zero, copied
+ *                verbatim, in flattened (row-major) element order; nnz entries
+ *   chunk_prefix uint64; one entry per 4096-element chunk; entry c is the
+ *                number of non-zero elements before chunk c (exclusive; entry
+ *                0 is 0; there is no trailing total).  It replaces the single
+ *                running counter j of Algorithm 2 so that chunks decode
+ *                independently.
+ *
+ * "Zero" means an all-zero bit pattern: -0.0, NaN, infinities and subnormals
+ * are kept, so decompress(compress(x)) is x bit for bit.
+ *
+ * General rules for every call below
+ *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
+ *     The caller owns every buffer; the library allocates nothing, keeps no
+ *     state between calls, and neither synchronises nor prints.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL
+ *     for the default stream) on the current device.
+ *   - Tensors are flat contiguous arrays of n elements (Algorithm 1 flattens
+ *     the tensor first; the shape is the caller's metadata).
+ *   - dense / values / y / gradient pointers and the bitmap pointer must be
+ *     16-byte aligned, chunk_prefix and nnz_out 8-byte aligned.
+ *   - The return value reports what the host can see: BT_OK, an argument
+ *     error (nothing was launched), or BT_ERR_CUDA if the launch itself
+ *     failed.  Conditions only the device can see are written to *dev_status
+ *     (when that pointer is not NULL).
+ *   - n == 0 is valid: *nnz_out = 0 and *dev_status = BT_OK are written,
+ *     nothing else is touched.
+ *   - Buffers of one call must not overlap, except where a parameter says it
+ *     may alias another.
+ */
+#ifndef BITTRAIN_H
+#define BITTRAIN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BT_CHUNK_ELEMS 4096u
+
+/* element types: the codec proper only needs the width, the ReLU pair the format */
+enum { BT_F32 = 0, BT_F16 = 1, BT_BF16 = 2 };
+
+enum {
+    BT_OK = 0,
+    BT_ERR_NULL = 1,       /* a required pointer is NULL                               */
+    BT_ERR_DTYPE = 2,      /* unknown element type                                     */
+    BT_ERR_ALIGN = 3,      /* a pointer breaks the alignment rule above                */
+    BT_ERR_WORKSPACE = 4,  /* workspace smaller than bt_workspace_bytes(n)             */
+    BT_ERR_CAPACITY = 5,   /* device: nnz > values_capacity (see bt_compress)          */
+    BT_ERR_TIMEOUT = 6,    /* device: a bounded wait inside the kernel ran out         */
+    BT_ERR_CUDA = 7        /* the CUDA runtime reported an error at launch             */
+};
+
+/*
+ * Size in bytes of the compressed form: 4*ceil(n/32) + nnz*sizeof(dtype) +
+ * 8*ceil(n/4096).  This is M_b of section 3.2 (element bytes times the
+ * non-zero count plus one bit per element) with whole bitmap words and the
+ * chunk prefix array added.  Pure host arithmetic; returns 0 for an unknown
+ * dtype.
+ */
+size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype);
+
+/*
+ * Bytes of device scratch bt_compress / bt_relu_fwd_compress need for n
+ * elements (the tile descriptors of the single-pass scan plus a small header).
+ * The contents need no initialisation and are unspecified after a call.  Two
+ * calls that run concurrently must not share a workspace.  No counterpart in
+ * the paper (its scan is sequential).
+ */
+size_t bt_workspace_bytes(uint64_t n);
+
+/*
+ * Algorithm 1 (dense -> bitmap).  Reads dense[0..n), writes bitmap
+ * (ceil(n/32) words), values[0..nnz), chunk_prefix (ceil(n/4096) entries) and
+ * *nnz_out.  values_capacity is the number of ELEMENTS the values buffer can
+ * hold; n always suffices.  If nnz exceeds it, stores past the capacity are
+ * suppressed, bitmap, chunk_prefix and *nnz_out are still complete and
+ * correct, and *dev_status = BT_ERR_CAPACITY, so the caller can run again with
+ * a buffer of nnz elements.  values[nnz..capacity) is left untouched or
+ * unspecified.  *dev_status = BT_ERR_TIMEOUT means an internal bounded wait
+ * gave up and every output is undefined.
+ */
+int bt_compress(const void *dense, uint64_t n, int dtype,
+                uint32_t *bitmap, void *values, uint64_t values_capacity,
+                uint64_t *chunk_prefix, uint64_t *nnz_out,
+                void *workspace, size_t workspace_bytes,
+                int32_t *dev_status, void *stream);
+
+/*
+ * Algorithm 2 (bitmap -> dense).  dense_out[i] = bit i set ? the next value :
+ * all-zero bits.  Chunks are decoded independently from chunk_prefix; values
+ * must hold at least the nnz elements the bitmap calls for.
+ */
+int bt_decompress(const uint32_t *bitmap, const void *values,
+                  const uint64_t *chunk_prefix, uint64_t n, int dtype,
+                  void *dense_out, void *stream);
+
+/*
+ * ReLU forward fused with Algorithm 1: y[i] = (x[i] <= 0) ? +0 : x[i] under
+ * IEEE comparison (so -0, negatives and -inf give +0 and a NaN passes through
+ * with its payload), and y is stashed in compressed form in the same pass
+ * (ReLU is the source of the sparsity, section 3.1; the activation is saved in
+ * the forward pass, section 3.2).  y_out may be NULL (only the stash is
+ * written) and may alias pre_act (in-place ReLU).  Other parameters as
+ * bt_compress.
+ */
+int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out,
+                         uint32_t *bitmap, void *values, uint64_t values_capacity,
+                         uint64_t *chunk_prefix, uint64_t *nnz_out,
+                         void *workspace, size_t workspace_bytes,
+                         int32_t *dev_status, void *stream);
+
+/*
+ * ReLU backward from the stash: grad_in[i] = bit i set ? grad_out[i] : +0.
+ * The backward pass restores activations to form gradients (section 3.2); for
+ * ReLU itself only the bitmap is needed.  A select, not a multiply: masked
+ * lanes are +0 even where grad_out is negative, infinite or NaN.  grad_in may
+ * alias grad_out.
+ */
+int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
+                            uint64_t n, int dtype, void *grad_in, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITTRAIN_H */

@@ -1,0 +1,157 @@
+"""Thin ctypes binding of libbittrain.so: same names as the C ABI, argument
+marshalling only.  Every step of the codec runs in the library's CUDA kernels;
+there is no fallback: if the shared object is missing this module raises.
+
+Tensors are torch CUDA tensors (device memory and streams are torch's); the
+functions pass their data pointers, the element count and the current stream.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+BT_F32, BT_F16, BT_BF16 = 0, 1, 2
+BT_OK, BT_ERR_NULL, BT_ERR_DTYPE, BT_ERR_ALIGN, BT_ERR_WORKSPACE, BT_ERR_CAPACITY, BT_ERR_TIMEOUT, BT_ERR_CUDA = range(8)
+STATUS_NAMES = ["BT_OK", "BT_ERR_NULL", "BT_ERR_DTYPE", "BT_ERR_ALIGN", "BT_ERR_WORKSPACE", "BT_ERR_CAPACITY",
+                "BT_ERR_TIMEOUT", "BT_ERR_CUDA"]
+CHUNK = 4096
+
+DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_BF16}
+EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
+           "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap")
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class BitTrainError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{call} returned {name}")
+        self.status = status
+
+
+def library_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """Load libbittrain.so (built in-tree by build.build_library()).  No fallback."""
+    global _lib
+    if _lib is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: build it with "
+                              "`python -m paper_2110_15362_b200.build` (needs nvcc); there is no CPU fallback")
+        L = ctypes.CDLL(path)
+        u64, vp, i32, sz = ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.bt_compressed_bytes.restype = sz
+        L.bt_compressed_bytes.argtypes = [u64, u64, i32]
+        L.bt_workspace_bytes.restype = sz
+        L.bt_workspace_bytes.argtypes = [u64]
+        L.bt_compress.restype = i32
+        L.bt_compress.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_decompress.restype = i32
+        L.bt_decompress.argtypes = [vp, vp, vp, u64, i32, vp, vp]
+        L.bt_relu_fwd_compress.restype = i32
+        L.bt_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_relu_bwd_from_bitmap.restype = i32
+        L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(call: str, status: int, check: bool) -> int:
+    if check and status != BT_OK:
+        raise BitTrainError(call, status)
+    return status
+
+
+def bt_compressed_bytes(n: int, nnz: int, dtype) -> int:
+    code = DTYPE_CODE.get(dtype, dtype)
+    return int(lib().bt_compressed_bytes(n, nnz, code))
+
+
+def bt_workspace_bytes(n: int) -> int:
+    return int(lib().bt_workspace_bytes(n))
+
+
+def bt_compress(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,
+                nnz_out: torch.Tensor, workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                *, n: Optional[int] = None, values_capacity: Optional[int] = None, stream=None,
+                check: bool = True) -> int:
+    n = dense.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    st = lib().bt_compress(_ptr(dense), n, DTYPE_CODE[dense.dtype], _ptr(bitmap), _ptr(values), cap,
+                           _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace),
+                           workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream))
+    return _check("bt_compress", st, check)
+
+
+def bt_relu_fwd_compress(pre_act: torch.Tensor, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
+                         values: torch.Tensor, chunk_prefix: torch.Tensor, nnz_out: torch.Tensor,
+                         workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                         *, n: Optional[int] = None, values_capacity: Optional[int] = None, stream=None,
+                         check: bool = True) -> int:
+    n = pre_act.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    st = lib().bt_relu_fwd_compress(_ptr(pre_act), n, DTYPE_CODE[pre_act.dtype], _ptr(y_out), _ptr(bitmap),
+                                    _ptr(values), cap, _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _ptr(dev_status),
+                                    _stream(stream))
+    return _check("bt_relu_fwd_compress", st, check)
+
+
+def bt_decompress(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor, dense_out: torch.Tensor,
+                  *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    n = dense_out.numel() if n is None else n
+    st = lib().bt_decompress(_ptr(bitmap), _ptr(values), _ptr(chunk_prefix), n, DTYPE_CODE[dense_out.dtype],
+                             _ptr(dense_out), _stream(stream))
+    return _check("bt_decompress", st, check)
+
+
+def bt_relu_bwd_from_bitmap(bitmap: torch.Tensor, grad_out: torch.Tensor, grad_in: torch.Tensor,
+                            *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    n = grad_out.numel() if n is None else n
+    st = lib().bt_relu_bwd_from_bitmap(_ptr(bitmap), _ptr(grad_out), n, DTYPE_CODE[grad_out.dtype], _ptr(grad_in),
+                                       _stream(stream))
+    return _check("bt_relu_bwd_from_bitmap", st, check)
+
+
+class Stash:
+    """Device buffers for one compressed tensor (allocation helper, no arithmetic)."""
+
+    def __init__(self, n: int, dtype: torch.dtype, device="cuda", values_capacity: Optional[int] = None):
+        self.n, self.dtype = n, dtype
+        cap = n if values_capacity is None else values_capacity
+        self.bitmap = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
+        self.values = torch.empty(cap, dtype=dtype, device=device)
+        self.chunk_prefix = torch.empty((n + CHUNK - 1) // CHUNK, dtype=torch.int64, device=device)
+        self.nnz_out = torch.empty(1, dtype=torch.int64, device=device)
+        self.dev_status = torch.empty(1, dtype=torch.int32, device=device)
+
+    @property
+    def nnz(self) -> int:
+        return int(self.nnz_out.item())
+
+    @property
+    def status(self) -> int:
+        return int(self.dev_status.item())
+
+
+def new_workspace(n: int, device="cuda") -> torch.Tensor:
+    return torch.empty(bt_workspace_bytes(n), dtype=torch.uint8, device=device)

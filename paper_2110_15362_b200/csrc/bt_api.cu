@@ -1,0 +1,116 @@
+// The extern "C" boundary: argument checks on the host, then one launch.
+#include "bt_internal.cuh"
+
+namespace {
+
+inline int elem_size_of(int dtype)
+{
+    switch (dtype) {
+    case BT_F32: return 4;
+    case BT_F16: return 2;
+    case BT_BF16: return 2;
+    default: return 0;
+    }
+}
+
+inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+inline uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+
+int compress_common(const void *src, uint64_t n, int dtype, bool relu, void *y, uint32_t *bitmap, void *values,
+                    uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
+                    size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    if (elem_size_of(dtype) == 0) return BT_ERR_DTYPE;
+    if (!nnz_out) return BT_ERR_NULL;
+    if (!aligned(nnz_out, 8) || !aligned(dev_status, 4)) return BT_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (n == 0) {
+        if (cudaMemsetAsync(nnz_out, 0, sizeof(uint64_t), s) != cudaSuccess) return BT_ERR_CUDA;
+        if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), s) != cudaSuccess) return BT_ERR_CUDA;
+        return BT_OK;
+    }
+    if (!src || !bitmap || !chunk_prefix || !workspace) return BT_ERR_NULL;
+    if (!values && values_capacity != 0) return BT_ERR_NULL;
+    if (!aligned(src, 16) || !aligned(y, 16) || !aligned(bitmap, 16) || !aligned(values, 16) ||
+        !aligned(chunk_prefix, 8) || !aligned(workspace, 16))
+        return BT_ERR_ALIGN;
+    if (workspace_bytes < bt_workspace_bytes(n)) return BT_ERR_WORKSPACE;
+
+    bt::CompressArgs a;
+    a.src        = src;
+    a.y          = y;
+    a.bitmap     = bitmap;
+    a.values     = values;
+    a.capacity   = values_capacity;
+    a.prefix     = chunk_prefix;
+    a.nnz_out    = nnz_out;
+    a.dev_status = dev_status;
+    a.ws_header  = static_cast<uint32_t *>(workspace);
+    a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
+    a.n          = n;
+    return bt::launch_compress(a, dtype, relu, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return 0;
+    return static_cast<size_t>(4 * ceil_div(n, 32) + nnz * static_cast<uint64_t>(es) + 8 * ceil_div(n, BT_CHUNK_ELEMS));
+}
+
+size_t bt_workspace_bytes(uint64_t n)
+{
+    return bt::kWsHeaderBytes + 8 * static_cast<size_t>(ceil_div(n, bt::kMinTileElems));
+}
+
+int bt_compress(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void *values, uint64_t values_capacity,
+                uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace, size_t workspace_bytes,
+                int32_t *dev_status, void *stream)
+{
+    return compress_common(dense, n, dtype, false, nullptr, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream);
+}
+
+int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out, uint32_t *bitmap, void *values,
+                         uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
+                         size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    return compress_common(pre_act, n, dtype, true, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream);
+}
+
+int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix, uint64_t n, int dtype,
+                  void *dense_out, void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !chunk_prefix || !dense_out) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
+        return BT_ERR_ALIGN;
+    // values may be NULL only when the bitmap has no set bit; the kernel then never reads it
+    return bt::launch_decompress(bitmap, values, chunk_prefix, n, es, dense_out, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
+int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out, uint64_t n, int dtype, void *grad_in,
+                            void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !grad_out || !grad_in) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(grad_out, 16) || !aligned(grad_in, 16)) return BT_ERR_ALIGN;
+    return bt::launch_relu_bwd(bitmap, grad_out, n, es, grad_in, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,165 @@
+// Shared declarations of the CUDA side of the codec: launcher prototypes, the
+// workspace layout and thin wrappers over the sm_100a PTX the kernels use
+// (mbarrier, 1-D bulk async copies, relaxed device-scope loads and stores).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bittrain.h"
+
+namespace bt {
+
+// ---------------------------------------------------------------- workspace layout
+// [0]   uint32  ticket     next tile to hand out
+// [1]   uint32  abort      set once a bounded wait ran out; every CTA then leaves
+// [2..] reserved
+// then one 64-bit descriptor per tile: (value << 2) | state
+constexpr size_t   kWsHeaderBytes = 256;
+constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;   // descriptors are sized for the smallest tile
+constexpr uint64_t kStateInvalid = 0, kStateAggregate = 1, kStateInclusive = 2;
+
+struct CompressArgs {
+    const void *src;        // dense input (pre-activation for the fused form)
+    void       *y;          // optional dense ReLU output
+    uint32_t   *bitmap;
+    void       *values;
+    uint64_t    capacity;   // in elements
+    uint64_t   *prefix;
+    uint64_t   *nnz_out;
+    int32_t    *dev_status;
+    uint32_t   *ws_header;
+    uint64_t   *ws_desc;
+    uint64_t    n;
+};
+
+cudaError_t launch_compress(const CompressArgs &a, int dtype, bool relu, cudaStream_t s);
+cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *prefix,
+                              uint64_t n, int elem_size, void *out, cudaStream_t s);
+cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size,
+                            void *gin, cudaStream_t s);
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+
+// makes the barrier initialisation and earlier generic-proxy shared-memory
+// writes visible to the async proxy (the bulk-copy engine)
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// 1-D bulk async copy global -> this CTA's shared memory, completing on an mbarrier.
+// Both addresses 16-byte aligned, bytes a non-zero multiple of 16.
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gmem_src, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_addr(smem_dst)),
+        "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
+        : "memory");
+}
+
+// 1-D bulk async copy this CTA's shared memory -> global (bulk-group completion).
+__device__ __forceinline__ void bulk_store(void *gmem_dst, const void *smem_src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst),
+                 "r"(smem_addr(smem_src)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_all()
+{
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t *p)
+{
+    uint64_t v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(uint64_t *p, uint64_t v)
+{
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_u32(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
+__device__ __forceinline__ uint32_t lanemask_lt()
+{
+    uint32_t m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+// ---------------------------------------------------------------- ReLU on bit patterns
+// keep(x) = !(x <= 0) under IEEE comparison: positive (non-zero magnitude, sign
+// clear) or NaN (magnitude above the exponent mask, either sign).
+template <int DT>
+struct ReluKeep;
+template <>
+struct ReluKeep<BT_F32> {
+    __device__ static __forceinline__ bool keep(uint32_t u)
+    {
+        return (static_cast<int32_t>(u) > 0) | (u > 0xFF800000u);
+    }
+};
+template <>
+struct ReluKeep<BT_F16> {
+    __device__ static __forceinline__ bool keep(uint32_t u)   // u holds a 16-bit pattern
+    {
+        return ((u - 1u) < 0x7FFFu) | (u > 0xFC00u);
+    }
+};
+template <>
+struct ReluKeep<BT_BF16> {
+    __device__ static __forceinline__ bool keep(uint32_t u)
+    {
+        return ((u - 1u) < 0x7FFFu) | (u > 0xFF80u);
+    }
+};
+
+}  // namespace bt

@@ -1,0 +1,99 @@
+// ReLU backward from the stashed bitmap: grad_in[i] = bit i ? grad_out[i] : +0.
+// A pure streaming select: every thread moves 16-byte vectors (4 fp32 or 8
+// 16-bit elements, i.e. 4 or 8 consecutive bits of one bitmap word), several
+// independent vectors in flight per thread.
+#include "bt_internal.cuh"
+
+namespace bt {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll  = 4;   // independent 16-byte vectors per thread
+
+template <typename U>
+__device__ __forceinline__ uint4 select_vec(uint4 g, uint32_t bits);
+
+template <>
+__device__ __forceinline__ uint4 select_vec<uint32_t>(uint4 g, uint32_t bits)
+{
+    g.x = (bits & 1u) ? g.x : 0u;
+    g.y = (bits & 2u) ? g.y : 0u;
+    g.z = (bits & 4u) ? g.z : 0u;
+    g.w = (bits & 8u) ? g.w : 0u;
+    return g;
+}
+
+// two 16-bit lanes per register: build a byte-pair mask from two bits
+__device__ __forceinline__ uint32_t mask2(uint32_t two_bits)
+{
+    return ((two_bits & 1u) ? 0x0000FFFFu : 0u) | ((two_bits & 2u) ? 0xFFFF0000u : 0u);
+}
+
+template <>
+__device__ __forceinline__ uint4 select_vec<uint16_t>(uint4 g, uint32_t bits)
+{
+    g.x &= mask2(bits);
+    g.y &= mask2(bits >> 2);
+    g.z &= mask2(bits >> 4);
+    g.w &= mask2(bits >> 6);
+    return g;
+}
+
+template <typename U>
+__global__ void __launch_bounds__(kThreads)
+relu_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *gout, const uint64_t n, U *gin)
+{
+    constexpr int      kVec  = 16 / sizeof(U);
+    constexpr uint32_t kMask = (1u << kVec) - 1u;
+    const uint64_t vecs      = n / kVec;                       // whole 16-byte vectors
+    const uint64_t block0    = static_cast<uint64_t>(blockIdx.x) * (kThreads * kUnroll);
+
+    uint4    g[kUnroll];
+    uint32_t w[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const uint64_t v = block0 + u * kThreads + threadIdx.x;
+        if (v < vecs) {
+            g[u] = reinterpret_cast<const uint4 *>(gout)[v];
+            w[u] = bitmap[(v * kVec) >> 5];
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const uint64_t v = block0 + u * kThreads + threadIdx.x;
+        if (v < vecs) {
+            const uint32_t bits = (w[u] >> ((v * kVec) & 31u)) & kMask;
+            reinterpret_cast<uint4 *>(gin)[v] = select_vec<U>(g[u], bits);
+        }
+    }
+    // the last n % kVec elements, one by one
+    if (blockIdx.x == 0 && threadIdx.x < n - vecs * kVec) {
+        const uint64_t i = vecs * kVec + threadIdx.x;
+        const bool set   = (bitmap[i >> 5] >> (i & 31u)) & 1u;
+        gin[i]           = set ? gout[i] : U(0);
+    }
+}
+
+template <typename U>
+cudaError_t launch_typed(const uint32_t *bitmap, const void *gout, uint64_t n, void *gin, cudaStream_t stream)
+{
+    constexpr int  kVec = 16 / sizeof(U);
+    const uint64_t vecs = n / kVec;
+    uint64_t       grid = (vecs + kThreads * kUnroll - 1) / (kThreads * kUnroll);
+    if (grid == 0) grid = 1;
+    if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    relu_bwd_kernel<U><<<static_cast<unsigned>(grid), kThreads, 0, stream>>>(bitmap, static_cast<const U *>(gout), n,
+                                                                             static_cast<U *>(gin));
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size, void *gin,
+                            cudaStream_t stream)
+{
+    return elem_size == 4 ? launch_typed<uint32_t>(bitmap, gout, n, gin, stream)
+                          : launch_typed<uint16_t>(bitmap, gout, n, gin, stream);
+}
+
+}  // namespace bt

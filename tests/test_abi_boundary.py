@@ -1,0 +1,92 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports
+every symbol the header declares, and its host arithmetic and argument checks
+behave as documented (no kernel is launched on an argument error)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2110_15362_b200 import binding as B
+from paper_2110_15362_b200 import build
+
+HEADER = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "bittrain.h")
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build_library()
+    return B.lib()
+
+
+def declared_functions():
+    text = re.sub(r"/\*.*?\*/", "", open(HEADER).read(), flags=re.S)
+    return sorted(set(re.findall(r"\b(bt_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = declared_functions()
+    assert set(B.EXPORTS) <= set(names) and len(names) >= 6
+    for name in names:
+        assert hasattr(L, name), name
+
+
+def test_compressed_bytes_closed_form(L, oracle):
+    for dt, es in ((B.BT_F32, 4), (B.BT_F16, 2), (B.BT_BF16, 2)):
+        for n, nnz in ((0, 0), (1, 1), (31, 7), (32, 32), (33, 0), (4096, 100), (4097, 4097), (200704, 100352),
+                       (1 << 28, 1 << 27), (3 * 4096 + 17, 12)):
+            got = L.bt_compressed_bytes(n, nnz, dt)
+            assert got == 4 * ((n + 31) // 32) + nnz * es + 8 * ((n + 4095) // 4096)
+            assert got == oracle.compressed_bytes(n, nnz, es)
+            if n % 32 == 0:
+                assert got == n // 8 + nnz * es + 8 * ((n + 4095) // 4096)
+    assert L.bt_compressed_bytes(100, 10, 99) == 0
+    assert L.bt_compressed_bytes(200704, 100352, B.BT_F32) == 426888
+
+
+def test_workspace_bytes_grows_with_n(L):
+    assert L.bt_workspace_bytes(0) > 0
+    assert L.bt_workspace_bytes(1 << 28) >= 8 * ((1 << 28) // 8192)
+    assert L.bt_workspace_bytes(1 << 20) <= L.bt_workspace_bytes(1 << 21)
+
+
+def test_argument_errors_are_reported_before_any_launch(L):
+    # 16-byte aligned fake addresses: never dereferenced, because every call below fails its checks first
+    A = 0x10000
+    ws = L.bt_workspace_bytes(8192)
+    ok_args = dict(dense=A, n=8192, dt=B.BT_F32, bitmap=A, values=A, cap=8192, prefix=A, nnz=A, ws=A, wsb=ws,
+                   status=A, stream=None)
+
+    def call(**kw):
+        a = dict(ok_args, **kw)
+        return L.bt_compress(a["dense"], a["n"], a["dt"], a["bitmap"], a["values"], a["cap"], a["prefix"], a["nnz"],
+                             a["ws"], a["wsb"], a["status"], a["stream"])
+
+    assert call(dt=7) == B.BT_ERR_DTYPE
+    assert call(dense=None) == B.BT_ERR_NULL
+    assert call(bitmap=None) == B.BT_ERR_NULL
+    assert call(prefix=None) == B.BT_ERR_NULL
+    assert call(nnz=None) == B.BT_ERR_NULL
+    assert call(ws=None) == B.BT_ERR_NULL
+    assert call(values=None) == B.BT_ERR_NULL
+    assert call(dense=A + 4) == B.BT_ERR_ALIGN
+    assert call(values=A + 8) == B.BT_ERR_ALIGN
+    assert call(prefix=A + 4) == B.BT_ERR_ALIGN
+    assert call(nnz=A + 4) == B.BT_ERR_ALIGN
+    assert call(wsb=ws - 1) == B.BT_ERR_WORKSPACE
+    assert L.bt_decompress(A, A, A, 10, 9, A, None) == B.BT_ERR_DTYPE
+    assert L.bt_decompress(None, A, A, 10, B.BT_F16, A, None) == B.BT_ERR_NULL
+    assert L.bt_decompress(A, A, A, 10, B.BT_F16, A + 2, None) == B.BT_ERR_ALIGN
+    assert L.bt_decompress(A, A, A, 0, B.BT_F16, None, None) == B.BT_OK          # n == 0 touches nothing
+    assert L.bt_relu_bwd_from_bitmap(A, None, 10, B.BT_F32, A, None) == B.BT_ERR_NULL
+    assert L.bt_relu_bwd_from_bitmap(A, A, 10, 5, A, None) == B.BT_ERR_DTYPE
+    assert L.bt_relu_bwd_from_bitmap(A, A + 2, 10, B.BT_BF16, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_relu_bwd_from_bitmap(None, None, 0, B.BT_BF16, None, None) == B.BT_OK
+    assert L.bt_relu_fwd_compress(A, 8192, B.BT_F32, A + 4, A, A, 8192, A, A, A, ws, A, None) == B.BT_ERR_ALIGN
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "library_path", lambda: str(tmp_path / "nope.so"))
+    with pytest.raises(ImportError):
+        B.lib()

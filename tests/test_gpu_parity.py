@@ -1,0 +1,141 @@
+"""GPU parity: every output of every C-ABI entry point, bit for bit, against the
+CPU oracle on the same seeded inputs.  All calls go through the ctypes binding
+of libbittrain.so."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2110_15362_b200 import binding as B
+from paper_2110_15362_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+KINDS = ["f32", "f16", "bf16"]
+SIZES = list(W.EDGE_SIZES) + [200704, 8192 * 37 + 5, 1 << 20]
+
+
+@pytest.fixture(scope="module")
+def G():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from tests import gpu_util
+    B.lib()
+    return gpu_util
+
+
+def assert_same_compressed(g, c):
+    assert g.guards_ok
+    assert g.status == B.BT_OK
+    assert g.nnz == c.nnz
+    assert np.array_equal(g.bitmap, c.bitmap)
+    assert np.array_equal(g.prefix, c.prefix)
+    assert np.array_equal(g.values, c.values)
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("n", SIZES)
+def test_compress_decompress_edge_sizes(G, oracle, kind, n):
+    x = W.random_patterns(n, kind, 0.5, seed=1000 + n)
+    c = oracle.compress(x)
+    g = G.gpu_compress(G.from_raw(x, kind))
+    assert_same_compressed(g, c)
+    out, ok = G.gpu_decompress(c.bitmap, c.values, c.prefix, n, kind)
+    assert ok and np.array_equal(out, x)
+    assert B.bt_compressed_bytes(n, g.nnz, G.TDT[kind]) == oracle.compressed_bytes(n, c.nnz, x.dtype.itemsize)
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("zf", [0.0, 0.25, 0.9, 0.99, 1.0])
+def test_compress_decompress_sparsity_levels(G, oracle, kind, zf):
+    n = 8192 * 301 + 4097 + 13        # many tiles per CTA is not reached here, many CTAs are; ragged tail
+    x = W.random_patterns(n, kind, zf, seed=int(zf * 100) + 5)
+    c = oracle.compress(x)
+    g = G.gpu_compress(G.from_raw(x, kind))
+    assert_same_compressed(g, c)
+    out, ok = G.gpu_decompress(g.bitmap, g.values, g.prefix, n, kind)
+    assert ok and np.array_equal(out, x)
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("n", [0, 1, 33, 4097, 8192 * 3 + 1000, 200704, 8192 * 150 + 77])
+@pytest.mark.parametrize("mode", ["stash_only", "with_y", "in_place"])
+def test_relu_fwd_compress(G, oracle, kind, n, mode):
+    x = W.random_patterns(n, kind, 0.1, seed=2000 + n)
+    y_ref, c = oracle.relu_fwd_compress(x, kind)
+    xt = G.from_raw(x, kind)
+    g = G.gpu_compress(xt, relu=True, want_y=(mode == "with_y"), in_place=(mode == "in_place"))
+    assert_same_compressed(g, c)
+    if mode == "stash_only":
+        assert g.y is None
+        assert np.array_equal(W.raw_numpy(xt), x)           # the input is left alone
+    else:
+        assert np.array_equal(g.y, y_ref)
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("n", [0, 1, 7, 33, 4097, 8192 * 3 + 1003, 200704, (1 << 20) + 5])
+@pytest.mark.parametrize("in_place", [False, True])
+def test_relu_bwd_from_bitmap(G, oracle, kind, n, in_place):
+    x = W.random_patterns(n, kind, 0.3, seed=3000 + n)
+    gr = W.random_patterns(n, kind, 0.05, seed=4000 + n)    # gradients with NaN, inf, -0 patterns inside
+    _, c = oracle.relu_fwd_compress(x, kind)
+    ref = oracle.relu_bwd_from_bitmap(c.bitmap, gr)
+    if n == 0:
+        bm = np.zeros(1, np.uint32)
+    else:
+        bm = c.bitmap
+    out, ok = G.gpu_relu_bwd(bm, G.from_raw(gr, kind) if n else torch.empty(0, dtype=G.TDT[kind], device="cuda"),
+                             in_place=in_place)
+    assert ok and np.array_equal(out, ref)
+
+
+def test_cfg1_round_trip(G, oracle):
+    x = W.cfg1("cuda")
+    xr = W.raw_numpy(x)
+    c = oracle.compress(xr)
+    g = G.gpu_compress(x)
+    assert_same_compressed(g, c)
+    out, ok = G.gpu_decompress(g.bitmap, g.values, g.prefix, x.numel(), "f32")
+    assert ok and np.array_equal(out, xr)
+    assert B.bt_compressed_bytes(x.numel(), g.nnz, torch.float32) == x.numel() // 8 + 4 * g.nnz + 8 * 49
+
+
+@pytest.mark.parametrize("variant", ["iid", "clustered"])
+@pytest.mark.parametrize("s", W.SPARSITY_SWEEP)
+def test_cfg3_reduced(G, oracle, variant, s):
+    n = 1 << 22
+    idx = W.SPARSITY_SWEEP.index(s)
+    x = (W.cfg3_iid if variant == "iid" else W.cfg3_clustered)(n, s, idx, "cuda")
+    xr = W.raw_numpy(x)
+    c = oracle.compress(xr)
+    g = G.gpu_compress(x)
+    assert_same_compressed(g, c)
+    out, ok = G.gpu_decompress(g.bitmap, g.values, g.prefix, n, "f32")
+    assert ok and np.array_equal(out, xr)
+
+
+def test_capacity_overflow_reports_and_stays_in_bounds(G, oracle):
+    n = 8192 * 20 + 100
+    x = W.random_patterns(n, "f32", 0.5, seed=77)
+    c = oracle.compress(x)
+    cap = c.nnz // 2
+    g = G.gpu_compress(G.from_raw(x, "f32"), capacity=cap)
+    assert g.guards_ok                                  # nothing written past the capacity
+    assert g.status == B.BT_ERR_CAPACITY
+    assert g.nnz == c.nnz                               # the true count is still reported
+    assert np.array_equal(g.bitmap, c.bitmap) and np.array_equal(g.prefix, c.prefix)
+    assert np.array_equal(g.values_all[:cap], c.values[:cap])
+
+
+def test_workspace_is_reusable_without_clearing(G, oracle):
+    n = 8192 * 40 + 1
+    ws = B.new_workspace(n)
+    ws.fill_(0xFF)                                      # garbage in: the call must not depend on it
+    for seed in (1, 2, 3):
+        x = W.random_patterns(n, "f16", 0.6, seed=seed)
+        c = oracle.compress(x)
+        st = B.Stash(n, torch.float16)
+        B.bt_compress(G.from_raw(x, "f16"), st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        torch.cuda.synchronize()
+        assert st.nnz == c.nnz and st.status == B.BT_OK
+        assert np.array_equal(W.raw_numpy(st.values[:c.nnz]), c.values)
+        assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), c.prefix)
