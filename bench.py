@@ -1,0 +1,532 @@
+#!/usr/bin/env python3
+"""Benchmark of the sparse-bitmap codec hot path on B200.
+
+One "step" is one pass of the whole path over one batch of synthetic
+activations shaped like a ResNet-18 at batch 32 (17 post-ReLU tensors, fp32,
+about half zeros): in forward order every layer is stashed twice -- once with
+bt_compress (from the post-ReLU activation) and once with bt_relu_fwd_compress
+(from the pre-activation) -- and in reverse order every layer is restored with
+bt_decompress and its ReLU gradient formed with bt_relu_bwd_from_bitmap.  The
+metric is dense-equivalent GB/s: the dense bytes of every tensor an entry point
+consumed or produced (N * sizeof(dtype) per call), summed over the step,
+divided by the step time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
+runs the same batch shard on its own GPU -- data-parallel replicas compress
+their own activations, there is no data-path collective -- and the value is the
+sum over ranks divided by the slowest rank's time (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "codec_dense_equivalent_throughput"
+UNIT = "GB/s"
+WORKLOAD = "cfg2_resnet18_b32_f32"
+OPS = ("bt_compress", "bt_relu_fwd_compress", "bt_decompress", "bt_relu_bwd_from_bitmap")
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=200)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    p.add_argument("--batch", type=int, default=32, help="batch of the ResNet-18-shaped set (32 = the named config)")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-large", action="store_true", help="skip the per-kernel runs on 1 GiB tensors")
+    p.add_argument("--no-e2e", action="store_true")
+    return p.parse_args()
+
+
+# ------------------------------------------------------------------------------------------
+# clocks: read-only NVML sampling in a thread while the timed region runs
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples = []          # (host time, sm MHz, reasons bitmask)
+        self.period = period_s
+        self._stop = threading.Event()
+        self.ok = False
+        self.sm_max = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = self._handle(index)
+            self.sm_max = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def _handle(self, index):
+        import torch
+        try:
+            uuid = str(torch.cuda.get_device_properties(index).uuid)
+            uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+            return self.nv.nvmlDeviceGetHandleByUUID(uuid)
+        except Exception:
+            return self.nv.nvmlDeviceGetHandleByIndex(index)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                mhz = int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                try:
+                    r = int(self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                self.samples.append((time.time(), mhz, r))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.ok:
+            self.thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self.ok and self.thread.is_alive():
+            self.thread.join(timeout=1.0)
+
+    def summary(self, t0: float, t1: float) -> dict:
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        note = "sampled during the timed region"
+        if not inside:
+            inside = self.samples[-3:]
+            note = "timed region shorter than the sampling period: nearest samples"
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "note": "NVML unavailable"}
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        reasons = [name for bit, name in self.REASONS.items() if mask & bit and name != "gpu_idle"]
+        return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.sm_max,
+                "reasons": reasons, "samples": len(inside), "note": note}
+
+
+# ------------------------------------------------------------------------------------------
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def algorithmic_bytes(op: str, n: int, nnz: int, es: int, with_y: bool = False) -> int:
+    """Bytes the method itself must move for one call (dense tensor, bitmap, packed values, prefix)."""
+    compressed = 4 * ((n + 31) // 32) + nnz * es + 8 * ((n + 4095) // 4096)
+    if op in ("bt_compress", "bt_decompress"):
+        return n * es + compressed
+    if op == "bt_relu_fwd_compress":
+        return n * es + compressed + (n * es if with_y else 0)
+    if op == "bt_relu_bwd_from_bitmap":
+        return 2 * n * es + 4 * ((n + 31) // 32)
+    raise ValueError(op)
+
+
+class Cfg2Step:
+    """Device-resident state of one step over the ResNet-18-shaped activation set."""
+
+    def __init__(self, dev, batch: int):
+        import torch
+        from paper_2110_15362_b200 import binding as B
+        from paper_2110_15362_b200 import workloads as W
+        self.B, self.torch = B, torch
+        self.shapes = W.resnet18_shapes(batch)
+        self.layers = []
+        n_max = max(W.numel(s) for s in self.shapes)
+        for i, shape, n in W.iter_layers(self.shapes):
+            pre = W.cfg2_preact(i, shape, dev).reshape(-1)
+            act = torch.clamp_min(pre, 0.0)                     # == W.cfg2_layer(i, shape): same seed
+            grad = W.cfg2_grad(i, shape, dev).reshape(-1)
+            self.layers.append(dict(n=n, pre=pre, act=act, grad=grad,
+                                    stash_a=B.Stash(n, torch.float32, dev), stash_b=B.Stash(n, torch.float32, dev)))
+        self.restored = torch.empty(n_max, dtype=torch.float32, device=dev)
+        self.gin = torch.empty(n_max, dtype=torch.float32, device=dev)
+        self.ws = B.new_workspace(n_max, dev)
+        self.total_elems = sum(l["n"] for l in self.layers)
+        self.dense_bytes_per_step = len(OPS) * 4 * self.total_elems
+        self.launches_per_step = len(OPS) * len(self.layers)
+
+    def run(self, rec=None):
+        """One step.  `rec(op, layer_index)` brackets a call with CUDA events when given."""
+        B = self.B
+        for i, l in enumerate(self.layers):
+            a, b = l["stash_a"], l["stash_b"]
+            if rec: rec("bt_compress", i, True)
+            B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.ws, a.dev_status)
+            if rec: rec("bt_compress", i, False)
+            if rec: rec("bt_relu_fwd_compress", i, True)
+            B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.ws,
+                                   b.dev_status)
+            if rec: rec("bt_relu_fwd_compress", i, False)
+        for i in range(len(self.layers) - 1, -1, -1):
+            l = self.layers[i]
+            a, b = l["stash_a"], l["stash_b"]
+            n = l["n"]
+            if rec: rec("bt_decompress", i, True)
+            B.bt_decompress(a.bitmap, a.values, a.chunk_prefix, self.restored[:n])
+            if rec: rec("bt_decompress", i, False)
+            if rec: rec("bt_relu_bwd_from_bitmap", i, True)
+            B.bt_relu_bwd_from_bitmap(b.bitmap, l["grad"], self.gin[:n])
+            if rec: rec("bt_relu_bwd_from_bitmap", i, False)
+
+    def check(self):
+        """After a step: device status words are clean and both stashes of a layer agree."""
+        torch = self.torch
+        for l in self.layers:
+            a, b = l["stash_a"], l["stash_b"]
+            assert a.status == 0 and b.status == 0, "device status not BT_OK"
+            assert a.nnz == b.nnz, "the two stashes of a layer disagree"
+        last = self.layers[0]
+        assert torch.equal(self.restored[:last["n"]].view(torch.int32), last["act"].view(torch.int32)), \
+            "round trip is not bit exact"
+
+    def nnz(self):
+        return [l["stash_a"].nnz for l in self.layers]
+
+
+def per_kernel_pass(step: Cfg2Step, steps: int):
+    """Same steps, eager launches, CUDA events on the launching stream around every call."""
+    import torch
+    stream = torch.cuda.current_stream()
+    pending = {}
+    records = []
+
+    def rec(op, i, begin):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record(stream)
+        if begin:
+            pending[(op, i)] = ev
+        else:
+            records.append((op, i, pending.pop((op, i)), ev))
+
+    for _ in range(steps):
+        step.run(rec)
+    torch.cuda.synchronize()
+    per_op = {op: {"ms": 0.0, "launches": 0} for op in OPS}
+    per_layer = {}
+    for op, i, e0, e1 in records:
+        ms = e0.elapsed_time(e1)
+        per_op[op]["ms"] += ms
+        per_op[op]["launches"] += 1
+        per_layer.setdefault((op, i), []).append(ms)
+    return per_op, per_layer
+
+
+def large_tensor_kernels(dev, peak_gbs: float):
+    """Every kernel alone on a 1 GiB fp32 tensor (2^28 elements, half zeros) and on the largest
+    VGG-16-shaped bf16 tensor: the sizes at which the kernels are held to the HBM roofline."""
+    import torch
+    from paper_2110_15362_b200 import binding as B
+    from paper_2110_15362_b200 import workloads as W
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def time_call(fn, reps=10):
+        best = []
+        for _ in range(3):
+            fn()
+        for _ in range(reps):
+            flush.fill_(1)                       # evict L2 between timed launches
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            best.append(e0.elapsed_time(e1))
+        return statistics.median(best), min(best)
+
+    for label, kind, n in (("f32_2^28_s0.5", "f32", 1 << 28), ("bf16_64x64x224x224", "bf16", 64 * 64 * 224 * 224)):
+        if kind == "f32":
+            x = W.cfg3_iid(n, 0.5, 2, dev)
+            pre = x
+        else:
+            pre = W.cfg4_preact(0, (n,), kind, dev)
+            x = torch.relu(pre)
+        es = x.element_size()
+        st = B.Stash(n, x.dtype, dev)
+        ws = B.new_workspace(n, dev)
+        dense = torch.empty_like(x)
+        res = {}
+        ms, best = time_call(lambda: B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws,
+                                                   st.dev_status))
+        nnz = st.nnz
+        res["bt_compress"] = (ms, best, algorithmic_bytes("bt_compress", n, nnz, es))
+        ms, best = time_call(lambda: B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, dense))
+        assert torch.equal(dense.view(torch.int16 if es == 2 else torch.int32),
+                           x.view(torch.int16 if es == 2 else torch.int32))
+        res["bt_decompress"] = (ms, best, algorithmic_bytes("bt_decompress", n, nnz, es))
+        ms, best = time_call(lambda: B.bt_relu_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix,
+                                                            st.nnz_out, ws, st.dev_status))
+        res["bt_relu_fwd_compress"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, es))
+        ms, best = time_call(lambda: B.bt_relu_fwd_compress(pre, dense, st.bitmap, st.values, st.chunk_prefix,
+                                                            st.nnz_out, ws, st.dev_status))
+        res["bt_relu_fwd_compress+y"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, es, True))
+        ms, best = time_call(lambda: B.bt_relu_bwd_from_bitmap(st.bitmap, x, dense))
+        res["bt_relu_bwd_from_bitmap"] = (ms, best, algorithmic_bytes("bt_relu_bwd_from_bitmap", n, 0, es))
+        out[label] = {op: {"ms_median": round(ms, 4), "ms_best": round(best, 4),
+                           "moved_gbs": round(by / ms / 1e6, 1),
+                           "dense_equiv_gbs": round(n * es / ms / 1e6, 1),
+                           "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
+                           "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
+                      for op, (ms, best, by) in res.items()}
+        del x, pre, st, ws, dense
+        torch.cuda.empty_cache()
+    return out
+
+
+# ------------------------------------------------------------------------------------------
+def oracle_step(layers_np, indices):
+    """The CPU oracle on the given layers, same four operations per layer; returns seconds."""
+    from oracle import bt_oracle as O
+    t0 = time.perf_counter()
+    stashes = []
+    for i in indices:
+        act, pre, grad = layers_np[i]
+        a = O.compress(act)
+        _, b = O.relu_fwd_compress(pre, "f32", want_y=False)
+        stashes.append((i, a, b))
+    for i, a, b in reversed(stashes):
+        O.decompress(a)
+        O.relu_bwd_from_bitmap(b.bitmap, layers_np[i][2])
+    return time.perf_counter() - t0
+
+
+def host_layers(batch, indices):
+    import torch
+    from paper_2110_15362_b200 import workloads as W
+    shapes = W.resnet18_shapes(batch)
+    out = {}
+    for i in indices:
+        pre = W.cfg2_preact(i, shapes[i], "cpu")
+        out[i] = (W.raw_numpy(torch.clamp_min(pre, 0.0)), W.raw_numpy(pre), W.raw_numpy(W.cfg2_grad(i, shapes[i], "cpu")))
+    return out, shapes
+
+
+def run_reference(args):
+    """The oracle, as it stands, on host cores; each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2110_15362_b200 import workloads as W
+    sample = [1]                                                # one [B,64,56,56] layer per step
+    layers, shapes = host_layers(args.batch, sample)
+    elems = sum(W.numel(shapes[i]) for i in sample)
+    for _ in range(min(args.warmup, 1)):
+        oracle_step(layers, sample)
+    t = [oracle_step(layers, sample) for _ in range(args.steps)]
+    total = sum(t)
+    value = len(OPS) * 4 * elems * args.steps / total / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": round(1e3 * total / args.steps, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch": args.batch,
+                       "ops_per_layer": list(OPS)},
+            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "layer 1 of 17 ([%d,64,56,56], %d elements) per step, all four operations; "
+                                       "host has %d cores" % (args.batch, elems, os.cpu_count())},
+            "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2110_15362_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.lib()
+    peak, peak_kind = measured_peak_gbs()
+
+    step = Cfg2Step(dev, args.batch)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(max(args.warmup, 3)):
+            step.run()
+    torch.cuda.synchronize()
+    step.check()
+    nnz = step.nnz()
+
+    # the whole step as one CUDA graph: 68 kernel launches replayed without host work in between
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step.run()
+    for _ in range(max(args.warmup, 3)):
+        graph.replay()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        graph.replay()
+    e1.record()
+    barrier()
+    t1 = time.time()
+    ms_total = e0.elapsed_time(e1)
+    step.check()
+    clocks = sampler.summary(t0, t1)
+
+    # per-kernel durations: the same steps launched eagerly with events around every call
+    per_op, per_layer = per_kernel_pass(step, min(args.steps, 20))
+
+    # end to end: inputs start in pinned host memory, results end in host memory, every step
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(step, graph, min(args.steps, 10), world)
+    sampler.stop()
+
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+        if e2e is not None:
+            t = torch.tensor([e2e["ms"]], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e["ms"] = float(t.item())
+
+    if rank == 0:
+        ms_step = ms_total / args.steps
+        value = world * step.dense_bytes_per_step / (ms_step * 1e-3) / 1e9
+        # roofline of the dominant kernel class
+        dom = max(per_op, key=lambda k: per_op[k]["ms"])
+        alg = sum(algorithmic_bytes(dom, l["n"], z, 4) for l, z in zip(step.layers, nnz))
+        launches = per_op[dom]["launches"]
+        avg_ms = per_op[dom]["ms"] / launches
+        achieved = (alg / len(step.layers)) / (avg_ms * 1e-3) / 1e9
+        # the largest layer alone (98 MiB dense), the launch closest to the sizes the roofline bar is set for
+        big_ms = statistics.median(per_layer[(dom, 0)])
+        big_alg = algorithmic_bytes(dom, step.layers[0]["n"], nnz[0], 4)
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "batch": args.batch, "layers": len(step.layers),
+                       "elements_per_step": step.total_elems, "zero_fraction": round(
+                           1.0 - sum(nnz) / step.total_elems, 4),
+                       "ops_per_layer": list(OPS), "launch": "one CUDA graph per step",
+                       "l2": "per-step working set %.2f GB exceeds the 126 MB L2; no flush between steps"
+                             % (7 * 4 * step.total_elems / 1e9),
+                       "parallelism": "dp%d" % world if world > 1 else "single"},
+            "clocks": clocks,
+            "gpu_launches": step.launches_per_step * args.steps,
+            "roofline": {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak,
+                         "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": peak_kind,
+                         "traffic": None,
+                         "avg_launch_ms": round(avg_ms, 5), "launches_timed": launches,
+                         "largest_layer": {"elements": step.layers[0]["n"], "ms": round(big_ms, 5),
+                                           "achieved": round(big_alg / big_ms / 1e6, 1),
+                                           "frac": round(big_alg / big_ms / 1e6 / peak, 4)},
+                         "per_op_ms_per_step": {k: round(v["ms"] / max(1, v["launches"]) * len(step.layers), 5)
+                                                for k, v in per_op.items()}},
+        }
+        if e2e is not None:
+            e2e_ms = e2e["ms"] / e2e["steps"]
+            line["e2e"] = {"value": round(world * step.dense_bytes_per_step / (e2e_ms * 1e-3) / 1e9, 3),
+                           "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "ms_per_step": round(e2e_ms, 3), "steps": e2e["steps"]}
+        if world == 1 and not args.no_large:
+            line["large_tensor_kernels"] = large_tensor_kernels(dev, peak)
+        if world == 1 and not args.no_cpu_baseline:
+            idx = list(range(len(step.layers)))
+            layers, _ = host_layers(args.batch, idx)
+            secs = oracle_step(layers, idx)
+            line["cpu_baseline"] = {"value": round(step.dense_bytes_per_step / secs / 1e9, 4), "unit": UNIT,
+                                    "cores": 1, "kind": "oracle",
+                                    "sample": "one full step (17 layers, %d elements, four operations each), "
+                                              "single thread; host has %d cores" % (step.total_elems, os.cpu_count()),
+                                    "seconds": round(secs, 2)}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(step: Cfg2Step, graph, steps: int, world: int):
+    """Step time with the inputs coming from pinned host memory and the results (restored
+    activation and input gradient of every layer, the nnz words) going back to host memory."""
+    import torch
+    host = []
+    for l in step.layers:
+        host.append(dict(act=l["act"].cpu().pin_memory(), pre=l["pre"].cpu().pin_memory(),
+                         grad=l["grad"].cpu().pin_memory(),
+                         nnz=torch.empty(1, dtype=torch.int64).pin_memory()))
+    n_max = step.restored.numel()
+    out_restored = torch.empty(n_max, dtype=torch.float32).pin_memory()
+    out_gin = torch.empty(n_max, dtype=torch.float32).pin_memory()
+    h2d = sum(3 * 4 * l["n"] for l in step.layers)
+    d2h = sum(8 for _ in step.layers) + 2 * 4 * step.layers[0]["n"]
+
+    def one():
+        for l, h in zip(step.layers, host):
+            l["act"].copy_(h["act"], non_blocking=True)
+            l["pre"].copy_(h["pre"], non_blocking=True)
+            l["grad"].copy_(h["grad"], non_blocking=True)
+        graph.replay()
+        for l, h in zip(step.layers, host):
+            h["nnz"].copy_(l["stash_a"].nnz_out, non_blocking=True)
+        n0 = step.layers[0]["n"]
+        out_restored[:n0].copy_(step.restored[:n0], non_blocking=True)
+        out_gin[:n0].copy_(step.gin[:n0], non_blocking=True)
+
+    for _ in range(2):
+        one()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    return {"ms": e0.elapsed_time(e1), "steps": steps, "h2d": h2d, "d2h": d2h}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
