@@ -11,7 +11,7 @@
 namespace bt {
 
 // ---------------------------------------------------------------- workspace layout
-// [0]   uint32  ticket     next tile to hand out
+// [0]   uint32  reserved
 // [1]   uint32  abort      set once a bounded wait ran out; every CTA then leaves
 // [2..] reserved
 // then one 64-bit descriptor per tile: (value << 2) | state
