@@ -14,10 +14,10 @@ namespace bt {
 // [0]   uint32  reserved
 // [1]   uint32  abort      set once a bounded wait ran out; every CTA then leaves
 // [2..] reserved
-// then one 64-bit descriptor per tile: (value << 2) | state
+// then one 64-bit total per wave of tiles, then one 64-bit descriptor per tile
+// (both sized for the smallest tile, so at most 2 words per 4096 elements)
 constexpr size_t   kWsHeaderBytes = 256;
-constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;   // descriptors are sized for the smallest tile
-constexpr uint64_t kStateInvalid = 0, kStateAggregate = 1, kStateInclusive = 2;
+constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;
 
 struct CompressArgs {
     const void *src;        // dense input (pre-activation for the fused form)
@@ -29,7 +29,8 @@ struct CompressArgs {
     uint64_t   *nnz_out;
     int32_t    *dev_status;
     uint32_t   *ws_header;
-    uint64_t   *ws_desc;
+    uint64_t   *ws_desc;    // wave totals, then tile descriptors
+    uint32_t    ws_waves;   // number of wave totals
     uint64_t    n;
 };
 
