@@ -5,21 +5,23 @@
 // The grid is launched cooperatively with exactly as many CTAs (G) as fit on
 // the device at once, so all of them are co-resident, and CTA b takes tiles
 // b, b+G, b+2G, ...: iteration j of every CTA together forms "wave j", G
-// consecutive tiles.  A CTA is kWarps worker warps plus one scan warp.  Tiles
-// are staged into shared memory by 1-D bulk async copies through a ring of
-// kStages buffers.  Each worker warp owns 1024 consecutive elements of the tile
-// = 32 bitmap words:
+// consecutive tiles.  Tiles are staged into shared memory by 1-D bulk async
+// copies through a ring of kStages slots, and the warps of a CTA are
+// specialised: one load warp (a single lane issues the bulk copies), kWarps
+// compactor warps, one scan warp, kWarps copier warps.
 //
-//   step k of a warp:  lane l reads element 32k+l from shared memory;
+// Compactor warp w owns kTile / kWarps consecutive elements of the tile:
+//
+//   step k of a warp:  lane l reads element 32k+l of its segment from shared memory;
 //                      ballot(non-zero) IS bitmap word k (LSB first);
 //                      popc(ballot & lanemask_lt) is the lane's rank;
 //                      non-zero lanes write the element back IN PLACE at
 //                      [run + rank] of the warp's own segment (always at or
 //                      before the position being read, so nothing unread is
-//                      overwritten).
+//                      overwritten); all shared accesses are conflict-free.
 //
-// After 32 steps lane k holds word k (one coalesced 128-byte bitmap store) and
-// the segment's first `run` slots hold the packed values.
+// The ballots are parked in shared memory by lane 0 and leave as one coalesced
+// bitmap store per warp; the segment's first `run` slots hold the packed values.
 //
 // Prefix.  The exclusive base of tile (wave j, CTA b) is
 //     sum of the totals of waves 0..j-1  +  sum of the counts of CTAs 0..b-1 in wave j.
@@ -32,23 +34,25 @@
 // compaction of the following tiles.  No tile waits on another tile's base:
 // only on counts, which never wait on anything but the data.
 //
-// The warps of a CTA never meet at a CTA-wide barrier; they hand work over
-// through mbarriers:
-//   full[s]     the bulk copy into stage s has landed            (copy engine -> workers)
-//   counted[s]  every worker has posted its packed count         (workers -> scan warp)
-//   ready[s]    base and warp offsets of the tile are in shared  (scan warp -> workers)
-// Each worker copies its packed slots of a tile out to values[base + warp
-// offset ...] kLag iterations after compacting it; the last worker warp out of
-// a stage refills it.
+// The warps of a CTA never meet at a CTA-wide barrier; a ring slot goes round
+// through four mbarriers:
+//   full[s]     the bulk copy has landed                   (copy engine -> compactors)
+//   counted[s]  every compactor has posted its count       (compactors  -> scan warp)
+//   ready[s]    base and segment offsets are in shared     (scan warp   -> copiers)
+//   empty[s]    every copier has copied its segment out    (copiers     -> load warp)
+// Copier warp w copies segment w's packed slots to values[base + offset ...].
+// The scan warp works on three tiles at a time (publish, read, finish), so the
+// compactors run about three tiles ahead of the copiers and nobody waits for a
+// round trip to L2.
 #include <cstdlib>
 #include <mutex>
+#include <type_traits>
 
 #include "bt_internal.cuh"
 
 namespace bt {
 namespace {
 
-constexpr int      kWarpElems  = 1024;                // 32 steps x 32 lanes
 constexpr uint32_t kFull       = 0xFFFFFFFFu;
 constexpr uint64_t kWaitNs     = 2000000000ull;       // bound of every in-kernel wait: 2 s
 constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
@@ -119,40 +123,130 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     }
 }
 
-// What the scan warp holds in flight for one tile: the descriptors of the lower CTAs of the
-// tile's wave (lane l, window k <-> CTA l + 32k) and the total word of the previous wave.
-struct PendingScan {
-    uint64_t d[kMaxWindows];
-    uint64_t prev_wave;
-};
+// shared-memory accesses by 32-bit shared address, kept in program order among themselves
+template <typename U>
+__device__ __forceinline__ uint32_t lds_elem(uint32_t addr)
+{
+    uint32_t v;
+    if constexpr (sizeof(U) == 4) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    else asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));   // zero-extended
+    return v;
+}
+// store `v` at `addr` in the lanes where keep != 0 (a predicated store, never a branch)
+template <typename U>
+__device__ __forceinline__ void sts_elem_if(uint32_t addr, uint32_t v, uint32_t keep)
+{
+    if constexpr (sizeof(U) == 4)
+        asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u32 [%0], %1;\n\t}" ::"r"(addr), "r"(v),
+                     "r"(keep));
+    else
+        asm volatile("{\n\t.reg .pred q;\n\t.reg .b16 h;\n\tsetp.ne.u32 q, %2, 0;\n\tcvt.u16.u32 h, %1;\n\t@q st.shared.u16 [%0], h;\n\t}" ::"r"(addr),
+                     "r"(v), "r"(keep));
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v));
+}
+
+// ---------------------------------------------------------------------------------------------
+// One warp compacts its segment of kSteps * 32 elements in place.  Returns the number of packed
+// values.  The ballot of step k goes to the shared word at words_addr + 4k (every lane stores the
+// same value to the same address: one wavefront, no predicate).  `y` (fused form with dense
+// output) points at the segment's first element of the dense ReLU output, `yvalid` is how many of
+// them exist.  seg_addr / words_addr are shared-window addresses.
+//
+// The loads of a batch of 8 steps are issued before the stores of the batch before it: a store of
+// step k lands below element 32(k+1) and a later batch reads at or above it, so they never meet.
+template <typename U, int RELU_DT, bool WRITE_Y, int kSteps>
+__device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, const uint32_t words_addr,
+                                                    const uint32_t lane, const uint32_t lt, U *y,
+                                                    const uint32_t yvalid)
+{
+    constexpr int      kBatch = kSteps < 8 ? kSteps : 8;
+    constexpr uint32_t kES    = sizeof(U);
+    const uint32_t     in0    = seg_addr + lane * kES;
+    uint32_t           out    = seg_addr;               // address of the next free packed slot
+    uint32_t           v[kBatch], vn[kBatch];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) v[j] = lds_elem<U>(in0 + j * 32 * kES);
+#pragma unroll
+    for (int kb = 0; kb < kSteps; kb += kBatch) {
+        if (kb + kBatch < kSteps) {
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) vn[j] = lds_elem<U>(in0 + (kb + kBatch + j) * 32 * kES);
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            uint32_t x = v[j];
+            if constexpr (RELU_DT >= 0) {
+                x = ReluKeep<RELU_DT>::keep(x) ? x : 0u;
+                if constexpr (WRITE_Y) {
+                    const uint32_t e = (kb + j) * 32 + lane;
+                    if (e < yvalid) y[e] = static_cast<U>(x);
+                }
+            }
+            const uint32_t b = __ballot_sync(kFull, x != 0u);
+            sts_u32(words_addr + 4 * (kb + j), b);
+            sts_elem_if<U>(out + kES * __popc(b & lt), x, x);
+            out += kES * __popc(b);
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) v[j] = vn[j];
+    }
+    return (out - seg_addr) / kES;
+}
+
+// One warp copies the `cnt` packed slots of its segment to out[0..cnt): contiguous, coalesced.
+template <typename U, bool kGuard>
+__device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, const uint32_t lane, const uint32_t cnt,
+                                                 U *__restrict__ out, const uint64_t room)
+{
+    uint32_t j = lane;
+    for (; j + 96 < cnt; j += 128) {
+        const U v0 = seg[j], v1 = seg[j + 32], v2 = seg[j + 64], v3 = seg[j + 96];
+        if (!kGuard || j < room) out[j] = v0;
+        if (!kGuard || j + 32 < room) out[j + 32] = v1;
+        if (!kGuard || j + 64 < room) out[j + 64] = v2;
+        if (!kGuard || j + 96 < room) out[j + 96] = v3;
+    }
+    for (; j < cnt; j += 32) {
+        const U v = seg[j];
+        if (!kGuard || j < room) out[j] = v;
+    }
+}
 
 // U: uint32_t (4-byte elements) or uint16_t (2-byte elements).
 // RELU_DT: -1 for the plain compressor, else the element type whose ReLU is fused in.
-// kLag: how many iterations the copy-out of a tile trails its compaction (>= 2: the scan of a
-// tile is issued one iteration and finished two iterations after the tile was counted).
-template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kStages, int kLag>
-__global__ void __launch_bounds__(kWarps * 32 + 32) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
+// kWarps compactor warps and as many copier warps, kSeg elements per warp, kStages ring slots.
+template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages>
+__global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
 {
-    constexpr int kTile          = kWarps * kWarpElems;
+    constexpr int kTile          = kWarps * kSeg;
+    constexpr int kSteps         = kSeg / 32;
     constexpr int kChunksPerTile = kTile / BT_CHUNK_ELEMS;
-    constexpr int kWarpsPerChunk = BT_CHUNK_ELEMS / kWarpElems;
-    constexpr int kScanWarp      = kWarps;          // warp index of the scan warp
-    constexpr int kWorkerThreads = kWarps * 32;
+    constexpr int kWarpsPerChunk = BT_CHUNK_ELEMS / kSeg;
+    constexpr int kCompactThreads = kWarps * 32;
+    // warp roles
+    constexpr int kFirstCopier = kWarps;
+    constexpr int kScanWarp    = 2 * kWarps;
+    constexpr int kLoadWarp    = 2 * kWarps + 1;
+    static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
     static_assert(kTile % BT_CHUNK_ELEMS == 0, "a tile holds whole chunks");
     static_assert(kWarps <= 32, "one lane per warp count");
-    static_assert(kLag >= 2, "a tile's base is known two iterations after its count");
-    static_assert(kStages >= kLag + 2, "one stage compacting, kLag awaiting copy-out, at least one loading");
+    static_assert(kStages >= 4, "loading, compacting, awaiting its base, copying out");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     U *const tiles = reinterpret_cast<U *>(smem_raw);
 
-    __shared__ __align__(8) uint64_t s_full[kStages];
-    __shared__ __align__(8) uint64_t s_counted[kStages];
-    __shared__ __align__(8) uint64_t s_ready[kStages];
-    __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the stage
-    __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each warp
-    __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each warp in the tile
-    __shared__ uint32_t          s_done[kStages];          // warps that finished copying the stage out
+    __shared__ __align__(8) uint64_t s_full[kStages];      // the bulk copy has landed            (copy engine -> compactors)
+    __shared__ __align__(8) uint64_t s_counted[kStages];   // every compactor posted its count    (compactors -> scan warp)
+    __shared__ __align__(8) uint64_t s_ready[kStages];     // base and offsets are in shared      (scan warp -> copiers)
+    __shared__ __align__(8) uint64_t s_empty[kStages];     // every copier is done with the slot  (copiers -> load warp)
+    __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
+    __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
+    __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
+    __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
+    __shared__ uint32_t          s_words[kWarps][kSteps];  // ballots of the segment a warp is compacting
     __shared__ volatile uint32_t s_abort;
 
     const uint32_t tid  = threadIdx.x;
@@ -164,18 +258,14 @@ __global__ void __launch_bounds__(kWarps * 32 + 32) compress_kernel(const Compre
     const uint64_t n    = a.n;
 #ifdef BT_PROFILE
     unsigned long long prof[16] = {};
+#define PROF_FLUSH(lo, hi)                                                                                       \
+    if (lane == 0)                                                                                               \
+        for (int k_ = (lo); k_ < (hi); ++k_)                                                                     \
+            atomicAdd(reinterpret_cast<unsigned long long *>(a.ws_header) + 8 + k_, prof[k_]);
+#else
+#define PROF_FLUSH(lo, hi)
 #endif
 
-    // Issue the bulk load of tile t into stage s (one thread).
-    auto issue_load = [&](uint32_t s, uint32_t t) {
-        const uint64_t first = static_cast<uint64_t>(t) * kTile;
-        const uint64_t left  = n - first;
-        const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
-        const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
-        fence_proxy_async();                       // earlier generic accesses to this stage come first
-        mbar_arrive_expect_tx(&s_full[s], bytes);  // bytes == 0 simply completes the phase
-        if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
-    };
     // tile of iteration `it` of this CTA (64-bit so that running past the end cannot wrap)
     auto tile_of = [&](uint32_t it) { return cta + static_cast<uint64_t>(it) * G; };
 
@@ -185,257 +275,249 @@ __global__ void __launch_bounds__(kWarps * 32 + 32) compress_kernel(const Compre
             mbar_init(&s_full[s], 1);
             mbar_init(&s_counted[s], kWarps);
             mbar_init(&s_ready[s], 1);
-            s_done[s] = 0;
+            mbar_init(&s_empty[s], kWarps);
         }
         fence_proxy_async();
-        for (int s = 0; s < kStages; ++s)
-            if (tile_of(s) < num_tiles) issue_load(s, static_cast<uint32_t>(tile_of(s)));
     }
     __syncthreads();
 
+    if (warp == kLoadWarp) {
+        // ------------------------------------------------------------ load warp (one lane)
+        if (lane == 0) {
+            bool ok = true;
+            for (uint32_t it = 0; ok; ++it) {
+                const uint64_t t64 = tile_of(it);
+                if (t64 >= num_tiles) break;
+                const uint32_t s = it % kStages;
+                if (it >= static_cast<uint32_t>(kStages)) {
+                    PROF_T(c0);
+                    ok = mbar_wait(&s_empty[s], ((it / kStages) - 1) & 1u, &s_abort);
+                    PROF_T(c1);
+                    PROF_ADD(4, c1 - c0);
+                    if (!ok) break;
+                }
+                const uint64_t first = t64 * kTile;
+                const uint64_t left  = n - first;
+                const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
+                const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
+                fence_proxy_async();                       // the copiers' and compactors' accesses to the slot come first
+                mbar_arrive_expect_tx(&s_full[s], bytes);  // bytes == 0 simply completes the phase
+                if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
+            }
+            if (!ok) {
+                // a bounded wait ran out somewhere in this CTA: before leaving, let the bulk copies that
+                // may still be in flight into its shared memory land (bounded, short)
+                for (int s = 0; s < kStages; ++s) {
+                    mbar_wait<false>(&s_full[s], 0, &s_abort, 20000000ull);
+                    mbar_wait<false>(&s_full[s], 1, &s_abort, 20000000ull);
+                }
+            }
+            PROF_FLUSH(4, 5);
+        }
+        return;
+    }
+
     if (warp == kScanWarp) {
         // ------------------------------------------------------------ scan warp
-        uint64_t *const wave_total   = a.ws_desc;                  // one word per wave
-        uint64_t *const desc         = a.ws_desc + a.ws_waves;     // one word per tile: (count << 1) | 1
-        const uint64_t  chunks_total = (n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
-        const uint32_t *abort_flag   = a.ws_header + 1;
+        uint64_t *const       wave_total   = a.ws_desc;                  // one word per wave
+        uint64_t *const       desc         = a.ws_desc + a.ws_waves;     // one word per tile: (count << 1) | 1
+        const uint64_t        chunks_total = (n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
+        const uint32_t *const abort_flag   = a.ws_header + 1;
+        uint64_t              waves_before = 0;    // sum of the totals of the waves before the tile being finished
+        bool                  failed       = false;
 
-        uint64_t    waves_before = 0;     // sum of the totals of all waves before the pending tile's wave
-        PendingScan pend;                 // loads in flight for the pending tile (iteration it - 1)
-        uint32_t    pend_agg = 0, pend_chunk_off = 0;   // of the pending tile: its count; this lane's chunk offset
-        bool        failed = false;
-
-        // Start the scan of tile (wave j, this CTA): one batch of independent loads.
-        auto start_scan = [&](uint32_t j) {
+        // Three tiles are in the scan pipeline at any time.  In iteration `it` the warp
+        //   (a) takes the counts of tile `it` and publishes them,
+        //   (b) issues the loads for tile `it - 1`, whose wave every CTA published about an iteration ago,
+        //   (c) finishes tile `it - 2` from the loads issued an iteration ago and hands it to the copiers.
+        // d[slot][k], lane l <-> descriptor of CTA l + 32k of the tile's wave; w[slot]: total word of the
+        // wave before it.  Tile j uses slot j & 1.
+        uint64_t d[2][kMaxWindows], w[2] = {0, 0};
 #pragma unroll
-            for (int k = 0; k < kMaxWindows; ++k) {
-                const uint32_t b = lane + 32u * k;
-                pend.d[k] = (b < cta) ? ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + b) : 1ull;
+        for (int k = 0; k < kMaxWindows; ++k) d[0][k] = d[1][k] = 1ull;
+        const uint32_t last_it = static_cast<uint32_t>((num_tiles - 1 - cta) / G);   // this CTA's last iteration
+
+        auto step = [&](auto parity, const uint32_t it) -> bool {
+            // parity == it & 1; tile it - 1 loads into slot kLoad, tile it - 2 is finished from slot kDone
+            constexpr int kLoad = 1 - decltype(parity)::value, kDone = decltype(parity)::value;
+            if (it <= last_it) {
+                // ---- (a)
+                const uint32_t s = it % kStages;
+                PROF_T(c0);
+                if (!mbar_wait(&s_counted[s], (it / kStages) & 1u, &s_abort)) {
+                    failed = true;
+                    return false;
+                }
+                PROF_T(c1);
+                PROF_ADD(8, c1 - c0);
+                const uint32_t c   = lane < kWarps ? s_cnt[s][lane] : 0u;
+                uint32_t       inc = c;
+#pragma unroll
+                for (int o = 1; o < kWarps; o <<= 1) {
+                    const uint32_t u = __shfl_up_sync(kFull, inc, o);
+                    if (lane >= static_cast<uint32_t>(o)) inc += u;
+                }
+                const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
+                if (lane == 0) {
+                    st_relaxed_u64(desc + tile_of(it), (static_cast<uint64_t>(agg) << 1) | 1ull);
+                    red_add_u64(wave_total + it, (1ull << kCountShift) + agg);
+                    s_agg[s] = agg;
+                }
+                if (lane < kWarps) s_off[s][lane] = inc - c;
             }
-            pend.prev_wave = (j > 0) ? ld_relaxed_u64(wave_total + (j - 1)) : (static_cast<uint64_t>(G) << kCountShift);
-        };
-        // Finish it: everything normally arrived long ago; entries that had not been published
-        // when the batch was issued are polled (bounded).  Publishes base and offsets to the workers.
-        auto finish_scan = [&](uint32_t j) -> bool {
-            uint64_t part  = 0;
-            uint32_t polls = 0;
-            uint64_t t0    = 0;
+            if (it >= 2 && it - 2 <= last_it) {
+                // ---- (c) first, so that its registers are free for (b)
+                const uint32_t j     = it - 2;
+                uint32_t       polls = 0;
+                uint64_t       t0    = 0;
+                for (;;) {
+                    bool missing = j > 0 && (w[kDone] >> kCountShift) != G;
 #pragma unroll
-            for (int k = 0; k < kMaxWindows; ++k) {
-                const uint32_t b = lane + 32u * k;
-                while (__any_sync(kFull, (pend.d[k] & 1ull) == 0)) {
+                    for (int k = 0; k < kMaxWindows; ++k) missing |= (d[kDone][k] & 1ull) == 0;
+                    if (!__any_sync(kFull, missing)) break;
                     PROF_ADD(11, 1);
                     __nanosleep(100);
                     if ((++polls & 255u) == 0) {
                         if (t0 == 0) t0 = now_ns();
-                        const bool give_up = (now_ns() - t0 > kWaitNs) || ld_relaxed_u32(abort_flag) != 0;
-                        if (__any_sync(kFull, give_up)) return false;
+                        if (__any_sync(kFull, (now_ns() - t0 > kWaitNs) || ld_relaxed_u32(abort_flag) != 0)) {
+                            failed = true;
+                            break;
+                        }
                     }
-                    if ((pend.d[k] & 1ull) == 0) pend.d[k] = ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + b);
+#pragma unroll
+                    for (int k = 0; k < kMaxWindows; ++k)
+                        if ((d[kDone][k] & 1ull) == 0)
+                            d[kDone][k] = ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + lane + 32u * k);
+                    if (j > 0 && (w[kDone] >> kCountShift) != G) w[kDone] = ld_relaxed_u64(wave_total + (j - 1));
                 }
-                part += pend.d[k] >> 1;
-            }
-            while ((pend.prev_wave >> kCountShift) != G) {           // uniform: every lane loaded the same word
-                PROF_ADD(12, 1);
-                __nanosleep(100);
-                if ((++polls & 255u) == 0) {
-                    if (t0 == 0) t0 = now_ns();
-                    if ((now_ns() - t0 > kWaitNs) || ld_relaxed_u32(abort_flag) != 0) return false;
+                if (failed) return false;
+                uint64_t part = 0;
+#pragma unroll
+                for (int k = 0; k < kMaxWindows; ++k) part += d[kDone][k] >> 1;
+                if (j > 0) waves_before += w[kDone] & ((1ull << kCountShift) - 1);
+                const uint64_t base = waves_before + warp_sum_u64(part);
+                const uint32_t ps   = j % kStages;
+                const uint64_t pt   = tile_of(j);
+                // exclusive count in front of each chunk of that tile
+                if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
+                    const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
+                    if (ch < chunks_total) a.prefix[ch] = base + s_off[ps][lane];
                 }
-                pend.prev_wave = ld_relaxed_u64(wave_total + (j - 1));
+                if (pt == num_tiles - 1 && lane == 0) {
+                    const uint64_t nnz = base + s_agg[ps];
+                    *a.nnz_out = nnz;
+                    __threadfence();
+                    const bool aborted = ld_relaxed_u32(abort_flag) != 0;
+                    if (a.dev_status)
+                        *a.dev_status = aborted ? BT_ERR_TIMEOUT : (nnz > a.capacity ? BT_ERR_CAPACITY : BT_OK);
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    s_base[ps] = base;
+                    mbar_arrive(&s_ready[ps]);                       // the copiers may take the tile
+                }
             }
-            if (j > 0) waves_before += pend.prev_wave & ((1ull << kCountShift) - 1);
-            const uint64_t base = waves_before + warp_sum_u64(part);
-            const uint32_t s    = j % kStages;
-            const uint64_t t    = tile_of(j);
-            if (lane == 0) s_base[s] = base;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&s_ready[s]);                 // workers may copy the tile out
-            // exclusive count in front of each chunk of this tile
-            if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
-                const uint64_t ch = t * kChunksPerTile + lane / kWarpsPerChunk;
-                if (ch < chunks_total) a.prefix[ch] = base + pend_chunk_off;
+            if (it >= 1 && it - 1 <= last_it) {
+                // ---- (b) one batch of independent loads
+                const uint32_t j = it - 1;
+#pragma unroll
+                for (int k = 0; k < kMaxWindows; ++k) {
+                    const uint32_t b = lane + 32u * k;
+                    d[kLoad][k] = (b < cta) ? ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + b) : 1ull;
+                }
+                w[kLoad] = (j > 0) ? ld_relaxed_u64(wave_total + (j - 1)) : 0ull;
             }
-            if (t == num_tiles - 1 && lane == 0) {
-                const uint64_t nnz = base + pend_agg;
-                *a.nnz_out = nnz;
-                __threadfence();
-                const bool aborted = ld_relaxed_u32(abort_flag) != 0;
-                if (a.dev_status)
-                    *a.dev_status = aborted ? BT_ERR_TIMEOUT : (nnz > a.capacity ? BT_ERR_CAPACITY : BT_OK);
-            }
-            return true;
+            return it < last_it + 2;
         };
 
-        uint32_t it = 0;
-        for (;; ++it) {
-            const uint64_t t64 = tile_of(it);
-            if (t64 >= num_tiles) break;
-            const uint32_t s = it % kStages;
-
-            PROF_T(c0);
-            if (!mbar_wait(&s_counted[s], (it / kStages) & 1u, &s_abort)) {
-                failed = true;
-                break;
-            }
-            PROF_T(c1);
-            if (lane == 0) DBG_MARK(it, 4, now_ns());
-            const uint32_t c   = lane < kWarps ? s_cnt[s][lane] : 0u;
-            uint32_t       inc = c;
-#pragma unroll
-            for (int o = 1; o < kWarps; o <<= 1) {
-                const uint32_t u = __shfl_up_sync(kFull, inc, o);
-                if (lane >= static_cast<uint32_t>(o)) inc += u;
-            }
-            const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
-            if (lane == 0) {
-                st_relaxed_u64(desc + t64, (static_cast<uint64_t>(agg) << 1) | 1ull);
-                red_add_u64(wave_total + it, (1ull << kCountShift) + agg);
-            }
-            if (lane < kWarps) s_off[s][lane] = inc - c;
-
-            // the tile counted one iteration ago: its loads have been in flight since then
-            if (it > 0 && !finish_scan(it - 1)) {
-                failed = true;
-                break;
-            }
-            if (lane == 0) DBG_MARK(it, 5, now_ns());
-            pend_agg       = agg;
-            pend_chunk_off = inc - c;
-            start_scan(it);
-            PROF_T(c2);
-            PROF_ADD(8, c1 - c0);
-            PROF_ADD(9, c2 - c1);
+        for (uint32_t it = 0;; it += 2) {
+            if (!step(std::integral_constant<int, 0>{}, it)) break;
+            if (!step(std::integral_constant<int, 1>{}, it + 1)) break;
         }
-        if (!failed && it > 0 && !finish_scan(it - 1)) failed = true;
         if (failed && lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort);
-#ifdef BT_PROFILE
-        if (lane == 0)
-            for (int k = 8; k < 13; ++k) atomicAdd(reinterpret_cast<unsigned long long *>(a.ws_header) + 8 + k, prof[k]);
-#endif
+        PROF_FLUSH(8, 13);
         return;
     }
 
-    // ---------------------------------------------------------------- worker warps
-    const uint32_t lt          = lanemask_lt();
-    U *const       vals        = static_cast<U *>(a.values);
-    const uint64_t words_total = (n + 31) >> 5;
-    const uint64_t capacity    = a.capacity;
-
-    for (uint32_t it = 0;; ++it) {
-        const uint32_t s   = it % kStages;
-        const uint64_t t64 = tile_of(it);
-
-        if (t64 < num_tiles) {
-            const uint32_t t     = static_cast<uint32_t>(t64);
-            U *const       tile  = tiles + static_cast<size_t>(s) * kTile;
-            const uint64_t first = t64 * kTile;
+    if (warp >= kFirstCopier) {
+        // ------------------------------------------------------------ copier warps
+        const uint32_t seg      = warp - kFirstCopier;
+        U *const       vals     = static_cast<U *>(a.values);
+        const uint64_t capacity = a.capacity;
+        for (uint32_t it = 0;; ++it) {
+            if (tile_of(it) >= num_tiles) break;
+            const uint32_t s = it % kStages;
             PROF_T(c0);
-            if (!mbar_wait(&s_full[s], (it / kStages) & 1u, &s_abort)) {
-                if (lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort);
-                break;
-            }
+            if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort)) break;
             PROF_T(c1);
-            if (tid == 0) DBG_MARK(it, 0, now_ns());
-            if (n - first < static_cast<uint64_t>(kTile)) {
-                // ragged last tile: fetch what the 16-byte granular bulk copy left out, zero the rest
-                const uint32_t have    = static_cast<uint32_t>(n - first);
-                const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
-                for (uint32_t e = by_bulk + tid; e < static_cast<uint32_t>(kTile); e += kWorkerThreads)
-                    tile[e] = (e < have) ? src[first + e] : U(0);
-                asm volatile("bar.sync %0, %1;" ::"n"(kBarWorkers), "n"(kWorkerThreads) : "memory");
-            }
-
-            // ---- per-warp in-place compaction of 1024 elements
-            U *const seg    = tile + warp * kWarpElems;
-            uint32_t run    = 0;
-            uint32_t myword = 0;
-#pragma unroll 1
-            for (int kb = 0; kb < 32; kb += 8) {
-                uint32_t v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) v[j] = seg[(kb + j) * 32 + lane];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint32_t x = v[j];
-                    if constexpr (RELU_DT >= 0) {
-                        x = ReluKeep<RELU_DT>::keep(x) ? x : 0u;
-                        if constexpr (WRITE_Y) {
-                            const uint64_t g = first + warp * kWarpElems + (kb + j) * 32 + lane;
-                            if (g < n) static_cast<U *>(a.y)[g] = static_cast<U>(x);
-                        }
-                    }
-                    const bool     p = x != 0u;
-                    const uint32_t b = __ballot_sync(kFull, p);
-                    if (lane == static_cast<uint32_t>(kb + j)) myword = b;
-                    if (p) seg[run + __popc(b & lt)] = static_cast<U>(x);
-                    run += __popc(b);
-                }
-            }
-            {
-                const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * 32 + lane;
-                if (w < words_total) a.bitmap[w] = myword;
-            }
-            if (lane == 0) {
-                s_cnt[s][warp] = run;
-                mbar_arrive(&s_counted[s]);                   // hand the count to the scan warp
-            }
-            PROF_T(c2);
-            if (tid == 0) DBG_MARK(it, 1, now_ns());
-            PROF_ADD(0, c1 - c0);
-            PROF_ADD(1, c2 - c1);
-        }
-
-        if (it >= static_cast<uint32_t>(kLag)) {
-            // ---- copy the packed slots of the tile compacted kLag iterations ago out, contiguous in values[]
-            const uint32_t pit = it - kLag;
-            if (tile_of(pit) >= num_tiles) {
-#ifdef BT_PROFILE
-                if (lane == 0 && warp == 0)
-                    for (int k = 0; k < 4; ++k)
-                        atomicAdd(reinterpret_cast<unsigned long long *>(a.ws_header) + 8 + k, prof[k]);
-#endif
-                return;                                        // every tile of this CTA is out
-            }
-            const uint32_t ps = pit % kStages;
-            PROF_T(c3);
-            if (!mbar_wait(&s_ready[ps], (pit / kStages) & 1u, &s_abort)) break;
-            PROF_T(c4);
-            if (tid == 0) DBG_MARK(pit, 2, now_ns());
-            const U *const pseg = tiles + static_cast<size_t>(ps) * kTile + warp * kWarpElems;
-            const uint32_t cnt  = s_cnt[ps][warp];
-            const uint64_t dst  = s_base[ps] + s_off[ps][warp];
-            if (dst + cnt <= capacity) {
-                for (uint32_t j = lane; j < cnt; j += 32) vals[dst + j] = pseg[j];
-            } else {
-                for (uint32_t j = lane; j < cnt; j += 32)
-                    if (dst + j < capacity) vals[dst + j] = pseg[j];
-            }
+            const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
+            const uint32_t cnt  = s_cnt[s][seg];
+            const uint64_t dst  = s_base[s] + s_off[s][seg];
+            if (dst + cnt <= capacity)
+                copy_out_segment<U, false>(pseg, lane, cnt, vals + dst, 0);
+            else
+                copy_out_segment<U, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
             __syncwarp();
-            if (lane == 0) {
-                __threadfence_block();
-                if (atomicAdd(&s_done[ps], 1u) == kWarps - 1) {
-                    // last warp out of this stage refills it with the tile it holds kStages iterations on
-                    __threadfence_block();
-                    s_done[ps]        = 0;
-                    const uint64_t nt = tile_of(pit + kStages);
-                    if (nt < num_tiles) issue_load(ps, static_cast<uint32_t>(nt));
-                }
-            }
-            PROF_T(c5);
-            if (tid == 0) DBG_MARK(pit, 3, now_ns());
-            PROF_ADD(2, c4 - c3);
-            PROF_ADD(3, c5 - c4);
+            asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
+            if (lane == 0) mbar_arrive(&s_empty[s]);
+            PROF_T(c2);
+            PROF_ADD(2, c1 - c0);
+            PROF_ADD(3, c2 - c1);
         }
+        if (seg == 0) { PROF_FLUSH(2, 4); }
+        return;
     }
 
-    // ---- only reached when a bounded wait ran out: before leaving, warp 0 lets the bulk copies
-    // that may still be in flight into this CTA's shared memory land (bounded, short)
-    if (warp == 0)
-        for (int s = 0; s < kStages; ++s) {
-            mbar_wait<false>(&s_full[s], 0, &s_abort, 20000000ull);
-            mbar_wait<false>(&s_full[s], 1, &s_abort, 20000000ull);
+    // ---------------------------------------------------------------- compactor warps
+    const uint32_t lt          = lanemask_lt();
+    const uint64_t words_total = (n + 31) >> 5;
+    for (uint32_t it = 0;; ++it) {
+        const uint64_t t64 = tile_of(it);
+        if (t64 >= num_tiles) break;
+        const uint32_t s     = it % kStages;
+        const uint32_t t     = static_cast<uint32_t>(t64);
+        U *const       tile  = tiles + static_cast<size_t>(s) * kTile;
+        const uint64_t first = t64 * kTile;
+        PROF_T(c0);
+        if (!mbar_wait(&s_full[s], (it / kStages) & 1u, &s_abort)) {
+            if (lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort);
+            break;
         }
+        PROF_T(c1);
+        if (n - first < static_cast<uint64_t>(kTile)) {
+            // ragged last tile: fetch what the 16-byte granular bulk copy left out, zero the rest
+            const uint32_t have    = static_cast<uint32_t>(n - first);
+            const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
+            for (uint32_t e = by_bulk + tid; e < static_cast<uint32_t>(kTile); e += kCompactThreads)
+                tile[e] = (e < have) ? src[first + e] : U(0);
+            asm volatile("bar.sync %0, %1;" ::"n"(kBarWorkers), "n"(kCompactThreads) : "memory");
+        }
+
+        // ---- in-place compaction of this warp's segment
+        const uint64_t e0     = first + warp * kSeg;                 // first element of the segment
+        uint32_t       yvalid = 0;
+        U             *y      = nullptr;
+        if constexpr (WRITE_Y) {
+            y      = static_cast<U *>(a.y) + e0;
+            yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
+        }
+        const uint32_t run = compact_segment<U, RELU_DT, WRITE_Y, kSteps>(
+            smem_addr(tile + warp * kSeg), smem_addr(&s_words[warp][0]), lane, lt, y, yvalid);
+        __syncwarp();
+        if (lane < kSteps) {
+            const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * kSteps + lane;
+            if (w < words_total) a.bitmap[w] = s_words[warp][lane];
+        }
+        __syncwarp();
+        if (lane == 0) {
+            s_cnt[s][warp] = run;
+            mbar_arrive(&s_counted[s]);                   // hand the count to the scan warp
+        }
+        PROF_T(c2);
+        PROF_ADD(0, c1 - c0);
+        PROF_ADD(1, c2 - c1);
+    }
+    if (warp == 0) { PROF_FLUSH(0, 2); }
 }
 
 // Launch shape of one kernel instantiation on one device: the opt-in shared
@@ -467,14 +549,14 @@ struct LaunchShape {
     }
 };
 
-template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kStages, int kLag>
+template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages>
 cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
 {
-    constexpr int kTile    = kWarps * kWarpElems;
-    constexpr int kThreads = kWarps * 32 + 32;
+    constexpr int kTile    = kWarps * kSeg;
+    constexpr int kThreads = kWarps * 64 + 64;
     constexpr size_t kSmem = static_cast<size_t>(kStages) * kTile * sizeof(U);
     static LaunchShape shape;   // one per instantiation
-    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, kWarps, kStages, kLag>;
+    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, kWarps, kSeg, kStages>;
 
     const uint32_t num_tiles = static_cast<uint32_t>((a.n + kTile - 1) / kTile);
     int            max_grid  = 0;
@@ -501,13 +583,12 @@ cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
     static const int cfg = [] { const char *e = getenv("BT_CFG"); return e ? atoi(e) : 0; }();
     constexpr int B = sizeof(U) == 4 ? 1 : 2;   // 16-bit tiles are half the bytes: room for twice the stages
     switch (cfg) {
-    case 1: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 6 * B, 2>(a, stream);      // 1 CTA/SM, 3 loading
-    case 2: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 6 * B, 3>(a, stream);      // 1 CTA/SM, lag 3
-    case 3: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 6 * B, 2>(a, stream);      // 2 CTAs/SM
-    case 4: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 4 * B, 2>(a, stream);      // 3 CTAs/SM
-    case 5: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 7 * B, 2>(a, stream);      // 1 CTA/SM, 4 loading
-    case 6: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 7 * B, 3>(a, stream);      // 2 CTAs/SM, lag 3
-    default: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 5 * B, 2>(a, stream);     // 1 CTA/SM, 2 loading
+    case 1: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 6 * B>(a, stream);
+    case 2: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 5 * B>(a, stream);
+    case 3: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 1024, 7 * B>(a, stream);      // 4096-element tiles, 2 CTAs/SM
+    case 4: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 512, 12 * B>(a, stream);      // 4096-element tiles, 8 x 512
+    case 5: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 1024, 12 * B>(a, stream);     // 4096-element tiles, 1 CTA/SM
+    default: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7 * B>(a, stream);
     }
 }
 
