@@ -580,16 +580,15 @@ cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
 template <typename U, int RELU_DT, bool WRITE_Y>
 cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
 {
+    // 8 compactor + 8 copier warps, 8192-element tiles, a ring of 192 KB: one CTA per SM
+    constexpr int kStages = sizeof(U) == 4 ? 6 : 12;
+#ifdef BT_PROFILE
     static const int cfg = [] { const char *e = getenv("BT_CFG"); return e ? atoi(e) : 0; }();
-    constexpr int B = sizeof(U) == 4 ? 1 : 2;   // 16-bit tiles are half the bytes: room for twice the stages
-    switch (cfg) {
-    case 1: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 6 * B>(a, stream);
-    case 2: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 5 * B>(a, stream);
-    case 3: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 1024, 7 * B>(a, stream);      // 4096-element tiles, 2 CTAs/SM
-    case 4: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 512, 12 * B>(a, stream);      // 4096-element tiles, 8 x 512
-    case 5: return launch_shaped<U, RELU_DT, WRITE_Y, 4, 1024, 12 * B>(a, stream);     // 4096-element tiles, 1 CTA/SM
-    default: return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7 * B>(a, stream);
-    }
+    if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, kStages + 1>(a, stream);
+    if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, kStages - 1>(a, stream);
+    if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 512, kStages>(a, stream);
+#endif
+    return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, kStages>(a, stream);
 }
 
 }  // namespace
