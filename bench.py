@@ -123,6 +123,27 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------
+# DRAM bytes per launch (read + write) of the dominant kernel class over one step of this workload, from the ncu
+# capture summarised in profiles/bench_cfg2_launch_list.md (bytes; None where no capture exists)
+NCU_TRAFFIC_PER_LAUNCH = {"bt_compress": 18.26e6, "bt_relu_fwd_compress": 18.28e6}
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time: the job is as fast as its slowest GPU."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(dense_bytes_per_rank_step: int, world: int, ms_per_step: float) -> float:
+    """Dense-equivalent GB/s of the whole job: every rank processes its own batch shard (weak scaling)."""
+    return world * dense_bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -416,18 +437,13 @@ def run_ours(args):
         e2e = run_e2e(step, graph, min(args.steps, 10), world)
     sampler.stop()
 
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-        if e2e is not None:
-            t = torch.tensor([e2e["ms"]], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e["ms"] = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
+    if e2e is not None:
+        e2e["ms"] = max_over_ranks(e2e["ms"], world, dev)
 
     if rank == 0:
         ms_step = ms_total / args.steps
-        value = world * step.dense_bytes_per_step / (ms_step * 1e-3) / 1e9
+        value = whole_job_value(step.dense_bytes_per_step, world, ms_step)
         # roofline of the dominant kernel class
         dom = max(per_op, key=lambda k: per_op[k]["ms"])
         alg = sum(algorithmic_bytes(dom, l["n"], z, 4) for l, z in zip(step.layers, nnz))
@@ -452,7 +468,8 @@ def run_ours(args):
             "gpu_launches": step.launches_per_step * args.steps,
             "roofline": {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak,
                          "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": peak_kind,
-                         "traffic": None,
+                         "traffic": NCU_TRAFFIC_PER_LAUNCH.get(dom),
+                         "algorithmic_bytes_per_launch": round(alg / len(step.layers)),
                          "avg_launch_ms": round(avg_ms, 5), "launches_timed": launches,
                          "largest_layer": {"elements": step.layers[0]["n"], "ms": round(big_ms, 5),
                                            "achieved": round(big_alg / big_ms / 1e6, 1),
@@ -462,7 +479,7 @@ def run_ours(args):
         }
         if e2e is not None:
             e2e_ms = e2e["ms"] / e2e["steps"]
-            line["e2e"] = {"value": round(world * step.dense_bytes_per_step / (e2e_ms * 1e-3) / 1e9, 3),
+            line["e2e"] = {"value": round(whole_job_value(step.dense_bytes_per_step, world, e2e_ms), 3),
                            "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": round(e2e_ms, 3), "steps": e2e["steps"]}
         if world == 1 and not args.no_large:
