@@ -481,7 +481,8 @@ def run_ours(args):
             e2e_ms = e2e["ms"] / e2e["steps"]
             line["e2e"] = {"value": round(whole_job_value(step.dense_bytes_per_step, world, e2e_ms), 3),
                            "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                           "ms_per_step": round(e2e_ms, 3), "steps": e2e["steps"]}
+                           "ms_per_step": round(e2e_ms, 3), "steps": e2e["steps"],
+                           "api": "bt_*_host entry points, pinned host buffers"}
         if world == 1 and not args.no_large:
             line["large_tensor_kernels"] = large_tensor_kernels(dev, peak)
         if world == 1 and not args.no_cpu_baseline:
@@ -499,35 +500,46 @@ def run_ours(args):
 
 
 def run_e2e(step: Cfg2Step, graph, steps: int, world: int):
-    """Step time with the inputs coming from pinned host memory and the results (restored
-    activation and input gradient of every layer, the nnz words) going back to host memory."""
+    """The same step through the host-buffer entry points of the C ABI: every tensor the step consumes
+    starts in pinned host memory and every tensor it produces (both stashes, the restored activation, the
+    input gradient) ends there; the host<->device copies happen inside the calls, inside the timed region."""
     import torch
-    host = []
-    for l in step.layers:
-        host.append(dict(act=l["act"].cpu().pin_memory(), pre=l["pre"].cpu().pin_memory(),
-                         grad=l["grad"].cpu().pin_memory(),
-                         nnz=torch.empty(1, dtype=torch.int64).pin_memory()))
+    B = step.B
+    dev = step.restored.device
     n_max = step.restored.numel()
+    staging = torch.empty(B.bt_host_staging_bytes(n_max, torch.float32), dtype=torch.uint8, device=dev)
+    host = []
+    h2d = d2h = 0
+    for l in step.layers:
+        n = l["n"]
+        h = dict(act=l["act"].cpu().pin_memory(), pre=l["pre"].cpu().pin_memory(), grad=l["grad"].cpu().pin_memory())
+        for tag in ("a", "b"):
+            h["bitmap_" + tag] = torch.empty((n + 31) // 32, dtype=torch.int32).pin_memory()
+            h["values_" + tag] = torch.empty(n, dtype=torch.float32).pin_memory()
+            h["prefix_" + tag] = torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory()
+            h["nnz_" + tag] = torch.zeros(1, dtype=torch.int64).pin_memory()
+        host.append(h)
     out_restored = torch.empty(n_max, dtype=torch.float32).pin_memory()
     out_gin = torch.empty(n_max, dtype=torch.float32).pin_memory()
-    h2d = sum(3 * 4 * l["n"] for l in step.layers)
-    d2h = sum(8 for _ in step.layers) + 2 * 4 * step.layers[0]["n"]
+    for l, z in zip(step.layers, step.nnz()):
+        n = l["n"]
+        comp = B.bt_compressed_bytes(n, z, torch.float32)
+        h2d += 4 * n + 4 * n + comp + (4 * ((n + 31) // 32) + 4 * n)      # compress, fused forward, decompress, backward
+        d2h += (comp + 8) + (comp + 8) + 4 * n + 4 * n
 
     def one():
         for l, h in zip(step.layers, host):
-            l["act"].copy_(h["act"], non_blocking=True)
-            l["pre"].copy_(h["pre"], non_blocking=True)
-            l["grad"].copy_(h["grad"], non_blocking=True)
-        graph.replay()
-        for l, h in zip(step.layers, host):
-            h["nnz"].copy_(l["stash_a"].nnz_out, non_blocking=True)
-        n0 = step.layers[0]["n"]
-        out_restored[:n0].copy_(step.restored[:n0], non_blocking=True)
-        out_gin[:n0].copy_(step.gin[:n0], non_blocking=True)
+            B.bt_compress_host(h["act"], h["bitmap_a"], h["values_a"], h["prefix_a"], h["nnz_a"], staging)
+            B.bt_relu_fwd_compress_host(h["pre"], None, h["bitmap_b"], h["values_b"], h["prefix_b"], h["nnz_b"], staging)
+        for l, h in zip(reversed(step.layers), reversed(host)):
+            n = l["n"]
+            B.bt_decompress_host(h["bitmap_a"], h["values_a"], h["prefix_a"], int(h["nnz_a"].item()),
+                                 out_restored[:n], staging)
+            B.bt_relu_bwd_from_bitmap_host(h["bitmap_b"], h["grad"], out_gin[:n], staging)
 
-    for _ in range(2):
-        one()
+    one()
     torch.cuda.synchronize()
+    assert torch.equal(out_restored[:step.layers[0]["n"]].view(torch.int32), host[0]["act"].view(torch.int32))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(steps):

@@ -134,6 +134,44 @@ int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out
 int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
                             uint64_t n, int dtype, void *grad_in, void *stream);
 
+/*
+ * Host-buffer forms.  The paper's own implementation keeps the stash in host
+ * memory (section 4, "Implementation Details": std::bitset and std::vector);
+ * these calls serve callers whose dense tensors or stashes live there.  Every
+ * `host_*` pointer is a HOST pointer (pinned memory is copied fastest, pageable
+ * memory works), `dev_staging` is a DEVICE buffer of at least
+ * bt_host_staging_bytes(n, dtype) bytes, 256-byte aligned, owned by the caller
+ * and free for reuse after the call.  Each call copies its inputs to the
+ * staging area, runs the same kernels as the device forms, copies the results
+ * back and SYNCHRONISES the stream before it returns (the packed values can be
+ * copied only once nnz is known), so device-side conditions (BT_ERR_CAPACITY,
+ * BT_ERR_TIMEOUT) arrive in the return value.  host_values_capacity counts
+ * elements; if nnz exceeds it the first host_values_capacity values are
+ * copied, *host_nnz holds the true count and BT_ERR_CAPACITY is returned.
+ * Otherwise arguments mean what they mean in the device forms.
+ */
+size_t bt_host_staging_bytes(uint64_t n, int dtype);
+
+int bt_compress_host(const void *host_dense, uint64_t n, int dtype,
+                     uint32_t *host_bitmap, void *host_values, uint64_t host_values_capacity,
+                     uint64_t *host_chunk_prefix, uint64_t *host_nnz,
+                     void *dev_staging, size_t dev_staging_bytes, void *stream);
+
+/* nnz: number of packed values in host_values (as returned by the compressor) */
+int bt_decompress_host(const uint32_t *host_bitmap, const void *host_values,
+                       const uint64_t *host_chunk_prefix, uint64_t nnz, uint64_t n, int dtype,
+                       void *host_dense_out, void *dev_staging, size_t dev_staging_bytes, void *stream);
+
+/* host_y_out may be NULL */
+int bt_relu_fwd_compress_host(const void *host_pre_act, uint64_t n, int dtype, void *host_y_out,
+                              uint32_t *host_bitmap, void *host_values, uint64_t host_values_capacity,
+                              uint64_t *host_chunk_prefix, uint64_t *host_nnz,
+                              void *dev_staging, size_t dev_staging_bytes, void *stream);
+
+int bt_relu_bwd_from_bitmap_host(const uint32_t *host_bitmap, const void *host_grad_out,
+                                 uint64_t n, int dtype, void *host_grad_in,
+                                 void *dev_staging, size_t dev_staging_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

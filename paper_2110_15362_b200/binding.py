@@ -23,7 +23,8 @@ CHUNK = 4096
 
 DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_BF16}
 EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
-           "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap")
+           "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
+           "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -61,6 +62,16 @@ def lib() -> ctypes.CDLL:
         L.bt_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
         L.bt_relu_bwd_from_bitmap.restype = i32
         L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
+        L.bt_host_staging_bytes.restype = sz
+        L.bt_host_staging_bytes.argtypes = [u64, i32]
+        L.bt_compress_host.restype = i32
+        L.bt_compress_host.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp]
+        L.bt_decompress_host.restype = i32
+        L.bt_decompress_host.argtypes = [vp, vp, vp, u64, u64, i32, vp, vp, sz, vp]
+        L.bt_relu_fwd_compress_host.restype = i32
+        L.bt_relu_fwd_compress_host.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp]
+        L.bt_relu_bwd_from_bitmap_host.restype = i32
+        L.bt_relu_bwd_from_bitmap_host.argtypes = [vp, vp, u64, i32, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -130,6 +141,51 @@ def bt_relu_bwd_from_bitmap(bitmap: torch.Tensor, grad_out: torch.Tensor, grad_i
     st = lib().bt_relu_bwd_from_bitmap(_ptr(bitmap), _ptr(grad_out), n, DTYPE_CODE[grad_out.dtype], _ptr(grad_in),
                                        _stream(stream))
     return _check("bt_relu_bwd_from_bitmap", st, check)
+
+
+# ---- host-buffer forms: `host_*` are CPU tensors (pinned for speed), `staging` a CUDA uint8 tensor
+def bt_host_staging_bytes(n: int, dtype) -> int:
+    return int(lib().bt_host_staging_bytes(n, DTYPE_CODE.get(dtype, dtype)))
+
+
+def _nbytes(t: torch.Tensor) -> int:
+    return t.numel() * t.element_size()
+
+
+def bt_compress_host(host_dense: torch.Tensor, host_bitmap: torch.Tensor, host_values: torch.Tensor,
+                     host_chunk_prefix: torch.Tensor, host_nnz: torch.Tensor, staging: torch.Tensor,
+                     *, stream=None, check: bool = True) -> int:
+    st = lib().bt_compress_host(_ptr(host_dense), host_dense.numel(), DTYPE_CODE[host_dense.dtype], _ptr(host_bitmap),
+                                _ptr(host_values), host_values.numel(), _ptr(host_chunk_prefix), _ptr(host_nnz),
+                                _ptr(staging), _nbytes(staging), _stream(stream))
+    return _check("bt_compress_host", st, check)
+
+
+def bt_relu_fwd_compress_host(host_pre_act: torch.Tensor, host_y_out: Optional[torch.Tensor],
+                              host_bitmap: torch.Tensor, host_values: torch.Tensor, host_chunk_prefix: torch.Tensor,
+                              host_nnz: torch.Tensor, staging: torch.Tensor, *, stream=None, check: bool = True) -> int:
+    st = lib().bt_relu_fwd_compress_host(_ptr(host_pre_act), host_pre_act.numel(), DTYPE_CODE[host_pre_act.dtype],
+                                         _ptr(host_y_out), _ptr(host_bitmap), _ptr(host_values), host_values.numel(),
+                                         _ptr(host_chunk_prefix), _ptr(host_nnz), _ptr(staging), _nbytes(staging),
+                                         _stream(stream))
+    return _check("bt_relu_fwd_compress_host", st, check)
+
+
+def bt_decompress_host(host_bitmap: torch.Tensor, host_values: torch.Tensor, host_chunk_prefix: torch.Tensor,
+                       nnz: int, host_dense_out: torch.Tensor, staging: torch.Tensor, *, stream=None,
+                       check: bool = True) -> int:
+    st = lib().bt_decompress_host(_ptr(host_bitmap), _ptr(host_values), _ptr(host_chunk_prefix), nnz,
+                                  host_dense_out.numel(), DTYPE_CODE[host_dense_out.dtype], _ptr(host_dense_out),
+                                  _ptr(staging), _nbytes(staging), _stream(stream))
+    return _check("bt_decompress_host", st, check)
+
+
+def bt_relu_bwd_from_bitmap_host(host_bitmap: torch.Tensor, host_grad_out: torch.Tensor, host_grad_in: torch.Tensor,
+                                 staging: torch.Tensor, *, stream=None, check: bool = True) -> int:
+    st = lib().bt_relu_bwd_from_bitmap_host(_ptr(host_bitmap), _ptr(host_grad_out), host_grad_out.numel(),
+                                            DTYPE_CODE[host_grad_out.dtype], _ptr(host_grad_in), _ptr(staging),
+                                            _nbytes(staging), _stream(stream))
+    return _check("bt_relu_bwd_from_bitmap_host", st, check)
 
 
 class Stash:
