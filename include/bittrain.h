@@ -62,7 +62,8 @@ enum {
     BT_ERR_WORKSPACE = 4,  /* workspace smaller than bt_workspace_bytes(n)             */
     BT_ERR_CAPACITY = 5,   /* device: nnz > values_capacity (see bt_compress)          */
     BT_ERR_TIMEOUT = 6,    /* device: a bounded wait inside the kernel ran out         */
-    BT_ERR_CUDA = 7        /* the CUDA runtime reported an error at launch             */
+    BT_ERR_CUDA = 7,       /* the CUDA runtime reported an error at launch             */
+    BT_ERR_TOO_LARGE = 8   /* n exceeds what the call can handle (bt_compress_noalloc) */
 };
 
 /*
@@ -133,6 +134,39 @@ int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out
  */
 int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
                             uint64_t n, int dtype, void *grad_in, void *stream);
+
+/*
+ * bt_compress for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: its implementation runs on the host and allocates freely.)
+ *
+ * Who needs it: code that runs where asking for device memory is not an
+ * option -- a training hook called while the framework's allocator is frozen
+ * (every byte of a memory plan already handed out, or a region in which an
+ * allocation would synchronise the device or simply fail), or a plug-in that
+ * receives its input and output buffers from a runtime that owns the device
+ * memory and gives it no way to request a workspace.  bt_compress wants such a
+ * workspace; here it is built into the library instead: a 262,400-byte array in
+ * device memory that every GPU which loads the library holds until the process
+ * exits.  That fixes the largest tensor: n <= BT_NOALLOC_MAX_ELEMS (2^26
+ * elements); a larger n returns BT_ERR_TOO_LARGE and nothing is launched.
+ *
+ * The call allocates nothing and frees nothing, on the host path or on the
+ * device.  The caller still passes every input and output buffer; arguments,
+ * outputs and *dev_status are exactly those of bt_compress without the two
+ * workspace parameters.  The first call on each device looks up the array's
+ * device address (one runtime query, made with that device current) -- make
+ * that first call outside any stream capture; later calls only launch.  All
+ * calls on a device share the one array: the part a call uses is cleared at
+ * its start, so nothing depends on the previous call's contents, but two calls
+ * whose execution overlaps on the GPU (different streams) race on it and give
+ * undefined results -- keep them on one stream or order them with events.
+ */
+#define BT_NOALLOC_MAX_ELEMS (1ull << 26)
+
+int bt_compress_noalloc(const void *dense, uint64_t n, int dtype,
+                        uint32_t *bitmap, void *values, uint64_t values_capacity,
+                        uint64_t *chunk_prefix, uint64_t *nnz_out,
+                        int32_t *dev_status, void *stream);
 
 /*
  * Host-buffer forms.  The paper's own implementation keeps the stash in host

@@ -16,15 +16,17 @@ import torch
 from . import build as _build
 
 BT_F32, BT_F16, BT_BF16 = 0, 1, 2
-BT_OK, BT_ERR_NULL, BT_ERR_DTYPE, BT_ERR_ALIGN, BT_ERR_WORKSPACE, BT_ERR_CAPACITY, BT_ERR_TIMEOUT, BT_ERR_CUDA = range(8)
+(BT_OK, BT_ERR_NULL, BT_ERR_DTYPE, BT_ERR_ALIGN, BT_ERR_WORKSPACE, BT_ERR_CAPACITY, BT_ERR_TIMEOUT, BT_ERR_CUDA,
+ BT_ERR_TOO_LARGE) = range(9)
 STATUS_NAMES = ["BT_OK", "BT_ERR_NULL", "BT_ERR_DTYPE", "BT_ERR_ALIGN", "BT_ERR_WORKSPACE", "BT_ERR_CAPACITY",
-                "BT_ERR_TIMEOUT", "BT_ERR_CUDA"]
+                "BT_ERR_TIMEOUT", "BT_ERR_CUDA", "BT_ERR_TOO_LARGE"]
+NOALLOC_MAX_ELEMS = 1 << 26
 CHUNK = 4096
 
 DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_BF16}
 EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
-           "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host")
+           "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -62,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.bt_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
         L.bt_relu_bwd_from_bitmap.restype = i32
         L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
+        L.bt_compress_noalloc.restype = i32
+        L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
         L.bt_host_staging_bytes.argtypes = [u64, i32]
         L.bt_compress_host.restype = i32
@@ -111,6 +115,18 @@ def bt_compress(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor,
                            _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace),
                            workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream))
     return _check("bt_compress", st, check)
+
+
+def bt_compress_noalloc(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,
+                        nnz_out: torch.Tensor, dev_status: Optional[torch.Tensor] = None, *, n: Optional[int] = None,
+                        values_capacity: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """bt_compress without a workspace argument: the scratch is a fixed array inside the library, so the
+    call allocates nothing (for callers that may not); n is limited to NOALLOC_MAX_ELEMS."""
+    n = dense.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    st = lib().bt_compress_noalloc(_ptr(dense), n, DTYPE_CODE[dense.dtype], _ptr(bitmap), _ptr(values), cap,
+                                   _ptr(chunk_prefix), _ptr(nnz_out), _ptr(dev_status), _stream(stream))
+    return _check("bt_compress_noalloc", st, check)
 
 
 def bt_relu_fwd_compress(pre_act: torch.Tensor, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
