@@ -1,0 +1,201 @@
+"""Parity at the full sizes of the five workload configurations, in the launch configuration the
+benchmark times (the library's own launch shapes, one stream).  A tensor of up to a gigabyte is too
+much for the single-threaded oracle, so each one is checked three ways: (1) the oracle on randomly
+sampled 4096-element chunks (bitmap words, packed values, prefix entry, restored elements), (2) torch
+routines on the GPU over the whole tensor (boolean indexing, packed bits, chunk counts, relu, where) as
+an independent full-size check, (3) properties that hold at any size (nnz == popcount(bitmap), the
+round trip is the identity bit for bit, bytes formula).  The small layers of configuration 2 go through
+the oracle whole."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2110_15362_b200 import binding as B
+from paper_2110_15362_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+IV = {2: torch.int16, 4: torch.int32}
+
+
+def bits_of(t):
+    return t.view(IV[t.element_size()])
+
+
+def torch_bitmap(mask: torch.Tensor) -> torch.Tensor:
+    """LSB-first uint32 words of a boolean vector, built with torch on the GPU in slices."""
+    n = mask.numel()
+    out = torch.empty((n + 31) // 32, dtype=torch.int32, device=mask.device)
+    shifts = torch.arange(32, device=mask.device, dtype=torch.int64)
+    step = 1 << 24
+    for lo in range(0, n, step):
+        m = mask[lo:lo + step]
+        pad = (-m.numel()) % 32
+        if pad:
+            m = torch.nn.functional.pad(m, (0, pad))
+        w = (m.view(-1, 32).to(torch.int64) << shifts).sum(dim=1)
+        out[lo // 32: lo // 32 + w.numel()] = w.to(torch.int32)
+    return out
+
+
+def torch_prefix(mask: torch.Tensor) -> torch.Tensor:
+    n = mask.numel()
+    pad = (-n) % 4096
+    m = torch.nn.functional.pad(mask, (0, pad)) if pad else mask
+    per_chunk = m.view(-1, 4096).sum(dim=1, dtype=torch.int64)
+    return torch.cumsum(per_chunk, 0) - per_chunk
+
+
+def check_against_torch(st: B.Stash, y: torch.Tensor):
+    """Whole-tensor check of a stash of y (y already post-ReLU where that applies)."""
+    mask = bits_of(y) != 0
+    nnz = int(mask.sum().item())
+    assert st.status == B.BT_OK and st.nnz == nnz
+    assert torch.equal(st.bitmap, torch_bitmap(mask))
+    assert torch.equal(st.chunk_prefix, torch_prefix(mask))
+    assert torch.equal(bits_of(st.values[:nnz]), bits_of(y)[mask])
+    # nnz == popcount(bitmap), by a different route than the packing above
+    b = st.bitmap.view(torch.uint8)
+    pop = sum(int(((b >> k) & 1).sum(dtype=torch.int64).item()) for k in range(8))
+    assert pop == nnz
+    n = y.numel()
+    assert B.bt_compressed_bytes(n, nnz, y.dtype) == 4 * ((n + 31) // 32) + nnz * y.element_size() + 8 * ((n + 4095) // 4096)
+    return nnz
+
+
+def check_sampled_chunks(oracle, st: B.Stash, y: torch.Tensor, restored, seed: int, samples: int = 24):
+    n = y.numel()
+    chunks = (n + 4095) // 4096
+    rng = np.random.default_rng(seed)
+    picks = sorted(set(rng.integers(0, chunks, size=samples).tolist()) | {0, chunks - 1})
+    prefix = st.chunk_prefix
+    nnz = st.nnz
+    for c in picks:
+        lo, hi = c * 4096, min(n, (c + 1) * 4096)
+        ref = oracle.compress(W.raw_numpy(y[lo:hi]))
+        words = W.raw_numpy(st.bitmap[lo // 32:(hi + 31) // 32]).view(np.uint32)
+        assert np.array_equal(words, ref.bitmap), c
+        start = int(prefix[c].item())
+        end = int(prefix[c + 1].item()) if c + 1 < chunks else nnz
+        assert end - start == ref.nnz, c
+        assert np.array_equal(W.raw_numpy(st.values[start:end]), ref.values), c
+        if restored is not None:
+            assert np.array_equal(W.raw_numpy(restored[lo:hi]), W.raw_numpy(y[lo:hi])), c
+
+
+def compress(x, ws=None):
+    n = x.numel()
+    st = B.Stash(n, x.dtype, DEV)
+    B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws if ws is not None else B.new_workspace(n, DEV),
+                  st.dev_status)
+    return st
+
+
+def decompress(st, like):
+    out = torch.empty_like(like)
+    B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, out)
+    return out
+
+
+def test_cfg2_resnet18_batch32_every_layer_against_the_oracle(oracle):
+    for i, shape, n in W.iter_layers(W.resnet18_shapes(32)):
+        x = W.cfg2_layer(i, shape, DEV).reshape(-1)
+        st = compress(x)
+        back = decompress(st, x)
+        torch.cuda.synchronize()
+        if n <= 8_000_000:                                   # small enough for the oracle, whole
+            ref = oracle.compress(W.raw_numpy(x))
+            assert st.nnz == ref.nnz and st.status == B.BT_OK
+            assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), ref.bitmap)
+            assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), ref.prefix)
+            assert np.array_equal(W.raw_numpy(st.values[:ref.nnz]), ref.values)
+        else:
+            check_against_torch(st, x)
+            check_sampled_chunks(oracle, st, x, back, seed=i)
+        assert torch.equal(bits_of(back), bits_of(x))
+
+
+@pytest.mark.parametrize("variant", ["iid", "clustered"])
+@pytest.mark.parametrize("s", W.SPARSITY_SWEEP)
+def test_cfg3_one_gibibyte_sparsity_sweep(oracle, variant, s):
+    n = 1 << 28
+    idx = W.SPARSITY_SWEEP.index(s)
+    x = (W.cfg3_iid if variant == "iid" else W.cfg3_clustered)(n, s, idx, DEV)
+    st = compress(x)
+    back = decompress(st, x)
+    nnz = check_against_torch(st, x)
+    assert abs((1 - nnz / n) - s) < 0.02
+    assert torch.equal(bits_of(back), bits_of(x))
+    check_sampled_chunks(oracle, st, x, back, seed=17 + idx)
+    # the bitmap-masked gradient at the same size
+    g = W.cfg2_grad(idx, (n,), DEV)
+    gin = torch.empty_like(g)
+    B.bt_relu_bwd_from_bitmap(st.bitmap, g, gin)
+    assert torch.equal(bits_of(gin), bits_of(torch.where(bits_of(x) != 0, g, torch.zeros((), device=DEV))))
+    del x, st, back, g, gin
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("kind", ["bf16", "f16"])
+def test_cfg4_vgg16_batch64_fused_relu_pair(oracle, kind):
+    shapes = W.vgg16_shapes(64)
+    seen = set()
+    for i, shape, n in W.iter_layers(shapes):
+        if shape in seen and i not in (0, len(shapes) - 1):
+            continue                                         # one tensor per distinct shape (plus first and last)
+        seen.add(shape)
+        pre = W.cfg4_preact(i, shape, kind, DEV).reshape(-1)
+        g = W.cfg4_grad(i, shape, kind, DEV).reshape(-1)
+        y_ref = (torch.relu(pre) + 0.0).to(pre.dtype)        # +0.0: torch.relu keeps the sign of -0.0
+        ws = B.new_workspace(n, DEV)
+        # stash only
+        st = B.Stash(n, pre.dtype, DEV)
+        B.bt_relu_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        check_against_torch(st, y_ref)
+        check_sampled_chunks(oracle, st, y_ref, None, seed=40 + i, samples=12)
+        # with the dense output
+        st2 = B.Stash(n, pre.dtype, DEV)
+        y = torch.empty_like(pre)
+        B.bt_relu_fwd_compress(pre, y, st2.bitmap, st2.values, st2.chunk_prefix, st2.nnz_out, ws, st2.dev_status)
+        assert torch.equal(bits_of(y), bits_of(y_ref))
+        assert torch.equal(st2.bitmap, st.bitmap) and st2.nnz == st.nnz
+        assert torch.equal(bits_of(st2.values[:st.nnz]), bits_of(st.values[:st.nnz]))
+        # backward from the bitmap
+        gin = torch.empty_like(g)
+        B.bt_relu_bwd_from_bitmap(st.bitmap, g, gin)
+        assert torch.equal(bits_of(gin), bits_of(torch.where(pre > 0, g, torch.zeros((), device=DEV, dtype=g.dtype))))
+        del pre, g, y, y_ref, st, st2, gin
+        torch.cuda.empty_cache()
+
+
+def test_cfg5_mobilenetv2_batch128_forward_then_reverse(oracle):
+    shapes = W.mobilenetv2_shapes(128)
+    fractions = W.cfg5_zero_fractions(len(shapes))
+    assert len(shapes) == 35 and sum(W.numel(s) for s in shapes) == 781541376
+    n_max = max(W.numel(s) for s in shapes)
+    ws = B.new_workspace(n_max, DEV)
+    stashes, nnzs, total_bytes = [], [], 0
+    for i, shape, n in W.iter_layers(shapes):                 # forward order, one stream
+        x = W.cfg5_layer(i, shape, fractions[i], DEV).reshape(-1)
+        st = B.Stash(n, x.dtype, DEV, values_capacity=n)
+        B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        nnz = int((bits_of(x) != 0).sum().item())
+        assert st.nnz == nnz and st.status == B.BT_OK
+        assert abs((1 - nnz / n) - fractions[i]) < 0.02
+        if i % 6 == 0:
+            check_sampled_chunks(oracle, st, x, None, seed=70 + i, samples=8)
+        # keep the exact-size stash, as a training step would (values trimmed to nnz)
+        st.values = st.values[:nnz].clone()
+        stashes.append((i, shape, n, st))
+        nnzs.append(nnz)
+        total_bytes += B.bt_compressed_bytes(n, nnz, torch.float32)
+        del x
+    dense_bytes = 4 * sum(n for _, _, n, _ in stashes)
+    assert total_bytes == sum(n // 8 + 4 * z + 8 * (n // 4096) for (_, _, n, _), z in zip(stashes, nnzs))
+    assert 0.15 * dense_bytes < total_bytes < 0.36 * dense_bytes      # 70-85 % zeros: about 18-33 % of dense
+    for i, shape, n, st in reversed(stashes):                # restore in reverse order
+        back = torch.empty(n, dtype=torch.float32, device=DEV)
+        B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, back)
+        x = W.cfg5_layer(i, shape, fractions[i], DEV).reshape(-1)
+        assert torch.equal(bits_of(back), bits_of(x))
+        del back, x
