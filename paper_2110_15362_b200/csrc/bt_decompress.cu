@@ -4,13 +4,15 @@
 //
 // One warp, one quarter chunk (1024 elements = 32 bitmap words):
 //   - lane l loads the 4 words 4l..4l+3 of the WHOLE chunk (one 512-byte
-//     coalesced read) to count the non-zeros in front of this warp's quarter;
-//   - lane l keeps word l of its own quarter and an exclusive scan of the 32
-//     word popcounts;
-//   - the quarter is written with 16-byte stores: per store a lane owns kVec
-//     consecutive elements, i.e. kVec consecutive bits of one word; the rank
-//     of its first set bit is  chunk base + warp base + word offset +
-//     popc(lower bits of the word),  and the set bits gather from values[].
+//     coalesced read, issued together with the read of chunk_prefix[c]); the
+//     popcounts of the lanes in front of this warp's quarter give the count in
+//     front of it, and four shuffles hand lane l word l of its own quarter, so
+//     the only dependent round trip left is the gather itself;
+//   - a warp scan of the 32 word popcounts gives word offsets;
+//   - the quarter is written with 16-byte stores: a lane owns kE consecutive
+//     elements, i.e. kE consecutive bits of one word; the rank of its first set
+//     bit is  chunk base + quarter base + word offset + popc(lower bits of the
+//     word),  and the set bits gather from values[] at consecutive addresses.
 #include "bt_internal.cuh"
 
 namespace bt {
@@ -18,93 +20,104 @@ namespace {
 
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 
-template <typename U>
-struct Vec16;
-template <>
-struct Vec16<uint32_t> {
-    static constexpr int kVec = 4;
-};
-template <>
-struct Vec16<uint16_t> {
-    static constexpr int kVec = 8;
-};
-
-template <typename U, int kWarps>
+// kE: elements a lane decodes per step (a multiple of one 16-byte vector)
+template <typename U, int kE, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
 decompress_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values,
                   const uint64_t *__restrict__ prefix, const uint64_t n, U *__restrict__ out)
 {
-    constexpr int kVec          = Vec16<U>::kVec;          // elements per 16-byte store
-    constexpr int kLanesPerWord = 32 / kVec;               // lanes that share one bitmap word
-    constexpr int kWordsPerStep = 32 / kLanesPerWord;      // words one warp-wide store covers
+    constexpr int kVec          = 16 / sizeof(U);          // elements per 16-byte store
+    constexpr int kLanesPerWord = 32 / kE;                 // lanes that share one bitmap word
+    constexpr int kWordsPerStep = kE;                      // words one warp-wide step covers (32 * kE / 32)
     constexpr int kSteps        = 32 / kWordsPerStep;
+    static_assert(kE % kVec == 0 && 32 % kE == 0 && kE < 32, "a lane takes whole vectors of one word");
 
-    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t lane        = threadIdx.x & 31u;
     const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
-    const uint64_t quarters = (n + 1023) >> 10;
+    const uint64_t quarters    = (n + 1023) >> 10;
     if (warp_global >= quarters) return;
 
-    const uint64_t chunk = warp_global >> 2;
-    const uint32_t q     = static_cast<uint32_t>(warp_global & 3u);
+    const uint64_t chunk       = warp_global >> 2;
+    const uint32_t q           = static_cast<uint32_t>(warp_global & 3u);
     const uint64_t words_total = (n + 31) >> 5;
-    const uint64_t cw0 = chunk * 128;                      // first word of the chunk
+    const uint64_t w0          = chunk * 128 + 4 * lane;   // this lane's four words of the chunk
+
+    // the chunk's 128 words (zero past the end of the bitmap) and its prefix entry: independent loads
+    uint4 w4 = make_uint4(0, 0, 0, 0);
+    if (w0 + 3 < words_total) {
+        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
+    } else {
+        if (w0 < words_total) w4.x = bitmap[w0];
+        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
+        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
+    }
+    const uint64_t chunk_base = prefix[chunk];
 
     // non-zeros of the chunk in front of this quarter
-    uint32_t before = 0;
-    if (q != 0 && lane < 8 * q) {
-        const uint4 w4 = *reinterpret_cast<const uint4 *>(bitmap + cw0 + 4 * lane);   // whole quarters precede: in range
-        before = __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w);
-    }
+    uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(kFull, before, o);
 
-    const uint64_t wi   = cw0 + 32 * q + lane;
-    const uint32_t word = wi < words_total ? bitmap[wi] : 0u;
-    uint32_t       incl = __popc(word);
+    // lane l takes word l of its own quarter: component l & 3 of lane 8q + (l >> 2)
+    const int      src = 8 * q + (lane >> 2);
+    const uint32_t c0 = __shfl_sync(kFull, w4.x, src), c1 = __shfl_sync(kFull, w4.y, src);
+    const uint32_t c2 = __shfl_sync(kFull, w4.z, src), c3 = __shfl_sync(kFull, w4.w, src);
+    const uint32_t word = (lane & 2u) ? ((lane & 1u) ? c3 : c2) : ((lane & 1u) ? c1 : c0);
+
+    uint32_t incl = __popc(word);
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const uint32_t u = __shfl_up_sync(kFull, incl, o);
         if (lane >= static_cast<uint32_t>(o)) incl += u;
     }
     const uint32_t excl = incl - __popc(word);
-    const uint64_t base = prefix[chunk] + before;
+    const U *const vp   = values + (chunk_base + before);   // packed values of this quarter
 
-    const uint64_t e0      = warp_global << 10;            // first element of the quarter
-    const uint32_t sub     = lane % kLanesPerWord;         // which kVec-bit group of the word
-    const uint32_t shift   = sub * kVec;
+    const uint64_t e0    = warp_global << 10;               // first element of the quarter
+    const uint32_t shift = (lane % kLanesPerWord) * kE;     // which kE-bit group of the word
+    // all gathers of the quarter are issued before the first store, so that a lane has up to 32
+    // independent loads in flight
+    U e[kSteps][kE];
 #pragma unroll
     for (int k = 0; k < kSteps; ++k) {
-        const int      src_lane = k * kWordsPerStep + lane / kLanesPerWord;
-        const uint32_t w        = __shfl_sync(kFull, word, src_lane);
-        const uint32_t wex      = __shfl_sync(kFull, excl, src_lane);
-        const uint32_t bits     = (w >> shift) & ((1u << kVec) - 1u);
-        uint64_t       idx      = base + wex + __popc(w & ((1u << shift) - 1u));
-        U              e[kVec];
+        const int      from = k * kWordsPerStep + lane / kLanesPerWord;
+        const uint32_t w    = __shfl_sync(kFull, word, from);
+        const uint32_t wex  = __shfl_sync(kFull, excl, from);
+        const uint32_t bits = (w >> shift) & ((1u << kE) - 1u);
+        uint32_t       off  = wex + __popc(w & ((1u << shift) - 1u));
 #pragma unroll
-        for (int j = 0; j < kVec; ++j) {
+        for (int j = 0; j < kE; ++j) {
             const bool set = (bits >> j) & 1u;
-            e[j]           = set ? values[idx] : U(0);
-            idx += set;
+            e[k][j]        = set ? vp[off] : U(0);
+            off += set;
         }
-        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kVec) + lane * kVec;
-        if (eo + kVec <= n) {
-            uint4 pack;
-            if constexpr (kVec == 4) {
-                pack = make_uint4(e[0], e[1], e[2], e[3]);
-            } else {
-                pack = make_uint4(e[0] | (uint32_t(e[1]) << 16), e[2] | (uint32_t(e[3]) << 16),
-                                  e[4] | (uint32_t(e[5]) << 16), e[6] | (uint32_t(e[7]) << 16));
-            }
-            *reinterpret_cast<uint4 *>(out + eo) = pack;
-        } else {
+    }
 #pragma unroll
-            for (int j = 0; j < kVec; ++j)
-                if (eo + j < n) out[eo + j] = e[j];
+    for (int k = 0; k < kSteps; ++k) {
+        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+#pragma unroll
+        for (int v = 0; v < kE / kVec; ++v) {
+            const uint64_t at = eo + v * kVec;
+            const U       *ev = e[k] + v * kVec;
+            if (at + kVec <= n) {
+                uint4 pack;
+                if constexpr (kVec == 4) {
+                    pack = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+                } else {
+                    pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
+                                      ev[4] | (uint32_t(ev[5]) << 16), ev[6] | (uint32_t(ev[7]) << 16));
+                }
+                *reinterpret_cast<uint4 *>(out + at) = pack;
+            } else {
+#pragma unroll
+                for (int j = 0; j < kVec; ++j)
+                    if (at + j < n) out[at + j] = ev[j];
+            }
         }
     }
 }
 
-template <typename U>
+template <typename U, int kE>
 cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *prefix, uint64_t n, void *out,
                          cudaStream_t stream)
 {
@@ -112,7 +125,7 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint6
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-    decompress_kernel<U, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
+    decompress_kernel<U, kE, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
         bitmap, static_cast<const U *>(values), prefix, n, static_cast<U *>(out));
     return cudaGetLastError();
 }
@@ -122,8 +135,13 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint6
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *prefix, uint64_t n,
                               int elem_size, void *out, cudaStream_t stream)
 {
-    return elem_size == 4 ? launch_typed<uint32_t>(bitmap, values, prefix, n, out, stream)
-                          : launch_typed<uint16_t>(bitmap, values, prefix, n, out, stream);
+#ifdef BT_DECOMP_E32
+    constexpr int kE32 = BT_DECOMP_E32, kE16 = BT_DECOMP_E16;
+#else
+    constexpr int kE32 = 4, kE16 = 8;
+#endif
+    return elem_size == 4 ? launch_typed<uint32_t, kE32>(bitmap, values, prefix, n, out, stream)
+                          : launch_typed<uint16_t, kE16>(bitmap, values, prefix, n, out, stream);
 }
 
 }  // namespace bt
