@@ -129,7 +129,7 @@ __device__ __forceinline__ uint32_t lds_elem(uint32_t addr)
 {
     uint32_t v;
     if constexpr (sizeof(U) == 4) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    else asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(addr));   // zero-extended
+    else asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(addr));   // sign-extended (see ReluKeep)
     return v;
 }
 // store `v` at `addr` in the lanes where keep != 0 (a predicated store, never a branch)
@@ -157,7 +157,7 @@ __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v)
 //
 // The loads of a batch of 8 steps are issued before the stores of the batch before it: a store of
 // step k lands below element 32(k+1) and a later batch reads at or above it, so they never meet.
-template <typename U, int RELU_DT, bool WRITE_Y, int kSteps>
+template <typename U, int RELU_DT, bool WRITE_Y, bool kGuardY, int kSteps>
 __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, const uint32_t words_addr,
                                                     const uint32_t lane, const uint32_t lt, U *y,
                                                     const uint32_t yvalid)
@@ -182,7 +182,7 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, con
                 x = ReluKeep<RELU_DT>::keep(x) ? x : 0u;
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
-                    if (e < yvalid) y[e] = static_cast<U>(x);
+                    if (!kGuardY || e < yvalid) y[e] = static_cast<U>(x);
                 }
             }
             const uint32_t b = __ballot_sync(kFull, x != 0u);
@@ -501,8 +501,12 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
             y      = static_cast<U *>(a.y) + e0;
             yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
         }
-        const uint32_t run = compact_segment<U, RELU_DT, WRITE_Y, kSteps>(
-            smem_addr(tile + warp * kSeg), smem_addr(&s_words[warp][0]), lane, lt, y, yvalid);
+        const uint32_t seg_addr = smem_addr(tile + warp * kSeg), words_addr = smem_addr(&s_words[warp][0]);
+        uint32_t       run;
+        if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
+            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, words_addr, lane, lt, y, yvalid);
+        else
+            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, words_addr, lane, lt, y, yvalid);
         __syncwarp();
         if (lane < kSteps) {
             const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * kSteps + lane;

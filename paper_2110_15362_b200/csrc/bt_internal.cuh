@@ -148,18 +148,20 @@ struct ReluKeep<BT_F32> {
         return (static_cast<int32_t>(u) > 0) | (u > 0xFF800000u);
     }
 };
+// The 16-bit forms take the pattern SIGN-EXTENDED to 32 bits (as `ld.shared.s16` delivers it): positive
+// is then one signed compare, a negative NaN one unsigned compare against the sign-extended -inf.
 template <>
 struct ReluKeep<BT_F16> {
-    __device__ static __forceinline__ bool keep(uint32_t u)   // u holds a 16-bit pattern
+    __device__ static __forceinline__ bool keep(uint32_t u)
     {
-        return ((u - 1u) < 0x7FFFu) | (u > 0xFC00u);
+        return (static_cast<int32_t>(u) > 0) | (u > 0xFFFFFC00u);
     }
 };
 template <>
 struct ReluKeep<BT_BF16> {
     __device__ static __forceinline__ bool keep(uint32_t u)
     {
-        return ((u - 1u) < 0x7FFFu) | (u > 0xFF80u);
+        return (static_cast<int32_t>(u) > 0) | (u > 0xFFFFFF80u);
     }
 };
 
