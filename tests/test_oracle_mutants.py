@@ -1,0 +1,108 @@
+"""Shows that the pins are not vacuous: each plausible mistake is planted into a COPY of the oracle's C
+source (one text substitution), the copy is compiled, and at least one of the independent pins -- numpy
+library routines, closed forms, torch.relu / torch.where -- must notice.  The shipped oracle is untouched."""
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2110_15362_b200 import workloads as W
+
+SRC = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle", "bt_oracle.c")
+
+MUTANTS = {
+    "msb_first_bit_order": ("(uint32_t)1 << (i & 31);                     /* push 1 bit */",
+                            "(uint32_t)1 << (31 - (i & 31));"),
+    "inclusive_prefix": ("if (i % CHUNK_ELEMS == 0) prefix[i / CHUNK_ELEMS] = j;\n        const unsigned char *e = src + i * (uint64_t)elem_size;\n        if (all_bytes_zero(e, elem_size)) {",
+                         "if (i % CHUNK_ELEMS == CHUNK_ELEMS - 1) prefix[i / CHUNK_ELEMS] = j;\n        const unsigned char *e = src + i * (uint64_t)elem_size;\n        if (all_bytes_zero(e, elem_size)) {"),
+    "float_compare_drops_negative_zero": ("if (p[b] != 0) return 0;", "if (p[b] != 0 && !(b == elem_size - 1 && p[b] == 0x80)) return 0;"),
+    "decode_skips_counter": ("memcpy(e, val + j * (uint64_t)elem_size, (size_t)elem_size);\n            j += 1;\n        } else {\n            memset(e, 0, (size_t)elem_size);\n        }\n    }\n}\n\nvoid oracle_decompress_chunked",
+                             "memcpy(e, val + j * (uint64_t)elem_size, (size_t)elem_size);\n            j += (i % 97 != 0);\n        } else {\n            memset(e, 0, (size_t)elem_size);\n        }\n    }\n}\n\nvoid oracle_decompress_chunked"),
+    "relu_keeps_negatives": ("return f <= 0.0f; }\n    case ORACLE_F64", "return f == 0.0f; }\n    case ORACLE_F64"),
+    "bwd_multiplies_instead_of_selecting": ("memset(o + i * (uint64_t)elem_size, 0, (size_t)elem_size);\n    }\n}\n\n/* M_b",
+                                            "memmove(o + i * (uint64_t)elem_size, g + i * (uint64_t)elem_size, (size_t)elem_size);\n    }\n}\n\n/* M_b"),
+    "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
+    "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
+}
+
+
+def build_mutant(tmp_path, name):
+    old, new = MUTANTS[name]
+    text = open(SRC).read()
+    assert text.count(old) == 1, f"mutation site of {name} not found exactly once"
+    c = tmp_path / f"{name}.c"
+    c.write_text(text.replace(old, new))
+    so = tmp_path / f"{name}.so"
+    subprocess.check_call(["gcc", "-O1", "-std=c11", "-shared", "-fPIC", "-I", os.path.dirname(SRC), "-o", str(so), str(c)])
+    L = ctypes.CDLL(str(so))
+    u64, vp, i32 = ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int
+    L.oracle_compress.restype = u64
+    L.oracle_compress.argtypes = [vp, u64, i32, vp, vp, vp]
+    L.oracle_decompress.argtypes = [vp, vp, u64, i32, vp]
+    L.oracle_relu_fwd_compress.restype = u64
+    L.oracle_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp]
+    L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
+    L.oracle_compressed_bytes.restype = u64
+    L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
+    return L
+
+
+def p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def pins_hold(L) -> bool:
+    """A compact rerun of the independent pins against library `L`; False as soon as one fails."""
+    n = 2 * 4096 + 77
+    x = W.random_patterns(n, "f32", 0.5, seed=1)
+    x[5] = 0x80000000                                             # a negative zero must survive
+    nz = x != 0
+    bitmap = np.zeros((n + 31) // 32, np.uint32)
+    values = np.zeros(n, np.uint32)
+    prefix = np.zeros((n + 4095) // 4096, np.uint64)
+    nnz = L.oracle_compress(p(x), n, 4, p(bitmap), p(values), p(prefix))
+    packed = np.packbits(nz, bitorder="little")
+    ref_bitmap = np.concatenate([packed, np.zeros((-packed.size) % 4, np.uint8)]).view("<u4")
+    per_chunk = np.add.reduceat(nz.astype(np.uint64), np.arange(0, n, 4096))
+    ref_prefix = np.concatenate([[0], np.cumsum(per_chunk)[:-1]]).astype(np.uint64)
+    if nnz != int(nz.sum()) or not np.array_equal(bitmap, ref_bitmap) or not np.array_equal(values[:nnz], x[nz]) \
+            or not np.array_equal(prefix, ref_prefix):
+        return False
+    back = np.empty(n, np.uint32)
+    L.oracle_decompress(p(bitmap), p(values), n, 4, p(back))
+    if not np.array_equal(back, x):
+        return False
+    # ReLU pair against torch
+    t = torch.randn(n, generator=torch.Generator().manual_seed(3)) * 2
+    t[::53] = 0.0
+    xr = W.raw_numpy(t)
+    y = np.empty(n, np.uint32)
+    L.oracle_relu_fwd_compress(p(xr), n, 0, p(y), p(bitmap), p(values), p(prefix))
+    if not np.array_equal(y, W.raw_numpy(torch.relu(t) + 0.0)):
+        return False
+    g = torch.randn(n, generator=torch.Generator().manual_seed(4))
+    gin = np.empty(n, np.uint32)
+    L.oracle_relu_bwd_from_bitmap(p(bitmap), p(W.raw_numpy(g)), n, 4, p(gin))
+    if not np.array_equal(gin, W.raw_numpy(torch.where(t > 0, g, torch.zeros(())))):
+        return False
+    # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
+    if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
+        return False
+    mb = (L.oracle_compressed_bytes(2408448, 1204224, 4) - 8 * (2408448 // 4096)) / 2 ** 20
+    return abs(mb - 4.88) <= 0.005
+
+
+def test_the_unmutated_source_passes(tmp_path):
+    MUTANTS["identity"] = ("#define CHUNK_ELEMS 4096u", "#define CHUNK_ELEMS 4096u")
+    try:
+        assert pins_hold(build_mutant(tmp_path, "identity"))
+    finally:
+        del MUTANTS["identity"]
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_every_planted_mistake_is_caught(tmp_path, name):
+    assert not pins_hold(build_mutant(tmp_path, name)), f"the pins did not notice: {name}"
