@@ -44,6 +44,8 @@
 // The scan warp works on three tiles at a time (publish, read, finish), so the
 // compactors run about three tiles ahead of the copiers and nobody waits for a
 // round trip to L2.
+#include <cooperative_groups.h>
+
 #include <cstdlib>
 #include <mutex>
 #include <type_traits>
@@ -281,28 +283,45 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
     }
     __syncthreads();
 
+    // bulk copy of tile `it` of this CTA into its ring slot (issued by lane 0 of the load warp)
+    auto issue_load = [&](const uint32_t it) {
+        const uint32_t s     = it % kStages;
+        const uint64_t first = tile_of(it) * kTile;
+        const uint64_t left  = n - first;
+        const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
+        const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
+        fence_proxy_async();                       // the copiers' and compactors' accesses to the slot come first
+        mbar_arrive_expect_tx(&s_full[s], bytes);  // bytes == 0 simply completes the phase
+        if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
+    };
+
+    // The workspace arrives with unspecified contents.  Every CTA zeroes its share of it (abort flag, wave
+    // totals, tile descriptors) and the grid meets once before anyone publishes a count; the first ring of
+    // tiles is requested before that, so the copies travel while the grid meets.
+    if (warp == kLoadWarp && lane == 0) {
+        for (uint32_t it = 0; it < static_cast<uint32_t>(kStages) && tile_of(it) < num_tiles; ++it) issue_load(it);
+    }
+    {
+        uint64_t *const ws    = reinterpret_cast<uint64_t *>(a.ws_header);
+        const uint64_t  words = kWsHeaderBytes / 8 + a.ws_waves + num_tiles;
+        for (uint64_t i = static_cast<uint64_t>(cta) * blockDim.x + tid; i < words; i += static_cast<uint64_t>(G) * blockDim.x)
+            ws[i] = 0;
+    }
+    cooperative_groups::this_grid().sync();
+
     if (warp == kLoadWarp) {
         // ------------------------------------------------------------ load warp (one lane)
         if (lane == 0) {
             bool ok = true;
-            for (uint32_t it = 0; ok; ++it) {
-                const uint64_t t64 = tile_of(it);
-                if (t64 >= num_tiles) break;
+            for (uint32_t it = kStages; ok; ++it) {
+                if (tile_of(it) >= num_tiles) break;
                 const uint32_t s = it % kStages;
-                if (it >= static_cast<uint32_t>(kStages)) {
-                    PROF_T(c0);
-                    ok = mbar_wait(&s_empty[s], ((it / kStages) - 1) & 1u, &s_abort);
-                    PROF_T(c1);
-                    PROF_ADD(4, c1 - c0);
-                    if (!ok) break;
-                }
-                const uint64_t first = t64 * kTile;
-                const uint64_t left  = n - first;
-                const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
-                const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
-                fence_proxy_async();                       // the copiers' and compactors' accesses to the slot come first
-                mbar_arrive_expect_tx(&s_full[s], bytes);  // bytes == 0 simply completes the phase
-                if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
+                PROF_T(c0);
+                ok = mbar_wait(&s_empty[s], ((it / kStages) - 1) & 1u, &s_abort);
+                PROF_T(c1);
+                PROF_ADD(4, c1 - c0);
+                if (!ok) break;
+                issue_load(it);
             }
             if (!ok) {
                 // a bounded wait ran out somewhere in this CTA: before leaving, let the bulk copies that
@@ -569,9 +588,6 @@ cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
     if (max_grid > 32 * kMaxWindows) max_grid = 32 * kMaxWindows;
     const uint32_t grid  = num_tiles < static_cast<uint32_t>(max_grid) ? num_tiles : static_cast<uint32_t>(max_grid);
     const uint32_t waves = (num_tiles + grid - 1) / grid;
-    // abort flag, wave totals and tile descriptors start at zero
-    e = cudaMemsetAsync(a.ws_header, 0, kWsHeaderBytes + 8 * (static_cast<size_t>(num_tiles) + waves), stream);
-    if (e != cudaSuccess) return e;
     // cooperative launch: the runtime guarantees that all `grid` CTAs are resident together
     CompressArgs args = a;
     args.ws_waves     = waves;
