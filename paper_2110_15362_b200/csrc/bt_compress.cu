@@ -295,32 +295,19 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
         if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
     };
 
-    // The workspace arrives with unspecified contents.  Every CTA zeroes its share of it (abort flag, wave
-    // totals, tile descriptors) and the grid meets once before anyone publishes a count; the first ring of
-    // tiles is requested before that, so the copies travel while the grid meets.
-    if (warp == kLoadWarp && lane == 0) {
-        for (uint32_t it = 0; it < static_cast<uint32_t>(kStages) && tile_of(it) < num_tiles; ++it) issue_load(it);
-    }
-    {
-        uint64_t *const ws    = reinterpret_cast<uint64_t *>(a.ws_header);
-        const uint64_t  words = kWsHeaderBytes / 8 + a.ws_waves + num_tiles;
-        for (uint64_t i = static_cast<uint64_t>(cta) * blockDim.x + tid; i < words; i += static_cast<uint64_t>(G) * blockDim.x)
-            ws[i] = 0;
-    }
-    cooperative_groups::this_grid().sync();
-
     if (warp == kLoadWarp) {
         // ------------------------------------------------------------ load warp (one lane)
         if (lane == 0) {
             bool ok = true;
-            for (uint32_t it = kStages; ok; ++it) {
+            for (uint32_t it = 0; ok; ++it) {
                 if (tile_of(it) >= num_tiles) break;
-                const uint32_t s = it % kStages;
-                PROF_T(c0);
-                ok = mbar_wait(&s_empty[s], ((it / kStages) - 1) & 1u, &s_abort);
-                PROF_T(c1);
-                PROF_ADD(4, c1 - c0);
-                if (!ok) break;
+                if (it >= static_cast<uint32_t>(kStages)) {
+                    PROF_T(c0);
+                    ok = mbar_wait(&s_empty[it % kStages], ((it / kStages) - 1) & 1u, &s_abort);
+                    PROF_T(c1);
+                    PROF_ADD(4, c1 - c0);
+                    if (!ok) break;
+                }
                 issue_load(it);
             }
             if (!ok) {
@@ -344,6 +331,26 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
         const uint32_t *const abort_flag   = a.ws_header + 1;
         uint64_t              waves_before = 0;    // sum of the totals of the waves before the tile being finished
         bool                  failed       = false;
+
+        // The workspace arrives with unspecified contents.  The scan warps zero it between them (abort flag,
+        // wave totals, tile descriptors) and meet once, at the grid barrier word the runtime gives every
+        // cooperative launch, before any of them publishes a count.  Only they touch the workspace, so the
+        // other warps start on the data at once and the meeting hides behind the first tile.
+        // The word follows the usual sense-reversing count: CTA 0 adds 2^31 - (G - 1), every other CTA adds 1,
+        // so bit 31 flips exactly when all G have arrived and the low bits are back where they started.
+        unsigned int *const grid_bar = &cooperative_groups::details::get_grid_workspace()->barrier;
+        uint32_t            bar_old  = 0;
+        bool                grid_met = false;
+        {
+            uint64_t *const ws    = reinterpret_cast<uint64_t *>(a.ws_header);
+            const uint64_t  words = kWsHeaderBytes / 8 + a.ws_waves + num_tiles;
+            for (uint64_t i = static_cast<uint64_t>(cta) * 32 + lane; i < words; i += static_cast<uint64_t>(G) * 32) ws[i] = 0;
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t add = cta == 0 ? 0x80000000u - (G - 1) : 1u;
+                asm volatile("atom.add.release.gpu.u32 %0, [%1], %2;" : "=r"(bar_old) : "l"(grid_bar), "r"(add) : "memory");
+            }
+        }
 
         // Three tiles are in the scan pipeline at any time.  In iteration `it` the warp
         //   (a) takes the counts of tile `it` and publishes them,
@@ -377,6 +384,27 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
                     if (lane >= static_cast<uint32_t>(o)) inc += u;
                 }
                 const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
+                if (!grid_met) {
+                    // first publication: every scan warp must have finished zeroing
+                    bool met = true;
+                    if (lane == 0) {
+                        const uint64_t t0 = now_ns();
+                        for (;;) {
+                            uint32_t cur;
+                            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(grid_bar) : "memory");
+                            if ((cur ^ bar_old) & 0x80000000u) break;
+                            if (now_ns() - t0 > kWaitNs) {
+                                met = false;
+                                break;
+                            }
+                        }
+                    }
+                    if (!__shfl_sync(kFull, met, 0)) {
+                        failed = true;
+                        return false;
+                    }
+                    grid_met = true;
+                }
                 if (lane == 0) {
                     st_relaxed_u64(desc + tile_of(it), (static_cast<uint64_t>(agg) << 1) | 1ull);
                     red_add_u64(wave_total + it, (1ull << kCountShift) + agg);
