@@ -189,28 +189,29 @@ class Cfg2Step:
         self.dense_bytes_per_step = len(OPS) * 4 * self.total_elems
         self.launches_per_step = len(OPS) * len(self.layers)
 
-    def run(self, rec=None):
-        """One step.  `rec(op, layer_index)` brackets a call with CUDA events when given."""
+    def run(self, only_op=None, only_layer=None):
+        """One step (forward over the layers, backward in reverse).  `only_op` / `only_layer` restrict it to
+        one operation and / or one layer, for the per-operation timing passes."""
         B = self.B
+
+        def want(op, i):
+            return (only_op is None or op == only_op) and (only_layer is None or i == only_layer)
+
         for i, l in enumerate(self.layers):
             a, b = l["stash_a"], l["stash_b"]
-            if rec: rec("bt_compress", i, True)
-            B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.ws, a.dev_status)
-            if rec: rec("bt_compress", i, False)
-            if rec: rec("bt_relu_fwd_compress", i, True)
-            B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.ws,
-                                   b.dev_status)
-            if rec: rec("bt_relu_fwd_compress", i, False)
+            if want("bt_compress", i):
+                B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.ws, a.dev_status)
+            if want("bt_relu_fwd_compress", i):
+                B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.ws,
+                                       b.dev_status)
         for i in range(len(self.layers) - 1, -1, -1):
             l = self.layers[i]
             a, b = l["stash_a"], l["stash_b"]
             n = l["n"]
-            if rec: rec("bt_decompress", i, True)
-            B.bt_decompress(a.bitmap, a.values, a.chunk_prefix, self.restored[:n])
-            if rec: rec("bt_decompress", i, False)
-            if rec: rec("bt_relu_bwd_from_bitmap", i, True)
-            B.bt_relu_bwd_from_bitmap(b.bitmap, l["grad"], self.gin[:n])
-            if rec: rec("bt_relu_bwd_from_bitmap", i, False)
+            if want("bt_decompress", i):
+                B.bt_decompress(a.bitmap, a.values, a.chunk_prefix, self.restored[:n])
+            if want("bt_relu_bwd_from_bitmap", i):
+                B.bt_relu_bwd_from_bitmap(b.bitmap, l["grad"], self.gin[:n])
 
     def check(self):
         """After a step: device status words are clean and both stashes of a layer agree."""
@@ -228,30 +229,48 @@ class Cfg2Step:
 
 
 def per_kernel_pass(step: Cfg2Step, steps: int):
-    """Same steps, eager launches, CUDA events on the launching stream around every call."""
+    """Device time of each operation: the step's launches of ONE operation (all 17 layers, in the step's
+    order) captured as a CUDA graph of their own and replayed `steps` times between two CUDA events on the
+    launching stream, so the figure holds what the whole-step graph holds for that operation (kernel time
+    and the device's launch latency between dependent kernels) and no host overhead.  The inputs of one
+    such pass (0.3 GB and more) exceed the L2.  The largest layer is timed the same way on its own,
+    with the L2 flushed before every replay."""
     import torch
-    stream = torch.cuda.current_stream()
-    pending = {}
-    records = []
-
-    def rec(op, i, begin):
-        ev = torch.cuda.Event(enable_timing=True)
-        ev.record(stream)
-        if begin:
-            pending[(op, i)] = ev
-        else:
-            records.append((op, i, pending.pop((op, i)), ev))
-
-    for _ in range(steps):
-        step.run(rec)
-    torch.cuda.synchronize()
-    per_op = {op: {"ms": 0.0, "launches": 0} for op in OPS}
-    per_layer = {}
-    for op, i, e0, e1 in records:
-        ms = e0.elapsed_time(e1)
-        per_op[op]["ms"] += ms
-        per_op[op]["launches"] += 1
-        per_layer.setdefault((op, i), []).append(ms)
+    dev = step.restored.device
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    per_op, per_layer = {}, {}
+    side = torch.cuda.Stream()
+    for op in OPS:
+        graphs = []
+        for only in (None, 0):
+            g = torch.cuda.CUDAGraph()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step.run(only_op=op, only_layer=only)          # warm-up outside the capture
+            torch.cuda.current_stream().wait_stream(side)
+            with torch.cuda.graph(g):
+                step.run(only_op=op, only_layer=only)
+            graphs.append(g)
+        whole, big = graphs
+        for _ in range(3):
+            whole.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            whole.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        per_op[op] = {"ms": e0.elapsed_time(e1), "launches": steps * len(step.layers)}
+        times = []
+        for _ in range(max(5, min(steps, 20))):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            big.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        per_layer[(op, 0)] = times
     return per_op, per_layer
 
 
@@ -428,7 +447,7 @@ def run_ours(args):
     step.check()
     clocks = sampler.summary(t0, t1)
 
-    # per-kernel durations: the same steps launched eagerly with events around every call
+    # per-operation device time: one CUDA graph per operation, replayed between two events
     per_op, per_layer = per_kernel_pass(step, min(args.steps, 20))
 
     # end to end: inputs start in pinned host memory, results end in host memory, every step
