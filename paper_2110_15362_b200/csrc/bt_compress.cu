@@ -220,8 +220,8 @@ __device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, cons
 // U: uint32_t (4-byte elements) or uint16_t (2-byte elements).
 // RELU_DT: -1 for the plain compressor, else the element type whose ReLU is fused in.
 // kWarps compactor warps and as many copier warps, kSeg elements per warp, kStages ring slots.
-template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages>
-__global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
+template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages, int kCopiers>
+__global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
 {
     constexpr int kTile          = kWarps * kSeg;
     constexpr int kSteps         = kSeg / 32;
@@ -230,8 +230,10 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
     constexpr int kCompactThreads = kWarps * 32;
     // warp roles
     constexpr int kFirstCopier = kWarps;
-    constexpr int kScanWarp    = 2 * kWarps;
-    constexpr int kLoadWarp    = 2 * kWarps + 1;
+    constexpr int kScanWarp    = kWarps + kCopiers;       // and kScanWarp + 1
+    constexpr int kLoadWarp    = kWarps + kCopiers + 2;
+    constexpr int kSegsPerCopier = kWarps / kCopiers;
+    static_assert(kWarps % kCopiers == 0, "equal shares for the copier warps");
     static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
     static_assert(kTile % BT_CHUNK_ELEMS == 0, "a tile holds whole chunks");
     static_assert(kWarps <= 32, "one lane per warp count");
@@ -244,6 +246,7 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
     __shared__ __align__(8) uint64_t s_counted[kStages];   // every compactor posted its count    (compactors -> scan warp)
     __shared__ __align__(8) uint64_t s_ready[kStages];     // base and offsets are in shared      (scan warp -> copiers)
     __shared__ __align__(8) uint64_t s_empty[kStages];     // every copier is done with the slot  (copiers -> load warp)
+    __shared__ __align__(8) uint64_t s_go;                 // the grid has met                    (scan warp 0 -> scan warp 1)
     __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
     __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
     __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
@@ -277,8 +280,9 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
             mbar_init(&s_full[s], 1);
             mbar_init(&s_counted[s], kWarps);
             mbar_init(&s_ready[s], 1);
-            mbar_init(&s_empty[s], kWarps);
+            mbar_init(&s_empty[s], kCopiers);
         }
+        mbar_init(&s_go, 1);
         fence_proxy_async();
     }
     __syncthreads();
@@ -323,56 +327,77 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
         return;
     }
 
-    if (warp == kScanWarp) {
-        // ------------------------------------------------------------ scan warp
+    if (warp == kScanWarp || warp == kScanWarp + 1) {
+        // ------------------------------------------------------------ scan warps
+        // Two warps share the scan: warp p takes this CTA's tiles p, p + 2, p + 4, ...  A warp's turn for
+        // tile j is
+        //   (a) wait until the compactors have counted tile j, publish the count,
+        //   (c) finish tile j - 2 (its own previous tile) from the loads of its previous turn and hand it
+        //       to the copiers,
+        //   (b) wait until tile j + 1 is counted -- about one tile later, when every CTA has published
+        //       wave j -- and issue, in ONE batch of independent loads, the reads of the descriptors of
+        //       wave j and of the totals of waves j - 1 and j - 2.
+        // The loads of (b) are used a whole tile later, in (c) of the next turn, so the round trip to L2
+        // (1.3 us under load, longer than one tile) never stalls a turn for long: a turn has two tiles' time.
+        // (One warp doing every tile cannot hide that round trip however deep its software pipeline is:
+        // its loads of consecutive tiles retire through the same scoreboard.)
+        const uint32_t        p            = warp - kScanWarp;
         uint64_t *const       wave_total   = a.ws_desc;                  // one word per wave
         uint64_t *const       desc         = a.ws_desc + a.ws_waves;     // one word per tile: (count << 1) | 1
         const uint64_t        chunks_total = (n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
         const uint32_t *const abort_flag   = a.ws_header + 1;
-        uint64_t              waves_before = 0;    // sum of the totals of the waves before the tile being finished
+        const uint32_t        last_it      = static_cast<uint32_t>((num_tiles - 1 - cta) / G);   // this CTA's last iteration
+        uint64_t              waves_before = 0;    // sum of the totals of the waves before this warp's previous tile
         bool                  failed       = false;
 
-        // The workspace arrives with unspecified contents.  The scan warps zero it between them (abort flag,
-        // wave totals, tile descriptors) and meet once, at the grid barrier word the runtime gives every
-        // cooperative launch, before any of them publishes a count.  Only they touch the workspace, so the
-        // other warps start on the data at once and the meeting hides behind the first tile.
-        // The word follows the usual sense-reversing count: CTA 0 adds 2^31 - (G - 1), every other CTA adds 1,
-        // so bit 31 flips exactly when all G have arrived and the low bits are back where they started.
-        unsigned int *const grid_bar = &cooperative_groups::details::get_grid_workspace()->barrier;
-        uint32_t            bar_old  = 0;
-        bool                grid_met = false;
-        {
-            uint64_t *const ws    = reinterpret_cast<uint64_t *>(a.ws_header);
-            const uint64_t  words = kWsHeaderBytes / 8 + a.ws_waves + num_tiles;
+        if (p == 0) {
+            // The workspace arrives with unspecified contents.  The first scan warps of the grid zero it between
+            // them (abort flag, wave totals, tile descriptors) and meet once, at the grid barrier word the runtime
+            // gives every cooperative launch, before any count is published.  Only the scan warps touch the
+            // workspace, so the other warps start on the data at once and the meeting hides behind the first tile.
+            // The word follows the usual sense-reversing count: CTA 0 adds 2^31 - (G - 1), every other CTA adds 1,
+            // so bit 31 flips exactly when all G have arrived and the low bits are back where they started.
+            unsigned int *const grid_bar = &cooperative_groups::details::get_grid_workspace()->barrier;
+            uint64_t *const     ws       = reinterpret_cast<uint64_t *>(a.ws_header);
+            const uint64_t      words    = kWsHeaderBytes / 8 + a.ws_waves + num_tiles;
             for (uint64_t i = static_cast<uint64_t>(cta) * 32 + lane; i < words; i += static_cast<uint64_t>(G) * 32) ws[i] = 0;
             __syncwarp();
+            bool met = true;
             if (lane == 0) {
+                uint32_t       bar_old;
                 const uint32_t add = cta == 0 ? 0x80000000u - (G - 1) : 1u;
                 asm volatile("atom.add.release.gpu.u32 %0, [%1], %2;" : "=r"(bar_old) : "l"(grid_bar), "r"(add) : "memory");
+                const uint64_t t0 = now_ns();
+                for (;;) {
+                    uint32_t cur;
+                    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(grid_bar) : "memory");
+                    if ((cur ^ bar_old) & 0x80000000u) break;
+                    if (now_ns() - t0 > kWaitNs) {
+                        met = false;
+                        break;
+                    }
+                }
+                if (met) mbar_arrive(&s_go);                          // the other scan warp may publish too
             }
+            failed = !__shfl_sync(kFull, met, 0);
+        } else {
+            failed = !mbar_wait(&s_go, 0, &s_abort);
         }
 
-        // Three tiles are in the scan pipeline at any time.  In iteration `it` the warp
-        //   (a) takes the counts of tile `it` and publishes them,
-        //   (b) issues the loads for tile `it - 1`, whose wave every CTA published about an iteration ago,
-        //   (c) finishes tile `it - 2` from the loads issued an iteration ago and hands it to the copiers.
-        // d[slot][k], lane l <-> descriptor of CTA l + 32k of the tile's wave; w[slot]: total word of the
-        // wave before it.  Tile j uses slot j & 1.
-        uint64_t d[2][kMaxWindows], w[2] = {0, 0};
+        // d[k], lane l <-> descriptor of CTA l + 32k of the wave of this warp's previous tile;
+        // w1, w2: total words of the one and the two waves before it
+        uint64_t d[kMaxWindows], w1 = 0, w2 = 0;
 #pragma unroll
-        for (int k = 0; k < kMaxWindows; ++k) d[0][k] = d[1][k] = 1ull;
-        const uint32_t last_it = static_cast<uint32_t>((num_tiles - 1 - cta) / G);   // this CTA's last iteration
+        for (int k = 0; k < kMaxWindows; ++k) d[k] = 1ull;
 
-        auto step = [&](auto parity, const uint32_t it) -> bool {
-            // parity == it & 1; tile it - 1 loads into slot kLoad, tile it - 2 is finished from slot kDone
-            constexpr int kLoad = 1 - decltype(parity)::value, kDone = decltype(parity)::value;
-            if (it <= last_it) {
+        for (uint32_t j = p; !failed && j <= last_it + 2; j += 2) {
+            if (j <= last_it) {
                 // ---- (a)
-                const uint32_t s = it % kStages;
+                const uint32_t s = j % kStages;
                 PROF_T(c0);
-                if (!mbar_wait(&s_counted[s], (it / kStages) & 1u, &s_abort)) {
+                if (!mbar_wait(&s_counted[s], (j / kStages) & 1u, &s_abort)) {
                     failed = true;
-                    return false;
+                    break;
                 }
                 PROF_T(c1);
                 PROF_ADD(8, c1 - c0);
@@ -384,43 +409,22 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
                     if (lane >= static_cast<uint32_t>(o)) inc += u;
                 }
                 const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
-                if (!grid_met) {
-                    // first publication: every scan warp must have finished zeroing
-                    bool met = true;
-                    if (lane == 0) {
-                        const uint64_t t0 = now_ns();
-                        for (;;) {
-                            uint32_t cur;
-                            asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(grid_bar) : "memory");
-                            if ((cur ^ bar_old) & 0x80000000u) break;
-                            if (now_ns() - t0 > kWaitNs) {
-                                met = false;
-                                break;
-                            }
-                        }
-                    }
-                    if (!__shfl_sync(kFull, met, 0)) {
-                        failed = true;
-                        return false;
-                    }
-                    grid_met = true;
-                }
                 if (lane == 0) {
-                    st_relaxed_u64(desc + tile_of(it), (static_cast<uint64_t>(agg) << 1) | 1ull);
-                    red_add_u64(wave_total + it, (1ull << kCountShift) + agg);
+                    st_relaxed_u64(desc + tile_of(j), (static_cast<uint64_t>(agg) << 1) | 1ull);
+                    red_add_u64(wave_total + j, (1ull << kCountShift) + agg);
                     s_agg[s] = agg;
                 }
                 if (lane < kWarps) s_off[s][lane] = inc - c;
             }
-            if (it >= 2 && it - 2 <= last_it) {
-                // ---- (c) first, so that its registers are free for (b)
-                const uint32_t j     = it - 2;
+            if (j >= 2) {
+                // ---- (c): tile j - 2 <= last_it
+                const uint32_t f     = j - 2;
                 uint32_t       polls = 0;
                 uint64_t       t0    = 0;
                 for (;;) {
-                    bool missing = j > 0 && (w[kDone] >> kCountShift) != G;
+                    bool missing = (f > 0 && (w1 >> kCountShift) != G) || (f > 1 && (w2 >> kCountShift) != G);
 #pragma unroll
-                    for (int k = 0; k < kMaxWindows; ++k) missing |= (d[kDone][k] & 1ull) == 0;
+                    for (int k = 0; k < kMaxWindows; ++k) missing |= (d[k] & 1ull) == 0;
                     if (!__any_sync(kFull, missing)) break;
                     PROF_ADD(11, 1);
                     __nanosleep(100);
@@ -433,18 +437,19 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
                     }
 #pragma unroll
                     for (int k = 0; k < kMaxWindows; ++k)
-                        if ((d[kDone][k] & 1ull) == 0)
-                            d[kDone][k] = ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + lane + 32u * k);
-                    if (j > 0 && (w[kDone] >> kCountShift) != G) w[kDone] = ld_relaxed_u64(wave_total + (j - 1));
+                        if ((d[k] & 1ull) == 0) d[k] = ld_relaxed_u64(desc + static_cast<uint64_t>(f) * G + lane + 32u * k);
+                    if (f > 0 && (w1 >> kCountShift) != G) w1 = ld_relaxed_u64(wave_total + (f - 1));
+                    if (f > 1 && (w2 >> kCountShift) != G) w2 = ld_relaxed_u64(wave_total + (f - 2));
                 }
-                if (failed) return false;
+                if (failed) break;
                 uint64_t part = 0;
 #pragma unroll
-                for (int k = 0; k < kMaxWindows; ++k) part += d[kDone][k] >> 1;
-                if (j > 0) waves_before += w[kDone] & ((1ull << kCountShift) - 1);
+                for (int k = 0; k < kMaxWindows; ++k) part += d[k] >> 1;
+                // the waves in front of tile f: those in front of tile f - 2, and waves f - 2 and f - 1
+                waves_before += (w1 & ((1ull << kCountShift) - 1)) + (w2 & ((1ull << kCountShift) - 1));
                 const uint64_t base = waves_before + warp_sum_u64(part);
-                const uint32_t ps   = j % kStages;
-                const uint64_t pt   = tile_of(j);
+                const uint32_t ps   = f % kStages;
+                const uint64_t pt   = tile_of(f);
                 // exclusive count in front of each chunk of that tile
                 if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
                     const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
@@ -464,31 +469,29 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
                     mbar_arrive(&s_ready[ps]);                       // the copiers may take the tile
                 }
             }
-            if (it >= 1 && it - 1 <= last_it) {
-                // ---- (b) one batch of independent loads
-                const uint32_t j = it - 1;
+            if (j <= last_it) {
+                // ---- (b): a tile later (when the other scan warp's next tile is counted, if there is one)
+                if (j + 1 <= last_it && !mbar_wait(&s_counted[(j + 1) % kStages], ((j + 1) / kStages) & 1u, &s_abort)) {
+                    failed = true;
+                    break;
+                }
 #pragma unroll
                 for (int k = 0; k < kMaxWindows; ++k) {
                     const uint32_t b = lane + 32u * k;
-                    d[kLoad][k] = (b < cta) ? ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + b) : 1ull;
+                    d[k] = (b < cta) ? ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + b) : 1ull;
                 }
-                w[kLoad] = (j > 0) ? ld_relaxed_u64(wave_total + (j - 1)) : 0ull;
+                w1 = (j > 0) ? ld_relaxed_u64(wave_total + (j - 1)) : 0ull;
+                w2 = (j > 1) ? ld_relaxed_u64(wave_total + (j - 2)) : 0ull;
             }
-            return it < last_it + 2;
-        };
-
-        for (uint32_t it = 0;; it += 2) {
-            if (!step(std::integral_constant<int, 0>{}, it)) break;
-            if (!step(std::integral_constant<int, 1>{}, it + 1)) break;
         }
         if (failed && lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort);
-        PROF_FLUSH(8, 13);
+        if (p == 0) { PROF_FLUSH(8, 13); }
         return;
     }
 
     if (warp >= kFirstCopier) {
         // ------------------------------------------------------------ copier warps
-        const uint32_t seg      = warp - kFirstCopier;
+        const uint32_t copier   = warp - kFirstCopier;
         U *const       vals     = static_cast<U *>(a.values);
         const uint64_t capacity = a.capacity;
         for (uint32_t it = 0;; ++it) {
@@ -497,13 +500,18 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
             PROF_T(c0);
             if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort)) break;
             PROF_T(c1);
-            const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
-            const uint32_t cnt  = s_cnt[s][seg];
-            const uint64_t dst  = s_base[s] + s_off[s][seg];
-            if (dst + cnt <= capacity)
-                copy_out_segment<U, false>(pseg, lane, cnt, vals + dst, 0);
-            else
-                copy_out_segment<U, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
+            const uint64_t base = s_base[s];
+#pragma unroll
+            for (int q = 0; q < kSegsPerCopier; ++q) {
+                const uint32_t seg  = copier * kSegsPerCopier + q;
+                const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
+                const uint32_t cnt  = s_cnt[s][seg];
+                const uint64_t dst  = base + s_off[s][seg];
+                if (dst + cnt <= capacity)
+                    copy_out_segment<U, false>(pseg, lane, cnt, vals + dst, 0);
+                else
+                    copy_out_segment<U, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
+            }
             __syncwarp();
             asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
             if (lane == 0) mbar_arrive(&s_empty[s]);
@@ -511,7 +519,7 @@ __global__ void __launch_bounds__(kWarps * 64 + 64) compress_kernel(const Compre
             PROF_ADD(2, c1 - c0);
             PROF_ADD(3, c2 - c1);
         }
-        if (seg == 0) { PROF_FLUSH(2, 4); }
+        if (copier == 0) { PROF_FLUSH(2, 4); }
         return;
     }
 
@@ -600,14 +608,14 @@ struct LaunchShape {
     }
 };
 
-template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages>
+template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages, int kCopiers>
 cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
 {
     constexpr int kTile    = kWarps * kSeg;
-    constexpr int kThreads = kWarps * 64 + 64;
+    constexpr int kThreads = (kWarps + kCopiers + 3) * 32;
     constexpr size_t kSmem = static_cast<size_t>(kStages) * kTile * sizeof(U);
     static LaunchShape shape;   // one per instantiation
-    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, kWarps, kSeg, kStages>;
+    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, kWarps, kSeg, kStages, kCopiers>;
 
     const uint32_t num_tiles = static_cast<uint32_t>((a.n + kTile - 1) / kTile);
     int            max_grid  = 0;
@@ -628,15 +636,24 @@ cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
 template <typename U, int RELU_DT, bool WRITE_Y>
 cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
 {
-    // 8 compactor + 8 copier warps, 8192-element tiles, a ring of 192 KB: one CTA per SM
-    constexpr int kStages = sizeof(U) == 4 ? 6 : 12;
+    // One CTA per SM, the ring takes nearly all of its shared memory.
+    //   4-byte elements: 8 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 7 stages;
+    //   2-byte elements: 16 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 6 stages --
+    //   a 2-byte tile takes as many compaction steps per byte again, so it gets twice the warps.
 #ifdef BT_PROFILE
     static const int cfg = [] { const char *e = getenv("BT_CFG"); return e ? atoi(e) : 0; }();
-    if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, kStages + 1>(a, stream);
-    if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, kStages - 1>(a, stream);
-    if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 512, kStages>(a, stream);
+    if constexpr (sizeof(U) == 4) {
+        if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 6, 8>(a, stream);
+        if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 4>(a, stream);
+        if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 512, 7, 8>(a, stream);
+    } else {
+        if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 12, 8>(a, stream);
+        if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 12, 1024, 8, 6>(a, stream);
+        if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 1024, 6, 16>(a, stream);
+    }
 #endif
-    return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, kStages>(a, stream);
+    if constexpr (sizeof(U) == 4) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 8>(a, stream);
+    else return launch_shaped<U, RELU_DT, WRITE_Y, 16, 1024, 6, 8>(a, stream);
 }
 
 }  // namespace
