@@ -145,30 +145,29 @@ __device__ __forceinline__ void sts_elem_if(uint32_t addr, uint32_t v, uint32_t 
         asm volatile("{\n\t.reg .pred q;\n\t.reg .b16 h;\n\tsetp.ne.u32 q, %2, 0;\n\tcvt.u16.u32 h, %1;\n\t@q st.shared.u16 [%0], h;\n\t}" ::"r"(addr),
                      "r"(v), "r"(keep));
 }
-__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v)
-{
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v));
-}
 
 // ---------------------------------------------------------------------------------------------
 // One warp compacts its segment of kSteps * 32 elements in place.  Returns the number of packed
-// values.  The ballot of step k goes to the shared word at words_addr + 4k (every lane stores the
-// same value to the same address: one wavefront, no predicate).  `y` (fused form with dense
-// output) points at the segment's first element of the dense ReLU output, `yvalid` is how many of
-// them exist.  seg_addr / words_addr are shared-window addresses.
+// values; lane k leaves with the ballot of step k, which is bitmap word k of the segment, in `word`
+// (kept in registers through a tree of selects: a store to shared memory per step costs more).
+// `y` (fused form with dense output) points at the segment's first element of the dense ReLU
+// output, `yvalid` is how many of them exist.  seg_addr is a shared-window address.
 //
 // The loads of a batch of 8 steps are issued before the stores of the batch before it: a store of
 // step k lands below element 32(k+1) and a later batch reads at or above it, so they never meet.
 template <typename U, int RELU_DT, bool WRITE_Y, bool kGuardY, int kSteps>
-__device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, const uint32_t words_addr,
-                                                    const uint32_t lane, const uint32_t lt, U *y,
-                                                    const uint32_t yvalid)
+__device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uint32_t &word, const uint32_t lane,
+                                                    const uint32_t lt, U *y, const uint32_t yvalid)
 {
-    constexpr int      kBatch = kSteps < 8 ? kSteps : 8;
+    constexpr int      kBatch = 8;
+    static_assert(kSteps % kBatch == 0 && kSteps <= 32, "whole batches; one bitmap word per lane");
     constexpr uint32_t kES    = sizeof(U);
     const uint32_t     in0    = seg_addr + lane * kES;
     uint32_t           out    = seg_addr;               // address of the next free packed slot
     uint32_t           v[kBatch], vn[kBatch];
+    uint32_t   bb[kBatch];
+    const bool l0 = lane & 1u, l1 = lane & 2u, l2 = lane & 4u;
+    word = 0;
 #pragma unroll
     for (int j = 0; j < kBatch; ++j) v[j] = lds_elem<U>(in0 + j * 32 * kES);
 #pragma unroll
@@ -188,9 +187,21 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, con
                 }
             }
             const uint32_t b = __ballot_sync(kFull, x != 0u);
-            sts_u32(words_addr + 4 * (kb + j), b);
-            sts_elem_if<U>(out + kES * __popc(b & lt), x, x);
+            bb[j] = b;
+            if (x != 0u) {
+                const uint32_t at = out + kES * __popc(b & lt);
+                if constexpr (kES == 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"(x));
+                else asm volatile("st.shared.u16 [%0], %1;" ::"r"(at), "h"(static_cast<uint16_t>(x)));
+            }
             out += kES * __popc(b);
+        }
+        {
+            // lane kb + j keeps ballot j of this batch: a binary tree of selects over the low lane bits
+            static_assert(kBatch == 8, "the select tree is written for batches of 8 ballots");
+            const uint32_t t0 = l0 ? bb[1] : bb[0], t1 = l0 ? bb[3] : bb[2], t2 = l0 ? bb[5] : bb[4], t3 = l0 ? bb[7] : bb[6];
+            const uint32_t u0 = l1 ? t1 : t0, u1 = l1 ? t3 : t2;
+            const uint32_t w  = l2 ? u1 : u0;
+            word = (lane >> 3) == static_cast<uint32_t>(kb / 8) ? w : word;
         }
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) v[j] = vn[j];
@@ -251,7 +262,6 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
     __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
     __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
-    __shared__ uint32_t          s_words[kWarps][kSteps];  // ballots of the segment a warp is compacting
     __shared__ volatile uint32_t s_abort;
 
     const uint32_t tid  = threadIdx.x;
@@ -556,16 +566,15 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             y      = static_cast<U *>(a.y) + e0;
             yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
         }
-        const uint32_t seg_addr = smem_addr(tile + warp * kSeg), words_addr = smem_addr(&s_words[warp][0]);
-        uint32_t       run;
+        const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
+        uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, words_addr, lane, lt, y, yvalid);
+            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid);
         else
-            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, words_addr, lane, lt, y, yvalid);
-        __syncwarp();
+            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid);
         if (lane < kSteps) {
             const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * kSteps + lane;
-            if (w < words_total) a.bitmap[w] = s_words[warp][lane];
+            if (w < words_total) a.bitmap[w] = word;
         }
         __syncwarp();
         if (lane == 0) {
