@@ -134,17 +134,6 @@ __device__ __forceinline__ uint32_t lds_elem(uint32_t addr)
     else asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(addr));   // sign-extended (see ReluKeep)
     return v;
 }
-// store `v` at `addr` in the lanes where keep != 0 (a predicated store, never a branch)
-template <typename U>
-__device__ __forceinline__ void sts_elem_if(uint32_t addr, uint32_t v, uint32_t keep)
-{
-    if constexpr (sizeof(U) == 4)
-        asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q st.shared.u32 [%0], %1;\n\t}" ::"r"(addr), "r"(v),
-                     "r"(keep));
-    else
-        asm volatile("{\n\t.reg .pred q;\n\t.reg .b16 h;\n\tsetp.ne.u32 q, %2, 0;\n\tcvt.u16.u32 h, %1;\n\t@q st.shared.u16 [%0], h;\n\t}" ::"r"(addr),
-                     "r"(v), "r"(keep));
-}
 
 // ---------------------------------------------------------------------------------------------
 // One warp compacts its segment of kSteps * 32 elements in place.  Returns the number of packed
