@@ -172,6 +172,59 @@ uint64_t oracle_relu_fwd_compress(const void *pre_act, uint64_t n, int kind,
     return j;
 }
 
+/* Is this element "<= tau" under IEEE comparison?  (false for NaN)  The element is
+ * widened exactly (binary16 / bfloat16 -> binary32, binary64 stays, tau widens
+ * to binary64), so the decision is taken on exact values of both sides. */
+static int le_tau(const unsigned char *e, int kind, float tau)
+{
+    switch (kind) {
+    case ORACLE_F32: { float f; memcpy(&f, e, 4); return f <= tau; }
+    case ORACLE_F64: { double d; memcpy(&d, e, 8); return d <= (double)tau; }
+    case ORACLE_F16: { uint16_t h; memcpy(&h, e, 2); return oracle_half_to_float(h) <= tau; }
+    case ORACLE_BF16: {
+        uint16_t h; memcpy(&h, e, 2);
+        uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4);
+        return f <= tau;
+    }
+    default: return 0;
+    }
+}
+
+/* Activation pruning joined to the stash (section 4, "Combining BitTrain with
+ * Activation Pruning"): only activations that exceed a close-to-zero threshold
+ * tau are stored, the others are taken to be zero.  y = (x <= tau) ? +0 : x --
+ * "exceeds" read as a strict comparison, so that tau = 0 is the ReLU above, and
+ * a NaN, which neither exceeds nor falls below anything, is kept.  Then
+ * Algorithm 1 on y. */
+uint64_t oracle_prune_fwd_compress(const void *x, uint64_t n, int kind, float tau,
+                                   void *y, uint32_t *bitmap, void *values,
+                                   uint64_t *prefix)
+{
+    int elem_size = oracle_elem_size(kind);
+    const unsigned char *src = (const unsigned char *)x;
+    unsigned char *yo = (unsigned char *)y;
+    unsigned char *val = (unsigned char *)values;
+    uint64_t words = (n + 31) / 32;
+    uint64_t j = 0;
+    unsigned char act[8];
+
+    for (uint64_t w = 0; w < words; ++w) bitmap[w] = 0;
+
+    for (uint64_t i = 0; i < n; ++i) {
+        if (i % CHUNK_ELEMS == 0) prefix[i / CHUNK_ELEMS] = j;
+        const unsigned char *e = src + i * (uint64_t)elem_size;
+        if (le_tau(e, kind, tau)) memset(act, 0, (size_t)elem_size);
+        else                      memcpy(act, e, (size_t)elem_size);
+        if (yo) memcpy(yo + i * (uint64_t)elem_size, act, (size_t)elem_size);
+        if (!all_bytes_zero(act, elem_size)) {
+            memcpy(val + j * (uint64_t)elem_size, act, (size_t)elem_size);
+            j += 1;
+            bitmap[i >> 5] |= (uint32_t)1 << (i & 31);
+        }
+    }
+    return j;
+}
+
 /* The ReLU gradient needs only the bitmap: a select, not a multiply, so that a
  * masked lane is +0 whatever the upstream gradient holds (-x, inf, NaN). */
 void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,

@@ -53,6 +53,13 @@ uint64_t oracle_relu_fwd_compress(const void *pre_act, uint64_t n, int kind,
                                   void *y, uint32_t *bitmap, void *values,
                                   uint64_t *prefix);
 
+/* Activation pruning with threshold tau joined to the stash: y = (x <= tau) ? +0 : x
+ * (the element widened exactly, IEEE comparison, NaN kept), then Algorithm 1 on
+ * y.  tau = 0 is oracle_relu_fwd_compress.  y may be NULL.  Returns nnz. */
+uint64_t oracle_prune_fwd_compress(const void *x, uint64_t n, int kind, float tau,
+                                   void *y, uint32_t *bitmap, void *values,
+                                   uint64_t *prefix);
+
 /* grad_in[i] = bit i ? grad_out[i] (raw copy) : +0 */
 void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
                                  uint64_t n, int elem_size, void *grad_in);

@@ -55,6 +55,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_decompress_chunked.argtypes = [vp, vp, vp, u64, i32, vp]
         L.oracle_relu_fwd_compress.restype = u64
         L.oracle_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp]
+        L.oracle_prune_fwd_compress.restype = u64
+        L.oracle_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, vp]
         L.oracle_relu_bwd_from_bitmap.restype = None
         L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
         L.oracle_compressed_bytes.restype = u64
@@ -115,6 +117,21 @@ def relu_fwd_compress(pre_act: np.ndarray, kind: str, want_y: bool = True):
     prefix = np.full((n + CHUNK - 1) // CHUNK, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64)
     nnz = int(lib().oracle_relu_fwd_compress(_ptr(x), n, KINDS[kind], _ptr(y), _ptr(bitmap),
                                               _ptr(values), _ptr(prefix)))
+    return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
+
+
+def prune_fwd_compress(x: np.ndarray, kind: str, tau: float, want_y: bool = True):
+    """Activation pruning with threshold `tau` (a binary32 value) joined to the stash.
+    Returns (y or None, Compressed).  `x` holds raw patterns of `kind`."""
+    xr = _raw(x)
+    assert xr.dtype.itemsize == ELEM_SIZE[kind]
+    n = xr.size
+    y = np.empty(n, dtype=xr.dtype) if want_y else None
+    bitmap = np.full((n + 31) // 32, 0xDEADBEEF, dtype=np.uint32)
+    values = np.empty(n, dtype=xr.dtype)
+    prefix = np.full((n + CHUNK - 1) // CHUNK, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64)
+    nnz = int(lib().oracle_prune_fwd_compress(_ptr(xr), n, KINDS[kind], ctypes.c_float(tau), _ptr(y), _ptr(bitmap),
+                                               _ptr(values), _ptr(prefix)))
     return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
 
 

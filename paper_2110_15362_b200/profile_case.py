@@ -1,0 +1,67 @@
+"""One small, seeded invocation of a kernel, for profiler captures.
+
+    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|decompress|relu_bwd> \
+           [--log2n 26] [--zeros 0.5] [--reps 3]
+
+runs `reps` repetitions of one entry point on a tensor of 2**log2n elements (default 2**26: 256 MiB of
+fp32, larger than the 126 MB L2 and small enough for a multi-pass capture), prints the non-zero count and
+the device status, and exits non-zero if the status is not BT_OK.  The 4-byte input is
+`workloads.cfg3_iid` (independent zeros with the given fraction); the 2-byte input is the ReLU of
+`workloads.cfg4_preact` (about half zeros).  A profiler is pointed at the kernel by name, e.g.
+
+    ncu --set full --clock-control none -k regex:compress_kernel -s 1 -c 1 -o report \
+        python -m paper_2110_15362_b200.profile_case f32 compress
+"""
+from __future__ import annotations
+
+import argparse
+import sys
+
+import torch
+
+from . import binding as B
+from . import workloads as W
+
+
+def main(argv=None) -> int:
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("dtype", choices=["f32", "f16", "bf16"])
+    ap.add_argument("op", choices=["compress", "relu", "relu_y", "decompress", "relu_bwd"])
+    ap.add_argument("--log2n", type=int, default=26)
+    ap.add_argument("--zeros", type=float, default=0.5)
+    ap.add_argument("--reps", type=int, default=3)
+    args = ap.parse_args(argv)
+
+    dev = torch.device("cuda")
+    n = 1 << args.log2n
+    if args.dtype == "f32":
+        x = W.cfg3_iid(n, args.zeros, 2, dev)
+    else:
+        x = torch.relu(W.cfg4_preact(0, (n,), args.dtype, dev))
+    st = B.Stash(n, x.dtype, dev)
+    ws = B.new_workspace(n, dev)
+    d = torch.empty_like(x)
+
+    def compress():
+        B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+
+    for _ in range(args.reps):
+        if args.op == "compress":
+            compress()
+        elif args.op == "relu":
+            B.bt_relu_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif args.op == "relu_y":
+            B.bt_relu_fwd_compress(x, d, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif args.op == "decompress":
+            compress()
+            B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, d)
+        else:
+            compress()
+            B.bt_relu_bwd_from_bitmap(st.bitmap, x, d)
+    torch.cuda.synchronize()
+    print("nnz", st.nnz, "status", st.status)
+    return 0 if st.status == B.BT_OK else 1
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -207,6 +207,31 @@ def random_patterns(n: int, kind: str, zero_fraction: float, seed: int, with_spe
     return x
 
 
+# pruning thresholds of the paper's activation-pruning study (section 4, Figure 9)
+PRUNE_THRESHOLDS = (0.0, 0.01, 0.05, 0.1)
+
+
+def near_threshold_patterns(n: int, kind: str, taus=PRUNE_THRESHOLDS, seed: int = 0) -> np.ndarray:
+    """Raw patterns of `kind` for the pruning tests: close-to-zero activations of both signs (the bulk of
+    a network's activations), and, sprinkled in, each threshold as the element type rounds it, its two
+    neighbours in that type, the special patterns and exact zeros.  Draws only; no comparison is made here."""
+    es = 4 if kind == "f32" else 2
+    tdt = TORCH_DTYPES[kind]
+    g = torch.Generator().manual_seed(seed)
+    body = (torch.randn(n, generator=g) * 0.08).to(tdt)
+    x = raw_numpy(body).copy()
+    if n:
+        rng = np.random.default_rng(seed + 1)
+        edge = []
+        for t in taus:
+            r = int(raw_numpy(torch.tensor([t], dtype=torch.float32).to(tdt))[0])
+            edge += [r, r + 1, max(r - 1, 0), r | (1 << (8 * es - 1))]
+        pool = np.array(edge + list(SPECIALS[kind]) + [0, 0, 0], dtype=_NP_UINT[es])
+        where = rng.integers(0, n, size=max(1, n // 5))
+        x[where] = pool[rng.integers(0, len(pool), size=where.size)]
+    return x
+
+
 def iter_layers(shapes) -> Iterator[Tuple[int, Tuple[int, ...], int]]:
     for i, s in enumerate(shapes):
         yield i, tuple(s), numel(s)

@@ -24,6 +24,12 @@ MUTANTS = {
     "relu_keeps_negatives": ("return f <= 0.0f; }\n    case ORACLE_F64", "return f == 0.0f; }\n    case ORACLE_F64"),
     "bwd_multiplies_instead_of_selecting": ("memset(o + i * (uint64_t)elem_size, 0, (size_t)elem_size);\n    }\n}\n\n/* M_b",
                                             "memmove(o + i * (uint64_t)elem_size, g + i * (uint64_t)elem_size, (size_t)elem_size);\n    }\n}\n\n/* M_b"),
+    "prune_compare_not_strict": ("return f <= tau; }\n    case ORACLE_F64: { double d; memcpy(&d, e, 8); return d <= (double)tau; }",
+                                 "return f < tau; }\n    case ORACLE_F64: { double d; memcpy(&d, e, 8); return d <= (double)tau; }"),
+    "prune_by_magnitude": ("case ORACLE_F32: { float f; memcpy(&f, e, 4); return f <= tau; }",
+                           "case ORACLE_F32: { float f; memcpy(&f, e, 4); return (f < 0 ? -f : f) <= tau; }"),
+    "prune_drops_nan": ("case ORACLE_F32: { float f; memcpy(&f, e, 4); return f <= tau; }",
+                        "case ORACLE_F32: { float f; memcpy(&f, e, 4); return !(f > tau); }"),
     "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
     "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
 }
@@ -45,6 +51,8 @@ def build_mutant(tmp_path, name):
     L.oracle_relu_fwd_compress.restype = u64
     L.oracle_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp]
     L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
+    L.oracle_prune_fwd_compress.restype = u64
+    L.oracle_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, vp]
     L.oracle_compressed_bytes.restype = u64
     L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
     return L
@@ -87,6 +95,14 @@ def pins_hold(L) -> bool:
     gin = np.empty(n, np.uint32)
     L.oracle_relu_bwd_from_bitmap(p(bitmap), p(W.raw_numpy(g)), n, 4, p(gin))
     if not np.array_equal(gin, W.raw_numpy(torch.where(t > 0, g, torch.zeros(())))):
+        return False
+    # pruning: torch.where on a tensor with close-to-zero values of both signs, the threshold itself and a NaN
+    tp = torch.randn(n, generator=torch.Generator().manual_seed(5)) * 0.08
+    tp[:4] = torch.tensor([0.05, float("nan"), -0.2, 0.0])
+    tau = torch.tensor(0.05, dtype=torch.float32)
+    yp = np.empty(n, np.uint32)
+    L.oracle_prune_fwd_compress(p(W.raw_numpy(tp)), n, 0, ctypes.c_float(0.05), p(yp), p(bitmap), p(values), p(prefix))
+    if not np.array_equal(yp, W.raw_numpy(torch.where(tp <= tau, torch.zeros(()), tp))):
         return False
     # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
     if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
