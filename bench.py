@@ -333,6 +333,28 @@ def large_tensor_kernels(dev, peak_gbs: float):
                       for op, (ms, best, by) in res.items()}
         del x, pre, st, ws, dense
         torch.cuda.empty_cache()
+
+    # activation pruning fused with the stash (the next row of the scope after the hot path): one pass
+    # over 2^28 close-to-zero fp32 pre-activations per threshold of the paper's study
+    n = 1 << 28
+    pre = W.prune_preact(n, dev)
+    st = B.Stash(n, pre.dtype, dev)
+    ws = B.new_workspace(n, dev)
+    rows = {}
+    for tau in W.PRUNE_THRESHOLDS:
+        ms, best = time_call(lambda: B.bt_prune_fwd_compress(pre, tau, None, st.bitmap, st.values, st.chunk_prefix,
+                                                             st.nnz_out, ws, st.dev_status))
+        nnz = st.nnz
+        by = algorithmic_bytes("bt_relu_fwd_compress", n, nnz, 4)
+        rows["tau=%g" % tau] = {"ms_median": round(ms, 4), "ms_best": round(best, 4),
+                                "zero_fraction": round(1.0 - nnz / n, 4),
+                                "stash_bytes_over_dense": round(B.bt_compressed_bytes(n, nnz, pre.dtype) / (4.0 * n), 4),
+                                "moved_gbs": round(by / ms / 1e6, 1),
+                                "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
+                                "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
+    out["f32_2^28_bt_prune_fwd_compress_N(0,0.15)"] = rows
+    del pre, st, ws
+    torch.cuda.empty_cache()
     return out
 
 

@@ -126,6 +126,28 @@ int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out
                          int32_t *dev_status, void *stream);
 
 /*
+ * Activation pruning fused with Algorithm 1 (section 4, "Combining BitTrain
+ * with Activation Pruning": only activations that exceed a close-to-zero
+ * threshold are stored, the others are taken to be zero; the paper studies
+ * thresholds 0, 0.01, 0.05 and 0.1).  y[i] = (x[i] <= tau) ? +0 : x[i] under
+ * IEEE comparison, the element widened exactly to binary32 and compared with
+ * the binary32 tau: "exceeds" is read as a strict comparison, so tau = 0 is
+ * exactly bt_relu_fwd_compress, and a NaN (which neither exceeds nor falls
+ * below anything) is kept with its payload.  tau may be negative; a NaN tau
+ * prunes nothing.  Applied to an activation that is already non-negative this
+ * is the thresholded compressor; applied to a pre-activation it is ReLU and
+ * pruning in one pass.  y_out may be NULL and may alias x.  Lossy by design
+ * for tau > 0; what is kept is kept bit for bit.  Other parameters, outputs and
+ * *dev_status as bt_compress.  The backward pass is bt_relu_bwd_from_bitmap /
+ * bt_decompress on the stash, unchanged.
+ */
+int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void *y_out,
+                          uint32_t *bitmap, void *values, uint64_t values_capacity,
+                          uint64_t *chunk_prefix, uint64_t *nnz_out,
+                          void *workspace, size_t workspace_bytes,
+                          int32_t *dev_status, void *stream);
+
+/*
  * ReLU backward from the stash: grad_in[i] = bit i set ? grad_out[i] : +0.
  * The backward pass restores activations to form gradients (section 3.2); for
  * ReLU itself only the bitmap is needed.  A select, not a multiply: masked

@@ -26,7 +26,8 @@ CHUNK = 4096
 DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_BF16}
 EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
-           "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc")
+           "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
+           "bt_prune_fwd_compress")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -64,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.bt_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
         L.bt_relu_bwd_from_bitmap.restype = i32
         L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
+        L.bt_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -142,6 +144,21 @@ def bt_relu_fwd_compress(pre_act: torch.Tensor, y_out: Optional[torch.Tensor], b
                                     _stream(stream))
     return _check("bt_relu_fwd_compress", st, check)
 
+
+
+def bt_prune_fwd_compress(x: torch.Tensor, tau: float, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
+                          values: torch.Tensor, chunk_prefix: torch.Tensor, nnz_out: torch.Tensor,
+                          workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                          *, n: Optional[int] = None, values_capacity: Optional[int] = None, stream=None,
+                          check: bool = True) -> int:
+    """Activation pruning fused with the stash: elements <= tau (a binary32 threshold) become +0."""
+    n = x.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    st = lib().bt_prune_fwd_compress(_ptr(x), n, DTYPE_CODE[x.dtype], ctypes.c_float(tau), _ptr(y_out), _ptr(bitmap),
+                                     _ptr(values), cap, _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _ptr(dev_status),
+                                     _stream(stream))
+    return _check("bt_prune_fwd_compress", st, check)
 
 def bt_decompress(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor, dense_out: torch.Tensor,
                   *, n: Optional[int] = None, stream=None, check: bool = True) -> int:

@@ -17,7 +17,7 @@ inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintp
 
 inline uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
 
-int compress_common(const void *src, uint64_t n, int dtype, bool relu, void *y, uint32_t *bitmap, void *values,
+int compress_common(const void *src, uint64_t n, int dtype, bool relu, float tau, void *y, uint32_t *bitmap, void *values,
                     uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
                     size_t workspace_bytes, int32_t *dev_status, void *stream)
 {
@@ -49,6 +49,7 @@ int compress_common(const void *src, uint64_t n, int dtype, bool relu, void *y, 
     a.ws_header  = static_cast<uint32_t *>(workspace);
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
+    a.tau        = tau;
     a.n          = n;
     return bt::launch_compress(a, dtype, relu, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
@@ -73,7 +74,7 @@ int bt_compress(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void
                 uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace, size_t workspace_bytes,
                 int32_t *dev_status, void *stream)
 {
-    return compress_common(dense, n, dtype, false, nullptr, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+    return compress_common(dense, n, dtype, false, 0.0f, nullptr, bitmap, values, values_capacity, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream);
 }
 
@@ -81,7 +82,15 @@ int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out
                          uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
                          size_t workspace_bytes, int32_t *dev_status, void *stream)
 {
-    return compress_common(pre_act, n, dtype, true, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+    return compress_common(pre_act, n, dtype, true, 0.0f, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream);
+}
+
+int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void *y_out, uint32_t *bitmap, void *values,
+                          uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
+                          size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    return compress_common(x, n, dtype, true, tau, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream);
 }
 

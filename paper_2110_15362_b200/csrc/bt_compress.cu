@@ -131,7 +131,7 @@ __device__ __forceinline__ uint32_t lds_elem(uint32_t addr)
 {
     uint32_t v;
     if constexpr (sizeof(U) == 4) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    else asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(addr));   // sign-extended (see ReluKeep)
+    else asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(addr));   // sign-extended
     return v;
 }
 
@@ -146,7 +146,7 @@ __device__ __forceinline__ uint32_t lds_elem(uint32_t addr)
 // step k lands below element 32(k+1) and a later batch reads at or above it, so they never meet.
 template <typename U, int RELU_DT, bool WRITE_Y, bool kGuardY, int kSteps>
 __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uint32_t &word, const uint32_t lane,
-                                                    const uint32_t lt, U *y, const uint32_t yvalid)
+                                                    const uint32_t lt, U *y, const uint32_t yvalid, const float tau)
 {
     constexpr int      kBatch = 8;
     static_assert(kSteps % kBatch == 0 && kSteps <= 32, "whole batches; one bitmap word per lane");
@@ -169,7 +169,7 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
         for (int j = 0; j < kBatch; ++j) {
             uint32_t x = v[j];
             if constexpr (RELU_DT >= 0) {
-                x = ReluKeep<RELU_DT>::keep(x) ? x : 0u;
+                x = KeepAbove<RELU_DT>::keep(x, tau) ? x : 0u;
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
                     if (!kGuardY || e < yvalid) y[e] = static_cast<U>(x);
@@ -558,9 +558,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
         uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid);
+            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau);
         else
-            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid);
+            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau);
         if (lane < kSteps) {
             const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * kSteps + lane;
             if (w < words_total) a.bitmap[w] = word;

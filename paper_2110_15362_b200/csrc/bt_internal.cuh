@@ -31,6 +31,7 @@ struct CompressArgs {
     uint32_t   *ws_header;
     uint64_t   *ws_desc;    // wave totals, then tile descriptors
     uint32_t    ws_waves;   // number of wave totals
+    float       tau;        // fused forms: elements <= tau become +0 (0 for plain ReLU)
     uint64_t    n;
 };
 
@@ -136,33 +137,28 @@ __device__ __forceinline__ uint32_t lanemask_lt()
     return m;
 }
 
-// ---------------------------------------------------------------- ReLU on bit patterns
-// keep(x) = !(x <= 0) under IEEE comparison: positive (non-zero magnitude, sign
-// clear) or NaN (magnitude above the exponent mask, either sign).
+// ---------------------------------------------------------------- keep what exceeds the threshold
+// keep(x, tau) = !(x <= tau) under IEEE comparison, the element widened exactly to binary32: true for
+// values above tau and for NaN.  tau = 0 is the ReLU decision (positive or NaN).  The 16-bit forms take
+// the pattern in the low half of the register (the upper half may hold a sign extension).
 template <int DT>
-struct ReluKeep;
+struct KeepAbove;
 template <>
-struct ReluKeep<BT_F32> {
-    __device__ static __forceinline__ bool keep(uint32_t u)
-    {
-        return (static_cast<int32_t>(u) > 0) | (u > 0xFF800000u);
-    }
+struct KeepAbove<BT_F32> {
+    __device__ static __forceinline__ bool keep(uint32_t u, float tau) { return !(__uint_as_float(u) <= tau); }
 };
-// The 16-bit forms take the pattern SIGN-EXTENDED to 32 bits (as `ld.shared.s16` delivers it): positive
-// is then one signed compare, a negative NaN one unsigned compare against the sign-extended -inf.
 template <>
-struct ReluKeep<BT_F16> {
-    __device__ static __forceinline__ bool keep(uint32_t u)
+struct KeepAbove<BT_F16> {
+    __device__ static __forceinline__ bool keep(uint32_t u, float tau)
     {
-        return (static_cast<int32_t>(u) > 0) | (u > 0xFFFFFC00u);
+        float f;
+        asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(static_cast<unsigned short>(u)));
+        return !(f <= tau);
     }
 };
 template <>
-struct ReluKeep<BT_BF16> {
-    __device__ static __forceinline__ bool keep(uint32_t u)
-    {
-        return (static_cast<int32_t>(u) > 0) | (u > 0xFFFFFF80u);
-    }
+struct KeepAbove<BT_BF16> {
+    __device__ static __forceinline__ bool keep(uint32_t u, float tau) { return !(__uint_as_float(u << 16) <= tau); }
 };
 
 }  // namespace bt

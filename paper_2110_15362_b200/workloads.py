@@ -207,6 +207,14 @@ def random_patterns(n: int, kind: str, zero_fraction: float, seed: int, with_spe
     return x
 
 
+def prune_preact(n: int, device="cpu", seed: int = 0) -> torch.Tensor:
+    """fp32 pre-activations for the pruning measurement: N(0, 0.15), so that half are not positive and
+    about three quarters do not exceed 0.1 -- the paper's observation that more than 70 % of a network's
+    activations are close to zero (section 3.1, activation histogram)."""
+    g = _gen(900 + seed, device)
+    return torch.randn(n, generator=g, device=device) * 0.15
+
+
 # pruning thresholds of the paper's activation-pruning study (section 4, Figure 9)
 PRUNE_THRESHOLDS = (0.0, 0.01, 0.05, 0.1)
 

@@ -54,7 +54,8 @@ class GpuCompressed:
 
 
 def gpu_compress(x: torch.Tensor, relu: bool = False, want_y: bool = False, capacity=None,
-                 in_place: bool = False, keep_device: bool = False):
+                 in_place: bool = False, keep_device: bool = False, tau=None):
+    """`tau` given: bt_prune_fwd_compress with that threshold (want_y / in_place as for the ReLU form)."""
     n = x.numel()
     cap = n if capacity is None else capacity
     bitmap = Guarded((n + 31) // 32, torch.int32)
@@ -64,7 +65,7 @@ def gpu_compress(x: torch.Tensor, relu: bool = False, want_y: bool = False, capa
     status = Guarded(1, torch.int32)
     ws = B.new_workspace(n)
     y = None
-    if relu:
+    if relu or tau is not None:
         if in_place:
             y_t = x
         elif want_y:
@@ -72,8 +73,12 @@ def gpu_compress(x: torch.Tensor, relu: bool = False, want_y: bool = False, capa
             y_t = y.inner
         else:
             y_t = None
-        B.bt_relu_fwd_compress(x, y_t, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws, status.inner,
-                               n=n, values_capacity=cap)
+        if tau is not None:
+            B.bt_prune_fwd_compress(x, tau, y_t, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws,
+                                    status.inner, n=n, values_capacity=cap)
+        else:
+            B.bt_relu_fwd_compress(x, y_t, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws, status.inner,
+                                   n=n, values_capacity=cap)
     else:
         B.bt_compress(x, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws, status.inner,
                       n=n, values_capacity=cap)
