@@ -125,7 +125,7 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # DRAM bytes per launch (read + write) of the dominant kernel class over one step of this workload, from the ncu
 # capture summarised in profiles/bench_cfg2_launch_list.md (bytes; None where no capture exists)
-NCU_TRAFFIC_PER_LAUNCH = {"bt_compress": 18.26e6, "bt_relu_fwd_compress": 18.28e6}
+NCU_TRAFFIC_PER_LAUNCH = {"bt_compress": 20.57e6, "bt_relu_fwd_compress": 20.61e6, "bt_decompress": 13.88e6}
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:

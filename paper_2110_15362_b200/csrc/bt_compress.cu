@@ -1,49 +1,52 @@
-// Algorithm 1 (dense -> bitmap) and its ReLU-fused form as ONE compaction pass:
-// a persistent-CTA stream compaction whose prefix sum rides on the wave
-// structure of the grid.
+// Algorithm 1 (dense -> bitmap) and its fused forms (ReLU, activation pruning) as ONE
+// compaction pass: a persistent-CTA stream compaction whose prefix sum rides on the
+// wave structure of the grid.
 //
 // The grid is launched cooperatively with exactly as many CTAs (G) as fit on
 // the device at once, so all of them are co-resident, and CTA b takes tiles
 // b, b+G, b+2G, ...: iteration j of every CTA together forms "wave j", G
-// consecutive tiles.  Tiles are staged into shared memory by 1-D bulk async
-// copies through a ring of kStages slots, and the warps of a CTA are
-// specialised: one load warp (a single lane issues the bulk copies), kWarps
-// compactor warps, one scan warp, kWarps copier warps.
+// consecutive tiles.  The warps of a CTA are specialised: one load warp,
+// kWarps compactor warps, two scan warps, kCopiers copier warps.
 //
-// Compactor warp w owns kTile / kWarps consecutive elements of the tile:
+// Compaction.  Compactor warp w owns segment w (1024 elements) of the tile:
 //
-//   step k of a warp:  lane l reads element 32k+l of its segment from shared memory;
-//                      ballot(non-zero) IS bitmap word k (LSB first);
-//                      popc(ballot & lanemask_lt) is the lane's rank;
-//                      non-zero lanes write the element back IN PLACE at
-//                      [run + rank] of the warp's own segment (always at or
-//                      before the position being read, so nothing unread is
-//                      overwritten); all shared accesses are conflict-free.
+//   step k:  lane l reads element 32k+l (conflict-free shared load);
+//            ballot(non-zero) IS bitmap word k (LSB first), kept by lane k;
+//            popc(ballot & lanemask_lt) is the lane's rank;
+//            non-zero lanes store the element at [run + rank] of the same
+//            segment -- in place: the write position never passes the read
+//            position, and a batch's loads are issued before the previous
+//            batch's stores;
+//            run += popc(ballot).
 //
-// The ballots are parked in shared memory by lane 0 and leave as one coalesced
-// bitmap store per warp; the segment's first `run` slots hold the packed values.
+// After 32 steps the segment's first `run` entries hold the packed values and
+// lane k holds bitmap word k: one coalesced 128-byte bitmap store per warp.
 //
 // Prefix.  The exclusive base of tile (wave j, CTA b) is
 //     sum of the totals of waves 0..j-1  +  sum of the counts of CTAs 0..b-1 in wave j.
-// As soon as a tile is compacted its scan warp publishes the tile count in a
-// descriptor and adds it (with a 1 in a counter field) to the wave's total with
-// one fire-and-forget reduction.  One iteration later -- when every CTA has
-// long published wave j -- it reads the b descriptors of its own wave and the
-// now complete total of wave j-1 in ONE batch of independent loads, and uses
-// them an iteration after that, so the round trip to L2 hides behind the
-// compaction of the following tiles.  No tile waits on another tile's base:
-// only on counts, which never wait on anything but the data.
+// As soon as a tile is counted a scan warp publishes the count in a descriptor
+// and adds it (with a 1 in a counter field) to the wave's total with one
+// fire-and-forget reduction.  About one tile later -- when every CTA has
+// published wave j -- it reads the b descriptors of its wave and the now
+// complete totals of the waves before it in ONE batch of independent loads,
+// and uses them a tile after that.  The two scan warps alternate tiles, so
+// that each has two tiles' time for that round trip to L2.  No tile waits on
+// another tile's base: only on counts, which never wait on anything but data.
 //
-// The warps of a CTA never meet at a CTA-wide barrier; a ring slot goes round
-// through four mbarriers:
-//   full[s]     the bulk copy has landed                   (copy engine -> compactors)
-//   counted[s]  every compactor has posted its count       (compactors  -> scan warp)
-//   ready[s]    base and segment offsets are in shared     (scan warp   -> copiers)
-//   empty[s]    every copier has copied its segment out    (copiers     -> load warp)
-// Copier warp w copies segment w's packed slots to values[base + offset ...].
-// The scan warp works on three tiles at a time (publish, read, finish), so the
-// compactors run about three tiles ahead of the copiers and nobody waits for a
-// round trip to L2.
+// Pipeline.  The warps of a CTA never meet at a CTA-wide barrier after the
+// prologue; a ring slot goes round through four mbarriers:
+//   full[s]     the bulk copy of the tile has landed         (copy engine -> compactors)
+//   counted[s]  every compactor has posted its count         (compactors  -> scan warps)
+//   ready[s]    base and segment offsets are in shared       (scan warp   -> copiers)
+//   empty[s]    every copier has copied its segments out     (copiers     -> load warp)
+// Copier warp c copies its segments' packed values to values[base + offset ...].
+// With a ring of 6 or 7 tiles the load warp runs several tiles ahead of the
+// compactors and the compactors several tiles ahead of the copiers, so nobody
+// waits for a round trip to L2 or to HBM.
+//
+// Workspace.  It arrives with unspecified contents; the scan warps zero it and
+// meet once at the grid barrier word of the cooperative launch before the
+// first count is published, while the other warps already work on the data.
 #include <cooperative_groups.h>
 
 #include <cstdlib>
