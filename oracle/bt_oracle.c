@@ -225,6 +225,34 @@ uint64_t oracle_prune_fwd_compress(const void *x, uint64_t n, int kind, float ta
     return j;
 }
 
+/* Double-mask batch normalisation (section 3.1: the zero pattern of the
+ * normalisation layer's INPUT is applied as a mask to its OUTPUT, which carries
+ * the sparsity through the layer).  The mask is the bitmap the input's stash
+ * already holds, so the output's stash reuses it and only needs the vector of
+ * values: walk the elements as Algorithm 1 does, but push x[i] where bit i of
+ * the mask is 1 -- whatever x[i] is -- instead of testing x[i].  y, when asked
+ * for, is the masked dense tensor.  Returns the number of values pushed (the
+ * number of set bits among the first n). */
+uint64_t oracle_mask_compress(const void *x, uint64_t n, int elem_size,
+                              const uint32_t *mask_bitmap, void *y, void *values)
+{
+    const unsigned char *src = (const unsigned char *)x;
+    unsigned char *yo = (unsigned char *)y;
+    unsigned char *val = (unsigned char *)values;
+    uint64_t j = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const unsigned char *e = src + i * (uint64_t)elem_size;
+        if ((mask_bitmap[i >> 5] >> (i & 31)) & 1u) {
+            memcpy(val + j * (uint64_t)elem_size, e, (size_t)elem_size);
+            j += 1;
+            if (yo) memcpy(yo + i * (uint64_t)elem_size, e, (size_t)elem_size);
+        } else if (yo) {
+            memset(yo + i * (uint64_t)elem_size, 0, (size_t)elem_size);
+        }
+    }
+    return j;
+}
+
 /* The ReLU gradient needs only the bitmap: a select, not a multiply, so that a
  * masked lane is +0 whatever the upstream gradient holds (-x, inf, NaN). */
 void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,

@@ -60,6 +60,13 @@ uint64_t oracle_prune_fwd_compress(const void *x, uint64_t n, int kind, float ta
                                    void *y, uint32_t *bitmap, void *values,
                                    uint64_t *prefix);
 
+/* Double-mask batch normalisation: values = the elements of x at the set bits
+ * of mask_bitmap, in element order (pushed whatever their value); y (may be
+ * NULL) = x at set bits, +0 elsewhere.  The stash of the result is
+ * (mask_bitmap, values, the mask's own prefix array).  Returns the count. */
+uint64_t oracle_mask_compress(const void *x, uint64_t n, int elem_size,
+                              const uint32_t *mask_bitmap, void *y, void *values);
+
 /* grad_in[i] = bit i ? grad_out[i] (raw copy) : +0 */
 void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
                                  uint64_t n, int elem_size, void *grad_in);

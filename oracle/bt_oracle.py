@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp]
         L.oracle_prune_fwd_compress.restype = u64
         L.oracle_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, vp]
+        L.oracle_mask_compress.restype = u64
+        L.oracle_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp]
         L.oracle_relu_bwd_from_bitmap.restype = None
         L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
         L.oracle_compressed_bytes.restype = u64
@@ -133,6 +135,18 @@ def prune_fwd_compress(x: np.ndarray, kind: str, tau: float, want_y: bool = True
     nnz = int(lib().oracle_prune_fwd_compress(_ptr(xr), n, KINDS[kind], ctypes.c_float(tau), _ptr(y), _ptr(bitmap),
                                                _ptr(values), _ptr(prefix)))
     return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
+
+
+def mask_compress(x: np.ndarray, mask_bitmap: np.ndarray, want_y: bool = True):
+    """Double-mask form: returns (y or None, values) for raw patterns `x` under `mask_bitmap`."""
+    xr = _raw(x)
+    n = xr.size
+    bm = np.ascontiguousarray(mask_bitmap, dtype=np.uint32)
+    assert bm.size >= (n + 31) // 32
+    y = np.empty(n, dtype=xr.dtype) if want_y else None
+    values = np.empty(n, dtype=xr.dtype)
+    cnt = int(lib().oracle_mask_compress(_ptr(xr), n, xr.dtype.itemsize, _ptr(bm), _ptr(y), _ptr(values)))
+    return y, values[:cnt].copy()
 
 
 def relu_bwd_from_bitmap(bitmap: np.ndarray, grad_out: np.ndarray) -> np.ndarray:

@@ -30,6 +30,10 @@ MUTANTS = {
                            "case ORACLE_F32: { float f; memcpy(&f, e, 4); return (f < 0 ? -f : f) <= tau; }"),
     "prune_drops_nan": ("case ORACLE_F32: { float f; memcpy(&f, e, 4); return f <= tau; }",
                         "case ORACLE_F32: { float f; memcpy(&f, e, 4); return !(f > tau); }"),
+    "mask_drops_zero_values": ("if ((mask_bitmap[i >> 5] >> (i & 31)) & 1u) {\n            memcpy(val",
+                               "if (((mask_bitmap[i >> 5] >> (i & 31)) & 1u) && !all_bytes_zero(e, elem_size)) {\n            memcpy(val"),
+    "mask_msb_first": ("if ((mask_bitmap[i >> 5] >> (i & 31)) & 1u) {\n            memcpy(val",
+                       "if ((mask_bitmap[i >> 5] >> (31 - (i & 31))) & 1u) {\n            memcpy(val"),
     "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
     "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
 }
@@ -53,6 +57,8 @@ def build_mutant(tmp_path, name):
     L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
     L.oracle_prune_fwd_compress.restype = u64
     L.oracle_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, vp]
+    L.oracle_mask_compress.restype = u64
+    L.oracle_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp]
     L.oracle_compressed_bytes.restype = u64
     L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
     return L
@@ -103,6 +109,16 @@ def pins_hold(L) -> bool:
     yp = np.empty(n, np.uint32)
     L.oracle_prune_fwd_compress(p(W.raw_numpy(tp)), n, 0, ctypes.c_float(0.05), p(yp), p(bitmap), p(values), p(prefix))
     if not np.array_equal(yp, W.raw_numpy(torch.where(tp <= tau, torch.zeros(()), tp))):
+        return False
+    # double mask: numpy boolean indexing under a mask that also covers zero elements
+    rng = np.random.default_rng(9)
+    mask = rng.random(n) < 0.4
+    mp = np.packbits(mask, bitorder="little")
+    mbm = np.concatenate([mp, np.zeros((-mp.size) % 4, np.uint8)]).view("<u4").copy()
+    ym = np.empty(n, np.uint32)
+    vm = np.zeros(n, np.uint32)
+    cnt = L.oracle_mask_compress(p(x), n, 4, p(mbm), p(ym), p(vm))
+    if cnt != int(mask.sum()) or not np.array_equal(vm[:cnt], x[mask]) or not np.array_equal(ym, np.where(mask, x, 0)):
         return False
     # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
     if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
