@@ -325,6 +325,16 @@ def large_tensor_kernels(dev, peak_gbs: float):
         res["bt_relu_fwd_compress+y"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, es, True))
         ms, best = time_call(lambda: B.bt_relu_bwd_from_bitmap(st.bitmap, x, dense))
         res["bt_relu_bwd_from_bitmap"] = (ms, best, algorithmic_bytes("bt_relu_bwd_from_bitmap", n, 0, es))
+        # double-mask form (a "next" row): the stash of x masks a dense tensor of the same shape
+        B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        nnz = st.nnz
+        masked_vals = torch.empty(nnz, dtype=x.dtype, device=dev)
+        by = n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + nnz * es
+        ms, best = time_call(lambda: B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, None, masked_vals))
+        res["bt_mask_compress"] = (ms, best, by)
+        ms, best = time_call(lambda: B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, dense, masked_vals))
+        res["bt_mask_compress+y"] = (ms, best, by + n * es)
+        del masked_vals
         out[label] = {op: {"ms_median": round(ms, 4), "ms_best": round(best, 4),
                            "moved_gbs": round(by / ms / 1e6, 1),
                            "dense_equiv_gbs": round(n * es / ms / 1e6, 1),

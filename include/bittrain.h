@@ -148,6 +148,26 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
                           int32_t *dev_status, void *stream);
 
 /*
+ * Double-mask batch normalisation support (section 3.1: the zero pattern of
+ * the normalisation layer's input is applied as a mask to its output, which
+ * carries the sparsity through the layer).  mask_bitmap / mask_chunk_prefix are
+ * the bitmap and prefix array of the INPUT's stash (as bt_compress or
+ * bt_relu_fwd_compress wrote them); x is the layer's dense output.  Writes
+ * values[k] = x[i] for the k-th set bit i, in element order, whatever x[i] is
+ * (a zero under a set bit is stored as a value), so that (mask_bitmap, values,
+ * mask_chunk_prefix) is the stash of the masked output -- bitmap, prefix array
+ * and nnz are shared with the input's stash and are not written again -- and
+ * bt_decompress restores it.  y_out, if not NULL, receives the masked dense
+ * tensor (x at set bits, +0 elsewhere) and may alias x.  values must hold the
+ * mask's nnz elements; stores at or beyond values_capacity are suppressed.
+ * Bits of the last bitmap word beyond n are ignored.  No workspace, no scan:
+ * ranks come from the prefix array.
+ */
+int bt_mask_compress(const void *x, uint64_t n, int dtype,
+                     const uint32_t *mask_bitmap, const uint64_t *mask_chunk_prefix,
+                     void *y_out, void *values, uint64_t values_capacity, void *stream);
+
+/*
  * ReLU backward from the stash: grad_in[i] = bit i set ? grad_out[i] : +0.
  * The backward pass restores activations to form gradients (section 3.2); for
  * ReLU itself only the bitmap is needed.  A select, not a multiply: masked

@@ -27,7 +27,7 @@ DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_B
 EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
-           "bt_prune_fwd_compress")
+           "bt_prune_fwd_compress", "bt_mask_compress")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -66,6 +66,9 @@ def lib() -> ctypes.CDLL:
         L.bt_relu_bwd_from_bitmap.restype = i32
         L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
         L.bt_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_prune_fwd_compress.restype = i32
+        L.bt_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp, u64, vp]
+        L.bt_mask_compress.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -159,6 +162,17 @@ def bt_prune_fwd_compress(x: torch.Tensor, tau: float, y_out: Optional[torch.Ten
                                      workspace.numel() * workspace.element_size(), _ptr(dev_status),
                                      _stream(stream))
     return _check("bt_prune_fwd_compress", st, check)
+
+def bt_mask_compress(x: torch.Tensor, mask_bitmap: torch.Tensor, mask_chunk_prefix: torch.Tensor,
+                     y_out: Optional[torch.Tensor], values: torch.Tensor, *, n: Optional[int] = None,
+                     values_capacity: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """Double-mask form: the values of x at the set bits of an existing stash's bitmap (and the masked dense y)."""
+    n = x.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    st = lib().bt_mask_compress(_ptr(x), n, DTYPE_CODE[x.dtype], _ptr(mask_bitmap), _ptr(mask_chunk_prefix),
+                                _ptr(y_out), _ptr(values), cap, _stream(stream))
+    return _check("bt_mask_compress", st, check)
+
 
 def bt_decompress(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor, dense_out: torch.Tensor,
                   *, n: Optional[int] = None, stream=None, check: bool = True) -> int:

@@ -110,6 +110,23 @@ int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *ch
                : BT_ERR_CUDA;
 }
 
+int bt_mask_compress(const void *x, uint64_t n, int dtype, const uint32_t *mask_bitmap, const uint64_t *mask_chunk_prefix,
+                     void *y_out, void *values, uint64_t values_capacity, void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!x || !mask_bitmap || !mask_chunk_prefix) return BT_ERR_NULL;
+    if (!values && values_capacity != 0) return BT_ERR_NULL;
+    if (!aligned(x, 16) || !aligned(y_out, 16) || !aligned(mask_bitmap, 16) || !aligned(values, 16) ||
+        !aligned(mask_chunk_prefix, 8))
+        return BT_ERR_ALIGN;
+    return bt::launch_mask_gather(x, mask_bitmap, mask_chunk_prefix, n, es, y_out, values, values_capacity,
+                                  static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
 int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out, uint64_t n, int dtype, void *grad_in,
                             void *stream)
 {

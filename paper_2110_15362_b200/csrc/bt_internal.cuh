@@ -38,6 +38,8 @@ struct CompressArgs {
 cudaError_t launch_compress(const CompressArgs &a, int dtype, bool relu, cudaStream_t s);
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *prefix,
                               uint64_t n, int elem_size, void *out, cudaStream_t s);
+cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,
+                               int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t s);
 cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size,
                             void *gin, cudaStream_t s);
 

@@ -1,0 +1,203 @@
+// Double-mask batch normalisation support (section 3.1): the zero pattern of a
+// normalisation layer's input, which that input's stash already holds as a
+// bitmap, is applied to the layer's output.  The output's stash reuses the
+// bitmap and its chunk prefix array, so all this pass has to produce is the
+// vector of values: x[i] at every set bit, in element order.
+//
+// Ranks come from the existing prefix array plus popcounts inside the chunk, so
+// there is no scan and no communication: the mirror image of the decompressor.
+// One warp, one quarter chunk (1024 elements = 32 bitmap words):
+//   - lane l loads the 4 words 4l..4l+3 of the WHOLE chunk together with
+//     chunk_prefix[c]; the popcounts of the lanes in front of this warp's quarter
+//     give the count in front of it, four shuffles hand lane l word l of its own
+//     quarter, a warp scan of the 32 word popcounts gives word offsets;
+//   - the quarter of x is read with 16-byte loads (all of them issued before the
+//     first store): a lane owns kE consecutive elements, i.e. kE consecutive bits
+//     of one word; the rank of its first set bit is  chunk base + quarter base +
+//     word offset + popc(lower bits of the word);  its set elements go to the
+//     warp's staging area in shared memory at that rank (the lanes' runs abut),
+//     shifted so that a staged element and its place in values[] have the same
+//     position within a 16-byte vector;
+//   - the staged run leaves for values[] with 16-byte stores (single elements at
+//     its ragged ends): scattered 2-byte stores straight to global memory ran at
+//     a third of the bandwidth;
+//   - optionally the masked dense tensor leaves with 16-byte stores.
+#include "bt_internal.cuh"
+
+namespace bt {
+namespace {
+
+constexpr uint32_t kFull = 0xFFFFFFFFu;
+
+template <typename U, int kE, int kWarps, bool WRITE_Y>
+__global__ void __launch_bounds__(kWarps * 32)
+mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64_t *__restrict__ prefix,
+                   const uint64_t n, U *y, U *__restrict__ values, const uint64_t capacity)   // y may alias x
+{
+    constexpr int kVec          = 16 / sizeof(U);          // elements per 16-byte vector
+    constexpr int kLanesPerWord = 32 / kE;
+    constexpr int kWordsPerStep = kE;
+    constexpr int kSteps        = 32 / kWordsPerStep;
+    static_assert(kE % kVec == 0 && 32 % kE == 0 && kE < 32, "a lane takes whole vectors of one word");
+
+    const uint32_t lane        = threadIdx.x & 31u;
+    const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    const uint64_t quarters    = (n + 1023) >> 10;
+    if (warp_global >= quarters) return;
+
+    const uint64_t chunk       = warp_global >> 2;
+    const uint32_t q           = static_cast<uint32_t>(warp_global & 3u);
+    const uint64_t words_total = (n + 31) >> 5;
+    const uint64_t w0          = chunk * 128 + 4 * lane;   // this lane's four words of the chunk
+    const uint64_t e0          = warp_global << 10;        // first element of the quarter
+
+    // the quarter of x first: these loads do not depend on the bitmap
+    U e[kSteps][kE];
+#pragma unroll
+    for (int k = 0; k < kSteps; ++k) {
+        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+#pragma unroll
+        for (int v = 0; v < kE / kVec; ++v) {
+            const uint64_t at = eo + v * kVec;
+            U             *ev = e[k] + v * kVec;
+            if (at + kVec <= n) {
+                const uint4 pack = *reinterpret_cast<const uint4 *>(x + at);
+                if constexpr (kVec == 4) {
+                    ev[0] = pack.x, ev[1] = pack.y, ev[2] = pack.z, ev[3] = pack.w;
+                } else {
+                    ev[0] = static_cast<U>(pack.x), ev[1] = static_cast<U>(pack.x >> 16);
+                    ev[2] = static_cast<U>(pack.y), ev[3] = static_cast<U>(pack.y >> 16);
+                    ev[4] = static_cast<U>(pack.z), ev[5] = static_cast<U>(pack.z >> 16);
+                    ev[6] = static_cast<U>(pack.w), ev[7] = static_cast<U>(pack.w >> 16);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kVec; ++j) ev[j] = at + j < n ? x[at + j] : U(0);
+            }
+        }
+    }
+
+    // the chunk's 128 words (zero past the end of the bitmap) and its prefix entry
+    uint4 w4 = make_uint4(0, 0, 0, 0);
+    if (w0 + 3 < words_total) {
+        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
+    } else {
+        if (w0 < words_total) w4.x = bitmap[w0];
+        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
+        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
+    }
+    const uint64_t chunk_base = prefix[chunk];
+
+    uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(kFull, before, o);
+
+    // lane l takes word l of its own quarter: component l & 3 of lane 8q + (l >> 2)
+    const int      src = 8 * q + (lane >> 2);
+    const uint32_t c0 = __shfl_sync(kFull, w4.x, src), c1 = __shfl_sync(kFull, w4.y, src);
+    const uint32_t c2 = __shfl_sync(kFull, w4.z, src), c3 = __shfl_sync(kFull, w4.w, src);
+    uint32_t       word = (lane & 2u) ? ((lane & 1u) ? c3 : c2) : ((lane & 1u) ? c1 : c0);
+    // bits past the end of the tensor do not count (a well-formed bitmap has none)
+    const uint64_t word_first = e0 + 32ull * lane;
+    if (word_first >= n) word = 0;
+    else if (n - word_first < 32) word &= (1u << static_cast<uint32_t>(n - word_first)) - 1u;
+
+    uint32_t incl = __popc(word);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t u = __shfl_up_sync(kFull, incl, o);
+        if (lane >= static_cast<uint32_t>(o)) incl += u;
+    }
+    const uint32_t excl = incl - __popc(word);
+    const uint64_t vbase = chunk_base + before;             // rank of the quarter's first set bit
+
+    // staging area of this warp: 1024 elements plus one vector of slack for the alignment shift
+    __shared__ __align__(16) U s_stage[kWarps][1024 + kVec];
+    U *const       stage = s_stage[threadIdx.x >> 5];
+    const uint32_t skew  = static_cast<uint32_t>(vbase % kVec);   // staged index i <-> values[vbase - skew + i]
+    const uint32_t total = __shfl_sync(kFull, incl, 31);          // set bits of the quarter
+
+    const uint32_t shift = (lane % kLanesPerWord) * kE;     // which kE-bit group of the word
+#pragma unroll
+    for (int k = 0; k < kSteps; ++k) {
+        const int      from = k * kWordsPerStep + lane / kLanesPerWord;
+        const uint32_t w    = __shfl_sync(kFull, word, from);
+        const uint32_t wex  = __shfl_sync(kFull, excl, from);
+        const uint32_t bits = (w >> shift) & ((1u << kE) - 1u);
+        uint32_t       off  = skew + wex + __popc(w & ((1u << shift) - 1u));
+#pragma unroll
+        for (int j = 0; j < kE; ++j) {
+            const bool set = (bits >> j) & 1u;
+            if (set) stage[off] = e[k][j];
+            off += set;
+            if constexpr (WRITE_Y) e[k][j] = set ? e[k][j] : U(0);
+        }
+        if constexpr (WRITE_Y) {
+            const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+#pragma unroll
+            for (int v = 0; v < kE / kVec; ++v) {
+                const uint64_t at = eo + v * kVec;
+                const U       *ev = e[k] + v * kVec;
+                if (at + kVec <= n) {
+                    uint4 pack;
+                    if constexpr (kVec == 4) {
+                        pack = make_uint4(ev[0], ev[1], ev[2], ev[3]);
+                    } else {
+                        pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
+                                          ev[4] | (uint32_t(ev[5]) << 16), ev[6] | (uint32_t(ev[7]) << 16));
+                    }
+                    *reinterpret_cast<uint4 *>(y + at) = pack;
+                } else {
+#pragma unroll
+                    for (int j = 0; j < kVec; ++j)
+                        if (at + j < n) y[at + j] = ev[j];
+                }
+            }
+        }
+    }
+    __syncwarp();
+
+    // staged [skew, skew + total) -> values[vbase, vbase + total), clipped to the capacity
+    const uint64_t gbase = vbase - skew;                    // a multiple of kVec: staged vector v <-> values + gbase + v * kVec
+    const uint32_t end   = skew + total;
+    const uint32_t vecs  = (end + kVec - 1) / kVec;
+    for (uint32_t v = lane; v < vecs; v += 32) {
+        const uint32_t lo = v * kVec, hi = lo + kVec;
+        const uint64_t g  = gbase + lo;
+        if (lo >= skew && hi <= end && g + kVec <= capacity) {
+            *reinterpret_cast<uint4 *>(values + g) = *reinterpret_cast<const uint4 *>(stage + lo);
+        } else {
+#pragma unroll
+            for (int j = 0; j < kVec; ++j)
+                if (lo + j >= skew && lo + j < end && g + j < capacity) values[g + j] = stage[lo + j];
+        }
+    }
+}
+
+template <typename U, int kE>
+cudaError_t launch_typed(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n, void *y,
+                         void *values, uint64_t capacity, cudaStream_t stream)
+{
+    constexpr int  kWarps   = 8;
+    const uint64_t quarters = (n + 1023) >> 10;
+    const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
+    if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    if (y)
+        mask_gather_kernel<U, kE, kWarps, true><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
+            static_cast<const U *>(x), bitmap, prefix, n, static_cast<U *>(y), static_cast<U *>(values), capacity);
+    else
+        mask_gather_kernel<U, kE, kWarps, false><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
+            static_cast<const U *>(x), bitmap, prefix, n, nullptr, static_cast<U *>(values), capacity);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,
+                               int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t stream)
+{
+    return elem_size == 4 ? launch_typed<uint32_t, 4>(x, bitmap, prefix, n, y, values, capacity, stream)
+                          : launch_typed<uint16_t, 8>(x, bitmap, prefix, n, y, values, capacity, stream);
+}
+
+}  // namespace bt

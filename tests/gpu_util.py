@@ -114,3 +114,27 @@ def gpu_relu_bwd(bitmap: np.ndarray, g: torch.Tensor, in_place: bool = False):
     B.bt_relu_bwd_from_bitmap(bm, g, out.inner, n=n)
     torch.cuda.synchronize()
     return out.raw(), out.guards_intact()
+
+
+def gpu_mask_compress(x: torch.Tensor, bitmap: np.ndarray, prefix: np.ndarray, nnz: int, mode: str = "with_y",
+                      capacity=None):
+    """bt_mask_compress under the given stash bitmap / prefix; returns (values[:nnz], y or None, guards intact).
+    mode: "stash_only", "with_y" or "in_place" (y written over x)."""
+    n = x.numel()
+    cap = nnz if capacity is None else capacity
+    bm = torch.from_numpy(bitmap.view(np.int32).copy()).cuda()
+    pf = torch.from_numpy(prefix.view(np.int64).copy()).cuda()
+    values = Guarded(max(cap, 1), x.dtype)
+    y = None
+    if mode == "with_y":
+        y = Guarded(n, x.dtype)
+        y_t = y.inner
+    elif mode == "in_place":
+        y_t = x
+    else:
+        y_t = None
+    B.bt_mask_compress(x, bm, pf, y_t, values.inner, n=n, values_capacity=cap)
+    torch.cuda.synchronize()
+    ok = values.guards_intact() and (y is None or y.guards_intact())
+    y_raw = y.raw() if y is not None else (W.raw_numpy(x) if mode == "in_place" else None)
+    return values.raw()[:min(nnz, cap)], y_raw, ok
