@@ -297,9 +297,13 @@ def large_tensor_kernels(dev, peak_gbs: float):
             best.append(e0.elapsed_time(e1))
         return statistics.median(best), min(best)
 
-    for label, kind, n in (("f32_2^28_s0.5", "f32", 1 << 28), ("bf16_64x64x224x224", "bf16", 64 * 64 * 224 * 224)):
+    for label, kind, n in (("f32_2^28_s0.5", "f32", 1 << 28), ("bf16_64x64x224x224", "bf16", 64 * 64 * 224 * 224),
+                           ("f64_2^27_s0.5", "f64", 1 << 27)):
         if kind == "f32":
             x = W.cfg3_iid(n, 0.5, 2, dev)
+            pre = x
+        elif kind == "f64":
+            x = W.cfg3_iid(n, 0.5, 3, dev).double()
             pre = x
         else:
             pre = W.cfg4_preact(0, (n,), kind, dev)
@@ -314,8 +318,8 @@ def large_tensor_kernels(dev, peak_gbs: float):
         nnz = st.nnz
         res["bt_compress"] = (ms, best, algorithmic_bytes("bt_compress", n, nnz, es))
         ms, best = time_call(lambda: B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, dense))
-        assert torch.equal(dense.view(torch.int16 if es == 2 else torch.int32),
-                           x.view(torch.int16 if es == 2 else torch.int32))
+        iv = {2: torch.int16, 4: torch.int32, 8: torch.int64}[es]
+        assert torch.equal(dense.view(iv), x.view(iv))
         res["bt_decompress"] = (ms, best, algorithmic_bytes("bt_decompress", n, nnz, es))
         ms, best = time_call(lambda: B.bt_relu_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix,
                                                             st.nnz_out, ws, st.dev_status))

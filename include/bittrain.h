@@ -51,8 +51,9 @@ extern "C" {
 
 #define BT_CHUNK_ELEMS 4096u
 
-/* element types: the codec proper only needs the width, the ReLU pair the format */
-enum { BT_F32 = 0, BT_F16 = 1, BT_BF16 = 2 };
+/* element types: the codec proper only needs the width, the ReLU pair the format
+ * (the paper's format covers the usual floating-point widths, double included) */
+enum { BT_F32 = 0, BT_F16 = 1, BT_BF16 = 2, BT_F64 = 3 };
 
 enum {
     BT_OK = 0,
@@ -130,8 +131,8 @@ int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out
  * with Activation Pruning": only activations that exceed a close-to-zero
  * threshold are stored, the others are taken to be zero; the paper studies
  * thresholds 0, 0.01, 0.05 and 0.1).  y[i] = (x[i] <= tau) ? +0 : x[i] under
- * IEEE comparison, the element widened exactly to binary32 and compared with
- * the binary32 tau: "exceeds" is read as a strict comparison, so tau = 0 is
+ * IEEE comparison, the element widened exactly to binary32 (for BT_F64, tau
+ * widened to binary64) and compared with the binary32 tau: "exceeds" is read as a strict comparison, so tau = 0 is
  * exactly bt_relu_fwd_compress, and a NaN (which neither exceeds nor falls
  * below anything) is kept with its payload.  tau may be negative; a NaN tau
  * prunes nothing.  Applied to an activation that is already non-negative this

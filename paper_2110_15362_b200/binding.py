@@ -15,7 +15,7 @@ import torch
 
 from . import build as _build
 
-BT_F32, BT_F16, BT_BF16 = 0, 1, 2
+BT_F32, BT_F16, BT_BF16, BT_F64 = 0, 1, 2, 3
 (BT_OK, BT_ERR_NULL, BT_ERR_DTYPE, BT_ERR_ALIGN, BT_ERR_WORKSPACE, BT_ERR_CAPACITY, BT_ERR_TIMEOUT, BT_ERR_CUDA,
  BT_ERR_TOO_LARGE) = range(9)
 STATUS_NAMES = ["BT_OK", "BT_ERR_NULL", "BT_ERR_DTYPE", "BT_ERR_ALIGN", "BT_ERR_WORKSPACE", "BT_ERR_CAPACITY",
@@ -23,7 +23,7 @@ STATUS_NAMES = ["BT_OK", "BT_ERR_NULL", "BT_ERR_DTYPE", "BT_ERR_ALIGN", "BT_ERR_
 NOALLOC_MAX_ELEMS = 1 << 26
 CHUNK = 4096
 
-DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_BF16}
+DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_BF16, torch.float64: BT_F64}
 EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",

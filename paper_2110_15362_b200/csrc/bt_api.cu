@@ -9,6 +9,7 @@ inline int elem_size_of(int dtype)
     case BT_F32: return 4;
     case BT_F16: return 2;
     case BT_BF16: return 2;
+    case BT_F64: return 8;
     default: return 0;
     }
 }

@@ -129,11 +129,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 }
 
 // shared-memory accesses by 32-bit shared address, kept in program order among themselves
+// register type that holds one element: 64 bits for 8-byte elements, 32 bits otherwise
 template <typename U>
-__device__ __forceinline__ uint32_t lds_elem(uint32_t addr)
+using Reg = std::conditional_t<sizeof(U) == 8, uint64_t, uint32_t>;
+
+template <typename U>
+__device__ __forceinline__ Reg<U> lds_elem(uint32_t addr)
 {
-    uint32_t v;
-    if constexpr (sizeof(U) == 4) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    Reg<U> v;
+    if constexpr (sizeof(U) == 8) asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr));
+    else if constexpr (sizeof(U) == 4) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     else asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(addr));   // sign-extended
     return v;
 }
@@ -156,8 +161,8 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
     constexpr uint32_t kES    = sizeof(U);
     const uint32_t     in0    = seg_addr + lane * kES;
     uint32_t           out    = seg_addr;               // address of the next free packed slot
-    uint32_t           v[kBatch], vn[kBatch];
-    uint32_t   bb[kBatch];
+    Reg<U>             v[kBatch], vn[kBatch];
+    uint32_t           bb[kBatch];
     const bool l0 = lane & 1u, l1 = lane & 2u, l2 = lane & 4u;
     word = 0;
 #pragma unroll
@@ -170,19 +175,20 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
         }
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
-            uint32_t x = v[j];
+            Reg<U> x = v[j];
             if constexpr (RELU_DT >= 0) {
-                x = KeepAbove<RELU_DT>::keep(x, tau) ? x : 0u;
+                x = KeepAbove<RELU_DT>::keep(x, tau) ? x : Reg<U>(0);
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
                     if (!kGuardY || e < yvalid) y[e] = static_cast<U>(x);
                 }
             }
-            const uint32_t b = __ballot_sync(kFull, x != 0u);
+            const uint32_t b = __ballot_sync(kFull, x != Reg<U>(0));
             bb[j] = b;
-            if (x != 0u) {
+            if (x != Reg<U>(0)) {
                 const uint32_t at = out + kES * __popc(b & lt);
-                if constexpr (kES == 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"(x));
+                if constexpr (kES == 8) asm volatile("st.shared.u64 [%0], %1;" ::"r"(at), "l"(x));
+                else if constexpr (kES == 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"(x));
                 else asm volatile("st.shared.u16 [%0], %1;" ::"r"(at), "h"(static_cast<uint16_t>(x)));
             }
             out += kES * __popc(b);
@@ -638,12 +644,14 @@ template <typename U, int RELU_DT, bool WRITE_Y>
 cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
 {
     // One CTA per SM, the ring takes nearly all of its shared memory.
+    //   8-byte elements: 8 compactor warps x 512 elements (32 KB tiles), 8 copiers, 7 stages;
     //   4-byte elements: 8 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 7 stages;
     //   2-byte elements: 16 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 6 stages --
     //   a 2-byte tile takes as many compaction steps per byte again, so it gets twice the warps.
 #ifdef BT_PROFILE
     static const int cfg = [] { const char *e = getenv("BT_CFG"); return e ? atoi(e) : 0; }();
-    if constexpr (sizeof(U) == 4) {
+    if constexpr (sizeof(U) == 8) {
+    } else if constexpr (sizeof(U) == 4) {
         if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 6, 8>(a, stream);
         if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 4>(a, stream);
         if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 512, 7, 8>(a, stream);
@@ -653,7 +661,8 @@ cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
         if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 1024, 6, 16>(a, stream);
     }
 #endif
-    if constexpr (sizeof(U) == 4) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 8>(a, stream);
+    if constexpr (sizeof(U) == 8) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 512, 7, 8>(a, stream);
+    else if constexpr (sizeof(U) == 4) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 8>(a, stream);
     else return launch_shaped<U, RELU_DT, WRITE_Y, 16, 1024, 6, 8>(a, stream);
 }
 
@@ -672,10 +681,13 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, bool relu, cudaStr
 {
     const bool y = a.y != nullptr;
     if (!relu) {
-        return dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(a, stream)
-                               : launch_typed<uint16_t, -1, false>(a, stream);
+        return dtype == BT_F64   ? launch_typed<uint64_t, -1, false>(a, stream)
+               : dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(a, stream)
+                                 : launch_typed<uint16_t, -1, false>(a, stream);
     }
     switch (dtype) {
+    case BT_F64:
+        return y ? launch_typed<uint64_t, BT_F64, true>(a, stream) : launch_typed<uint64_t, BT_F64, false>(a, stream);
     case BT_F32:
         return y ? launch_typed<uint32_t, BT_F32, true>(a, stream) : launch_typed<uint32_t, BT_F32, false>(a, stream);
     case BT_F16:

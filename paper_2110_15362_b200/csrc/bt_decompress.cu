@@ -20,7 +20,7 @@ namespace {
 
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 
-// kE: elements a lane decodes per step (a multiple of one 16-byte vector)
+// kE: elements a lane decodes per step (a multiple of one 16-byte vector: 2 for 8-byte, 4 for 4-byte, 8 for 2-byte elements)
 template <typename U, int kE, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
 decompress_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values,
@@ -101,7 +101,10 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ val
             const U       *ev = e[k] + v * kVec;
             if (at + kVec <= n) {
                 uint4 pack;
-                if constexpr (kVec == 4) {
+                if constexpr (kVec == 2) {
+                    pack = make_uint4(static_cast<uint32_t>(ev[0]), static_cast<uint32_t>(ev[0] >> 32),
+                                      static_cast<uint32_t>(ev[1]), static_cast<uint32_t>(ev[1] >> 32));
+                } else if constexpr (kVec == 4) {
                     pack = make_uint4(ev[0], ev[1], ev[2], ev[3]);
                 } else {
                     pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
@@ -140,6 +143,7 @@ cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const 
 #else
     constexpr int kE32 = 4, kE16 = 8;
 #endif
+    if (elem_size == 8) return launch_typed<uint64_t, 2>(bitmap, values, prefix, n, out, stream);
     return elem_size == 4 ? launch_typed<uint32_t, kE32>(bitmap, values, prefix, n, out, stream)
                           : launch_typed<uint16_t, kE16>(bitmap, values, prefix, n, out, stream);
 }

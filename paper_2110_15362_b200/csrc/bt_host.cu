@@ -8,7 +8,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
-inline int    elem_size_of(int dtype) { return dtype == BT_F32 ? 4 : (dtype == BT_F16 || dtype == BT_BF16) ? 2 : 0; }
+inline int    elem_size_of(int dtype) { return dtype == BT_F64 ? 8 : dtype == BT_F32 ? 4 : (dtype == BT_F16 || dtype == BT_BF16) ? 2 : 0; }
 
 // Carves the staging area; every region starts 256-byte aligned.
 struct Staging {

@@ -140,7 +140,7 @@ __device__ __forceinline__ uint32_t lanemask_lt()
 }
 
 // ---------------------------------------------------------------- keep what exceeds the threshold
-// keep(x, tau) = !(x <= tau) under IEEE comparison, the element widened exactly to binary32: true for
+// keep(x, tau) = !(x <= tau) under IEEE comparison, the element widened exactly to binary32 (binary64 elements: tau widened to binary64): true for
 // values above tau and for NaN.  tau = 0 is the ReLU decision (positive or NaN).  The 16-bit forms take
 // the pattern in the low half of the register (the upper half may hold a sign extension).
 template <int DT>
@@ -148,6 +148,13 @@ struct KeepAbove;
 template <>
 struct KeepAbove<BT_F32> {
     __device__ static __forceinline__ bool keep(uint32_t u, float tau) { return !(__uint_as_float(u) <= tau); }
+};
+template <>
+struct KeepAbove<BT_F64> {
+    __device__ static __forceinline__ bool keep(uint64_t u, float tau)
+    {
+        return !(__longlong_as_double(static_cast<long long>(u)) <= static_cast<double>(tau));
+    }
 };
 template <>
 struct KeepAbove<BT_F16> {

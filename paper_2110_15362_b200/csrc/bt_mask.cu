@@ -62,7 +62,10 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
             U             *ev = e[k] + v * kVec;
             if (at + kVec <= n) {
                 const uint4 pack = *reinterpret_cast<const uint4 *>(x + at);
-                if constexpr (kVec == 4) {
+                if constexpr (kVec == 2) {
+                    ev[0] = pack.x | (static_cast<uint64_t>(pack.y) << 32);
+                    ev[1] = pack.z | (static_cast<uint64_t>(pack.w) << 32);
+                } else if constexpr (kVec == 4) {
                     ev[0] = pack.x, ev[1] = pack.y, ev[2] = pack.z, ev[3] = pack.w;
                 } else {
                     ev[0] = static_cast<U>(pack.x), ev[1] = static_cast<U>(pack.x >> 16);
@@ -140,7 +143,10 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
                 const U       *ev = e[k] + v * kVec;
                 if (at + kVec <= n) {
                     uint4 pack;
-                    if constexpr (kVec == 4) {
+                    if constexpr (kVec == 2) {
+                        pack = make_uint4(static_cast<uint32_t>(ev[0]), static_cast<uint32_t>(ev[0] >> 32),
+                                          static_cast<uint32_t>(ev[1]), static_cast<uint32_t>(ev[1] >> 32));
+                    } else if constexpr (kVec == 4) {
                         pack = make_uint4(ev[0], ev[1], ev[2], ev[3]);
                     } else {
                         pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
@@ -178,7 +184,7 @@ template <typename U, int kE>
 cudaError_t launch_typed(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n, void *y,
                          void *values, uint64_t capacity, cudaStream_t stream)
 {
-    constexpr int  kWarps   = 8;
+    constexpr int  kWarps   = sizeof(U) == 8 ? 4 : 8;   // the staging area of a CTA stays below 48 KB
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
@@ -196,6 +202,7 @@ cudaError_t launch_typed(const void *x, const uint32_t *bitmap, const uint64_t *
 cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,
                                int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t stream)
 {
+    if (elem_size == 8) return launch_typed<uint64_t, 2>(x, bitmap, prefix, n, y, values, capacity, stream);
     return elem_size == 4 ? launch_typed<uint32_t, 4>(x, bitmap, prefix, n, y, values, capacity, stream)
                           : launch_typed<uint16_t, 8>(x, bitmap, prefix, n, y, values, capacity, stream);
 }

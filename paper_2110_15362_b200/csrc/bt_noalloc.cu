@@ -46,7 +46,7 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
                                    uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out,
                                    int32_t *dev_status, void *stream)
 {
-    if (dtype != BT_F32 && dtype != BT_F16 && dtype != BT_BF16) return BT_ERR_DTYPE;
+    if (dtype != BT_F32 && dtype != BT_F16 && dtype != BT_BF16 && dtype != BT_F64) return BT_ERR_DTYPE;
     if (n > BT_NOALLOC_MAX_ELEMS) return BT_ERR_TOO_LARGE;      // the built-in scratch cannot describe more tiles
     if (!nnz_out) return BT_ERR_NULL;
     if (!aligned(nnz_out, 8) || !aligned(dev_status, 4)) return BT_ERR_ALIGN;

@@ -1,6 +1,6 @@
 // ReLU backward from the stashed bitmap: grad_in[i] = bit i ? grad_out[i] : +0.
-// A pure streaming select: every thread moves 16-byte vectors (4 fp32 or 8
-// 16-bit elements, i.e. 4 or 8 consecutive bits of one bitmap word), several
+// A pure streaming select: every thread moves 16-byte vectors (2 fp64, 4 fp32 or
+// 8 16-bit elements, i.e. 2, 4 or 8 consecutive bits of one bitmap word), several
 // independent vectors in flight per thread.
 #include "bt_internal.cuh"
 
@@ -20,6 +20,14 @@ __device__ __forceinline__ uint4 select_vec<uint32_t>(uint4 g, uint32_t bits)
     g.y = (bits & 2u) ? g.y : 0u;
     g.z = (bits & 4u) ? g.z : 0u;
     g.w = (bits & 8u) ? g.w : 0u;
+    return g;
+}
+
+template <>
+__device__ __forceinline__ uint4 select_vec<uint64_t>(uint4 g, uint32_t bits)
+{
+    if (!(bits & 1u)) g.x = g.y = 0u;
+    if (!(bits & 2u)) g.z = g.w = 0u;
     return g;
 }
 
@@ -92,8 +100,9 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *gout, uint64_t n, v
 cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size, void *gin,
                             cudaStream_t stream)
 {
-    return elem_size == 4 ? launch_typed<uint32_t>(bitmap, gout, n, gin, stream)
-                          : launch_typed<uint16_t>(bitmap, gout, n, gin, stream);
+    return elem_size == 8   ? launch_typed<uint64_t>(bitmap, gout, n, gin, stream)
+           : elem_size == 4 ? launch_typed<uint32_t>(bitmap, gout, n, gin, stream)
+                            : launch_typed<uint16_t>(bitmap, gout, n, gin, stream);
 }
 
 }  // namespace bt

@@ -18,11 +18,12 @@ from typing import Dict, Iterator, List, Sequence, Tuple
 import numpy as np
 import torch
 
-TORCH_DTYPES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+TORCH_DTYPES = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16, "f64": torch.float64}
 _INT_VIEW = {1: torch.uint8, 2: torch.int16, 4: torch.int32, 8: torch.int64}
 _NP_UINT = {2: np.uint16, 4: np.uint32, 8: np.uint64}
 
 SPARSITY_SWEEP = (0.0, 0.25, 0.5, 0.7, 0.9, 0.99)
+ELEM_BYTES = {"f32": 4, "f16": 2, "bf16": 2, "f64": 8}
 
 
 def raw_numpy(t: torch.Tensor) -> np.ndarray:
@@ -187,7 +188,11 @@ SPECIAL_F16 = (0x0000, 0x8000, 0x3C00, 0xBC00, 0x0001, 0x8001, 0x7C00, 0xFC00, 0
                0x7C01, 0xFC01)
 SPECIAL_BF16 = (0x0000, 0x8000, 0x3F80, 0xBF80, 0x0001, 0x8001, 0x7F80, 0xFF80, 0x7FC0, 0xFFC1,
                 0x7F81, 0xFF81)
-SPECIALS = {"f32": SPECIAL_F32, "f16": SPECIAL_F16, "bf16": SPECIAL_BF16}
+SPECIAL_F64 = (0x0000000000000000, 0x8000000000000000, 0x3FF0000000000000, 0xBFF0000000000000,
+               0x0000000000000001, 0x8000000000000001, 0x7FF0000000000000, 0xFFF0000000000000,
+               0x7FF8000000000000, 0xFFF8000000000001, 0x7FF0000000000001, 0xFFF0000000000001,
+               0x0000000100000000, 0x00000000FFFFFFFF)          # the last two: non-zero in one 32-bit half only
+SPECIALS = {"f32": SPECIAL_F32, "f16": SPECIAL_F16, "bf16": SPECIAL_BF16, "f64": SPECIAL_F64}
 
 
 def random_patterns(n: int, kind: str, zero_fraction: float, seed: int, with_specials: bool = True
@@ -196,9 +201,12 @@ def random_patterns(n: int, kind: str, zero_fraction: float, seed: int, with_spe
     subnormals and negative values all occur), zeroed at Bernoulli(zero_fraction)
     positions, with the special patterns (signed zeros, infinities, NaNs, smallest
     subnormals) sprinkled in."""
-    es = 4 if kind == "f32" else 2
+    es = ELEM_BYTES[kind]
     rng = np.random.default_rng(seed)
-    x = rng.integers(0, 1 << (8 * es), size=n, dtype=np.uint64).astype(_NP_UINT[es])
+    if es == 8:
+        x = rng.integers(0, 1 << 63, size=n, dtype=np.uint64) | (rng.integers(0, 2, size=n, dtype=np.uint64) << np.uint64(63))
+    else:
+        x = rng.integers(0, 1 << (8 * es), size=n, dtype=np.uint64).astype(_NP_UINT[es])
     x[rng.random(n) < zero_fraction] = 0
     if with_specials and n:
         sp = np.array(SPECIALS[kind], dtype=_NP_UINT[es])
@@ -223,7 +231,7 @@ def near_threshold_patterns(n: int, kind: str, taus=PRUNE_THRESHOLDS, seed: int 
     """Raw patterns of `kind` for the pruning tests: close-to-zero activations of both signs (the bulk of
     a network's activations), and, sprinkled in, each threshold as the element type rounds it, its two
     neighbours in that type, the special patterns and exact zeros.  Draws only; no comparison is made here."""
-    es = 4 if kind == "f32" else 2
+    es = ELEM_BYTES[kind]
     tdt = TORCH_DTYPES[kind]
     g = torch.Generator().manual_seed(seed)
     body = (torch.randn(n, generator=g) * 0.08).to(tdt)

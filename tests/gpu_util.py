@@ -9,7 +9,7 @@ from paper_2110_15362_b200 import binding as B
 from paper_2110_15362_b200 import workloads as W
 
 GUARD = 64            # guard elements on each side of every output buffer
-TDT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+TDT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16, "f64": torch.float64}
 _INT = {2: torch.int16, 4: torch.int32, 8: torch.int64}
 
 
@@ -39,7 +39,7 @@ class Guarded:
 def from_raw(x: np.ndarray, kind: str, device="cuda") -> torch.Tensor:
     """Device tensor of torch dtype `kind` holding exactly the raw patterns in x."""
     es = x.dtype.itemsize
-    t = torch.from_numpy(x.view({2: np.int16, 4: np.int32}[es]).copy()).to(device)
+    t = torch.from_numpy(x.view({2: np.int16, 4: np.int32, 8: np.int64}[es]).copy()).to(device)
     return t.view(TDT[kind])
 
 

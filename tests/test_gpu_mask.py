@@ -10,7 +10,7 @@ from paper_2110_15362_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
 
-KINDS = ["f32", "f16", "bf16"]
+KINDS = ["f32", "f16", "bf16", "f64"]
 
 
 @pytest.fixture(scope="module")

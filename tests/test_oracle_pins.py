@@ -158,10 +158,10 @@ def test_half_widening_matches_numpy_for_every_pattern(oracle):
     assert np.isnan(got[nan].view(np.float32)).all()
 
 
-@pytest.mark.parametrize("kind", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("kind", ["f32", "f16", "bf16", "f64"])
 def test_relu_fwd_matches_torch_relu(oracle, kind):
     n = 2 * 4096 + 77
-    t = (torch.randn(n, generator=torch.Generator().manual_seed(11)) * 3).to(W.TORCH_DTYPES[kind])
+    t = (torch.randn(n, generator=torch.Generator().manual_seed(11), dtype=torch.float64) * 3).to(W.TORCH_DTYPES[kind])
     t[::97] = 0.0
     t[5::101] = -0.0
     t[7] = float("inf"); t[8] = float("-inf")
@@ -169,12 +169,12 @@ def test_relu_fwd_matches_torch_relu(oracle, kind):
     y, c = oracle.relu_fwd_compress(x, kind)
     # torch.relu keeps the sign of -0.0; adding +0.0 (exact in every precision) turns
     # that one case into +0.0, which is the reading taken here, and changes nothing else.
-    y_ref = W.raw_numpy((torch.relu(t.float()) + 0.0).to(t.dtype))
+    y_ref = W.raw_numpy((torch.relu(t.double()) + 0.0).to(t.dtype))
     assert np.array_equal(y, y_ref)
-    assert not (y == (0x8000 if x.dtype.itemsize == 2 else 0x80000000)).any()      # no -0.0 survives
+    assert not (y == (1 << (8 * x.dtype.itemsize - 1))).any()                       # no -0.0 survives
     # bit i == (x[i] > 0), the ReLU derivative mask
     bits = np.unpackbits(c.bitmap.view(np.uint8), bitorder="little")[:n].astype(bool)
-    assert np.array_equal(bits, (t.float() > 0).numpy())
+    assert np.array_equal(bits, (t.double() > 0).numpy())
     # and the compressed form is the plain compressor applied to y
     c2 = oracle.compress(y)
     assert c.nnz == c2.nnz and all(np.array_equal(a, b) for a, b in zip(c[:3], c2[:3]))
@@ -182,14 +182,14 @@ def test_relu_fwd_matches_torch_relu(oracle, kind):
     assert y_none is None and all(np.array_equal(a, b) for a, b in zip(c[:3], c3[:3]))
 
 
-@pytest.mark.parametrize("kind", ["f32", "f16", "bf16"])
+@pytest.mark.parametrize("kind", ["f32", "f16", "bf16", "f64"])
 def test_relu_fwd_special_patterns(oracle, kind):
     """+-0, negatives, -inf -> +0; positives incl. subnormals and +inf unchanged; NaN kept with payload."""
-    es = 4 if kind == "f32" else 2
+    es = W.ELEM_BYTES[kind]
     sp = np.array(W.SPECIALS[kind], dtype=UINT[es])
     y, c = oracle.relu_fwd_compress(sp, kind)
     sign = 1 << (8 * es - 1)
-    expmask = {"f32": 0x7F800000, "f16": 0x7C00, "bf16": 0x7F80}[kind]
+    expmask = {"f32": 0x7F800000, "f16": 0x7C00, "bf16": 0x7F80, "f64": 0x7FF0000000000000}[kind]
     for xin, yout in zip(sp.tolist(), y.tolist()):
         mag = xin & (sign - 1)
         is_nan = mag > expmask
