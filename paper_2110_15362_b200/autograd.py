@@ -1,0 +1,190 @@
+"""The stash wired into PyTorch's autograd: activations that a layer saves for its backward pass are kept
+in the sparse-bitmap form and restored when the backward pass asks for them (the integration the paper
+names as its first contribution and, for GPUs, as future work: section 1 and the conclusion).
+
+Two pieces, both thin wrappers around the C-ABI calls (no arithmetic here):
+
+* ``stash_saved_activations()`` -- a ``torch.autograd.graph.saved_tensors_hooks`` context.  Every eligible
+  tensor saved inside it (CUDA, floating point, contiguous, large enough, not a parameter) is compressed
+  with ``bt_compress``; only the bitmap, the chunk prefix array and exactly ``nnz`` values stay alive.  On
+  the way back ``bt_decompress`` rebuilds the tensor bit for bit, so gradients are unchanged.  A tensor
+  that would not shrink (too few zeros) is kept as it is.
+* ``relu_stash(x)`` -- a ReLU whose forward pass writes the activation and its stash in one kernel
+  (``bt_relu_fwd_compress``) and whose backward pass needs only the bitmap
+  (``bt_relu_bwd_from_bitmap``).  Inside the context above its stash is shared with the next layer's saved
+  input, so the activation is compressed once.
+
+Getting the exact ``nnz`` to size the values costs one device-to-host read per packed tensor.
+"""
+from __future__ import annotations
+
+import weakref
+from typing import Dict, Optional, Tuple
+
+import torch
+
+from . import binding as B
+
+__all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash"]
+
+
+class PackedActivation:
+    """What replaces a saved tensor: the stash and the metadata needed to rebuild it."""
+
+    __slots__ = ("bitmap", "values", "chunk_prefix", "shape", "dtype", "device", "nnz", "__weakref__")
+
+    def __init__(self, bitmap, values, chunk_prefix, shape, dtype, device, nnz):
+        self.bitmap, self.values, self.chunk_prefix = bitmap, values, chunk_prefix
+        self.shape, self.dtype, self.device, self.nnz = shape, dtype, device, nnz
+
+    @property
+    def numel(self) -> int:
+        n = 1
+        for s in self.shape:
+            n *= s
+        return n
+
+    def nbytes(self) -> int:
+        return B.bt_compressed_bytes(self.numel, self.nnz, self.dtype)
+
+    def unpack(self) -> torch.Tensor:
+        out = torch.empty(self.shape, dtype=self.dtype, device=self.device)
+        B.bt_decompress(self.bitmap, self.values, self.chunk_prefix, out.view(-1))
+        return out
+
+
+class _Scratch:
+    """Per-device reusable buffers of the packing calls: workspace and a full-capacity values buffer."""
+
+    def __init__(self):
+        self.ws: Dict[torch.device, torch.Tensor] = {}
+        self.values: Dict[Tuple[torch.device, torch.dtype], torch.Tensor] = {}
+
+    def workspace(self, n: int, device) -> torch.Tensor:
+        need = B.bt_workspace_bytes(n)
+        ws = self.ws.get(device)
+        if ws is None or ws.numel() < need:
+            ws = self.ws[device] = torch.empty(need, dtype=torch.uint8, device=device)
+        return ws
+
+    def full_values(self, n: int, dtype, device) -> torch.Tensor:
+        key = (device, dtype)
+        v = self.values.get(key)
+        if v is None or v.numel() < n:
+            v = self.values[key] = torch.empty(n, dtype=dtype, device=device)
+        return v
+
+
+def _compress(flat: torch.Tensor, scratch: _Scratch, relu_into: Optional[torch.Tensor] = None):
+    """Runs the (fused) compressor on a flat tensor; returns bitmap, exact-size values, prefix, nnz."""
+    n, dev = flat.numel(), flat.device
+    bitmap = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
+    prefix = torch.empty((n + B.CHUNK - 1) // B.CHUNK, dtype=torch.int64, device=dev)
+    nnz_out = torch.empty(1, dtype=torch.int64, device=dev)
+    status = torch.empty(1, dtype=torch.int32, device=dev)
+    full = scratch.full_values(n, flat.dtype, dev)
+    ws = scratch.workspace(n, dev)
+    if relu_into is None:
+        B.bt_compress(flat, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
+    else:
+        B.bt_relu_fwd_compress(flat, relu_into, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
+    nnz = int(nnz_out.item())                       # the one host read: sizes the values exactly
+    st = int(status.item())
+    if st != B.BT_OK:
+        raise B.BitTrainError("bt_compress (autograd stash)", st)
+    return bitmap, full[:nnz].clone(), prefix, nnz
+
+
+class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
+    """Context manager: saved activations are kept compressed between the forward and the backward pass."""
+
+    def __init__(self, min_numel: int = 1 << 14, min_saving: float = 0.1):
+        self.min_numel, self.min_saving = min_numel, min_saving
+        self.scratch = _Scratch()
+        self.packed_bytes = 0            # bytes kept in compressed form so far
+        self.dense_bytes = 0             # bytes the same tensors would have taken
+        self._shared: Dict[int, Tuple[weakref.ref, weakref.ref]] = {}
+        super().__init__(self._pack, self._unpack)
+
+    # ---- sharing of one stash between several saves of the same tensor object
+    # The table holds weak references only: a stash lives as long as the tensor object it belongs to (which
+    # carries it as an attribute) or a saved-tensor slot of the graph, and is freed with them.
+    def share(self, tensor: torch.Tensor, packed: PackedActivation) -> None:
+        tensor._bt_packed = packed
+        self._shared[id(tensor)] = (weakref.ref(tensor), weakref.ref(packed))
+
+    def _lookup(self, tensor: torch.Tensor) -> Optional[PackedActivation]:
+        hit = self._shared.get(id(tensor))
+        if hit is None:
+            return None
+        ref, packed_ref = hit
+        packed = packed_ref()
+        if ref() is tensor and packed is not None:
+            return packed
+        del self._shared[id(tensor)]     # the id was recycled by another object
+        return None
+
+    def _eligible(self, t: torch.Tensor) -> bool:
+        return (t.is_cuda and t.dtype in B.DTYPE_CODE and t.is_contiguous() and t.numel() >= self.min_numel
+                and not isinstance(t, torch.nn.Parameter) and not (t.requires_grad and t.is_leaf))
+
+    def _pack(self, t: torch.Tensor):
+        if not self._eligible(t):
+            return t
+        shared = self._lookup(t)
+        if shared is not None:
+            return shared
+        n, es = t.numel(), t.element_size()
+        bitmap, values, prefix, nnz = _compress(t.detach().view(-1), self.scratch)
+        if B.bt_compressed_bytes(n, nnz, t.dtype) > (1.0 - self.min_saving) * n * es:
+            return t                                  # too few zeros: the stash would not be smaller
+        packed = PackedActivation(bitmap, values, prefix, tuple(t.shape), t.dtype, t.device, nnz)
+        self.share(t, packed)
+        self.packed_bytes += packed.nbytes()
+        self.dense_bytes += n * es
+        return packed
+
+    @staticmethod
+    def _unpack(obj):
+        return obj.unpack() if isinstance(obj, PackedActivation) else obj
+
+    def __enter__(self):
+        super().__enter__()
+        return self
+
+    def __exit__(self, *exc):
+        self._shared.clear()
+        return super().__exit__(*exc)
+
+
+class ReLUStash(torch.autograd.Function):
+    """ReLU with the stash fused into its forward pass; the backward pass reads only the bitmap."""
+
+    @staticmethod
+    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None):
+        xc = x.contiguous()
+        y = torch.empty_like(xc)
+        scratch = hooks.scratch if hooks is not None else _Scratch()
+        bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1))
+        ctx.save_for_backward(bitmap)     # released with the graph, like any saved tensor
+        if hooks is not None:
+            # the next layer will save y as its input: hand it this stash instead of compressing y again
+            packed = PackedActivation(bitmap, values, prefix, tuple(y.shape), y.dtype, y.device, nnz)
+            hooks.share(y, packed)
+            hooks.packed_bytes += packed.nbytes()
+            hooks.dense_bytes += y.numel() * y.element_size()
+        return y
+
+    @staticmethod
+    def backward(ctx, grad: torch.Tensor):
+        g = grad.contiguous()
+        gin = torch.empty_like(g)
+        (bitmap,) = ctx.saved_tensors
+        B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gin.view(-1))
+        return gin, None
+
+
+def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None) -> torch.Tensor:
+    """ReLU through the fused kernel.  Pass the active ``stash_saved_activations`` context as ``hooks`` to let
+    the following layer reuse the stash for its saved input."""
+    return ReLUStash.apply(x, hooks)

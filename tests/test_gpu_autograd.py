@@ -1,0 +1,121 @@
+"""The stash inside PyTorch's autograd: saved activations are compressed between the passes, gradients are
+bit-identical to plain PyTorch (the codec is lossless), and the peak memory of a ReLU network drops."""
+import pytest
+import torch
+
+from paper_2110_15362_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def A():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    B.lib()
+    from paper_2110_15362_b200 import autograd
+    return autograd
+
+
+def mlp(width, depth, seed, dtype=torch.float32):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return [(torch.randn(width, width, generator=g, device="cuda", dtype=dtype) / width ** 0.5).requires_grad_()
+            for _ in range(depth)]
+
+
+def run(weights, x, relu, hooks=None):
+    h = x
+    for w in weights:
+        h = relu(h @ w)
+    loss = (h * h).sum()
+    loss.backward()
+    grads = [w.grad.clone() for w in weights]
+    for w in weights:
+        w.grad = None
+    return loss.detach().clone(), grads
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16, torch.float64])
+def test_gradients_are_bit_identical(A, dtype):
+    weights = mlp(512, 4, seed=1, dtype=dtype)
+    x = torch.randn(2048, 512, device="cuda", dtype=dtype, generator=torch.Generator(device="cuda").manual_seed(2))
+    ref_loss, ref = run(weights, x, torch.relu)
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        loss1, g1 = run(weights, x, torch.relu)
+        assert hooks.dense_bytes > 0 and hooks.packed_bytes < 0.7 * hooks.dense_bytes
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        loss2, g2 = run(weights, x, lambda t: A.relu_stash(t, hooks))
+    loss3, g3 = run(weights, x, A.relu_stash)                       # the fused ReLU alone, no hooks
+    for loss, grads in ((loss1, g1), (loss2, g2), (loss3, g3)):
+        assert torch.equal(loss, ref_loss)
+        for a, b in zip(grads, ref):
+            assert torch.equal(a, b)
+
+
+def test_pack_unpack_round_trip_and_skips(A):
+    hooks = A.stash_saved_activations(min_numel=1024)
+    t = torch.relu(torch.randn(64, 4096, device="cuda"))
+    p = hooks._pack(t)
+    assert isinstance(p, A.PackedActivation) and p.nnz == int(torch.count_nonzero(t))
+    assert p.values.numel() == p.nnz                                # exact-size storage
+    assert torch.equal(hooks._unpack(p).view(torch.int32), t.view(torch.int32))
+    assert hooks._pack(t) is p                                      # the same tensor object is packed once
+    dense = torch.randn(64, 4096, device="cuda")                   # no zeros: not worth a stash
+    assert hooks._pack(dense) is dense
+    small = torch.zeros(10, device="cuda")
+    assert hooks._pack(small) is small
+    param = torch.nn.Parameter(torch.zeros(1 << 16, device="cuda"))
+    assert hooks._pack(param) is param
+    cpu = torch.zeros(1 << 16)
+    assert hooks._pack(cpu) is cpu
+    view = torch.zeros(256, 512, device="cuda").t()                # not contiguous
+    assert hooks._pack(view) is view
+
+
+def test_conv_network_trains_and_matches(A):
+    torch.backends.cudnn.deterministic = True
+    g = torch.Generator(device="cuda").manual_seed(3)
+    w1 = (torch.randn(32, 3, 3, 3, generator=g, device="cuda") * 0.2).requires_grad_()
+    w2 = (torch.randn(64, 32, 3, 3, generator=g, device="cuda") * 0.05).requires_grad_()
+    x = torch.randn(16, 3, 64, 64, generator=g, device="cuda")
+
+    def step(relu):
+        h = relu(torch.nn.functional.conv2d(x, w1, padding=1))
+        h = torch.nn.functional.max_pool2d(h, 2)
+        h = relu(torch.nn.functional.conv2d(h, w2, padding=1))
+        h.square().mean().backward()
+        out = (w1.grad.clone(), w2.grad.clone())
+        w1.grad = w2.grad = None
+        return out
+
+    ref = step(torch.relu)
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        got = step(lambda t: A.relu_stash(t, hooks))
+        assert hooks.packed_bytes > 0
+    for a, b in zip(got, ref):
+        assert torch.equal(a, b)
+
+
+def test_peak_memory_drops(A):
+    width, depth, batch = 1024, 32, 16384                             # 64 MiB per fp32 activation, 2 GiB saved by plain PyTorch
+    weights = mlp(width, depth, seed=5)
+    x = torch.randn(batch, width, device="cuda", generator=torch.Generator(device="cuda").manual_seed(6))
+
+    def peak(fn):
+        torch.cuda.synchronize()
+        torch.cuda.empty_cache()
+        torch.cuda.reset_peak_memory_stats()
+        base = torch.cuda.memory_allocated()
+        fn()
+        torch.cuda.synchronize()
+        return torch.cuda.max_memory_allocated() - base
+
+    def plain():
+        run(weights, x, torch.relu)
+
+    def stashed():
+        with A.stash_saved_activations() as hooks:
+            run(weights, x, lambda t: A.relu_stash(t, hooks))
+
+    plain(); stashed()                                                # warm up allocator and cuBLAS workspaces
+    p0, p1 = peak(plain), peak(stashed)
+    assert p1 < 0.75 * p0, (p0, p1)
