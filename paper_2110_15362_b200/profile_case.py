@@ -1,6 +1,6 @@
 """One small, seeded invocation of a kernel, for profiler captures.
 
-    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|decompress|relu_bwd> \
+    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|prune|decompress|relu_bwd|mask|mask_y> \
            [--log2n 26] [--zeros 0.5] [--reps 3]
 
 runs `reps` repetitions of one entry point on a tensor of 2**log2n elements (default 2**26: 256 MiB of
@@ -25,8 +25,9 @@ from . import workloads as W
 
 def main(argv=None) -> int:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("dtype", choices=["f32", "f16", "bf16"])
-    ap.add_argument("op", choices=["compress", "relu", "relu_y", "decompress", "relu_bwd"])
+    ap.add_argument("dtype", choices=["f32", "f16", "bf16", "f64"])
+    ap.add_argument("op", choices=["compress", "relu", "relu_y", "prune", "decompress", "relu_bwd", "mask", "mask_y"])
+    ap.add_argument("--tau", type=float, default=0.1)
     ap.add_argument("--log2n", type=int, default=26)
     ap.add_argument("--zeros", type=float, default=0.5)
     ap.add_argument("--reps", type=int, default=3)
@@ -35,7 +36,9 @@ def main(argv=None) -> int:
     dev = torch.device("cuda")
     n = 1 << args.log2n
     if args.dtype == "f32":
-        x = W.cfg3_iid(n, args.zeros, 2, dev)
+        x = W.prune_preact(n, dev) if args.op == "prune" else W.cfg3_iid(n, args.zeros, 2, dev)
+    elif args.dtype == "f64":
+        x = W.cfg3_iid(n, args.zeros, 3, dev).double()
     else:
         x = torch.relu(W.cfg4_preact(0, (n,), args.dtype, dev))
     st = B.Stash(n, x.dtype, dev)
@@ -52,6 +55,12 @@ def main(argv=None) -> int:
             B.bt_relu_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
         elif args.op == "relu_y":
             B.bt_relu_fwd_compress(x, d, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif args.op == "prune":
+            B.bt_prune_fwd_compress(x, args.tau, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws,
+                                    st.dev_status)
+        elif args.op in ("mask", "mask_y"):
+            compress()
+            B.bt_mask_compress(x, st.bitmap, st.chunk_prefix, d if args.op == "mask_y" else None, st.values)
         elif args.op == "decompress":
             compress()
             B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, d)
