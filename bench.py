@@ -537,7 +537,7 @@ def run_ours(args):
             line["e2e"] = {"value": round(whole_job_value(step.dense_bytes_per_step, world, e2e_ms), 3),
                            "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": round(e2e_ms, 3), "steps": e2e["steps"],
-                           "api": "bt_*_host entry points, pinned host buffers"}
+                           "api": "bt_*_host entry points, pinned host buffers, %d host threads" % e2e["workers"]}
         if world == 1 and not args.no_large:
             line["large_tensor_kernels"] = large_tensor_kernels(dev, peak)
         if world == 1 and not args.no_cpu_baseline:
@@ -554,15 +554,20 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_e2e(step: Cfg2Step, graph, steps: int, world: int):
+def run_e2e(step: Cfg2Step, graph, steps: int, world: int, workers: int = int(os.environ.get("BT_E2E_WORKERS", "4"))):
     """The same step through the host-buffer entry points of the C ABI: every tensor the step consumes
     starts in pinned host memory and every tensor it produces (both stashes, the restored activation, the
-    input gradient) ends there; the host<->device copies happen inside the calls, inside the timed region."""
+    input gradient) ends there; the host<->device copies happen inside the calls, inside the timed region.
+
+    The calls are synchronous, so a few host threads (each with its own stream, staging area and output
+    buffers) work on different layers at once: one call's host->device copy overlaps another's
+    device->host copy and kernels.  All forward calls of a step finish before its backward calls start."""
+    import queue
+    from concurrent.futures import ThreadPoolExecutor
     import torch
     B = step.B
     dev = step.restored.device
     n_max = step.restored.numel()
-    staging = torch.empty(B.bt_host_staging_bytes(n_max, torch.float32), dtype=torch.uint8, device=dev)
     host = []
     h2d = d2h = 0
     for l in step.layers:
@@ -574,34 +579,60 @@ def run_e2e(step: Cfg2Step, graph, steps: int, world: int):
             h["prefix_" + tag] = torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory()
             h["nnz_" + tag] = torch.zeros(1, dtype=torch.int64).pin_memory()
         host.append(h)
-    out_restored = torch.empty(n_max, dtype=torch.float32).pin_memory()
-    out_gin = torch.empty(n_max, dtype=torch.float32).pin_memory()
     for l, z in zip(step.layers, step.nnz()):
         n = l["n"]
         comp = B.bt_compressed_bytes(n, z, torch.float32)
         h2d += 4 * n + 4 * n + comp + (4 * ((n + 31) // 32) + 4 * n)      # compress, fused forward, decompress, backward
         d2h += (comp + 8) + (comp + 8) + 4 * n + 4 * n
 
-    def one():
-        for l, h in zip(step.layers, host):
-            B.bt_compress_host(h["act"], h["bitmap_a"], h["values_a"], h["prefix_a"], h["nnz_a"], staging)
-            B.bt_relu_fwd_compress_host(h["pre"], None, h["bitmap_b"], h["values_b"], h["prefix_b"], h["nnz_b"], staging)
-        for l, h in zip(reversed(step.layers), reversed(host)):
-            n = l["n"]
-            B.bt_decompress_host(h["bitmap_a"], h["values_a"], h["prefix_a"], int(h["nnz_a"].item()),
-                                 out_restored[:n], staging)
-            B.bt_relu_bwd_from_bitmap_host(h["bitmap_b"], h["grad"], out_gin[:n], staging)
+    # per-thread resources, handed out through a queue
+    pool = queue.SimpleQueue()
+    for _ in range(workers):
+        pool.put(dict(stream=torch.cuda.Stream(device=dev),
+                      staging=torch.empty(B.bt_host_staging_bytes(n_max, torch.float32), dtype=torch.uint8, device=dev),
+                      restored=torch.empty(n_max, dtype=torch.float32).pin_memory(),
+                      gin=torch.empty(n_max, dtype=torch.float32).pin_memory()))
+    check = {}
 
-    one()
-    torch.cuda.synchronize()
-    assert torch.equal(out_restored[:step.layers[0]["n"]].view(torch.int32), host[0]["act"].view(torch.int32))
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
+    def call(task):
+        kind, i = task
+        r = pool.get()
+        try:
+            torch.cuda.set_device(dev)
+            h, s, n = host[i], r["stream"], step.layers[i]["n"]
+            if kind == "compress":
+                B.bt_compress_host(h["act"], h["bitmap_a"], h["values_a"], h["prefix_a"], h["nnz_a"], r["staging"], stream=s)
+            elif kind == "fused":
+                B.bt_relu_fwd_compress_host(h["pre"], None, h["bitmap_b"], h["values_b"], h["prefix_b"], h["nnz_b"],
+                                            r["staging"], stream=s)
+            elif kind == "decompress":
+                B.bt_decompress_host(h["bitmap_a"], h["values_a"], h["prefix_a"], int(h["nnz_a"].item()),
+                                     r["restored"][:n], r["staging"], stream=s)
+                if i == 0:
+                    check["ok"] = torch.equal(r["restored"][:n].view(torch.int32), h["act"].view(torch.int32))
+            else:
+                B.bt_relu_bwd_from_bitmap_host(h["bitmap_b"], h["grad"], r["gin"][:n], r["staging"], stream=s)
+        finally:
+            pool.put(r)
+
+    order = sorted(range(len(step.layers)), key=lambda i: -step.layers[i]["n"])     # large layers first
+    fwd = [(k, i) for i in order for k in ("compress", "fused")]
+    bwd = [(k, i) for i in order for k in ("decompress", "backward")]
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        def one():
+            list(ex.map(call, fwd))
+            list(ex.map(call, bwd))
         one()
-    e1.record()
-    torch.cuda.synchronize()
-    return {"ms": e0.elapsed_time(e1), "steps": steps, "h2d": h2d, "d2h": d2h}
+        torch.cuda.synchronize()
+        assert check.get("ok"), "end-to-end round trip is not bit exact"
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            one()
+        # every call has synchronised its own stream before returning; the closing event follows them all
+        e1.record()
+        torch.cuda.synchronize()
+    return {"ms": e0.elapsed_time(e1), "steps": steps, "h2d": h2d, "d2h": d2h, "workers": workers}
 
 
 def main():
