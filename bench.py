@@ -48,6 +48,9 @@ def parse_args():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-large", action="store_true", help="skip the per-kernel runs on 1 GiB tensors")
     p.add_argument("--no-e2e", action="store_true")
+    p.add_argument("--chains", type=int, choices=(1, 2, 4), default=2,
+                   help="independent chains of the step's graph: 2 = plain codec / fused pair on two streams, "
+                        "4 = each of them split into even and odd layers")
     return p.parse_args()
 
 
@@ -182,17 +185,28 @@ class Cfg2Step:
             grad = W.cfg2_grad(i, shape, dev).reshape(-1)
             self.layers.append(dict(n=n, pre=pre, act=act, grad=grad,
                                     stash_a=B.Stash(n, torch.float32, dev), stash_b=B.Stash(n, torch.float32, dev)))
-        self.restored = torch.empty(n_max, dtype=torch.float32, device=dev)
-        self.gin = torch.empty(n_max, dtype=torch.float32, device=dev)
-        self.ws = B.new_workspace(n_max, dev)
+        # one output buffer and one workspace per chain (at most four chains); chain 0 restores the activations
+        self.outs = [torch.empty(n_max, dtype=torch.float32, device=dev) for _ in range(4)]
+        self.wss = [B.new_workspace(n_max, dev) for _ in range(4)]
+        self.restored, self.gin, self.ws = self.outs[0], self.outs[1], self.wss[0]
         self.total_elems = sum(l["n"] for l in self.layers)
         self.dense_bytes_per_step = len(OPS) * 4 * self.total_elems
         self.launches_per_step = len(OPS) * len(self.layers)
 
-    def run(self, only_op=None, only_layer=None):
+    def run(self, only_op=None, only_layer=None, streams=None):
         """One step (forward over the layers, backward in reverse).  `only_op` / `only_layer` restrict it to
-        one operation and / or one layer, for the per-operation timing passes."""
+        one operation and / or one layer, for the per-operation timing passes.  With `streams` (a list of 2
+        or 4 streams, the first being the current one) the step runs as independent chains -- the plain codec
+        (compress ... decompress) and the fused pair (fused forward ... ReLU backward), each optionally split
+        into even and odd layers -- every chain with its own stream, workspace and output buffer, so that one
+        chain's launch latency hides behind another's kernels."""
         B = self.B
+        k = 1 if not streams else len(streams)
+
+        def chain(family, i):                       # family 0: plain codec, 1: fused pair
+            if k == 1:
+                return 0
+            return family if k == 2 else 2 * family + (i & 1)
 
         def want(op, i):
             return (only_op is None or op == only_op) and (only_layer is None or i == only_layer)
@@ -200,18 +214,25 @@ class Cfg2Step:
         for i, l in enumerate(self.layers):
             a, b = l["stash_a"], l["stash_b"]
             if want("bt_compress", i):
-                B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.ws, a.dev_status)
+                c = chain(0, i)
+                B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.wss[c], a.dev_status,
+                              stream=streams[c] if streams else None)
             if want("bt_relu_fwd_compress", i):
-                B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.ws,
-                                       b.dev_status)
+                c = chain(1, i)
+                B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.wss[c],
+                                       b.dev_status, stream=streams[c] if streams else None)
         for i in range(len(self.layers) - 1, -1, -1):
             l = self.layers[i]
             a, b = l["stash_a"], l["stash_b"]
             n = l["n"]
             if want("bt_decompress", i):
-                B.bt_decompress(a.bitmap, a.values, a.chunk_prefix, self.restored[:n])
+                c = chain(0, i)
+                B.bt_decompress(a.bitmap, a.values, a.chunk_prefix, self.outs[c if k > 1 else 0][:n],
+                                stream=streams[c] if streams else None)
             if want("bt_relu_bwd_from_bitmap", i):
-                B.bt_relu_bwd_from_bitmap(b.bitmap, l["grad"], self.gin[:n])
+                c = chain(1, i)
+                B.bt_relu_bwd_from_bitmap(b.bitmap, l["grad"], self.outs[c if k > 1 else 1][:n],
+                                          stream=streams[c] if streams else None)
 
     def check(self):
         """After a step: device status words are clean and both stashes of a layer agree."""
@@ -456,8 +477,17 @@ def run_ours(args):
 
     # the whole step as one CUDA graph: 68 kernel launches replayed without host work in between
     graph = torch.cuda.CUDAGraph()
+    branches = [torch.cuda.Stream() for _ in range(args.chains - 1)]
     with torch.cuda.graph(graph):
-        step.run()
+        if args.chains > 1:
+            main_stream = torch.cuda.current_stream()
+            for b in branches:
+                b.wait_stream(main_stream)               # fork
+            step.run(streams=[main_stream] + branches)
+            for b in branches:
+                main_stream.wait_stream(b)               # join
+        else:
+            step.run()
     for _ in range(max(args.warmup, 3)):
         graph.replay()
     torch.cuda.synchronize()
@@ -515,7 +545,11 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "batch": args.batch, "layers": len(step.layers),
                        "elements_per_step": step.total_elems, "zero_fraction": round(
                            1.0 - sum(nnz) / step.total_elems, 4),
-                       "ops_per_layer": list(OPS), "launch": "one CUDA graph per step",
+                       "ops_per_layer": list(OPS),
+                       "launch": "one CUDA graph per step" + (", %d independent chains on %d streams (plain codec / fused "
+                                                              "pair%s)" % (args.chains, args.chains, ", even / odd layers"
+                                                                           if args.chains == 4 else "")
+                                                              if args.chains > 1 else ""),
                        "l2": "per-step working set %.2f GB exceeds the 126 MB L2; no flush between steps"
                              % (7 * 4 * step.total_elems / 1e9),
                        "parallelism": "dp%d" % world if world > 1 else "single"},
