@@ -246,6 +246,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
     static_assert(kTile % BT_CHUNK_ELEMS == 0, "a tile holds whole chunks");
     static_assert(kWarps <= 32, "one lane per warp count");
+    // A scan warp makes tile j ready only in its turn for tile j + 2, after that tile has been counted, so
+    // tiles j, j + 1 and j + 2 must hold slots at once: three stages are the minimum that cannot deadlock,
+    // the fourth keeps the bulk copy of the next tile in flight.
     static_assert(kStages >= 4, "loading, compacting, awaiting its base, copying out");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
