@@ -8,15 +8,15 @@ from paper_2110_15362_b200 import binding as B
 from paper_2110_15362_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
-TDT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
+TDT = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16, "f64": torch.float64}
 
 
 def host_tensor(raw: np.ndarray, kind: str) -> torch.Tensor:
-    t = torch.from_numpy(raw.view({2: np.int16, 4: np.int32}[raw.dtype.itemsize]).copy()).view(TDT[kind])
+    t = torch.from_numpy(raw.view({2: np.int16, 4: np.int32, 8: np.int64}[raw.dtype.itemsize]).copy()).view(TDT[kind])
     return t.pin_memory()
 
 
-@pytest.mark.parametrize("kind", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("kind", ["f32", "bf16", "f16", "f64"])
 @pytest.mark.parametrize("n", [0, 1, 33, 4097, 8192 * 5 + 123, 200704])
 def test_host_round_trip_and_relu_pair(oracle, kind, n):
     assert torch.cuda.is_available()

@@ -19,7 +19,7 @@ def outputs(st: B.Stash):
     return (nnz, st.status, W.raw_numpy(st.bitmap), W.raw_numpy(st.chunk_prefix), W.raw_numpy(st.values[:nnz]))
 
 
-@pytest.mark.parametrize("kind", ["f32", "bf16"])
+@pytest.mark.parametrize("kind", ["f32", "bf16", "f64"])
 def test_noalloc_matches_bt_compress_on_two_calls_in_a_row(kind):
     assert torch.cuda.is_available()
     L = B.lib()
@@ -27,7 +27,7 @@ def test_noalloc_matches_bt_compress_on_two_calls_in_a_row(kind):
     sizes = (8192 * 37 + 4097 + 5, 200704)                    # second call smaller: stale scratch beyond it must not matter
     for call, n in enumerate(sizes):
         raw = W.random_patterns(n, kind, 0.5, seed=31337 + call)
-        x = torch.from_numpy(raw.view({2: np.int16, 4: np.int32}[raw.dtype.itemsize]).copy()).cuda().view(dt)
+        x = torch.from_numpy(raw.view({2: np.int16, 4: np.int32, 8: np.int64}[raw.dtype.itemsize]).copy()).cuda().view(dt)
         ref, got = B.Stash(n, dt), B.Stash(n, dt)
         B.bt_compress(x, ref.bitmap, ref.values, ref.chunk_prefix, ref.nnz_out, B.new_workspace(n), ref.dev_status)
         expect = outputs(ref)
