@@ -212,6 +212,34 @@ int bt_compress_noalloc(const void *dense, uint64_t n, int dtype,
                         int32_t *dev_status, void *stream);
 
 /*
+ * Arena forms (no counterpart in the paper; they serve a training loop that stashes one activation after
+ * another).  A stash needs exactly nnz values, but nnz is known only on the device; sizing a buffer from
+ * it costs a device-to-host read per tensor.  Here the caller owns one arena (a device buffer of
+ * arena_bytes bytes, 16-byte aligned) and one device word, *arena_cursor, holding the number of bytes in
+ * use (set it to 0, or back to an earlier value, with a device write in stream order).  A call reads the
+ * cursor c, writes its packed values at arena + c, and -- if all nnz values fit behind the cursor --
+ * stores c in *values_offset_out and advances the cursor to c + nnz * sizeof(dtype), rounded up to 16
+ * bytes.  If they do not fit, *dev_status = BT_ERR_CAPACITY, the cursor and *values_offset_out stay as
+ * they were, bitmap, chunk_prefix and *nnz_out are still complete.  For n == 0 the offset is the cursor
+ * and the cursor does not move.  Calls that share an arena must be ordered on the device (one stream, or
+ * events).  bt_prune_fwd_compress_arena with tau = 0 is the fused ReLU forward.  All other parameters as
+ * in bt_compress / bt_prune_fwd_compress / bt_decompress.
+ */
+int bt_compress_arena(const void *dense, uint64_t n, int dtype, uint32_t *bitmap,
+                      void *arena, uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offset_out,
+                      uint64_t *chunk_prefix, uint64_t *nnz_out,
+                      void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+int bt_prune_fwd_compress_arena(const void *x, uint64_t n, int dtype, float tau, void *y_out, uint32_t *bitmap,
+                                void *arena, uint64_t arena_bytes, uint64_t *arena_cursor,
+                                uint64_t *values_offset_out, uint64_t *chunk_prefix, uint64_t *nnz_out,
+                                void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+/* values_offset: the device word a *_arena compressor wrote (byte offset of the values inside the arena) */
+int bt_decompress_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
+                        const uint64_t *chunk_prefix, uint64_t n, int dtype, void *dense_out, void *stream);
+
+/*
  * Host-buffer forms.  The paper's own implementation keeps the stash in host
  * memory (section 4, "Implementation Details": std::bitset and std::vector);
  * these calls serve callers whose dense tensors or stashes live there.  Every

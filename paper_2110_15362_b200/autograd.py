@@ -14,7 +14,11 @@ Two pieces, both thin wrappers around the C-ABI calls (no arithmetic here):
   (``bt_relu_bwd_from_bitmap``).  Inside the context above its stash is shared with the next layer's saved
   input, so the activation is compressed once.
 
-Getting the exact ``nnz`` to size the values costs one device-to-host read per packed tensor.
+Getting the exact ``nnz`` to size the values costs one device-to-host read per packed tensor.  With
+``stash_saved_activations(arena_bytes=...)`` the values go instead behind a device-side cursor into one
+pre-allocated arena (the ``*_arena`` entry points): no host read in the forward pass; the device status
+words are checked once, when the backward pass first asks for a tensor.  The cursor is reset on entering
+the context, so one context entry covers one forward / backward pass.
 """
 from __future__ import annotations
 
@@ -29,13 +33,16 @@ __all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUSta
 
 
 class PackedActivation:
-    """What replaces a saved tensor: the stash and the metadata needed to rebuild it."""
+    """What replaces a saved tensor: the stash and the metadata needed to rebuild it.  `values` is either the
+    exact-size vector of values, or (arena mode) None with `arena`, `offset` (device word) and `owner` set."""
 
-    __slots__ = ("bitmap", "values", "chunk_prefix", "shape", "dtype", "device", "nnz", "__weakref__")
+    __slots__ = ("bitmap", "values", "chunk_prefix", "shape", "dtype", "device", "nnz", "arena", "offset", "owner",
+                 "__weakref__")
 
-    def __init__(self, bitmap, values, chunk_prefix, shape, dtype, device, nnz):
+    def __init__(self, bitmap, values, chunk_prefix, shape, dtype, device, nnz, arena=None, offset=None, owner=None):
         self.bitmap, self.values, self.chunk_prefix = bitmap, values, chunk_prefix
         self.shape, self.dtype, self.device, self.nnz = shape, dtype, device, nnz
+        self.arena, self.offset, self.owner = arena, offset, owner
 
     @property
     def numel(self) -> int:
@@ -45,11 +52,17 @@ class PackedActivation:
         return n
 
     def nbytes(self) -> int:
-        return B.bt_compressed_bytes(self.numel, self.nnz, self.dtype)
+        """Bytes of the stash (arena mode: reads nnz from the device)."""
+        nnz = int(self.nnz.item()) if isinstance(self.nnz, torch.Tensor) else self.nnz
+        return B.bt_compressed_bytes(self.numel, nnz, self.dtype)
 
     def unpack(self) -> torch.Tensor:
         out = torch.empty(self.shape, dtype=self.dtype, device=self.device)
-        B.bt_decompress(self.bitmap, self.values, self.chunk_prefix, out.view(-1))
+        if self.arena is not None:
+            self.owner.check_statuses()
+            B.bt_decompress_arena(self.bitmap, self.arena, self.offset, self.chunk_prefix, out.view(-1))
+        else:
+            B.bt_decompress(self.bitmap, self.values, self.chunk_prefix, out.view(-1))
         return out
 
 
@@ -95,11 +108,36 @@ def _compress(flat: torch.Tensor, scratch: _Scratch, relu_into: Optional[torch.T
     return bitmap, full[:nnz].clone(), prefix, nnz
 
 
-class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
-    """Context manager: saved activations are kept compressed between the forward and the backward pass."""
+def _compress_arena(flat: torch.Tensor, owner, relu_into: Optional[torch.Tensor] = None):
+    """Arena form of `_compress`: nothing is read back; returns bitmap, prefix, nnz word, offset word."""
+    n, dev = flat.numel(), flat.device
+    bitmap = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
+    prefix = torch.empty((n + B.CHUNK - 1) // B.CHUNK, dtype=torch.int64, device=dev)
+    words = torch.empty(2, dtype=torch.int64, device=dev)               # nnz, byte offset of the values
+    status = torch.empty(1, dtype=torch.int32, device=dev)
+    ws = owner.scratch.workspace(n, dev)
+    if relu_into is None:
+        B.bt_compress_arena(flat, bitmap, owner.arena, owner.cursor, words[1:], prefix, words[:1], ws, status, n=n)
+    else:
+        B.bt_prune_fwd_compress_arena(flat, 0.0, relu_into, bitmap, owner.arena, owner.cursor, words[1:], prefix,
+                                      words[:1], ws, status, n=n)
+    owner.statuses.append(status)
+    return bitmap, prefix, words[:1], words[1:]
 
-    def __init__(self, min_numel: int = 1 << 14, min_saving: float = 0.1):
+
+class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
+    """Context manager: saved activations are kept compressed between the forward and the backward pass.
+    `arena_bytes`: keep all values in one pre-allocated arena of that size behind a device-side cursor (no
+    host read per tensor; a RuntimeError at the first unpack if the arena was too small)."""
+
+    def __init__(self, min_numel: int = 1 << 14, min_saving: float = 0.1, arena_bytes: Optional[int] = None,
+                 device="cuda"):
         self.min_numel, self.min_saving = min_numel, min_saving
+        self.arena = self.cursor = None
+        self.statuses: list = []
+        if arena_bytes is not None:
+            self.arena = torch.empty((arena_bytes + 15) // 16 * 16, dtype=torch.uint8, device=device)
+            self.cursor = torch.zeros(1, dtype=torch.int64, device=device)
         self.scratch = _Scratch()
         self.packed_bytes = 0            # bytes kept in compressed form so far
         self.dense_bytes = 0             # bytes the same tensors would have taken
@@ -128,6 +166,15 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
         return (t.is_cuda and t.dtype in B.DTYPE_CODE and t.is_contiguous() and t.numel() >= self.min_numel
                 and not isinstance(t, torch.nn.Parameter) and not (t.requires_grad and t.is_leaf))
 
+    def check_statuses(self) -> None:
+        """Arena mode: one host read for all stashes made so far; raises if any did not fit."""
+        if self.statuses:
+            worst = int(torch.cat(self.statuses).max().item())
+            self.statuses.clear()
+            if worst != B.BT_OK:
+                raise RuntimeError("stash arena too small or a stash call failed: %s" %
+                                   B.BitTrainError("bt_*_arena", worst))
+
     def _pack(self, t: torch.Tensor):
         if not self._eligible(t):
             return t
@@ -135,6 +182,13 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
         if shared is not None:
             return shared
         n, es = t.numel(), t.element_size()
+        if self.arena is not None:
+            bitmap, prefix, nnz_word, off_word = _compress_arena(t.detach().view(-1), self)
+            packed = PackedActivation(bitmap, None, prefix, tuple(t.shape), t.dtype, t.device, nnz_word,
+                                      arena=self.arena, offset=off_word, owner=self)
+            self.share(t, packed)
+            self.dense_bytes += n * es
+            return packed
         bitmap, values, prefix, nnz = _compress(t.detach().view(-1), self.scratch)
         if B.bt_compressed_bytes(n, nnz, t.dtype) > (1.0 - self.min_saving) * n * es:
             return t                                  # too few zeros: the stash would not be smaller
@@ -149,6 +203,9 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
         return obj.unpack() if isinstance(obj, PackedActivation) else obj
 
     def __enter__(self):
+        if self.cursor is not None:
+            self.cursor.zero_()                 # a new pass: the arena is empty again
+            self.statuses.clear()
         super().__enter__()
         return self
 
@@ -164,6 +221,13 @@ class ReLUStash(torch.autograd.Function):
     def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None):
         xc = x.contiguous()
         y = torch.empty_like(xc)
+        if hooks is not None and hooks.arena is not None:
+            bitmap, prefix, nnz_word, off_word = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1))
+            ctx.save_for_backward(bitmap)
+            hooks.share(y, PackedActivation(bitmap, None, prefix, tuple(y.shape), y.dtype, y.device, nnz_word,
+                                            arena=hooks.arena, offset=off_word, owner=hooks))
+            hooks.dense_bytes += y.numel() * y.element_size()
+            return y
         scratch = hooks.scratch if hooks is not None else _Scratch()
         bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1))
         ctx.save_for_backward(bitmap)     # released with the graph, like any saved tensor

@@ -27,7 +27,8 @@ DTYPE_CODE = {torch.float32: BT_F32, torch.float16: BT_F16, torch.bfloat16: BT_B
 EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
-           "bt_prune_fwd_compress", "bt_mask_compress")
+           "bt_prune_fwd_compress", "bt_mask_compress", "bt_compress_arena", "bt_prune_fwd_compress_arena",
+           "bt_decompress_arena")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -69,6 +70,12 @@ def lib() -> ctypes.CDLL:
         L.bt_prune_fwd_compress.restype = i32
         L.bt_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp, u64, vp]
         L.bt_mask_compress.restype = i32
+        L.bt_compress_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.bt_compress_arena.restype = i32
+        L.bt_prune_fwd_compress_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.bt_prune_fwd_compress_arena.restype = i32
+        L.bt_decompress_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
+        L.bt_decompress_arena.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -172,6 +179,41 @@ def bt_mask_compress(x: torch.Tensor, mask_bitmap: torch.Tensor, mask_chunk_pref
     st = lib().bt_mask_compress(_ptr(x), n, DTYPE_CODE[x.dtype], _ptr(mask_bitmap), _ptr(mask_chunk_prefix),
                                 _ptr(y_out), _ptr(values), cap, _stream(stream))
     return _check("bt_mask_compress", st, check)
+
+
+def bt_compress_arena(dense: torch.Tensor, bitmap: torch.Tensor, arena: torch.Tensor, arena_cursor: torch.Tensor,
+                      values_offset_out: torch.Tensor, chunk_prefix: torch.Tensor, nnz_out: torch.Tensor,
+                      workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None, *, n: Optional[int] = None,
+                      stream=None, check: bool = True) -> int:
+    """bt_compress whose values go behind the cursor of a caller-owned arena (a uint8 device tensor)."""
+    n = dense.numel() if n is None else n
+    st = lib().bt_compress_arena(_ptr(dense), n, DTYPE_CODE[dense.dtype], _ptr(bitmap), _ptr(arena), _nbytes(arena),
+                                 _ptr(arena_cursor), _ptr(values_offset_out), _ptr(chunk_prefix), _ptr(nnz_out),
+                                 _ptr(workspace), _nbytes(workspace), _ptr(dev_status), _stream(stream))
+    return _check("bt_compress_arena", st, check)
+
+
+def bt_prune_fwd_compress_arena(x: torch.Tensor, tau: float, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
+                                arena: torch.Tensor, arena_cursor: torch.Tensor, values_offset_out: torch.Tensor,
+                                chunk_prefix: torch.Tensor, nnz_out: torch.Tensor, workspace: torch.Tensor,
+                                dev_status: Optional[torch.Tensor] = None, *, n: Optional[int] = None, stream=None,
+                                check: bool = True) -> int:
+    """Fused forward (tau = 0: ReLU) whose values go behind the cursor of a caller-owned arena."""
+    n = x.numel() if n is None else n
+    st = lib().bt_prune_fwd_compress_arena(_ptr(x), n, DTYPE_CODE[x.dtype], ctypes.c_float(tau), _ptr(y_out),
+                                           _ptr(bitmap), _ptr(arena), _nbytes(arena), _ptr(arena_cursor),
+                                           _ptr(values_offset_out), _ptr(chunk_prefix), _ptr(nnz_out),
+                                           _ptr(workspace), _nbytes(workspace), _ptr(dev_status), _stream(stream))
+    return _check("bt_prune_fwd_compress_arena", st, check)
+
+
+def bt_decompress_arena(bitmap: torch.Tensor, arena: torch.Tensor, values_offset: torch.Tensor,
+                        chunk_prefix: torch.Tensor, dense_out: torch.Tensor, *, n: Optional[int] = None, stream=None,
+                        check: bool = True) -> int:
+    n = dense_out.numel() if n is None else n
+    st = lib().bt_decompress_arena(_ptr(bitmap), _ptr(arena), _ptr(values_offset), _ptr(chunk_prefix), n,
+                                   DTYPE_CODE[dense_out.dtype], _ptr(dense_out), _stream(stream))
+    return _check("bt_decompress_arena", st, check)
 
 
 def bt_decompress(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor, dense_out: torch.Tensor,

@@ -18,15 +18,27 @@ inline bool aligned(const void *p, uintptr_t a) { return (reinterpret_cast<uintp
 
 inline uint64_t ceil_div(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
 
+struct Arena {
+    uint64_t *cursor     = nullptr;   // device word: bytes of the arena in use
+    uint64_t *offset_out = nullptr;   // device word: receives the byte offset of this call's values
+    uint64_t  bytes      = 0;
+};
+
 int compress_common(const void *src, uint64_t n, int dtype, bool relu, float tau, void *y, uint32_t *bitmap, void *values,
                     uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
-                    size_t workspace_bytes, int32_t *dev_status, void *stream)
+                    size_t workspace_bytes, int32_t *dev_status, void *stream, const Arena &arena = Arena())
 {
     if (elem_size_of(dtype) == 0) return BT_ERR_DTYPE;
     if (!nnz_out) return BT_ERR_NULL;
     if (!aligned(nnz_out, 8) || !aligned(dev_status, 4)) return BT_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (arena.cursor && (!arena.offset_out || !aligned(arena.cursor, 8) || !aligned(arena.offset_out, 8)))
+        return arena.offset_out ? BT_ERR_ALIGN : BT_ERR_NULL;
     if (n == 0) {
+        // nothing is pushed: the values of an empty tensor start where the cursor stands
+        if (arena.cursor &&
+            cudaMemcpyAsync(arena.offset_out, arena.cursor, sizeof(uint64_t), cudaMemcpyDeviceToDevice, s) != cudaSuccess)
+            return BT_ERR_CUDA;
         if (cudaMemsetAsync(nnz_out, 0, sizeof(uint64_t), s) != cudaSuccess) return BT_ERR_CUDA;
         if (dev_status && cudaMemsetAsync(dev_status, 0, sizeof(int32_t), s) != cudaSuccess) return BT_ERR_CUDA;
         return BT_OK;
@@ -51,6 +63,9 @@ int compress_common(const void *src, uint64_t n, int dtype, bool relu, float tau
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
     a.tau        = tau;
+    a.arena_cursor      = arena.cursor;
+    a.values_offset_out = arena.offset_out;
+    a.arena_bytes       = arena.bytes;
     a.n          = n;
     return bt::launch_compress(a, dtype, relu, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
@@ -95,6 +110,45 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
                            workspace, workspace_bytes, dev_status, stream);
 }
 
+int bt_compress_arena(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void *arena, uint64_t arena_bytes,
+                      uint64_t *arena_cursor, uint64_t *values_offset_out, uint64_t *chunk_prefix, uint64_t *nnz_out,
+                      void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    if (!arena_cursor) return BT_ERR_NULL;
+    Arena ar;
+    ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
+    return compress_common(dense, n, dtype, false, 0.0f, nullptr, bitmap, arena, arena_bytes, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream, ar);
+}
+
+int bt_prune_fwd_compress_arena(const void *x, uint64_t n, int dtype, float tau, void *y_out, uint32_t *bitmap, void *arena,
+                                uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offset_out,
+                                uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace, size_t workspace_bytes,
+                                int32_t *dev_status, void *stream)
+{
+    if (!arena_cursor) return BT_ERR_NULL;
+    Arena ar;
+    ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
+    return compress_common(x, n, dtype, true, tau, y_out, bitmap, arena, arena_bytes, chunk_prefix, nnz_out, workspace,
+                           workspace_bytes, dev_status, stream, ar);
+}
+
+int bt_decompress_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
+                        const uint64_t *chunk_prefix, uint64_t n, int dtype, void *dense_out, void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !chunk_prefix || !dense_out || !arena || !values_offset) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
+        !aligned(dense_out, 16))
+        return BT_ERR_ALIGN;
+    return bt::launch_decompress(bitmap, arena, values_offset, chunk_prefix, n, es, dense_out,
+                                 static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
 int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix, uint64_t n, int dtype,
                   void *dense_out, void *stream)
 {
@@ -105,7 +159,7 @@ int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *ch
     if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
         return BT_ERR_ALIGN;
     // values may be NULL only when the bitmap has no set bit; the kernel then never reads it
-    return bt::launch_decompress(bitmap, values, chunk_prefix, n, es, dense_out, static_cast<cudaStream_t>(stream)) ==
+    return bt::launch_decompress(bitmap, values, nullptr, chunk_prefix, n, es, dense_out, static_cast<cudaStream_t>(stream)) ==
                    cudaSuccess
                ? BT_OK
                : BT_ERR_CUDA;

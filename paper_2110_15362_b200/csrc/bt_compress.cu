@@ -264,6 +264,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
     __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
     __shared__ volatile uint32_t s_abort;
+    __shared__ uint64_t          s_arena_c0;               // arena forms: the cursor as this launch found it
 
     const uint32_t tid  = threadIdx.x;
     const uint32_t lane = tid & 31u;
@@ -286,7 +287,10 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     auto tile_of = [&](uint32_t it) { return cta + static_cast<uint64_t>(it) * G; };
 
     if (tid == 0) {
-        s_abort = 0;
+        // Read before the barrier below: the kernel's one update of the cursor follows the last tile's base,
+        // which needs a publication from every CTA, and a CTA publishes only after this barrier.
+        s_arena_c0 = a.arena_cursor ? *reinterpret_cast<const volatile uint64_t *>(a.arena_cursor) : 0;
+        s_abort    = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&s_full[s], 1);
             mbar_init(&s_counted[s], kWarps);
@@ -471,8 +475,18 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                     *a.nnz_out = nnz;
                     __threadfence();
                     const bool aborted = ld_relaxed_u32(abort_flag) != 0;
+                    uint64_t capacity = a.capacity;
+                    if (a.arena_cursor) {
+                        // arena form: the room left behind the cursor; the cursor moves only when everything fitted
+                        const uint64_t c0 = s_arena_c0;
+                        capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(U) : 0;
+                        if (!aborted && nnz <= capacity) {
+                            *a.values_offset_out = c0;
+                            *a.arena_cursor      = c0 + ((nnz * sizeof(U) + 15) & ~15ull);
+                        }
+                    }
                     if (a.dev_status)
-                        *a.dev_status = aborted ? BT_ERR_TIMEOUT : (nnz > a.capacity ? BT_ERR_CAPACITY : BT_OK);
+                        *a.dev_status = aborted ? BT_ERR_TIMEOUT : (nnz > capacity ? BT_ERR_CAPACITY : BT_OK);
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -503,8 +517,13 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     if (warp >= kFirstCopier) {
         // ------------------------------------------------------------ copier warps
         const uint32_t copier   = warp - kFirstCopier;
-        U *const       vals     = static_cast<U *>(a.values);
-        const uint64_t capacity = a.capacity;
+        U             *vals     = static_cast<U *>(a.values);
+        uint64_t       capacity = a.capacity;
+        if (a.arena_cursor) {
+            const uint64_t c0 = s_arena_c0;
+            vals              = reinterpret_cast<U *>(static_cast<unsigned char *>(a.values) + c0);
+            capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(U) : 0;
+        }
         for (uint32_t it = 0;; ++it) {
             if (tile_of(it) >= num_tiles) break;
             const uint32_t s = it % kStages;

@@ -23,8 +23,9 @@ constexpr uint32_t kFull = 0xFFFFFFFFu;
 // kE: elements a lane decodes per step (a multiple of one 16-byte vector: 2 for 8-byte, 4 for 4-byte, 8 for 2-byte elements)
 template <typename U, int kE, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
-decompress_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values,
-                  const uint64_t *__restrict__ prefix, const uint64_t n, U *__restrict__ out)
+decompress_kernel(const uint32_t *__restrict__ bitmap, const U *values,
+                  const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
+                  U *__restrict__ out)
 {
     constexpr int kVec          = 16 / sizeof(U);          // elements per 16-byte store
     constexpr int kLanesPerWord = 32 / kE;                 // lanes that share one bitmap word
@@ -52,6 +53,8 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ val
         if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
     }
     const uint64_t chunk_base = prefix[chunk];
+    // arena form: the packed values start *values_offset bytes into `values`
+    if (values_offset) values = reinterpret_cast<const U *>(reinterpret_cast<const unsigned char *>(values) + *values_offset);
 
     // non-zeros of the chunk in front of this quarter
     uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
@@ -121,31 +124,31 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ val
 }
 
 template <typename U, int kE>
-cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *prefix, uint64_t n, void *out,
-                         cudaStream_t stream)
+cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
+                         const uint64_t *prefix, uint64_t n, void *out, cudaStream_t stream)
 {
     constexpr int  kWarps   = 8;
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     decompress_kernel<U, kE, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
-        bitmap, static_cast<const U *>(values), prefix, n, static_cast<U *>(out));
+        bitmap, static_cast<const U *>(values), values_offset, prefix, n, static_cast<U *>(out));
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *prefix, uint64_t n,
-                              int elem_size, void *out, cudaStream_t stream)
+cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
+                              const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t stream)
 {
 #ifdef BT_DECOMP_E32
     constexpr int kE32 = BT_DECOMP_E32, kE16 = BT_DECOMP_E16;
 #else
     constexpr int kE32 = 4, kE16 = 8;
 #endif
-    if (elem_size == 8) return launch_typed<uint64_t, 2>(bitmap, values, prefix, n, out, stream);
-    return elem_size == 4 ? launch_typed<uint32_t, kE32>(bitmap, values, prefix, n, out, stream)
-                          : launch_typed<uint16_t, kE16>(bitmap, values, prefix, n, out, stream);
+    if (elem_size == 8) return launch_typed<uint64_t, 2>(bitmap, values, values_offset, prefix, n, out, stream);
+    return elem_size == 4 ? launch_typed<uint32_t, kE32>(bitmap, values, values_offset, prefix, n, out, stream)
+                          : launch_typed<uint16_t, kE16>(bitmap, values, values_offset, prefix, n, out, stream);
 }
 
 }  // namespace bt

@@ -32,12 +32,19 @@ struct CompressArgs {
     uint64_t   *ws_desc;    // wave totals, then tile descriptors
     uint32_t    ws_waves;   // number of wave totals
     float       tau;        // fused forms: elements <= tau become +0 (0 for plain ReLU)
+    // arena forms: `values` is the arena's base, the packed values go to values + *arena_cursor (bytes);
+    // on success the kernel stores the old cursor in *values_offset_out and advances the cursor past the
+    // values (rounded up to 16 bytes).  All three are NULL / 0 for the plain forms.
+    uint64_t   *arena_cursor;
+    uint64_t   *values_offset_out;
+    uint64_t    arena_bytes;
     uint64_t    n;
 };
 
 cudaError_t launch_compress(const CompressArgs &a, int dtype, bool relu, cudaStream_t s);
-cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *prefix,
-                              uint64_t n, int elem_size, void *out, cudaStream_t s);
+// values_offset: NULL, or a device word holding the byte offset of the packed values inside `values`
+cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
+                              const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t s);
 cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,
                                int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t s);
 cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size,

@@ -78,6 +78,7 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(scratch) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
     a.tau        = 0.0f;
+    a.arena_cursor = nullptr, a.values_offset_out = nullptr, a.arena_bytes = 0;
     a.n          = n;
     // the launcher clears the part of the scratch this call uses (it keeps the last call's contents otherwise)
     return bt::launch_compress(a, dtype, false, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;

@@ -119,3 +119,25 @@ def test_peak_memory_drops(A):
     plain(); stashed()                                                # warm up allocator and cuBLAS workspaces
     p0, p1 = peak(plain), peak(stashed)
     assert p1 < 0.75 * p0, (p0, p1)
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_arena_mode_matches_and_reports_overflow(A, fused):
+    weights = mlp(512, 4, seed=7)
+    x = torch.randn(4096, 512, device="cuda", generator=torch.Generator(device="cuda").manual_seed(8))
+    ref_loss, ref = run(weights, x, torch.relu)
+    hooks = A.stash_saved_activations(min_numel=1024, arena_bytes=64 << 20)
+    for _ in range(2):                                               # the arena is reused pass after pass
+        with hooks:
+            loss, grads = run(weights, x, (lambda t: A.relu_stash(t, hooks)) if fused else torch.relu)
+        assert torch.equal(loss, ref_loss)
+        for a, b in zip(grads, ref):
+            assert torch.equal(a, b)
+        used = int(hooks.cursor.item())
+        assert 0 < used < 0.7 * hooks.dense_bytes / 2 + (1 << 20) or used < hooks.dense_bytes
+    small = A.stash_saved_activations(min_numel=1024, arena_bytes=1 << 20)        # far too small
+    with pytest.raises(RuntimeError, match="arena too small"):
+        with small:
+            run(weights, x, torch.relu)
+    for w in weights:
+        w.grad = None
