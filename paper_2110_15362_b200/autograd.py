@@ -218,9 +218,13 @@ class ReLUStash(torch.autograd.Function):
     """ReLU with the stash fused into its forward pass; the backward pass reads only the bitmap."""
 
     @staticmethod
-    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None):
-        xc = x.contiguous()
-        y = torch.empty_like(xc)
+    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False):
+        if inplace and x.is_contiguous():
+            xc = y = x                   # the kernel may write the activation over its input
+            ctx.mark_dirty(x)
+        else:
+            xc = x.contiguous()
+            y = torch.empty_like(xc)
         if hooks is not None and hooks.arena is not None:
             bitmap, prefix, nnz_word, off_word = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1))
             ctx.save_for_backward(bitmap)
@@ -245,10 +249,11 @@ class ReLUStash(torch.autograd.Function):
         gin = torch.empty_like(g)
         (bitmap,) = ctx.saved_tensors
         B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gin.view(-1))
-        return gin, None
+        return gin, None, None
 
 
-def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None) -> torch.Tensor:
+def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False) -> torch.Tensor:
     """ReLU through the fused kernel.  Pass the active ``stash_saved_activations`` context as ``hooks`` to let
-    the following layer reuse the stash for its saved input."""
-    return ReLUStash.apply(x, hooks)
+    the following layer reuse the stash for its saved input.  ``inplace=True`` writes the activation over ``x``
+    (like ``torch.relu_``: only where ``x`` is not needed again, e.g. the output of a convolution)."""
+    return ReLUStash.apply(x, hooks, inplace)

@@ -141,3 +141,24 @@ def test_arena_mode_matches_and_reports_overflow(A, fused):
             run(weights, x, torch.relu)
     for w in weights:
         w.grad = None
+
+
+def test_inplace_relu_stash_matches(A):
+    weights = mlp(256, 3, seed=9)
+    x = torch.randn(1024, 256, device="cuda", generator=torch.Generator(device="cuda").manual_seed(10))
+    ref_loss, ref = run(weights, x, torch.relu)
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        loss, grads = run(weights, x, lambda t: A.relu_stash(t, hooks, inplace=True))
+    assert torch.equal(loss, ref_loss)
+    for a, b in zip(grads, ref):
+        assert torch.equal(a, b)
+
+
+def test_vgg_demo_runs_and_losses_agree(A, capsys):
+    import json
+    from paper_2110_15362_b200 import demo_vgg_step
+    assert demo_vgg_step.main(["--batch", "2", "--size", "64", "--arena-gib", "0.25"]) == 0
+    out = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
+    assert out["plain"]["loss"] == pytest.approx(out["stashed"]["loss"], rel=1e-3)
+    assert out["plain"]["loss"] == pytest.approx(out["stashed_arena"]["loss"], rel=1e-3)
+    assert 0.3 < out["saved_activation_bytes_over_dense"] < 0.8
