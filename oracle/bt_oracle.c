@@ -253,6 +253,98 @@ uint64_t oracle_mask_compress(const void *x, uint64_t n, int elem_size,
     return j;
 }
 
+/* Compare an element with 6 after exact widening: sets *ge6 (x >= 6) and *lt6
+ * (x < 6); both are 0 for a NaN. */
+static void cmp_six(const unsigned char *e, int kind, int *ge6, int *lt6)
+{
+    double d = 0.0;
+    switch (kind) {
+    case ORACLE_F32: { float f; memcpy(&f, e, 4); d = (double)f; break; }
+    case ORACLE_F64: { memcpy(&d, e, 8); break; }
+    case ORACLE_F16: { uint16_t h; memcpy(&h, e, 2); d = (double)oracle_half_to_float(h); break; }
+    case ORACLE_BF16: {
+        uint16_t h; memcpy(&h, e, 2);
+        uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4); d = (double)f; break;
+    }
+    default: break;
+    }
+    *ge6 = d >= 6.0;
+    *lt6 = d < 6.0;
+}
+
+/* the value 6 in the element type (exact in all four) */
+static void six_pattern(int kind, unsigned char *out)
+{
+    switch (kind) {
+    case ORACLE_F32: { float f = 6.0f; memcpy(out, &f, 4); break; }
+    case ORACLE_F64: { double d = 6.0; memcpy(out, &d, 8); break; }
+    case ORACLE_F16: { uint16_t h = 0x4600; memcpy(out, &h, 2); break; }     /* 1.5 * 2^2 */
+    case ORACLE_BF16: { uint16_t h = 0x40C0; memcpy(out, &h, 2); break; }    /* top half of 0x40C00000 */
+    default: break;
+    }
+}
+
+/* ReLU6 (the activation of the MobileNetV2 family among the paper's models)
+ * joined to the stash: y = (x <= 0) ? +0 : (x >= 6 ? 6 : x); a NaN fails both
+ * comparisons and is kept.  Then Algorithm 1 on y. */
+uint64_t oracle_relu6_fwd_compress(const void *pre_act, uint64_t n, int kind,
+                                   void *y, uint32_t *bitmap, void *values,
+                                   uint64_t *prefix)
+{
+    int elem_size = oracle_elem_size(kind);
+    const unsigned char *src = (const unsigned char *)pre_act;
+    unsigned char *yo = (unsigned char *)y;
+    unsigned char *val = (unsigned char *)values;
+    uint64_t words = (n + 31) / 32;
+    uint64_t j = 0;
+    unsigned char act[8];
+
+    for (uint64_t w = 0; w < words; ++w) bitmap[w] = 0;
+
+    for (uint64_t i = 0; i < n; ++i) {
+        if (i % CHUNK_ELEMS == 0) prefix[i / CHUNK_ELEMS] = j;
+        const unsigned char *e = src + i * (uint64_t)elem_size;
+        int ge6, lt6;
+        cmp_six(e, kind, &ge6, &lt6);
+        if (le_zero(e, kind)) memset(act, 0, (size_t)elem_size);
+        else if (ge6)         six_pattern(kind, act);
+        else                  memcpy(act, e, (size_t)elem_size);
+        if (yo) memcpy(yo + i * (uint64_t)elem_size, act, (size_t)elem_size);
+        if (!all_bytes_zero(act, elem_size)) {
+            memcpy(val + j * (uint64_t)elem_size, act, (size_t)elem_size);
+            j += 1;
+            bitmap[i >> 5] |= (uint32_t)1 << (i & 31);
+        }
+    }
+    return j;
+}
+
+/* ReLU6 backward from the stash: the gradient passes where 0 < x < 6, i.e.
+ * where the bit is set and the stashed activation is below 6 (a stashed 6 is a
+ * saturated unit, a stashed NaN compares false); a select, as for ReLU.  Walks
+ * the values with the single running counter of Algorithm 2. */
+void oracle_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values,
+                                 uint64_t n, int kind, const void *grad_out,
+                                 void *grad_in)
+{
+    int elem_size = oracle_elem_size(kind);
+    const unsigned char *val = (const unsigned char *)values;
+    const unsigned char *g = (const unsigned char *)grad_out;
+    unsigned char *o = (unsigned char *)grad_in;
+    uint64_t j = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        int pass = 0;
+        if ((bitmap[i >> 5] >> (i & 31)) & 1u) {
+            int ge6, lt6;
+            cmp_six(val + j * (uint64_t)elem_size, kind, &ge6, &lt6);
+            pass = lt6;
+            j += 1;
+        }
+        if (pass) memmove(o + i * (uint64_t)elem_size, g + i * (uint64_t)elem_size, (size_t)elem_size);
+        else      memset(o + i * (uint64_t)elem_size, 0, (size_t)elem_size);
+    }
+}
+
 /* The ReLU gradient needs only the bitmap: a select, not a multiply, so that a
  * masked lane is +0 whatever the upstream gradient holds (-x, inf, NaN). */
 void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,

@@ -67,6 +67,17 @@ uint64_t oracle_prune_fwd_compress(const void *x, uint64_t n, int kind, float ta
 uint64_t oracle_mask_compress(const void *x, uint64_t n, int elem_size,
                               const uint32_t *mask_bitmap, void *y, void *values);
 
+/* ReLU6 joined to the stash: y = (x <= 0) ? +0 : (x >= 6 ? 6 : x), NaN kept, then
+ * Algorithm 1 on y.  y may be NULL.  Returns nnz. */
+uint64_t oracle_relu6_fwd_compress(const void *pre_act, uint64_t n, int kind,
+                                   void *y, uint32_t *bitmap, void *values,
+                                   uint64_t *prefix);
+
+/* ReLU6 backward: grad_in[i] = (bit i set and its stashed value < 6) ? grad_out[i] : +0 */
+void oracle_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values,
+                                 uint64_t n, int kind, const void *grad_out,
+                                 void *grad_in);
+
 /* grad_in[i] = bit i ? grad_out[i] (raw copy) : +0 */
 void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
                                  uint64_t n, int elem_size, void *grad_in);

@@ -59,6 +59,10 @@ def lib() -> ctypes.CDLL:
         L.oracle_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, vp]
         L.oracle_mask_compress.restype = u64
         L.oracle_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp]
+        L.oracle_relu6_fwd_compress.restype = u64
+        L.oracle_relu6_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp]
+        L.oracle_relu6_bwd_from_stash.restype = None
+        L.oracle_relu6_bwd_from_stash.argtypes = [vp, vp, u64, i32, vp, vp]
         L.oracle_relu_bwd_from_bitmap.restype = None
         L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
         L.oracle_compressed_bytes.restype = u64
@@ -147,6 +151,30 @@ def mask_compress(x: np.ndarray, mask_bitmap: np.ndarray, want_y: bool = True):
     values = np.empty(n, dtype=xr.dtype)
     cnt = int(lib().oracle_mask_compress(_ptr(xr), n, xr.dtype.itemsize, _ptr(bm), _ptr(y), _ptr(values)))
     return y, values[:cnt].copy()
+
+
+def relu6_fwd_compress(pre_act: np.ndarray, kind: str, want_y: bool = True):
+    """ReLU6 joined to the stash.  Returns (y or None, Compressed)."""
+    x = _raw(pre_act)
+    assert x.dtype.itemsize == ELEM_SIZE[kind]
+    n = x.size
+    y = np.empty(n, dtype=x.dtype) if want_y else None
+    bitmap = np.full((n + 31) // 32, 0xDEADBEEF, dtype=np.uint32)
+    values = np.empty(n, dtype=x.dtype)
+    prefix = np.full((n + CHUNK - 1) // CHUNK, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64)
+    nnz = int(lib().oracle_relu6_fwd_compress(_ptr(x), n, KINDS[kind], _ptr(y), _ptr(bitmap), _ptr(values),
+                                               _ptr(prefix)))
+    return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
+
+
+def relu6_bwd_from_stash(c: Compressed, kind: str, grad_out: np.ndarray) -> np.ndarray:
+    g = _raw(grad_out)
+    assert g.size == c.n and g.dtype.itemsize == ELEM_SIZE[kind]
+    out = np.empty_like(g)
+    bm = np.ascontiguousarray(c.bitmap, dtype=np.uint32)
+    vals = np.ascontiguousarray(c.values)
+    lib().oracle_relu6_bwd_from_stash(_ptr(bm), _ptr(vals), c.n, KINDS[kind], _ptr(g), _ptr(out))
+    return out
 
 
 def relu_bwd_from_bitmap(bitmap: np.ndarray, grad_out: np.ndarray) -> np.ndarray:

@@ -34,6 +34,8 @@ MUTANTS = {
                                "if (((mask_bitmap[i >> 5] >> (i & 31)) & 1u) && !all_bytes_zero(e, elem_size)) {\n            memcpy(val"),
     "mask_msb_first": ("if ((mask_bitmap[i >> 5] >> (i & 31)) & 1u) {\n            memcpy(val",
                        "if ((mask_bitmap[i >> 5] >> (31 - (i & 31))) & 1u) {\n            memcpy(val"),
+    "relu6_never_saturates": ("else if (ge6)         six_pattern(kind, act);", "else if (ge6 && 0)    six_pattern(kind, act);"),
+    "relu6_bwd_passes_saturated_units": ("            pass = lt6;\n", "            pass = 1;\n"),
     "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
     "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
 }
@@ -57,6 +59,9 @@ def build_mutant(tmp_path, name):
     L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
     L.oracle_prune_fwd_compress.restype = u64
     L.oracle_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, vp]
+    L.oracle_relu6_fwd_compress.restype = u64
+    L.oracle_relu6_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp]
+    L.oracle_relu6_bwd_from_stash.argtypes = [vp, vp, u64, i32, vp, vp]
     L.oracle_mask_compress.restype = u64
     L.oracle_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp]
     L.oracle_compressed_bytes.restype = u64
@@ -119,6 +124,18 @@ def pins_hold(L) -> bool:
     vm = np.zeros(n, np.uint32)
     cnt = L.oracle_mask_compress(p(x), n, 4, p(mbm), p(ym), p(vm))
     if cnt != int(mask.sum()) or not np.array_equal(vm[:cnt], x[mask]) or not np.array_equal(ym, np.where(mask, x, 0)):
+        return False
+    # ReLU6 pair against torch
+    t6 = torch.randn(n, generator=torch.Generator().manual_seed(6)) * 4
+    t6[:3] = torch.tensor([6.0, 7.5, 0.0])
+    y6 = np.empty(n, np.uint32)
+    nnz6 = L.oracle_relu6_fwd_compress(p(W.raw_numpy(t6)), n, 0, p(y6), p(bitmap), p(values), p(prefix))
+    if not np.array_equal(y6, W.raw_numpy(torch.nn.functional.relu6(t6) + 0.0)):
+        return False
+    g6 = torch.randn(n, generator=torch.Generator().manual_seed(7))
+    gin6 = np.empty(n, np.uint32)
+    L.oracle_relu6_bwd_from_stash(p(bitmap), p(values[:nnz6].copy()), n, 0, p(W.raw_numpy(g6)), p(gin6))
+    if not np.array_equal(gin6, W.raw_numpy(torch.where((t6 > 0) & (t6 < 6), g6, torch.zeros(())))):
         return False
     # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
     if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
