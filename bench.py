@@ -350,6 +350,13 @@ def large_tensor_kernels(dev, peak_gbs: float):
         res["bt_relu_fwd_compress+y"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, es, True))
         ms, best = time_call(lambda: B.bt_relu_bwd_from_bitmap(st.bitmap, x, dense))
         res["bt_relu_bwd_from_bitmap"] = (ms, best, algorithmic_bytes("bt_relu_bwd_from_bitmap", n, 0, es))
+        # ReLU6 pair (a "next" row): fused forward, stash only, and the backward that consults the stashed values
+        ms, best = time_call(lambda: B.bt_relu6_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix,
+                                                             st.nnz_out, ws, st.dev_status))
+        nnz6 = st.nnz
+        res["bt_relu6_fwd_compress"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, nnz6, es))
+        ms, best = time_call(lambda: B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, x, dense))
+        res["bt_relu6_bwd_from_stash"] = (ms, best, 2 * n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + nnz6 * es)
         # double-mask form (a "next" row): the stash of x masks a dense tensor of the same shape
         B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
         nnz = st.nnz

@@ -149,6 +149,26 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
                           int32_t *dev_status, void *stream);
 
 /*
+ * ReLU6 (the activation of the MobileNetV2 family among the paper's models) fused with Algorithm 1:
+ * y[i] = (x[i] <= 0) ? +0 : (x[i] >= 6 ? 6 : x[i]) under IEEE comparison of the exactly widened element
+ * (a NaN fails both comparisons and is kept), stashed in the same pass.  Parameters as
+ * bt_relu_fwd_compress.
+ */
+int bt_relu6_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out,
+                          uint32_t *bitmap, void *values, uint64_t values_capacity,
+                          uint64_t *chunk_prefix, uint64_t *nnz_out,
+                          void *workspace, size_t workspace_bytes,
+                          int32_t *dev_status, void *stream);
+
+/*
+ * ReLU6 backward from the stash: grad_in[i] = (bit i set and its stashed value < 6) ? grad_out[i] : +0.
+ * The bitmap alone cannot tell a saturated unit (stashed value 6) from an active one, so the values and
+ * the chunk prefix array are read as well.  A select, not a multiply.  grad_in may alias grad_out.
+ */
+int bt_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix,
+                            const void *grad_out, uint64_t n, int dtype, void *grad_in, void *stream);
+
+/*
  * Double-mask batch normalisation support (section 3.1: the zero pattern of
  * the normalisation layer's input is applied as a mask to its output, which
  * carries the sparsity through the layer).  mask_bitmap / mask_chunk_prefix are

@@ -28,7 +28,7 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
            "bt_prune_fwd_compress", "bt_mask_compress", "bt_compress_arena", "bt_prune_fwd_compress_arena",
-           "bt_decompress_arena")
+           "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
         L.bt_prune_fwd_compress_arena.restype = i32
         L.bt_decompress_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
         L.bt_decompress_arena.restype = i32
+        L.bt_relu6_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_relu6_fwd_compress.restype = i32
+        L.bt_relu6_bwd_from_stash.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
+        L.bt_relu6_bwd_from_stash.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -214,6 +218,28 @@ def bt_decompress_arena(bitmap: torch.Tensor, arena: torch.Tensor, values_offset
     st = lib().bt_decompress_arena(_ptr(bitmap), _ptr(arena), _ptr(values_offset), _ptr(chunk_prefix), n,
                                    DTYPE_CODE[dense_out.dtype], _ptr(dense_out), _stream(stream))
     return _check("bt_decompress_arena", st, check)
+
+
+def bt_relu6_fwd_compress(pre_act: torch.Tensor, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
+                          values: torch.Tensor, chunk_prefix: torch.Tensor, nnz_out: torch.Tensor,
+                          workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                          *, n: Optional[int] = None, values_capacity: Optional[int] = None, stream=None,
+                          check: bool = True) -> int:
+    n = pre_act.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    st = lib().bt_relu6_fwd_compress(_ptr(pre_act), n, DTYPE_CODE[pre_act.dtype], _ptr(y_out), _ptr(bitmap),
+                                     _ptr(values), cap, _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace),
+                                     _nbytes(workspace), _ptr(dev_status), _stream(stream))
+    return _check("bt_relu6_fwd_compress", st, check)
+
+
+def bt_relu6_bwd_from_stash(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,
+                            grad_out: torch.Tensor, grad_in: torch.Tensor, *, n: Optional[int] = None, stream=None,
+                            check: bool = True) -> int:
+    n = grad_out.numel() if n is None else n
+    st = lib().bt_relu6_bwd_from_stash(_ptr(bitmap), _ptr(values), _ptr(chunk_prefix), _ptr(grad_out), n,
+                                       DTYPE_CODE[grad_out.dtype], _ptr(grad_in), _stream(stream))
+    return _check("bt_relu6_bwd_from_stash", st, check)
 
 
 def bt_decompress(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor, dense_out: torch.Tensor,

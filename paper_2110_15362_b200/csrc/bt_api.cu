@@ -24,7 +24,7 @@ struct Arena {
     uint64_t  bytes      = 0;
 };
 
-int compress_common(const void *src, uint64_t n, int dtype, bool relu, float tau, void *y, uint32_t *bitmap, void *values,
+int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau, void *y, uint32_t *bitmap, void *values,
                     uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
                     size_t workspace_bytes, int32_t *dev_status, void *stream, const Arena &arena = Arena())
 {
@@ -67,7 +67,7 @@ int compress_common(const void *src, uint64_t n, int dtype, bool relu, float tau
     a.values_offset_out = arena.offset_out;
     a.arena_bytes       = arena.bytes;
     a.n          = n;
-    return bt::launch_compress(a, dtype, relu, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+    return bt::launch_compress(a, dtype, fused, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
 
 }  // namespace
@@ -90,7 +90,7 @@ int bt_compress(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void
                 uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace, size_t workspace_bytes,
                 int32_t *dev_status, void *stream)
 {
-    return compress_common(dense, n, dtype, false, 0.0f, nullptr, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+    return compress_common(dense, n, dtype, 0, 0.0f, nullptr, bitmap, values, values_capacity, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream);
 }
 
@@ -98,7 +98,7 @@ int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out
                          uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
                          size_t workspace_bytes, int32_t *dev_status, void *stream)
 {
-    return compress_common(pre_act, n, dtype, true, 0.0f, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+    return compress_common(pre_act, n, dtype, 1, 0.0f, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream);
 }
 
@@ -106,8 +106,32 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
                           uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
                           size_t workspace_bytes, int32_t *dev_status, void *stream)
 {
-    return compress_common(x, n, dtype, true, tau, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+    return compress_common(x, n, dtype, 1, tau, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream);
+}
+
+int bt_relu6_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out, uint32_t *bitmap, void *values,
+                          uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
+                          size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    return compress_common(pre_act, n, dtype, 2, 0.0f, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream);
+}
+
+int bt_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix,
+                            const void *grad_out, uint64_t n, int dtype, void *grad_in, void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !chunk_prefix || !grad_out || !grad_in) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(grad_out, 16) ||
+        !aligned(grad_in, 16))
+        return BT_ERR_ALIGN;
+    return bt::launch_relu6_bwd(bitmap, values, chunk_prefix, grad_out, n, dtype, grad_in,
+                                static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
 }
 
 int bt_compress_arena(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void *arena, uint64_t arena_bytes,
@@ -117,7 +141,7 @@ int bt_compress_arena(const void *dense, uint64_t n, int dtype, uint32_t *bitmap
     if (!arena_cursor) return BT_ERR_NULL;
     Arena ar;
     ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
-    return compress_common(dense, n, dtype, false, 0.0f, nullptr, bitmap, arena, arena_bytes, chunk_prefix, nnz_out,
+    return compress_common(dense, n, dtype, 0, 0.0f, nullptr, bitmap, arena, arena_bytes, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream, ar);
 }
 
@@ -129,7 +153,7 @@ int bt_prune_fwd_compress_arena(const void *x, uint64_t n, int dtype, float tau,
     if (!arena_cursor) return BT_ERR_NULL;
     Arena ar;
     ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
-    return compress_common(x, n, dtype, true, tau, y_out, bitmap, arena, arena_bytes, chunk_prefix, nnz_out, workspace,
+    return compress_common(x, n, dtype, 1, tau, y_out, bitmap, arena, arena_bytes, chunk_prefix, nnz_out, workspace,
                            workspace_bytes, dev_status, stream, ar);
 }
 

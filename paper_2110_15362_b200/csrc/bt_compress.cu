@@ -177,7 +177,7 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
         for (int j = 0; j < kBatch; ++j) {
             Reg<U> x = v[j];
             if constexpr (RELU_DT >= 0) {
-                x = KeepAbove<RELU_DT>::keep(x, tau) ? x : Reg<U>(0);
+                x = fused_forward<RELU_DT>(x, tau);
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
                     if (!kGuardY || e < yvalid) y[e] = static_cast<U>(x);
@@ -227,7 +227,7 @@ __device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, cons
 }
 
 // U: uint32_t (4-byte elements) or uint16_t (2-byte elements).
-// RELU_DT: -1 for the plain compressor, else the element type whose ReLU is fused in.
+// RELU_DT: -1 for the plain compressor, else the number of the fused forward form (element type, + 4 for ReLU6).
 // kWarps compactor warps and as many copier warps, kSeg elements per warp, kStages ring slots.
 template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages, int kCopiers>
 __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
@@ -699,13 +699,28 @@ extern "C" int bt_debug_set_buffer(void *buf, unsigned int it0)
 }
 #endif
 
-cudaError_t launch_compress(const CompressArgs &a, int dtype, bool relu, cudaStream_t stream)
+cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStream_t stream)
 {
+    // fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0), 2 ReLU6
     const bool y = a.y != nullptr;
-    if (!relu) {
+    if (fused == 0) {
         return dtype == BT_F64   ? launch_typed<uint64_t, -1, false>(a, stream)
                : dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(a, stream)
                                  : launch_typed<uint16_t, -1, false>(a, stream);
+    }
+    constexpr int k6 = kFusedRelu6;
+    if (fused == 2) {
+        switch (dtype) {
+        case BT_F64:
+            return y ? launch_typed<uint64_t, k6 + BT_F64, true>(a, stream) : launch_typed<uint64_t, k6 + BT_F64, false>(a, stream);
+        case BT_F32:
+            return y ? launch_typed<uint32_t, k6 + BT_F32, true>(a, stream) : launch_typed<uint32_t, k6 + BT_F32, false>(a, stream);
+        case BT_F16:
+            return y ? launch_typed<uint16_t, k6 + BT_F16, true>(a, stream) : launch_typed<uint16_t, k6 + BT_F16, false>(a, stream);
+        default:
+            return y ? launch_typed<uint16_t, k6 + BT_BF16, true>(a, stream)
+                     : launch_typed<uint16_t, k6 + BT_BF16, false>(a, stream);
+        }
     }
     switch (dtype) {
     case BT_F64:

@@ -41,12 +41,15 @@ struct CompressArgs {
     uint64_t    n;
 };
 
-cudaError_t launch_compress(const CompressArgs &a, int dtype, bool relu, cudaStream_t s);
+// fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0), 2 ReLU6
+cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStream_t s);
 // values_offset: NULL, or a device word holding the byte offset of the packed values inside `values`
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                               const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t s);
 cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,
                                int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t s);
+cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
+                             uint64_t n, int dtype, void *gin, cudaStream_t s);
 cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size,
                             void *gin, cudaStream_t s);
 
@@ -146,35 +149,70 @@ __device__ __forceinline__ uint32_t lanemask_lt()
     return m;
 }
 
-// ---------------------------------------------------------------- keep what exceeds the threshold
-// keep(x, tau) = !(x <= tau) under IEEE comparison, the element widened exactly to binary32 (binary64 elements: tau widened to binary64): true for
-// values above tau and for NaN.  tau = 0 is the ReLU decision (positive or NaN).  The 16-bit forms take
-// the pattern in the low half of the register (the upper half may hold a sign extension).
+// ---------------------------------------------------------------- decisions of the fused forward forms
+// Elem<DT>::widen(u): the element's value, widened exactly (binary16 / bfloat16 -> binary32; binary32 and
+// binary64 as they are).  The 16-bit forms take the pattern in the low half of the register (the upper half
+// may hold a sign extension).  Elem<DT>::kSix: the pattern of 6.0 in the element type (exact in all four).
 template <int DT>
-struct KeepAbove;
+struct Elem;
 template <>
-struct KeepAbove<BT_F32> {
-    __device__ static __forceinline__ bool keep(uint32_t u, float tau) { return !(__uint_as_float(u) <= tau); }
+struct Elem<BT_F32> {
+    static constexpr uint32_t kSix = 0x40C00000u;
+    __device__ static __forceinline__ float widen(uint32_t u) { return __uint_as_float(u); }
 };
 template <>
-struct KeepAbove<BT_F64> {
-    __device__ static __forceinline__ bool keep(uint64_t u, float tau)
-    {
-        return !(__longlong_as_double(static_cast<long long>(u)) <= static_cast<double>(tau));
-    }
+struct Elem<BT_F64> {
+    static constexpr uint64_t kSix = 0x4018000000000000ull;
+    __device__ static __forceinline__ double widen(uint64_t u) { return __longlong_as_double(static_cast<long long>(u)); }
 };
 template <>
-struct KeepAbove<BT_F16> {
-    __device__ static __forceinline__ bool keep(uint32_t u, float tau)
+struct Elem<BT_F16> {
+    static constexpr uint32_t kSix = 0x4600u;
+    __device__ static __forceinline__ float widen(uint32_t u)
     {
         float f;
         asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(static_cast<unsigned short>(u)));
-        return !(f <= tau);
+        return f;
     }
 };
 template <>
-struct KeepAbove<BT_BF16> {
-    __device__ static __forceinline__ bool keep(uint32_t u, float tau) { return !(__uint_as_float(u << 16) <= tau); }
+struct Elem<BT_BF16> {
+    static constexpr uint32_t kSix = 0x40C0u;
+    __device__ static __forceinline__ float widen(uint32_t u) { return __uint_as_float(u << 16); }
 };
+
+// v >= 6 as an opaque 0/1 (false for a NaN).  Written as inline PTX on purpose: given the comparison and the
+// select that follows it in C++, the compiler may fuse the two into a floating-point minimum, which returns the
+// canonical NaN for a NaN input and so loses the payload and sign that the format keeps.
+__device__ __forceinline__ uint32_t at_least_six(float v)
+{
+    uint32_t r;
+    asm("{\n\t.reg .pred p;\n\tsetp.ge.f32 p, %1, 0f40C00000;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "f"(v));
+    return r;
+}
+__device__ __forceinline__ uint32_t at_least_six(double v)
+{
+    uint32_t r;
+    asm("{\n\t.reg .pred p;\n\tsetp.ge.f64 p, %1, 0d4018000000000000;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "d"(v));
+    return r;
+}
+
+// The fused forward forms are numbered by one template argument: -1 none (plain compressor), DT (0..3) keep
+// what exceeds the threshold (tau = 0: ReLU), 4 + DT ReLU6.
+constexpr int kFusedRelu6 = 4;
+
+// y = (x <= tau) ? +0 : x, and for ReLU6 additionally 6 where x >= 6; IEEE comparisons, so a NaN is kept.
+template <int FUSED, typename R>
+__device__ __forceinline__ R fused_forward(R x, float tau)
+{
+    constexpr int DT   = FUSED & 3;
+    const auto    v    = Elem<DT>::widen(x);
+    const bool    drop = v <= static_cast<decltype(v)>(tau);
+    if constexpr (FUSED >= kFusedRelu6) {
+        const uint32_t saturated = at_least_six(v);
+        x                        = saturated ? static_cast<R>(Elem<DT>::kSix) : x;     // selects, no branches
+    }
+    return drop ? R(0) : x;
+}
 
 }  // namespace bt

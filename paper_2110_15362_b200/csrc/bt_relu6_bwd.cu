@@ -1,0 +1,170 @@
+// ReLU6 backward from the stash: grad_in[i] = (bit i set and the stashed
+// activation is below 6) ? grad_out[i] : +0.  Unlike plain ReLU, the bitmap alone
+// does not say whether a unit is saturated (its stashed value is 6), so the
+// values are consulted: the decompressor's rank arithmetic (chunk prefix entry +
+// popcounts, no communication between warps), a gather of the stashed values of
+// the set bits, one comparison each, and a select on the gradient, which moves
+// in 16-byte vectors.
+//
+// One warp, one quarter chunk (1024 elements = 32 bitmap words); a lane owns kE
+// consecutive elements per step, i.e. kE consecutive bits of one word.
+#include "bt_internal.cuh"
+
+namespace bt {
+namespace {
+
+constexpr uint32_t kFull = 0xFFFFFFFFu;
+
+template <typename U, int DT, int kE, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32)
+relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values, const uint64_t *__restrict__ prefix,
+                 const U *gout, const uint64_t n, U *gin)   // gin may alias gout
+{
+    constexpr int kVec          = 16 / sizeof(U);
+    constexpr int kLanesPerWord = 32 / kE;
+    constexpr int kWordsPerStep = kE;
+    constexpr int kSteps        = 32 / kWordsPerStep;
+    static_assert(kE % kVec == 0 && 32 % kE == 0 && kE < 32, "a lane takes whole vectors of one word");
+
+    const uint32_t lane        = threadIdx.x & 31u;
+    const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    const uint64_t quarters    = (n + 1023) >> 10;
+    if (warp_global >= quarters) return;
+
+    const uint64_t chunk       = warp_global >> 2;
+    const uint32_t q           = static_cast<uint32_t>(warp_global & 3u);
+    const uint64_t words_total = (n + 31) >> 5;
+    const uint64_t w0          = chunk * 128 + 4 * lane;
+    const uint64_t e0          = warp_global << 10;
+
+    // the quarter of the gradient first: these loads do not depend on the stash
+    U g[kSteps][kE];
+#pragma unroll
+    for (int k = 0; k < kSteps; ++k) {
+        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+#pragma unroll
+        for (int v = 0; v < kE / kVec; ++v) {
+            const uint64_t at = eo + v * kVec;
+            U             *gv = g[k] + v * kVec;
+            if (at + kVec <= n) {
+                const uint4 pack = *reinterpret_cast<const uint4 *>(gout + at);
+                if constexpr (kVec == 2) {
+                    gv[0] = pack.x | (static_cast<uint64_t>(pack.y) << 32);
+                    gv[1] = pack.z | (static_cast<uint64_t>(pack.w) << 32);
+                } else if constexpr (kVec == 4) {
+                    gv[0] = pack.x, gv[1] = pack.y, gv[2] = pack.z, gv[3] = pack.w;
+                } else {
+                    gv[0] = static_cast<U>(pack.x), gv[1] = static_cast<U>(pack.x >> 16);
+                    gv[2] = static_cast<U>(pack.y), gv[3] = static_cast<U>(pack.y >> 16);
+                    gv[4] = static_cast<U>(pack.z), gv[5] = static_cast<U>(pack.z >> 16);
+                    gv[6] = static_cast<U>(pack.w), gv[7] = static_cast<U>(pack.w >> 16);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < kVec; ++j) gv[j] = at + j < n ? gout[at + j] : U(0);
+            }
+        }
+    }
+
+    uint4 w4 = make_uint4(0, 0, 0, 0);
+    if (w0 + 3 < words_total) {
+        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
+    } else {
+        if (w0 < words_total) w4.x = bitmap[w0];
+        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
+        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
+    }
+    const uint64_t chunk_base = prefix[chunk];
+
+    uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(kFull, before, o);
+
+    const int      src = 8 * q + (lane >> 2);
+    const uint32_t c0 = __shfl_sync(kFull, w4.x, src), c1 = __shfl_sync(kFull, w4.y, src);
+    const uint32_t c2 = __shfl_sync(kFull, w4.z, src), c3 = __shfl_sync(kFull, w4.w, src);
+    uint32_t       word = (lane & 2u) ? ((lane & 1u) ? c3 : c2) : ((lane & 1u) ? c1 : c0);
+    // bits past the end of the tensor do not count (a well-formed bitmap has none)
+    const uint64_t word_first = e0 + 32ull * lane;
+    if (word_first >= n) word = 0;
+    else if (n - word_first < 32) word &= (1u << static_cast<uint32_t>(n - word_first)) - 1u;
+
+    uint32_t incl = __popc(word);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t u = __shfl_up_sync(kFull, incl, o);
+        if (lane >= static_cast<uint32_t>(o)) incl += u;
+    }
+    const uint32_t excl = incl - __popc(word);
+    const U *const vp   = values + (chunk_base + before);
+
+    const uint32_t shift = (lane % kLanesPerWord) * kE;
+#pragma unroll
+    for (int k = 0; k < kSteps; ++k) {
+        const int      from = k * kWordsPerStep + lane / kLanesPerWord;
+        const uint32_t w    = __shfl_sync(kFull, word, from);
+        const uint32_t wex  = __shfl_sync(kFull, excl, from);
+        const uint32_t bits = (w >> shift) & ((1u << kE) - 1u);
+        uint32_t       off  = wex + __popc(w & ((1u << shift) - 1u));
+#pragma unroll
+        for (int j = 0; j < kE; ++j) {
+            const bool set  = (bits >> j) & 1u;
+            const U    v    = set ? vp[off] : U(0);                   // a predicated load, as in the decompressor
+            const auto a    = Elem<DT>::widen(v);
+            const bool pass = set & (a < static_cast<decltype(a)>(6));   // false for a stashed 6 and for a NaN
+            off += set;
+            g[k][j] = pass ? g[k][j] : U(0);
+        }
+        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+#pragma unroll
+        for (int v = 0; v < kE / kVec; ++v) {
+            const uint64_t at = eo + v * kVec;
+            const U       *gv = g[k] + v * kVec;
+            if (at + kVec <= n) {
+                uint4 pack;
+                if constexpr (kVec == 2) {
+                    pack = make_uint4(static_cast<uint32_t>(gv[0]), static_cast<uint32_t>(gv[0] >> 32),
+                                      static_cast<uint32_t>(gv[1]), static_cast<uint32_t>(gv[1] >> 32));
+                } else if constexpr (kVec == 4) {
+                    pack = make_uint4(gv[0], gv[1], gv[2], gv[3]);
+                } else {
+                    pack = make_uint4(gv[0] | (uint32_t(gv[1]) << 16), gv[2] | (uint32_t(gv[3]) << 16),
+                                      gv[4] | (uint32_t(gv[5]) << 16), gv[6] | (uint32_t(gv[7]) << 16));
+                }
+                *reinterpret_cast<uint4 *>(gin + at) = pack;
+            } else {
+#pragma unroll
+                for (int j = 0; j < kVec; ++j)
+                    if (at + j < n) gin[at + j] = gv[j];
+            }
+        }
+    }
+}
+
+template <typename U, int DT, int kE>
+cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
+                         uint64_t n, void *gin, cudaStream_t stream)
+{
+    constexpr int  kWarps   = 8;
+    const uint64_t quarters = (n + 1023) >> 10;
+    const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
+    if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    relu6_bwd_kernel<U, DT, kE, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
+        bitmap, static_cast<const U *>(values), prefix, static_cast<const U *>(gout), n, static_cast<U *>(gin));
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
+                             uint64_t n, int dtype, void *gin, cudaStream_t stream)
+{
+    switch (dtype) {
+    case BT_F64: return launch_typed<uint64_t, BT_F64, 2>(bitmap, values, prefix, gout, n, gin, stream);
+    case BT_F32: return launch_typed<uint32_t, BT_F32, 4>(bitmap, values, prefix, gout, n, gin, stream);
+    case BT_F16: return launch_typed<uint16_t, BT_F16, 8>(bitmap, values, prefix, gout, n, gin, stream);
+    default: return launch_typed<uint16_t, BT_BF16, 8>(bitmap, values, prefix, gout, n, gin, stream);
+    }
+}
+
+}  // namespace bt
