@@ -368,3 +368,78 @@ uint64_t oracle_compressed_bytes(uint64_t n, uint64_t nnz, int elem_size)
     uint64_t chunks = (n + CHUNK_ELEMS - 1) / CHUNK_ELEMS;
     return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;
 }
+
+/* binary32 -> binary16, round to nearest, ties to even (IEEE 754 conversion).
+ * Above the largest half (65504) by half a unit in the last place or more:
+ * infinity.  At or below 2^-25: zero (2^-25 is the tie between 0 and the
+ * smallest subnormal, and 0 is the even one).  A NaN becomes the one quiet
+ * NaN 0x7FFF, sign and payload dropped (the reading taken for the narrowed
+ * stash).  Works on the bit pattern; no floating-point operation involved. */
+uint16_t oracle_float_to_half(uint32_t u)
+{
+    uint32_t sign = (u >> 16) & 0x8000u;
+    uint32_t a    = u & 0x7FFFFFFFu;
+    if (a > 0x7F800000u) return 0x7FFFu;
+    if (a >= 0x477FF000u) return (uint16_t)(sign | 0x7C00u);     /* >= 65520 (and inf) */
+    if (a <= 0x33000000u) return (uint16_t)sign;                 /* <= 2^-25 */
+    uint32_t expo = a >> 23;
+    uint32_t q, rem, half;
+    if (expo < 113u) {
+        /* below 2^-14: a half subnormal, q units of 2^-24.  With the hidden bit
+         * the value is m * 2^(expo-150), i.e. m >> (126 - expo) units. */
+        uint32_t m     = (a & 0x7FFFFFu) | 0x800000u;
+        uint32_t shift = 126u - expo;                            /* 14 .. 24 */
+        q    = m >> shift;
+        rem  = m & ((1u << shift) - 1u);
+        half = 1u << (shift - 1u);
+    } else {
+        /* normal half: rebias 127 -> 15, keep 10 mantissa bits, round on the 13 dropped */
+        q    = ((expo - 112u) << 10) | ((a >> 13) & 0x3FFu);
+        rem  = a & 0x1FFFu;
+        half = 0x1000u;
+    }
+    if (rem > half || (rem == half && (q & 1u))) q += 1u;        /* a carry runs into the exponent as it should */
+    return (uint16_t)(sign | q);
+}
+
+/* binary32 -> bfloat16 (the top 16 bits), round to nearest, ties to even; a
+ * value that rounds past the largest finite bfloat16 becomes infinity by the
+ * same carry; a NaN becomes 0x7FFF. */
+uint16_t oracle_float_to_bfloat16(uint32_t u)
+{
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FFFu;
+    uint32_t q = u >> 16, rem = u & 0xFFFFu;
+    if (rem > 0x8000u || (rem == 0x8000u && (q & 1u))) q += 1u;
+    return (uint16_t)q;
+}
+
+/* Down-cast on stash: the tensor is binary32, the stashed values are 16 bits
+ * wide.  act = fused ? ((x <= tau) ? +0 : x) : x; bit i is set where the
+ * binary32 pattern of act is not all-zero -- so bitmap, prefix and the count
+ * are those of the full-precision stash -- and the value pushed is act
+ * narrowed to to_kind (ORACLE_F16 or ORACLE_BF16), which may be a zero when
+ * act underflows.  y (binary32, may be NULL) receives act.  Returns nnz. */
+uint64_t oracle_narrow_compress(const void *x, uint64_t n, int to_kind, int fused, float tau,
+                                void *y, uint32_t *bitmap, uint16_t *values, uint64_t *prefix)
+{
+    const unsigned char *src = (const unsigned char *)x;
+    unsigned char *yo = (unsigned char *)y;
+    uint64_t words = (n + 31) / 32;
+    uint64_t j = 0;
+
+    for (uint64_t w = 0; w < words; ++w) bitmap[w] = 0;
+
+    for (uint64_t i = 0; i < n; ++i) {
+        if (i % CHUNK_ELEMS == 0) prefix[i / CHUNK_ELEMS] = j;
+        uint32_t u;
+        memcpy(&u, src + 4 * i, 4);
+        if (fused && le_tau(src + 4 * i, ORACLE_F32, tau)) u = 0;
+        if (yo) memcpy(yo + 4 * i, &u, 4);
+        if (u != 0) {
+            values[j] = to_kind == ORACLE_F16 ? oracle_float_to_half(u) : oracle_float_to_bfloat16(u);
+            j += 1;
+            bitmap[i >> 5] |= (uint32_t)1 << (i & 31);
+        }
+    }
+    return j;
+}

@@ -85,6 +85,19 @@ void oracle_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
 /* M_b of section 3.2 generalised: bitmap words + values + prefix entries */
 uint64_t oracle_compressed_bytes(uint64_t n, uint64_t nnz, int elem_size);
 
+/* Down-cast on stash (the low-precision study of the paper's evaluation, as a
+ * hybrid: binary32 tensor, 16-bit stashed values).  act = fused ? ((x <= tau) ?
+ * +0 : x) : x; bitmap / prefix / count are those of act in binary32; values[k]
+ * is the k-th non-zero of act narrowed to to_kind (ORACLE_F16 / ORACLE_BF16)
+ * by the conversions below.  y (binary32, may be NULL) = act.  Returns nnz. */
+uint64_t oracle_narrow_compress(const void *x, uint64_t n, int to_kind, int fused, float tau,
+                                void *y, uint32_t *bitmap, uint16_t *values, uint64_t *prefix);
+
+/* binary32 pattern -> binary16 / bfloat16 pattern: round to nearest, ties to
+ * even; overflow to infinity; every NaN to 0x7FFF */
+uint16_t oracle_float_to_half(uint32_t bits);
+uint16_t oracle_float_to_bfloat16(uint32_t bits);
+
 /* exact widening of one IEEE binary16 pattern to binary32 (used by the ReLU test) */
 float oracle_half_to_float(uint16_t h);
 

@@ -67,6 +67,12 @@ def lib() -> ctypes.CDLL:
         L.oracle_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp]
         L.oracle_compressed_bytes.restype = u64
         L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
+        L.oracle_narrow_compress.restype = u64
+        L.oracle_narrow_compress.argtypes = [vp, u64, i32, i32, ctypes.c_float, vp, vp, vp, vp]
+        L.oracle_float_to_half.restype = ctypes.c_uint16
+        L.oracle_float_to_half.argtypes = [ctypes.c_uint32]
+        L.oracle_float_to_bfloat16.restype = ctypes.c_uint16
+        L.oracle_float_to_bfloat16.argtypes = [ctypes.c_uint32]
         L.oracle_half_to_float.restype = ctypes.c_float
         L.oracle_half_to_float.argtypes = [ctypes.c_uint16]
         _lib = L
@@ -183,6 +189,29 @@ def relu_bwd_from_bitmap(bitmap: np.ndarray, grad_out: np.ndarray) -> np.ndarray
     bm = np.ascontiguousarray(bitmap, dtype=np.uint32)
     lib().oracle_relu_bwd_from_bitmap(_ptr(bm), _ptr(g), g.size, g.dtype.itemsize, _ptr(out))
     return out
+
+
+def narrow_compress(x: np.ndarray, to_kind: str, fused: bool = False, tau: float = 0.0, want_y: bool = False):
+    """Down-cast on stash: `x` holds binary32 patterns; the stashed values are `to_kind` ("f16" / "bf16")
+    patterns.  Returns (y or None, Compressed) with `values` of dtype uint16."""
+    x = _raw(x)
+    assert x.dtype.itemsize == 4 and to_kind in ("f16", "bf16")
+    n = x.size
+    y = np.empty(n, dtype=x.dtype) if want_y else None
+    bitmap = np.full((n + 31) // 32, 0xDEADBEEF, dtype=np.uint32)
+    values = np.empty(n, dtype=np.uint16)
+    prefix = np.full((n + CHUNK - 1) // CHUNK, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64)
+    nnz = int(lib().oracle_narrow_compress(_ptr(x), n, KINDS[to_kind], int(fused), float(np.float32(tau)), _ptr(y),
+                                            _ptr(bitmap), _ptr(values), _ptr(prefix)))
+    return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
+
+
+def float_to_half(bits: int) -> int:
+    return int(lib().oracle_float_to_half(bits))
+
+
+def float_to_bfloat16(bits: int) -> int:
+    return int(lib().oracle_float_to_bfloat16(bits))
 
 
 def compressed_bytes(n: int, nnz: int, elem_size: int) -> int:

@@ -36,6 +36,13 @@ MUTANTS = {
                        "if ((mask_bitmap[i >> 5] >> (31 - (i & 31))) & 1u) {\n            memcpy(val"),
     "relu6_never_saturates": ("else if (ge6)         six_pattern(kind, act);", "else if (ge6 && 0)    six_pattern(kind, act);"),
     "relu6_bwd_passes_saturated_units": ("            pass = lt6;\n", "            pass = 1;\n"),
+    "narrow_truncates_instead_of_rounding": ("if (rem > half || (rem == half && (q & 1u))) q += 1u;        /* a carry",
+                                             "if (0) q += 1u;        /* a carry"),
+    "narrow_half_ties_away_from_zero": ("if (rem > half || (rem == half && (q & 1u))) q += 1u;        /* a carry",
+                                        "if (rem >= half) q += 1u;        /* a carry"),
+    "narrow_bf16_ties_away_from_zero": ("if (rem > 0x8000u || (rem == 0x8000u && (q & 1u))) q += 1u;", "if (rem >= 0x8000u) q += 1u;"),
+    "narrow_tests_zero_after_the_cast": ("        if (u != 0) {\n            values[j] = to_kind",
+                                         "        if ((to_kind == ORACLE_F16 ? oracle_float_to_half(u) : oracle_float_to_bfloat16(u)) & 0x7FFFu) {\n            values[j] = to_kind"),
     "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
     "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
 }
@@ -66,6 +73,8 @@ def build_mutant(tmp_path, name):
     L.oracle_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp]
     L.oracle_compressed_bytes.restype = u64
     L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
+    L.oracle_narrow_compress.restype = u64
+    L.oracle_narrow_compress.argtypes = [vp, u64, i32, i32, ctypes.c_float, vp, vp, vp, vp]
     return L
 
 
@@ -137,6 +146,16 @@ def pins_hold(L) -> bool:
     L.oracle_relu6_bwd_from_stash(p(bitmap), p(values[:nnz6].copy()), n, 0, p(W.raw_numpy(g6)), p(gin6))
     if not np.array_equal(gin6, W.raw_numpy(torch.where((t6 > 0) & (t6 < 6), g6, torch.zeros(())))):
         return False
+    # down-cast on stash against numpy (binary16) and torch (bfloat16), with ties and an underflow
+    tn = torch.randn(n, generator=torch.Generator().manual_seed(8))
+    xn = W.raw_numpy(tn).copy()
+    xn[:6] = np.array([0x3F801000, 0x3F803000, 0x3F808000, 0x3F818000, 0x2F000000, 0], dtype=np.uint32)
+    for to_kind, ref in ((1, xn.view(np.float32).astype(np.float16).view(np.uint16)),
+                         (2, torch.from_numpy(xn.view(np.int32)).view(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))):
+        v16 = np.zeros(n, np.uint16)
+        nn_ = L.oracle_narrow_compress(p(xn), n, to_kind, 0, 0.0, None, p(bitmap), p(v16), p(prefix))
+        if nn_ != int(np.count_nonzero(xn)) or not np.array_equal(v16[:nn_], ref[xn != 0]):
+            return False
     # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
     if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
         return False
