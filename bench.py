@@ -357,6 +357,18 @@ def large_tensor_kernels(dev, peak_gbs: float):
         res["bt_relu6_fwd_compress"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, nnz6, es))
         ms, best = time_call(lambda: B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, x, dense))
         res["bt_relu6_bwd_from_stash"] = (ms, best, 2 * n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + nnz6 * es)
+        if kind == "f32":
+            # down-cast on stash (a "next" row): float32 tensor, 16-bit stashed values
+            for to, tdt in (("f16", torch.float16), ("bf16", torch.bfloat16)):
+                v16 = torch.empty(n, dtype=tdt, device=dev)
+                ms, best = time_call(lambda: B.bt_compress_narrow(x, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws,
+                                                                  st.dev_status))
+                by16 = n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + st.nnz * 2
+                res["bt_compress_narrow_" + to] = (ms, best, by16)
+                ms, best = time_call(lambda: B.bt_prune_fwd_compress_narrow(pre, 0.0, None, st.bitmap, v16, st.chunk_prefix,
+                                                                            st.nnz_out, ws, st.dev_status))
+                res["bt_prune_fwd_compress_narrow_" + to] = (ms, best, by16)
+                del v16
         # double-mask form (a "next" row): the stash of x masks a dense tensor of the same shape
         B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
         nnz = st.nnz

@@ -149,6 +149,34 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
                           int32_t *dev_status, void *stream);
 
 /*
+ * Down-cast on stash (the evaluation's "Combining BitTrain with Low Precision"
+ * study stores half-precision activation values in the bitmap format; these
+ * two calls are its hybrid form for a training run that computes in binary32):
+ * the tensor is BT_F32, the stashed values are to_dtype (BT_F16 or BT_BF16).
+ * bitmap, chunk_prefix and *nnz_out are exactly those bt_compress /
+ * bt_prune_fwd_compress give for the binary32 tensor -- the zero test is on
+ * the binary32 pattern, so bt_relu_bwd_from_bitmap is unchanged -- and
+ * values[k] (16 bits each; values_capacity counts 16-bit elements) is the k-th
+ * kept element converted with round-to-nearest-even: overflow gives +-inf, a
+ * magnitude of 2^-25 or less gives +-0 in binary16 (a zero stored under a set
+ * bit), every NaN gives 0x7FFF.  bt_decompress with to_dtype restores the
+ * narrowed dense tensor; bt_compressed_bytes(n, nnz, to_dtype) is the stash's
+ * size.  y_out (BT_F32, may be NULL, may alias x) receives the unnarrowed
+ * activation.  Lossy by design; no arena and no host-buffer form.  Other
+ * parameters and *dev_status as bt_compress.
+ */
+int bt_compress_narrow(const void *dense, uint64_t n, int to_dtype,
+                       uint32_t *bitmap, void *values, uint64_t values_capacity,
+                       uint64_t *chunk_prefix, uint64_t *nnz_out,
+                       void *workspace, size_t workspace_bytes,
+                       int32_t *dev_status, void *stream);
+int bt_prune_fwd_compress_narrow(const void *x, uint64_t n, int to_dtype, float tau, void *y_out,
+                                 uint32_t *bitmap, void *values, uint64_t values_capacity,
+                                 uint64_t *chunk_prefix, uint64_t *nnz_out,
+                                 void *workspace, size_t workspace_bytes,
+                                 int32_t *dev_status, void *stream);
+
+/*
  * ReLU6 (the activation of the MobileNetV2 family among the paper's models) fused with Algorithm 1:
  * y[i] = (x[i] <= 0) ? +0 : (x[i] >= 6 ? 6 : x[i]) under IEEE comparison of the exactly widened element
  * (a NaN fails both comparisons and is kept), stashed in the same pass.  Parameters as

@@ -28,7 +28,8 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap", "bt_host_staging_bytes", "bt_compress_host",
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
            "bt_prune_fwd_compress", "bt_mask_compress", "bt_compress_arena", "bt_prune_fwd_compress_arena",
-           "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash")
+           "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
+           "bt_prune_fwd_compress_narrow")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.bt_relu6_fwd_compress.restype = i32
         L.bt_relu6_bwd_from_stash.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
         L.bt_relu6_bwd_from_stash.restype = i32
+        L.bt_compress_narrow.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_compress_narrow.restype = i32
+        L.bt_prune_fwd_compress_narrow.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_prune_fwd_compress_narrow.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -173,6 +178,35 @@ def bt_prune_fwd_compress(x: torch.Tensor, tau: float, y_out: Optional[torch.Ten
                                      workspace.numel() * workspace.element_size(), _ptr(dev_status),
                                      _stream(stream))
     return _check("bt_prune_fwd_compress", st, check)
+
+def bt_compress_narrow(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,
+                       nnz_out: torch.Tensor, workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                       *, n: Optional[int] = None, values_capacity: Optional[int] = None, stream=None,
+                       check: bool = True) -> int:
+    """Down-cast on stash: a float32 tensor whose stashed values take the (16-bit) dtype of `values`."""
+    n = dense.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    assert dense.dtype == torch.float32
+    st = lib().bt_compress_narrow(_ptr(dense), n, DTYPE_CODE[values.dtype], _ptr(bitmap), _ptr(values), cap,
+                                  _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace), _nbytes(workspace),
+                                  _ptr(dev_status), _stream(stream))
+    return _check("bt_compress_narrow", st, check)
+
+
+def bt_prune_fwd_compress_narrow(x: torch.Tensor, tau: float, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
+                                 values: torch.Tensor, chunk_prefix: torch.Tensor, nnz_out: torch.Tensor,
+                                 workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                                 *, n: Optional[int] = None, values_capacity: Optional[int] = None, stream=None,
+                                 check: bool = True) -> int:
+    """Fused forward (tau = 0: ReLU) of a float32 tensor whose stashed values take the 16-bit dtype of `values`."""
+    n = x.numel() if n is None else n
+    cap = values.numel() if values_capacity is None else values_capacity
+    assert x.dtype == torch.float32
+    st = lib().bt_prune_fwd_compress_narrow(_ptr(x), n, DTYPE_CODE[values.dtype], ctypes.c_float(tau), _ptr(y_out),
+                                            _ptr(bitmap), _ptr(values), cap, _ptr(chunk_prefix), _ptr(nnz_out),
+                                            _ptr(workspace), _nbytes(workspace), _ptr(dev_status), _stream(stream))
+    return _check("bt_prune_fwd_compress_narrow", st, check)
+
 
 def bt_mask_compress(x: torch.Tensor, mask_bitmap: torch.Tensor, mask_chunk_prefix: torch.Tensor,
                      y_out: Optional[torch.Tensor], values: torch.Tensor, *, n: Optional[int] = None,

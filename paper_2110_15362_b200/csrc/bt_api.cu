@@ -26,9 +26,10 @@ struct Arena {
 
 int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau, void *y, uint32_t *bitmap, void *values,
                     uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
-                    size_t workspace_bytes, int32_t *dev_status, void *stream, const Arena &arena = Arena())
+                    size_t workspace_bytes, int32_t *dev_status, void *stream, const Arena &arena = Arena(), int cast = 0)
 {
     if (elem_size_of(dtype) == 0) return BT_ERR_DTYPE;
+    if (cast != 0 && (dtype != BT_F32 || (cast != BT_F16 && cast != BT_BF16))) return BT_ERR_DTYPE;
     if (!nnz_out) return BT_ERR_NULL;
     if (!aligned(nnz_out, 8) || !aligned(dev_status, 4)) return BT_ERR_ALIGN;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -62,6 +63,7 @@ int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau
     a.ws_header  = static_cast<uint32_t *>(workspace);
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
+    a.cast       = cast;
     a.tau        = tau;
     a.arena_cursor      = arena.cursor;
     a.values_offset_out = arena.offset_out;
@@ -108,6 +110,24 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
 {
     return compress_common(x, n, dtype, 1, tau, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
                            workspace, workspace_bytes, dev_status, stream);
+}
+
+int bt_compress_narrow(const void *dense, uint64_t n, int to_dtype, uint32_t *bitmap, void *values,
+                       uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace,
+                       size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    if (to_dtype != BT_F16 && to_dtype != BT_BF16) return BT_ERR_DTYPE;
+    return compress_common(dense, n, BT_F32, 0, 0.0f, nullptr, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream, Arena(), to_dtype);
+}
+
+int bt_prune_fwd_compress_narrow(const void *x, uint64_t n, int to_dtype, float tau, void *y_out, uint32_t *bitmap,
+                                 void *values, uint64_t values_capacity, uint64_t *chunk_prefix, uint64_t *nnz_out,
+                                 void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    if (to_dtype != BT_F16 && to_dtype != BT_BF16) return BT_ERR_DTYPE;
+    return compress_common(x, n, BT_F32, 1, tau, y_out, bitmap, values, values_capacity, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream, Arena(), to_dtype);
 }
 
 int bt_relu6_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out, uint32_t *bitmap, void *values,

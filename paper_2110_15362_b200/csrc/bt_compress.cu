@@ -207,29 +207,52 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
     return (out - seg_addr) / kES;
 }
 
-// One warp copies the `cnt` packed slots of its segment to out[0..cnt): contiguous, coalesced.
-template <typename U, bool kGuard>
-__device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, const uint32_t lane, const uint32_t cnt,
-                                                 U *__restrict__ out, const uint64_t room)
+// Down-cast on stash: a binary32 pattern narrowed to binary16 (CAST 1) or bfloat16 (CAST 2), round to nearest
+// even by the hardware conversion, every NaN to the one quiet NaN 0x7FFF.  CAST 0 passes the element through.
+template <int CAST, typename U>
+__device__ __forceinline__ auto narrowed(const U v)
 {
+    if constexpr (CAST == 0) {
+        return v;
+    } else {
+        static_assert(sizeof(U) == 4, "the narrowing forms take binary32 tensors");
+        const float f = __uint_as_float(v);
+        uint16_t    h;
+        if constexpr (CAST == 1) asm("cvt.rn.f16.f32 %0, %1;" : "=h"(h) : "f"(f));
+        else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(f));
+        return (v & 0x7FFFFFFFu) > 0x7F800000u ? static_cast<uint16_t>(0x7FFFu) : h;
+    }
+}
+template <int CAST, typename U>
+using Stored = std::conditional_t<CAST == 0, U, uint16_t>;
+
+// One warp copies the `cnt` packed slots of its segment to out[0..cnt): contiguous, coalesced.
+template <typename U, int CAST, bool kGuard>
+__device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, const uint32_t lane, const uint32_t cnt,
+                                                 Stored<CAST, U> *__restrict__ out, const uint64_t room)
+{
+    // (Pairing narrowed values into 4-byte stores was measured and is no faster: at half zeros the narrowing
+    // forms run at the speed of the compaction, not of the copy-out.)
     uint32_t j = lane;
     for (; j + 96 < cnt; j += 128) {
-        const U v0 = seg[j], v1 = seg[j + 32], v2 = seg[j + 64], v3 = seg[j + 96];
+        const auto v0 = narrowed<CAST>(seg[j]), v1 = narrowed<CAST>(seg[j + 32]), v2 = narrowed<CAST>(seg[j + 64]),
+                   v3 = narrowed<CAST>(seg[j + 96]);
         if (!kGuard || j < room) out[j] = v0;
         if (!kGuard || j + 32 < room) out[j + 32] = v1;
         if (!kGuard || j + 64 < room) out[j + 64] = v2;
         if (!kGuard || j + 96 < room) out[j + 96] = v3;
     }
     for (; j < cnt; j += 32) {
-        const U v = seg[j];
+        const auto v = narrowed<CAST>(seg[j]);
         if (!kGuard || j < room) out[j] = v;
     }
 }
 
 // U: uint32_t (4-byte elements) or uint16_t (2-byte elements).
 // RELU_DT: -1 for the plain compressor, else the number of the fused forward form (element type, + 4 for ReLU6).
+// CAST: 0, or the 16-bit type the copiers narrow the packed binary32 values to (1 binary16, 2 bfloat16).
 // kWarps compactor warps and as many copier warps, kSeg elements per warp, kStages ring slots.
-template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages, int kCopiers>
+template <typename U, int RELU_DT, bool WRITE_Y, int CAST, int kWarps, int kSeg, int kStages, int kCopiers>
 __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
 {
     constexpr int kTile          = kWarps * kSeg;
@@ -479,10 +502,10 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                     if (a.arena_cursor) {
                         // arena form: the room left behind the cursor; the cursor moves only when everything fitted
                         const uint64_t c0 = s_arena_c0;
-                        capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(U) : 0;
+                        capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(Stored<CAST, U>) : 0;
                         if (!aborted && nnz <= capacity) {
                             *a.values_offset_out = c0;
-                            *a.arena_cursor      = c0 + ((nnz * sizeof(U) + 15) & ~15ull);
+                            *a.arena_cursor      = c0 + ((nnz * sizeof(Stored<CAST, U>) + 15) & ~15ull);
                         }
                     }
                     if (a.dev_status)
@@ -517,12 +540,13 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     if (warp >= kFirstCopier) {
         // ------------------------------------------------------------ copier warps
         const uint32_t copier   = warp - kFirstCopier;
-        U             *vals     = static_cast<U *>(a.values);
+        using V                 = Stored<CAST, U>;
+        V             *vals     = static_cast<V *>(a.values);
         uint64_t       capacity = a.capacity;
         if (a.arena_cursor) {
             const uint64_t c0 = s_arena_c0;
-            vals              = reinterpret_cast<U *>(static_cast<unsigned char *>(a.values) + c0);
-            capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(U) : 0;
+            vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(a.values) + c0);
+            capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(V) : 0;
         }
         for (uint32_t it = 0;; ++it) {
             if (tile_of(it) >= num_tiles) break;
@@ -538,9 +562,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 const uint32_t cnt  = s_cnt[s][seg];
                 const uint64_t dst  = base + s_off[s][seg];
                 if (dst + cnt <= capacity)
-                    copy_out_segment<U, false>(pseg, lane, cnt, vals + dst, 0);
+                    copy_out_segment<U, CAST, false>(pseg, lane, cnt, vals + dst, 0);
                 else
-                    copy_out_segment<U, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
+                    copy_out_segment<U, CAST, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
             }
             __syncwarp();
             asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
@@ -637,14 +661,14 @@ struct LaunchShape {
     }
 };
 
-template <typename U, int RELU_DT, bool WRITE_Y, int kWarps, int kSeg, int kStages, int kCopiers>
+template <typename U, int RELU_DT, bool WRITE_Y, int CAST, int kWarps, int kSeg, int kStages, int kCopiers>
 cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
 {
     constexpr int kTile    = kWarps * kSeg;
     constexpr int kThreads = (kWarps + kCopiers + 3) * 32;
     constexpr size_t kSmem = static_cast<size_t>(kStages) * kTile * sizeof(U);
     static LaunchShape shape;   // one per instantiation
-    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, kWarps, kSeg, kStages, kCopiers>;
+    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, CAST, kWarps, kSeg, kStages, kCopiers>;
 
     const uint32_t num_tiles = static_cast<uint32_t>((a.n + kTile - 1) / kTile);
     int            max_grid  = 0;
@@ -662,7 +686,7 @@ cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
                                        stream);
 }
 
-template <typename U, int RELU_DT, bool WRITE_Y>
+template <typename U, int RELU_DT, bool WRITE_Y, int CAST = 0>
 cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
 {
     // One CTA per SM, the ring takes nearly all of its shared memory.
@@ -674,18 +698,18 @@ cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
     static const int cfg = [] { const char *e = getenv("BT_CFG"); return e ? atoi(e) : 0; }();
     if constexpr (sizeof(U) == 8) {
     } else if constexpr (sizeof(U) == 4) {
-        if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 6, 8>(a, stream);
-        if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 4>(a, stream);
-        if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 512, 7, 8>(a, stream);
+        if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 1024, 6, 8>(a, stream);
+        if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 1024, 7, 4>(a, stream);
+        if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 16, 512, 7, 8>(a, stream);
     } else {
-        if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 12, 8>(a, stream);
-        if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, 12, 1024, 8, 6>(a, stream);
-        if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, 16, 1024, 6, 16>(a, stream);
+        if (cfg == 1) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 1024, 12, 8>(a, stream);
+        if (cfg == 2) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 12, 1024, 8, 6>(a, stream);
+        if (cfg == 3) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 16, 1024, 6, 16>(a, stream);
     }
 #endif
-    if constexpr (sizeof(U) == 8) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 512, 7, 8>(a, stream);
-    else if constexpr (sizeof(U) == 4) return launch_shaped<U, RELU_DT, WRITE_Y, 8, 1024, 7, 8>(a, stream);
-    else return launch_shaped<U, RELU_DT, WRITE_Y, 16, 1024, 6, 8>(a, stream);
+    if constexpr (sizeof(U) == 8) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 512, 7, 8>(a, stream);
+    else if constexpr (sizeof(U) == 4) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 1024, 7, 8>(a, stream);
+    else return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 16, 1024, 6, 8>(a, stream);
 }
 
 }  // namespace
@@ -703,6 +727,14 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStr
 {
     // fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0), 2 ReLU6
     const bool y = a.y != nullptr;
+    if (a.cast != 0) {
+        // down-cast on stash: binary32 tensors, plain and threshold forms
+        if (dtype != BT_F32 || fused == 2 || a.arena_cursor) return cudaErrorInvalidValue;
+        const bool h = a.cast == BT_F16;
+        if (fused == 0) return h ? launch_typed<uint32_t, -1, false, 1>(a, stream) : launch_typed<uint32_t, -1, false, 2>(a, stream);
+        if (y) return h ? launch_typed<uint32_t, BT_F32, true, 1>(a, stream) : launch_typed<uint32_t, BT_F32, true, 2>(a, stream);
+        return h ? launch_typed<uint32_t, BT_F32, false, 1>(a, stream) : launch_typed<uint32_t, BT_F32, false, 2>(a, stream);
+    }
     if (fused == 0) {
         return dtype == BT_F64   ? launch_typed<uint64_t, -1, false>(a, stream)
                : dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(a, stream)

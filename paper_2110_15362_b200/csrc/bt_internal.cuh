@@ -31,6 +31,7 @@ struct CompressArgs {
     uint32_t   *ws_header;
     uint64_t   *ws_desc;    // wave totals, then tile descriptors
     uint32_t    ws_waves;   // number of wave totals
+    int         cast;       // 0, or the 16-bit type (BT_F16 / BT_BF16) the stashed values of a binary32 tensor are narrowed to
     float       tau;        // fused forms: elements <= tau become +0 (0 for plain ReLU)
     // arena forms: `values` is the arena's base, the packed values go to values + *arena_cursor (bytes);
     // on success the kernel stores the old cursor in *values_offset_out and advances the cursor past the

@@ -77,6 +77,7 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
     a.ws_header  = static_cast<uint32_t *>(scratch);
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(scratch) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
+    a.cast       = 0;
     a.tau        = 0.0f;
     a.arena_cursor = nullptr, a.values_offset_out = nullptr, a.arena_bytes = 0;
     a.n          = n;

@@ -1,6 +1,6 @@
 """One small, seeded invocation of a kernel, for profiler captures.
 
-    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|prune|decompress|relu_bwd|mask|mask_y> \
+    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|prune|narrow|relu6|relu6_bwd|decompress|relu_bwd|mask|mask_y> \
            [--log2n 26] [--zeros 0.5] [--reps 3]
 
 runs `reps` repetitions of one entry point on a tensor of 2**log2n elements (default 2**26: 256 MiB of
@@ -26,7 +26,7 @@ from . import workloads as W
 def main(argv=None) -> int:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("dtype", choices=["f32", "f16", "bf16", "f64"])
-    ap.add_argument("op", choices=["compress", "relu", "relu_y", "prune", "decompress", "relu_bwd", "mask", "mask_y"])
+    ap.add_argument("op", choices=["compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd", "decompress", "relu_bwd", "mask", "mask_y"])
     ap.add_argument("--tau", type=float, default=0.1)
     ap.add_argument("--log2n", type=int, default=26)
     ap.add_argument("--zeros", type=float, default=0.5)
@@ -44,6 +44,7 @@ def main(argv=None) -> int:
     st = B.Stash(n, x.dtype, dev)
     ws = B.new_workspace(n, dev)
     d = torch.empty_like(x)
+    v16 = torch.empty(n, dtype=torch.float16, device=dev) if args.op == "narrow" else None
 
     def compress():
         B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
@@ -58,6 +59,13 @@ def main(argv=None) -> int:
         elif args.op == "prune":
             B.bt_prune_fwd_compress(x, args.tau, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws,
                                     st.dev_status)
+        elif args.op == "narrow":                            # float32 tensor, float16 stashed values
+            B.bt_compress_narrow(x, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif args.op == "relu6":
+            B.bt_relu6_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif args.op == "relu6_bwd":
+            B.bt_relu6_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+            B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, x, d)
         elif args.op in ("mask", "mask_y"):
             compress()
             B.bt_mask_compress(x, st.bitmap, st.chunk_prefix, d if args.op == "mask_y" else None, st.values)

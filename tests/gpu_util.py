@@ -54,12 +54,13 @@ class GpuCompressed:
 
 
 def gpu_compress(x: torch.Tensor, relu: bool = False, want_y: bool = False, capacity=None,
-                 in_place: bool = False, keep_device: bool = False, tau=None):
-    """`tau` given: bt_prune_fwd_compress with that threshold (want_y / in_place as for the ReLU form)."""
+                 in_place: bool = False, keep_device: bool = False, tau=None, narrow=None):
+    """`tau` given: bt_prune_fwd_compress with that threshold (want_y / in_place as for the ReLU form).
+    `narrow` ("f16" / "bf16"): the down-cast-on-stash entry points (float32 input, 16-bit values)."""
     n = x.numel()
     cap = n if capacity is None else capacity
     bitmap = Guarded((n + 31) // 32, torch.int32)
-    values = Guarded(cap, x.dtype)
+    values = Guarded(cap, TDT[narrow] if narrow else x.dtype)
     prefix = Guarded((n + 4095) // 4096, torch.int64)
     nnz = Guarded(1, torch.int64)
     status = Guarded(1, torch.int32)
@@ -73,12 +74,18 @@ def gpu_compress(x: torch.Tensor, relu: bool = False, want_y: bool = False, capa
             y_t = y.inner
         else:
             y_t = None
-        if tau is not None:
+        if narrow:
+            B.bt_prune_fwd_compress_narrow(x, 0.0 if tau is None else tau, y_t, bitmap.inner, values.inner, prefix.inner,
+                                           nnz.inner, ws, status.inner, n=n, values_capacity=cap)
+        elif tau is not None:
             B.bt_prune_fwd_compress(x, tau, y_t, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws,
                                     status.inner, n=n, values_capacity=cap)
         else:
             B.bt_relu_fwd_compress(x, y_t, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws, status.inner,
                                    n=n, values_capacity=cap)
+    elif narrow:
+        B.bt_compress_narrow(x, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws, status.inner,
+                             n=n, values_capacity=cap)
     else:
         B.bt_compress(x, bitmap.inner, values.inner, prefix.inner, nnz.inner, ws, status.inner,
                       n=n, values_capacity=cap)
