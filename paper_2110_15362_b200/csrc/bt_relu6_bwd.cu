@@ -7,7 +7,10 @@
 // in 16-byte vectors.
 //
 // One warp, one quarter chunk (1024 elements = 32 bitmap words); a lane owns kE
-// consecutive elements per step, i.e. kE consecutive bits of one word.
+// consecutive elements per step, i.e. kE consecutive bits of one word.  The
+// gradient is fetched kBlk steps at a time, ahead of the gather that depends on
+// the stash (all steps at once for 2- and 4-byte elements; 8-byte elements take
+// four rounds, or the registers would halve the occupancy).
 #include "bt_internal.cuh"
 
 namespace bt {
@@ -15,7 +18,7 @@ namespace {
 
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 
-template <typename U, int DT, int kE, int kWarps>
+template <typename U, int DT, int kE, int kBlk, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
 relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values, const uint64_t *__restrict__ prefix,
                  const U *gout, const uint64_t n, U *gin)   // gin may alias gout
@@ -25,6 +28,7 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     constexpr int kWordsPerStep = kE;
     constexpr int kSteps        = 32 / kWordsPerStep;
     static_assert(kE % kVec == 0 && 32 % kE == 0 && kE < 32, "a lane takes whole vectors of one word");
+    static_assert(kSteps % kBlk == 0, "whole rounds");
 
     const uint32_t lane        = threadIdx.x & 31u;
     const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
@@ -37,34 +41,37 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     const uint64_t w0          = chunk * 128 + 4 * lane;
     const uint64_t e0          = warp_global << 10;
 
-    // the quarter of the gradient first: these loads do not depend on the stash
-    U g[kSteps][kE];
+    // kBlk steps of the gradient: these loads do not depend on the stash
+    U    g[kBlk][kE];
+    auto fetch = [&](const int k0) {
 #pragma unroll
-    for (int k = 0; k < kSteps; ++k) {
-        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+        for (int k = 0; k < kBlk; ++k) {
+            const uint64_t eo = e0 + static_cast<uint64_t>(k0 + k) * (32 * kE) + lane * kE;
 #pragma unroll
-        for (int v = 0; v < kE / kVec; ++v) {
-            const uint64_t at = eo + v * kVec;
-            U             *gv = g[k] + v * kVec;
-            if (at + kVec <= n) {
-                const uint4 pack = *reinterpret_cast<const uint4 *>(gout + at);
-                if constexpr (kVec == 2) {
-                    gv[0] = pack.x | (static_cast<uint64_t>(pack.y) << 32);
-                    gv[1] = pack.z | (static_cast<uint64_t>(pack.w) << 32);
-                } else if constexpr (kVec == 4) {
-                    gv[0] = pack.x, gv[1] = pack.y, gv[2] = pack.z, gv[3] = pack.w;
+            for (int v = 0; v < kE / kVec; ++v) {
+                const uint64_t at = eo + v * kVec;
+                U             *gv = g[k] + v * kVec;
+                if (at + kVec <= n) {
+                    const uint4 pack = *reinterpret_cast<const uint4 *>(gout + at);
+                    if constexpr (kVec == 2) {
+                        gv[0] = pack.x | (static_cast<uint64_t>(pack.y) << 32);
+                        gv[1] = pack.z | (static_cast<uint64_t>(pack.w) << 32);
+                    } else if constexpr (kVec == 4) {
+                        gv[0] = pack.x, gv[1] = pack.y, gv[2] = pack.z, gv[3] = pack.w;
+                    } else {
+                        gv[0] = static_cast<U>(pack.x), gv[1] = static_cast<U>(pack.x >> 16);
+                        gv[2] = static_cast<U>(pack.y), gv[3] = static_cast<U>(pack.y >> 16);
+                        gv[4] = static_cast<U>(pack.z), gv[5] = static_cast<U>(pack.z >> 16);
+                        gv[6] = static_cast<U>(pack.w), gv[7] = static_cast<U>(pack.w >> 16);
+                    }
                 } else {
-                    gv[0] = static_cast<U>(pack.x), gv[1] = static_cast<U>(pack.x >> 16);
-                    gv[2] = static_cast<U>(pack.y), gv[3] = static_cast<U>(pack.y >> 16);
-                    gv[4] = static_cast<U>(pack.z), gv[5] = static_cast<U>(pack.z >> 16);
-                    gv[6] = static_cast<U>(pack.w), gv[7] = static_cast<U>(pack.w >> 16);
-                }
-            } else {
 #pragma unroll
-                for (int j = 0; j < kVec; ++j) gv[j] = at + j < n ? gout[at + j] : U(0);
+                    for (int j = 0; j < kVec; ++j) gv[j] = at + j < n ? gout[at + j] : U(0);
+                }
             }
         }
-    }
+    };
+    fetch(0);
 
     uint4 w4 = make_uint4(0, 0, 0, 0);
     if (w0 + 3 < words_total) {
@@ -100,8 +107,10 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
 
     const uint32_t shift = (lane % kLanesPerWord) * kE;
 #pragma unroll
-    for (int k = 0; k < kSteps; ++k) {
-        const int      from = k * kWordsPerStep + lane / kLanesPerWord;
+    for (int kk = 0; kk < kSteps; ++kk) {
+        const int k = kk % kBlk;                              // row of g
+        if (kk != 0 && k == 0) fetch(kk);
+        const int      from = kk * kWordsPerStep + lane / kLanesPerWord;
         const uint32_t w    = __shfl_sync(kFull, word, from);
         const uint32_t wex  = __shfl_sync(kFull, excl, from);
         const uint32_t bits = (w >> shift) & ((1u << kE) - 1u);
@@ -115,7 +124,7 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
             off += set;
             g[k][j] = pass ? g[k][j] : U(0);
         }
-        const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
+        const uint64_t eo = e0 + static_cast<uint64_t>(kk) * (32 * kE) + lane * kE;
 #pragma unroll
         for (int v = 0; v < kE / kVec; ++v) {
             const uint64_t at = eo + v * kVec;
@@ -141,7 +150,7 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     }
 }
 
-template <typename U, int DT, int kE>
+template <typename U, int DT, int kE, int kBlk>
 cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
                          uint64_t n, void *gin, cudaStream_t stream)
 {
@@ -149,7 +158,7 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint6
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-    relu6_bwd_kernel<U, DT, kE, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
+    relu6_bwd_kernel<U, DT, kE, kBlk, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
         bitmap, static_cast<const U *>(values), prefix, static_cast<const U *>(gout), n, static_cast<U *>(gin));
     return cudaGetLastError();
 }
@@ -160,10 +169,10 @@ cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const u
                              uint64_t n, int dtype, void *gin, cudaStream_t stream)
 {
     switch (dtype) {
-    case BT_F64: return launch_typed<uint64_t, BT_F64, 2>(bitmap, values, prefix, gout, n, gin, stream);
-    case BT_F32: return launch_typed<uint32_t, BT_F32, 4>(bitmap, values, prefix, gout, n, gin, stream);
-    case BT_F16: return launch_typed<uint16_t, BT_F16, 8>(bitmap, values, prefix, gout, n, gin, stream);
-    default: return launch_typed<uint16_t, BT_BF16, 8>(bitmap, values, prefix, gout, n, gin, stream);
+    case BT_F64: return launch_typed<uint64_t, BT_F64, 2, 2>(bitmap, values, prefix, gout, n, gin, stream);
+    case BT_F32: return launch_typed<uint32_t, BT_F32, 4, 2>(bitmap, values, prefix, gout, n, gin, stream);
+    case BT_F16: return launch_typed<uint16_t, BT_F16, 8, 4>(bitmap, values, prefix, gout, n, gin, stream);
+    default: return launch_typed<uint16_t, BT_BF16, 8, 4>(bitmap, values, prefix, gout, n, gin, stream);
     }
 }
 
