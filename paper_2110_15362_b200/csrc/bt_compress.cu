@@ -291,7 +291,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
 
     const uint32_t tid  = threadIdx.x;
     const uint32_t lane = tid & 31u;
-    const uint32_t warp = tid >> 5;
+    // broadcast from lane 0 so that the compiler knows the role branches below are warp-uniform and may keep
+    // warp-uniform values (ballots, their counts, the running output position) on the uniform datapath
+    const uint32_t warp = __shfl_sync(kFull, tid >> 5, 0);
     const uint32_t G    = gridDim.x;
     const uint32_t cta  = blockIdx.x;
     const U *const src  = static_cast<const U *>(a.src);
