@@ -199,3 +199,72 @@ def test_cfg5_mobilenetv2_batch128_forward_then_reverse(oracle):
         x = W.cfg5_layer(i, shape, fractions[i], DEV).reshape(-1)
         assert torch.equal(bits_of(back), bits_of(x))
         del back, x
+
+
+def test_more_than_two_to_the_32_elements(oracle):
+    """Element indices, bitmap word indices and packed offsets beyond 32 bits: a bf16 tensor of 2^32 + 70001
+    elements (8.6 GB dense, ragged against words, chunks and tiles).  Checked in slices with torch, on sampled
+    chunks with the oracle (the last chunks lie beyond element 2^32), and through every kernel of the path."""
+    n = (1 << 32) + 70001
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 << 30:
+        pytest.skip("needs about 45 GB of free device memory")
+    step = 1 << 28
+    pre = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    for k, lo in enumerate(range(0, n, step)):                # seeded, slice by slice
+        m = min(step, n - lo)
+        pre[lo:lo + m] = torch.randn(m, generator=torch.Generator(device=DEV).manual_seed(9000 + k), device=DEV,
+                                     dtype=torch.float32).to(torch.bfloat16)
+    st = B.Stash(n, pre.dtype, DEV)
+    ws = B.new_workspace(n, DEV)
+    y = torch.empty_like(pre)
+    B.bt_relu_fwd_compress(pre, y, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+    torch.cuda.synchronize()
+    assert st.status == B.BT_OK
+    nnz = st.nnz
+    # whole tensor, slice by slice: the dense output, the bitmap, the prefix array and the packed values
+    total = 0
+    for lo in range(0, n, step):
+        hi = min(n, lo + step)
+        y_ref = torch.clamp_min(pre[lo:hi].float(), 0.0).to(torch.bfloat16)
+        y_ref = torch.where(y_ref == 0, torch.zeros_like(y_ref), y_ref)                 # +0 for -0.0
+        assert torch.equal(bits_of(y[lo:hi]), bits_of(y_ref))
+        mask = bits_of(y_ref) != 0
+        assert torch.equal(st.bitmap[lo // 32:(hi + 31) // 32], torch_bitmap(mask))       # slices start on word boundaries
+        c0, c1 = lo // 4096, (hi + 4095) // 4096
+        assert torch.equal(st.chunk_prefix[c0:c1], torch_prefix(mask) + total)
+        cnt = int(mask.sum().item())
+        assert torch.equal(bits_of(st.values[total:total + cnt]), bits_of(y_ref)[mask])
+        total += cnt
+        del y_ref, mask
+    assert total == nnz and nnz > (1 << 31)                  # packed offsets pass 2^31 as well
+    check_sampled_chunks(oracle, st, y, None, seed=5, samples=16)
+    chunks = (n + 4095) // 4096
+    for c in (chunks - 1, chunks - 2, (1 << 32) // 4096, (1 << 32) // 4096 - 1):          # around element 2^32 and the ragged end
+        lo, hi = c * 4096, min(n, (c + 1) * 4096)
+        ref = oracle.compress(W.raw_numpy(y[lo:hi]))
+        start = int(st.chunk_prefix[c].item())
+        assert np.array_equal(W.raw_numpy(st.bitmap[lo // 32:(hi + 31) // 32]).view(np.uint32), ref.bitmap)
+        assert np.array_equal(W.raw_numpy(st.values[start:start + ref.nnz]), ref.values)
+    # the plain compressor on y gives the same stash
+    st2 = B.Stash(n, pre.dtype, DEV)
+    B.bt_compress(y, st2.bitmap, st2.values, st2.chunk_prefix, st2.nnz_out, ws, st2.dev_status)
+    assert st2.status == B.BT_OK and st2.nnz == nnz
+    assert torch.equal(st2.bitmap, st.bitmap) and torch.equal(st2.chunk_prefix, st.chunk_prefix)
+    assert torch.equal(bits_of(st2.values[:nnz]), bits_of(st.values[:nnz]))
+    del st2
+    # restore, masked gradient (in place), masked gather
+    back = torch.empty_like(y)
+    B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, back)
+    assert torch.equal(bits_of(back), bits_of(y))
+    B.bt_relu_bwd_from_bitmap(st.bitmap, pre, back)           # the pre-activation doubles as the gradient
+    for lo in range(0, n, step):
+        hi = min(n, lo + step)
+        assert torch.equal(bits_of(back[lo:hi]), bits_of(torch.where(bits_of(y[lo:hi]) != 0, pre[lo:hi],
+                                                                     torch.zeros((), device=DEV, dtype=pre.dtype))))
+    vals = torch.empty(nnz, dtype=pre.dtype, device=DEV)
+    B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, None, vals)
+    torch.cuda.synchronize()
+    assert torch.equal(bits_of(vals), bits_of(st.values[:nnz]))   # where a bit is set, pre == y
+    del pre, y, back, vals, st, ws
+    torch.cuda.empty_cache()
