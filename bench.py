@@ -368,6 +368,8 @@ def large_tensor_kernels(dev, peak_gbs: float):
                 ms, best = time_call(lambda: B.bt_prune_fwd_compress_narrow(pre, 0.0, None, st.bitmap, v16, st.chunk_prefix,
                                                                             st.nnz_out, ws, st.dev_status))
                 res["bt_prune_fwd_compress_narrow_" + to] = (ms, best, by16)
+                ms, best = time_call(lambda: B.bt_decompress_widen(st.bitmap, v16, st.chunk_prefix, dense))
+                res["bt_decompress_widen_" + to] = (ms, best, by16)
                 del v16
         # double-mask form (a "next" row): the stash of x masks a dense tensor of the same shape
         B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)

@@ -177,6 +177,17 @@ int bt_prune_fwd_compress_narrow(const void *x, uint64_t n, int to_dtype, float 
                                  int32_t *dev_status, void *stream);
 
 /*
+ * Algorithm 2 on a narrowed stash, straight into a BT_F32 tensor: dense_out[i]
+ * = the stashed 16-bit value of element i (from_dtype: BT_F16 or BT_BF16)
+ * widened to binary32 -- exact for both types, a NaN keeps its sign and its
+ * payload moves into the upper mantissa bits -- where bit i is set, +0
+ * elsewhere.  The result equals bt_decompress in from_dtype followed by a cast
+ * to binary32.  Other parameters as bt_decompress.
+ */
+int bt_decompress_widen(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix,
+                        uint64_t n, int from_dtype, void *dense_out, void *stream);
+
+/*
  * ReLU6 (the activation of the MobileNetV2 family among the paper's models) fused with Algorithm 1:
  * y[i] = (x[i] <= 0) ? +0 : (x[i] >= 6 ? 6 : x[i]) under IEEE comparison of the exactly widened element
  * (a NaN fails both comparisons and is kept), stashed in the same pass.  Parameters as

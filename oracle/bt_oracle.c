@@ -443,3 +443,28 @@ uint64_t oracle_narrow_compress(const void *x, uint64_t n, int to_kind, int fuse
     }
     return j;
 }
+
+/* Restoring a narrowed stash into a binary32 tensor: Algorithm 2 with each
+ * 16-bit value widened on the way (binary16 -> binary32 and bfloat16 ->
+ * binary32 are both exact, NaN payloads shift into the upper mantissa bits);
+ * elements whose bit is clear are +0. */
+void oracle_widen_decompress(const uint32_t *bitmap, const uint16_t *values, uint64_t n,
+                             int from_kind, void *dense_f32)
+{
+    unsigned char *out = (unsigned char *)dense_f32;
+    uint64_t j = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        uint32_t u = 0;
+        if ((bitmap[i >> 5] >> (i & 31)) & 1u) {
+            uint16_t h = values[j];
+            j += 1;
+            if (from_kind == ORACLE_F16) {
+                float f = oracle_half_to_float(h);
+                memcpy(&u, &f, 4);
+            } else {
+                u = (uint32_t)h << 16;
+            }
+        }
+        memcpy(out + 4 * i, &u, 4);
+    }
+}

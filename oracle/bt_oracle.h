@@ -93,6 +93,10 @@ uint64_t oracle_compressed_bytes(uint64_t n, uint64_t nnz, int elem_size);
 uint64_t oracle_narrow_compress(const void *x, uint64_t n, int to_kind, int fused, float tau,
                                 void *y, uint32_t *bitmap, uint16_t *values, uint64_t *prefix);
 
+/* Algorithm 2 on a narrowed stash, each value widened exactly to binary32 */
+void oracle_widen_decompress(const uint32_t *bitmap, const uint16_t *values, uint64_t n,
+                             int from_kind, void *dense_f32);
+
 /* binary32 pattern -> binary16 / bfloat16 pattern: round to nearest, ties to
  * even; overflow to infinity; every NaN to 0x7FFF */
 uint16_t oracle_float_to_half(uint32_t bits);

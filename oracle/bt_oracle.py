@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
         L.oracle_narrow_compress.restype = u64
         L.oracle_narrow_compress.argtypes = [vp, u64, i32, i32, ctypes.c_float, vp, vp, vp, vp]
+        L.oracle_widen_decompress.restype = None
+        L.oracle_widen_decompress.argtypes = [vp, vp, u64, i32, vp]
         L.oracle_float_to_half.restype = ctypes.c_uint16
         L.oracle_float_to_half.argtypes = [ctypes.c_uint32]
         L.oracle_float_to_bfloat16.restype = ctypes.c_uint16
@@ -204,6 +206,15 @@ def narrow_compress(x: np.ndarray, to_kind: str, fused: bool = False, tau: float
     nnz = int(lib().oracle_narrow_compress(_ptr(x), n, KINDS[to_kind], int(fused), float(np.float32(tau)), _ptr(y),
                                             _ptr(bitmap), _ptr(values), _ptr(prefix)))
     return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
+
+
+def widen_decompress(c: Compressed, from_kind: str) -> np.ndarray:
+    """The binary32 tensor (raw uint32 patterns) a narrowed stash restores to."""
+    assert c.values.dtype == np.uint16 and from_kind in ("f16", "bf16")
+    out = np.full(c.n, 0xDEADBEEF, dtype=np.uint32)
+    vals = np.ascontiguousarray(c.values) if c.values.size else np.zeros(1, np.uint16)
+    lib().oracle_widen_decompress(_ptr(c.bitmap), _ptr(vals), c.n, KINDS[from_kind], _ptr(out))
+    return out
 
 
 def float_to_half(bits: int) -> int:

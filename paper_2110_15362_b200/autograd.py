@@ -19,6 +19,12 @@ Getting the exact ``nnz`` to size the values costs one device-to-host read per p
 pre-allocated arena (the ``*_arena`` entry points): no host read in the forward pass; the device status
 words are checked once, when the backward pass first asks for a tensor.  The cursor is reset on entering
 the context, so one context entry covers one forward / backward pass.
+
+``relu6_stash(x)`` is the same for ReLU6 (``bt_relu6_fwd_compress`` / ``bt_relu6_bwd_from_stash``; its backward
+pass reads the stashed values as well, which are the ones the next layer's saved input shares).  With
+``stash_saved_activations(narrow=torch.float16)`` (or ``torch.bfloat16``) float32 activations are stashed with
+16-bit values (``bt_compress_narrow`` / ``bt_decompress_widen``): lossy -- what the backward pass gets back is
+the activation rounded to the narrow type -- and not combined with the arena.
 """
 from __future__ import annotations
 
@@ -29,7 +35,7 @@ import torch
 
 from . import binding as B
 
-__all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash"]
+__all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash", "relu6_stash", "ReLU6Stash"]
 
 
 class PackedActivation:
@@ -54,13 +60,15 @@ class PackedActivation:
     def nbytes(self) -> int:
         """Bytes of the stash (arena mode: reads nnz from the device)."""
         nnz = int(self.nnz.item()) if isinstance(self.nnz, torch.Tensor) else self.nnz
-        return B.bt_compressed_bytes(self.numel, nnz, self.dtype)
+        return B.bt_compressed_bytes(self.numel, nnz, self.dtype if self.values is None else self.values.dtype)
 
     def unpack(self) -> torch.Tensor:
         out = torch.empty(self.shape, dtype=self.dtype, device=self.device)
         if self.arena is not None:
             self.owner.check_statuses()
             B.bt_decompress_arena(self.bitmap, self.arena, self.offset, self.chunk_prefix, out.view(-1))
+        elif self.values.dtype != self.dtype:          # a narrowed stash of a float32 tensor
+            B.bt_decompress_widen(self.bitmap, self.values, self.chunk_prefix, out.view(-1))
         else:
             B.bt_decompress(self.bitmap, self.values, self.chunk_prefix, out.view(-1))
         return out
@@ -88,16 +96,27 @@ class _Scratch:
         return v
 
 
-def _compress(flat: torch.Tensor, scratch: _Scratch, relu_into: Optional[torch.Tensor] = None):
-    """Runs the (fused) compressor on a flat tensor; returns bitmap, exact-size values, prefix, nnz."""
+def _compress(flat: torch.Tensor, scratch: _Scratch, relu_into: Optional[torch.Tensor] = None,
+              narrow: Optional[torch.dtype] = None, relu6: bool = False):
+    """Runs the (fused) compressor on a flat tensor; returns bitmap, exact-size values, prefix, nnz.  `narrow`:
+    16-bit dtype of the stashed values of a float32 tensor.  `relu6`: the fused form is ReLU6 (needs relu_into)."""
     n, dev = flat.numel(), flat.device
+    if narrow is not None and flat.dtype != torch.float32:
+        narrow = None
     bitmap = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
     prefix = torch.empty((n + B.CHUNK - 1) // B.CHUNK, dtype=torch.int64, device=dev)
     nnz_out = torch.empty(1, dtype=torch.int64, device=dev)
     status = torch.empty(1, dtype=torch.int32, device=dev)
-    full = scratch.full_values(n, flat.dtype, dev)
+    full = scratch.full_values(n, narrow or flat.dtype, dev)
     ws = scratch.workspace(n, dev)
-    if relu_into is None:
+    if relu6:
+        B.bt_relu6_fwd_compress(flat, relu_into, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
+    elif narrow is not None and relu_into is None:
+        B.bt_compress_narrow(flat, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
+    elif narrow is not None:
+        B.bt_prune_fwd_compress_narrow(flat, 0.0, relu_into, bitmap, full, prefix, nnz_out, ws, status, n=n,
+                                       values_capacity=n)
+    elif relu_into is None:
         B.bt_compress(flat, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
     else:
         B.bt_relu_fwd_compress(flat, relu_into, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
@@ -128,11 +147,16 @@ def _compress_arena(flat: torch.Tensor, owner, relu_into: Optional[torch.Tensor]
 class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
     """Context manager: saved activations are kept compressed between the forward and the backward pass.
     `arena_bytes`: keep all values in one pre-allocated arena of that size behind a device-side cursor (no
-    host read per tensor; a RuntimeError at the first unpack if the arena was too small)."""
+    host read per tensor; a RuntimeError at the first unpack if the arena was too small).  `narrow`
+    (torch.float16 / torch.bfloat16): float32 activations are stashed with values of that type (lossy)."""
 
     def __init__(self, min_numel: int = 1 << 14, min_saving: float = 0.1, arena_bytes: Optional[int] = None,
-                 device="cuda"):
-        self.min_numel, self.min_saving = min_numel, min_saving
+                 device="cuda", narrow: Optional[torch.dtype] = None):
+        if narrow not in (None, torch.float16, torch.bfloat16):
+            raise ValueError("narrow must be torch.float16 or torch.bfloat16")
+        if narrow is not None and arena_bytes is not None:
+            raise ValueError("the narrowing forms have no arena variant")
+        self.min_numel, self.min_saving, self.narrow = min_numel, min_saving, narrow
         self.arena = self.cursor = None
         self.statuses: list = []
         if arena_bytes is not None:
@@ -189,8 +213,8 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
             self.share(t, packed)
             self.dense_bytes += n * es
             return packed
-        bitmap, values, prefix, nnz = _compress(t.detach().view(-1), self.scratch)
-        if B.bt_compressed_bytes(n, nnz, t.dtype) > (1.0 - self.min_saving) * n * es:
+        bitmap, values, prefix, nnz = _compress(t.detach().view(-1), self.scratch, narrow=self.narrow)
+        if B.bt_compressed_bytes(n, nnz, values.dtype) > (1.0 - self.min_saving) * n * es:
             return t                                  # too few zeros: the stash would not be smaller
         packed = PackedActivation(bitmap, values, prefix, tuple(t.shape), t.dtype, t.device, nnz)
         self.share(t, packed)
@@ -233,7 +257,8 @@ class ReLUStash(torch.autograd.Function):
             hooks.dense_bytes += y.numel() * y.element_size()
             return y
         scratch = hooks.scratch if hooks is not None else _Scratch()
-        bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1))
+        bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1),
+                                                narrow=hooks.narrow if hooks is not None else None)
         ctx.save_for_backward(bitmap)     # released with the graph, like any saved tensor
         if hooks is not None:
             # the next layer will save y as its input: hand it this stash instead of compressing y again
@@ -257,3 +282,40 @@ def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None,
     the following layer reuse the stash for its saved input.  ``inplace=True`` writes the activation over ``x``
     (like ``torch.relu_``: only where ``x`` is not needed again, e.g. the output of a convolution)."""
     return ReLUStash.apply(x, hooks, inplace)
+
+
+class ReLU6Stash(torch.autograd.Function):
+    """ReLU6 with the stash fused into its forward pass; the backward pass reads the bitmap and the stashed
+    values (a stored 6 marks a saturated unit).  Always exact-size values (one host read), also inside an
+    arena context; never narrowed (the backward pass compares the stored values with 6)."""
+
+    @staticmethod
+    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False):
+        if inplace and x.is_contiguous():
+            xc = y = x
+            ctx.mark_dirty(x)
+        else:
+            xc = x.contiguous()
+            y = torch.empty_like(xc)
+        scratch = hooks.scratch if hooks is not None else _Scratch()
+        bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1), relu6=True)
+        ctx.save_for_backward(bitmap, values, prefix)
+        if hooks is not None:
+            packed = PackedActivation(bitmap, values, prefix, tuple(y.shape), y.dtype, y.device, nnz)
+            hooks.share(y, packed)
+            hooks.packed_bytes += packed.nbytes()
+            hooks.dense_bytes += y.numel() * y.element_size()
+        return y
+
+    @staticmethod
+    def backward(ctx, grad: torch.Tensor):
+        g = grad.contiguous()
+        gin = torch.empty_like(g)
+        bitmap, values, prefix = ctx.saved_tensors
+        B.bt_relu6_bwd_from_stash(bitmap, values, prefix, g.view(-1), gin.view(-1))
+        return gin, None, None
+
+
+def relu6_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False) -> torch.Tensor:
+    """ReLU6 through the fused kernel; arguments as for ``relu_stash``."""
+    return ReLU6Stash.apply(x, hooks, inplace)

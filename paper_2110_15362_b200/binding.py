@@ -29,7 +29,7 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
            "bt_prune_fwd_compress", "bt_mask_compress", "bt_compress_arena", "bt_prune_fwd_compress_arena",
            "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
-           "bt_prune_fwd_compress_narrow")
+           "bt_prune_fwd_compress_narrow", "bt_decompress_widen")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.bt_compress_narrow.restype = i32
         L.bt_prune_fwd_compress_narrow.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
         L.bt_prune_fwd_compress_narrow.restype = i32
+        L.bt_decompress_widen.argtypes = [vp, vp, vp, u64, i32, vp, vp]
+        L.bt_decompress_widen.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -206,6 +208,16 @@ def bt_prune_fwd_compress_narrow(x: torch.Tensor, tau: float, y_out: Optional[to
                                             _ptr(bitmap), _ptr(values), cap, _ptr(chunk_prefix), _ptr(nnz_out),
                                             _ptr(workspace), _nbytes(workspace), _ptr(dev_status), _stream(stream))
     return _check("bt_prune_fwd_compress_narrow", st, check)
+
+
+def bt_decompress_widen(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor, dense_out: torch.Tensor,
+                        *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """Restores a narrowed stash (16-bit `values`) into a float32 tensor."""
+    n = dense_out.numel() if n is None else n
+    assert dense_out.dtype == torch.float32
+    st = lib().bt_decompress_widen(_ptr(bitmap), _ptr(values), _ptr(chunk_prefix), n, DTYPE_CODE[values.dtype],
+                                   _ptr(dense_out), _stream(stream))
+    return _check("bt_decompress_widen", st, check)
 
 
 def bt_mask_compress(x: torch.Tensor, mask_bitmap: torch.Tensor, mask_chunk_prefix: torch.Tensor,

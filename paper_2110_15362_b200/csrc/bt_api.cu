@@ -209,6 +209,20 @@ int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *ch
                : BT_ERR_CUDA;
 }
 
+int bt_decompress_widen(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix, uint64_t n,
+                        int from_dtype, void *dense_out, void *stream)
+{
+    if (from_dtype != BT_F16 && from_dtype != BT_BF16) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !chunk_prefix || !dense_out) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
+        return BT_ERR_ALIGN;
+    return bt::launch_decompress_widen(bitmap, values, chunk_prefix, n, from_dtype, dense_out,
+                                       static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
 int bt_mask_compress(const void *x, uint64_t n, int dtype, const uint32_t *mask_bitmap, const uint64_t *mask_chunk_prefix,
                      void *y_out, void *values, uint64_t values_capacity, void *stream)
 {

@@ -13,6 +13,8 @@
 //     elements, i.e. kE consecutive bits of one word; the rank of its first set
 //     bit is  chunk base + quarter base + word offset + popc(lower bits of the
 //     word),  and the set bits gather from values[] at consecutive addresses.
+#include <type_traits>
+
 #include "bt_internal.cuh"
 
 namespace bt {
@@ -21,9 +23,25 @@ namespace {
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 
 // kE: elements a lane decodes per step (a multiple of one 16-byte vector: 2 for 8-byte, 4 for 4-byte, 8 for 2-byte elements)
-template <typename U, int kE, int kGrp, int kWarps>
+// WIDEN: 0, or the 16-bit type of the stashed values of a binary32 tensor (1 binary16, 2 bfloat16): the value
+// is widened exactly on its way out (the restore side of the down-cast on stash).
+template <int WIDEN>
+__device__ __forceinline__ uint32_t widened(const uint16_t h)
+{
+    if constexpr (WIDEN == 1) {
+        float f;
+        asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(h));
+        // a NaN keeps its sign and payload (written out, not left to the conversion instruction)
+        const uint32_t nan = (static_cast<uint32_t>(h & 0x8000u) << 16) | 0x7F800000u | (static_cast<uint32_t>(h & 0x3FFu) << 13);
+        return (h & 0x7FFFu) > 0x7C00u ? nan : __float_as_uint(f);
+    } else {
+        return static_cast<uint32_t>(h) << 16;
+    }
+}
+
+template <typename U, int kE, int kGrp, int kWarps, int WIDEN = 0>
 __global__ void __launch_bounds__(kWarps * 32)
-decompress_kernel(const uint32_t *__restrict__ bitmap, const U *values,
+decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<WIDEN != 0, uint16_t, U> *values,
                   const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
                   U *__restrict__ out)
 {
@@ -54,7 +72,8 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const U *values,
     }
     const uint64_t chunk_base = prefix[chunk];
     // arena form: the packed values start *values_offset bytes into `values`
-    if (values_offset) values = reinterpret_cast<const U *>(reinterpret_cast<const unsigned char *>(values) + *values_offset);
+    using V = std::conditional_t<WIDEN != 0, uint16_t, U>;   // type of a stashed value
+    if (values_offset) values = reinterpret_cast<const V *>(reinterpret_cast<const unsigned char *>(values) + *values_offset);
 
     // non-zeros of the chunk in front of this quarter
     uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
@@ -74,7 +93,7 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const U *values,
         if (lane >= static_cast<uint32_t>(o)) incl += u;
     }
     const uint32_t excl = incl - __popc(word);
-    const U *const vp   = values + (chunk_base + before);   // packed values of this quarter
+    const V *const vp   = values + (chunk_base + before);   // packed values of this quarter
 
     const uint64_t e0    = warp_global << 10;               // first element of the quarter
     const uint32_t shift = (lane % kLanesPerWord) * kE;     // which kE-bit group of the word
@@ -97,7 +116,8 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const U *values,
 #pragma unroll
         for (int j = 0; j < kE; ++j) {
             const bool set = (bits >> j) & 1u;
-            e[kk][j]       = set ? vp[off] : U(0);
+            if constexpr (WIDEN != 0) e[kk][j] = set ? widened<WIDEN>(vp[off]) : 0u;
+            else e[kk][j] = set ? vp[off] : U(0);
             off += set;
         }
     }
@@ -145,6 +165,22 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint6
 }
 
 }  // namespace
+
+cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *prefix, uint64_t n,
+                                    int from_dtype, void *out_f32, cudaStream_t stream)
+{
+    constexpr int  kWarps   = 8;
+    const uint64_t quarters = (n + 1023) >> 10;
+    const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
+    if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    const auto *v = static_cast<const uint16_t *>(values16);
+    auto       *o = static_cast<uint32_t *>(out_f32);
+    if (from_dtype == BT_F16)
+        decompress_kernel<uint32_t, 4, 8, kWarps, 1><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, nullptr, prefix, n, o);
+    else
+        decompress_kernel<uint32_t, 4, 8, kWarps, 2><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, nullptr, prefix, n, o);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                               const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t stream)

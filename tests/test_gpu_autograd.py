@@ -162,3 +162,57 @@ def test_vgg_demo_runs_and_losses_agree(A, capsys):
     assert out["plain"]["loss"] == pytest.approx(out["stashed"]["loss"], rel=1e-3)
     assert out["plain"]["loss"] == pytest.approx(out["stashed_arena"]["loss"], rel=1e-3)
     assert 0.3 < out["saved_activation_bytes_over_dense"] < 0.8
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_relu6_stash_gradients_are_bit_identical(A, dtype):
+    weights = mlp(512, 4, seed=5, dtype=dtype)
+    x = 3 * torch.randn(2048, 512, device="cuda", dtype=dtype, generator=torch.Generator(device="cuda").manual_seed(6))
+    relu6 = torch.nn.functional.relu6
+    ref_loss, ref = run(weights, x, relu6)
+    assert int((relu6(x @ weights[0]) == 6).sum()) > 1000           # the clamp is exercised
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        loss1, g1 = run(weights, x, lambda t: A.relu6_stash(t, hooks))
+        assert hooks.packed_bytes < 0.7 * hooks.dense_bytes
+    loss2, g2 = run(weights, x, A.relu6_stash)                      # without the hooks
+    with A.stash_saved_activations(min_numel=1024, arena_bytes=64 << 20) as hooks:
+        loss3, g3 = run(weights, x, lambda t: A.relu6_stash(t, hooks))      # inside an arena context: exact-size stashes
+    for loss, grads in ((loss1, g1), (loss2, g2), (loss3, g3)):
+        assert torch.equal(loss, ref_loss)
+        for a, b in zip(grads, ref):
+            assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("narrow", [torch.float16, torch.bfloat16])
+def test_narrowed_stash_is_the_rounded_activation(A, narrow):
+    """Lossy by design: what the backward pass sees is the activation rounded to the narrow type, so the
+    gradients equal those of a plain step whose saved activations are rounded the same way."""
+    weights = mlp(512, 3, seed=7)
+    x = torch.randn(2048, 512, device="cuda", generator=torch.Generator(device="cuda").manual_seed(8))
+    hooks = A.stash_saved_activations(min_numel=1024, narrow=narrow)
+    t = torch.relu(torch.randn(64, 4096, device="cuda"))
+    p = hooks._pack(t)
+    assert p.values.dtype == narrow and p.nnz == int(torch.count_nonzero(t))
+    assert torch.equal(hooks._unpack(p), t.to(narrow).float())
+    assert p.nbytes() == B.bt_compressed_bytes(t.numel(), p.nnz, narrow)
+
+    class RoundSaved(torch.autograd.graph.saved_tensors_hooks):     # the plain-PyTorch statement of the same thing
+        def __init__(self):
+            super().__init__(lambda s: s.to(narrow).float() if s.dtype == torch.float32 and s.numel() >= 1024
+                             and not (s.requires_grad and s.is_leaf) else s, lambda s: s)
+
+    def relu_by_mask(t):                                            # saves a boolean mask, which no hook rounds
+        return torch.where(t > 0, t, torch.zeros((), device=t.device))
+
+    with RoundSaved():
+        ref_loss, ref = run(weights, x, relu_by_mask)
+    with A.stash_saved_activations(min_numel=1024, narrow=narrow) as hooks:
+        loss1, g1 = run(weights, x, lambda t: A.relu_stash(t, hooks))
+        assert hooks.packed_bytes < 0.4 * hooks.dense_bytes         # half the zeros gone, the rest at half width
+    assert torch.equal(loss1, ref_loss)                             # the forward pass is not narrowed
+    for a, b in zip(g1, ref):
+        assert torch.equal(a, b)                                    # same rounded activations into the same GEMMs
+    _, exact = run(weights, x, torch.relu)
+    assert not torch.equal(g1[-1], exact[-1]) and torch.allclose(g1[-1], exact[-1], rtol=0.05, atol=0.5)
+    with pytest.raises(ValueError):
+        A.stash_saved_activations(narrow=narrow, arena_bytes=1 << 20)

@@ -46,6 +46,18 @@ def boundary_patterns(to_kind, seed):
     return x
 
 
+def widen_on_gpu(G, g, n, to_kind):
+    """bt_decompress_widen on a stash produced on the GPU; returns the raw binary32 patterns (guards checked)."""
+    bm = torch.from_numpy(g.bitmap.view(np.int32).copy()).cuda()
+    vals = G.from_raw(g.values if g.values.size else np.zeros(1, g.values.dtype), to_kind)
+    pf = torch.from_numpy(g.prefix.view(np.int64).copy()).cuda()
+    out = G.Guarded(n, torch.float32)
+    B.bt_decompress_widen(bm, vals, pf, out.inner, n=n)
+    torch.cuda.synchronize()
+    assert out.guards_intact()
+    return out.raw().view(np.uint32)
+
+
 @pytest.mark.parametrize("to_kind", TO)
 @pytest.mark.parametrize("n", [0, 1, 33, 1025, 4097, 16384 * 3 + 1001, 200704])
 def test_plain_form(G, oracle, to_kind, n):
@@ -57,6 +69,8 @@ def test_plain_form(G, oracle, to_kind, n):
         # the 16-bit stash goes through the unchanged decompressor
         out, ok = G.gpu_decompress(g.bitmap, g.values, g.prefix, n, to_kind)
         assert ok and np.array_equal(out.view(np.uint16), oracle.decompress(c))
+        # and through the widening one, straight into binary32
+        assert np.array_equal(widen_on_gpu(G, g, n, to_kind), oracle.widen_decompress(c, to_kind))
 
 
 @pytest.mark.parametrize("to_kind", TO)
@@ -67,6 +81,7 @@ def test_every_rounding_boundary(G, oracle, to_kind):
     assert_same(g, c)
     full = oracle.compress(x)                                        # structure: that of the binary32 stash
     assert np.array_equal(g.bitmap, full.bitmap) and np.array_equal(g.prefix, full.prefix) and g.nnz == full.nnz
+    assert np.array_equal(widen_on_gpu(G, g, x.size, to_kind), oracle.widen_decompress(c, to_kind))
 
 
 @pytest.mark.parametrize("to_kind", TO)

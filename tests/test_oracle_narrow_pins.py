@@ -108,3 +108,29 @@ def test_fused_threshold_form(oracle, to_kind, tau):
         assert c.values[np.flatnonzero(np.flatnonzero(keep.numpy()) == 7)[0]] == 0
     _, c2 = oracle.narrow_compress(x, to_kind, fused=True, tau=tau, want_y=False)
     assert np.array_equal(c2.values, c.values)
+
+
+@pytest.mark.parametrize("to_kind", ["f16", "bf16"])
+def test_widening_restore_matches_library_casts(oracle, to_kind):
+    """Restoring a narrowed stash into binary32 = the narrowed dense tensor cast up by numpy / torch (exact
+    casts), and narrowing the restored tensor again changes nothing."""
+    n = 3 * 4096 + 55
+    x = W.random_patterns(n, "f32", 0.4, seed=91)
+    _, c = oracle.narrow_compress(x, to_kind)
+    back = oracle.widen_decompress(c, to_kind)
+    dense16 = oracle.decompress(c)
+    if to_kind == "f16":
+        ref = dense16.view(np.float16).astype(np.float32).view(np.uint32)
+        nan = np.isnan(dense16.view(np.float16))
+        assert np.array_equal(back[~nan], ref[~nan])
+        assert (back[nan] == 0x7FFFE000).all() and nan.any()          # 0x7FFF widened: the payload moves up 13 bits
+    else:
+        ref = torch.from_numpy(dense16.view(np.int16)).view(torch.bfloat16).float().view(torch.int32).numpy().view(np.uint32)
+        nan = torch.isnan(torch.from_numpy(dense16.view(np.int16)).view(torch.bfloat16)).numpy()
+        assert np.array_equal(back[~nan], ref[~nan])
+        assert (back[nan] == 0x7FFF0000).all() and nan.any()
+    bits = np.unpackbits(c.bitmap.view(np.uint8), bitorder="little")[:n].astype(bool)
+    assert not back[~bits].any()
+    _, again = oracle.narrow_compress(back, to_kind)                 # idempotent on what survives as non-zero
+    keep = c.values != 0                                             # an underflow to +0 drops out; -0 keeps its bit
+    assert np.array_equal(again.values, c.values[keep])
