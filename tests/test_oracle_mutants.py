@@ -43,6 +43,8 @@ MUTANTS = {
     "narrow_bf16_ties_away_from_zero": ("if (rem > 0x8000u || (rem == 0x8000u && (q & 1u))) q += 1u;", "if (rem >= 0x8000u) q += 1u;"),
     "narrow_tests_zero_after_the_cast": ("        if (u != 0) {\n            values[j] = to_kind",
                                          "        if ((to_kind == ORACLE_F16 ? oracle_float_to_half(u) : oracle_float_to_bfloat16(u)) & 0x7FFFu) {\n            values[j] = to_kind"),
+    "widen_bf16_shifts_one_bit_short": ("            } else {\n                u = (uint32_t)h << 16;", "            } else {\n                u = (uint32_t)h << 15;"),
+    "widen_skips_the_value_counter": ("            uint16_t h = values[j];\n            j += 1;", "            uint16_t h = values[j];\n            j += (i % 89 != 0);"),
     "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
     "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
 }
@@ -75,6 +77,8 @@ def build_mutant(tmp_path, name):
     L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
     L.oracle_narrow_compress.restype = u64
     L.oracle_narrow_compress.argtypes = [vp, u64, i32, i32, ctypes.c_float, vp, vp, vp, vp]
+    L.oracle_widen_decompress.restype = None
+    L.oracle_widen_decompress.argtypes = [vp, vp, u64, i32, vp]
     return L
 
 
@@ -155,6 +159,13 @@ def pins_hold(L) -> bool:
         v16 = np.zeros(n, np.uint16)
         nn_ = L.oracle_narrow_compress(p(xn), n, to_kind, 0, 0.0, None, p(bitmap), p(v16), p(prefix))
         if nn_ != int(np.count_nonzero(xn)) or not np.array_equal(v16[:nn_], ref[xn != 0]):
+            return False
+        # and back up: the narrowed dense tensor cast to binary32 by the library (exact)
+        wide = np.empty(n, np.uint32)
+        L.oracle_widen_decompress(p(bitmap), p(v16), n, to_kind, p(wide))
+        dense16 = np.where(xn != 0, ref, 0).astype(np.uint16)
+        up = dense16.view(np.float16).astype(np.float32).view(np.uint32) if to_kind == 1 else dense16.astype(np.uint32) << 16
+        if not np.array_equal(wide, up):
             return False
     # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
     if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
