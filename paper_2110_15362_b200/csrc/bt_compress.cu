@@ -342,7 +342,8 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     if (warp == kLoadWarp) {
         // ------------------------------------------------------------ load warp (one lane)
         if (lane == 0) {
-            bool ok = true;
+            bool     ok     = true;
+            uint32_t issued = 0;
             for (uint32_t it = 0; ok; ++it) {
                 if (tile_of(it) >= num_tiles) break;
                 if (it >= static_cast<uint32_t>(kStages)) {
@@ -353,15 +354,13 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                     if (!ok) break;
                 }
                 issue_load(it);
+                issued = it + 1;
             }
-            if (!ok) {
-                // a bounded wait ran out somewhere in this CTA: before leaving, let the bulk copies that
-                // may still be in flight into its shared memory land (bounded, short)
-                for (int s = 0; s < kStages; ++s) {
-                    mbar_wait<false>(&s_full[s], 0, &s_abort, 20000000ull);
-                    mbar_wait<false>(&s_full[s], 1, &s_abort, 20000000ull);
-                }
-            }
+            // This lane stays until every bulk copy it issued has landed, whatever the other warps do (they may
+            // leave early once a bounded wait has run out somewhere): the CTA never retires with a copy into its
+            // shared memory in flight.  Only the last kStages copies can still be pending; each wait is bounded.
+            for (uint32_t it = issued > static_cast<uint32_t>(kStages) ? issued - kStages : 0; it < issued; ++it)
+                mbar_wait<false>(&s_full[it % kStages], (it / kStages) & 1u, &s_abort, 20000000ull);
             PROF_FLUSH(4, 5);
         }
         return;
