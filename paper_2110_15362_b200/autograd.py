@@ -20,6 +20,11 @@ pre-allocated arena (the ``*_arena`` entry points): no host read in the forward 
 words are checked once, when the backward pass first asks for a tensor.  The cursor is reset on entering
 the context, so one context entry covers one forward / backward pass.
 
+``double_mask(out, like)`` is the double-mask form for normalisation layers: ``out`` (e.g. a batch-norm output)
+is zeroed wherever ``like`` (the layer's input, a post-ReLU tensor) is zero, and its stash reuses the bitmap and
+the prefix array of ``like``'s stash (``bt_mask_compress``); the backward pass masks the gradient with the same
+bitmap.
+
 ``relu6_stash(x)`` is the same for ReLU6 (``bt_relu6_fwd_compress`` / ``bt_relu6_bwd_from_stash``; its backward
 pass reads the stashed values as well, which are the ones the next layer's saved input shares).  With
 ``stash_saved_activations(narrow=torch.float16)`` (or ``torch.bfloat16``) float32 activations are stashed with
@@ -35,7 +40,8 @@ import torch
 
 from . import binding as B
 
-__all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash", "relu6_stash", "ReLU6Stash"]
+__all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash", "relu6_stash", "ReLU6Stash",
+           "double_mask", "DoubleMask"]
 
 
 class PackedActivation:
@@ -319,3 +325,51 @@ class ReLU6Stash(torch.autograd.Function):
 def relu6_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False) -> torch.Tensor:
     """ReLU6 through the fused kernel; arguments as for ``relu_stash``."""
     return ReLU6Stash.apply(x, hooks, inplace)
+
+
+class DoubleMask(torch.autograd.Function):
+    """out masked by the zero pattern of `like` (double-mask batch normalisation): y = like != 0 ? out : +0.  The
+    stash of y shares the bitmap and the prefix array of like's stash and gets its own values; the backward pass
+    is the bitmap select.  `like` receives no gradient (the mask is a constant of the step)."""
+
+    @staticmethod
+    def forward(ctx, out: torch.Tensor, like: torch.Tensor, hooks: Optional[stash_saved_activations] = None,
+                inplace: bool = False):
+        if out.shape != like.shape or out.dtype != like.dtype:
+            raise ValueError("double_mask: the two tensors must agree in shape and dtype")
+        src = hooks._lookup(like) if hooks is not None else None
+        if src is None or src.arena is not None or src.values.dtype != like.dtype:
+            # no reusable stash of `like` (none yet, or one whose size only the device knows): make one
+            scratch = hooks.scratch if hooks is not None else _Scratch()
+            bitmap, values, prefix, nnz = _compress(like.detach().contiguous().view(-1), scratch)
+            src = PackedActivation(bitmap, values, prefix, tuple(like.shape), like.dtype, like.device, nnz)
+        if inplace and out.is_contiguous():
+            xc = y = out
+            ctx.mark_dirty(out)
+        else:
+            xc = out.contiguous()
+            y = torch.empty_like(xc)
+        values = torch.empty(max(src.nnz, 1), dtype=out.dtype, device=out.device)
+        B.bt_mask_compress(xc.view(-1), src.bitmap, src.chunk_prefix, y.view(-1), values, values_capacity=src.nnz)
+        ctx.save_for_backward(src.bitmap)
+        if hooks is not None:
+            packed = PackedActivation(src.bitmap, values[:src.nnz], src.chunk_prefix, tuple(y.shape), y.dtype, y.device,
+                                      src.nnz)
+            hooks.share(y, packed)
+            hooks.packed_bytes += src.nnz * y.element_size()          # bitmap and prefix are the source's
+            hooks.dense_bytes += y.numel() * y.element_size()
+        return y
+
+    @staticmethod
+    def backward(ctx, grad: torch.Tensor):
+        g = grad.contiguous()
+        gin = torch.empty_like(g)
+        (bitmap,) = ctx.saved_tensors
+        B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gin.view(-1))
+        return gin, None, None, None
+
+
+def double_mask(out: torch.Tensor, like: torch.Tensor, hooks: Optional[stash_saved_activations] = None,
+                inplace: bool = False) -> torch.Tensor:
+    """``out`` with zeros wherever ``like`` is zero, stashed under ``like``'s bitmap (see ``DoubleMask``)."""
+    return DoubleMask.apply(out, like, hooks, inplace)

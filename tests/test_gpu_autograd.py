@@ -216,3 +216,44 @@ def test_narrowed_stash_is_the_rounded_activation(A, narrow):
     assert not torch.equal(g1[-1], exact[-1]) and torch.allclose(g1[-1], exact[-1], rtol=0.05, atol=0.5)
     with pytest.raises(ValueError):
         A.stash_saved_activations(narrow=narrow, arena_bytes=1 << 20)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_double_mask_batch_norm_block(A, dtype):
+    """conv-free residual-style block: relu -> batch norm -> double mask -> linear.  Output, gradients and the
+    stash (shared bitmap, own values) equal the plain PyTorch statement y = where(h != 0, bn(h), 0)."""
+    g = torch.Generator(device="cuda").manual_seed(11)
+    x = torch.randn(4096, 256, device="cuda", dtype=dtype, generator=g)
+    w1 = (torch.randn(256, 256, device="cuda", dtype=dtype, generator=g) / 16).requires_grad_()
+    w2 = (torch.randn(256, 256, device="cuda", dtype=dtype, generator=g) / 16).requires_grad_()
+    gamma = torch.rand(256, device="cuda", dtype=dtype, generator=g).add_(0.5).requires_grad_()
+    beta = torch.randn(256, device="cuda", dtype=dtype, generator=g).requires_grad_()
+
+    def block(relu, mask):
+        h = relu(x @ w1)
+        b = torch.nn.functional.batch_norm(h, None, None, gamma, beta, training=True)
+        y = mask(b, h)
+        loss = ((y @ w2).float() ** 2).mean()
+        loss.backward()
+        grads = [p.grad.clone() for p in (w1, w2, gamma, beta)]
+        for p in (w1, w2, gamma, beta):
+            p.grad = None
+        return loss.detach().clone(), y.detach().clone(), grads
+
+    ref_loss, ref_y, ref = block(torch.relu, lambda b, h: torch.where(h != 0, b, torch.zeros((), device="cuda", dtype=dtype)))
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        loss, y, grads = block(lambda t: A.relu_stash(t, hooks), lambda b, h: A.double_mask(b, h, hooks))
+        assert hooks.packed_bytes < 0.7 * hooks.dense_bytes
+    loss2, y2, grads2 = block(torch.relu, A.double_mask)             # without hooks: the mask is derived on the spot
+    for l, yy, gg in ((loss, y, grads), (loss2, y2, grads2)):
+        assert torch.equal(l, ref_loss) and torch.equal(yy, ref_y)
+        for a, b in zip(gg, ref):
+            assert torch.equal(a, b)
+    # the stash of the masked output shares the source's bitmap and holds exactly its count of values
+    hooks = A.stash_saved_activations(min_numel=1024)
+    h = A.relu_stash(torch.randn(64, 4096, device="cuda", dtype=dtype), hooks)
+    b = torch.randn(64, 4096, device="cuda", dtype=dtype)
+    m = A.double_mask(b, h, hooks)
+    ph, pm = hooks._lookup(h), hooks._lookup(m)
+    assert pm.bitmap is ph.bitmap and pm.chunk_prefix is ph.chunk_prefix and pm.values.numel() == ph.nnz
+    assert torch.equal(hooks._unpack(pm), torch.where(h != 0, b, torch.zeros((), device="cuda", dtype=dtype)))
