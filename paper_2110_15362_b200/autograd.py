@@ -80,6 +80,16 @@ class PackedActivation:
         return out
 
 
+def _usable(t: torch.Tensor) -> bool:
+    """Can the library take this tensor as it is?  (contiguous and 16-byte aligned)"""
+    return t.is_contiguous() and t.data_ptr() % 16 == 0
+
+
+def _flat_input(t: torch.Tensor) -> torch.Tensor:
+    """The tensor itself if the library can take it, else a contiguous, aligned copy."""
+    return t if _usable(t) else t.clone(memory_format=torch.contiguous_format)
+
+
 class _Scratch:
     """Per-device reusable buffers of the packing calls: workspace and a full-capacity values buffer."""
 
@@ -194,6 +204,7 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
 
     def _eligible(self, t: torch.Tensor) -> bool:
         return (t.is_cuda and t.dtype in B.DTYPE_CODE and t.is_contiguous() and t.numel() >= self.min_numel
+                and t.data_ptr() % 16 == 0               # the library wants 16-byte aligned tensors (a view may not be)
                 and not isinstance(t, torch.nn.Parameter) and not (t.requires_grad and t.is_leaf))
 
     def check_statuses(self) -> None:
@@ -249,11 +260,11 @@ class ReLUStash(torch.autograd.Function):
 
     @staticmethod
     def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False):
-        if inplace and x.is_contiguous():
+        if inplace and _usable(x):
             xc = y = x                   # the kernel may write the activation over its input
             ctx.mark_dirty(x)
         else:
-            xc = x.contiguous()
+            xc = _flat_input(x)
             y = torch.empty_like(xc)
         if hooks is not None and hooks.arena is not None:
             bitmap, prefix, nnz_word, off_word = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1))
@@ -276,7 +287,7 @@ class ReLUStash(torch.autograd.Function):
 
     @staticmethod
     def backward(ctx, grad: torch.Tensor):
-        g = grad.contiguous()
+        g = _flat_input(grad)
         gin = torch.empty_like(g)
         (bitmap,) = ctx.saved_tensors
         B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gin.view(-1))
@@ -297,11 +308,11 @@ class ReLU6Stash(torch.autograd.Function):
 
     @staticmethod
     def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False):
-        if inplace and x.is_contiguous():
+        if inplace and _usable(x):
             xc = y = x
             ctx.mark_dirty(x)
         else:
-            xc = x.contiguous()
+            xc = _flat_input(x)
             y = torch.empty_like(xc)
         scratch = hooks.scratch if hooks is not None else _Scratch()
         bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1), relu6=True)
@@ -315,7 +326,7 @@ class ReLU6Stash(torch.autograd.Function):
 
     @staticmethod
     def backward(ctx, grad: torch.Tensor):
-        g = grad.contiguous()
+        g = _flat_input(grad)
         gin = torch.empty_like(g)
         bitmap, values, prefix = ctx.saved_tensors
         B.bt_relu6_bwd_from_stash(bitmap, values, prefix, g.view(-1), gin.view(-1))
@@ -341,13 +352,13 @@ class DoubleMask(torch.autograd.Function):
         if src is None or src.arena is not None or src.values.dtype != like.dtype:
             # no reusable stash of `like` (none yet, or one whose size only the device knows): make one
             scratch = hooks.scratch if hooks is not None else _Scratch()
-            bitmap, values, prefix, nnz = _compress(like.detach().contiguous().view(-1), scratch)
+            bitmap, values, prefix, nnz = _compress(_flat_input(like.detach()).view(-1), scratch)
             src = PackedActivation(bitmap, values, prefix, tuple(like.shape), like.dtype, like.device, nnz)
-        if inplace and out.is_contiguous():
+        if inplace and _usable(out):
             xc = y = out
             ctx.mark_dirty(out)
         else:
-            xc = out.contiguous()
+            xc = _flat_input(out)
             y = torch.empty_like(xc)
         values = torch.empty(max(src.nnz, 1), dtype=out.dtype, device=out.device)
         B.bt_mask_compress(xc.view(-1), src.bitmap, src.chunk_prefix, y.view(-1), values, values_capacity=src.nnz)
@@ -362,7 +373,7 @@ class DoubleMask(torch.autograd.Function):
 
     @staticmethod
     def backward(ctx, grad: torch.Tensor):
-        g = grad.contiguous()
+        g = _flat_input(grad)
         gin = torch.empty_like(g)
         (bitmap,) = ctx.saved_tensors
         B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gin.view(-1))

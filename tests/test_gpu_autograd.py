@@ -69,6 +69,8 @@ def test_pack_unpack_round_trip_and_skips(A):
     assert hooks._pack(cpu) is cpu
     view = torch.zeros(256, 512, device="cuda").t()                # not contiguous
     assert hooks._pack(view) is view
+    odd = torch.zeros((1 << 16) + 1, device="cuda")[1:]            # contiguous but not 16-byte aligned
+    assert odd.data_ptr() % 16 != 0 and hooks._pack(odd) is odd
 
 
 def test_conv_network_trains_and_matches(A):
@@ -257,3 +259,21 @@ def test_double_mask_batch_norm_block(A, dtype):
     ph, pm = hooks._lookup(h), hooks._lookup(m)
     assert pm.bitmap is ph.bitmap and pm.chunk_prefix is ph.chunk_prefix and pm.values.numel() == ph.nnz
     assert torch.equal(hooks._unpack(pm), torch.where(h != 0, b, torch.zeros((), device="cuda", dtype=dtype)))
+
+
+def test_views_that_the_library_cannot_take_are_copied(A):
+    """A contiguous but misaligned view and a transposed view go through the fused functions via a copy."""
+    base = torch.randn((1 << 16) + 1, device="cuda")
+    for x in (base[1:], torch.randn(256, 512, device="cuda").t()):
+        x = x.detach().requires_grad_()
+        ref = torch.relu(x)
+        ref.backward(torch.ones_like(ref))
+        gref, x.grad = x.grad.clone(), None
+        for fn, tref in ((A.relu_stash, ref), (A.relu6_stash, torch.nn.functional.relu6(x.detach()))):
+            y = fn(x)
+            assert torch.equal(y, tref)
+            y.backward(torch.ones_like(y))
+            assert torch.equal(x.grad, gref if fn is A.relu_stash else ((x.detach() > 0) & (x.detach() < 6)).float())
+            x.grad = None
+        m = A.double_mask(x.detach() + 1, x.detach().clamp_min(0))
+        assert torch.equal(m, torch.where(x.detach() > 0, x.detach() + 1, torch.zeros((), device="cuda")))
