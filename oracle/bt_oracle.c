@@ -468,3 +468,75 @@ void oracle_widen_decompress(const uint32_t *bitmap, const uint16_t *values, uin
         memcpy(out + 4 * i, &u, 4);
     }
 }
+
+/* The element widened to binary64 for an ordering decision (exact for all four kinds). */
+static double as_double(const unsigned char *e, int kind)
+{
+    switch (kind) {
+    case ORACLE_F32: { float f; memcpy(&f, e, 4); return (double)f; }
+    case ORACLE_F64: { double d; memcpy(&d, e, 8); return d; }
+    case ORACLE_F16: { uint16_t h; memcpy(&h, e, 2); return (double)oracle_half_to_float(h); }
+    default: {
+        uint16_t h; memcpy(&h, e, 2);
+        uint32_t u = (uint32_t)h << 16; float f; memcpy(&f, &u, 4);
+        return (double)f;
+    }
+    }
+}
+
+/* 2x2 max pooling, stride 2, of `planes` images of height x width elements (both
+ * even), row-major.  The window is visited in the order (0,0), (0,1), (1,0),
+ * (1,1); a later element replaces the current maximum when it is greater or
+ * when it is a NaN (so the first of equal maxima wins, and the last NaN wins):
+ * the rule of the framework's own pooling kernels, which the codes must agree
+ * with.  y (planes x height/2 x width/2) receives a raw copy of the winner,
+ * codes (may be NULL) its position 2*dy + dx, two bits per output, sixteen
+ * outputs per 32-bit word, output o in bits 2*(o%16).. of word o/16; unused
+ * bits of the last word are 0. */
+void oracle_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width,
+                           int kind, void *y, uint32_t *codes)
+{
+    int es = oracle_elem_size(kind);
+    const unsigned char *src = (const unsigned char *)x;
+    unsigned char *dst = (unsigned char *)y;
+    uint64_t ho = height / 2, wo = width / 2;
+    uint64_t outputs = planes * ho * wo;
+    if (codes)
+        for (uint64_t w = 0; w < (outputs + 15) / 16; ++w) codes[w] = 0;
+    uint64_t o = 0;
+    for (uint64_t p = 0; p < planes; ++p)
+        for (uint64_t r = 0; r < ho; ++r)
+            for (uint64_t c = 0; c < wo; ++c, ++o) {
+                uint64_t best_at = 0;
+                double   best    = 0.0;
+                unsigned best_k  = 0;
+                for (unsigned k = 0; k < 4; ++k) {
+                    uint64_t at = (p * height + 2 * r + (k >> 1)) * width + 2 * c + (k & 1);
+                    double   v  = as_double(src + at * (uint64_t)es, kind);
+                    if (k == 0 || v > best || v != v) {
+                        best = v; best_at = at; best_k = k;
+                    }
+                }
+                memcpy(dst + o * (uint64_t)es, src + best_at * (uint64_t)es, (size_t)es);
+                if (codes) codes[o >> 4] |= (uint32_t)best_k << (2 * (o & 15));
+            }
+}
+
+/* Its backward pass from the codes alone: the gradient of an output goes to the
+ * window position its code names, the other three positions get +0. */
+void oracle_maxpool2x2_bwd(const uint32_t *codes, const void *grad_out, uint64_t planes,
+                           uint64_t height, uint64_t width, int elem_size, void *grad_in)
+{
+    const unsigned char *g = (const unsigned char *)grad_out;
+    unsigned char *gi = (unsigned char *)grad_in;
+    uint64_t ho = height / 2, wo = width / 2;
+    memset(gi, 0, (size_t)(planes * height * width * (uint64_t)elem_size));
+    uint64_t o = 0;
+    for (uint64_t p = 0; p < planes; ++p)
+        for (uint64_t r = 0; r < ho; ++r)
+            for (uint64_t c = 0; c < wo; ++c, ++o) {
+                unsigned k  = (codes[o >> 4] >> (2 * (o & 15))) & 3u;
+                uint64_t at = (p * height + 2 * r + (k >> 1)) * width + 2 * c + (k & 1);
+                memcpy(gi + at * (uint64_t)elem_size, g + o * (uint64_t)elem_size, (size_t)elem_size);
+            }
+}

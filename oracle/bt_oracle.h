@@ -93,6 +93,17 @@ uint64_t oracle_compressed_bytes(uint64_t n, uint64_t nnz, int elem_size);
 uint64_t oracle_narrow_compress(const void *x, uint64_t n, int to_kind, int fused, float tau,
                                 void *y, uint32_t *bitmap, uint16_t *values, uint64_t *prefix);
 
+/* 2x2 / stride 2 max pooling of planes x height x width elements (height and
+ * width even) with a 2-bit code per output naming the winning window position
+ * (2*dy + dx; window order (0,0),(0,1),(1,0),(1,1); a later element wins when
+ * greater or NaN), sixteen codes per 32-bit word, LSB first.  The pooled output
+ * is what the stash then compresses; the codes replace the saved input and the
+ * index tensor in the backward pass. */
+void oracle_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width,
+                           int kind, void *y, uint32_t *codes);
+void oracle_maxpool2x2_bwd(const uint32_t *codes, const void *grad_out, uint64_t planes,
+                           uint64_t height, uint64_t width, int elem_size, void *grad_in);
+
 /* Algorithm 2 on a narrowed stash, each value widened exactly to binary32 */
 void oracle_widen_decompress(const uint32_t *bitmap, const uint16_t *values, uint64_t n,
                              int from_kind, void *dense_f32);

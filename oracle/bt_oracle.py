@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.oracle_compressed_bytes.argtypes = [u64, u64, i32]
         L.oracle_narrow_compress.restype = u64
         L.oracle_narrow_compress.argtypes = [vp, u64, i32, i32, ctypes.c_float, vp, vp, vp, vp]
+        L.oracle_maxpool2x2_fwd.restype = None
+        L.oracle_maxpool2x2_fwd.argtypes = [vp, u64, u64, u64, i32, vp, vp]
+        L.oracle_maxpool2x2_bwd.restype = None
+        L.oracle_maxpool2x2_bwd.argtypes = [vp, vp, u64, u64, u64, i32, vp]
         L.oracle_widen_decompress.restype = None
         L.oracle_widen_decompress.argtypes = [vp, vp, u64, i32, vp]
         L.oracle_float_to_half.restype = ctypes.c_uint16
@@ -206,6 +210,24 @@ def narrow_compress(x: np.ndarray, to_kind: str, fused: bool = False, tau: float
     nnz = int(lib().oracle_narrow_compress(_ptr(x), n, KINDS[to_kind], int(fused), float(np.float32(tau)), _ptr(y),
                                             _ptr(bitmap), _ptr(values), _ptr(prefix)))
     return y, Compressed(bitmap, values[:nnz].copy(), prefix, nnz, n)
+
+
+def maxpool2x2_fwd(x: np.ndarray, planes: int, height: int, width: int, kind: str):
+    """Returns (y, codes): the pooled raw patterns (planes * height/2 * width/2) and the 2-bit winner codes."""
+    x = _raw(x)
+    assert x.size == planes * height * width and height % 2 == 0 and width % 2 == 0
+    outputs = planes * (height // 2) * (width // 2)
+    y = np.empty(outputs, dtype=x.dtype)
+    codes = np.full((outputs + 15) // 16, 0xDEADBEEF, dtype=np.uint32)
+    lib().oracle_maxpool2x2_fwd(_ptr(x), planes, height, width, KINDS[kind], _ptr(y), _ptr(codes))
+    return y, codes
+
+
+def maxpool2x2_bwd(codes: np.ndarray, grad_out: np.ndarray, planes: int, height: int, width: int) -> np.ndarray:
+    g = _raw(grad_out)
+    gin = np.empty(planes * height * width, dtype=g.dtype)
+    lib().oracle_maxpool2x2_bwd(_ptr(codes), _ptr(g), planes, height, width, g.dtype.itemsize, _ptr(gin))
+    return gin
 
 
 def widen_decompress(c: Compressed, from_kind: str) -> np.ndarray:

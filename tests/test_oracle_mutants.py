@@ -45,6 +45,9 @@ MUTANTS = {
                                          "        if ((to_kind == ORACLE_F16 ? oracle_float_to_half(u) : oracle_float_to_bfloat16(u)) & 0x7FFFu) {\n            values[j] = to_kind"),
     "widen_bf16_shifts_one_bit_short": ("            } else {\n                u = (uint32_t)h << 16;", "            } else {\n                u = (uint32_t)h << 15;"),
     "widen_skips_the_value_counter": ("            uint16_t h = values[j];\n            j += 1;", "            uint16_t h = values[j];\n            j += (i % 89 != 0);"),
+    "maxpool_last_of_equal_maxima_wins": ("if (k == 0 || v > best || v != v) {", "if (k == 0 || v >= best || v != v) {"),
+    "maxpool_ignores_nan": ("if (k == 0 || v > best || v != v) {", "if (k == 0 || v > best) {"),
+    "maxpool_codes_column_major": ("codes[o >> 4] |= (uint32_t)best_k << (2 * (o & 15));", "codes[o >> 4] |= (uint32_t)(((best_k & 1) << 1) | (best_k >> 1)) << (2 * (o & 15));"),
     "bytes_forgets_prefix": ("return 4 * words + nnz * (uint64_t)elem_size + 8 * chunks;", "return 4 * words + nnz * (uint64_t)elem_size;"),
     "bytes_counts_bits_as_bytes": ("return 4 * words + nnz", "return 32 * words + nnz"),
 }
@@ -79,6 +82,8 @@ def build_mutant(tmp_path, name):
     L.oracle_narrow_compress.argtypes = [vp, u64, i32, i32, ctypes.c_float, vp, vp, vp, vp]
     L.oracle_widen_decompress.restype = None
     L.oracle_widen_decompress.argtypes = [vp, vp, u64, i32, vp]
+    L.oracle_maxpool2x2_fwd.restype = None
+    L.oracle_maxpool2x2_fwd.argtypes = [vp, u64, u64, u64, i32, vp, vp]
     return L
 
 
@@ -167,6 +172,19 @@ def pins_hold(L) -> bool:
         up = dense16.view(np.float16).astype(np.float32).view(np.uint32) if to_kind == 1 else dense16.astype(np.uint32) << 16
         if not np.array_equal(wide, up):
             return False
+    # 2x2 max pooling against torch: values and winner positions, with ties and a NaN
+    tp = torch.clamp_min(torch.randn(3, 8, 12, generator=torch.Generator().manual_seed(9)), 0.0)
+    tp[0, 0, 0] = float("nan"); tp[1, 2:4, 2:4] = 1.5
+    yp = np.empty(3 * 4 * 6, np.uint32)
+    cp = np.zeros((3 * 4 * 6 + 15) // 16, np.uint32)
+    L.oracle_maxpool2x2_fwd(p(W.raw_numpy(tp.reshape(-1))), 3, 8, 12, 0, p(yp), p(cp))
+    refp, idxp = torch.nn.functional.max_pool2d(tp.unsqueeze(0), 2, return_indices=True)
+    kk = (2 * (idxp[0] // 12 - 2 * torch.arange(4).view(1, 4, 1)) + (idxp[0] % 12 - 2 * torch.arange(6).view(1, 1, 6))).reshape(-1).numpy()
+    unpacked = (cp.repeat(16) >> np.tile(2 * np.arange(16, dtype=np.uint32), cp.size)) & 3
+    if not np.array_equal(unpacked[:kk.size], kk.astype(np.uint32)):
+        return False
+    if not np.array_equal(np.nan_to_num(yp.view(np.float32), nan=9.0), np.nan_to_num(refp.reshape(-1).numpy(), nan=9.0)):
+        return False
     # closed form and the first row of Table 1 (16,3,224,224 at 50 % non-zero: 4.88 MB without the prefix term)
     if L.oracle_compressed_bytes(200704, 100352, 4) != 200704 // 8 + 4 * 100352 + 8 * 49:
         return False
