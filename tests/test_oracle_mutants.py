@@ -174,7 +174,7 @@ def pins_hold(L) -> bool:
             return False
     # 2x2 max pooling against torch: values and winner positions, with ties and a NaN
     tp = torch.clamp_min(torch.randn(3, 8, 12, generator=torch.Generator().manual_seed(9)), 0.0)
-    tp[0, 0, 0] = float("nan"); tp[1, 2:4, 2:4] = 1.5
+    tp[0, 0, 1] = float("nan"); tp[0, 3, 2] = float("nan"); tp[1, 2:4, 2:4] = 1.5
     yp = np.empty(3 * 4 * 6, np.uint32)
     cp = np.zeros((3 * 4 * 6 + 15) // 16, np.uint32)
     L.oracle_maxpool2x2_fwd(p(W.raw_numpy(tp.reshape(-1))), 3, 8, 12, 0, p(yp), p(cp))
