@@ -411,6 +411,26 @@ def large_tensor_kernels(dev, peak_gbs: float):
     out["f32_2^28_bt_prune_fwd_compress_N(0,0.15)"] = rows
     del pre, st, ws
     torch.cuda.empty_cache()
+
+    # max pooling with winner codes (a "next" row): the first pooling layer of a VGG-16 at batch 32
+    rows = {}
+    for label, dt in (("f32", torch.float32), ("bf16", torch.bfloat16)):
+        x = torch.clamp_min(torch.randn(32, 64, 224, 224, device=dev, generator=torch.Generator(device=dev).manual_seed(900)),
+                            0).to(dt)
+        no, es = x.numel() // 4, x.element_size()
+        y = torch.empty(32, 64, 112, 112, dtype=dt, device=dev)
+        codes = torch.empty((no + 15) // 16, dtype=torch.int32, device=dev)
+        gin = torch.empty_like(x)
+        by = 5 * no * es + 4 * ((no + 15) // 16)
+        for op, fn in (("bt_maxpool2x2_fwd", lambda: B.bt_maxpool2x2_fwd(x, y, codes)),
+                       ("bt_maxpool2x2_bwd", lambda: B.bt_maxpool2x2_bwd(codes, y, gin))):
+            ms, best = time_call(fn)
+            rows[label + "_" + op] = {"ms_median": round(ms, 4), "ms_best": round(best, 4), "moved_gbs": round(by / ms / 1e6, 1),
+                                      "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
+                                      "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
+        del x, y, codes, gin
+        torch.cuda.empty_cache()
+    out["maxpool2x2_[32,64,224,224]"] = rows
     return out
 
 

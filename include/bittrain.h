@@ -64,7 +64,8 @@ enum {
     BT_ERR_CAPACITY = 5,   /* device: nnz > values_capacity (see bt_compress)          */
     BT_ERR_TIMEOUT = 6,    /* device: a bounded wait inside the kernel ran out         */
     BT_ERR_CUDA = 7,       /* the CUDA runtime reported an error at launch             */
-    BT_ERR_TOO_LARGE = 8   /* n exceeds what the call can handle (bt_compress_noalloc) */
+    BT_ERR_TOO_LARGE = 8,  /* n exceeds what the call can handle (bt_compress_noalloc) */
+    BT_ERR_SHAPE = 9       /* a dimension the call cannot take (bt_maxpool2x2_*: odd or zero) */
 };
 
 /*
@@ -175,6 +176,32 @@ int bt_prune_fwd_compress_narrow(const void *x, uint64_t n, int to_dtype, float 
                                  uint64_t *chunk_prefix, uint64_t *nnz_out,
                                  void *workspace, size_t workspace_bytes,
                                  int32_t *dev_status, void *stream);
+
+/*
+ * Max pooling with winner codes.  The evaluation's per-layer analysis finds the
+ * activations of max-pooling layers among the largest and sparsest; a
+ * framework keeps, for such a layer's backward pass, its input and an index
+ * tensor (8 bytes per output).  bt_maxpool2x2_fwd pools planes x height x width
+ * elements (row-major, e.g. N*C planes of an NCHW tensor; height and width even
+ * and non-zero, else BT_ERR_SHAPE) with a 2x2 window and stride 2 into y
+ * (planes x height/2 x width/2) and writes, if codes is not NULL, 2 bits per
+ * output naming the winning window position 2*dy + dx: sixteen outputs per
+ * 32-bit word, output o in bits 2*(o%16).. of word o/16, ceil(outputs/16)
+ * words, unused bits 0.  The window is visited in the order (0,0), (0,1),
+ * (1,0), (1,1) and a later element replaces the maximum when it is greater
+ * (IEEE comparison of the exactly widened values) or when it is a NaN: the
+ * first of equal maxima wins, a NaN wins over everything, the last NaN over an
+ * earlier one -- the positions a framework's index tensor would name.  y
+ * receives a raw copy of the winner (then stashed with bt_compress like any
+ * activation).  bt_maxpool2x2_bwd needs only the codes: grad_in (planes x
+ * height x width) gets grad_out[o] at the coded position of window o and +0
+ * at the other three; every element of grad_in is written.  x / y and
+ * grad_out / grad_in must not overlap.  Pointers 16-byte aligned.
+ */
+int bt_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width, int dtype,
+                      void *y, uint32_t *codes, void *stream);
+int bt_maxpool2x2_bwd(const uint32_t *codes, const void *grad_out, uint64_t planes, uint64_t height,
+                      uint64_t width, int dtype, void *grad_in, void *stream);
 
 /*
  * Algorithm 2 on a narrowed stash, straight into a BT_F32 tensor: dense_out[i]

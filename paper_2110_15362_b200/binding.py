@@ -17,9 +17,9 @@ from . import build as _build
 
 BT_F32, BT_F16, BT_BF16, BT_F64 = 0, 1, 2, 3
 (BT_OK, BT_ERR_NULL, BT_ERR_DTYPE, BT_ERR_ALIGN, BT_ERR_WORKSPACE, BT_ERR_CAPACITY, BT_ERR_TIMEOUT, BT_ERR_CUDA,
- BT_ERR_TOO_LARGE) = range(9)
+ BT_ERR_TOO_LARGE, BT_ERR_SHAPE) = range(10)
 STATUS_NAMES = ["BT_OK", "BT_ERR_NULL", "BT_ERR_DTYPE", "BT_ERR_ALIGN", "BT_ERR_WORKSPACE", "BT_ERR_CAPACITY",
-                "BT_ERR_TIMEOUT", "BT_ERR_CUDA", "BT_ERR_TOO_LARGE"]
+                "BT_ERR_TIMEOUT", "BT_ERR_CUDA", "BT_ERR_TOO_LARGE", "BT_ERR_SHAPE"]
 NOALLOC_MAX_ELEMS = 1 << 26
 CHUNK = 4096
 
@@ -29,7 +29,7 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
            "bt_prune_fwd_compress", "bt_mask_compress", "bt_compress_arena", "bt_prune_fwd_compress_arena",
            "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
-           "bt_prune_fwd_compress_narrow", "bt_decompress_widen")
+           "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -87,6 +87,10 @@ def lib() -> ctypes.CDLL:
         L.bt_prune_fwd_compress_narrow.restype = i32
         L.bt_decompress_widen.argtypes = [vp, vp, vp, u64, i32, vp, vp]
         L.bt_decompress_widen.restype = i32
+        L.bt_maxpool2x2_fwd.argtypes = [vp, u64, u64, u64, i32, vp, vp, vp]
+        L.bt_maxpool2x2_fwd.restype = i32
+        L.bt_maxpool2x2_bwd.argtypes = [vp, vp, u64, u64, u64, i32, vp, vp]
+        L.bt_maxpool2x2_bwd.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -218,6 +222,28 @@ def bt_decompress_widen(bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix
     st = lib().bt_decompress_widen(_ptr(bitmap), _ptr(values), _ptr(chunk_prefix), n, DTYPE_CODE[values.dtype],
                                    _ptr(dense_out), _stream(stream))
     return _check("bt_decompress_widen", st, check)
+
+
+def bt_maxpool2x2_fwd(x: torch.Tensor, y: torch.Tensor, codes: Optional[torch.Tensor], *, planes: Optional[int] = None,
+                      height: Optional[int] = None, width: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """2x2 / stride 2 max pooling of a contiguous (..., H, W) tensor into y, with 2-bit winner codes (int32 words,
+    ceil(outputs / 16) of them) if `codes` is given."""
+    height = x.shape[-2] if height is None else height
+    width = x.shape[-1] if width is None else width
+    planes = x.numel() // max(1, height * width) if planes is None else planes
+    st = lib().bt_maxpool2x2_fwd(_ptr(x), planes, height, width, DTYPE_CODE[x.dtype], _ptr(y), _ptr(codes), _stream(stream))
+    return _check("bt_maxpool2x2_fwd", st, check)
+
+
+def bt_maxpool2x2_bwd(codes: torch.Tensor, grad_out: torch.Tensor, grad_in: torch.Tensor, *, planes: Optional[int] = None,
+                      height: Optional[int] = None, width: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """The pooling's backward pass from the codes alone; grad_in has the (..., H, W) shape of the pooled tensor's input."""
+    height = grad_in.shape[-2] if height is None else height
+    width = grad_in.shape[-1] if width is None else width
+    planes = grad_in.numel() // max(1, height * width) if planes is None else planes
+    st = lib().bt_maxpool2x2_bwd(_ptr(codes), _ptr(grad_out), planes, height, width, DTYPE_CODE[grad_out.dtype],
+                                 _ptr(grad_in), _stream(stream))
+    return _check("bt_maxpool2x2_bwd", st, check)
 
 
 def bt_mask_compress(x: torch.Tensor, mask_bitmap: torch.Tensor, mask_chunk_prefix: torch.Tensor,

@@ -53,6 +53,10 @@ cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint
                                int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t s);
 cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
                              uint64_t n, int dtype, void *gin, cudaStream_t s);
+cudaError_t launch_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width, int dtype, void *y,
+                                  uint32_t *codes, cudaStream_t s);
+cudaError_t launch_maxpool2x2_bwd(const uint32_t *codes, const void *gout, uint64_t planes, uint64_t height, uint64_t width,
+                                  int elem_size, void *gin, cudaStream_t s);
 cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size,
                             void *gin, cudaStream_t s);
 
@@ -197,6 +201,25 @@ __device__ __forceinline__ uint32_t at_least_six(double v)
 {
     uint32_t r;
     asm("{\n\t.reg .pred p;\n\tsetp.ge.f64 p, %1, 0d4018000000000000;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "d"(v));
+    return r;
+}
+
+// (v > b) || isnan(v) as an opaque 0/1, for the same reason: a compare-and-select chain written in C++ may
+// become a floating-point maximum, which does not keep a NaN's payload.
+__device__ __forceinline__ uint32_t greater_or_nan(float v, float b)
+{
+    uint32_t r;
+    asm("{\n\t.reg .pred p, q;\n\tsetp.gt.f32 p, %1, %2;\n\tsetp.nan.f32 q, %1, %1;\n\tor.pred p, p, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "f"(v), "f"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t greater_or_nan(double v, double b)
+{
+    uint32_t r;
+    asm("{\n\t.reg .pred p, q;\n\tsetp.gt.f64 p, %1, %2;\n\tsetp.nan.f64 q, %1, %1;\n\tor.pred p, p, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "d"(v), "d"(b));
     return r;
 }
 
