@@ -25,6 +25,10 @@ is zeroed wherever ``like`` (the layer's input, a post-ReLU tensor) is zero, and
 the prefix array of ``like``'s stash (``bt_mask_compress``); the backward pass masks the gradient with the same
 bitmap.
 
+``maxpool2x2_stash(x)`` is a 2x2 / stride 2 max pooling that keeps 2 bits per output for its backward pass
+(``bt_maxpool2x2_fwd`` / ``bt_maxpool2x2_bwd``) instead of its input and an index tensor: behind a ``relu_stash``
+the values of the pooled layer's input are then held by nothing, only its bitmap.
+
 ``relu6_stash(x)`` is the same for ReLU6 (``bt_relu6_fwd_compress`` / ``bt_relu6_bwd_from_stash``; its backward
 pass reads the stashed values as well, which are the ones the next layer's saved input shares).  With
 ``stash_saved_activations(narrow=torch.float16)`` (or ``torch.bfloat16``) float32 activations are stashed with
@@ -41,7 +45,7 @@ import torch
 from . import binding as B
 
 __all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash", "relu6_stash", "ReLU6Stash",
-           "double_mask", "DoubleMask"]
+           "double_mask", "DoubleMask", "maxpool2x2_stash", "MaxPool2x2Stash"]
 
 
 class PackedActivation:
@@ -384,3 +388,33 @@ def double_mask(out: torch.Tensor, like: torch.Tensor, hooks: Optional[stash_sav
                 inplace: bool = False) -> torch.Tensor:
     """``out`` with zeros wherever ``like`` is zero, stashed under ``like``'s bitmap (see ``DoubleMask``)."""
     return DoubleMask.apply(out, like, hooks, inplace)
+
+
+class MaxPool2x2Stash(torch.autograd.Function):
+    """2x2 / stride 2 max pooling of a (..., H, W) tensor (H and W even) whose backward pass needs only 2 bits per
+    output.  The pooled output is an ordinary tensor: inside the hooks context the next layer's save compresses it."""
+
+    @staticmethod
+    def forward(ctx, x: torch.Tensor):
+        if x.dim() < 2 or x.shape[-1] % 2 or x.shape[-2] % 2 or x.numel() == 0:
+            raise ValueError("maxpool2x2_stash: the last two dimensions must be even and non-empty")
+        xc = _flat_input(x)
+        y = torch.empty(xc.shape[:-2] + (xc.shape[-2] // 2, xc.shape[-1] // 2), dtype=x.dtype, device=x.device)
+        codes = torch.empty((y.numel() + 15) // 16, dtype=torch.int32, device=x.device)
+        B.bt_maxpool2x2_fwd(xc, y, codes)
+        ctx.save_for_backward(codes)
+        ctx.in_shape = tuple(xc.shape)
+        return y
+
+    @staticmethod
+    def backward(ctx, grad: torch.Tensor):
+        (codes,) = ctx.saved_tensors
+        g = _flat_input(grad)
+        gin = torch.empty(ctx.in_shape, dtype=g.dtype, device=g.device)
+        B.bt_maxpool2x2_bwd(codes, g, gin)
+        return gin
+
+
+def maxpool2x2_stash(x: torch.Tensor) -> torch.Tensor:
+    """``torch.nn.functional.max_pool2d(x, 2)`` with a 2-bit-per-output backward record (see ``MaxPool2x2Stash``)."""
+    return MaxPool2x2Stash.apply(x)

@@ -4,9 +4,10 @@
 
 Builds the thirteen 3x3 convolutions and five 2x2 max-pools of VGG-16 (no batch normalisation, a small
 linear head), runs forward + backward three ways -- plain PyTorch (in-place ReLU), saved activations
-stashed (exact-size values, one host read per tensor), saved activations stashed into an arena (no host
-read) -- and prints one JSON line with the bytes kept for the saved ReLU outputs relative to their dense
-size, the peak device memory above the model's own tensors and the step time of each.  The peak also
+stashed (exact-size values, one host read per tensor), the same with the pooling layers keeping 2-bit winner
+codes instead of their input and an index tensor, and that with the values in an arena (no host read) -- and prints one JSON line with the bytes kept for the saved ReLU outputs relative to their dense
+size, the device memory held between the forward and the backward pass, the peak above the model's own tensors
+and the step time of each.  The peak also
 holds what no stash touches: the transients of the widest layer (its pre-activation, its gradients, the
 restored activation) and the max-pool indices, so it drops by less than the saved activations do.  The paper
 measures the training-memory footprint of such models on ImageNet / CIFAR-10 with pre-trained weights; with
@@ -25,6 +26,7 @@ import torch.nn.functional as F
 from . import autograd as A
 from . import binding as B
 
+HELD = []          # device bytes allocated at the end of each forward pass (read by measure())
 CFG = (64, 64, "M", 128, 128, "M", 256, 256, 256, "M", 512, 512, 512, "M", 512, 512, 512, "M")
 
 
@@ -41,16 +43,18 @@ def make_weights(dtype, device, seed=0):
     return ws, head
 
 
-def step(x, ws, head, relu):
+def step(x, ws, head, relu, pool=lambda t: F.max_pool2d(t, 2)):
     h, k = x, 0
     for c in CFG:
         if c == "M":
-            h = F.max_pool2d(h, 2)
+            h = pool(h)
         else:
             h = relu(F.conv2d(h, ws[k], padding=1))
             k += 1
     logits = F.linear(h.mean(dim=(2, 3)), head)
     loss = logits.float().square().mean()
+    del h, logits
+    HELD.append(torch.cuda.memory_allocated())                # what the graph holds between the two passes
     loss.backward()
     for w in ws + [head]:
         w.grad = None
@@ -73,7 +77,9 @@ def measure(fn, reps=3):
         ms = e0.elapsed_time(e1)
         best = ms if best is None else min(best, ms)
         peak = max(peak, torch.cuda.max_memory_allocated() - base)
-    return {"peak_mib": round(peak / 2 ** 20, 1), "step_ms": round(best, 2), "loss": loss}
+        held = HELD[-1] - base
+    return {"held_after_forward_mib": round(held / 2 ** 20, 1), "peak_mib": round(peak / 2 ** 20, 1),
+            "step_ms": round(best, 2), "loss": loss}
 
 
 def main(argv=None) -> int:
@@ -95,19 +101,42 @@ def main(argv=None) -> int:
            "size": args.size, "dtype": args.dtype}
     out["plain"] = measure(lambda: step(x, ws, head, torch.relu_))
 
+    def scratch_mib(hooks):
+        t = list(hooks.scratch.ws.values()) + list(hooks.scratch.values.values())
+        return round(sum(b.numel() * b.element_size() for b in t) / 2 ** 20, 1)
+
+    # one context object per variant, entered once per step: its scratch (workspace and a full-capacity values
+    # buffer) is allocated by the warm-up step and reported on its own
+    hooks1 = A.stash_saved_activations()
+
     def stashed():
-        with A.stash_saved_activations() as hooks:
-            loss = step(x, ws, head, lambda t: A.relu_stash(t, hooks, inplace=True))
-            out["saved_activation_bytes_over_dense"] = round(hooks.packed_bytes / max(1, hooks.dense_bytes), 4)
+        with hooks1:
+            before = hooks1.packed_bytes, hooks1.dense_bytes
+            loss = step(x, ws, head, lambda t: A.relu_stash(t, hooks1, inplace=True))
+            out["saved_activation_bytes_over_dense"] = round((hooks1.packed_bytes - before[0]) /
+                                                             max(1, hooks1.dense_bytes - before[1]), 4)
         return loss
 
     out["stashed"] = measure(stashed)
+    out["stashed"]["scratch_mib"] = scratch_mib(hooks1)
+    del hooks1
+    torch.cuda.empty_cache()
+    hooks2 = A.stash_saved_activations()
+
+    def stashed_pool():
+        with hooks2:
+            return step(x, ws, head, lambda t: A.relu_stash(t, hooks2, inplace=True), A.maxpool2x2_stash)
+
+    out["stashed_pool_codes"] = measure(stashed_pool)
+    out["stashed_pool_codes"]["scratch_mib"] = scratch_mib(hooks2)
+    del hooks2
+    torch.cuda.empty_cache()
 
     arena_hooks = A.stash_saved_activations(arena_bytes=int(args.arena_gib * 2 ** 30))
 
     def arena():
         with arena_hooks:
-            return step(x, ws, head, lambda t: A.relu_stash(t, arena_hooks, inplace=True))
+            return step(x, ws, head, lambda t: A.relu_stash(t, arena_hooks, inplace=True), A.maxpool2x2_stash)
 
     out["stashed_arena"] = measure(arena)
     out["stashed_arena"]["arena_used_mib"] = round(int(arena_hooks.cursor.item()) / 2 ** 20, 1)

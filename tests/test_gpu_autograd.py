@@ -163,7 +163,11 @@ def test_vgg_demo_runs_and_losses_agree(A, capsys):
     out = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
     assert out["plain"]["loss"] == pytest.approx(out["stashed"]["loss"], rel=1e-3)
     assert out["plain"]["loss"] == pytest.approx(out["stashed_arena"]["loss"], rel=1e-3)
+    assert out["plain"]["loss"] == pytest.approx(out["stashed_pool_codes"]["loss"], rel=1e-3)
     assert 0.3 < out["saved_activation_bytes_over_dense"] < 0.8
+    # what the graph holds between the two passes shrinks, most with the pooling layers on winner codes
+    assert out["stashed_pool_codes"]["held_after_forward_mib"] < out["stashed"]["held_after_forward_mib"] \
+        < out["plain"]["held_after_forward_mib"]
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
@@ -277,3 +281,33 @@ def test_views_that_the_library_cannot_take_are_copied(A):
             x.grad = None
         m = A.double_mask(x.detach() + 1, x.detach().clamp_min(0))
         assert torch.equal(m, torch.where(x.detach() > 0, x.detach() + 1, torch.zeros((), device="cuda")))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_maxpool_stash_matches_torch(A, dtype):
+    x = torch.randn(8, 16, 28, 36, device="cuda", generator=torch.Generator(device="cuda").manual_seed(21)).clamp_min_(0).to(dtype)
+    w = (torch.randn(16, 16, 3, 3, device="cuda", generator=torch.Generator(device="cuda").manual_seed(22)) / 12).to(dtype).requires_grad_()
+
+    def run_net(relu, pool, hooks=None):
+        xx = x.clone().requires_grad_()
+        h = pool(relu(torch.nn.functional.conv2d(xx, w, padding=1)))
+        h = pool(relu(torch.nn.functional.conv2d(h, w, padding=1)))
+        loss = h.float().square().mean()
+        loss.backward()
+        out = (loss.detach().clone(), xx.grad.clone(), w.grad.clone())
+        w.grad = None
+        return out
+
+    torch.backends.cudnn.deterministic = True
+    ref = run_net(torch.relu, lambda t: torch.nn.functional.max_pool2d(t, 2))
+    got = run_net(torch.relu, A.maxpool2x2_stash)
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        got2 = run_net(lambda t: A.relu_stash(t, hooks), A.maxpool2x2_stash)
+    for g in (got, got2):
+        for a, b in zip(g, ref):
+            assert torch.equal(a, b)
+    with pytest.raises(ValueError):
+        A.maxpool2x2_stash(torch.zeros(2, 3, 5, 4, device="cuda"))
+    # a non-contiguous input is taken through a copy
+    xt = torch.randn(4, 6, 8, 10, device="cuda").transpose(0, 1)
+    assert torch.equal(A.maxpool2x2_stash(xt), torch.nn.functional.max_pool2d(xt, 2))
