@@ -179,6 +179,7 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
         self.min_numel, self.min_saving, self.narrow = min_numel, min_saving, narrow
         self.arena = self.cursor = None
         self.statuses: list = []
+        self.loose_statuses: list = []   # status words of bitmap-only calls (BT_ERR_CAPACITY expected)
         if arena_bytes is not None:
             self.arena = torch.empty((arena_bytes + 15) // 16 * 16, dtype=torch.uint8, device=device)
             self.cursor = torch.zeros(1, dtype=torch.int64, device=device)
@@ -212,7 +213,14 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
                 and not isinstance(t, torch.nn.Parameter) and not (t.requires_grad and t.is_leaf))
 
     def check_statuses(self) -> None:
-        """Arena mode: one host read for all stashes made so far; raises if any did not fit."""
+        """One host read for all status words collected so far; raises if an arena stash did not fit or a call
+        failed."""
+        if self.loose_statuses:
+            words = torch.cat(self.loose_statuses)
+            self.loose_statuses.clear()
+            bad = words[(words != B.BT_OK) & (words != B.BT_ERR_CAPACITY)]
+            if bad.numel():
+                raise RuntimeError("a bitmap-only stash call failed: %s" % B.BitTrainError("bt_relu_fwd_compress", int(bad[0].item())))
         if self.statuses:
             worst = int(torch.cat(self.statuses).max().item())
             self.statuses.clear()
@@ -256,6 +264,8 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
 
     def __exit__(self, *exc):
         self._shared.clear()
+        if exc[0] is None:
+            self.check_statuses()
         return super().__exit__(*exc)
 
 
@@ -263,13 +273,31 @@ class ReLUStash(torch.autograd.Function):
     """ReLU with the stash fused into its forward pass; the backward pass reads only the bitmap."""
 
     @staticmethod
-    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False):
+    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False,
+                keep_values: bool = True):
         if inplace and _usable(x):
             xc = y = x                   # the kernel may write the activation over its input
             ctx.mark_dirty(x)
         else:
             xc = _flat_input(x)
             y = torch.empty_like(xc)
+        if not keep_values:
+            # nobody will ask for the activation again (e.g. it only feeds a pooling layer that keeps winner codes):
+            # the bitmap is all this ReLU's backward pass needs, so the values are not stored at all
+            n, dev = xc.numel(), xc.device
+            bitmap = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
+            prefix = torch.empty((n + B.CHUNK - 1) // B.CHUNK, dtype=torch.int64, device=dev)
+            nnz_out = torch.empty(1, dtype=torch.int64, device=dev)
+            status = torch.empty(1, dtype=torch.int32, device=dev)
+            scratch = hooks.scratch if hooks is not None else _Scratch()
+            B.bt_relu_fwd_compress(xc.view(-1), y.view(-1), bitmap, None, prefix, nnz_out, scratch.workspace(n, dev), status,
+                                   n=n, values_capacity=0)
+            if hooks is not None:
+                hooks.loose_statuses.append(status)     # BT_ERR_CAPACITY is the expected answer here
+            elif int(status.item()) not in (B.BT_OK, B.BT_ERR_CAPACITY):
+                raise B.BitTrainError("bt_relu_fwd_compress (bitmap only)", int(status.item()))
+            ctx.save_for_backward(bitmap)
+            return y
         if hooks is not None and hooks.arena is not None:
             bitmap, prefix, nnz_word, off_word = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1))
             ctx.save_for_backward(bitmap)
@@ -295,14 +323,17 @@ class ReLUStash(torch.autograd.Function):
         gin = torch.empty_like(g)
         (bitmap,) = ctx.saved_tensors
         B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gin.view(-1))
-        return gin, None, None
+        return gin, None, None, None
 
 
-def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False) -> torch.Tensor:
+def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False,
+               keep_values: bool = True) -> torch.Tensor:
     """ReLU through the fused kernel.  Pass the active ``stash_saved_activations`` context as ``hooks`` to let
     the following layer reuse the stash for its saved input.  ``inplace=True`` writes the activation over ``x``
-    (like ``torch.relu_``: only where ``x`` is not needed again, e.g. the output of a convolution)."""
-    return ReLUStash.apply(x, hooks, inplace)
+    (like ``torch.relu_``: only where ``x`` is not needed again, e.g. the output of a convolution).
+    ``keep_values=False`` keeps the bitmap only: for an activation that no later layer saves (one that feeds
+    ``maxpool2x2_stash``, say); a layer that does save it compresses it itself."""
+    return ReLUStash.apply(x, hooks, inplace, keep_values)
 
 
 class ReLU6Stash(torch.autograd.Function):

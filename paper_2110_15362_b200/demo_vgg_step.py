@@ -43,13 +43,15 @@ def make_weights(dtype, device, seed=0):
     return ws, head
 
 
-def step(x, ws, head, relu, pool=lambda t: F.max_pool2d(t, 2)):
+def step(x, ws, head, relu, pool=lambda t: F.max_pool2d(t, 2), relu_before_pool=None):
+    """`relu_before_pool`: the activation used where a pooling layer follows (default: `relu`)."""
     h, k = x, 0
-    for c in CFG:
+    for i, c in enumerate(CFG):
         if c == "M":
             h = pool(h)
         else:
-            h = relu(F.conv2d(h, ws[k], padding=1))
+            act = relu_before_pool if relu_before_pool is not None and CFG[i + 1] == "M" else relu
+            h = act(F.conv2d(h, ws[k], padding=1))
             k += 1
     logits = F.linear(h.mean(dim=(2, 3)), head)
     loss = logits.float().square().mean()
@@ -125,7 +127,8 @@ def main(argv=None) -> int:
 
     def stashed_pool():
         with hooks2:
-            return step(x, ws, head, lambda t: A.relu_stash(t, hooks2, inplace=True), A.maxpool2x2_stash)
+            return step(x, ws, head, lambda t: A.relu_stash(t, hooks2, inplace=True), A.maxpool2x2_stash,
+                        lambda t: A.relu_stash(t, hooks2, inplace=True, keep_values=False))
 
     out["stashed_pool_codes"] = measure(stashed_pool)
     out["stashed_pool_codes"]["scratch_mib"] = scratch_mib(hooks2)
@@ -136,7 +139,8 @@ def main(argv=None) -> int:
 
     def arena():
         with arena_hooks:
-            return step(x, ws, head, lambda t: A.relu_stash(t, arena_hooks, inplace=True), A.maxpool2x2_stash)
+            return step(x, ws, head, lambda t: A.relu_stash(t, arena_hooks, inplace=True), A.maxpool2x2_stash,
+                        lambda t: A.relu_stash(t, arena_hooks, inplace=True, keep_values=False))
 
     out["stashed_arena"] = measure(arena)
     out["stashed_arena"]["arena_used_mib"] = round(int(arena_hooks.cursor.item()) / 2 ** 20, 1)

@@ -303,7 +303,16 @@ def test_maxpool_stash_matches_torch(A, dtype):
     got = run_net(torch.relu, A.maxpool2x2_stash)
     with A.stash_saved_activations(min_numel=1024) as hooks:
         got2 = run_net(lambda t: A.relu_stash(t, hooks), A.maxpool2x2_stash)
-    for g in (got, got2):
+    with A.stash_saved_activations(min_numel=1024) as hooks:             # bitmap-only ReLU in front of the pooling
+        got3 = run_net(lambda t: A.relu_stash(t, hooks, keep_values=False), A.maxpool2x2_stash)
+        assert hooks.loose_statuses and hooks._lookup(torch.zeros(1)) is None
+    assert not hooks.loose_statuses                                       # checked on leaving the context
+    with A.stash_saved_activations(min_numel=1024, arena_bytes=32 << 20) as hooks:
+        got4 = run_net(lambda t: A.relu_stash(t, hooks, keep_values=False), A.maxpool2x2_stash)
+        used = int(hooks.cursor.item())
+    got5 = run_net(lambda t: A.relu_stash(t, keep_values=False), A.maxpool2x2_stash)
+    assert used < 32 << 20
+    for g in (got, got2, got3, got4, got5):
         for a, b in zip(g, ref):
             assert torch.equal(a, b)
     with pytest.raises(ValueError):
