@@ -1,6 +1,6 @@
 """One small, seeded invocation of a kernel, for profiler captures.
 
-    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|prune|narrow|relu6|relu6_bwd|decompress|relu_bwd|mask|mask_y> \
+    python -m paper_2110_15362_b200.profile_case <f32|f16|bf16> <compress|relu|relu_y|prune|narrow|relu6|relu6_bwd|decompress|relu_bwd|mask|mask_y|maxpool|maxpool_bwd> \
            [--log2n 26] [--zeros 0.5] [--reps 3]
 
 runs `reps` repetitions of one entry point on a tensor of 2**log2n elements (default 2**26: 256 MiB of
@@ -26,7 +26,7 @@ from . import workloads as W
 def main(argv=None) -> int:
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("dtype", choices=["f32", "f16", "bf16", "f64"])
-    ap.add_argument("op", choices=["compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd", "decompress", "relu_bwd", "mask", "mask_y"])
+    ap.add_argument("op", choices=["compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd", "decompress", "relu_bwd", "mask", "mask_y", "maxpool", "maxpool_bwd"])
     ap.add_argument("--tau", type=float, default=0.1)
     ap.add_argument("--log2n", type=int, default=26)
     ap.add_argument("--zeros", type=float, default=0.5)
@@ -48,6 +48,18 @@ def main(argv=None) -> int:
 
     def compress():
         B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+
+    if args.op in ("maxpool", "maxpool_bwd"):                # the tensor seen as rows of 256 elements
+        xp = x.view(-1, n // 256 // 64, 256)
+        yp = torch.empty(xp.shape[0], xp.shape[1] // 2, 128, dtype=x.dtype, device=dev)
+        codes = torch.empty((yp.numel() + 15) // 16, dtype=torch.int32, device=dev)
+        for _ in range(args.reps):
+            B.bt_maxpool2x2_fwd(xp, yp, codes)
+            if args.op == "maxpool_bwd":
+                B.bt_maxpool2x2_bwd(codes, yp, d.view_as(xp))
+        torch.cuda.synchronize()
+        print("pooled", tuple(yp.shape), "non-zero", int(torch.count_nonzero(yp)))
+        return 0
 
     for _ in range(args.reps):
         if args.op == "compress":
