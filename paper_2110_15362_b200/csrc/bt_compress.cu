@@ -61,7 +61,8 @@ namespace {
 constexpr uint32_t kFull       = 0xFFFFFFFFu;
 constexpr uint64_t kWaitNs     = 2000000000ull;       // bound of every in-kernel wait: 2 s
 constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
-constexpr int      kMaxWindows = 10;                  // the grid never exceeds 32 * kMaxWindows CTAs
+constexpr int      kMaxWindows = 5;                   // the grid never exceeds 32 * kMaxWindows = 160 CTAs (a B200 has 148 SMs);
+                                                      // ten windows cost 2 % on the ResNet-shaped step for predicated-off loads
 constexpr int      kCountShift = 40;                  // wave total word: (tiles added << 40) | sum of counts
 
 #ifdef BT_PROFILE
