@@ -80,7 +80,9 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype);
 /*
  * Bytes of device scratch bt_compress / bt_relu_fwd_compress need for n
  * elements (the tile descriptors of the single-pass scan plus a small header).
- * The contents need no initialisation and are unspecified after a call.  Two
+ * The contents need no initialisation and are unspecified after a call: a
+ * word counts as written by the running call only if it carries that call's
+ * 64-bit tag, which no other call shares.  Two
  * calls that run concurrently must not share a workspace.  No counterpart in
  * the paper (its scan is sequential).
  */
@@ -274,7 +276,7 @@ int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
  * allocation would synchronise the device or simply fail), or a plug-in that
  * receives its input and output buffers from a runtime that owns the device
  * memory and gives it no way to request a workspace.  bt_compress wants such a
- * workspace; here it is built into the library instead: a 262,400-byte array in
+ * workspace; here it is built into the library instead: a 393,488-byte array in
  * device memory that every GPU which loads the library holds until the process
  * exits.  That fixes the largest tensor: n <= BT_NOALLOC_MAX_ELEMS (2^26
  * elements); a larger n returns BT_ERR_TOO_LARGE and nothing is launched.
@@ -285,8 +287,8 @@ int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
  * workspace parameters.  The first call on each device looks up the array's
  * device address (one runtime query, made with that device current) -- make
  * that first call outside any stream capture; later calls only launch.  All
- * calls on a device share the one array: the part a call uses is cleared at
- * its start, so nothing depends on the previous call's contents, but two calls
+ * calls on a device share the one array: nothing in it outlives a call
+ * (its words are tagged per call), but two calls
  * whose execution overlaps on the GPU (different streams) race on it and give
  * undefined results -- keep them on one stream or order them with events.
  */

@@ -60,9 +60,10 @@ int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau
     a.prefix     = chunk_prefix;
     a.nnz_out    = nnz_out;
     a.dev_status = dev_status;
-    a.ws_header  = static_cast<uint32_t *>(workspace);
+    a.ws_header  = static_cast<uint64_t *>(workspace);
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
+    a.call_tag   = 0;
     a.cast       = cast;
     a.tau        = tau;
     a.arena_cursor      = arena.cursor;
@@ -85,7 +86,7 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype)
 
 size_t bt_workspace_bytes(uint64_t n)
 {
-    return bt::kWsHeaderBytes + 16 * static_cast<size_t>(ceil_div(n, bt::kMinTileElems));
+    return bt::kWsHeaderBytes + 16 + 24 * static_cast<size_t>(ceil_div(n, bt::kMinTileElems));
 }
 
 int bt_compress(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void *values, uint64_t values_capacity,

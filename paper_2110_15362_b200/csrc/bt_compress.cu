@@ -44,11 +44,19 @@
 // compactors and the compactors several tiles ahead of the copiers, so nobody
 // waits for a round trip to L2 or to HBM.
 //
-// Workspace.  It arrives with unspecified contents; the scan warps zero it and
-// meet once at the grid barrier word of the cooperative launch before the
-// first count is published, while the other warps already work on the data.
+// Workspace.  It arrives with unspecified contents and is not cleared.  A tile's
+// descriptor carries the launch's 64-bit tag in both of its halves, and a reader
+// takes only descriptors with its own launch's tag; so counts are published and
+// read from the first tile on.  Only the wave totals, being sums, need zeroed
+// words: the last copier warp of every CTA zeroes a share of them and the grid
+// meets once at the barrier word of the cooperative launch; until that meeting
+// is over the scan warps park their contributions to totals in shared memory,
+// and the copier warp adds them afterwards.  A launch of one wave has no totals
+// and no meeting.
 #include <cooperative_groups.h>
 
+#include <atomic>
+#include <chrono>
 #include <cstdlib>
 #include <mutex>
 #include <type_traits>
@@ -61,8 +69,9 @@ namespace {
 constexpr uint32_t kFull       = 0xFFFFFFFFu;
 constexpr uint64_t kWaitNs     = 2000000000ull;       // bound of every in-kernel wait: 2 s
 constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
-constexpr int      kMaxWindows = 5;                   // the grid never exceeds 32 * kMaxWindows = 160 CTAs (a B200 has 148 SMs);
-                                                      // ten windows cost 2 % on the ResNet-shaped step for predicated-off loads
+constexpr int      kMaxWindows = 5;                   // the grid never exceeds 32 * kMaxWindows CTAs
+constexpr int      kHdrSeq     = 0;                   // header words (64-bit): launch sequence number,
+constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out)
 constexpr int      kCountShift = 40;                  // wave total word: (tiles added << 40) | sum of counts
 
 #ifdef BT_PROFILE
@@ -105,11 +114,26 @@ __device__ __forceinline__ void red_add_u64(uint64_t *p, uint64_t v)
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
-// Raise the abort flag (shared and global) and report the timeout.
-__device__ __noinline__ void raise_timeout(uint32_t *ws_header, int32_t *dev_status, volatile uint32_t *s_abort)
+// A bijective mixer of 64-bit words (the finaliser of splitmix64).
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t x)
+{
+    x ^= x >> 30;
+    x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27;
+    x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return x;
+}
+
+// Raise the abort flag (shared, and global under this launch's tag if a scan warp got as far as reading it),
+// move the workspace's sequence number so that the next launch cannot take this one's words for its own, and
+// report the timeout.
+__device__ __noinline__ void raise_timeout(uint64_t *ws_header, int32_t *dev_status, volatile uint32_t *s_abort,
+                                           const uint64_t tag)
 {
     *s_abort = 1u;
-    st_relaxed_u32(ws_header + 1, 1u);
+    if (tag) st_relaxed_u64(ws_header + kHdrAbort, tag);
+    red_add_u64(ws_header + kHdrSeq, 1ull << 32);
     __threadfence();
     if (dev_status) *reinterpret_cast<volatile int32_t *>(dev_status) = BT_ERR_TIMEOUT;
 }
@@ -282,12 +306,15 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     __shared__ __align__(8) uint64_t s_counted[kStages];   // every compactor posted its count    (compactors -> scan warp)
     __shared__ __align__(8) uint64_t s_ready[kStages];     // base and offsets are in shared      (scan warp -> copiers)
     __shared__ __align__(8) uint64_t s_empty[kStages];     // every copier is done with the slot  (copiers -> load warp)
-    __shared__ __align__(8) uint64_t s_go;                 // the grid has met                    (scan warp 0 -> scan warp 1)
     __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
     __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
     __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
     __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
     __shared__ volatile uint32_t s_abort;
+    __shared__ volatile uint64_t s_tag;                    // this launch's tag once a scan warp has it, else 0
+    __shared__ volatile uint32_t s_met;                    // the grid has met: wave totals may be added to
+    __shared__ unsigned long long s_held[8];               // contributions to wave totals held back until then
+    __shared__ uint32_t          s_held_wave[8];           //   and the waves they belong to (slot = iteration & 7)
     __shared__ uint64_t          s_arena_c0;               // arena forms: the cursor as this launch found it
 
     const uint32_t tid  = threadIdx.x;
@@ -317,13 +344,15 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         // which needs a publication from every CTA, and a CTA publishes only after this barrier.
         s_arena_c0 = a.arena_cursor ? *reinterpret_cast<const volatile uint64_t *>(a.arena_cursor) : 0;
         s_abort    = 0;
+        s_tag      = 0;
+        s_met      = 0;
+        for (int k = 0; k < 8; ++k) s_held[k] = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&s_full[s], 1);
             mbar_init(&s_counted[s], kWarps);
             mbar_init(&s_ready[s], 1);
             mbar_init(&s_empty[s], kCopiers);
         }
-        mbar_init(&s_go, 1);
         fence_proxy_async();
     }
     __syncthreads();
@@ -387,54 +416,53 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         // (1.3 us under load, longer than one tile) never stalls a turn for long: a turn has two tiles' time.
         // (One warp doing every tile cannot hide that round trip however deep its software pipeline is:
         // its loads of consecutive tiles retire through the same scoreboard.)
-        const uint32_t        p            = warp - kScanWarp;
-        uint64_t *const       wave_total   = a.ws_desc;                  // one word per wave
-        uint64_t *const       desc         = a.ws_desc + a.ws_waves;     // one word per tile: (count << 1) | 1
-        const uint64_t        chunks_total = (n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
-        const uint32_t *const abort_flag   = a.ws_header + 1;
-        const uint32_t        last_it      = static_cast<uint32_t>((num_tiles - 1 - cta) / G);   // this CTA's last iteration
-        uint64_t              waves_before = 0;    // sum of the totals of the waves before this warp's previous tile
-        bool                  failed       = false;
+        const uint32_t  p            = warp - kScanWarp;
+        const bool      multi        = num_tiles > G;              // more than one wave: wave totals are in use
+        uint64_t *const wave_total   = a.ws_desc;                  // one word per wave
+        uint64_t *const desc         = a.ws_desc + a.ws_waves;     // two words per tile
+        const uint64_t  chunks_total = (n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
+        const uint32_t  last_it      = static_cast<uint32_t>((num_tiles - 1 - cta) / G);   // this CTA's last iteration
+        uint64_t        waves_before = 0;    // sum of the totals of the waves before this warp's previous tile
+        bool            failed       = false;
 
-        if (p == 0) {
-            // The workspace arrives with unspecified contents.  The first scan warps of the grid zero it between
-            // them (abort flag, wave totals, tile descriptors) and meet once, at the grid barrier word the runtime
-            // gives every cooperative launch, before any count is published.  Only the scan warps touch the
-            // workspace, so the other warps start on the data at once and the meeting hides behind the first tile.
-            // The word follows the usual sense-reversing count: CTA 0 adds 2^31 - (G - 1), every other CTA adds 1,
-            // so bit 31 flips exactly when all G have arrived and the low bits are back where they started.
-            unsigned int *const grid_bar = &cooperative_groups::details::get_grid_workspace()->barrier;
-            uint64_t *const     ws       = reinterpret_cast<uint64_t *>(a.ws_header);
-            const uint64_t      words    = kWsHeaderBytes / 8 + a.ws_waves + num_tiles;
-            for (uint64_t i = static_cast<uint64_t>(cta) * 32 + lane; i < words; i += static_cast<uint64_t>(G) * 32) ws[i] = 0;
-            __syncwarp();
-            bool met = true;
-            if (lane == 0) {
-                uint32_t       bar_old;
-                const uint32_t add = cta == 0 ? 0x80000000u - (G - 1) : 1u;
-                asm volatile("atom.add.release.gpu.u32 %0, [%1], %2;" : "=r"(bar_old) : "l"(grid_bar), "r"(add) : "memory");
-                const uint64_t t0 = now_ns();
-                for (;;) {
-                    uint32_t cur;
-                    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(grid_bar) : "memory");
-                    if ((cur ^ bar_old) & 0x80000000u) break;
-                    if (now_ns() - t0 > kWaitNs) {
-                        met = false;
-                        break;
-                    }
-                }
-                if (met) mbar_arrive(&s_go);                          // the other scan warp may publish too
+        // The tag of this launch.  Both scan warps read the same sequence number: it changes only once every CTA
+        // has published all its counts, or two seconds into a failure.
+        uint64_t seq = 0;
+        if (lane == 0) seq = ld_relaxed_u64(a.ws_header + kHdrSeq);
+        seq                   = __shfl_sync(kFull, seq, 0);
+        const uint64_t tag    = mix64(a.call_tag + seq * 0x9E3779B97F4A7C15ull) | 1ull;
+        const uint64_t tag_w0 = tag & 0xFFFFFFFF00000000ull, tag_w1 = tag << 32;
+        if (p == 0 && lane == 0) s_tag = tag;
+        auto valid = [&](const uint64_t w0, const uint64_t w1) {
+            return ((w0 ^ tag_w0) >> 32) == 0 && ((w1 ^ tag_w1) >> 32) == 0 && static_cast<uint32_t>(w0) == static_cast<uint32_t>(w1);
+        };
+
+        // Wave totals are sums made by reductions, so their words must be zero first, and the grid must have met
+        // after the zeroing before anyone adds.  That meeting is a copier warp's job (below): until it is over, a
+        // scan warp parks its contribution in shared memory and goes on -- the tagged descriptors need no clearing,
+        // so counts are published and read without waiting for the meeting.
+        auto add_to_total = [&](const uint32_t wave, const unsigned long long contribution) {     // lane 0 only
+            if (s_met) {
+                red_add_u64(wave_total + wave, contribution);
+                return;
             }
-            failed = !__shfl_sync(kFull, met, 0);
-        } else {
-            failed = !mbar_wait(&s_go, 0, &s_abort);
-        }
+            const uint32_t slot = wave & 7u;
+            s_held_wave[slot]   = wave;
+            __threadfence_block();
+            atomicExch(&s_held[slot], contribution);
+            __threadfence_block();
+            if (s_met) {
+                // the meeting ended meanwhile: whoever takes the parked value out adds it
+                const unsigned long long v = atomicExch(&s_held[slot], 0ull);
+                if (v) red_add_u64(wave_total + wave, v);
+            }
+        };
 
-        // d[k], lane l <-> descriptor of CTA l + 32k of the wave of this warp's previous tile;
+        // d0[k], d1[k], lane l <-> descriptor of CTA l + 32k of the wave of this warp's previous tile;
         // w1, w2: total words of the one and the two waves before it
-        uint64_t d[kMaxWindows], w1 = 0, w2 = 0;
+        uint64_t d0[kMaxWindows], d1[kMaxWindows], w1 = 0, w2 = 0;
 #pragma unroll
-        for (int k = 0; k < kMaxWindows; ++k) d[k] = 1ull;
+        for (int k = 0; k < kMaxWindows; ++k) d0[k] = tag_w0, d1[k] = tag_w1;
 
         for (uint32_t j = p; !failed && j <= last_it + 2; j += 2) {
             if (j <= last_it) {
@@ -456,11 +484,11 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 }
                 const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
                 if (lane == 0) {
-                    st_relaxed_u64(desc + tile_of(j), (static_cast<uint64_t>(agg) << 1) | 1ull);
-                    red_add_u64(wave_total + j, (1ull << kCountShift) + agg);
+                    st_relaxed_2xu64(desc + 2 * tile_of(j), tag_w0 | agg, tag_w1 | agg);
                     s_agg[s] = agg;
                 }
                 if (lane < kWarps) s_off[s][lane] = inc - c;
+                if (multi && lane == 0) add_to_total(j, (1ull << kCountShift) + agg);
             }
             if (j >= 2) {
                 // ---- (c): tile j - 2 <= last_it
@@ -470,27 +498,28 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 for (;;) {
                     bool missing = (f > 0 && (w1 >> kCountShift) != G) || (f > 1 && (w2 >> kCountShift) != G);
 #pragma unroll
-                    for (int k = 0; k < kMaxWindows; ++k) missing |= (d[k] & 1ull) == 0;
+                    for (int k = 0; k < kMaxWindows; ++k) missing |= !valid(d0[k], d1[k]);
                     if (!__any_sync(kFull, missing)) break;
                     PROF_ADD(11, 1);
                     __nanosleep(100);
                     if ((++polls & 255u) == 0) {
                         if (t0 == 0) t0 = now_ns();
-                        if (__any_sync(kFull, (now_ns() - t0 > kWaitNs) || ld_relaxed_u32(abort_flag) != 0)) {
+                        if (__any_sync(kFull, (now_ns() - t0 > kWaitNs) || ld_relaxed_u64(a.ws_header + kHdrAbort) == tag)) {
                             failed = true;
                             break;
                         }
                     }
 #pragma unroll
                     for (int k = 0; k < kMaxWindows; ++k)
-                        if ((d[k] & 1ull) == 0) d[k] = ld_relaxed_u64(desc + static_cast<uint64_t>(f) * G + lane + 32u * k);
+                        if (!valid(d0[k], d1[k]))
+                            ld_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(f) * G + lane + 32u * k), d0[k], d1[k]);
                     if (f > 0 && (w1 >> kCountShift) != G) w1 = ld_relaxed_u64(wave_total + (f - 1));
                     if (f > 1 && (w2 >> kCountShift) != G) w2 = ld_relaxed_u64(wave_total + (f - 2));
                 }
                 if (failed) break;
                 uint64_t part = 0;
 #pragma unroll
-                for (int k = 0; k < kMaxWindows; ++k) part += d[k] >> 1;
+                for (int k = 0; k < kMaxWindows; ++k) part += static_cast<uint32_t>(d0[k]);
                 // the waves in front of tile f: those in front of tile f - 2, and waves f - 2 and f - 1
                 waves_before += (w1 & ((1ull << kCountShift) - 1)) + (w2 & ((1ull << kCountShift) - 1));
                 const uint64_t base = waves_before + warp_sum_u64(part);
@@ -505,7 +534,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                     const uint64_t nnz = base + s_agg[ps];
                     *a.nnz_out = nnz;
                     __threadfence();
-                    const bool aborted = ld_relaxed_u32(abort_flag) != 0;
+                    const bool aborted = ld_relaxed_u64(a.ws_header + kHdrAbort) == tag;
                     uint64_t capacity = a.capacity;
                     if (a.arena_cursor) {
                         // arena form: the room left behind the cursor; the cursor moves only when everything fitted
@@ -518,6 +547,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                     }
                     if (a.dev_status)
                         *a.dev_status = aborted ? BT_ERR_TIMEOUT : (nnz > capacity ? BT_ERR_CAPACITY : BT_OK);
+                    // every CTA has published all its counts by now, so every CTA has read the sequence number:
+                    // the next launch on this workspace gets another tag
+                    red_add_u64(a.ws_header + kHdrSeq, 1ull);
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -534,13 +566,14 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
 #pragma unroll
                 for (int k = 0; k < kMaxWindows; ++k) {
                     const uint32_t b = lane + 32u * k;
-                    d[k] = (b < cta) ? ld_relaxed_u64(desc + static_cast<uint64_t>(j) * G + b) : 1ull;
+                    if (b < cta) ld_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(j) * G + b), d0[k], d1[k]);
+                    else d0[k] = tag_w0, d1[k] = tag_w1;             // not in front of this CTA: a valid count of 0
                 }
                 w1 = (j > 0) ? ld_relaxed_u64(wave_total + (j - 1)) : 0ull;
                 w2 = (j > 1) ? ld_relaxed_u64(wave_total + (j - 2)) : 0ull;
             }
         }
-        if (failed && lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort);
+        if (failed && lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort, s_tag);
         if (p == 0) { PROF_FLUSH(8, 13); }
         return;
     }
@@ -555,6 +588,45 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             const uint64_t c0 = s_arena_c0;
             vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(a.values) + c0);
             capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(V) : 0;
+        }
+        if (copier == kCopiers - 1 && num_tiles > G) {
+            // The meeting: this warp has nothing to copy for the first microseconds.  It zeroes this CTA's share of
+            // the wave totals, arrives at the grid barrier word the runtime gives every cooperative launch (the
+            // sense-reversing count grid.sync() uses: CTA 0 adds 2^31 - (G - 1), every other CTA adds 1, bit 31
+            // flips when all have arrived), waits for the flip (bounded), and then adds what the scan warps have
+            // parked meanwhile.
+            static_assert(kStages + 1 <= 8, "one parking slot per tile that can be counted before the meeting is over");
+            uint64_t *const     wave_total = a.ws_desc;
+            unsigned int *const grid_bar   = &cooperative_groups::details::get_grid_workspace()->barrier;
+            for (uint32_t i = cta * 32 + lane; i < a.ws_waves; i += G * 32) wave_total[i] = 0;
+            __syncwarp();
+            if (lane == 0) {
+                uint32_t       bar_old;
+                const uint32_t add = cta == 0 ? 0x80000000u - (G - 1) : 1u;
+                asm volatile("atom.add.release.gpu.u32 %0, [%1], %2;" : "=r"(bar_old) : "l"(grid_bar), "r"(add) : "memory");
+                const uint64_t t0 = now_ns();
+                bool           ok = true;
+                for (;;) {
+                    uint32_t cur;
+                    asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(grid_bar) : "memory");
+                    if ((cur ^ bar_old) & 0x80000000u) break;
+                    if (s_abort || now_ns() - t0 > kWaitNs) {
+                        ok = false;
+                        break;
+                    }
+                }
+                if (ok) {
+                    s_met = 1;
+                    __threadfence_block();
+                    for (int k = 0; k < 8; ++k) {
+                        const unsigned long long v = atomicExch(&s_held[k], 0ull);
+                        if (v) red_add_u64(wave_total + s_held_wave[k], v);
+                    }
+                } else {
+                    raise_timeout(a.ws_header, a.dev_status, &s_abort, s_tag);
+                }
+            }
+            __syncwarp();
         }
         for (uint32_t it = 0;; ++it) {
             if (tile_of(it) >= num_tiles) break;
@@ -597,7 +669,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         const uint64_t first = t64 * kTile;
         PROF_T(c0);
         if (!mbar_wait(&s_full[s], (it / kStages) & 1u, &s_abort)) {
-            if (lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort);
+            if (lane == 0) raise_timeout(a.ws_header, a.dev_status, &s_abort, s_tag);
             break;
         }
         PROF_T(c1);
@@ -638,6 +710,16 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         PROF_ADD(1, c2 - c1);
     }
     if (warp == 0) { PROF_FLUSH(0, 2); }
+}
+
+// A value no other call of this process gets: a counter that starts at a salt drawn from the clock and the
+// address space, so that words left in recycled memory by another run of the library do not line up either.
+uint64_t next_call_tag()
+{
+    static std::atomic<uint64_t> counter{
+        mix64(static_cast<uint64_t>(std::chrono::steady_clock::now().time_since_epoch().count()) ^
+              mix64(reinterpret_cast<uintptr_t>(&counter)))};
+    return counter.fetch_add(1, std::memory_order_relaxed);
 }
 
 // Launch shape of one kernel instantiation on one device: the opt-in shared
@@ -687,7 +769,11 @@ cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
     const uint32_t waves = (num_tiles + grid - 1) / grid;
     // cooperative launch: the runtime guarantees that all `grid` CTAs are resident together
     CompressArgs args = a;
-    args.ws_waves     = waves;
+    args.ws_waves     = (waves + 1) & ~1u;            // an even number of total words keeps the descriptors 16-byte aligned
+    args.call_tag     = next_call_tag();
+#ifdef BT_PROFILE
+    if (cudaError_t pe = cudaMemsetAsync(a.ws_header + 8, 0, kWsHeaderBytes - 64, stream); pe != cudaSuccess) return pe;
+#endif
     uint32_t     nt   = num_tiles;
     void *params[] = {&args, &nt};
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kernel), dim3(grid), dim3(kThreads), params, kSmem,

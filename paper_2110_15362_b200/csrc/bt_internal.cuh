@@ -11,11 +11,19 @@
 namespace bt {
 
 // ---------------------------------------------------------------- workspace layout
-// [0]   uint32  reserved
-// [1]   uint32  abort      set once a bounded wait ran out; every CTA then leaves
-// [2..] reserved
-// then one 64-bit total per wave of tiles, then one 64-bit descriptor per tile
-// (both sized for the smallest tile, so at most 2 words per 4096 elements)
+// The workspace arrives with unspecified contents.  It holds
+//   a 256-byte header, 64-bit words: [0] seq, the launch sequence number of this workspace; [1] abort, equal to
+//     the launch's tag once a bounded wait of that launch ran out; [8..] counters of the profile build;
+//   one 64-bit total per wave of tiles (an even number of words), zeroed by the launch itself before use;
+//   one 16-byte descriptor per tile, never cleared: word 0 = (tag >> 32) << 32 | count, word 1 = (tag & 0xFFFFFFFF)
+//     << 32 | count.  A reader takes a descriptor only if both halves carry its own launch's tag and agree on
+//     the count (the two halves may be written and read separately).
+// tag = mix64(call_tag + seq * odd) | 1: call_tag comes from the host (a process-wide counter: two calls never
+// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (the CTA of
+// the last tile adds 1 once all counts are in; a CTA that gives up adds 2^32), so replays of one captured launch
+// -- same call_tag -- get different tags too.  Memory this library never wrote matches by chance only: 2^-64
+// per word for the tag, and the repeated count on top.
+// Sized for the smallest tile: 24 bytes per 4096 elements.
 constexpr size_t   kWsHeaderBytes = 256;
 constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;
 
@@ -28,9 +36,10 @@ struct CompressArgs {
     uint64_t   *prefix;
     uint64_t   *nnz_out;
     int32_t    *dev_status;
-    uint32_t   *ws_header;
+    uint64_t   *ws_header;
     uint64_t   *ws_desc;    // wave totals, then tile descriptors
-    uint32_t    ws_waves;   // number of wave totals
+    uint32_t    ws_waves;   // number of wave-total words (even; set by launch_compress)
+    uint64_t    call_tag;   // unique to the call (set by launch_compress)
     int         cast;       // 0, or the 16-bit type (BT_F16 / BT_BF16) the stashed values of a binary32 tensor are narrowed to
     float       tau;        // fused forms: elements <= tau become +0 (0 for plain ReLU)
     // arena forms: `values` is the arena's base, the packed values go to values + *arena_cursor (bytes);
@@ -136,6 +145,15 @@ __device__ __forceinline__ uint64_t ld_relaxed_u64(const uint64_t *p)
 __device__ __forceinline__ void st_relaxed_u64(uint64_t *p, uint64_t v)
 {
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+// 16-byte descriptor accesses (the two halves may be performed separately: each is self-validating)
+__device__ __forceinline__ void ld_relaxed_2xu64(const uint64_t *p, uint64_t &w0, uint64_t &w1)
+{
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(w0), "=l"(w1) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_2xu64(uint64_t *p, uint64_t w0, uint64_t w1)
+{
+    asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(w0), "l"(w1) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t *p)
 {

@@ -6,7 +6,7 @@
 // allocation would synchronise or fail), or a plug-in that is handed its input and output buffers
 // by a runtime that owns the device memory and offers no way to ask for more.  For them the scratch
 // lives here, in a file-scope device array that every GPU loading this library carries until the
-// process exits (kScratchBytes, a quarter of a megabyte), which bounds the tensor size to
+// process exits (kScratchBytes, three eighths of a megabyte), which bounds the tensor size to
 // BT_NOALLOC_MAX_ELEMS elements.
 #include <mutex>
 
@@ -15,7 +15,7 @@
 namespace {
 
 // scratch for at most BT_NOALLOC_MAX_ELEMS elements: the same layout bt_workspace_bytes() sizes
-constexpr size_t kScratchBytes = bt::kWsHeaderBytes + 16 * (BT_NOALLOC_MAX_ELEMS / bt::kMinTileElems);
+constexpr size_t kScratchBytes = bt::kWsHeaderBytes + 16 + 24 * (BT_NOALLOC_MAX_ELEMS / bt::kMinTileElems);
 
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
@@ -74,9 +74,10 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
     a.prefix     = chunk_prefix;
     a.nnz_out    = nnz_out;
     a.dev_status = dev_status;
-    a.ws_header  = static_cast<uint32_t *>(scratch);
+    a.ws_header  = static_cast<uint64_t *>(scratch);
     a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(scratch) + bt::kWsHeaderBytes);
     a.ws_waves   = 0;
+    a.call_tag   = 0;
     a.cast       = 0;
     a.tau        = 0.0f;
     a.arena_cursor = nullptr, a.values_offset_out = nullptr, a.arena_bytes = 0;
