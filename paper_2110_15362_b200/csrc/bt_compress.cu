@@ -313,8 +313,12 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     __shared__ volatile uint32_t s_abort;
     __shared__ volatile uint64_t s_tag;                    // this launch's tag once a scan warp has it, else 0
     __shared__ volatile uint32_t s_met;                    // the grid has met: wave totals may be added to
-    __shared__ unsigned long long s_held[8];               // contributions to wave totals held back until then
-    __shared__ uint32_t          s_held_wave[8];           //   and the waves they belong to (slot = iteration & 7)
+    // Contributions to wave totals held back until then, and the waves they belong to.  Tile j can be counted before
+    // the meeting is over only while j <= kStages (tile kStages + 1 needs the slot of tile 1, whose base needs a
+    // total), so kStages + 1 slots, indexed by the wave modulo that, never collide.
+    constexpr uint32_t kHeld = kStages + 1;
+    __shared__ unsigned long long s_held[kHeld];
+    __shared__ uint32_t          s_held_wave[kHeld];
     __shared__ uint64_t          s_arena_c0;               // arena forms: the cursor as this launch found it
 
     const uint32_t tid  = threadIdx.x;
@@ -346,7 +350,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         s_abort    = 0;
         s_tag      = 0;
         s_met      = 0;
-        for (int k = 0; k < 8; ++k) s_held[k] = 0;
+        for (uint32_t k = 0; k < kHeld; ++k) s_held[k] = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&s_full[s], 1);
             mbar_init(&s_counted[s], kWarps);
@@ -446,7 +450,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 red_add_u64(wave_total + wave, contribution);
                 return;
             }
-            const uint32_t slot = wave & 7u;
+            const uint32_t slot = wave % kHeld;
             s_held_wave[slot]   = wave;
             __threadfence_block();
             atomicExch(&s_held[slot], contribution);
@@ -595,7 +599,6 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             // sense-reversing count grid.sync() uses: CTA 0 adds 2^31 - (G - 1), every other CTA adds 1, bit 31
             // flips when all have arrived), waits for the flip (bounded), and then adds what the scan warps have
             // parked meanwhile.
-            static_assert(kStages + 1 <= 8, "one parking slot per tile that can be counted before the meeting is over");
             uint64_t *const     wave_total = a.ws_desc;
             unsigned int *const grid_bar   = &cooperative_groups::details::get_grid_workspace()->barrier;
             for (uint32_t i = cta * 32 + lane; i < a.ws_waves; i += G * 32) wave_total[i] = 0;
@@ -618,7 +621,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 if (ok) {
                     s_met = 1;
                     __threadfence_block();
-                    for (int k = 0; k < 8; ++k) {
+                    for (uint32_t k = 0; k < kHeld; ++k) {
                         const unsigned long long v = atomicExch(&s_held[k], 0ull);
                         if (v) red_add_u64(wave_total + s_held_wave[k], v);
                     }
