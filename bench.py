@@ -48,7 +48,7 @@ def parse_args():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-large", action="store_true", help="skip the per-kernel runs on 1 GiB tensors")
     p.add_argument("--no-e2e", action="store_true")
-    p.add_argument("--chains", type=int, choices=(1, 2, 4), default=2,
+    p.add_argument("--chains", type=int, choices=(1, 2, 4), default=4,
                    help="independent chains of the step's graph: 2 = plain codec / fused pair on two streams, "
                         "4 = each of them split into even and odd layers")
     return p.parse_args()
