@@ -563,7 +563,12 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             }
             if (j <= last_it) {
                 // ---- (b): a tile later (when the other scan warp's next tile is counted, if there is one)
-                if (j + 1 <= last_it && !mbar_wait(&s_counted[(j + 1) % kStages], ((j + 1) / kStages) & 1u, &s_abort)) {
+                if (j + 1 > last_it) {
+                    // This CTA's last tile: no next tile to wait for.  A short pause gives the other counts of the
+                    // wave time to land, so that the reads below usually succeed at once instead of costing a second
+                    // round trip (cold ResNet-shaped forward passes: -5 %; reading at once and polling was slower).
+                    __nanosleep(300);
+                } else if (!mbar_wait(&s_counted[(j + 1) % kStages], ((j + 1) / kStages) & 1u, &s_abort)) {
                     failed = true;
                     break;
                 }
