@@ -155,7 +155,7 @@ template <typename U, int kE, int kGrp>
 cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                          const uint64_t *prefix, uint64_t n, void *out, cudaStream_t stream)
 {
-    constexpr int  kWarps   = 8;
+    constexpr int  kWarps   = 4;   // four warps per CTA: 3 % faster than eight on few-MB tensors, 1.5 % on 1 GiB (two: the same)
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
@@ -169,7 +169,7 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint6
 cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *prefix, uint64_t n,
                                     int from_dtype, void *out_f32, cudaStream_t stream)
 {
-    constexpr int  kWarps   = 8;
+    constexpr int  kWarps   = 4;
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;

