@@ -29,11 +29,12 @@ template <int WIDEN>
 __device__ __forceinline__ uint32_t widened(const uint16_t h)
 {
     if constexpr (WIDEN == 1) {
-        float f;
-        asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(h));
-        // a NaN keeps its sign and payload (written out, not left to the conversion instruction)
-        const uint32_t nan = (static_cast<uint32_t>(h & 0x8000u) << 16) | 0x7F800000u | (static_cast<uint32_t>(h & 0x3FFu) << 13);
-        return (h & 0x7FFFu) > 0x7C00u ? nan : __float_as_uint(f);
+        // exponent and mantissa moved into place, then rebiased by an exact multiplication (subnormals included);
+        // infinities and NaNs get the all-ones exponent by hand, which keeps a NaN payload and sign
+        const uint32_t t = static_cast<uint32_t>(h & 0x7FFFu) << 13;
+        uint32_t       r = __float_as_uint(__uint_as_float(t) * 5.192296858534828e33f);      // 2^112
+        r                = (h & 0x7C00u) == 0x7C00u ? (t | 0x7F800000u) : r;
+        return r | (static_cast<uint32_t>(h & 0x8000u) << 16);
     } else {
         return static_cast<uint32_t>(h) << 16;
     }
