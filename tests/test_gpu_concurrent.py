@@ -38,3 +38,53 @@ def test_two_streams_compress_concurrently(oracle, n):
             assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), c.bitmap)
             assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), c.prefix)
             assert np.array_equal(W.raw_numpy(st.values[:c.nnz]), c.values)
+
+
+def test_graph_replays_share_one_workspace_across_sizes():
+    """A captured graph of launches of different sizes and element types that share ONE workspace, replayed many
+    times with the inputs changed in between: every replay's words in the workspace must be told from the
+    previous replay's (same captured arguments) and from the other launches' (other sizes, same memory)."""
+    B.lib()
+    dev = torch.device("cuda")
+    sizes = [(8192 * 300 + 11, torch.float32), (8192 * 3 + 5, torch.float32), (16384 * 200 + 3, torch.bfloat16),
+             (8192 * 149, torch.float32), (77, torch.float32), (4096 * 148 * 3 + 1, torch.float64)]
+    xs = [torch.zeros(n, dtype=dt, device=dev) for n, dt in sizes]
+    stashes = [B.Stash(n, dt, dev) for n, dt in sizes]
+    ws = B.new_workspace(max(n for n, _ in sizes), dev)
+    ws.random_(0, 255)
+    gen = torch.Generator(device=dev).manual_seed(5)
+
+    def refill():
+        for x in xs:
+            t = torch.randn(x.numel(), device=dev, generator=gen)
+            x.copy_(torch.where(torch.rand(x.numel(), device=dev, generator=gen) < 0.6, torch.zeros((), device=dev), t).to(x.dtype))
+
+    def launch_all():
+        for x, st in zip(xs, stashes):
+            B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+
+    refill()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        launch_all()                                          # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        launch_all()
+    iv = {2: torch.int16, 4: torch.int32, 8: torch.int64}
+    for rep in range(40):
+        refill()
+        g.replay()
+        if rep % 3 == 0:
+            g.replay()                                        # the same inputs twice in a row as well
+        torch.cuda.synchronize()
+        for x, st in zip(xs, stashes):
+            bits = x.view(iv[x.element_size()])
+            mask = bits != 0
+            nnz = int(mask.sum())
+            assert st.status == B.BT_OK and st.nnz == nnz, (rep, x.numel())
+            assert torch.equal(st.values[:nnz].view(bits.dtype), bits[mask]), (rep, x.numel())
+            back = torch.empty_like(x)
+            B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, back)
+            assert torch.equal(back.view(bits.dtype), bits), (rep, x.numel())
