@@ -82,6 +82,6 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
     a.tau        = 0.0f;
     a.arena_cursor = nullptr, a.values_offset_out = nullptr, a.arena_bytes = 0;
     a.n          = n;
-    // the launcher clears the part of the scratch this call uses (it keeps the last call's contents otherwise)
+    // nothing in the scratch is cleared between calls: the kernel tells this call's words by their tag
     return bt::launch_compress(a, dtype, false, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
