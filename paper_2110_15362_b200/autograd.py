@@ -256,16 +256,16 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
         return obj.unpack() if isinstance(obj, PackedActivation) else obj
 
     def __enter__(self):
+        # status words the previous pass left unchecked (its backward pass may have run outside the context, or
+        # asked for nothing): one host read here, where no launch of the new pass is waiting behind it
+        self.check_statuses()
         if self.cursor is not None:
             self.cursor.zero_()                 # a new pass: the arena is empty again
-            self.statuses.clear()
         super().__enter__()
         return self
 
     def __exit__(self, *exc):
         self._shared.clear()
-        if exc[0] is None:
-            self.check_statuses()
         return super().__exit__(*exc)
 
 

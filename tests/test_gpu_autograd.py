@@ -306,7 +306,8 @@ def test_maxpool_stash_matches_torch(A, dtype):
     with A.stash_saved_activations(min_numel=1024) as hooks:             # bitmap-only ReLU in front of the pooling
         got3 = run_net(lambda t: A.relu_stash(t, hooks, keep_values=False), A.maxpool2x2_stash)
         assert hooks.loose_statuses and hooks._lookup(torch.zeros(1)) is None
-    assert not hooks.loose_statuses                                       # checked on leaving the context
+    hooks.check_statuses()                                                # also done on entering the next pass
+    assert not hooks.loose_statuses
     with A.stash_saved_activations(min_numel=1024, arena_bytes=32 << 20) as hooks:
         got4 = run_net(lambda t: A.relu_stash(t, hooks, keep_values=False), A.maxpool2x2_stash)
         used = int(hooks.cursor.item())
