@@ -97,9 +97,10 @@ def _flat_input(t: torch.Tensor) -> torch.Tensor:
 class _Scratch:
     """Per-device reusable buffers of the packing calls: workspace and a full-capacity values buffer."""
 
-    def __init__(self):
+    def __init__(self, two_pass: bool = True):
         self.ws: Dict[torch.device, torch.Tensor] = {}
         self.values: Dict[Tuple[torch.device, torch.dtype], torch.Tensor] = {}
+        self.two_pass = two_pass         # exact-size values without a full-capacity buffer (see _compress)
 
     def workspace(self, n: int, device) -> torch.Tensor:
         need = B.bt_workspace_bytes(n)
@@ -127,8 +128,27 @@ def _compress(flat: torch.Tensor, scratch: _Scratch, relu_into: Optional[torch.T
     prefix = torch.empty((n + B.CHUNK - 1) // B.CHUNK, dtype=torch.int64, device=dev)
     nnz_out = torch.empty(1, dtype=torch.int64, device=dev)
     status = torch.empty(1, dtype=torch.int32, device=dev)
-    full = scratch.full_values(n, narrow or flat.dtype, dev)
     ws = scratch.workspace(n, dev)
+    if scratch.two_pass and narrow is None:
+        # Two passes instead of a values buffer of full capacity: the compressor with no room for values gives
+        # bitmap, prefix and nnz (BT_ERR_CAPACITY is its expected answer), the host reads nnz, and the masked
+        # gather fills a buffer of exactly that size from the activation.  Costs the gather (cheaper than a
+        # compaction); saves a buffer as large as the largest activation for the whole step.
+        if relu6:
+            B.bt_relu6_fwd_compress(flat, relu_into, bitmap, None, prefix, nnz_out, ws, status, n=n, values_capacity=0)
+        elif relu_into is None:
+            B.bt_compress(flat, bitmap, None, prefix, nnz_out, ws, status, n=n, values_capacity=0)
+        else:
+            B.bt_relu_fwd_compress(flat, relu_into, bitmap, None, prefix, nnz_out, ws, status, n=n, values_capacity=0)
+        nnz = int(nnz_out.item())
+        st = int(status.item())
+        if st not in (B.BT_OK, B.BT_ERR_CAPACITY):
+            raise B.BitTrainError("bt_compress (autograd stash)", st)
+        values = torch.empty(nnz, dtype=flat.dtype, device=dev)
+        if nnz:
+            B.bt_mask_compress(flat if relu_into is None else relu_into, bitmap, prefix, None, values, n=n)
+        return bitmap, values, prefix, nnz
+    full = scratch.full_values(n, narrow or flat.dtype, dev)
     if relu6:
         B.bt_relu6_fwd_compress(flat, relu_into, bitmap, full, prefix, nnz_out, ws, status, n=n, values_capacity=n)
     elif narrow is not None and relu_into is None:
@@ -168,10 +188,12 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
     """Context manager: saved activations are kept compressed between the forward and the backward pass.
     `arena_bytes`: keep all values in one pre-allocated arena of that size behind a device-side cursor (no
     host read per tensor; a RuntimeError at the first unpack if the arena was too small).  `narrow`
-    (torch.float16 / torch.bfloat16): float32 activations are stashed with values of that type (lossy)."""
+    (torch.float16 / torch.bfloat16): float32 activations are stashed with values of that type (lossy).
+    `two_pass` (exact-size mode): size the values by a first pass without values and fill them with a masked
+    gather, instead of compacting into a buffer of full capacity that stays allocated (default)."""
 
     def __init__(self, min_numel: int = 1 << 14, min_saving: float = 0.1, arena_bytes: Optional[int] = None,
-                 device="cuda", narrow: Optional[torch.dtype] = None):
+                 device="cuda", narrow: Optional[torch.dtype] = None, two_pass: bool = True):
         if narrow not in (None, torch.float16, torch.bfloat16):
             raise ValueError("narrow must be torch.float16 or torch.bfloat16")
         if narrow is not None and arena_bytes is not None:
@@ -183,7 +205,7 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
         if arena_bytes is not None:
             self.arena = torch.empty((arena_bytes + 15) // 16 * 16, dtype=torch.uint8, device=device)
             self.cursor = torch.zeros(1, dtype=torch.int64, device=device)
-        self.scratch = _Scratch()
+        self.scratch = _Scratch(two_pass)
         self.packed_bytes = 0            # bytes kept in compressed form so far
         self.dense_bytes = 0             # bytes the same tensors would have taken
         self._shared: Dict[int, Tuple[weakref.ref, weakref.ref]] = {}
