@@ -165,8 +165,8 @@ int bt_prune_fwd_compress(const void *x, uint64_t n, int dtype, float tau, void 
  * bit), every NaN gives 0x7FFF.  bt_decompress with to_dtype restores the
  * narrowed dense tensor; bt_compressed_bytes(n, nnz, to_dtype) is the stash's
  * size.  y_out (BT_F32, may be NULL, may alias x) receives the unnarrowed
- * activation.  Lossy by design; no arena and no host-buffer form.  Other
- * parameters and *dev_status as bt_compress.
+ * activation.  Lossy by design; no host-buffer form (arena forms below).
+ * Other parameters and *dev_status as bt_compress.
  */
 int bt_compress_narrow(const void *dense, uint64_t n, int to_dtype,
                        uint32_t *bitmap, void *values, uint64_t values_capacity,
@@ -326,6 +326,38 @@ int bt_prune_fwd_compress_arena(const void *x, uint64_t n, int dtype, float tau,
 /* values_offset: the device word a *_arena compressor wrote (byte offset of the values inside the arena) */
 int bt_decompress_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
                         const uint64_t *chunk_prefix, uint64_t n, int dtype, void *dense_out, void *stream);
+
+/*
+ * Arena forms of the later calls.  The narrowing compressors push 16-bit values: the cursor advances by
+ * 2 * nnz bytes rounded up to 16, and the room behind the cursor is counted in 16-bit elements;
+ * bt_decompress_widen_arena (or bt_decompress_arena with the 16-bit type) reads them back.  The ReLU6
+ * pair pushes and reads values of the tensor's own type.  Everything else as in the arena forms above
+ * and in bt_compress_narrow / bt_prune_fwd_compress_narrow / bt_decompress_widen / bt_relu6_fwd_compress
+ * / bt_relu6_bwd_from_stash.
+ */
+int bt_compress_narrow_arena(const void *dense, uint64_t n, int to_dtype, uint32_t *bitmap,
+                             void *arena, uint64_t arena_bytes, uint64_t *arena_cursor,
+                             uint64_t *values_offset_out, uint64_t *chunk_prefix, uint64_t *nnz_out,
+                             void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+int bt_prune_fwd_compress_narrow_arena(const void *x, uint64_t n, int to_dtype, float tau, void *y_out,
+                                       uint32_t *bitmap, void *arena, uint64_t arena_bytes,
+                                       uint64_t *arena_cursor, uint64_t *values_offset_out,
+                                       uint64_t *chunk_prefix, uint64_t *nnz_out,
+                                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+int bt_decompress_widen_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
+                              const uint64_t *chunk_prefix, uint64_t n, int from_dtype, void *dense_out,
+                              void *stream);
+
+int bt_relu6_fwd_compress_arena(const void *pre_act, uint64_t n, int dtype, void *y_out, uint32_t *bitmap,
+                                void *arena, uint64_t arena_bytes, uint64_t *arena_cursor,
+                                uint64_t *values_offset_out, uint64_t *chunk_prefix, uint64_t *nnz_out,
+                                void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream);
+
+int bt_relu6_bwd_from_stash_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
+                                  const uint64_t *chunk_prefix, const void *grad_out, uint64_t n, int dtype,
+                                  void *grad_in, void *stream);
 
 /*
  * Host-buffer forms.  The paper's own implementation keeps the stash in host

@@ -33,7 +33,8 @@ the values of the pooled layer's input are then held by nothing, only its bitmap
 pass reads the stashed values as well, which are the ones the next layer's saved input shares).  With
 ``stash_saved_activations(narrow=torch.float16)`` (or ``torch.bfloat16``) float32 activations are stashed with
 16-bit values (``bt_compress_narrow`` / ``bt_decompress_widen``): lossy -- what the backward pass gets back is
-the activation rounded to the narrow type -- and not combined with the arena.
+the activation rounded to the narrow type.  Both work inside an arena context as well (the ``*_arena`` forms of
+those calls); a ReLU6 stash is never narrowed.
 """
 from __future__ import annotations
 
@@ -50,15 +51,18 @@ __all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUSta
 
 class PackedActivation:
     """What replaces a saved tensor: the stash and the metadata needed to rebuild it.  `values` is either the
-    exact-size vector of values, or (arena mode) None with `arena`, `offset` (device word) and `owner` set."""
+    exact-size vector of values, or (arena mode) None with `arena`, `offset` (device word), `owner` and `stored`
+    (the dtype of the values in the arena) set."""
 
     __slots__ = ("bitmap", "values", "chunk_prefix", "shape", "dtype", "device", "nnz", "arena", "offset", "owner",
-                 "__weakref__")
+                 "stored", "__weakref__")
 
-    def __init__(self, bitmap, values, chunk_prefix, shape, dtype, device, nnz, arena=None, offset=None, owner=None):
+    def __init__(self, bitmap, values, chunk_prefix, shape, dtype, device, nnz, arena=None, offset=None, owner=None,
+                 stored=None):
         self.bitmap, self.values, self.chunk_prefix = bitmap, values, chunk_prefix
         self.shape, self.dtype, self.device, self.nnz = shape, dtype, device, nnz
         self.arena, self.offset, self.owner = arena, offset, owner
+        self.stored = stored if stored is not None else (dtype if values is None else values.dtype)
 
     @property
     def numel(self) -> int:
@@ -70,13 +74,17 @@ class PackedActivation:
     def nbytes(self) -> int:
         """Bytes of the stash (arena mode: reads nnz from the device)."""
         nnz = int(self.nnz.item()) if isinstance(self.nnz, torch.Tensor) else self.nnz
-        return B.bt_compressed_bytes(self.numel, nnz, self.dtype if self.values is None else self.values.dtype)
+        return B.bt_compressed_bytes(self.numel, nnz, self.stored)
 
     def unpack(self) -> torch.Tensor:
         out = torch.empty(self.shape, dtype=self.dtype, device=self.device)
         if self.arena is not None:
             self.owner.check_statuses()
-            B.bt_decompress_arena(self.bitmap, self.arena, self.offset, self.chunk_prefix, out.view(-1))
+            if self.stored != self.dtype:              # a narrowed stash of a float32 tensor
+                B.bt_decompress_widen_arena(self.bitmap, self.arena, self.offset, self.chunk_prefix, self.stored,
+                                            out.view(-1))
+            else:
+                B.bt_decompress_arena(self.bitmap, self.arena, self.offset, self.chunk_prefix, out.view(-1))
         elif self.values.dtype != self.dtype:          # a narrowed stash of a float32 tensor
             B.bt_decompress_widen(self.bitmap, self.values, self.chunk_prefix, out.view(-1))
         else:
@@ -167,21 +175,32 @@ def _compress(flat: torch.Tensor, scratch: _Scratch, relu_into: Optional[torch.T
     return bitmap, full[:nnz].clone(), prefix, nnz
 
 
-def _compress_arena(flat: torch.Tensor, owner, relu_into: Optional[torch.Tensor] = None):
-    """Arena form of `_compress`: nothing is read back; returns bitmap, prefix, nnz word, offset word."""
+def _compress_arena(flat: torch.Tensor, owner, relu_into: Optional[torch.Tensor] = None, relu6: bool = False):
+    """Arena form of `_compress`: nothing is read back; returns bitmap, prefix, nnz word, offset word and the
+    dtype of the values pushed (the owner's narrow type for a float32 tensor, except under ReLU6)."""
     n, dev = flat.numel(), flat.device
+    narrow = owner.narrow if (flat.dtype == torch.float32 and not relu6) else None
     bitmap = torch.empty((n + 31) // 32, dtype=torch.int32, device=dev)
     prefix = torch.empty((n + B.CHUNK - 1) // B.CHUNK, dtype=torch.int64, device=dev)
     words = torch.empty(2, dtype=torch.int64, device=dev)               # nnz, byte offset of the values
     status = torch.empty(1, dtype=torch.int32, device=dev)
     ws = owner.scratch.workspace(n, dev)
-    if relu_into is None:
+    if relu6:
+        B.bt_relu6_fwd_compress_arena(flat, relu_into, bitmap, owner.arena, owner.cursor, words[1:], prefix, words[:1],
+                                      ws, status, n=n)
+    elif narrow is not None and relu_into is None:
+        B.bt_compress_narrow_arena(flat, narrow, bitmap, owner.arena, owner.cursor, words[1:], prefix, words[:1], ws,
+                                   status, n=n)
+    elif narrow is not None:
+        B.bt_prune_fwd_compress_narrow_arena(flat, narrow, 0.0, relu_into, bitmap, owner.arena, owner.cursor, words[1:],
+                                             prefix, words[:1], ws, status, n=n)
+    elif relu_into is None:
         B.bt_compress_arena(flat, bitmap, owner.arena, owner.cursor, words[1:], prefix, words[:1], ws, status, n=n)
     else:
         B.bt_prune_fwd_compress_arena(flat, 0.0, relu_into, bitmap, owner.arena, owner.cursor, words[1:], prefix,
                                       words[:1], ws, status, n=n)
     owner.statuses.append(status)
-    return bitmap, prefix, words[:1], words[1:]
+    return bitmap, prefix, words[:1], words[1:], narrow or flat.dtype
 
 
 class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
@@ -196,8 +215,6 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
                  device="cuda", narrow: Optional[torch.dtype] = None, two_pass: bool = True):
         if narrow not in (None, torch.float16, torch.bfloat16):
             raise ValueError("narrow must be torch.float16 or torch.bfloat16")
-        if narrow is not None and arena_bytes is not None:
-            raise ValueError("the narrowing forms have no arena variant")
         self.min_numel, self.min_saving, self.narrow = min_numel, min_saving, narrow
         self.arena = self.cursor = None
         self.statuses: list = []
@@ -258,9 +275,9 @@ class stash_saved_activations(torch.autograd.graph.saved_tensors_hooks):
             return shared
         n, es = t.numel(), t.element_size()
         if self.arena is not None:
-            bitmap, prefix, nnz_word, off_word = _compress_arena(t.detach().view(-1), self)
+            bitmap, prefix, nnz_word, off_word, stored = _compress_arena(t.detach().view(-1), self)
             packed = PackedActivation(bitmap, None, prefix, tuple(t.shape), t.dtype, t.device, nnz_word,
-                                      arena=self.arena, offset=off_word, owner=self)
+                                      arena=self.arena, offset=off_word, owner=self, stored=stored)
             self.share(t, packed)
             self.dense_bytes += n * es
             return packed
@@ -321,10 +338,10 @@ class ReLUStash(torch.autograd.Function):
             ctx.save_for_backward(bitmap)
             return y
         if hooks is not None and hooks.arena is not None:
-            bitmap, prefix, nnz_word, off_word = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1))
+            bitmap, prefix, nnz_word, off_word, stored = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1))
             ctx.save_for_backward(bitmap)
             hooks.share(y, PackedActivation(bitmap, None, prefix, tuple(y.shape), y.dtype, y.device, nnz_word,
-                                            arena=hooks.arena, offset=off_word, owner=hooks))
+                                            arena=hooks.arena, offset=off_word, owner=hooks, stored=stored))
             hooks.dense_bytes += y.numel() * y.element_size()
             return y
         scratch = hooks.scratch if hooks is not None else _Scratch()
@@ -360,8 +377,8 @@ def relu_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None,
 
 class ReLU6Stash(torch.autograd.Function):
     """ReLU6 with the stash fused into its forward pass; the backward pass reads the bitmap and the stashed
-    values (a stored 6 marks a saturated unit).  Always exact-size values (one host read), also inside an
-    arena context; never narrowed (the backward pass compares the stored values with 6)."""
+    values (a stored 6 marks a saturated unit).  Exact-size values (one host read), or inside an arena context
+    values in the arena; never narrowed (the backward pass compares the stored values with 6)."""
 
     @staticmethod
     def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None, inplace: bool = False):
@@ -371,6 +388,16 @@ class ReLU6Stash(torch.autograd.Function):
         else:
             xc = _flat_input(x)
             y = torch.empty_like(xc)
+        ctx.owner = None
+        if hooks is not None and hooks.arena is not None:
+            bitmap, prefix, nnz_word, off_word, stored = _compress_arena(xc.view(-1), hooks, relu_into=y.view(-1),
+                                                                         relu6=True)
+            ctx.owner = hooks
+            ctx.save_for_backward(bitmap, off_word, prefix)
+            hooks.share(y, PackedActivation(bitmap, None, prefix, tuple(y.shape), y.dtype, y.device, nnz_word,
+                                            arena=hooks.arena, offset=off_word, owner=hooks, stored=stored))
+            hooks.dense_bytes += y.numel() * y.element_size()
+            return y
         scratch = hooks.scratch if hooks is not None else _Scratch()
         bitmap, values, prefix, nnz = _compress(xc.view(-1), scratch, relu_into=y.view(-1), relu6=True)
         ctx.save_for_backward(bitmap, values, prefix)
@@ -386,7 +413,11 @@ class ReLU6Stash(torch.autograd.Function):
         g = _flat_input(grad)
         gin = torch.empty_like(g)
         bitmap, values, prefix = ctx.saved_tensors
-        B.bt_relu6_bwd_from_stash(bitmap, values, prefix, g.view(-1), gin.view(-1))
+        if ctx.owner is not None:                      # arena mode: `values` is the offset word
+            ctx.owner.check_statuses()
+            B.bt_relu6_bwd_from_stash_arena(bitmap, ctx.owner.arena, values, prefix, g.view(-1), gin.view(-1))
+        else:
+            B.bt_relu6_bwd_from_stash(bitmap, values, prefix, g.view(-1), gin.view(-1))
         return gin, None, None
 
 

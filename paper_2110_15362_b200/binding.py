@@ -29,7 +29,9 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_decompress_host", "bt_relu_fwd_compress_host", "bt_relu_bwd_from_bitmap_host", "bt_compress_noalloc",
            "bt_prune_fwd_compress", "bt_mask_compress", "bt_compress_arena", "bt_prune_fwd_compress_arena",
            "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
-           "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd")
+           "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd",
+           "bt_compress_narrow_arena", "bt_prune_fwd_compress_narrow_arena", "bt_decompress_widen_arena",
+           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -91,6 +93,17 @@ def lib() -> ctypes.CDLL:
         L.bt_maxpool2x2_fwd.restype = i32
         L.bt_maxpool2x2_bwd.argtypes = [vp, vp, u64, u64, u64, i32, vp, vp]
         L.bt_maxpool2x2_bwd.restype = i32
+        L.bt_compress_narrow_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.bt_compress_narrow_arena.restype = i32
+        L.bt_prune_fwd_compress_narrow_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz,
+                                                         vp, vp]
+        L.bt_prune_fwd_compress_narrow_arena.restype = i32
+        L.bt_decompress_widen_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
+        L.bt_decompress_widen_arena.restype = i32
+        L.bt_relu6_fwd_compress_arena.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.bt_relu6_fwd_compress_arena.restype = i32
+        L.bt_relu6_bwd_from_stash_arena.argtypes = [vp, vp, vp, vp, vp, u64, i32, vp, vp]
+        L.bt_relu6_bwd_from_stash_arena.restype = i32
         L.bt_compress_noalloc.restype = i32
         L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
         L.bt_host_staging_bytes.restype = sz
@@ -290,6 +303,69 @@ def bt_decompress_arena(bitmap: torch.Tensor, arena: torch.Tensor, values_offset
     st = lib().bt_decompress_arena(_ptr(bitmap), _ptr(arena), _ptr(values_offset), _ptr(chunk_prefix), n,
                                    DTYPE_CODE[dense_out.dtype], _ptr(dense_out), _stream(stream))
     return _check("bt_decompress_arena", st, check)
+
+
+def bt_compress_narrow_arena(dense: torch.Tensor, to_dtype: torch.dtype, bitmap: torch.Tensor, arena: torch.Tensor,
+                             arena_cursor: torch.Tensor, values_offset_out: torch.Tensor, chunk_prefix: torch.Tensor,
+                             nnz_out: torch.Tensor, workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                             *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """bt_compress_narrow whose 16-bit values (of `to_dtype`) go behind the cursor of a caller-owned arena."""
+    n = dense.numel() if n is None else n
+    assert dense.dtype == torch.float32
+    st = lib().bt_compress_narrow_arena(_ptr(dense), n, DTYPE_CODE[to_dtype], _ptr(bitmap), _ptr(arena), _nbytes(arena),
+                                        _ptr(arena_cursor), _ptr(values_offset_out), _ptr(chunk_prefix), _ptr(nnz_out),
+                                        _ptr(workspace), _nbytes(workspace), _ptr(dev_status), _stream(stream))
+    return _check("bt_compress_narrow_arena", st, check)
+
+
+def bt_prune_fwd_compress_narrow_arena(x: torch.Tensor, to_dtype: torch.dtype, tau: float, y_out: Optional[torch.Tensor],
+                                       bitmap: torch.Tensor, arena: torch.Tensor, arena_cursor: torch.Tensor,
+                                       values_offset_out: torch.Tensor, chunk_prefix: torch.Tensor, nnz_out: torch.Tensor,
+                                       workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,
+                                       *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """bt_prune_fwd_compress_narrow whose 16-bit values (of `to_dtype`) go behind the cursor of a caller-owned arena."""
+    n = x.numel() if n is None else n
+    assert x.dtype == torch.float32
+    st = lib().bt_prune_fwd_compress_narrow_arena(_ptr(x), n, DTYPE_CODE[to_dtype], ctypes.c_float(tau), _ptr(y_out),
+                                                  _ptr(bitmap), _ptr(arena), _nbytes(arena), _ptr(arena_cursor),
+                                                  _ptr(values_offset_out), _ptr(chunk_prefix), _ptr(nnz_out),
+                                                  _ptr(workspace), _nbytes(workspace), _ptr(dev_status), _stream(stream))
+    return _check("bt_prune_fwd_compress_narrow_arena", st, check)
+
+
+def bt_decompress_widen_arena(bitmap: torch.Tensor, arena: torch.Tensor, values_offset: torch.Tensor,
+                              chunk_prefix: torch.Tensor, from_dtype: torch.dtype, dense_out: torch.Tensor,
+                              *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """Restores a narrowed stash whose 16-bit values (of `from_dtype`) sit in an arena into a float32 tensor."""
+    n = dense_out.numel() if n is None else n
+    assert dense_out.dtype == torch.float32
+    st = lib().bt_decompress_widen_arena(_ptr(bitmap), _ptr(arena), _ptr(values_offset), _ptr(chunk_prefix), n,
+                                         DTYPE_CODE[from_dtype], _ptr(dense_out), _stream(stream))
+    return _check("bt_decompress_widen_arena", st, check)
+
+
+def bt_relu6_fwd_compress_arena(pre_act: torch.Tensor, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,
+                                arena: torch.Tensor, arena_cursor: torch.Tensor, values_offset_out: torch.Tensor,
+                                chunk_prefix: torch.Tensor, nnz_out: torch.Tensor, workspace: torch.Tensor,
+                                dev_status: Optional[torch.Tensor] = None, *, n: Optional[int] = None, stream=None,
+                                check: bool = True) -> int:
+    """Fused ReLU6 forward whose values go behind the cursor of a caller-owned arena."""
+    n = pre_act.numel() if n is None else n
+    st = lib().bt_relu6_fwd_compress_arena(_ptr(pre_act), n, DTYPE_CODE[pre_act.dtype], _ptr(y_out), _ptr(bitmap),
+                                           _ptr(arena), _nbytes(arena), _ptr(arena_cursor), _ptr(values_offset_out),
+                                           _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace), _nbytes(workspace),
+                                           _ptr(dev_status), _stream(stream))
+    return _check("bt_relu6_fwd_compress_arena", st, check)
+
+
+def bt_relu6_bwd_from_stash_arena(bitmap: torch.Tensor, arena: torch.Tensor, values_offset: torch.Tensor,
+                                  chunk_prefix: torch.Tensor, grad_out: torch.Tensor, grad_in: torch.Tensor,
+                                  *, n: Optional[int] = None, stream=None, check: bool = True) -> int:
+    """ReLU6 backward from a stash whose values sit in an arena."""
+    n = grad_out.numel() if n is None else n
+    st = lib().bt_relu6_bwd_from_stash_arena(_ptr(bitmap), _ptr(arena), _ptr(values_offset), _ptr(chunk_prefix),
+                                             _ptr(grad_out), n, DTYPE_CODE[grad_out.dtype], _ptr(grad_in), _stream(stream))
+    return _check("bt_relu6_bwd_from_stash_arena", st, check)
 
 
 def bt_relu6_fwd_compress(pre_act: torch.Tensor, y_out: Optional[torch.Tensor], bitmap: torch.Tensor,

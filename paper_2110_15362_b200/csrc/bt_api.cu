@@ -149,7 +149,7 @@ int bt_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values, const ui
     if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(grad_out, 16) ||
         !aligned(grad_in, 16))
         return BT_ERR_ALIGN;
-    return bt::launch_relu6_bwd(bitmap, values, chunk_prefix, grad_out, n, dtype, grad_in,
+    return bt::launch_relu6_bwd(bitmap, values, nullptr, chunk_prefix, grad_out, n, dtype, grad_in,
                                 static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? BT_OK
                : BT_ERR_CUDA;
@@ -194,6 +194,76 @@ int bt_decompress_arena(const uint32_t *bitmap, const void *arena, const uint64_
                : BT_ERR_CUDA;
 }
 
+int bt_compress_narrow_arena(const void *dense, uint64_t n, int to_dtype, uint32_t *bitmap, void *arena,
+                             uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offset_out,
+                             uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace, size_t workspace_bytes,
+                             int32_t *dev_status, void *stream)
+{
+    if (to_dtype != BT_F16 && to_dtype != BT_BF16) return BT_ERR_DTYPE;
+    if (!arena_cursor) return BT_ERR_NULL;
+    Arena ar;
+    ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
+    return compress_common(dense, n, BT_F32, 0, 0.0f, nullptr, bitmap, arena, arena_bytes, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream, ar, to_dtype);
+}
+
+int bt_prune_fwd_compress_narrow_arena(const void *x, uint64_t n, int to_dtype, float tau, void *y_out, uint32_t *bitmap,
+                                       void *arena, uint64_t arena_bytes, uint64_t *arena_cursor,
+                                       uint64_t *values_offset_out, uint64_t *chunk_prefix, uint64_t *nnz_out,
+                                       void *workspace, size_t workspace_bytes, int32_t *dev_status, void *stream)
+{
+    if (to_dtype != BT_F16 && to_dtype != BT_BF16) return BT_ERR_DTYPE;
+    if (!arena_cursor) return BT_ERR_NULL;
+    Arena ar;
+    ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
+    return compress_common(x, n, BT_F32, 1, tau, y_out, bitmap, arena, arena_bytes, chunk_prefix, nnz_out, workspace,
+                           workspace_bytes, dev_status, stream, ar, to_dtype);
+}
+
+int bt_relu6_fwd_compress_arena(const void *pre_act, uint64_t n, int dtype, void *y_out, uint32_t *bitmap, void *arena,
+                                uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offset_out,
+                                uint64_t *chunk_prefix, uint64_t *nnz_out, void *workspace, size_t workspace_bytes,
+                                int32_t *dev_status, void *stream)
+{
+    if (!arena_cursor) return BT_ERR_NULL;
+    Arena ar;
+    ar.cursor = arena_cursor, ar.offset_out = values_offset_out, ar.bytes = arena_bytes;
+    return compress_common(pre_act, n, dtype, 2, 0.0f, y_out, bitmap, arena, arena_bytes, chunk_prefix, nnz_out,
+                           workspace, workspace_bytes, dev_status, stream, ar);
+}
+
+int bt_decompress_widen_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
+                              const uint64_t *chunk_prefix, uint64_t n, int from_dtype, void *dense_out, void *stream)
+{
+    if (from_dtype != BT_F16 && from_dtype != BT_BF16) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !chunk_prefix || !dense_out || !arena || !values_offset) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
+        !aligned(dense_out, 16))
+        return BT_ERR_ALIGN;
+    return bt::launch_decompress_widen(bitmap, arena, values_offset, chunk_prefix, n, from_dtype, dense_out,
+                                       static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
+int bt_relu6_bwd_from_stash_arena(const uint32_t *bitmap, const void *arena, const uint64_t *values_offset,
+                                  const uint64_t *chunk_prefix, const void *grad_out, uint64_t n, int dtype,
+                                  void *grad_in, void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (n == 0) return BT_OK;
+    if (!bitmap || !chunk_prefix || !grad_out || !grad_in || !arena || !values_offset) return BT_ERR_NULL;
+    if (!aligned(bitmap, 16) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
+        !aligned(grad_out, 16) || !aligned(grad_in, 16))
+        return BT_ERR_ALIGN;
+    return bt::launch_relu6_bwd(bitmap, arena, values_offset, chunk_prefix, grad_out, n, dtype, grad_in,
+                                static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? BT_OK
+               : BT_ERR_CUDA;
+}
+
 int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *chunk_prefix, uint64_t n, int dtype,
                   void *dense_out, void *stream)
 {
@@ -218,7 +288,7 @@ int bt_decompress_widen(const uint32_t *bitmap, const void *values, const uint64
     if (!bitmap || !chunk_prefix || !dense_out) return BT_ERR_NULL;
     if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
         return BT_ERR_ALIGN;
-    return bt::launch_decompress_widen(bitmap, values, chunk_prefix, n, from_dtype, dense_out,
+    return bt::launch_decompress_widen(bitmap, values, nullptr, chunk_prefix, n, from_dtype, dense_out,
                                        static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? BT_OK
                : BT_ERR_CUDA;

@@ -831,7 +831,7 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStr
     const bool y = a.y != nullptr;
     if (a.cast != 0) {
         // down-cast on stash: binary32 tensors, plain and threshold forms
-        if (dtype != BT_F32 || fused == 2 || a.arena_cursor) return cudaErrorInvalidValue;
+        if (dtype != BT_F32 || fused == 2) return cudaErrorInvalidValue;
         const bool h = a.cast == BT_F16;
         if (fused == 0) return h ? launch_typed<uint32_t, -1, false, 1>(a, stream) : launch_typed<uint32_t, -1, false, 2>(a, stream);
         if (y) return h ? launch_typed<uint32_t, BT_F32, true, 1>(a, stream) : launch_typed<uint32_t, BT_F32, true, 2>(a, stream);

@@ -167,8 +167,8 @@ cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint6
 
 }  // namespace
 
-cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *prefix, uint64_t n,
-                                    int from_dtype, void *out_f32, cudaStream_t stream)
+cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *values_offset,
+                                    const uint64_t *prefix, uint64_t n, int from_dtype, void *out_f32, cudaStream_t stream)
 {
     constexpr int  kWarps   = 4;
     const uint64_t quarters = (n + 1023) >> 10;
@@ -177,9 +177,9 @@ cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16
     const auto *v = static_cast<const uint16_t *>(values16);
     auto       *o = static_cast<uint32_t *>(out_f32);
     if (from_dtype == BT_F16)
-        decompress_kernel<uint32_t, 4, 8, kWarps, 1><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, nullptr, prefix, n, o);
+        decompress_kernel<uint32_t, 4, 8, kWarps, 1><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, values_offset, prefix, n, o);
     else
-        decompress_kernel<uint32_t, 4, 8, kWarps, 2><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, nullptr, prefix, n, o);
+        decompress_kernel<uint32_t, 4, 8, kWarps, 2><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, values_offset, prefix, n, o);
     return cudaGetLastError();
 }
 

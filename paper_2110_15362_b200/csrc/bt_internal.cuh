@@ -56,12 +56,12 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStr
 // values_offset: NULL, or a device word holding the byte offset of the packed values inside `values`
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                               const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t s);
-cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *prefix, uint64_t n,
-                                    int from_dtype, void *out_f32, cudaStream_t s);
+cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *values_offset,
+                                    const uint64_t *prefix, uint64_t n, int from_dtype, void *out_f32, cudaStream_t s);
 cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,
                                int elem_size, void *y, void *values, uint64_t capacity, cudaStream_t s);
-cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
-                             uint64_t n, int dtype, void *gin, cudaStream_t s);
+cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
+                             const uint64_t *prefix, const void *gout, uint64_t n, int dtype, void *gin, cudaStream_t s);
 cudaError_t launch_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width, int dtype, void *y,
                                   uint32_t *codes, cudaStream_t s);
 cudaError_t launch_maxpool2x2_bwd(const uint32_t *codes, const void *gout, uint64_t planes, uint64_t height, uint64_t width,

@@ -21,9 +21,12 @@ constexpr uint32_t kFull = 0xFFFFFFFFu;
 
 template <typename U, int DT, int kE, int kBlk, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
-relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values, const uint64_t *__restrict__ prefix,
-                 const U *gout, const uint64_t n, U *gin)   // gin may alias gout
+relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ values,
+                 const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const U *gout,
+                 const uint64_t n, U *gin)   // gin may alias gout
 {
+    // arena form: the packed values start *values_offset bytes into `values`
+    if (values_offset) values = reinterpret_cast<const U *>(reinterpret_cast<const unsigned char *>(values) + *values_offset);
     constexpr int kVec          = 16 / sizeof(U);
     constexpr int kLanesPerWord = 32 / kE;
     constexpr int kWordsPerStep = kE;
@@ -152,28 +155,29 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
 }
 
 template <typename U, int DT, int kE, int kBlk>
-cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
-                         uint64_t n, void *gin, cudaStream_t stream)
+cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *values_offset, const uint64_t *prefix,
+                         const void *gout, uint64_t n, void *gin, cudaStream_t stream)
 {
     constexpr int  kWarps   = 4;   // four warps per CTA: 1 to 4 % faster than eight
     const uint64_t quarters = (n + 1023) >> 10;
     const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     relu6_bwd_kernel<U, DT, kE, kBlk, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
-        bitmap, static_cast<const U *>(values), prefix, static_cast<const U *>(gout), n, static_cast<U *>(gin));
+        bitmap, static_cast<const U *>(values), values_offset, prefix, static_cast<const U *>(gout), n, static_cast<U *>(gin));
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *prefix, const void *gout,
-                             uint64_t n, int dtype, void *gin, cudaStream_t stream)
+cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
+                             const uint64_t *prefix, const void *gout, uint64_t n, int dtype, void *gin,
+                             cudaStream_t stream)
 {
     switch (dtype) {
-    case BT_F64: return launch_typed<uint64_t, BT_F64, 2, 2>(bitmap, values, prefix, gout, n, gin, stream);
-    case BT_F32: return launch_typed<uint32_t, BT_F32, 4, 2>(bitmap, values, prefix, gout, n, gin, stream);
-    case BT_F16: return launch_typed<uint16_t, BT_F16, 8, 4>(bitmap, values, prefix, gout, n, gin, stream);
-    default: return launch_typed<uint16_t, BT_BF16, 8, 4>(bitmap, values, prefix, gout, n, gin, stream);
+    case BT_F64: return launch_typed<uint64_t, BT_F64, 2, 2>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
+    case BT_F32: return launch_typed<uint32_t, BT_F32, 4, 2>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
+    case BT_F16: return launch_typed<uint16_t, BT_F16, 8, 4>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
+    default: return launch_typed<uint16_t, BT_BF16, 8, 4>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
     }
 }
 

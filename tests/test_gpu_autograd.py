@@ -182,7 +182,8 @@ def test_relu6_stash_gradients_are_bit_identical(A, dtype):
         assert hooks.packed_bytes < 0.7 * hooks.dense_bytes
     loss2, g2 = run(weights, x, A.relu6_stash)                      # without the hooks
     with A.stash_saved_activations(min_numel=1024, arena_bytes=64 << 20) as hooks:
-        loss3, g3 = run(weights, x, lambda t: A.relu6_stash(t, hooks))      # inside an arena context: exact-size stashes
+        loss3, g3 = run(weights, x, lambda t: A.relu6_stash(t, hooks))      # inside an arena context: values in the arena
+        assert 0 < int(hooks.cursor.item()) < 0.7 * hooks.dense_bytes and hooks.packed_bytes == 0
     for loss, grads in ((loss1, g1), (loss2, g2), (loss3, g3)):
         assert torch.equal(loss, ref_loss)
         for a, b in zip(grads, ref):
@@ -220,8 +221,15 @@ def test_narrowed_stash_is_the_rounded_activation(A, narrow):
         assert torch.equal(a, b)                                    # same rounded activations into the same GEMMs
     _, exact = run(weights, x, torch.relu)
     assert not torch.equal(g1[-1], exact[-1]) and torch.allclose(g1[-1], exact[-1], rtol=0.05, atol=0.5)
-    with pytest.raises(ValueError):
-        A.stash_saved_activations(narrow=narrow, arena_bytes=1 << 20)
+    # the same inside an arena: 16-bit values behind the cursor, no host read in the forward pass
+    with A.stash_saved_activations(min_numel=1024, narrow=narrow, arena_bytes=32 << 20) as hooks:
+        loss2, g2 = run(weights, x, lambda t: A.relu_stash(t, hooks))
+        assert 0 < int(hooks.cursor.item()) < 0.4 * hooks.dense_bytes
+    with A.stash_saved_activations(min_numel=1024, narrow=narrow, arena_bytes=32 << 20) as hooks:
+        loss3, g3 = run(weights, x, relu_by_mask)                   # the hooks alone (plain narrowing compressor)
+    assert torch.equal(loss2, ref_loss) and torch.equal(loss3, ref_loss)
+    for a, b, c in zip(g2, g3, ref):
+        assert torch.equal(a, c) and torch.equal(b, c)
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
