@@ -3,10 +3,11 @@
     python -m paper_2110_15362_b200.demo_vgg_step [--batch 32] [--size 224] [--dtype f32|bf16] [--arena-gib 8]
 
 Builds the thirteen 3x3 convolutions and five 2x2 max-pools of VGG-16 (no batch normalisation, a small
-linear head), runs forward + backward three ways -- plain PyTorch (in-place ReLU), saved activations
+linear head), runs forward + backward several ways -- plain PyTorch (in-place ReLU), saved activations
 stashed (exact-size values, one host read per tensor), the same with the pooling layers keeping 2-bit winner
-codes instead of their input and an index tensor, and that with the values in an arena (no host read) -- and prints one JSON line with the bytes kept for the saved ReLU outputs relative to their dense
-size, the device memory held between the forward and the backward pass, the peak above the model's own tensors
+codes instead of their input and an index tensor, that with the values in an arena (no host read), and (fp32
+only) the arena with the values down-cast to bfloat16 on stash, which is lossy in the gradients -- and prints one
+JSON line with the bytes kept for the saved ReLU outputs relative to their dense size, the device memory held between the forward and the backward pass, the peak above the model's own tensors
 and the step time of each.  The peak also
 holds what no stash touches: the transients of the widest layer (its pre-activation, its gradients, the
 restored activation) and the max-pool indices, so it drops by less than the saved activations do.  The paper
@@ -146,6 +147,18 @@ def main(argv=None) -> int:
     out["stashed_arena"]["arena_used_mib"] = round(int(arena_hooks.cursor.item()) / 2 ** 20, 1)
     out["stashed_arena"]["peak_mib_with_arena_used"] = round(out["stashed_arena"]["peak_mib"] +
                                                             out["stashed_arena"]["arena_used_mib"], 1)
+    if dtype == torch.float32:
+        del arena_hooks
+        torch.cuda.empty_cache()
+        narrow_hooks = A.stash_saved_activations(arena_bytes=int(args.arena_gib * 2 ** 30), narrow=torch.bfloat16)
+
+        def arena_narrow():
+            with narrow_hooks:
+                return step(x, ws, head, lambda t: A.relu_stash(t, narrow_hooks, inplace=True), A.maxpool2x2_stash,
+                            lambda t: A.relu_stash(t, narrow_hooks, inplace=True, keep_values=False))
+
+        out["stashed_arena_bf16_values"] = measure(arena_narrow)
+        out["stashed_arena_bf16_values"]["arena_used_mib"] = round(int(narrow_hooks.cursor.item()) / 2 ** 20, 1)
     print(json.dumps(out))
     return 0
 

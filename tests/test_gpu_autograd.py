@@ -164,6 +164,8 @@ def test_vgg_demo_runs_and_losses_agree(A, capsys):
     assert out["plain"]["loss"] == pytest.approx(out["stashed"]["loss"], rel=1e-3)
     assert out["plain"]["loss"] == pytest.approx(out["stashed_arena"]["loss"], rel=1e-3)
     assert out["plain"]["loss"] == pytest.approx(out["stashed_pool_codes"]["loss"], rel=1e-3)
+    assert out["plain"]["loss"] == pytest.approx(out["stashed_arena_bf16_values"]["loss"], rel=1e-3)   # forward not narrowed
+    assert out["stashed_arena_bf16_values"]["arena_used_mib"] < 0.6 * out["stashed_arena"]["arena_used_mib"]
     assert 0.3 < out["saved_activation_bytes_over_dense"] < 0.8
     # what the graph holds between the two passes shrinks, most with the pooling layers on winner codes
     assert out["stashed_pool_codes"]["held_after_forward_mib"] < out["stashed"]["held_after_forward_mib"] \
