@@ -27,7 +27,9 @@ bitmap.
 
 ``maxpool2x2_stash(x)`` is a 2x2 / stride 2 max pooling that keeps 2 bits per output for its backward pass
 (``bt_maxpool2x2_fwd`` / ``bt_maxpool2x2_bwd``) instead of its input and an index tensor: behind a ``relu_stash``
-the values of the pooled layer's input are then held by nothing, only its bitmap.
+the values of the pooled layer's input are then held by nothing, only its bitmap.  ``relu_maxpool2x2_stash(x)``
+does both layers with the pooling first (the maximum commutes with the ReLU): the full-size activation is never
+written and the fused ReLU + stash runs on the pooled quarter.
 
 ``relu6_stash(x)`` is the same for ReLU6 (``bt_relu6_fwd_compress`` / ``bt_relu6_bwd_from_stash``; its backward
 pass reads the stashed values as well, which are the ones the next layer's saved input shares).  With
@@ -46,7 +48,8 @@ import torch
 from . import binding as B
 
 __all__ = ["PackedActivation", "stash_saved_activations", "relu_stash", "ReLUStash", "relu6_stash", "ReLU6Stash",
-           "double_mask", "DoubleMask", "maxpool2x2_stash", "MaxPool2x2Stash"]
+           "double_mask", "DoubleMask", "maxpool2x2_stash", "MaxPool2x2Stash", "relu_maxpool2x2_stash",
+           "ReLUMaxPool2x2Stash"]
 
 
 class PackedActivation:
@@ -502,3 +505,54 @@ class MaxPool2x2Stash(torch.autograd.Function):
 def maxpool2x2_stash(x: torch.Tensor) -> torch.Tensor:
     """``torch.nn.functional.max_pool2d(x, 2)`` with a 2-bit-per-output backward record (see ``MaxPool2x2Stash``)."""
     return MaxPool2x2Stash.apply(x)
+
+
+class ReLUMaxPool2x2Stash(torch.autograd.Function):
+    """``max_pool2d(relu(x), 2)`` computed as ``relu(max_pool2d(x, 2))``: the maximum commutes with the ReLU, so the
+    pooling runs first, on the pre-activation, and the fused ReLU + stash runs on a quarter of the elements.  The
+    full-size activation is never written.  Kept for the backward pass: 2 bits per pooled output and the pooled
+    activation's bitmap; the pooled activation's stash is shared with the next layer's save.  Output and input
+    gradient are those of the two-step form: a window with a positive maximum has the same winner either way, and
+    a window without one has a zero output and an all-zero gradient whichever position its code names."""
+
+    @staticmethod
+    def forward(ctx, x: torch.Tensor, hooks: Optional[stash_saved_activations] = None):
+        if x.dim() < 2 or x.shape[-1] % 2 or x.shape[-2] % 2 or x.numel() == 0:
+            raise ValueError("relu_maxpool2x2_stash: the last two dimensions must be even and non-empty")
+        xc = _flat_input(x)
+        y = torch.empty(xc.shape[:-2] + (xc.shape[-2] // 2, xc.shape[-1] // 2), dtype=x.dtype, device=x.device)
+        codes = torch.empty((y.numel() + 15) // 16, dtype=torch.int32, device=x.device)
+        B.bt_maxpool2x2_fwd(xc, y, codes)
+        flat = y.view(-1)
+        if hooks is not None and hooks.arena is not None:
+            bitmap, prefix, nnz_word, off_word, stored = _compress_arena(flat, hooks, relu_into=flat)
+            hooks.share(y, PackedActivation(bitmap, None, prefix, tuple(y.shape), y.dtype, y.device, nnz_word,
+                                            arena=hooks.arena, offset=off_word, owner=hooks, stored=stored))
+            hooks.dense_bytes += y.numel() * y.element_size()
+        else:
+            scratch = hooks.scratch if hooks is not None else _Scratch()
+            bitmap, values, prefix, nnz = _compress(flat, scratch, relu_into=flat,
+                                                    narrow=hooks.narrow if hooks is not None else None)
+            if hooks is not None:
+                packed = PackedActivation(bitmap, values, prefix, tuple(y.shape), y.dtype, y.device, nnz)
+                hooks.share(y, packed)
+                hooks.packed_bytes += packed.nbytes()
+                hooks.dense_bytes += y.numel() * y.element_size()
+        ctx.save_for_backward(codes, bitmap)
+        ctx.in_shape = tuple(xc.shape)
+        return y
+
+    @staticmethod
+    def backward(ctx, grad: torch.Tensor):
+        codes, bitmap = ctx.saved_tensors
+        g = _flat_input(grad)
+        gp = torch.empty_like(g)
+        B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gp.view(-1))
+        gin = torch.empty(ctx.in_shape, dtype=g.dtype, device=g.device)
+        B.bt_maxpool2x2_bwd(codes, gp, gin)
+        return gin, None
+
+
+def relu_maxpool2x2_stash(x: torch.Tensor, hooks: Optional[stash_saved_activations] = None) -> torch.Tensor:
+    """``max_pool2d(relu(x), 2)`` with the pooling moved in front of the ReLU (see ``ReLUMaxPool2x2Stash``)."""
+    return ReLUMaxPool2x2Stash.apply(x, hooks)

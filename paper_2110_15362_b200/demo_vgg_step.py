@@ -5,8 +5,9 @@
 Builds the thirteen 3x3 convolutions and five 2x2 max-pools of VGG-16 (no batch normalisation, a small
 linear head), runs forward + backward several ways -- plain PyTorch (in-place ReLU), saved activations
 stashed (exact-size values, one host read per tensor), the same with the pooling layers keeping 2-bit winner
-codes instead of their input and an index tensor, that with the values in an arena (no host read), and (fp32
-only) the arena with the values down-cast to bfloat16 on stash, which is lossy in the gradients -- and prints one
+codes instead of their input and an index tensor, that with the values in an arena (no host read), the arena with
+each ReLU + pooling pair done pooling first (the full-size activation in front of a pooling layer is never
+written), and (fp32 only) the arena with the values down-cast to bfloat16 on stash, which is lossy in the gradients -- and prints one
 JSON line with the bytes kept for the saved ReLU outputs relative to their dense size, the device memory held between the forward and the backward pass, the peak above the model's own tensors
 and the step time of each.  The peak also
 holds what no stash touches: the transients of the widest layer (its pre-activation, its gradients, the
@@ -44,15 +45,20 @@ def make_weights(dtype, device, seed=0):
     return ws, head
 
 
-def step(x, ws, head, relu, pool=lambda t: F.max_pool2d(t, 2), relu_before_pool=None):
-    """`relu_before_pool`: the activation used where a pooling layer follows (default: `relu`)."""
+def step(x, ws, head, relu, pool=lambda t: F.max_pool2d(t, 2), relu_before_pool=None, relu_pool=None):
+    """`relu_before_pool`: the activation used where a pooling layer follows (default: `relu`).  `relu_pool`: one
+    call that does the activation and the pooling layer behind it (replaces both there)."""
     h, k = x, 0
     for i, c in enumerate(CFG):
         if c == "M":
-            h = pool(h)
+            if relu_pool is None:
+                h = pool(h)
         else:
-            act = relu_before_pool if relu_before_pool is not None and CFG[i + 1] == "M" else relu
-            h = act(F.conv2d(h, ws[k], padding=1))
+            h = F.conv2d(h, ws[k], padding=1)
+            if CFG[i + 1] == "M" and relu_pool is not None:
+                h = relu_pool(h)
+            else:
+                h = (relu_before_pool if relu_before_pool is not None and CFG[i + 1] == "M" else relu)(h)
             k += 1
     logits = F.linear(h.mean(dim=(2, 3)), head)
     loss = logits.float().square().mean()
@@ -147,8 +153,19 @@ def main(argv=None) -> int:
     out["stashed_arena"]["arena_used_mib"] = round(int(arena_hooks.cursor.item()) / 2 ** 20, 1)
     out["stashed_arena"]["peak_mib_with_arena_used"] = round(out["stashed_arena"]["peak_mib"] +
                                                             out["stashed_arena"]["arena_used_mib"], 1)
+    del arena_hooks
+    torch.cuda.empty_cache()
+    first_hooks = A.stash_saved_activations(arena_bytes=int(args.arena_gib * 2 ** 30))
+
+    def arena_pool_first():
+        with first_hooks:
+            return step(x, ws, head, lambda t: A.relu_stash(t, first_hooks, inplace=True),
+                        relu_pool=lambda t: A.relu_maxpool2x2_stash(t, first_hooks))
+
+    out["stashed_arena_pool_first"] = measure(arena_pool_first)
+    out["stashed_arena_pool_first"]["arena_used_mib"] = round(int(first_hooks.cursor.item()) / 2 ** 20, 1)
     if dtype == torch.float32:
-        del arena_hooks
+        del first_hooks
         torch.cuda.empty_cache()
         narrow_hooks = A.stash_saved_activations(arena_bytes=int(args.arena_gib * 2 ** 30), narrow=torch.bfloat16)
 

@@ -164,6 +164,8 @@ def test_vgg_demo_runs_and_losses_agree(A, capsys):
     assert out["plain"]["loss"] == pytest.approx(out["stashed"]["loss"], rel=1e-3)
     assert out["plain"]["loss"] == pytest.approx(out["stashed_arena"]["loss"], rel=1e-3)
     assert out["plain"]["loss"] == pytest.approx(out["stashed_pool_codes"]["loss"], rel=1e-3)
+    assert out["plain"]["loss"] == pytest.approx(out["stashed_arena_pool_first"]["loss"], rel=1e-3)
+    assert out["stashed_arena_pool_first"]["held_after_forward_mib"] <= out["stashed_arena"]["held_after_forward_mib"]
     assert out["plain"]["loss"] == pytest.approx(out["stashed_arena_bf16_values"]["loss"], rel=1e-3)   # forward not narrowed
     assert out["stashed_arena_bf16_values"]["arena_used_mib"] < 0.6 * out["stashed_arena"]["arena_used_mib"]
     assert 0.3 < out["saved_activation_bytes_over_dense"] < 0.8
@@ -323,7 +325,15 @@ def test_maxpool_stash_matches_torch(A, dtype):
         used = int(hooks.cursor.item())
     got5 = run_net(lambda t: A.relu_stash(t, keep_values=False), A.maxpool2x2_stash)
     assert used < 32 << 20
-    for g in (got, got2, got3, got4, got5):
+    # the two layers as one call, pooling first (the maximum commutes with the ReLU)
+    got6 = run_net(lambda t: t, A.relu_maxpool2x2_stash)
+    with A.stash_saved_activations(min_numel=1024) as hooks:
+        got7 = run_net(lambda t: t, lambda t: A.relu_maxpool2x2_stash(t, hooks))
+        assert hooks.packed_bytes > 0
+    with A.stash_saved_activations(min_numel=1024, arena_bytes=32 << 20) as hooks:
+        got8 = run_net(lambda t: t, lambda t: A.relu_maxpool2x2_stash(t, hooks))
+        assert 0 < int(hooks.cursor.item()) < 32 << 20
+    for g in (got, got2, got3, got4, got5, got6, got7, got8):
         for a, b in zip(g, ref):
             assert torch.equal(a, b)
     with pytest.raises(ValueError):
@@ -331,3 +341,37 @@ def test_maxpool_stash_matches_torch(A, dtype):
     # a non-contiguous input is taken through a copy
     xt = torch.randn(4, 6, 8, 10, device="cuda").transpose(0, 1)
     assert torch.equal(A.maxpool2x2_stash(xt), torch.nn.functional.max_pool2d(xt, 2))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16, torch.float64])
+def test_relu_and_pooling_commuted_is_bit_identical(A, dtype):
+    """relu_maxpool2x2_stash against max_pool2d(relu(x), 2) on inputs full of ties, windows without a positive
+    element, exact zeros and NaNs: output and input gradient agree bit for bit (no -0 among the inputs: the
+    framework's ReLU keeps that sign, the library's gives +0)."""
+    g = torch.Generator(device="cuda").manual_seed(31)
+    x = (torch.randint(-3, 4, (6, 5, 30, 44), device="cuda", generator=g).to(torch.float64) / 2).to(dtype)   # many ties
+    x[0, 0, :6] = -1.0                                                   # whole windows without a positive element
+    x[1, 1, 2:8, 4:12] = 0.0
+    pick = torch.rand(x.shape, device="cuda", generator=g) < 0.01
+    x[pick] = float("nan")
+    x[2, 2, 4, 4] = x[2, 2, 4, 5] = x[2, 2, 5, 4] = float("nan")          # several NaNs in one window
+    grad = torch.randn(6, 5, 15, 22, device="cuda", generator=g).to(dtype)
+    iv = {torch.float32: torch.int32, torch.bfloat16: torch.int16, torch.float64: torch.int64}[dtype]
+    xr = x.clone().requires_grad_()
+    ref = torch.nn.functional.max_pool2d(torch.relu(xr), 2)
+    ref.backward(grad)
+    for hooks in (None, A.stash_saved_activations(min_numel=64), A.stash_saved_activations(min_numel=64, arena_bytes=1 << 20)):
+        xs = x.clone().requires_grad_()
+        if hooks is None:
+            y = A.relu_maxpool2x2_stash(xs)
+            y.backward(grad)
+        else:
+            with hooks:
+                y = A.relu_maxpool2x2_stash(xs, hooks)
+                packed = hooks._lookup(y)
+                assert packed is not None and torch.equal(packed.unpack().view(iv), y.detach().view(iv))
+                y.backward(grad)
+        assert torch.equal(y.detach().view(iv), ref.detach().view(iv))
+        assert torch.equal(xs.grad.view(iv), xr.grad.view(iv))
+    with pytest.raises(ValueError):
+        A.relu_maxpool2x2_stash(torch.zeros(2, 3, 5, 4, device="cuda"))
