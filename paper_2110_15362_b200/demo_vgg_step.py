@@ -19,6 +19,7 @@ reports for ReLU layers, so the activation-memory ratio is comparable while accu
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import sys
 
@@ -73,7 +74,8 @@ def step(x, ws, head, relu, pool=lambda t: F.max_pool2d(t, 2), relu_before_pool=
 def measure(fn, reps=3):
     fn()                                                      # warm-up (cuDNN algorithm choice, allocator)
     torch.cuda.synchronize()
-    torch.cuda.empty_cache()
+    gc.collect()                                              # tensors kept alive only by reference cycles (a caller's
+    torch.cuda.empty_cache()                                  # earlier work) must not be freed in mid-measurement
     best, peak, loss = None, 0, None
     for _ in range(reps):
         torch.cuda.reset_peak_memory_stats()
