@@ -85,6 +85,49 @@ def test_argument_errors_are_reported_before_any_launch(L):
     assert L.bt_relu_fwd_compress(A, 8192, B.BT_F32, A + 4, A, A, 8192, A, A, A, ws, A, None) == B.BT_ERR_ALIGN
 
 
+def test_later_entry_points_check_their_arguments_before_any_launch(L):
+    """The calls added after the hot path (narrowing, widening, ReLU6, pooling, masked gather, arena forms): every
+    call below fails its host-side checks, so the fake addresses are never dereferenced."""
+    A = 0x10000
+    ws = L.bt_workspace_bytes(8192)
+    tail = (A, A, A, ws, A, None)                                   # chunk_prefix, nnz_out, workspace, bytes, status, stream
+    arena = (A, 1 << 20, A, A)                                      # arena, arena_bytes, cursor, values_offset_out
+    assert L.bt_compress_narrow(A, 8192, B.BT_F32, A, A, 8192, *tail) == B.BT_ERR_DTYPE
+    assert L.bt_compress_narrow(None, 8192, B.BT_F16, A, A, 8192, *tail) == B.BT_ERR_NULL
+    assert L.bt_prune_fwd_compress_narrow(A, 8192, B.BT_F64, 0.0, None, A, A, 8192, *tail) == B.BT_ERR_DTYPE
+    assert L.bt_prune_fwd_compress_narrow(A + 4, 8192, B.BT_BF16, 0.0, None, A, A, 8192, *tail) == B.BT_ERR_ALIGN
+    assert L.bt_decompress_widen(A, A, A, 10, B.BT_F32, A, None) == B.BT_ERR_DTYPE
+    assert L.bt_decompress_widen(A, A, None, 10, B.BT_F16, A, None) == B.BT_ERR_NULL
+    assert L.bt_decompress_widen(None, None, None, 0, B.BT_F16, None, None) == B.BT_OK
+    assert L.bt_relu6_fwd_compress(A, 8192, 11, None, A, A, 8192, *tail) == B.BT_ERR_DTYPE
+    assert L.bt_relu6_fwd_compress(A, 8192, B.BT_F32, None, None, A, 8192, *tail) == B.BT_ERR_NULL
+    assert L.bt_relu6_bwd_from_stash(A, A, A, None, 10, B.BT_F32, A, None) == B.BT_ERR_NULL
+    assert L.bt_relu6_bwd_from_stash(A, A, A, A, 10, B.BT_F32, A + 8, None) == B.BT_ERR_ALIGN
+    assert L.bt_mask_compress(None, 10, B.BT_F32, A, A, None, A, 10, None) == B.BT_ERR_NULL
+    assert L.bt_mask_compress(A, 10, 9, A, A, None, A, 10, None) == B.BT_ERR_DTYPE
+    assert L.bt_maxpool2x2_fwd(A, 4, 3, 8, B.BT_F32, A, A, None) == B.BT_ERR_SHAPE
+    assert L.bt_maxpool2x2_fwd(A, 4, 8, 0, B.BT_F32, A, A, None) == B.BT_ERR_SHAPE
+    assert L.bt_maxpool2x2_fwd(None, 4, 8, 8, B.BT_F32, A, A, None) == B.BT_ERR_NULL
+    assert L.bt_maxpool2x2_fwd(None, 0, 8, 8, B.BT_F32, None, None, None) == B.BT_OK
+    assert L.bt_maxpool2x2_bwd(A, A, 4, 8, 8, 13, A, None) == B.BT_ERR_DTYPE
+    # arena forms
+    assert L.bt_compress_arena(A, 8192, B.BT_F32, A, A, 1 << 20, None, A, *tail) == B.BT_ERR_NULL      # no cursor
+    assert L.bt_compress_arena(A, 8192, B.BT_F32, A, A, 1 << 20, A, None, *tail) == B.BT_ERR_NULL      # no offset word
+    assert L.bt_compress_arena(A, 8192, B.BT_F32, A, A, 1 << 20, A + 4, A, *tail) == B.BT_ERR_ALIGN
+    assert L.bt_prune_fwd_compress_arena(A, 8192, 9, 0.0, None, A, *arena, *tail) == B.BT_ERR_DTYPE
+    assert L.bt_decompress_arena(A, A, None, A, 10, B.BT_F32, A, None) == B.BT_ERR_NULL
+    assert L.bt_compress_narrow_arena(A, 8192, B.BT_F32, A, *arena, *tail) == B.BT_ERR_DTYPE
+    assert L.bt_compress_narrow_arena(A, 8192, B.BT_F16, A, A, 1 << 20, None, A, *tail) == B.BT_ERR_NULL
+    assert L.bt_prune_fwd_compress_narrow_arena(A, 8192, B.BT_F64, 0.0, None, A, *arena, *tail) == B.BT_ERR_DTYPE
+    assert L.bt_prune_fwd_compress_narrow_arena(A, 8192, B.BT_BF16, 0.0, A + 2, A, *arena, *tail) == B.BT_ERR_ALIGN
+    assert L.bt_relu6_fwd_compress_arena(A, 8192, B.BT_F32, None, A, A, 1 << 20, A, None, *tail) == B.BT_ERR_NULL
+    assert L.bt_decompress_widen_arena(A, A, A, A, 10, B.BT_F64, A, None) == B.BT_ERR_DTYPE
+    assert L.bt_decompress_widen_arena(A, A, None, A, 10, B.BT_F16, A, None) == B.BT_ERR_NULL
+    assert L.bt_relu6_bwd_from_stash_arena(A, A, None, A, A, 10, B.BT_F32, A, None) == B.BT_ERR_NULL
+    assert L.bt_relu6_bwd_from_stash_arena(A, A, A + 4, A, A, 10, B.BT_F32, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_relu6_bwd_from_stash_arena(None, None, None, None, None, 0, B.BT_F32, None, None) == B.BT_OK
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "library_path", lambda: str(tmp_path / "nope.so"))
