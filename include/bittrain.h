@@ -206,6 +206,18 @@ int bt_maxpool2x2_bwd(const uint32_t *codes, const void *grad_out, uint64_t plan
                       uint64_t width, int dtype, void *grad_in, void *stream);
 
 /*
+ * Backward pass of ReLU followed by this pooling, for a forward pass that pooled first (the maximum
+ * commutes with the ReLU: pool the pre-activation with bt_maxpool2x2_fwd, then run bt_relu_fwd_compress
+ * on the pooled quarter).  pooled_bitmap is the bitmap of the pooled activation's stash (bit o set: output
+ * o is non-zero after the ReLU).  grad_in gets grad_out[o] at the coded position of window o if bit o is
+ * set, and +0 everywhere else: bt_relu_bwd_from_bitmap and bt_maxpool2x2_bwd in one pass.  Other
+ * parameters as bt_maxpool2x2_bwd; pooled_bitmap 4-byte aligned, ceil(outputs / 32) words.
+ */
+int bt_maxpool2x2_bwd_masked(const uint32_t *codes, const uint32_t *pooled_bitmap, const void *grad_out,
+                             uint64_t planes, uint64_t height, uint64_t width, int dtype, void *grad_in,
+                             void *stream);
+
+/*
  * Algorithm 2 on a narrowed stash, straight into a BT_F32 tensor: dense_out[i]
  * = the stashed 16-bit value of element i (from_dtype: BT_F16 or BT_BF16)
  * widened to binary32 -- exact for both types, a NaN keeps its sign and its

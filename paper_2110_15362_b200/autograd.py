@@ -546,10 +546,8 @@ class ReLUMaxPool2x2Stash(torch.autograd.Function):
     def backward(ctx, grad: torch.Tensor):
         codes, bitmap = ctx.saved_tensors
         g = _flat_input(grad)
-        gp = torch.empty_like(g)
-        B.bt_relu_bwd_from_bitmap(bitmap, g.view(-1), gp.view(-1))
         gin = torch.empty(ctx.in_shape, dtype=g.dtype, device=g.device)
-        B.bt_maxpool2x2_bwd(codes, gp, gin)
+        B.bt_maxpool2x2_bwd_masked(codes, bitmap, g, gin)      # the ReLU's select and the pooling's scatter in one pass
         return gin, None
 
 

@@ -31,7 +31,7 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
            "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd",
            "bt_compress_narrow_arena", "bt_prune_fwd_compress_narrow_arena", "bt_decompress_widen_arena",
-           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena")
+           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.bt_maxpool2x2_fwd.restype = i32
         L.bt_maxpool2x2_bwd.argtypes = [vp, vp, u64, u64, u64, i32, vp, vp]
         L.bt_maxpool2x2_bwd.restype = i32
+        L.bt_maxpool2x2_bwd_masked.argtypes = [vp, vp, vp, u64, u64, u64, i32, vp, vp]
+        L.bt_maxpool2x2_bwd_masked.restype = i32
         L.bt_compress_narrow_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
         L.bt_compress_narrow_arena.restype = i32
         L.bt_prune_fwd_compress_narrow_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz,
@@ -257,6 +259,19 @@ def bt_maxpool2x2_bwd(codes: torch.Tensor, grad_out: torch.Tensor, grad_in: torc
     st = lib().bt_maxpool2x2_bwd(_ptr(codes), _ptr(grad_out), planes, height, width, DTYPE_CODE[grad_out.dtype],
                                  _ptr(grad_in), _stream(stream))
     return _check("bt_maxpool2x2_bwd", st, check)
+
+
+def bt_maxpool2x2_bwd_masked(codes: torch.Tensor, pooled_bitmap: torch.Tensor, grad_out: torch.Tensor, grad_in: torch.Tensor,
+                             *, planes: Optional[int] = None, height: Optional[int] = None, width: Optional[int] = None,
+                             stream=None, check: bool = True) -> int:
+    """Backward pass of ReLU + pooling done pooling first: the gradient of a pooled output whose bit in
+    `pooled_bitmap` is clear counts as zero."""
+    height = grad_in.shape[-2] if height is None else height
+    width = grad_in.shape[-1] if width is None else width
+    planes = grad_in.numel() // max(1, height * width) if planes is None else planes
+    st = lib().bt_maxpool2x2_bwd_masked(_ptr(codes), _ptr(pooled_bitmap), _ptr(grad_out), planes, height, width,
+                                        DTYPE_CODE[grad_out.dtype], _ptr(grad_in), _stream(stream))
+    return _check("bt_maxpool2x2_bwd_masked", st, check)
 
 
 def bt_mask_compress(x: torch.Tensor, mask_bitmap: torch.Tensor, mask_chunk_prefix: torch.Tensor,

@@ -326,20 +326,34 @@ int bt_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t 
                : BT_ERR_CUDA;
 }
 
-int bt_maxpool2x2_bwd(const uint32_t *codes, const void *grad_out, uint64_t planes, uint64_t height, uint64_t width, int dtype,
-                      void *grad_in, void *stream)
+namespace {
+int maxpool_bwd_common(const uint32_t *codes, const uint32_t *mask, bool masked, const void *grad_out, uint64_t planes,
+                       uint64_t height, uint64_t width, int dtype, void *grad_in, void *stream)
 {
     const int es = elem_size_of(dtype);
     if (es == 0) return BT_ERR_DTYPE;
     if (height == 0 || width == 0 || (height & 1) || (width & 1)) return BT_ERR_SHAPE;
     if (planes == 0) return BT_OK;
     if (planes > (1ull << 40) / height / width) return BT_ERR_TOO_LARGE;
-    if (!codes || !grad_out || !grad_in) return BT_ERR_NULL;
-    if (!aligned(codes, 4) || !aligned(grad_out, 16) || !aligned(grad_in, 16)) return BT_ERR_ALIGN;
-    return bt::launch_maxpool2x2_bwd(codes, grad_out, planes, height, width, es, grad_in, static_cast<cudaStream_t>(stream)) ==
-                   cudaSuccess
+    if (!codes || !grad_out || !grad_in || (masked && !mask)) return BT_ERR_NULL;
+    if (!aligned(codes, 4) || !aligned(mask, 4) || !aligned(grad_out, 16) || !aligned(grad_in, 16)) return BT_ERR_ALIGN;
+    return bt::launch_maxpool2x2_bwd(codes, mask, grad_out, planes, height, width, es, grad_in,
+                                     static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? BT_OK
                : BT_ERR_CUDA;
+}
+}  // namespace
+
+int bt_maxpool2x2_bwd(const uint32_t *codes, const void *grad_out, uint64_t planes, uint64_t height, uint64_t width, int dtype,
+                      void *grad_in, void *stream)
+{
+    return maxpool_bwd_common(codes, nullptr, false, grad_out, planes, height, width, dtype, grad_in, stream);
+}
+
+int bt_maxpool2x2_bwd_masked(const uint32_t *codes, const uint32_t *pooled_bitmap, const void *grad_out, uint64_t planes,
+                             uint64_t height, uint64_t width, int dtype, void *grad_in, void *stream)
+{
+    return maxpool_bwd_common(codes, pooled_bitmap, true, grad_out, planes, height, width, dtype, grad_in, stream);
 }
 
 int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out, uint64_t n, int dtype, void *grad_in,

@@ -64,8 +64,9 @@ cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const u
                              const uint64_t *prefix, const void *gout, uint64_t n, int dtype, void *gin, cudaStream_t s);
 cudaError_t launch_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width, int dtype, void *y,
                                   uint32_t *codes, cudaStream_t s);
-cudaError_t launch_maxpool2x2_bwd(const uint32_t *codes, const void *gout, uint64_t planes, uint64_t height, uint64_t width,
-                                  int elem_size, void *gin, cudaStream_t s);
+// mask: NULL, or a bitmap over the pooled outputs (the gradient of an output whose bit is clear counts as +0)
+cudaError_t launch_maxpool2x2_bwd(const uint32_t *codes, const uint32_t *mask, const void *gout, uint64_t planes,
+                                  uint64_t height, uint64_t width, int elem_size, void *gin, cudaStream_t s);
 cudaError_t launch_relu_bwd(const uint32_t *bitmap, const void *gout, uint64_t n, int elem_size,
                             void *gin, cudaStream_t s);
 

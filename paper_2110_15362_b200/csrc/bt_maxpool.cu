@@ -85,9 +85,10 @@ maxpool2x2_fwd_kernel(const U *__restrict__ x, const uint64_t outputs, const I w
 
 template <typename U, typename I>
 __global__ void __launch_bounds__(kThreads)
-maxpool2x2_bwd_kernel(const uint32_t *__restrict__ codes, const U *__restrict__ gout, const uint64_t outputs, const I wo,
-                      const I width, U *__restrict__ gin)
+maxpool2x2_bwd_kernel(const uint32_t *__restrict__ codes, const uint32_t *__restrict__ mask, const U *__restrict__ gout,
+                      const uint64_t outputs, const I wo, const I width, U *__restrict__ gin)
 {
+    // mask (may be NULL): bitmap over the outputs; the gradient of an output whose bit is clear counts as +0
     using P            = Pair<U>;
     const uint64_t o64 = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
     if (o64 >= outputs) return;
@@ -96,7 +97,8 @@ maxpool2x2_bwd_kernel(const uint32_t *__restrict__ codes, const U *__restrict__ 
     const I        col  = o - row * wo;
     const uint64_t at   = 2ull * row * width + 2ull * col;
     const uint32_t k    = (codes[o64 >> 4] >> (2u * (static_cast<uint32_t>(o64) & 15u))) & 3u;
-    const U        g    = gout[o64];
+    U              g    = gout[o64];
+    if (mask != nullptr && ((mask[o64 >> 5] >> (static_cast<uint32_t>(o64) & 31u)) & 1u) == 0) g = U(0);
     *reinterpret_cast<typename P::T *>(gin + at)         = P::make(k == 0 ? g : U(0), k == 1 ? g : U(0));
     *reinterpret_cast<typename P::T *>(gin + at + width) = P::make(k == 2 ? g : U(0), k == 3 ? g : U(0));
 }
@@ -173,8 +175,8 @@ maxpool2x2_fwd_vec_kernel(const U *__restrict__ x, const uint64_t groups, const 
 
 template <typename U, typename I>
 __global__ void __launch_bounds__(kThreads)
-maxpool2x2_bwd_vec_kernel(const uint32_t *__restrict__ codes, const U *__restrict__ gout, const uint64_t groups,
-                          const I groups_per_row, const I width, U *__restrict__ gin)
+maxpool2x2_bwd_vec_kernel(const uint32_t *__restrict__ codes, const uint32_t *__restrict__ mask, const U *__restrict__ gout,
+                          const uint64_t groups, const I groups_per_row, const I width, U *__restrict__ gin)
 {
     constexpr int  kOut = 8 / sizeof(U);
     const uint64_t g64  = static_cast<uint64_t>(blockIdx.x) * kThreads + threadIdx.x;
@@ -185,6 +187,8 @@ maxpool2x2_bwd_vec_kernel(const uint32_t *__restrict__ codes, const U *__restric
     const uint64_t at   = 2ull * row * width + 2ull * kOut * cg;
     const uint64_t o0   = g64 * kOut;
     const uint32_t bits = codes[o0 >> 4] >> (2u * (static_cast<uint32_t>(o0) & 15u));
+    // the kOut mask bits of this thread's outputs sit in one word (kOut divides 32)
+    const uint32_t live = mask != nullptr ? mask[o0 >> 5] >> (static_cast<uint32_t>(o0) & 31u) : 0xFFFFFFFFu;
     const uint2    gv   = *reinterpret_cast<const uint2 *>(gout + o0);
     U              gr[kOut], top[2 * kOut], bot[2 * kOut];
     if constexpr (sizeof(U) == 4) {
@@ -195,6 +199,7 @@ maxpool2x2_bwd_vec_kernel(const uint32_t *__restrict__ codes, const U *__restric
 #pragma unroll
     for (int j = 0; j < kOut; ++j) {
         const uint32_t k = (bits >> (2 * j)) & 3u;
+        gr[j]            = (live >> j) & 1u ? gr[j] : U(0);
         top[2 * j]       = k == 0 ? gr[j] : U(0);
         top[2 * j + 1]   = k == 1 ? gr[j] : U(0);
         bot[2 * j]       = k == 2 ? gr[j] : U(0);
@@ -235,8 +240,8 @@ cudaError_t fwd_typed(const void *x, uint64_t outputs, uint64_t wo, uint64_t wid
 }
 
 template <typename U>
-cudaError_t bwd_typed(const uint32_t *codes, const void *gout, uint64_t outputs, uint64_t wo, uint64_t width, uint64_t elements,
-                      void *gin, cudaStream_t s)
+cudaError_t bwd_typed(const uint32_t *codes, const uint32_t *mask, const void *gout, uint64_t outputs, uint64_t wo,
+                      uint64_t width, uint64_t elements, void *gin, cudaStream_t s)
 {
     if constexpr (sizeof(U) <= 4) {
         constexpr uint64_t kOut = 8 / sizeof(U);
@@ -245,11 +250,11 @@ cudaError_t bwd_typed(const uint32_t *codes, const void *gout, uint64_t outputs,
             if (vgrid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
             if (elements <= 0xFFFFFFFFull)
                 maxpool2x2_bwd_vec_kernel<U, uint32_t><<<static_cast<unsigned>(vgrid), kThreads, 0, s>>>(
-                    codes, static_cast<const U *>(gout), groups, static_cast<uint32_t>(per_row), static_cast<uint32_t>(width),
-                    static_cast<U *>(gin));
+                    codes, mask, static_cast<const U *>(gout), groups, static_cast<uint32_t>(per_row),
+                    static_cast<uint32_t>(width), static_cast<U *>(gin));
             else
                 maxpool2x2_bwd_vec_kernel<U, uint64_t><<<static_cast<unsigned>(vgrid), kThreads, 0, s>>>(
-                    codes, static_cast<const U *>(gout), groups, per_row, width, static_cast<U *>(gin));
+                    codes, mask, static_cast<const U *>(gout), groups, per_row, width, static_cast<U *>(gin));
             return cudaGetLastError();
         }
     }
@@ -257,10 +262,11 @@ cudaError_t bwd_typed(const uint32_t *codes, const void *gout, uint64_t outputs,
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     if (elements <= 0xFFFFFFFFull)
         maxpool2x2_bwd_kernel<U, uint32_t><<<static_cast<unsigned>(grid), kThreads, 0, s>>>(
-            codes, static_cast<const U *>(gout), outputs, static_cast<uint32_t>(wo), static_cast<uint32_t>(width), static_cast<U *>(gin));
+            codes, mask, static_cast<const U *>(gout), outputs, static_cast<uint32_t>(wo), static_cast<uint32_t>(width),
+            static_cast<U *>(gin));
     else
         maxpool2x2_bwd_kernel<U, uint64_t><<<static_cast<unsigned>(grid), kThreads, 0, s>>>(
-            codes, static_cast<const U *>(gout), outputs, wo, width, static_cast<U *>(gin));
+            codes, mask, static_cast<const U *>(gout), outputs, wo, width, static_cast<U *>(gin));
     return cudaGetLastError();
 }
 
@@ -278,13 +284,13 @@ cudaError_t launch_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t heigh
     }
 }
 
-cudaError_t launch_maxpool2x2_bwd(const uint32_t *codes, const void *gout, uint64_t planes, uint64_t height, uint64_t width,
-                                  int elem_size, void *gin, cudaStream_t s)
+cudaError_t launch_maxpool2x2_bwd(const uint32_t *codes, const uint32_t *mask, const void *gout, uint64_t planes,
+                                  uint64_t height, uint64_t width, int elem_size, void *gin, cudaStream_t s)
 {
     const uint64_t wo = width / 2, outputs = planes * (height / 2) * wo, elements = planes * height * width;
-    if (elem_size == 8) return bwd_typed<uint64_t>(codes, gout, outputs, wo, width, elements, gin, s);
-    return elem_size == 4 ? bwd_typed<uint32_t>(codes, gout, outputs, wo, width, elements, gin, s)
-                          : bwd_typed<uint16_t>(codes, gout, outputs, wo, width, elements, gin, s);
+    if (elem_size == 8) return bwd_typed<uint64_t>(codes, mask, gout, outputs, wo, width, elements, gin, s);
+    return elem_size == 4 ? bwd_typed<uint32_t>(codes, mask, gout, outputs, wo, width, elements, gin, s)
+                          : bwd_typed<uint16_t>(codes, mask, gout, outputs, wo, width, elements, gin, s);
 }
 
 }  // namespace bt

@@ -110,6 +110,9 @@ def test_later_entry_points_check_their_arguments_before_any_launch(L):
     assert L.bt_maxpool2x2_fwd(None, 4, 8, 8, B.BT_F32, A, A, None) == B.BT_ERR_NULL
     assert L.bt_maxpool2x2_fwd(None, 0, 8, 8, B.BT_F32, None, None, None) == B.BT_OK
     assert L.bt_maxpool2x2_bwd(A, A, 4, 8, 8, 13, A, None) == B.BT_ERR_DTYPE
+    assert L.bt_maxpool2x2_bwd_masked(A, None, A, 4, 8, 8, B.BT_F32, A, None) == B.BT_ERR_NULL
+    assert L.bt_maxpool2x2_bwd_masked(A, A + 2, A, 4, 8, 8, B.BT_F32, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_maxpool2x2_bwd_masked(A, A, A, 4, 8, 7, B.BT_F32, A, None) == B.BT_ERR_SHAPE
     # arena forms
     assert L.bt_compress_arena(A, 8192, B.BT_F32, A, A, 1 << 20, None, A, *tail) == B.BT_ERR_NULL      # no cursor
     assert L.bt_compress_arena(A, 8192, B.BT_F32, A, A, 1 << 20, A, None, *tail) == B.BT_ERR_NULL      # no offset word

@@ -55,6 +55,15 @@ def test_forward_and_backward_match_the_oracle(G, oracle, kind, shape):
                         planes=planes, height=h, width=w)
     torch.cuda.synchronize()
     assert gin.guards_intact() and np.array_equal(gin.raw(), oracle.maxpool2x2_bwd(c_ref, g, planes, h, w))
+    # masked form: the ReLU's select on the pooled gradient and the scatter in one pass
+    mask = oracle.compress(W.random_patterns(y_ref.size, kind, 0.5, seed=78, with_specials=False)).bitmap
+    gin2 = G.Guarded(n, G.TDT[kind])
+    B.bt_maxpool2x2_bwd_masked(torch.from_numpy(c_ref.view(np.int32).copy()).cuda(),
+                               torch.from_numpy(mask.view(np.int32).copy()).cuda(), G.from_raw(g, kind), gin2.inner,
+                               planes=planes, height=h, width=w)
+    torch.cuda.synchronize()
+    masked_g = oracle.relu_bwd_from_bitmap(mask, g)
+    assert gin2.guards_intact() and np.array_equal(gin2.raw(), oracle.maxpool2x2_bwd(c_ref, masked_g, planes, h, w))
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
