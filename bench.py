@@ -422,13 +422,15 @@ def large_tensor_kernels(dev, peak_gbs: float):
         codes = torch.empty((no + 15) // 16, dtype=torch.int32, device=dev)
         gin = torch.empty_like(x)
         by = 5 * no * es + 4 * ((no + 15) // 16)
+        pooled_bitmap = torch.randint(-2 ** 31, 2 ** 31 - 1, ((no + 31) // 32,), dtype=torch.int32, device=dev)
         for op, fn in (("bt_maxpool2x2_fwd", lambda: B.bt_maxpool2x2_fwd(x, y, codes)),
-                       ("bt_maxpool2x2_bwd", lambda: B.bt_maxpool2x2_bwd(codes, y, gin))):
+                       ("bt_maxpool2x2_bwd", lambda: B.bt_maxpool2x2_bwd(codes, y, gin)),
+                       ("bt_maxpool2x2_bwd_masked", lambda: B.bt_maxpool2x2_bwd_masked(codes, pooled_bitmap, y, gin))):
             ms, best = time_call(fn)
             rows[label + "_" + op] = {"ms_median": round(ms, 4), "ms_best": round(best, 4), "moved_gbs": round(by / ms / 1e6, 1),
                                       "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
                                       "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
-        del x, y, codes, gin
+        del x, y, codes, gin, pooled_bitmap
         torch.cuda.empty_cache()
     out["maxpool2x2_[32,64,224,224]"] = rows
     return out
