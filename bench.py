@@ -51,6 +51,9 @@ def parse_args():
     p.add_argument("--chains", type=int, choices=(1, 2, 4), default=4,
                    help="independent chains of the step's graph: 2 = plain codec / fused pair on two streams, "
                         "4 = each of them split into even and odd layers")
+    p.add_argument("--cta-budget", default="49,74",
+                   help="CTAs per compress launch when the step runs as several chains: 'small,large' for layers "
+                        "of at most / more than 800 tiles of 8192 elements (0 = one CTA per SM); see bt_set_max_ctas")
     return p.parse_args()
 
 
@@ -192,6 +195,12 @@ class Cfg2Step:
         self.total_elems = sum(l["n"] for l in self.layers)
         self.dense_bytes_per_step = len(OPS) * 4 * self.total_elems
         self.launches_per_step = len(OPS) * len(self.layers)
+        # CTAs per compress launch (small layers, large layers); (0, 0) = one CTA per SM.  A cooperative launch
+        # starts only when all its CTAs fit, so chains that are to overlap get a share of the SMs each.
+        self.cta_budget = (0, 0)
+
+    def cta_limit(self, n: int) -> int:
+        return self.cta_budget[0] if n <= 800 * 8192 else self.cta_budget[1]
 
     def run(self, only_op=None, only_layer=None, streams=None):
         """One step (forward over the layers, backward in reverse).  `only_op` / `only_layer` restrict it to
@@ -213,6 +222,7 @@ class Cfg2Step:
 
         for i, l in enumerate(self.layers):
             a, b = l["stash_a"], l["stash_b"]
+            B.bt_set_max_ctas(self.cta_limit(l["n"]))
             if want("bt_compress", i):
                 c = chain(0, i)
                 B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.wss[c], a.dev_status,
@@ -221,6 +231,7 @@ class Cfg2Step:
                 c = chain(1, i)
                 B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.wss[c],
                                        b.dev_status, stream=streams[c] if streams else None)
+        B.bt_set_max_ctas(0)
         for i in range(len(self.layers) - 1, -1, -1):
             l = self.layers[i]
             a, b = l["stash_a"], l["stash_b"]
@@ -249,29 +260,42 @@ class Cfg2Step:
         return [l["stash_a"].nnz for l in self.layers]
 
 
-def per_kernel_pass(step: Cfg2Step, steps: int):
+def per_kernel_pass(step: Cfg2Step, steps: int, chains: int = 1):
     """Device time of each operation: the step's launches of ONE operation (all 17 layers, in the step's
-    order) captured as a CUDA graph of their own and replayed `steps` times between two CUDA events on the
-    launching stream, so the figure holds what the whole-step graph holds for that operation (kernel time
-    and the device's launch latency between dependent kernels) and no host overhead.  The inputs of one
-    such pass (0.3 GB and more) exceed the L2.  The largest layer is timed the same way on its own,
-    with the L2 flushed before every replay."""
+    order and launch configuration: with four chains the operation's even and odd layers on two streams, with
+    the step's CTA budget) captured as a CUDA graph of their own and replayed `steps` times between two CUDA
+    events on the launching stream, so the figure holds what the whole-step graph holds for that operation
+    (kernel time, the device's launch latency between dependent kernels, the overlap of the operation's own
+    two chains) and no host overhead.  The inputs of one such pass (0.3 GB and more) exceed the L2.  The
+    largest layer is timed on its own, one launch with one CTA per SM, the L2 flushed before every replay."""
     import torch
     dev = step.restored.device
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     per_op, per_layer = {}, {}
     side = torch.cuda.Stream()
+    branches = [torch.cuda.Stream() for _ in range(3)] if chains == 4 else []
+    budget = step.cta_budget
     for op in OPS:
         graphs = []
         for only in (None, 0):
             g = torch.cuda.CUDAGraph()
+            step.cta_budget = budget if only is None else (0, 0)
             side.wait_stream(torch.cuda.current_stream())
             with torch.cuda.stream(side):
                 step.run(only_op=op, only_layer=only)          # warm-up outside the capture
             torch.cuda.current_stream().wait_stream(side)
             with torch.cuda.graph(g):
-                step.run(only_op=op, only_layer=only)
+                if branches and only is None:
+                    main_stream = torch.cuda.current_stream()
+                    for b in branches:
+                        b.wait_stream(main_stream)
+                    step.run(only_op=op, streams=[main_stream] + branches)
+                    for b in branches:
+                        main_stream.wait_stream(b)
+                else:
+                    step.run(only_op=op, only_layer=only)
             graphs.append(g)
+        step.cta_budget = budget
         whole, big = graphs
         for _ in range(3):
             whole.replay()
@@ -510,6 +534,8 @@ def run_ours(args):
     peak, peak_kind = measured_peak_gbs()
 
     step = Cfg2Step(dev, args.batch)
+    if args.chains > 1:
+        step.cta_budget = tuple(int(v) for v in args.cta_budget.split(","))
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
         for _ in range(max(args.warmup, 3)):
@@ -557,7 +583,7 @@ def run_ours(args):
     clocks = sampler.summary(t0, t1)
 
     # per-operation device time: one CUDA graph per operation, replayed between two events
-    per_op, per_layer = per_kernel_pass(step, min(args.steps, 20))
+    per_op, per_layer = per_kernel_pass(step, min(args.steps, 20), args.chains)
 
     # end to end: inputs start in pinned host memory, results end in host memory, every step
     e2e = None
@@ -581,6 +607,8 @@ def run_ours(args):
         # the largest layer alone (98 MiB dense), the launch closest to the sizes the roofline bar is set for
         big_ms = statistics.median(per_layer[(dom, 0)])
         big_alg = algorithmic_bytes(dom, step.layers[0]["n"], nnz[0], 4)
+        # all four operations together: the bytes the method must move in one step over the step's time
+        step_alg = sum(algorithmic_bytes(op, l["n"], z, 4) for op in OPS for l, z in zip(step.layers, nnz))
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
@@ -593,6 +621,9 @@ def run_ours(args):
                                                               "pair%s)" % (args.chains, args.chains, ", even / odd layers"
                                                                            if args.chains == 4 else "")
                                                               if args.chains > 1 else ""),
+                       "cta_budget": ("compress launches limited to %d CTAs (layers of at most 800 tiles) / %d CTAs "
+                                      "(larger layers; 0 = one per SM) so that the chains' cooperative launches are "
+                                      "resident side by side" % step.cta_budget) if any(step.cta_budget) else "one CTA per SM",
                        "l2": "per-step working set %.2f GB exceeds the 126 MB L2; no flush between steps"
                              % (7 * 4 * step.total_elems / 1e9),
                        "parallelism": "dp%d" % world if world > 1 else "single"},
@@ -607,7 +638,13 @@ def run_ours(args):
                                            "achieved": round(big_alg / big_ms / 1e6, 1),
                                            "frac": round(big_alg / big_ms / 1e6 / peak, 4)},
                          "per_op_ms_per_step": {k: round(v["ms"] / max(1, v["launches"]) * len(step.layers), 5)
-                                                for k, v in per_op.items()}},
+                                                for k, v in per_op.items()},
+                         "whole_step": {"algorithmic_bytes": step_alg,
+                                        "achieved": round(step_alg / (ms_step * 1e-3) / 1e9, 1),
+                                        "frac": round(step_alg / (ms_step * 1e-3) / 1e9 / peak, 4)},
+                         "how": "avg_launch_ms = time of the step's launches of this operation, in the step's launch "
+                                "configuration (its even / odd chains on two streams, the CTA budget), over their "
+                                "number; largest_layer = one launch alone, one CTA per SM, L2 flushed"},
         }
         if e2e is not None:
             e2e_ms = e2e["ms"] / e2e["steps"]

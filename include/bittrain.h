@@ -89,6 +89,22 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype);
 size_t bt_workspace_bytes(uint64_t n);
 
 /*
+ * Launch configuration for callers that keep several compress calls in flight
+ * (on several streams, or in the branches of a CUDA graph).  The compress
+ * kernel is launched cooperatively with one CTA per SM, and a cooperative
+ * launch starts only when all its CTAs can be resident: two launches of more
+ * than half the SMs each therefore run one after the other, whatever their
+ * streams.  bt_set_max_ctas(m) limits every later compress-family launch MADE
+ * BY THE CALLING THREAD to m CTAs (0: no limit, the default), so that
+ * floor(SMs / m) launches can run side by side, each somewhat slower than it
+ * would be alone.  Results do not depend on the limit.  Returns the limit it
+ * replaces, or -1 (and changes nothing) if m < 0.  Host-side state only: a
+ * launch captured into a CUDA graph keeps the limit it was captured with.
+ * No counterpart in the paper.
+ */
+int bt_set_max_ctas(int max_ctas);
+
+/*
  * Algorithm 1 (dense -> bitmap).  Reads dense[0..n), writes bitmap
  * (ceil(n/32) words), values[0..nnz), chunk_prefix (ceil(n/4096) entries) and
  * *nnz_out.  values_capacity is the number of ELEMENTS the values buffer can

@@ -84,6 +84,12 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype)
     return static_cast<size_t>(4 * ceil_div(n, 32) + nnz * static_cast<uint64_t>(es) + 8 * ceil_div(n, BT_CHUNK_ELEMS));
 }
 
+int bt_set_max_ctas(int max_ctas)
+{
+    if (max_ctas < 0) return -1;
+    return static_cast<int>(bt::set_compress_max_ctas(static_cast<uint32_t>(max_ctas)));
+}
+
 size_t bt_workspace_bytes(uint64_t n)
 {
     return bt::kWsHeaderBytes + 16 + 24 * static_cast<size_t>(ceil_div(n, bt::kMinTileElems));

@@ -730,6 +730,12 @@ uint64_t next_call_tag()
     return counter.fetch_add(1, std::memory_order_relaxed);
 }
 
+// The calling thread's limit on the CTAs of one compress launch (0: none).  A cooperative launch needs all its
+// CTAs resident at once and a CTA of this kernel fills an SM, so two launches of more than half the SMs each run
+// one after the other even on different streams; a caller that keeps several launches in flight gives each a
+// share of the SMs.
+thread_local uint32_t t_max_ctas = 0;
+
 // Launch shape of one kernel instantiation on one device: the opt-in shared
 // memory size is set and the number of co-resident CTAs is looked up once.
 struct LaunchShape {
@@ -773,6 +779,7 @@ cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
     cudaError_t    e         = shape.max_grid(kernel, kThreads, kSmem, max_grid);
     if (e != cudaSuccess) return e;
     if (max_grid > 32 * kMaxWindows) max_grid = 32 * kMaxWindows;
+    if (t_max_ctas != 0 && static_cast<uint32_t>(max_grid) > t_max_ctas) max_grid = static_cast<int>(t_max_ctas);
     const uint32_t grid  = num_tiles < static_cast<uint32_t>(max_grid) ? num_tiles : static_cast<uint32_t>(max_grid);
     const uint32_t waves = (num_tiles + grid - 1) / grid;
     // cooperative launch: the runtime guarantees that all `grid` CTAs are resident together
@@ -824,6 +831,13 @@ extern "C" int bt_debug_set_buffer(void *buf, unsigned int it0)
     return cudaMemcpyToSymbol(g_dbg_it0, &it0, sizeof(it0)) != cudaSuccess;
 }
 #endif
+
+uint32_t set_compress_max_ctas(uint32_t max_ctas)
+{
+    const uint32_t before = t_max_ctas;
+    t_max_ctas            = max_ctas;
+    return before;
+}
 
 cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStream_t stream)
 {

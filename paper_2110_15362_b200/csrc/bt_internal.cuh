@@ -53,6 +53,8 @@ struct CompressArgs {
 
 // fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0), 2 ReLU6
 cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStream_t s);
+// the calling thread's limit on the CTAs of one compress launch (0: none); returns the limit it replaces
+uint32_t set_compress_max_ctas(uint32_t max_ctas);
 // values_offset: NULL, or a device word holding the byte offset of the packed values inside `values`
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                               const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t s);

@@ -131,6 +131,18 @@ def test_later_entry_points_check_their_arguments_before_any_launch(L):
     assert L.bt_relu6_bwd_from_stash_arena(None, None, None, None, None, 0, B.BT_F32, None, None) == B.BT_OK
 
 
+def test_cta_limit_is_per_thread_host_state(L):
+    import threading
+    assert L.bt_set_max_ctas(0) == 0
+    assert L.bt_set_max_ctas(74) == 0 and L.bt_set_max_ctas(49) == 74
+    assert L.bt_set_max_ctas(-1) == -1 and L.bt_set_max_ctas(49) == 49          # a negative limit changes nothing
+    seen = []
+    t = threading.Thread(target=lambda: seen.append((L.bt_set_max_ctas(5), L.bt_set_max_ctas(0))))
+    t.start(), t.join()
+    assert seen == [(0, 5)]                                                      # another thread starts without a limit
+    assert L.bt_set_max_ctas(0) == 49
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
     monkeypatch.setattr(B, "library_path", lambda: str(tmp_path / "nope.so"))
