@@ -9,7 +9,10 @@ bt_compress (from the post-ReLU activation) and once with bt_relu_fwd_compress
 bt_decompress and its ReLU gradient formed with bt_relu_bwd_from_bitmap.  The
 metric is dense-equivalent GB/s: the dense bytes of every tensor an entry point
 consumed or produced (N * sizeof(dtype) per call), summed over the step,
-divided by the step time.
+divided by the step time.  The step is one CUDA graph of four independent chains
+(plain codec / fused pair, even / odd layers) on four streams; each compress
+launch is limited to a share of the SMs (bt_set_max_ctas) so that the chains'
+cooperative launches are resident side by side.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
