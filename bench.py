@@ -9,8 +9,8 @@ bt_compress (from the post-ReLU activation) and once with bt_relu_fwd_compress
 bt_decompress and its ReLU gradient formed with bt_relu_bwd_from_bitmap.  The
 metric is dense-equivalent GB/s: the dense bytes of every tensor an entry point
 consumed or produced (N * sizeof(dtype) per call), summed over the step,
-divided by the step time.  The step is one CUDA graph of four independent chains
-(plain codec / fused pair, even / odd layers) on four streams; each compress
+divided by the step time.  The step is one CUDA graph of eight independent chains
+(plain codec / fused pair, layers by index mod 4) on eight streams; each compress
 launch is limited to a share of the SMs (bt_set_max_ctas) so that the chains'
 cooperative launches are resident side by side.
 
@@ -51,10 +51,10 @@ def parse_args():
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-large", action="store_true", help="skip the per-kernel runs on 1 GiB tensors")
     p.add_argument("--no-e2e", action="store_true")
-    p.add_argument("--chains", type=int, choices=(1, 2, 4), default=4,
+    p.add_argument("--chains", type=int, choices=(1, 2, 4, 8), default=8,
                    help="independent chains of the step's graph: 2 = plain codec / fused pair on two streams, "
-                        "4 = each of them split into even and odd layers")
-    p.add_argument("--cta-budget", default="49,74",
+                        "4 = each of them split into even and odd layers, 8 = into layers by index mod 4")
+    p.add_argument("--cta-budget", default="24,74",
                    help="CTAs per compress launch when the step runs as several chains: 'small,large' for layers "
                         "of at most / more than 800 tiles of 8192 elements (0 = one CTA per SM); see bt_set_max_ctas")
     return p.parse_args()
@@ -191,9 +191,9 @@ class Cfg2Step:
             grad = W.cfg2_grad(i, shape, dev).reshape(-1)
             self.layers.append(dict(n=n, pre=pre, act=act, grad=grad,
                                     stash_a=B.Stash(n, torch.float32, dev), stash_b=B.Stash(n, torch.float32, dev)))
-        # one output buffer and one workspace per chain (at most four chains); chain 0 restores the activations
-        self.outs = [torch.empty(n_max, dtype=torch.float32, device=dev) for _ in range(4)]
-        self.wss = [B.new_workspace(n_max, dev) for _ in range(4)]
+        # one output buffer and one workspace per chain (at most eight chains); chain 0 restores the activations
+        self.outs = [torch.empty(n_max, dtype=torch.float32, device=dev) for _ in range(8)]
+        self.wss = [B.new_workspace(n_max, dev) for _ in range(8)]
         self.restored, self.gin, self.ws = self.outs[0], self.outs[1], self.wss[0]
         self.total_elems = sum(l["n"] for l in self.layers)
         self.dense_bytes_per_step = len(OPS) * 4 * self.total_elems
@@ -207,10 +207,10 @@ class Cfg2Step:
 
     def run(self, only_op=None, only_layer=None, streams=None):
         """One step (forward over the layers, backward in reverse).  `only_op` / `only_layer` restrict it to
-        one operation and / or one layer, for the per-operation timing passes.  With `streams` (a list of 2
-        or 4 streams, the first being the current one) the step runs as independent chains -- the plain codec
+        one operation and / or one layer, for the per-operation timing passes.  With `streams` (a list of 2,
+        4 or 8 streams, the first being the current one) the step runs as independent chains -- the plain codec
         (compress ... decompress) and the fused pair (fused forward ... ReLU backward), each optionally split
-        into even and odd layers -- every chain with its own stream, workspace and output buffer, so that one
+        into even and odd layers or into layers by index mod 4 -- every chain with its own stream, workspace and output buffer, so that one
         chain's launch latency hides behind another's kernels."""
         B = self.B
         k = 1 if not streams else len(streams)
@@ -218,7 +218,7 @@ class Cfg2Step:
         def chain(family, i):                       # family 0: plain codec, 1: fused pair
             if k == 1:
                 return 0
-            return family if k == 2 else 2 * family + (i & 1)
+            return family if k == 2 else (2 * family + (i & 1) if k == 4 else 4 * family + (i & 3))
 
         def want(op, i):
             return (only_op is None or op == only_op) and (only_layer is None or i == only_layer)
@@ -265,8 +265,8 @@ class Cfg2Step:
 
 def per_kernel_pass(step: Cfg2Step, steps: int, chains: int = 1):
     """Device time of each operation: the step's launches of ONE operation (all 17 layers, in the step's
-    order and launch configuration: with four chains the operation's even and odd layers on two streams, with
-    the step's CTA budget) captured as a CUDA graph of their own and replayed `steps` times between two CUDA
+    order and launch configuration: with four or eight chains the operation's own two or four chains on their
+    streams, with the step's CTA budget) captured as a CUDA graph of their own and replayed `steps` times between two CUDA
     events on the launching stream, so the figure holds what the whole-step graph holds for that operation
     (kernel time, the device's launch latency between dependent kernels, the overlap of the operation's own
     two chains) and no host overhead.  The inputs of one such pass (0.3 GB and more) exceed the L2.  The
@@ -276,7 +276,7 @@ def per_kernel_pass(step: Cfg2Step, steps: int, chains: int = 1):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     per_op, per_layer = {}, {}
     side = torch.cuda.Stream()
-    branches = [torch.cuda.Stream() for _ in range(3)] if chains == 4 else []
+    branches = [torch.cuda.Stream() for _ in range(chains - 1)] if chains >= 4 else []
     budget = step.cta_budget
     for op in OPS:
         graphs = []
@@ -621,8 +621,8 @@ def run_ours(args):
                            1.0 - sum(nnz) / step.total_elems, 4),
                        "ops_per_layer": list(OPS),
                        "launch": "one CUDA graph per step" + (", %d independent chains on %d streams (plain codec / fused "
-                                                              "pair%s)" % (args.chains, args.chains, ", even / odd layers"
-                                                                           if args.chains == 4 else "")
+                                                              "pair%s)" % (args.chains, args.chains, ", even / odd layers" if args.chains == 4
+                                                                           else ", layers by index mod 4" if args.chains == 8 else "")
                                                               if args.chains > 1 else ""),
                        "cta_budget": ("compress launches limited to %d CTAs (layers of at most 800 tiles) / %d CTAs "
                                       "(larger layers; 0 = one per SM) so that the chains' cooperative launches are "
@@ -646,7 +646,7 @@ def run_ours(args):
                                         "achieved": round(step_alg / (ms_step * 1e-3) / 1e9, 1),
                                         "frac": round(step_alg / (ms_step * 1e-3) / 1e9 / peak, 4)},
                          "how": "avg_launch_ms = time of the step's launches of this operation, in the step's launch "
-                                "configuration (its even / odd chains on two streams, the CTA budget), over their "
+                                "configuration (its own chains on their streams, the CTA budget), over their "
                                 "number; largest_layer = one launch alone, one CTA per SM, L2 flushed"},
         }
         if e2e is not None:
