@@ -268,3 +268,55 @@ def test_more_than_two_to_the_32_elements(oracle):
     assert torch.equal(bits_of(vals), bits_of(st.values[:nnz]))   # where a bit is set, pre == y
     del pre, y, back, vals, st, ws
     torch.cuda.empty_cache()
+
+
+def test_cfg2_step_in_the_launch_configuration_the_benchmark_times(oracle):
+    """The benchmark's own step object, captured as it is timed (one CUDA graph, eight chains on eight streams, 24
+    / 74 CTAs per compress launch) and replayed: both stashes of every layer against the oracle (the largest
+    layer against torch routines and on sampled chunks), the restored activations and the ReLU gradients."""
+    import bench
+    step = bench.Cfg2Step(DEV, 32)
+    step.cta_budget = (24, 74)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step.run()
+    torch.cuda.synchronize()
+    for l in step.layers:                                    # forget what the warm-up wrote
+        for st in (l["stash_a"], l["stash_b"]):
+            st.bitmap.zero_(), st.values.zero_(), st.chunk_prefix.zero_(), st.nnz_out.zero_()
+    graph = torch.cuda.CUDAGraph()
+    branches = [torch.cuda.Stream() for _ in range(7)]
+    with torch.cuda.graph(graph):
+        main = torch.cuda.current_stream()
+        for b in branches:
+            b.wait_stream(main)
+        step.run(streams=[main] + branches)
+        for b in branches:
+            main.wait_stream(b)
+    assert B.bt_set_max_ctas(0) == 0                         # the step leaves no limit behind
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    step.check()
+    for i, l in enumerate(step.layers):
+        x, n = l["act"], l["n"]
+        for st in (l["stash_a"], l["stash_b"]):
+            if n <= 8_000_000:
+                ref = oracle.compress(W.raw_numpy(x))
+                assert st.nnz == ref.nnz and st.status == B.BT_OK
+                assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), ref.bitmap)
+                assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), ref.prefix)
+                assert np.array_equal(W.raw_numpy(st.values[:ref.nnz]), ref.values)
+            else:
+                check_against_torch(st, x)
+                check_sampled_chunks(oracle, st, x, decompress(st, x), seed=i)
+    # the last layer each chain restored / differentiated is still in that chain's output buffer
+    for c in range(8):
+        fam, r = divmod(c, 4)
+        i = min(j for j in range(len(step.layers)) if j % 4 == r)         # backward runs in reverse: lowest index last
+        l = step.layers[i]
+        out = step.outs[c][:l["n"]]
+        if fam == 0:
+            assert torch.equal(bits_of(out), bits_of(l["act"]))
+        else:
+            assert torch.equal(bits_of(out), bits_of(torch.where(l["act"] != 0, l["grad"], torch.zeros_like(l["grad"]))))
