@@ -203,6 +203,9 @@ class Cfg2Step:
         self.cta_budget = (0, 0)
 
     def cta_limit(self, n: int) -> int:
+        if len(self.cta_budget) == 5:                        # experiments: one limit per layer size, smallest first
+            tiles = (n + 8191) // 8192
+            return self.cta_budget[sum(tiles > t for t in (100, 200, 400, 800))]
         return self.cta_budget[0] if n <= 800 * 8192 else self.cta_budget[1]
 
     def run(self, only_op=None, only_layer=None, streams=None):
@@ -624,9 +627,11 @@ def run_ours(args):
                                                               "pair%s)" % (args.chains, args.chains, ", even / odd layers" if args.chains == 4
                                                                            else ", layers by index mod 4" if args.chains == 8 else "")
                                                               if args.chains > 1 else ""),
-                       "cta_budget": ("compress launches limited to %d CTAs (layers of at most 800 tiles) / %d CTAs "
-                                      "(larger layers; 0 = one per SM) so that the chains' cooperative launches are "
-                                      "resident side by side" % step.cta_budget) if any(step.cta_budget) else "one CTA per SM",
+                       "cta_budget": (("compress launches limited to %d CTAs (layers of at most 800 tiles) / %d CTAs "
+                                       "(larger layers; 0 = one per SM) so that the chains' cooperative launches are "
+                                       "resident side by side" % step.cta_budget) if len(step.cta_budget) == 2
+                                      else "CTAs per compress launch by layer size: %s" % (step.cta_budget,))
+                       if any(step.cta_budget) else "one CTA per SM",
                        "l2": "per-step working set %.2f GB exceeds the 126 MB L2; no flush between steps"
                              % (7 * 4 * step.total_elems / 1e9),
                        "parallelism": "dp%d" % world if world > 1 else "single"},
