@@ -1,5 +1,5 @@
 """Randomised stress of the single-pass compaction protocol: random sizes (one element to tens of millions), zero
-fractions and element types; two fused launches at a time on two streams, each with its own workspace filled
+fractions, element types and CTA limits; two fused launches at a time on two streams, each with its own workspace filled
 with garbage and reused back to back; every output compared with torch routines on the GPU.  Runs for
 BT_STRESS_SECONDS (default 5; a 300-second run covers some 200 000 cases)."""
 import os
@@ -38,6 +38,7 @@ def test_random_concurrent_launches_match_torch():
         nnz = int(mask.sum())
         bm_ref, pf_ref, v_ref = torch_bitmap(mask), torch_prefix(mask), bits_of(y_ref)[mask]
         outs = []
+        B.bt_set_max_ctas(int(rng.choice([0, 0, 0, 2, 7, 24, 49, 74, 111])))       # a share of the SMs per launch, or none
         for k, st_ in enumerate(streams):
             st_.wait_stream(torch.cuda.current_stream())
             with torch.cuda.stream(st_):
@@ -51,9 +52,10 @@ def test_random_concurrent_launches_match_torch():
                 back = torch.empty_like(pre)
                 B.bt_decompress(stash.bitmap, stash.values, stash.chunk_prefix, back, stream=st_)
                 outs.append((stash, y, back))
+        limit = B.bt_set_max_ctas(0)
         torch.cuda.synchronize()
         for stash, y, back in outs:
-            where = f"case {cases}: n={n} zeros={s} {dt}"
+            where = f"case {cases}: n={n} zeros={s} {dt} max_ctas={limit}"
             assert stash.status == B.BT_OK and stash.nnz == nnz, where
             assert torch.equal(stash.bitmap, bm_ref) and torch.equal(stash.chunk_prefix, pf_ref), where
             assert torch.equal(bits_of(stash.values[:nnz]), v_ref), where
