@@ -89,6 +89,40 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype);
 size_t bt_workspace_bytes(uint64_t n);
 
 /*
+ * Batched forms of bt_compress and bt_relu_fwd_compress: `count` tensors of one element type in ONE
+ * pass.  Algorithm 1 runs per tensor -- every tensor gets its own bitmap, values, chunk_prefix
+ * (starting again at 0), *nnz_out and *dev_status, exactly what the single-tensor call writes -- but
+ * the tiles of all tensors are dealt to the same resident grid, so a training step that stashes many
+ * activations of a few megabytes each pays the fixed cost of a launch (a few microseconds: load,
+ * compact, exchange counts, copy out) once per batch, not once per tensor.  `items` is a HOST array
+ * read before the call returns; the pointers inside are device pointers with the alignment rules of
+ * bt_compress.  bt_compress_batch: y_out must be NULL in every item; bt_relu_fwd_compress_batch: y_out
+ * NULL in every item or in none (BT_ERR_SHAPE otherwise).  Tensors with n == 0 get *nnz_out = 0 and
+ * *dev_status = BT_OK.  More than 32 non-empty tensors are handled as several launches on `stream`.
+ * workspace_bytes >= bt_batch_workspace_bytes(n of every item); contents as for bt_workspace_bytes.
+ * Nothing is launched on an argument error.  No counterpart in the paper (its loop is sequential).
+ */
+typedef struct bt_batch_item {
+    const void *dense;          /* input: the activation, or the pre-activation for the fused form */
+    void *y_out;                /* fused form: dense output, may alias dense; else NULL            */
+    uint32_t *bitmap;
+    void *values;
+    uint64_t values_capacity;   /* in elements                                                     */
+    uint64_t *chunk_prefix;
+    uint64_t *nnz_out;
+    int32_t *dev_status;        /* may be NULL                                                     */
+    uint64_t n;
+} bt_batch_item;
+
+size_t bt_batch_workspace_bytes(const uint64_t *n /* host */, uint32_t count);
+
+int bt_compress_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype,
+                      void *workspace, size_t workspace_bytes, void *stream);
+
+int bt_relu_fwd_compress_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Launch configuration for callers that keep several compress calls in flight
  * (on several streams, or in the branches of a CUDA graph).  The compress
  * kernel is launched cooperatively with one CTA per SM, and a cooperative

@@ -46,31 +46,89 @@ int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau
     }
     if (!src || !bitmap || !chunk_prefix || !workspace) return BT_ERR_NULL;
     if (!values && values_capacity != 0) return BT_ERR_NULL;
-    if (!aligned(src, 16) || !aligned(y, 16) || !aligned(bitmap, 16) || !aligned(values, 16) ||
+    if (!aligned(src, 16) || !aligned(y, 16) || !aligned(bitmap, 4) || !aligned(values, 16) ||
         !aligned(chunk_prefix, 8) || !aligned(workspace, 16))
         return BT_ERR_ALIGN;
     if (workspace_bytes < bt_workspace_bytes(n)) return BT_ERR_WORKSPACE;
 
-    bt::CompressArgs a;
-    a.src        = src;
-    a.y          = y;
-    a.bitmap     = bitmap;
-    a.values     = values;
-    a.capacity   = values_capacity;
-    a.prefix     = chunk_prefix;
-    a.nnz_out    = nnz_out;
-    a.dev_status = dev_status;
-    a.ws_header  = static_cast<uint64_t *>(workspace);
-    a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
-    a.ws_waves   = 0;
-    a.call_tag   = 0;
-    a.cast       = cast;
-    a.tau        = tau;
-    a.arena_cursor      = arena.cursor;
-    a.values_offset_out = arena.offset_out;
-    a.arena_bytes       = arena.bytes;
-    a.n          = n;
-    return bt::launch_compress(a, dtype, fused, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+    bt::CompressJob j{};
+    j.src        = src;
+    j.y          = y;
+    j.bitmap     = bitmap;
+    j.values     = values;
+    j.capacity   = values_capacity;
+    j.prefix     = chunk_prefix;
+    j.nnz_out    = nnz_out;
+    j.dev_status = dev_status;
+    j.n          = n;
+    bt::CompressCommon c{};
+    c.cast              = cast;
+    c.tau               = tau;
+    c.arena_cursor      = arena.cursor;
+    c.values_offset_out = arena.offset_out;
+    c.arena_bytes       = arena.bytes;
+    return bt::launch_compress(c, &j, 1, workspace, dtype, fused, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+}
+
+// The batched forms: every tensor is checked before anything is launched; empty tensors get their nnz and status
+// words and take no part in the launches; the others go out kMaxBatch at a time, one launch after the other on
+// the stream, all through the same workspace.
+int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype, int fused, void *workspace,
+                          size_t workspace_bytes, void *stream)
+{
+    if (elem_size_of(dtype) == 0) return BT_ERR_DTYPE;
+    if (count == 0) return BT_OK;
+    if (!items) return BT_ERR_NULL;
+    uint64_t chunks = 0;
+    bool     any_y = false, all_y = true, any = false;
+    for (uint32_t k = 0; k < count; ++k) {
+        const bt_batch_item &it = items[k];
+        if (!it.nnz_out) return BT_ERR_NULL;
+        if (!aligned(it.nnz_out, 8) || !aligned(it.dev_status, 4)) return BT_ERR_ALIGN;
+        if (it.n == 0) continue;
+        if (!it.dense || !it.bitmap || !it.chunk_prefix) return BT_ERR_NULL;
+        if (!it.values && it.values_capacity != 0) return BT_ERR_NULL;
+        if (!aligned(it.dense, 16) || !aligned(it.y_out, 16) || !aligned(it.bitmap, 4) || !aligned(it.values, 16) ||
+            !aligned(it.chunk_prefix, 8))
+            return BT_ERR_ALIGN;
+        any = true;
+        any_y |= it.y_out != nullptr;
+        all_y &= it.y_out != nullptr;
+        chunks += ceil_div(it.n, BT_CHUNK_ELEMS);
+    }
+    if (fused == 0 && any_y) return BT_ERR_SHAPE;            // the plain compressor has no dense output
+    if (any_y && !all_y) return BT_ERR_SHAPE;                // a dense output for every tensor of a batch or for none
+    if (any && !workspace) return BT_ERR_NULL;
+    if (any && !aligned(workspace, 16)) return BT_ERR_ALIGN;
+    if (any && workspace_bytes < bt::compress_workspace_bytes(chunks)) return BT_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    bt::CompressJob    jobs[bt::kMaxBatch];
+    uint32_t           m = 0;
+    bt::CompressCommon c{};
+    for (uint32_t k = 0; k < count; ++k) {
+        const bt_batch_item &it = items[k];
+        if (it.n == 0) {
+            if (cudaMemsetAsync(it.nnz_out, 0, sizeof(uint64_t), s) != cudaSuccess) return BT_ERR_CUDA;
+            if (it.dev_status && cudaMemsetAsync(it.dev_status, 0, sizeof(int32_t), s) != cudaSuccess) return BT_ERR_CUDA;
+        } else {
+            bt::CompressJob &j = jobs[m++];
+            j                  = bt::CompressJob{};
+            j.src              = it.dense;
+            j.y                = fused ? it.y_out : nullptr;
+            j.bitmap           = it.bitmap;
+            j.values           = it.values;
+            j.capacity         = it.values_capacity;
+            j.prefix           = it.chunk_prefix;
+            j.nnz_out          = it.nnz_out;
+            j.dev_status       = it.dev_status;
+            j.n                = it.n;
+        }
+        if (m == bt::kMaxBatch || (k + 1 == count && m > 0)) {
+            if (bt::launch_compress(c, jobs, m, workspace, dtype, fused, s) != cudaSuccess) return BT_ERR_CUDA;
+            m = 0;
+        }
+    }
+    return BT_OK;
 }
 
 }  // namespace
@@ -90,9 +148,34 @@ int bt_set_max_ctas(int max_ctas)
     return static_cast<int>(bt::set_compress_max_ctas(static_cast<uint32_t>(max_ctas)));
 }
 
+#ifdef BT_TEST_HOOKS
+// Test builds only (never the product library): the bound of every wait inside the compress kernels, so that a
+// test can make a wait run out by itself and see the kernel return BT_ERR_TIMEOUT.
+uint64_t bt_test_set_wait_ns(uint64_t wait_ns) { return bt::set_compress_wait_ns(wait_ns); }
+#endif
+
 size_t bt_workspace_bytes(uint64_t n)
 {
-    return bt::kWsHeaderBytes + 16 + 24 * static_cast<size_t>(ceil_div(n, bt::kMinTileElems));
+    return bt::compress_workspace_bytes(ceil_div(n, BT_CHUNK_ELEMS));
+}
+
+size_t bt_batch_workspace_bytes(const uint64_t *n, uint32_t count)
+{
+    uint64_t chunks = 0;
+    for (uint32_t k = 0; n && k < count; ++k) chunks += ceil_div(n[k], BT_CHUNK_ELEMS);
+    return bt::compress_workspace_bytes(chunks);
+}
+
+int bt_compress_batch(const bt_batch_item *items, uint32_t count, int dtype, void *workspace, size_t workspace_bytes,
+                      void *stream)
+{
+    return compress_batch_common(items, count, dtype, 0, workspace, workspace_bytes, stream);
+}
+
+int bt_relu_fwd_compress_batch(const bt_batch_item *items, uint32_t count, int dtype, void *workspace,
+                               size_t workspace_bytes, void *stream)
+{
+    return compress_batch_common(items, count, dtype, 1, workspace, workspace_bytes, stream);
 }
 
 int bt_compress(const void *dense, uint64_t n, int dtype, uint32_t *bitmap, void *values, uint64_t values_capacity,

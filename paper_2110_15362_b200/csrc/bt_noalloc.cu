@@ -15,7 +15,7 @@
 namespace {
 
 // scratch for at most BT_NOALLOC_MAX_ELEMS elements: the same layout bt_workspace_bytes() sizes
-constexpr size_t kScratchBytes = bt::kWsHeaderBytes + 16 + 24 * (BT_NOALLOC_MAX_ELEMS / bt::kMinTileElems);
+constexpr size_t kScratchBytes = bt::compress_workspace_bytes(BT_NOALLOC_MAX_ELEMS / BT_CHUNK_ELEMS);
 
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
@@ -58,30 +58,23 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
     }
     if (!dense || !bitmap || !chunk_prefix) return BT_ERR_NULL;
     if (!values && values_capacity != 0) return BT_ERR_NULL;
-    if (!aligned(dense, 16) || !aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8))
+    if (!aligned(dense, 16) || !aligned(bitmap, 4) || !aligned(values, 16) || !aligned(chunk_prefix, 8))
         return BT_ERR_ALIGN;
 
     void     *scratch = nullptr;
     const int rc      = scratch_for_current_device(&scratch);   // first call on a device: looks the address up
     if (rc != BT_OK) return rc;
 
-    bt::CompressArgs a;
-    a.src        = dense;
-    a.y          = nullptr;
-    a.bitmap     = bitmap;
-    a.values     = values;
-    a.capacity   = values_capacity;
-    a.prefix     = chunk_prefix;
-    a.nnz_out    = nnz_out;
-    a.dev_status = dev_status;
-    a.ws_header  = static_cast<uint64_t *>(scratch);
-    a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(scratch) + bt::kWsHeaderBytes);
-    a.ws_waves   = 0;
-    a.call_tag   = 0;
-    a.cast       = 0;
-    a.tau        = 0.0f;
-    a.arena_cursor = nullptr, a.values_offset_out = nullptr, a.arena_bytes = 0;
-    a.n          = n;
+    bt::CompressJob j{};
+    j.src        = dense;
+    j.bitmap     = bitmap;
+    j.values     = values;
+    j.capacity   = values_capacity;
+    j.prefix     = chunk_prefix;
+    j.nnz_out    = nnz_out;
+    j.dev_status = dev_status;
+    j.n          = n;
+    bt::CompressCommon c{};
     // nothing in the scratch is cleared between calls: the kernel tells this call's words by their tag
-    return bt::launch_compress(a, dtype, false, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+    return bt::launch_compress(c, &j, 1, scratch, dtype, 0, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
