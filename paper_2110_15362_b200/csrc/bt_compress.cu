@@ -63,7 +63,8 @@ constexpr uint32_t kFull       = 0xFFFFFFFFu;
 constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
 constexpr int      kMaxWindows = kMaxGrid / 32;       // descriptor windows of 32 CTAs
 constexpr int      kHdrSeq     = 0;                   // header words (64-bit): launch sequence number,
-constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out)
+constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out),
+constexpr int      kHdrGo      = 2;                   //   go word (== the launch's tag once every CTA has arrived at the meeting)
 constexpr int      kCountShift = 40;                  // wave total word: (tiles added << 40) | sum of counts
 
 template <int kJobs>
@@ -140,9 +141,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = now_ns();
     for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 32; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if ((kStopOnAbort && *s_abort) || now_ns() - t0 > limit_ns) return false;
     }
 }
@@ -175,26 +174,6 @@ __device__ __forceinline__ uint4 lds_vec(uint32_t addr)
     return v;
 }
 __device__ __forceinline__ void sts_u8(uint32_t addr, uint32_t v) { asm volatile("st.shared.u8 [%0], %1;" ::"r"(addr), "r"(v)); }
-template <typename U>
-__device__ __forceinline__ void sts_elem(uint32_t addr, Reg<U> x)
-{
-    if constexpr (sizeof(U) == 8) asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(x));
-    else if constexpr (sizeof(U) == 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(x));
-    else asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(static_cast<uint16_t>(x)));
-}
-
-// if (cond) { store x at addr; addr += sizeof(U); } as predicated instructions (a branch per element costs more
-// than the element's other work)
-template <typename U>
-__device__ __forceinline__ void sts_elem_if(uint32_t &addr, Reg<U> x, uint32_t cond)
-{
-    if constexpr (sizeof(U) == 8)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u64 [%0], %1;\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(addr) : "l"(x), "r"(cond));
-    else if constexpr (sizeof(U) == 4)
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t}" : "+r"(addr) : "r"(x), "r"(cond));
-    else
-        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], %1;\n\t@p add.u32 %0, %0, 2;\n\t}" : "+r"(addr) : "h"(static_cast<uint16_t>(x)), "r"(cond));
-}
 
 // How a warp walks a segment: kVec elements per lane and step (one 16-byte vector), the counts of kPack
 // consecutive steps in kFieldBits-wide fields of one register (an inclusive warp sum of a field is at most
@@ -234,121 +213,240 @@ __device__ __forceinline__ uint4 repack(const Reg<U> (&e)[Vec<U>::kVec])
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// One warp compacts its segment of kSeg elements in place.  Returns the number of packed values; lane k
-// (k < kSeg / 32) leaves with bitmap word k of the segment in `word`.  `bm_addr` is the warp's staging area
-// for the bitmap (kSeg / 8 bytes of shared memory).  `y` (fused form with dense output) points at the
-// segment's first element of the dense output, `yvalid` is how many of them exist.  seg_addr and bm_addr are
-// shared-window addresses.
-//
-// The whole segment is in registers before the first packed value is stored, so reads and writes never meet.
-template <typename U, int FUSED, bool WRITE_Y, bool kGuardY, int kSeg>
-__device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, const uint32_t bm_addr, uint32_t &word,
-                                                    const uint32_t lane, U *y, const uint32_t yvalid, const float tau)
+// m |= bit where the 32-bit word / its low half / its high half / the 64-bit pair is not zero: a compare and a
+// predicated OR (written out because the compiler's own form, compare - select - OR, is one instruction longer,
+// and these run once per element)
+__device__ __forceinline__ void or_if_nz32(uint32_t &m, uint32_t x, uint32_t bit)
 {
-    using V                       = Vec<U>;
-    constexpr int      kVec       = V::kVec;
-    constexpr int      kPack      = V::kPack;
-    constexpr int      kFB        = V::kFieldBits;
-    constexpr int      kLPB       = V::kLanesPerByte;
-    constexpr int      kSteps     = kSeg / (32 * kVec);
-    constexpr uint32_t kES        = sizeof(U);
-    constexpr uint32_t kFieldMask = (1u << kFB) - 1u;
-    static_assert(kSteps % kPack == 0 && kSeg / 32 <= 32, "whole batches of steps; one bitmap word per lane");
-    static_assert(kLPB == 1 || kPack == 4, "the byte assembly below packs four steps");
-    constexpr int kBatches = kSteps / kPack;
-    const uint32_t in0 = seg_addr + lane * 16u;
-    // ---- phase 1: the whole segment into registers; masks, counts and bitmap bytes
-    Reg<U>   e[kSteps][kVec];
-    uint32_t m[kSteps];
-    uint32_t packed[kBatches];                       // the counts of a batch's steps, one per field
-    {
-        uint4 q[kSteps];
+    asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\t@p or.b32 %0, %0, %2;\n\t}" : "+r"(m) : "r"(x), "r"(bit));
+}
+__device__ __forceinline__ void or_if_nz_lo16(uint32_t &m, uint32_t x, uint32_t bit)
+{
+    asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tand.b32 t, %1, 0xFFFF;\n\tsetp.ne.u32 p, t, 0;\n\t@p or.b32 %0, %0, %2;\n\t}" : "+r"(m) : "r"(x), "r"(bit));
+}
+__device__ __forceinline__ void or_if_nz_hi16(uint32_t &m, uint32_t x, uint32_t bit)
+{
+    asm("{\n\t.reg .pred p;\n\tsetp.gt.u32 p, %1, 0xFFFF;\n\t@p or.b32 %0, %0, %2;\n\t}" : "+r"(m) : "r"(x), "r"(bit));
+}
+__device__ __forceinline__ void or_if_nz64(uint32_t &m, uint32_t lo, uint32_t hi, uint32_t bit)
+{
+    asm("{\n\t.reg .pred p;\n\t.reg .b32 t;\n\tor.b32 t, %1, %2;\n\tsetp.ne.u32 p, t, 0;\n\t@p or.b32 %0, %0, %3;\n\t}" : "+r"(m) : "r"(lo), "r"(hi), "r"(bit));
+}
+
+// the mask of a lane's vector: bit k set where its k-th element is not zero
+template <typename U>
+__device__ __forceinline__ uint32_t vec_mask(const uint4 &q)
+{
+    uint32_t m = 0;
+    if constexpr (sizeof(U) == 8) {
+        or_if_nz64(m, q.x, q.y, 1u), or_if_nz64(m, q.z, q.w, 2u);
+    } else if constexpr (sizeof(U) == 4) {
+        or_if_nz32(m, q.x, 1u), or_if_nz32(m, q.y, 2u), or_if_nz32(m, q.z, 4u), or_if_nz32(m, q.w, 8u);
+    } else {
+        or_if_nz_lo16(m, q.x, 1u), or_if_nz_hi16(m, q.x, 2u), or_if_nz_lo16(m, q.y, 4u), or_if_nz_hi16(m, q.y, 8u);
+        or_if_nz_lo16(m, q.z, 16u), or_if_nz_hi16(m, q.z, 32u), or_if_nz_lo16(m, q.w, 64u), or_if_nz_hi16(m, q.w, 128u);
+    }
+    return m;
+}
+
+// if (cond) { store the element at addr; addr += its size; } as predicated instructions (a branch per element
+// costs more than the element's other work); with kWrap, addr then wraps from `end` back by `ring` bytes
+template <bool kWrap>
+__device__ __forceinline__ void wrap_addr(uint32_t &addr, const uint32_t end, const uint32_t ring)
+{
+    if constexpr (kWrap) addr = addr >= end ? addr - ring : addr;
+}
+template <bool kWrap>
+__device__ __forceinline__ void sts32_if(uint32_t &addr, uint32_t x, uint32_t cond, const uint32_t end, const uint32_t ring)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t}" : "+r"(addr) : "r"(x), "r"(cond));
+    wrap_addr<kWrap>(addr, end, ring);
+}
+template <bool kWrap>
+__device__ __forceinline__ void sts64_if(uint32_t &addr, uint32_t lo, uint32_t hi, uint32_t cond, const uint32_t end, const uint32_t ring)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\t@p st.shared.v2.u32 [%0], {%1, %2};\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(addr) : "r"(lo), "r"(hi), "r"(cond));
+    wrap_addr<kWrap>(addr, end, ring);
+}
+// the two 16-bit elements of a word, each under its own condition
+template <bool kWrap>
+__device__ __forceinline__ void sts16x2_if(uint32_t &addr, uint32_t x, uint32_t cond_lo, uint32_t cond_hi, const uint32_t end, const uint32_t ring)
+{
+    if constexpr (!kWrap) {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\t"
+            "setp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], l;\n\t@p add.u32 %0, %0, 2;\n\t"
+            "setp.ne.u32 q, %3, 0;\n\t@q st.shared.u16 [%0], h;\n\t@q add.u32 %0, %0, 2;\n\t}"
+            : "+r"(addr)
+            : "r"(x), "r"(cond_lo), "r"(cond_hi));
+    } else {
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], l;\n\t@p add.u32 %0, %0, 2;\n\t}" : "+r"(addr) : "r"(x), "r"(cond_lo));
+        wrap_addr<true>(addr, end, ring);
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], h;\n\t@p add.u32 %0, %0, 2;\n\t}" : "+r"(addr) : "r"(x), "r"(cond_hi));
+        wrap_addr<true>(addr, end, ring);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The compaction of one segment of kSeg elements by one warp, in four steps that the kernel interleaves with
+// its hand-offs.  A lane takes one 16-byte vector per step (element (s * 32 + lane) * kVec + k of the segment
+// is its k-th of step s) and keeps it packed in four registers.
+template <typename U, int kSeg>
+struct Seg {
+    using V                              = Vec<U>;
+    static constexpr int      kVec       = V::kVec;
+    static constexpr int      kPack      = V::kPack;
+    static constexpr int      kFB        = V::kFieldBits;
+    static constexpr int      kLPB       = V::kLanesPerByte;
+    static constexpr int      kSteps     = kSeg / (32 * kVec);
+    static constexpr int      kBatches   = kSteps / kPack;
+    static constexpr int      kWords     = kSeg / 32;                 // bitmap words of the segment
+    static constexpr int      kWordsPerLane = (kWords + 31) / 32;
+    static constexpr uint32_t kES        = sizeof(U);
+    static constexpr uint32_t kFieldMask = (1u << kFB) - 1u;
+    static_assert(kSteps % kPack == 0 && kSteps >= kPack && kWords <= 64, "whole batches of steps; at most two bitmap words per lane");
+    static_assert(kLPB == 1 || kPack == 4, "the byte assembly packs four steps");
+};
+
+// (1) the segment into registers, the fused forward form applied, one mask per step (bit k: the lane's k-th
+// element of the step is kept, i.e. its pattern is not zero), the dense output written.
+template <typename U, int FUSED, bool WRITE_Y, bool kGuardY, int kSeg>
+__device__ __forceinline__ void segment_load(const uint32_t seg_addr, const uint32_t lane, uint4 (&q)[Seg<U, kSeg>::kSteps],
+                                             uint32_t (&m)[Seg<U, kSeg>::kSteps], U *y, const uint32_t yvalid, const float tau)
+{
+    using S = Seg<U, kSeg>;
 #pragma unroll
-        for (int s = 0; s < kSteps; ++s) q[s] = lds_vec(in0 + s * 512u);
+    for (int s = 0; s < S::kSteps; ++s) q[s] = lds_vec(seg_addr + lane * 16u + s * 512u);
 #pragma unroll
-        for (int s = 0; s < kSteps; ++s) {
-            unpack<U>(q[s], e[s]);
-            uint32_t mm = 0;
+    for (int s = 0; s < S::kSteps; ++s) {
+        if constexpr (FUSED >= 0) {
+            Reg<U> e[S::kVec];
+            unpack<U>(q[s], e);
 #pragma unroll
-            for (int k = 0; k < kVec; ++k) {
-                if constexpr (FUSED >= 0) e[s][k] = fused_forward<FUSED>(e[s][k], tau);
-                mm |= (e[s][k] != Reg<U>(0) ? 1u : 0u) << k;
-            }
-            if constexpr (FUSED >= 0 && WRITE_Y) {
-                const uint32_t at = (s * 32 + lane) * kVec;                // first element of the vector in the segment
-                if (!kGuardY || at + kVec <= yvalid) {
-                    *reinterpret_cast<uint4 *>(y + at) = repack<U>(e[s]);
+            for (int k = 0; k < S::kVec; ++k) e[k] = fused_forward<FUSED>(e[k], tau);
+            q[s] = repack<U>(e);
+            if constexpr (WRITE_Y) {
+                const uint32_t at = (s * 32 + lane) * S::kVec;                // first element of the vector in the segment
+                if (!kGuardY || at + S::kVec <= yvalid) {
+                    *reinterpret_cast<uint4 *>(y + at) = q[s];
                 } else {
 #pragma unroll
-                    for (int k = 0; k < kVec; ++k)
-                        if (at + k < yvalid) y[at + k] = static_cast<U>(e[s][k]);
+                    for (int k = 0; k < S::kVec; ++k)
+                        if (at + k < yvalid) y[at + k] = static_cast<U>(e[k]);
                 }
             }
-            m[s] = mm;
         }
+        m[s] = vec_mask<U>(q[s]);
     }
+}
+
+// (2) the masks are the bitmap: byte i of the segment's bitmap covers elements 8i .. 8i + 7.  The lanes behind a
+// byte combine their bits, the bytes go through a staging area (kSeg / 8 bytes of shared memory at bm_addr), and
+// lane k returns with bitmap words k * kWordsPerLane ... of the segment.
+template <typename U, int kSeg>
+__device__ __forceinline__ void segment_bitmap(const uint32_t (&m)[Seg<U, kSeg>::kSteps], const uint32_t bm_addr, const uint32_t lane,
+                                               uint32_t (&word)[Seg<U, kSeg>::kWordsPerLane])
+{
+    using S = Seg<U, kSeg>;
+    __syncwarp();                                   // the words of the segment before this one have been read
 #pragma unroll
-    for (int b = 0; b < kBatches; ++b) {
-        packed[b] = 0;
+    for (int b = 0; b < S::kSteps; b += S::kPack) {
+        if constexpr (S::kLPB == 1) {
 #pragma unroll
-        for (int p = 0; p < kPack; ++p) packed[b] |= static_cast<uint32_t>(__popc(m[b * kPack + p])) << (p * kFB);
-    }
-    // the masks are the bitmap: byte i of the segment's bitmap covers elements 8i .. 8i + 7
-#pragma unroll
-    for (int b = 0; b < kSteps; b += kPack) {
-        if constexpr (kLPB == 1) {
-#pragma unroll
-            for (int p = 0; p < kPack; ++p) sts_u8(bm_addr + (b + p) * 32u + lane, m[b + p]);
+            for (int p = 0; p < S::kPack; ++p) sts_u8(bm_addr + (b + p) * 32u + lane, m[b + p]);
         } else {
             // four steps' masks at a byte's distance, shifted to this lane's place in its byte; the lanes behind
             // one byte then hold four finished bytes (one per step) and share the four stores
             uint32_t four = m[b] | (m[b + 1] << 8) | (m[b + 2] << 16) | (m[b + 3] << 24);
-            four <<= kVec * (lane & (kLPB - 1));
+            four <<= S::kVec * (lane & (S::kLPB - 1));
 #pragma unroll
-            for (int o = 1; o < kLPB; o <<= 1) four |= __shfl_xor_sync(kFull, four, o);
-            if constexpr (kLPB == 2) {
+            for (int o = 1; o < S::kLPB; o <<= 1) four |= __shfl_xor_sync(kFull, four, o);
+            if constexpr (S::kLPB == 2) {
                 const uint32_t half = (lane & 1u) ? (four >> 16) : four;                 // even lane: steps b, b + 1
                 const uint32_t at   = bm_addr + (b + 2u * (lane & 1u)) * 16u + (lane >> 1);
                 sts_u8(at, half & 0xFFu);
                 sts_u8(at + 16u, (half >> 8) & 0xFFu);
             } else {
-                static_assert(kLPB == 4, "two or four lanes behind a byte");
+                static_assert(S::kLPB == 4, "two or four lanes behind a byte");
                 sts_u8(bm_addr + (b + (lane & 3u)) * 8u + (lane >> 2), (four >> (8u * (lane & 3u))) & 0xFFu);
             }
         }
     }
-    // ---- phase 2: one warp scan per batch of steps, the batches' scans side by side
-    uint32_t inc[kBatches];
+    __syncwarp();
+    if constexpr (S::kWordsPerLane == 1) {
+        word[0] = 0;
+        if (lane < static_cast<uint32_t>(S::kWords)) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(word[0]) : "r"(bm_addr + 4u * lane) : "memory");
+    } else {
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(word[0]), "=r"(word[1]) : "r"(bm_addr + 8u * lane) : "memory");
+    }
+}
+
+// (3) one warp scan per batch of steps (the counts of a batch's steps ride in the fields of one register), the
+// batches' scans side by side.  Leaves the inclusive sums in inc[], the lane's own counts in packed[]; returns
+// the number of kept elements of the segment.
+template <typename U, int kSeg>
+__device__ __forceinline__ uint32_t segment_scan(const uint32_t (&m)[Seg<U, kSeg>::kSteps], uint32_t (&inc)[Seg<U, kSeg>::kBatches],
+                                                 uint32_t (&packed)[Seg<U, kSeg>::kBatches], const uint32_t lane)
+{
+    using S = Seg<U, kSeg>;
 #pragma unroll
-    for (int b = 0; b < kBatches; ++b) inc[b] = packed[b];
+    for (int b = 0; b < S::kBatches; ++b) {
+        packed[b] = 0;
+#pragma unroll
+        for (int p = 0; p < S::kPack; ++p) packed[b] |= static_cast<uint32_t>(__popc(m[b * S::kPack + p])) << (p * S::kFB);
+        inc[b] = packed[b];
+    }
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        uint32_t u[kBatches];
+        uint32_t u[S::kBatches];
 #pragma unroll
-        for (int b = 0; b < kBatches; ++b) u[b] = __shfl_up_sync(kFull, inc[b], o);
+        for (int b = 0; b < S::kBatches; ++b) u[b] = __shfl_up_sync(kFull, inc[b], o);
 #pragma unroll
-        for (int b = 0; b < kBatches; ++b)
+        for (int b = 0; b < S::kBatches; ++b)
             if (lane >= static_cast<uint32_t>(o)) inc[b] += u[b];
     }
-    // ---- phase 3: every lane stores its surviving elements at its exclusive offset (predicated stores: no branches)
-    uint32_t out = seg_addr;                        // address of the next free packed slot (warp-uniform)
+    uint32_t cnt = 0;
 #pragma unroll
-    for (int b = 0; b < kBatches; ++b) {
+    for (int b = 0; b < S::kBatches; ++b) {
+        const uint32_t tot = __shfl_sync(kFull, inc[b], 31);
+#pragma unroll
+        for (int p = 0; p < S::kPack; ++p) cnt += (tot >> (p * S::kFB)) & S::kFieldMask;
+    }
+    return cnt;
+}
+
+// (4) every lane stores its kept elements at its exclusive offset behind `at0`, the shared-window address of the
+// segment's run in the ring of packed values [end - ring, end).  kWrap: the run crosses the ring's end.
+template <typename U, int kSeg, bool kWrap>
+__device__ __forceinline__ void segment_store(const uint4 (&q)[Seg<U, kSeg>::kSteps], const uint32_t (&m)[Seg<U, kSeg>::kSteps],
+                                              const uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t (&packed)[Seg<U, kSeg>::kBatches],
+                                              const uint32_t at0, const uint32_t end, const uint32_t ring)
+{
+    using S        = Seg<U, kSeg>;
+    uint32_t out = at0;                              // address of the step's first packed slot (warp-uniform)
+#pragma unroll
+    for (int b = 0; b < S::kBatches; ++b) {
         const uint32_t tot = __shfl_sync(kFull, inc[b], 31);
         const uint32_t exc = inc[b] - packed[b];
 #pragma unroll
-        for (int p = 0; p < kPack; ++p) {
-            uint32_t at = out + kES * ((exc >> (p * kFB)) & kFieldMask);
-#pragma unroll
-            for (int k = 0; k < kVec; ++k) sts_elem_if<U>(at, e[b * kPack + p][k], m[b * kPack + p] & (1u << k));
-            out += kES * ((tot >> (p * kFB)) & kFieldMask);
+        for (int p = 0; p < S::kPack; ++p) {
+            const uint4    &v  = q[b * S::kPack + p];
+            const uint32_t  mm = m[b * S::kPack + p];
+            uint32_t        at = out + S::kES * ((exc >> (p * S::kFB)) & S::kFieldMask);
+            wrap_addr<kWrap>(at, end, ring);
+            if constexpr (sizeof(U) == 8) {
+                sts64_if<kWrap>(at, v.x, v.y, mm & 1u, end, ring), sts64_if<kWrap>(at, v.z, v.w, mm & 2u, end, ring);
+            } else if constexpr (sizeof(U) == 4) {
+                sts32_if<kWrap>(at, v.x, mm & 1u, end, ring), sts32_if<kWrap>(at, v.y, mm & 2u, end, ring);
+                sts32_if<kWrap>(at, v.z, mm & 4u, end, ring), sts32_if<kWrap>(at, v.w, mm & 8u, end, ring);
+            } else {
+                sts16x2_if<kWrap>(at, v.x, mm & 1u, mm & 2u, end, ring), sts16x2_if<kWrap>(at, v.y, mm & 4u, mm & 8u, end, ring);
+                sts16x2_if<kWrap>(at, v.z, mm & 16u, mm & 32u, end, ring), sts16x2_if<kWrap>(at, v.w, mm & 64u, mm & 128u, end, ring);
+            }
+            out += S::kES * ((tot >> (p * S::kFB)) & S::kFieldMask);
+            wrap_addr<kWrap>(out, end, ring);
         }
     }
-    __syncwarp();
-    word = 0;
-    if (lane < static_cast<uint32_t>(kSeg / 32)) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(word) : "r"(bm_addr + 4u * lane) : "memory");
-    return (out - seg_addr) / kES;
 }
 
 // Down-cast on stash: a binary32 pattern narrowed to binary16 (CAST 1) or bfloat16 (CAST 2), round to nearest
@@ -370,23 +468,100 @@ __device__ __forceinline__ auto narrowed(const U v)
 template <int CAST, typename U>
 using Stored = std::conditional_t<CAST == 0, U, uint16_t>;
 
-// One warp copies the `cnt` packed slots of its segment to out[0..cnt): contiguous, coalesced.
-template <typename U, int CAST, bool kGuard>
-__device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, const uint32_t lane, const uint32_t cnt,
-                                                 Stored<CAST, U> *__restrict__ out, const uint64_t room)
+// The copier warps' share of a run of `cnt` packed values at src[0..cnt), element by element: warp `copier`, lane
+// `lane` takes elements copier * 32 + lane + 32 * kCopiers * i; each instruction moves 32 consecutive elements.
+template <typename U, int CAST, int kCopiers, bool kGuard>
+__device__ __forceinline__ void copy_out_elems(const U *__restrict__ src, const uint32_t first, const uint32_t cnt,
+                                               Stored<CAST, U> *__restrict__ out, const uint64_t room)
 {
-    uint32_t j = lane;
-    for (; j + 96 < cnt; j += 128) {
-        const auto v0 = narrowed<CAST>(seg[j]), v1 = narrowed<CAST>(seg[j + 32]), v2 = narrowed<CAST>(seg[j + 64]),
-                   v3 = narrowed<CAST>(seg[j + 96]);
+    constexpr uint32_t kStride = 32u * kCopiers;
+    uint32_t           j       = first;
+    for (; j + 3 * kStride < cnt; j += 4 * kStride) {
+        const auto v0 = narrowed<CAST>(src[j]), v1 = narrowed<CAST>(src[j + kStride]), v2 = narrowed<CAST>(src[j + 2 * kStride]),
+                   v3 = narrowed<CAST>(src[j + 3 * kStride]);
         if (!kGuard || j < room) out[j] = v0;
-        if (!kGuard || j + 32 < room) out[j + 32] = v1;
-        if (!kGuard || j + 64 < room) out[j + 64] = v2;
-        if (!kGuard || j + 96 < room) out[j + 96] = v3;
+        if (!kGuard || j + kStride < room) out[j + kStride] = v1;
+        if (!kGuard || j + 2 * kStride < room) out[j + 2 * kStride] = v2;
+        if (!kGuard || j + 3 * kStride < room) out[j + 3 * kStride] = v3;
     }
-    for (; j < cnt; j += 32) {
-        const auto v = narrowed<CAST>(seg[j]);
+    for (; j < cnt; j += kStride) {
+        const auto v = narrowed<CAST>(src[j]);
         if (!kGuard || j < room) out[j] = v;
+    }
+}
+
+// Words kWS .. kWS + 3 of the eight words {a, b}, shifted right by `bits` (0 or 16) into the next word: the 16-byte
+// vector that starts kWS words and bits / 8 bytes into a.
+template <int kWS>
+__device__ __forceinline__ uint4 window(const uint4 &a, const uint4 &b, const uint32_t bits)
+{
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    return make_uint4(__funnelshift_r(w[kWS], w[kWS + 1], bits), __funnelshift_r(w[kWS + 1], w[kWS + 2], bits),
+                      __funnelshift_r(w[kWS + 2], w[kWS + 3], bits), __funnelshift_r(w[kWS + 3], w[(kWS + 4) & 7], bits));
+}
+
+// The same share in 16-byte vectors: `out` is 16-byte aligned, the run starts `shift` bytes (a multiple of the
+// element size, < 16) into the 16-byte shared vector at src_vec.  A lane reads the two shared vectors its output
+// vector straddles and stores their window: 32 lanes move 512 bytes per instruction.  nvec whole vectors.
+template <int kCopiers, int kWS>
+__device__ __forceinline__ void copy_out_vecs_ws(const uint4 *__restrict__ src_vec, const uint32_t bits, const uint32_t first, const uint32_t nvec,
+                                                 uint4 *__restrict__ out)
+{
+    constexpr uint32_t kStride = 32u * kCopiers;
+    uint32_t           i       = first;
+    for (; i + kStride < nvec; i += 2 * kStride) {
+        const uint4 a0 = src_vec[i], b0 = src_vec[i + 1], a1 = src_vec[i + kStride], b1 = src_vec[i + kStride + 1];
+        out[i]           = window<kWS>(a0, b0, bits);
+        out[i + kStride] = window<kWS>(a1, b1, bits);
+    }
+    if (i < nvec) {
+        const uint4 a0 = src_vec[i], b0 = src_vec[i + 1];
+        out[i]         = window<kWS>(a0, b0, bits);
+    }
+}
+template <int kCopiers>
+__device__ __forceinline__ void copy_out_vecs(const uint4 *__restrict__ src_vec, const uint32_t shift, const uint32_t first, const uint32_t nvec,
+                                              uint4 *__restrict__ out)
+{
+    constexpr uint32_t kStride = 32u * kCopiers;
+    if (shift == 0) {
+        for (uint32_t i = first; i < nvec; i += kStride) out[i] = src_vec[i];
+        return;
+    }
+    const uint32_t bits = (shift & 2u) * 8u;
+    switch (shift >> 2) {
+    case 0: copy_out_vecs_ws<kCopiers, 0>(src_vec, bits, first, nvec, out); break;
+    case 1: copy_out_vecs_ws<kCopiers, 1>(src_vec, bits, first, nvec, out); break;
+    case 2: copy_out_vecs_ws<kCopiers, 2>(src_vec, bits, first, nvec, out); break;
+    default: copy_out_vecs_ws<kCopiers, 3>(src_vec, bits, first, nvec, out); break;
+    }
+}
+
+// One contiguous piece of a tile's run, `cnt` packed values at src (shared memory), to out[0..cnt) (global memory):
+// in 16-byte vectors where nothing stands in the way (values of the tensor's own type, room for all of them), the
+// few elements before the first and after the last whole output vector one by one.
+template <typename U, int CAST, int kCopiers, bool kGuard>
+__device__ __forceinline__ void copy_out_piece(const U *src, const uint32_t cnt, Stored<CAST, U> *out, const uint64_t room,
+                                               const uint32_t copier, const uint32_t lane)
+{
+    const uint32_t mine = copier * 32u + lane;
+    if constexpr (CAST != 0 || kGuard) {
+        copy_out_elems<U, CAST, kCopiers, kGuard>(src, mine, cnt, out, room);
+    } else {
+        constexpr uint32_t kVec = 16 / sizeof(U);
+        const uint32_t     lead = static_cast<uint32_t>((16u - (reinterpret_cast<uintptr_t>(out) & 15u)) & 15u) / sizeof(U);   // elements before the first aligned output vector
+        if (cnt < lead + 2 * kVec) {
+            copy_out_elems<U, 0, kCopiers, false>(src, mine, cnt, out, 0);
+            return;
+        }
+        const uint32_t nvec = (cnt - lead) / kVec;
+        const uint32_t done = lead + nvec * kVec;
+        if (mine < lead) out[mine] = src[mine];
+        // the tail goes to the last copier warp, the head to the first
+        if (copier == kCopiers - 1 && done + lane < cnt) out[done + lane] = src[done + lane];
+        const uintptr_t s0 = reinterpret_cast<uintptr_t>(src + lead);
+        copy_out_vecs<kCopiers>(reinterpret_cast<const uint4 *>(s0 & ~static_cast<uintptr_t>(15)), static_cast<uint32_t>(s0 & 15u), mine, nvec,
+                                reinterpret_cast<uint4 *>(out + lead));
     }
 }
 
@@ -427,6 +602,7 @@ __device__ __forceinline__ void walk_begin(Walk &w, const CompressParams<kJobs> 
 template <int kJobs>
 __device__ __forceinline__ void walk_next(Walk &w, const CompressParams<kJobs> &p, const uint32_t cta, const uint32_t G)
 {
+    if (!w.valid) return;
     ++w.j;
     if (static_cast<uint64_t>(w.v) + static_cast<uint64_t>(w.j) * G >= w.tiles) {
         ++w.k;
@@ -434,52 +610,67 @@ __device__ __forceinline__ void walk_next(Walk &w, const CompressParams<kJobs> &
     }
 }
 
+constexpr int kRec = 8;     // tiles of a CTA that can be between "counted" and "copied out" at once
+
 // U: uint64_t, uint32_t or uint16_t (the element's width).
 // FUSED: -1 for the plain compressor, else the number of the fused forward form (element type, + 4 for ReLU6).
 // CAST: 0, or the 16-bit type the copiers narrow the packed binary32 values to (1 binary16, 2 bfloat16).
 // kJobs: room for tensors in the kernel's parameters (1, or kMaxBatch for the batched forms).
-// kWarps compactor warps, kSeg elements per warp, kStages ring slots, kCopiers copier warps.
-template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kWarps, int kSeg, int kStages, int kCopiers>
-__global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32)
+// kGroups groups of kGW compactor warps (a group takes every kGroups-th tile of the CTA), kSeg elements per warp,
+// kIn slots of the ring of incoming tiles, kOutBytes of ring for the packed values, kCopiers copier warps.
+template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kGroups, int kGW, int kSeg, int kIn, int kOutBytes, int kCopiers>
+__global__ void __launch_bounds__((kGroups * kGW + kCopiers + 3) * 32)
 compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
 {
-    constexpr int kTile           = kWarps * kSeg;
+    using S                       = Seg<U, kSeg>;
+    constexpr int kWarps          = kGroups * kGW;           // compactor warps
+    constexpr int kTile           = kGW * kSeg;
     constexpr int kChunksPerTile  = kTile / BT_CHUNK_ELEMS;
     constexpr int kWarpsPerChunk  = BT_CHUNK_ELEMS / kSeg;
-    constexpr int kCompactThreads = kWarps * 32;
+    constexpr int kGroupThreads   = kGW * 32;
+    constexpr uint32_t kOutElems  = kOutBytes / sizeof(U);
+    constexpr int kMaxInFlight    = kIn - 1;                 // bulk copies outstanding per CTA
     // warp roles
-    constexpr int kFirstCopier   = kWarps;
-    constexpr int kScanWarp      = kWarps + kCopiers;       // and kScanWarp + 1
-    constexpr int kLoadWarp      = kWarps + kCopiers + 2;
-    constexpr int kSegsPerCopier = kWarps / kCopiers;
-    static_assert(kWarps % kCopiers == 0, "equal shares for the copier warps");
-    static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
+    constexpr int kFirstCopier = kWarps;
+    constexpr int kScanWarp    = kWarps + kCopiers;       // and kScanWarp + 1
+    constexpr int kLoadWarp    = kWarps + kCopiers + 2;
+    static_assert(kSeg % 32 == 0 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
     static_assert(kTile % BT_CHUNK_ELEMS == 0, "a tile holds whole chunks");
-    static_assert(kWarps <= 32, "one lane per warp count");
-    // A scan warp makes tile i ready only in its turn for tile i + 2, after that tile has been counted, so
-    // tiles i, i + 1 and i + 2 must hold slots at once: three stages are the minimum that cannot deadlock,
-    // the fourth keeps the bulk copy of the next tile in flight.
-    static_assert(kStages >= 4, "loading, compacting, awaiting its base, copying out");
+    static_assert(kGW <= 32, "one lane per warp count");
+    static_assert(kIn >= 2 && kIn > kGroups, "one tile landing while the groups read theirs");
+    // A scan warp makes tile i ready only in its turn for tile i + 2, after that tile has been counted, and a tile is
+    // counted before its packed values ask for room: so the runs of tiles i and i + 1 must fit the ring together.
+    static_assert(kOutElems >= 2 * kTile && kOutBytes % 16 == 0, "two whole tiles of packed values");
+    static_assert(kRec >= 4 && kRec > kGroups, "counted, awaiting its base (two turns), copying out");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    U *const tiles = reinterpret_cast<U *>(smem_raw);
+    U *const tiles   = reinterpret_cast<U *>(smem_raw);                           // kIn incoming tiles
+    U *const outring = tiles + static_cast<size_t>(kIn) * kTile;                  // ring of packed values
 
-    __shared__ __align__(8) uint64_t s_full[kStages];      // the bulk copy has landed            (copy engine -> compactors)
-    __shared__ __align__(8) uint64_t s_counted[kStages];   // every compactor posted its count    (compactors -> scan warp)
-    __shared__ __align__(8) uint64_t s_ready[kStages];     // base and offsets are in shared      (scan warp -> copiers)
-    __shared__ __align__(8) uint64_t s_empty[kStages];     // every copier is done with the slot  (copiers -> load warp)
-    __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
-    __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
-    __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
-    __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
+    __shared__ __align__(8) uint64_t s_full[kIn];          // the bulk copy has landed                     (copy engine -> compactors)
+    __shared__ __align__(8) uint64_t s_drained[kIn];       // every compactor has its segment in registers (compactors -> load warp)
+    __shared__ __align__(8) uint64_t s_counted[kRec];      // every compactor posted its count             (compactors -> scan warps, placer)
+    __shared__ __align__(8) uint64_t s_placed[kRec];       // the tile's run has its place in the ring     (placer -> compactors, next placer)
+    __shared__ __align__(8) uint64_t s_packed[kRec];       // every compactor stored its packed values     (compactors -> copiers)
+    __shared__ __align__(8) uint64_t s_ready[kRec];        // the tile's base is in shared                 (scan warp -> copiers)
+    __shared__ __align__(8) uint64_t s_copied[kRec];       // every copier is done with the tile's run     (copiers -> compactors)
+    __shared__ uint64_t          s_base[kRec];             // exclusive base of the tile
+    __shared__ uint32_t          s_cnt[kRec][kGW];         // packed count of each segment
+    __shared__ uint32_t          s_off[kRec][kGW];         // where each segment's run starts in the ring (elements)
+    __shared__ uint32_t          s_tot[kRec];              // packed count of the tile
+    __shared__ uint32_t          s_pos[kRec];              // where the tile's run starts in the ring (elements)
+    __shared__ uint32_t          s_end[kRec];              // elements ever put into the ring up to and including this tile
+    // what the placer of one tile hands to the placer of the next: where the next run starts, elements ever put into
+    // the ring and ever copied out of it, the oldest tile not yet seen copied out
+    __shared__ uint32_t          s_chain_pos, s_chain_alloc, s_chain_freed, s_chain_oldest;
     __shared__ __align__(16) unsigned char s_bits[kWarps][kSeg / 8];   // bitmap bytes of the segment a warp is compacting
     __shared__ volatile uint32_t s_abort;
     __shared__ volatile uint64_t s_tag;                    // this launch's tag once the first scan warp has it, else 0
     __shared__ volatile uint32_t s_met;                    // the grid has met: wave totals may be added to and read
     // Contributions to wave totals held back until then, and the total words they belong to.  This CTA's i-th tile
-    // can be counted before the meeting is over only while i <= kStages (tile kStages + 1 needs the slot of tile 1,
-    // whose base may need a total), so kStages + 1 slots, indexed by i modulo that, never collide.
-    constexpr uint32_t kHeld = kStages + 1;
+    // can be counted before the meeting is over only while i <= kRec (tile kRec + 1 needs the record of tile 1,
+    // whose base may need a total), so kRec + 1 slots, indexed by i modulo that, never collide.
+    constexpr uint32_t kHeld = kRec + 1;
     __shared__ unsigned long long s_held[kHeld];
     __shared__ uint32_t          s_held_word[kHeld];
     __shared__ uint64_t          s_arena_c0;               // arena forms: the cursor as this launch found it
@@ -501,12 +692,18 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         s_abort    = 0;
         s_tag      = 0;
         s_met      = 0;
+        s_chain_pos = 0, s_chain_alloc = 0, s_chain_freed = 0, s_chain_oldest = 0;
         for (uint32_t k = 0; k < kHeld; ++k) s_held[k] = 0;
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kIn; ++s) {
             mbar_init(&s_full[s], 1);
-            mbar_init(&s_counted[s], kWarps);
-            mbar_init(&s_ready[s], 1);
-            mbar_init(&s_empty[s], kCopiers);
+            mbar_init(&s_drained[s], kGW);
+        }
+        for (int r = 0; r < kRec; ++r) {
+            mbar_init(&s_counted[r], kGW);
+            mbar_init(&s_placed[r], 1);
+            mbar_init(&s_packed[r], kGW);
+            mbar_init(&s_ready[r], 1);
+            mbar_init(&s_copied[r], kCopiers);
         }
         fence_proxy_async();
     }
@@ -520,31 +717,30 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             Walk     w;
             walk_begin(w, p, cta, G);
             for (uint32_t it = 0; ok && w.valid; ++it, walk_next(w, p, cta, G)) {
-                if (it >= static_cast<uint32_t>(kStages)) {
-                    ok = mbar_wait(&s_empty[it % kStages], ((it / kStages) - 1) & 1u, &s_abort, wait_ns);
+                if (it >= static_cast<uint32_t>(kIn)) {
+                    ok = mbar_wait(&s_drained[it % kIn], ((it / kIn) - 1) & 1u, &s_abort, wait_ns);
                     if (!ok) break;
                 }
-                // Start-up pacing: at most two bulk copies outstanding per SM while the ring fills for the first
-                // time, as in steady state, where a copy is issued only as a slot frees.  Requesting the whole ring
-                // at once puts 33 MB in front of every other memory operation of the launch's first microseconds.
-                if (it >= 2u && it < static_cast<uint32_t>(kStages)) mbar_wait<false>(&s_full[(it - 2u) % kStages], 0, &s_abort, wait_ns);
+                // at most kMaxInFlight bulk copies outstanding: the answers to the scan warps' reads queue behind them
+                if (it >= static_cast<uint32_t>(kMaxInFlight))
+                    mbar_wait<false>(&s_full[(it - kMaxInFlight) % kIn], ((it - kMaxInFlight) / kIn) & 1u, &s_abort, wait_ns);
                 // bulk copy of the tile into its ring slot
-                const uint32_t s     = it % kStages;
+                const uint32_t s     = it % kIn;
                 const U *const src   = static_cast<const U *>(p.job[w.k].src);
                 const uint64_t first = static_cast<uint64_t>(w.tile(G)) * kTile;
                 const uint64_t left  = p.job[w.k].n - first;
                 const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
                 const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
-                fence_proxy_async();                       // the copiers' and compactors' accesses to the slot come first
+                fence_proxy_async();                       // the compactors' reads of the slot come first
                 mbar_arrive_expect_tx(&s_full[s], bytes);  // bytes == 0 simply completes the phase
                 if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
                 issued = it + 1;
             }
             // This lane stays until every bulk copy it issued has landed, whatever the other warps do (they may
             // leave early once a bounded wait has run out somewhere): the CTA never retires with a copy into its
-            // shared memory in flight.  Only the last kStages copies can still be pending; each wait is bounded.
-            for (uint32_t it = issued > static_cast<uint32_t>(kStages) ? issued - kStages : 0; it < issued; ++it)
-                mbar_wait<false>(&s_full[it % kStages], (it / kStages) & 1u, &s_abort, 20000000ull);
+            // shared memory in flight.  Only the last kIn copies can still be pending; each wait is bounded.
+            for (uint32_t it = issued > static_cast<uint32_t>(kIn) ? issued - kIn : 0; it < issued; ++it)
+                mbar_wait<false>(&s_full[it % kIn], (it / kIn) & 1u, &s_abort, 20000000ull);
         }
         return;
     }
@@ -560,7 +756,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         //       the wave of tile i -- and issue, in ONE batch of independent loads, the reads of the descriptors
         //       of that wave and of the totals of the two waves before it.
         // The loads of (b) are used a whole tile later, in (c) of the next turn, so the round trip to L2
-        // (1.3 us under load, longer than one tile) never stalls a turn for long: a turn has two tiles' time.
+        // (longer than one tile under load) never stalls a turn for long: a turn has two tiles' time.
         const uint32_t  q          = warp - kScanWarp;
         uint64_t *const wave_total = p.c.ws_total;
         uint64_t *const desc       = p.c.ws_desc;
@@ -576,7 +772,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         const uint32_t last_i = my_tiles - 1;       // every CTA has a tile: the grid is no larger than the tile count
 
         // The tag of this launch.  One warp reads the sequence number; it changes only once every CTA has arrived
-        // at the meeting, which a CTA does after this read.
+        // at the meeting (or, without one, published its count), which a CTA does after this read.
         uint64_t tag = 0;
         if (q == 0) {
             if (lane == 0) {
@@ -626,34 +822,33 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
 
         Walk cur;                                   // this warp's tile of the turn
         walk_begin(cur, p, cta, G);
-        if (q == 1 && cur.valid) walk_next(cur, p, cta, G);
-        uint32_t pk = 0, pj = 0, pv = 0;            // this warp's previous tile: tensor, wave, virtual CTA
+        if (q == 1) walk_next(cur, p, cta, G);
+        uint32_t pk = 0, pj = 0, pv = 0;            // this warp's previous tile: tensor, wave, virtual CTA,
+        uint32_t p_off = 0, p_agg = 0;              //   lane l < kGW: exclusive offset of its segment l; its count
         uint64_t waves_before = 0;                  // sum of the totals of the waves before the previous tile ...
         uint32_t waves_of     = 0xFFFFFFFFu;        // ... of this tensor
 
         for (uint32_t i = q; !failed && i <= last_i + 2; i += 2) {
             const bool has = i <= last_i;
+            uint32_t   c_off = 0, c_agg = 0;
             if (has) {
                 // ---- (a)
-                const uint32_t s = i % kStages;
-                if (!mbar_wait(&s_counted[s], (i / kStages) & 1u, &s_abort, wait_ns)) {
+                const uint32_t r = i % kRec;
+                if (!mbar_wait(&s_counted[r], (i / kRec) & 1u, &s_abort, wait_ns)) {
                     failed = true;
                     break;
                 }
-                const uint32_t c   = lane < kWarps ? s_cnt[s][lane] : 0u;
+                const uint32_t c   = lane < kGW ? s_cnt[r][lane] : 0u;
                 uint32_t       inc = c;
 #pragma unroll
-                for (int o = 1; o < kWarps; o <<= 1) {
+                for (int o = 1; o < kGW; o <<= 1) {
                     const uint32_t u = __shfl_up_sync(kFull, inc, o);
                     if (lane >= static_cast<uint32_t>(o)) inc += u;
                 }
-                const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
-                if (lane == 0) {
-                    st_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(p.job[cur.k].desc0) + cur.tile(G)), tag_w0 | agg, tag_w1 | agg);
-                    s_agg[s] = agg;
-                }
-                if (lane < kWarps) s_off[s][lane] = inc - c;
-                if (cur.tiles > G && lane == 0) add_to_total(i, p.job[cur.k].total0 + cur.j, (1ull << kCountShift) + agg);
+                c_agg = __shfl_sync(kFull, inc, kGW - 1);
+                c_off = inc - c;
+                if (lane == 0) st_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(p.job[cur.k].desc0) + cur.tile(G)), tag_w0 | c_agg, tag_w1 | c_agg);
+                if (cur.tiles > G && lane == 0) add_to_total(i, p.job[cur.k].total0 + cur.j, (1ull << kCountShift) + c_agg);
             }
             if (i >= 2) {
                 // ---- (c): this warp's previous tile, (pk, pj, pv)
@@ -691,15 +886,15 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 waves_before = (waves_of == pk ? waves_before : 0ull) + (w1 & ((1ull << kCountShift) - 1)) + (w2 & ((1ull << kCountShift) - 1));
                 waves_of     = pk;
                 const uint64_t base = waves_before + warp_sum_u64(part);
-                const uint32_t ps   = (i - 2) % kStages;
+                const uint32_t pr   = (i - 2) % kRec;
                 const uint64_t pt   = pv + static_cast<uint64_t>(pj) * G;
                 // exclusive count in front of each chunk of that tile
-                if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
+                if (lane < kGW && (lane % kWarpsPerChunk) == 0) {
                     const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
-                    if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + s_off[ps][lane];
+                    if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + p_off;
                 }
                 if (pt == jb.tiles - 1 && lane == 0) {
-                    const uint64_t nnz = base + s_agg[ps];
+                    const uint64_t nnz = base + p_agg;
                     *jb.nnz_out        = nnz;
                     __threadfence();
                     const bool aborted  = ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag;
@@ -725,10 +920,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                             *reinterpret_cast<volatile int32_t *>(jb.dev_status) = BT_ERR_TIMEOUT;
                     }
                 }
-                __syncwarp();
                 if (lane == 0) {
-                    s_base[ps] = base;
-                    mbar_arrive(&s_ready[ps]);                       // the copiers may take the tile
+                    s_base[pr] = base;
+                    mbar_arrive(&s_ready[pr]);                       // the copiers may take the tile
                 }
             }
             if (has) {
@@ -738,7 +932,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     // wave time to land, so that the reads below usually succeed at once instead of costing a second
                     // round trip.
                     __nanosleep(300);
-                } else if (!mbar_wait(&s_counted[(i + 1) % kStages], ((i + 1) / kStages) & 1u, &s_abort, wait_ns)) {
+                } else if (!mbar_wait(&s_counted[(i + 1) % kRec], ((i + 1) / kRec) & 1u, &s_abort, wait_ns)) {
                     failed = true;
                     break;
                 }
@@ -752,9 +946,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 const bool met = s_met != 0;
                 w1 = (cur.j > 0 && met) ? ld_relaxed_u64(wave_total + p.job[cur.k].total0 + (cur.j - 1)) : 0ull;
                 w2 = (cur.j > 1 && met) ? ld_relaxed_u64(wave_total + p.job[cur.k].total0 + (cur.j - 2)) : 0ull;
-                pk = cur.k, pj = cur.j, pv = cur.v;
+                pk = cur.k, pj = cur.j, pv = cur.v, p_off = c_off, p_agg = c_agg;
                 walk_next(cur, p, cta, G);
-                if (cur.valid) walk_next(cur, p, cta, G);
+                walk_next(cur, p, cta, G);
             }
         }
         if (failed && lane == 0) raise_timeout(p, &s_abort, tag);
@@ -767,9 +961,11 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         using V               = Stored<CAST, U>;
         if (copier == kCopiers - 1 && meet) {
             // The meeting: this warp has nothing to copy for the first microseconds.  It zeroes this CTA's share of
-            // the wave totals, writes the launch's tag into this CTA's arrival word and waits (bounded) until all G
-            // arrival words carry the tag: every CTA has then zeroed its share, and has read the sequence number.
-            // Then it adds what the scan warps have parked meanwhile, and CTA 0 moves the sequence number on.
+            // the wave totals and writes the launch's tag into this CTA's arrival word.  CTA 0 waits (bounded) until
+            // all G arrival words carry the tag -- every CTA has then zeroed its share, and has read the sequence
+            // number, which CTA 0 now moves on -- and writes the tag into the "go" word; the others wait for that
+            // word (one poller and one word per CTA: every CTA polling every arrival word makes a hot spot in L2
+            // that takes microseconds to cool).  Then the warp adds what the scan warps have parked meanwhile.
             uint64_t *const wave_total = p.c.ws_total;
             uint64_t *const arrive     = p.c.ws_header + kWsArriveWord;
             uint64_t        tag        = 0;
@@ -783,22 +979,40 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     __threadfence();
                     st_release_u64(arrive + cta, tag);
                 }
-                bool here[kMaxWindows];
-#pragma unroll
-                for (int k = 0; k < kMaxWindows; ++k) here[k] = lane + 32u * k >= G;
                 const uint64_t t0 = now_ns();
-                for (;;) {
-                    bool missing = false;
+                if (cta == 0) {
+                    bool here[kMaxWindows];
 #pragma unroll
-                    for (int k = 0; k < kMaxWindows; ++k) {
-                        if (!here[k]) here[k] = ld_acquire_u64(arrive + lane + 32u * k) == tag;
-                        missing |= !here[k];
+                    for (int k = 0; k < kMaxWindows; ++k) here[k] = lane + 32u * k >= G;
+                    for (;;) {
+                        bool missing = false;
+#pragma unroll
+                        for (int k = 0; k < kMaxWindows; ++k) {
+                            if (!here[k]) here[k] = ld_acquire_u64(arrive + lane + 32u * k) == tag;
+                            missing |= !here[k];
+                        }
+                        if (!__any_sync(kFull, missing)) break;
+                        if (__any_sync(kFull, s_abort != 0 || now_ns() - t0 > wait_ns)) {
+                            ok = false;
+                            break;
+                        }
                     }
-                    if (!__any_sync(kFull, missing)) break;
-                    if (__any_sync(kFull, s_abort != 0 || now_ns() - t0 > wait_ns)) {
-                        ok = false;
-                        break;
+                    if (ok && lane == 0) {
+                        __threadfence();
+                        st_release_u64(p.c.ws_header + kHdrGo, tag);
+                        red_add_u64(p.c.ws_header + kHdrSeq, 1ull);      // every CTA has read it: the next launch gets another tag
                     }
+                } else {
+                    if (lane == 0) {
+                        while (ld_acquire_u64(p.c.ws_header + kHdrGo) != tag) {
+                            if (s_abort != 0 || now_ns() - t0 > wait_ns) {
+                                ok = false;
+                                break;
+                            }
+                            __nanosleep(64);
+                        }
+                    }
+                    ok = __shfl_sync(kFull, ok ? 1 : 0, 0) != 0;
                 }
             }
             if (lane == 0) {
@@ -810,8 +1024,6 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                         const unsigned long long v = atomicExch(&s_held[k], 0ull);
                         if (v) red_add_u64(wave_total + s_held_word[k], v);
                     }
-                    // every CTA has read the sequence number: the next launch on this workspace gets another tag
-                    if (cta == 0) red_add_u64(p.c.ws_header + kHdrSeq, 1ull);
                 } else {
                     raise_timeout(p, &s_abort, tag);
                 }
@@ -821,8 +1033,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         Walk w;
         walk_begin(w, p, cta, G);
         for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
-            const uint32_t s = it % kStages;
-            if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort, wait_ns)) break;
+            const uint32_t r = it % kRec;
+            if (!mbar_wait(&s_ready[r], (it / kRec) & 1u, &s_abort, wait_ns)) break;
+            if (!mbar_wait(&s_packed[r], (it / kRec) & 1u, &s_abort, wait_ns)) break;
             V       *vals     = static_cast<V *>(p.job[w.k].values);
             uint64_t capacity = p.job[w.k].capacity;
             if (p.c.arena_cursor) {
@@ -830,38 +1043,48 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(p.job[w.k].values) + c0);
                 capacity          = c0 <= p.c.arena_bytes ? (p.c.arena_bytes - c0) / sizeof(V) : 0;
             }
-            const uint64_t base = s_base[s];
-#pragma unroll
-            for (int qq = 0; qq < kSegsPerCopier; ++qq) {
-                const uint32_t seg  = copier * kSegsPerCopier + qq;
-                const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
-                const uint32_t cnt  = s_cnt[s][seg];
-                const uint64_t dst  = base + s_off[s][seg];
-                if (dst + cnt <= capacity)
-                    copy_out_segment<U, CAST, false>(pseg, lane, cnt, vals + dst, 0);
-                else
-                    copy_out_segment<U, CAST, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
+            const uint64_t base  = s_base[r];
+            const uint32_t total = s_tot[r];
+            const uint32_t pos   = s_pos[r];
+            // the run may cross the ring's end: two pieces
+            const uint32_t head = total < kOutElems - pos ? total : kOutElems - pos;
+            if (base + total <= capacity) {
+                copy_out_piece<U, CAST, kCopiers, false>(outring + pos, head, vals + base, 0, copier, lane);
+                if (head < total) copy_out_piece<U, CAST, kCopiers, false>(outring, total - head, vals + base + head, 0, copier, lane);
+            } else {
+                const uint64_t room = base < capacity ? capacity - base : 0;
+                copy_out_piece<U, CAST, kCopiers, true>(outring + pos, head, vals + base, room, copier, lane);
+                if (head < total) copy_out_piece<U, CAST, kCopiers, true>(outring, total - head, vals + base + head, room > head ? room - head : 0, copier, lane);
             }
             __syncwarp();
-            asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
-            if (lane == 0) mbar_arrive(&s_empty[s]);
+            asm volatile("" ::: "memory");        // the copy-out stays above the release of the record
+            if (lane == 0) mbar_arrive(&s_copied[r]);
         }
         return;
     }
 
     // ---------------------------------------------------------------- compactor warps
-    const uint32_t bm_addr = smem_addr(&s_bits[warp][0]);
+    // kGroups groups of kGW warps; group g takes this CTA's tiles g, g + kGroups, ...; warp 0 of a group is the
+    // "placer" of its tiles: it gives the tile's run its place in the ring, behind the run of the tile before.
+    const uint32_t grp      = warp / kGW;
+    const uint32_t gw       = warp % kGW;
+    const uint32_t bm_addr  = smem_addr(&s_bits[warp][0]);
+    const uint32_t out_addr = smem_addr(outring);
+    const uint32_t out_end  = out_addr + kOutBytes;
+    bool           failed   = false;
     Walk           w;
     walk_begin(w, p, cta, G);
-    for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
+    for (uint32_t k = 0; k < grp; ++k) walk_next(w, p, cta, G);
+    for (uint32_t it = grp; w.valid; it += kGroups) {
         const CompressJob &jb    = p.job[w.k];
         const uint64_t     n     = jb.n;
         const uint64_t     t64   = w.tile(G);
-        const uint32_t     s     = it % kStages;
+        const uint32_t     s     = it % kIn;
+        const uint32_t     r     = it % kRec;
         U *const           tile  = tiles + static_cast<size_t>(s) * kTile;
         const uint64_t     first = t64 * kTile;
-        if (!mbar_wait(&s_full[s], (it / kStages) & 1u, &s_abort, wait_ns)) {
-            if (lane == 0) raise_timeout(p, &s_abort, s_tag);
+        if (!mbar_wait(&s_full[s], (it / kIn) & 1u, &s_abort, wait_ns)) {
+            failed = true;
             break;
         }
         if (n - first < static_cast<uint64_t>(kTile)) {
@@ -869,35 +1092,106 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             const U *const src     = static_cast<const U *>(jb.src);
             const uint32_t have    = static_cast<uint32_t>(n - first);
             const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
-            for (uint32_t e = by_bulk + tid; e < static_cast<uint32_t>(kTile); e += kCompactThreads)
+            for (uint32_t e = by_bulk + gw * 32u + lane; e < static_cast<uint32_t>(kTile); e += kGroupThreads)
                 tile[e] = (e < have) ? src[first + e] : U(0);
-            asm volatile("bar.sync %0, %1;" ::"n"(kBarWorkers), "n"(kCompactThreads) : "memory");
+            asm volatile("bar.sync %0, %1;" ::"r"(kBarWorkers + grp), "n"(kGroupThreads) : "memory");
         }
 
-        // ---- in-place compaction of this warp's segment
-        const uint64_t e0     = first + warp * kSeg;                 // first element of the segment
+        // ---- (1) the segment into registers; the slot goes back to the load warp
+        const uint64_t e0     = first + gw * kSeg;                   // first element of the segment
         uint32_t       yvalid = 0;
         U             *y      = nullptr;
         if constexpr (WRITE_Y) {
             y      = static_cast<U *>(jb.y) + e0;
             yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
         }
-        const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
-        uint32_t       run, word;
+        uint4          q[S::kSteps];
+        uint32_t       m[S::kSteps];
+        const uint32_t seg_addr = smem_addr(tile + gw * kSeg);
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, FUSED, WRITE_Y, false, kSeg>(seg_addr, bm_addr, word, lane, y, yvalid, p.c.tau);
+            segment_load<U, FUSED, WRITE_Y, false, kSeg>(seg_addr, lane, q, m, y, yvalid, p.c.tau);
         else
-            run = compact_segment<U, FUSED, WRITE_Y, true, kSeg>(seg_addr, bm_addr, word, lane, y, yvalid, p.c.tau);
-        if (lane < static_cast<uint32_t>(kSeg / 32)) {
-            const uint64_t wd = t64 * (kTile / 32) + warp * (kSeg / 32) + lane;
-            if (wd < ((n + 31) >> 5)) jb.bitmap[wd] = word;
+            segment_load<U, FUSED, WRITE_Y, true, kSeg>(seg_addr, lane, q, m, y, yvalid, p.c.tau);
+        __syncwarp();                                // the masks exist, so every lane's loads have returned
+        if (lane == 0) mbar_arrive(&s_drained[s]);
+
+        // ---- (3) count; the record of tile it - kRec must be free first
+        uint32_t inc[S::kBatches], packed[S::kBatches];
+        const uint32_t cnt = segment_scan<U, kSeg>(m, inc, packed, lane);
+        if (it >= static_cast<uint32_t>(kRec) && !mbar_wait(&s_copied[r], ((it / kRec) - 1) & 1u, &s_abort, wait_ns)) {
+            failed = true;
+            break;
         }
-        __syncwarp();
         if (lane == 0) {
-            s_cnt[s][warp] = run;
-            mbar_arrive(&s_counted[s]);                   // hand the count to the scan warp
+            s_cnt[r][gw] = cnt;
+            mbar_arrive(&s_counted[r]);                   // hand the count to the scan warp and to the placer
         }
+        // ---- (2) the bitmap, while the other warps count
+        uint32_t word[S::kWordsPerLane];
+        segment_bitmap<U, kSeg>(m, bm_addr, lane, word);
+        if (lane * S::kWordsPerLane < static_cast<uint32_t>(S::kWords)) {
+            const uint64_t wd = t64 * (kTile / 32) + gw * S::kWords + lane * S::kWordsPerLane;
+#pragma unroll
+            for (int k = 0; k < S::kWordsPerLane; ++k)
+                if (wd + k < ((n + 31) >> 5)) jb.bitmap[wd + k] = word[k];
+        }
+        if (gw == 0) {
+            // ---- the placer: the tile's run goes behind the run of the tile before it, once there is room
+            if (!mbar_wait(&s_counted[r], (it / kRec) & 1u, &s_abort, wait_ns) ||
+                (it > 0 && !mbar_wait(&s_placed[(it - 1) % kRec], ((it - 1) / kRec) & 1u, &s_abort, wait_ns))) {
+                failed = true;
+                break;
+            }
+            const uint32_t c   = lane < kGW ? s_cnt[r][lane] : 0u;
+            uint32_t       sum = c;
+#pragma unroll
+            for (int o = 1; o < kGW; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(kFull, sum, o);
+                if (lane >= static_cast<uint32_t>(o)) sum += u;
+            }
+            const uint32_t total = __shfl_sync(kFull, sum, kGW - 1);
+            uint32_t       pos = s_chain_pos, alloc = s_chain_alloc, freed = s_chain_freed, oldest = s_chain_oldest;
+            // tiles up to it - kRec have been copied out (every warp of this group waited for that above); the others
+            // are waited for as room is needed.  A record's s_end is read before the record is used again.
+            while (oldest + kRec <= it || alloc + total - freed > kOutElems) {
+                if (!mbar_wait(&s_copied[oldest % kRec], (oldest / kRec) & 1u, &s_abort, wait_ns)) {
+                    failed = true;
+                    break;
+                }
+                freed = s_end[oldest % kRec];
+                ++oldest;
+            }
+            if (failed) break;
+            if (lane < kGW) {
+                const uint32_t at = pos + (sum - c);
+                s_off[r][lane]    = at >= kOutElems ? at - kOutElems : at;
+            }
+            if (lane == 0) {
+                s_pos[r] = pos;
+                s_tot[r] = total;
+                s_end[r] = alloc + total;
+                const uint32_t next = pos + total;
+                s_chain_pos = next >= kOutElems ? next - kOutElems : next, s_chain_alloc = alloc + total, s_chain_freed = freed, s_chain_oldest = oldest;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s_placed[r]);
+        }
+        if (!mbar_wait(&s_placed[r], (it / kRec) & 1u, &s_abort, wait_ns)) {
+            failed = true;
+            break;
+        }
+        // ---- (4) the packed values into the ring
+        const uint32_t at = s_off[r][gw];
+        if (at + cnt <= kOutElems)
+            segment_store<U, kSeg, false>(q, m, inc, packed, out_addr + at * S::kES, out_end, kOutBytes);
+        else
+            segment_store<U, kSeg, true>(q, m, inc, packed, out_addr + at * S::kES, out_end, kOutBytes);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_packed[r]);         // hand the run to the copiers
+#pragma unroll
+        for (int k = 0; k < kGroups; ++k) walk_next(w, p, cta, G);
     }
+    if (failed && lane == 0) raise_timeout(p, &s_abort, s_tag);
 }
 
 // A value no other call of this process gets: a counter that starts at a salt drawn from the clock and the
@@ -948,14 +1242,14 @@ struct LaunchShape {
     }
 };
 
-template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kWarps, int kSeg, int kStages, int kCopiers>
+template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kGroups, int kGW, int kSeg, int kIn, int kOutBytes, int kCopiers>
 cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, cudaStream_t stream)
 {
-    constexpr int    kTile    = kWarps * kSeg;
-    constexpr int    kThreads = (kWarps + kCopiers + 3) * 32;
-    constexpr size_t kSmem    = static_cast<size_t>(kStages) * kTile * sizeof(U);
+    constexpr int    kTile    = kGW * kSeg;
+    constexpr int    kThreads = (kGroups * kGW + kCopiers + 3) * 32;
+    constexpr size_t kSmem    = static_cast<size_t>(kIn) * kTile * sizeof(U) + kOutBytes;
     static LaunchShape shape;   // one per instantiation
-    auto kernel = compress_kernel<U, FUSED, WRITE_Y, CAST, kJobs, kWarps, kSeg, kStages, kCopiers>;
+    auto kernel = compress_kernel<U, FUSED, WRITE_Y, CAST, kJobs, kGroups, kGW, kSeg, kIn, kOutBytes, kCopiers>;
     if (count == 0 || count > static_cast<uint32_t>(kJobs)) return cudaErrorInvalidValue;
 
     CompressParams<kJobs> p;
@@ -1002,23 +1296,17 @@ cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint
 template <typename U, int FUSED, bool WRITE_Y, int CAST = 0>
 cudaError_t launch_typed(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, cudaStream_t stream)
 {
-    // One CTA per SM, the ring takes nearly all of its shared memory.
-    //   8-byte elements: 8 compactor warps x 512 elements (32 KB tiles), 8 copiers, 7 stages;
-    //   4-byte elements: 8 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 7 stages;
-    //   2-byte elements: 16 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 6 stages.
-    // Batches (plain and ReLU forms only) run the instantiation with room for kMaxBatch tensors.
+    // One CTA per SM; the two rings take nearly all of its shared memory: 4 incoming tiles of 32 KB and 92 KB of
+    // packed values.  Two groups of 8 compactor warps (512 8-byte, 1024 4-byte or 2048 2-byte elements per warp),
+    // 4 copiers.  Batches (plain and ReLU forms only) run the instantiation with room for kMaxBatch tensors.
+    constexpr int  kSeg       = 4096 / sizeof(U);
+    constexpr int  kOut       = 92 * 1024;
     constexpr bool kBatchable = CAST == 0 && FUSED < kFusedRelu6;
     if constexpr (kBatchable) {
-        if (count > 1) {
-            if constexpr (sizeof(U) == 8) return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 8, 512, 7, 8>(c, jobs, count, workspace, stream);
-            else if constexpr (sizeof(U) == 4) return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 8, 1024, 7, 8>(c, jobs, count, workspace, stream);
-            else return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 16, 1024, 6, 8>(c, jobs, count, workspace, stream);
-        }
+        if (count > 1) return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 2, 8, kSeg, 4, kOut, 4>(c, jobs, count, workspace, stream);
     }
     if (count != 1) return cudaErrorInvalidValue;
-    if constexpr (sizeof(U) == 8) return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 8, 512, 7, 8>(c, jobs, count, workspace, stream);
-    else if constexpr (sizeof(U) == 4) return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 8, 1024, 7, 8>(c, jobs, count, workspace, stream);
-    else return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 16, 1024, 6, 8>(c, jobs, count, workspace, stream);
+    return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 2, 8, kSeg, 4, kOut, 4>(c, jobs, count, workspace, stream);
 }
 
 }  // namespace
