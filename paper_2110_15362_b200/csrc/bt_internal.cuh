@@ -11,25 +11,19 @@
 namespace bt {
 
 // ---------------------------------------------------------------- workspace layout
-// The workspace arrives with unspecified contents and is never cleared as a whole.  It holds, in 64-bit words,
+// The workspace arrives with unspecified contents and is never cleared.  It holds, in 64-bit words,
 //   a header of kWsHeaderBytes: [0] seq, the launch sequence number of this workspace; [1] abort, equal to the
-//     launch's tag once a bounded wait of that launch ran out; from kWsArriveWord on, one arrival word per CTA
-//     (the launch's tag once that CTA has zeroed its share of the wave totals: the grid's one meeting);
-//   one total per wave of tiles of every tensor of the launch (an even number of words), zeroed by the launch
-//     itself before use and read only after the meeting;
-//   one 16-byte descriptor per tile, never cleared: word 0 = (tag >> 32) << 32 | count, word 1 = (tag & 0xFFFFFFFF)
-//     << 32 | count.  A reader takes a descriptor only if both halves carry its own launch's tag and agree on
-//     the count (the two halves may be written and read separately).
+//     launch's tag once a bounded wait of that launch ran out; [8 ..] one word per tensor of the launch, equal
+//     to the tag once all tiles of that tensor have published their counts;
+//   eight words per tile (32 KB of elements): four pairs of words, each pair one 64-bit sum with half of the
+//     launch's tag in each word (bt_compress.cu has the layout).  A reader takes a pair only if both halves are
+//     those of its own launch.
 // tag = mix64(call_tag + seq * odd) | 1: call_tag comes from the host (a process-wide counter: two calls never
-// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (CTA 0 adds 1
-// once every CTA has arrived at the meeting, i.e. has read seq; a CTA that gives up adds 2^32), so replays of
+// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (its last
+// tile adds 1 once every tile has published, i.e. has read seq; a tile that gives up adds 2^32), so replays of
 // one captured launch -- same call_tag -- get different tags too.  Memory this library never wrote matches by
-// chance only: 2^-64 per word for the tag, and the repeated count on top.
-// Sized for the smallest tile: 24 bytes per 4096 elements.
-constexpr uint32_t kMaxGrid       = 160;                       // CTAs of one compress launch (32 * 5 descriptor windows)
-constexpr uint32_t kWsArriveWord  = 32;                        // first arrival word
-constexpr size_t   kWsHeaderBytes = 8 * (kWsArriveWord + kMaxGrid);
-constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;
+// chance only: 2^-64 per pair.
+constexpr size_t   kWsHeaderBytes = 512;
 constexpr uint32_t kMaxBatch      = 32;                        // tensors of one batched launch
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;             // bound of every in-kernel wait: 2 s
 
@@ -44,19 +38,13 @@ struct CompressJob {
     uint64_t   *nnz_out;
     int32_t    *dev_status;
     uint64_t    n;
-    // set by launch_compress:
-    uint32_t    tiles;      // number of tiles of the tensor
-    uint32_t    rot;        // the CTA that takes the tensor's tile 0 (tile t goes to CTA (rot + t) mod grid)
-    uint32_t    total0;     // index of the tensor's first wave-total word
-    uint32_t    desc0;      // index of the tensor's first tile descriptor
+    uint32_t    tiles;      // number of tiles (4096 elements) of the tensor; set by launch_compress
 };
 
 // What every tensor of a launch shares.
 struct CompressCommon {
-    uint64_t   *ws_header;
-    uint64_t   *ws_total;   // wave totals (set by launch_compress)
+    uint64_t   *ws_header;  // (set by launch_compress)
     uint64_t   *ws_desc;    // tile descriptors (set by launch_compress)
-    uint32_t    ws_totals;  // number of wave-total words (even; set by launch_compress)
     uint32_t    jobs;       // number of tensors
     uint64_t    call_tag;   // unique to the call (set by launch_compress)
     uint64_t    wait_ns;    // bound of every in-kernel wait (set by launch_compress)
@@ -76,9 +64,8 @@ struct CompressCommon {
 cudaError_t launch_compress(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, int dtype,
                             int fused, cudaStream_t s);
 // bytes of workspace for tensors holding `chunks` 4096-element chunks in all
-constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 16 + 24 * static_cast<size_t>(chunks); }
-// the calling thread's limit on the CTAs of one compress launch (0: none); returns the limit it replaces
-uint32_t set_compress_max_ctas(uint32_t max_ctas);
+// (64 bytes per tile, and a tile is at least one chunk)
+constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 64 * static_cast<size_t>(chunks); }
 // the bound of the compress kernels' waits for later launches of the process; returns the one it replaces
 // (reachable only from a test build of the library)
 uint64_t set_compress_wait_ns(uint64_t wait_ns);
