@@ -238,32 +238,23 @@ struct Seg {
     static_assert(kLPB == 1 || kPack == 4, "the byte assembly packs four steps");
 };
 
-// (1) the segment into registers (all loads first), the fused forward form applied, one mask per step (bit k:
-// the lane's k-th element of the step is kept, i.e. its pattern is not zero), the dense output written.  `src`
-// and `y` point at the segment's first element, `valid` is how many of its kSeg elements exist (the others
-// count as zeros).
+__device__ __forceinline__ void sts_vec(uint32_t addr, const uint4 &v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+}
+
+// (1) first pass over the segment (shared-window address seg_addr): the fused forward form applied in place (and
+// written to the dense output), one mask per step (bit k: the lane's k-th element of the step is kept, i.e. its
+// pattern is not zero).  Only the masks stay in registers.  `y` points at the segment's first element of the
+// dense output, `valid` is how many of the segment's kSeg elements exist (the others are zeros in shared memory).
 template <typename U, int FUSED, bool WRITE_Y, int kSeg>
-__device__ __forceinline__ void segment_load(const U *__restrict__ src, const uint32_t valid, const uint32_t lane, uint4 (&q)[Seg<U, kSeg>::kSteps],
-                                             uint32_t (&m)[Seg<U, kSeg>::kSteps], U *y, const float tau)
+__device__ __forceinline__ void segment_masks(const uint32_t seg_addr, const uint32_t valid, const uint32_t lane, uint32_t (&m)[Seg<U, kSeg>::kSteps],
+                                              U *y, const float tau)
 {
     using S = Seg<U, kSeg>;
-    if (valid == static_cast<uint32_t>(kSeg)) {
+    uint4 q[S::kSteps];
 #pragma unroll
-        for (int s = 0; s < S::kSteps; ++s) q[s] = ldg_vec(src + (s * 32 + lane) * S::kVec);
-    } else {
-#pragma unroll
-        for (int s = 0; s < S::kSteps; ++s) {
-            const uint32_t at = (s * 32 + lane) * S::kVec;
-            if (at + S::kVec <= valid) {
-                q[s] = ldg_vec(src + at);
-            } else {
-                Reg<U> e[S::kVec];
-#pragma unroll
-                for (int k = 0; k < S::kVec; ++k) e[k] = at + k < valid ? static_cast<Reg<U>>(src[at + k]) : Reg<U>(0);
-                q[s] = repack<U>(e);
-            }
-        }
-    }
+    for (int s = 0; s < S::kSteps; ++s) q[s] = lds_vec(seg_addr + (s * 32 + lane) * 16u);
 #pragma unroll
     for (int s = 0; s < S::kSteps; ++s) {
         if constexpr (FUSED >= 0) {
@@ -272,6 +263,7 @@ __device__ __forceinline__ void segment_load(const U *__restrict__ src, const ui
 #pragma unroll
             for (int k = 0; k < S::kVec; ++k) e[k] = fused_forward<FUSED>(e[k], tau);
             q[s] = repack<U>(e);
+            sts_vec(seg_addr + (s * 32 + lane) * 16u, q[s]);
             if constexpr (WRITE_Y) {
                 const uint32_t at = (s * 32 + lane) * S::kVec;                // first element of the vector in the segment
                 if (at + S::kVec <= valid) {
@@ -367,37 +359,45 @@ __device__ __forceinline__ void segment_scan(const uint32_t (&packed)[Seg<U, kSe
     }
 }
 
-// (4) every lane stores its kept elements at its exclusive offset behind `at0`, the shared-window address of the
-// segment's run in the staging area (kWrap: a ring [end - ring, end) whose end the run may cross; not used here).
-template <typename U, int kSeg, bool kWrap>
-__device__ __forceinline__ void segment_store(const uint4 (&q)[Seg<U, kSeg>::kSteps], const uint32_t (&m)[Seg<U, kSeg>::kSteps],
-                                              const uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t (&packed)[Seg<U, kSeg>::kBatches],
-                                              const uint32_t at0, const uint32_t end, const uint32_t ring)
+// (4) second pass: the segment is packed in place.  Every lane reads its vectors again and stores its kept
+// elements at its exclusive offset from the segment's start, with predicated instructions.  The loads of a batch
+// of steps are issued before the stores of the batch before it: a store of a batch lands below the batch's end
+// and a later batch reads at or above it, so they never meet.
+template <typename U, int kSeg>
+__device__ __forceinline__ void segment_pack(const uint32_t seg_addr, const uint32_t lane, const uint32_t (&m)[Seg<U, kSeg>::kSteps],
+                                             const uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t (&packed)[Seg<U, kSeg>::kBatches])
 {
     using S        = Seg<U, kSeg>;
-    uint32_t out = at0;                              // address of the step's first packed slot (warp-uniform)
+    uint32_t out = seg_addr;                         // address of the step's first packed slot (warp-uniform)
+    uint4    q[S::kPack], qn[S::kPack];
+#pragma unroll
+    for (int p = 0; p < S::kPack; ++p) q[p] = lds_vec(seg_addr + (p * 32 + lane) * 16u);
 #pragma unroll
     for (int b = 0; b < S::kBatches; ++b) {
+        if (b + 1 < S::kBatches) {
+#pragma unroll
+            for (int p = 0; p < S::kPack; ++p) qn[p] = lds_vec(seg_addr + (((b + 1) * S::kPack + p) * 32 + lane) * 16u);
+        }
         const uint32_t tot = __shfl_sync(kFull, inc[b], 31);
         const uint32_t exc = inc[b] - packed[b];
 #pragma unroll
         for (int p = 0; p < S::kPack; ++p) {
-            const uint4    &v  = q[b * S::kPack + p];
+            const uint4    &v  = q[p];
             const uint32_t  mm = m[b * S::kPack + p];
             uint32_t        at = out + S::kES * ((exc >> (p * S::kFB)) & S::kFieldMask);
-            wrap_addr<kWrap>(at, end, ring);
             if constexpr (sizeof(U) == 8) {
-                sts64_if<kWrap>(at, v.x, v.y, mm & 1u, end, ring), sts64_if<kWrap>(at, v.z, v.w, mm & 2u, end, ring);
+                sts64_if<false>(at, v.x, v.y, mm & 1u, 0, 0), sts64_if<false>(at, v.z, v.w, mm & 2u, 0, 0);
             } else if constexpr (sizeof(U) == 4) {
-                sts32_if<kWrap>(at, v.x, mm & 1u, end, ring), sts32_if<kWrap>(at, v.y, mm & 2u, end, ring);
-                sts32_if<kWrap>(at, v.z, mm & 4u, end, ring), sts32_if<kWrap>(at, v.w, mm & 8u, end, ring);
+                sts32_if<false>(at, v.x, mm & 1u, 0, 0), sts32_if<false>(at, v.y, mm & 2u, 0, 0);
+                sts32_if<false>(at, v.z, mm & 4u, 0, 0), sts32_if<false>(at, v.w, mm & 8u, 0, 0);
             } else {
-                sts16x2_if<kWrap>(at, v.x, mm & 1u, mm & 2u, end, ring), sts16x2_if<kWrap>(at, v.y, mm & 4u, mm & 8u, end, ring);
-                sts16x2_if<kWrap>(at, v.z, mm & 16u, mm & 32u, end, ring), sts16x2_if<kWrap>(at, v.w, mm & 64u, mm & 128u, end, ring);
+                sts16x2_if<false>(at, v.x, mm & 1u, mm & 2u, 0, 0), sts16x2_if<false>(at, v.y, mm & 4u, mm & 8u, 0, 0);
+                sts16x2_if<false>(at, v.z, mm & 16u, mm & 32u, 0, 0), sts16x2_if<false>(at, v.w, mm & 64u, mm & 128u, 0, 0);
             }
             out += S::kES * ((tot >> (p * S::kFB)) & S::kFieldMask);
-            wrap_addr<kWrap>(out, end, ring);
         }
+#pragma unroll
+        for (int p = 0; p < S::kPack; ++p) q[p] = qn[p];
     }
 }
 
@@ -558,7 +558,7 @@ struct TileShape {
     static constexpr int kSeg       = 4096 / sizeof(U);
     static constexpr int kTile      = kWarps * kSeg;
     static constexpr int kThreads   = kWarps * 32;
-    static constexpr int kMinBlocks = 4;
+    static constexpr int kMinBlocks = 6;
 };
 
 // U: uint64_t, uint32_t or uint16_t (the element's width).
@@ -578,8 +578,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     using S                      = Seg<U, kSeg>;
     using V                      = Stored<CAST, U>;
 
-    __shared__ __align__(16) U             s_stage[kTile];             // the tile's packed values
+    __shared__ __align__(128) U            s_tile[kTile];              // the tile as it lands; packed in place, segment by segment
     __shared__ __align__(16) unsigned char s_bits[kW][kSeg / 8];       // bitmap bytes of each warp's segment
+    __shared__ __align__(8) uint64_t       s_landed;                   // mbarrier: the bulk copy of the tile has landed
     __shared__ uint32_t                    s_wcnt[kW];                 // kept elements of each warp's segment
     __shared__ uint64_t                    s_tag;                      // the launch's tag
     __shared__ uint64_t                    s_excl;                     // the tile's exclusive prefix
@@ -596,36 +597,56 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     if constexpr (kJobs > 1) {
         while (t >= p.job[k].tiles) t -= p.job[k].tiles, ++k;
     }
-    const CompressJob &jb     = p.job[k];
-    const uint64_t     n      = jb.n;
-    const uint64_t     e0     = t * kTile + warp * kSeg;               // first element of this warp's segment
-    const uint32_t     valid  = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
-    uint64_t *const    desc   = p.c.ws_desc + kDescWords * static_cast<uint64_t>(blockIdx.x);
+    const CompressJob &jb    = p.job[k];
+    const uint64_t     n     = jb.n;
+    const uint64_t     first = t * kTile;                               // the tile's first element
+    const uint32_t     have  = n - first < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(n - first) : static_cast<uint32_t>(kTile);
+    const uint64_t     e0    = first + warp * kSeg;                     // first element of this warp's segment
+    const uint32_t     valid = have > warp * kSeg ? (have - warp * kSeg < static_cast<uint32_t>(kSeg) ? have - warp * kSeg : static_cast<uint32_t>(kSeg)) : 0u;
+    uint64_t *const    desc  = p.c.ws_desc + kDescWords * static_cast<uint64_t>(blockIdx.x);
+    const U *const     src   = static_cast<const U *>(jb.src) + first;
 
-    // ---- (1) the segment into registers.  The first thread also reads the workspace's sequence number (and the
-    // arena's cursor): every CTA does so before it publishes anything, and both change only after the last tile of
-    // the launch has seen a publication from every tile.
-    uint64_t seq = 0, c0 = 0;
+    // ---- the tile into shared memory: one bulk copy (whole 16-byte units; the few elements behind them and the
+    // zeros of a ragged last tile by ordinary stores).  The first thread also reads the workspace's sequence number
+    // (and the arena's cursor): every CTA does so before it publishes anything, and both change only after the last
+    // tile of the launch has seen a publication from every tile.
+    const uint32_t bytes = (have * static_cast<uint32_t>(sizeof(U))) & ~15u;
     if (tid == 0) {
-        seq = ld_relaxed_u64(p.c.ws_header + kHdrSeq);
-        if (p.c.arena_cursor) c0 = ld_relaxed_u64(p.c.arena_cursor);
+        mbar_init(&s_landed, 1);
+        fence_proxy_async();
+        mbar_arrive_expect_tx(&s_landed, bytes);
+        if (bytes) bulk_load(s_tile, src, bytes, &s_landed);
+        const uint64_t seq = ld_relaxed_u64(p.c.ws_header + kHdrSeq);
+        s_arena_c0         = p.c.arena_cursor ? ld_relaxed_u64(p.c.arena_cursor) : 0;
+        s_tag              = mix64(p.c.call_tag + seq * 0x9E3779B97F4A7C15ull) | 1ull;
+        s_failed           = 0;
     }
-    uint4    q[S::kSteps];
-    uint32_t m[S::kSteps];
-    segment_load<U, FUSED, WRITE_Y, kSeg>(static_cast<const U *>(jb.src) + e0, valid, lane, q, m, WRITE_Y ? static_cast<U *>(jb.y) + e0 : nullptr, p.c.tau);
+    if (have < static_cast<uint32_t>(kTile)) {
+        for (uint32_t e = bytes / sizeof(U) + tid; e < static_cast<uint32_t>(kTile); e += T::kThreads) s_tile[e] = e < have ? src[e] : U(0);
+    }
+    __syncthreads();                                 // the barrier is initialised; the tail is in place
+    {
+        const uint64_t t0 = now_ns();
+        while (!mbar_try_wait(&s_landed, 0)) {
+            if (now_ns() - t0 > p.c.wait_ns) {       // cannot happen unless the copy engine is stuck: leave without touching the tile
+                if (tid == 0) raise_timeout(p, s_tag);
+                return;
+            }
+        }
+    }
+
+    // ---- (1) first pass: masks (and the fused forward form)
+    const uint32_t seg_addr = smem_addr(s_tile + warp * kSeg);
+    uint32_t       m[S::kSteps];
+    segment_masks<U, FUSED, WRITE_Y, kSeg>(seg_addr, valid, lane, m, WRITE_Y ? static_cast<U *>(jb.y) + e0 : nullptr, p.c.tau);
 
     // ---- (3a) count, and out with the tile's count as early as possible: the tiles behind this one wait for it,
     // and every microsecond it is out before they ask saves them a second round trip to L2
     uint32_t       inc[S::kBatches], packed[S::kBatches];
     const uint32_t cnt = segment_count<U, kSeg>(m, packed);
     if (lane == 0) s_wcnt[warp] = cnt;
-    if (tid == 0) {
-        s_tag      = mix64(p.c.call_tag + seq * 0x9E3779B97F4A7C15ull) | 1ull;
-        s_arena_c0 = c0;
-        s_failed   = 0;
-    }
     __syncthreads();
-    // every warp: where its run starts in the staging area, and the tile's count
+    // every warp: where its run goes in the tensor's packed values relative to the tile's, and the tile's count
     uint32_t before = 0, total = 0;
 #pragma unroll
     for (int j = 0; j < kW; ++j) {
@@ -646,11 +667,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             if (wd + j < ((n + 31) >> 5)) jb.bitmap[wd + j] = word[j];
     }
 
-    // ---- (3b) the lanes' offsets
+    // ---- (3b) the lanes' offsets, (4) second pass: the segment packed in place
     segment_scan<U, kSeg>(packed, inc, lane);
-
-    // ---- (4) the packed values into the staging area
-    segment_store<U, kSeg, false>(q, m, inc, packed, smem_addr(s_stage + before), 0, 0);
+    segment_pack<U, kSeg>(seg_addr, lane, m, inc, packed);
 
     // ---- warp 0 gathers the tile's exclusive prefix.  With t = a + 64 b + 4096 c + 262144 d (digits of the tile's
     // number inside its tensor) it is the counts of the a tiles before it in its group of 64, of the b groups of 64
@@ -805,11 +824,14 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         vals               = reinterpret_cast<V *>(static_cast<unsigned char *>(jb.values) + cur);
         capacity           = cur <= p.c.arena_bytes ? (p.c.arena_bytes - cur) / sizeof(V) : 0;
     }
-    const uint64_t base = s_excl;
-    if (base + total <= capacity) {
-        copy_out_piece<U, CAST, kW, false>(s_stage, total, vals + base, 0, warp, lane);
+    // every warp copies its own run, which starts its segment
+    __syncwarp();
+    const uint64_t base = s_excl + before;
+    const U *const run  = s_tile + warp * kSeg;
+    if (base + cnt <= capacity) {
+        copy_out_piece<U, CAST, 1, false>(run, cnt, vals + base, 0, 0, lane);
     } else {
-        copy_out_piece<U, CAST, kW, true>(s_stage, total, vals + base, base < capacity ? capacity - base : 0, warp, lane);
+        copy_out_piece<U, CAST, 1, true>(run, cnt, vals + base, base < capacity ? capacity - base : 0, 0, lane);
     }
 }
 
