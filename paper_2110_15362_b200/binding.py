@@ -31,8 +31,7 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
            "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd",
            "bt_compress_narrow_arena", "bt_prune_fwd_compress_narrow_arena", "bt_decompress_widen_arena",
-           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked", "bt_batch_workspace_bytes",
-           "bt_compress_batch", "bt_relu_fwd_compress_batch")
+           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked", "bt_set_max_ctas")
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -60,6 +59,8 @@ def lib() -> ctypes.CDLL:
         u64, vp, i32, sz = ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
         L.bt_compressed_bytes.restype = sz
         L.bt_compressed_bytes.argtypes = [u64, u64, i32]
+        L.bt_set_max_ctas.restype = i32
+        L.bt_set_max_ctas.argtypes = [i32]
         L.bt_workspace_bytes.restype = sz
         L.bt_workspace_bytes.argtypes = [u64]
         L.bt_compress.restype = i32
@@ -200,6 +201,15 @@ def bt_prune_fwd_compress(x: torch.Tensor, tau: float, y_out: Optional[torch.Ten
                                      workspace.numel() * workspace.element_size(), _ptr(dev_status),
                                      _stream(stream))
     return _check("bt_prune_fwd_compress", st, check)
+
+def bt_set_max_ctas(max_ctas: int) -> int:
+    """Limits the CTAs of every later compress-family launch of the calling thread (0: no limit); returns the limit
+    it replaces."""
+    prev = lib().bt_set_max_ctas(int(max_ctas))
+    if prev < 0:
+        raise ValueError("bt_set_max_ctas: the limit must not be negative")
+    return prev
+
 
 def bt_compress_narrow(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,
                        nnz_out: torch.Tensor, workspace: torch.Tensor, dev_status: Optional[torch.Tensor] = None,

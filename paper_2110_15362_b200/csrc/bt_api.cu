@@ -142,6 +142,12 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype)
     return static_cast<size_t>(4 * ceil_div(n, 32) + nnz * static_cast<uint64_t>(es) + 8 * ceil_div(n, BT_CHUNK_ELEMS));
 }
 
+int bt_set_max_ctas(int max_ctas)
+{
+    if (max_ctas < 0) return -1;
+    return static_cast<int>(bt::set_compress_max_ctas(static_cast<uint32_t>(max_ctas)));
+}
+
 #ifdef BT_TEST_HOOKS
 // Test builds only (never the product library): the bound of every wait inside the compress kernels, so that a
 // test can make a wait run out by itself and see the kernel return BT_ERR_TIMEOUT.

@@ -1,41 +1,57 @@
-// Algorithm 1 (dense -> bitmap) and its fused forms (ReLU, activation pruning, ReLU6) as ONE pass
-// over one tensor or a batch of tensors: a single-pass stream compaction with decoupled look-back.
+// Algorithm 1 (dense -> bitmap) and its fused forms (ReLU, activation pruning, ReLU6) as ONE
+// compaction pass over one tensor or a batch of tensors: a persistent-CTA stream compaction whose
+// prefix sum rides on the wave structure of the grid.
 //
-// One CTA, one tile of 32 KB (4096 8-byte, 8192 4-byte or 16384 2-byte elements: whole chunks of the
-// prefix array), taken in the order of the block index.  The CTA's eight warps each own a segment of
-// the tile:
+// The grid is launched cooperatively with as many CTAs (G) as fit on the device at once, so all of
+// them are co-resident.  The tiles of a launch are dealt round robin: tile t of tensor k goes to CTA
+// (rot_k + t) mod G, where rot_k continues the deal of the tensor before it, so every CTA gets the
+// same share of a batch whatever the tensors' sizes.  Inside a tensor, tiles [jG, (j+1)G) form
+// "wave j"; a CTA takes at most one tile of a wave and takes its tiles in order.  The warps of a
+// CTA are specialised: one load warp, kWarps compactor warps, two scan warps, kCopiers copier warps.
 //
-//   - every lane loads its 16-byte vectors of the segment straight into registers (all of them
-//     before anything else: these loads are the kernel's bytes in flight) and keeps them there;
-//   - a kVec-bit mask per vector of the elements whose pattern is not zero (after the fused forward
-//     form, if any).  The masks ARE the bitmap: lanes that share a bitmap byte combine their bits
-//     with one or two shuffles, the bytes pass through a small staging area, and lane k stores
-//     word k of the segment -- one coalesced store per warp;
+// Compaction.  Compactor warp w owns segment w of the tile.  A lane takes one 16-byte vector of
+// the segment per step (kVec consecutive elements), so a warp covers 32 * kVec elements per step:
+//
+//   - one 16-byte shared load; a kVec-bit mask of the elements whose pattern is not zero (after
+//     the fused forward form, if any);
+//   - the masks ARE the bitmap: lanes that share a bitmap byte combine their bits with one or two
+//     shuffles and store the byte in a small staging area; at the end lane k reads word k of the
+//     segment back and the 32 words leave as one coalesced 128-byte store;
 //   - the counts of several steps ride in the fields of one register through ONE warp scan (five
-//     shuffles); the warps' counts meet in shared memory;
-//   - every lane stores its kept elements at its exclusive offset into the tile's staging area in
-//     shared memory, with predicated instructions;
-//   - meanwhile warp 0 publishes the tile's count and looks back over the tiles before it for its
-//     exclusive prefix (below); when it has it, all warps copy the staged run to
-//     values[prefix ...] in 16-byte vectors.
+//     shuffles) -- 2 steps for 2-byte, 4 steps for wider elements;
+//   - every lane stores its surviving elements, in place, at its exclusive offset behind the
+//     segment's running output position: the write position never passes the read position, and a
+//     batch's loads are issued before the stores of the batch before it.
 //
-// Prefix.  Every tile publishes its count in the workspace as soon as it is counted.  The last tile of
-// every group of 64 tiles adds up the group's counts and publishes the group's count, the last tile of
-// every group of 4096 tiles that of its group (from the 64 group counts below it), and so on.  With
-// t = a + 64 b + 4096 c + ... the exclusive prefix of tile t is the sum of a tile counts, b counts of
-// groups of 64, c counts of groups of 4096 ...: warp 0 reads them all at once, at most 63 per level, two
-// per lane.  No tile waits for another tile's PREFIX, so there is no chain of dependent round trips
-// through L2 along the tensor (a look-back over prefixes advances one window of tiles per round trip,
-// which at 8 TB/s is too slow for 32 KB tiles): a tile waits only for counts of tiles with a smaller
-// block index, which started no later than itself, and by the time it asks nearly all of them are
-// out.  The prefix restarts at every tensor of a batch.
+// Prefix.  The exclusive base of tile (tensor k, wave j, virtual CTA v) is
+//     sum of the totals of waves 0..j-1 of tensor k  +  sum of the counts of virtual CTAs 0..v-1 in wave j.
+// As soon as a tile is counted a scan warp publishes the count in a descriptor and adds it (with a
+// 1 in a counter field) to the wave's total with one fire-and-forget reduction.  About one tile
+// later -- when every CTA has published that wave -- it reads the v descriptors of its wave and the
+// now complete totals of the two waves before it in ONE batch of independent loads, and uses them a
+// tile after that.  The two scan warps alternate tiles, so that each has two tiles' time for that
+// round trip to L2.  No tile waits on another tile's base: only on counts, which never wait on
+// anything but data.
 //
-// Workspace.  It arrives with unspecified contents and is not cleared: a descriptor carries the
-// launch's 64-bit tag, half in each of its two words, and a reader takes only descriptors with its
-// own launch's tag.
+// Pipeline.  The warps of a CTA never meet at a CTA-wide barrier after the prologue; a ring slot
+// goes round through four mbarriers:
+//   full[s]     the bulk copy of the tile has landed         (copy engine -> compactors)
+//   counted[s]  every compactor has posted its count         (compactors  -> scan warps)
+//   ready[s]    base and segment offsets are in shared       (scan warp   -> copiers)
+//   empty[s]    every copier has copied its segments out     (copiers     -> load warp)
+// Copier warp c copies its segments' packed values to values[base + offset ...].
+//
+// Workspace.  It arrives with unspecified contents and is not cleared.  A tile's descriptor carries
+// the launch's 64-bit tag in both of its halves, and a reader takes only descriptors with its own
+// launch's tag; so counts are published and read from the first tile on.  Only the wave totals,
+// being sums, need zeroed words: the last copier warp of every CTA zeroes a share of them and
+// writes the launch's tag into the CTA's arrival word; when it has seen all G arrival words it
+// declares the grid met.  Until then the scan warps park their contributions to totals in shared
+// memory (the copier warp adds them afterwards) and take no total for read.
 #include <atomic>
 #include <chrono>
 #include <cstdlib>
+#include <mutex>
 #include <type_traits>
 
 #include "bt_internal.cuh"
@@ -43,10 +59,11 @@
 namespace bt {
 namespace {
 
-constexpr uint32_t kFull     = 0xFFFFFFFFu;
-constexpr int      kHdrSeq   = 0;                   // header words (64-bit): launch sequence number,
-constexpr int      kHdrAbort = 1;                   //   abort word (== the launch's tag once a wait ran out),
-constexpr int      kHdrDone  = 8;                   //   one word per tensor of the launch (== the tag once all its tiles have published)
+constexpr uint32_t kFull       = 0xFFFFFFFFu;
+constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
+constexpr int      kMaxWindows = kMaxGrid / 32;       // descriptor windows of 32 CTAs
+constexpr int      kHdrSeq     = 0;                   // header words (64-bit): launch sequence number,
+constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out)
 
 template <int kJobs>
 struct CompressParams {
@@ -68,9 +85,26 @@ __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v)
     return v;
 }
 
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
 __device__ __forceinline__ void red_add_u64(uint64_t *p, uint64_t v)
 {
     asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__device__ __forceinline__ uint64_t ld_acquire_u64(const uint64_t *p)
+{
+    uint64_t v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void st_release_u64(uint64_t *p, uint64_t v)
+{
+    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
 // A bijective mixer of 64-bit words (the finaliser of splitmix64).
@@ -84,12 +118,46 @@ __host__ __device__ __forceinline__ uint64_t mix64(uint64_t x)
     return x;
 }
 
-// 16 bytes from global memory that are read once: no line in L1
-__device__ __forceinline__ uint4 ldg_vec(const void *p)
+// Raise the abort flag (shared, and global under this launch's tag if the CTA got as far as reading it), move
+// the workspace's sequence number so that the next launch cannot take this one's words for its own, and report
+// the timeout in every tensor's status word.
+template <int kJobs>
+__device__ __noinline__ void raise_timeout(const CompressParams<kJobs> &p, volatile uint32_t *s_abort, const uint64_t tag)
 {
-    uint4 v;
-    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+    *s_abort = 1u;
+    if (tag) st_relaxed_u64(p.c.ws_header + kHdrAbort, tag);
+    red_add_u64(p.c.ws_header + kHdrSeq, 1ull << 32);
+    __threadfence();
+    for (uint32_t k = 0; k < p.c.jobs; ++k)
+        if (p.job[k].dev_status) *reinterpret_cast<volatile int32_t *>(p.job[k].dev_status) = BT_ERR_TIMEOUT;
+}
+
+// Bounded wait on an mbarrier phase.  False once the limit passed or the CTA is aborting.
+template <bool kStopOnAbort = true>
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *s_abort, const uint64_t limit_ns)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = now_ns();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((kStopOnAbort && *s_abort) || now_ns() - t0 > limit_ns) return false;
+    }
+}
+
+// The launch's tag as the first scan warp left it in shared memory (bounded wait; 0 if the CTA is aborting).
+__device__ __forceinline__ uint64_t wait_tag(volatile uint64_t *s_tag, volatile uint32_t *s_abort, const uint64_t limit_ns)
+{
+    uint64_t t = *s_tag;
+    if (t) return t;
+    const uint64_t t0 = now_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i) {
+            t = *s_tag;
+            if (t) return t;
+        }
+        if (*s_abort || now_ns() - t0 > limit_ns) return 0;
+    }
 }
 
 // register type that holds one element: 64 bits for 8-byte elements, 32 bits otherwise
@@ -238,23 +306,15 @@ struct Seg {
     static_assert(kLPB == 1 || kPack == 4, "the byte assembly packs four steps");
 };
 
-__device__ __forceinline__ void sts_vec(uint32_t addr, const uint4 &v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
-}
-
-// (1) first pass over the segment (shared-window address seg_addr): the fused forward form applied in place (and
-// written to the dense output), one mask per step (bit k: the lane's k-th element of the step is kept, i.e. its
-// pattern is not zero).  Only the masks stay in registers.  `y` points at the segment's first element of the
-// dense output, `valid` is how many of the segment's kSeg elements exist (the others are zeros in shared memory).
-template <typename U, int FUSED, bool WRITE_Y, int kSeg>
-__device__ __forceinline__ void segment_masks(const uint32_t seg_addr, const uint32_t valid, const uint32_t lane, uint32_t (&m)[Seg<U, kSeg>::kSteps],
-                                              U *y, const float tau)
+// (1) the segment into registers, the fused forward form applied, one mask per step (bit k: the lane's k-th
+// element of the step is kept, i.e. its pattern is not zero), the dense output written.
+template <typename U, int FUSED, bool WRITE_Y, bool kGuardY, int kSeg>
+__device__ __forceinline__ void segment_load(const uint32_t seg_addr, const uint32_t lane, uint4 (&q)[Seg<U, kSeg>::kSteps],
+                                             uint32_t (&m)[Seg<U, kSeg>::kSteps], U *y, const uint32_t yvalid, const float tau)
 {
     using S = Seg<U, kSeg>;
-    uint4 q[S::kSteps];
 #pragma unroll
-    for (int s = 0; s < S::kSteps; ++s) q[s] = lds_vec(seg_addr + (s * 32 + lane) * 16u);
+    for (int s = 0; s < S::kSteps; ++s) q[s] = lds_vec(seg_addr + lane * 16u + s * 512u);
 #pragma unroll
     for (int s = 0; s < S::kSteps; ++s) {
         if constexpr (FUSED >= 0) {
@@ -263,15 +323,14 @@ __device__ __forceinline__ void segment_masks(const uint32_t seg_addr, const uin
 #pragma unroll
             for (int k = 0; k < S::kVec; ++k) e[k] = fused_forward<FUSED>(e[k], tau);
             q[s] = repack<U>(e);
-            sts_vec(seg_addr + (s * 32 + lane) * 16u, q[s]);
             if constexpr (WRITE_Y) {
                 const uint32_t at = (s * 32 + lane) * S::kVec;                // first element of the vector in the segment
-                if (at + S::kVec <= valid) {
+                if (!kGuardY || at + S::kVec <= yvalid) {
                     *reinterpret_cast<uint4 *>(y + at) = q[s];
                 } else {
 #pragma unroll
                     for (int k = 0; k < S::kVec; ++k)
-                        if (at + k < valid) y[at + k] = static_cast<U>(e[k]);
+                        if (at + k < yvalid) y[at + k] = static_cast<U>(e[k]);
                 }
             }
         }
@@ -320,34 +379,21 @@ __device__ __forceinline__ void segment_bitmap(const uint32_t (&m)[Seg<U, kSeg>:
     }
 }
 
-// (3a) the lane's own counts, the counts of a batch's steps in the fields of one register; returns the number of
-// kept elements of the whole segment (the same in every lane)
+// (3) one warp scan per batch of steps (the counts of a batch's steps ride in the fields of one register), the
+// batches' scans side by side.  Leaves the inclusive sums in inc[], the lane's own counts in packed[]; returns
+// the number of kept elements of the segment.
 template <typename U, int kSeg>
-__device__ __forceinline__ uint32_t segment_count(const uint32_t (&m)[Seg<U, kSeg>::kSteps], uint32_t (&packed)[Seg<U, kSeg>::kBatches])
+__device__ __forceinline__ uint32_t segment_scan(const uint32_t (&m)[Seg<U, kSeg>::kSteps], uint32_t (&inc)[Seg<U, kSeg>::kBatches],
+                                                 uint32_t (&packed)[Seg<U, kSeg>::kBatches], const uint32_t lane)
 {
     using S = Seg<U, kSeg>;
-    uint32_t mine = 0;
 #pragma unroll
     for (int b = 0; b < S::kBatches; ++b) {
         packed[b] = 0;
 #pragma unroll
-        for (int p = 0; p < S::kPack; ++p) {
-            const uint32_t c = static_cast<uint32_t>(__popc(m[b * S::kPack + p]));
-            packed[b] |= c << (p * S::kFB);
-            mine += c;
-        }
+        for (int p = 0; p < S::kPack; ++p) packed[b] |= static_cast<uint32_t>(__popc(m[b * S::kPack + p])) << (p * S::kFB);
+        inc[b] = packed[b];
     }
-    return __reduce_add_sync(kFull, mine);
-}
-
-// (3b) one warp scan per batch of steps (the counts of a batch's steps ride in the fields of one register), the
-// batches' scans side by side.  Leaves the inclusive sums in inc[].
-template <typename U, int kSeg>
-__device__ __forceinline__ void segment_scan(const uint32_t (&packed)[Seg<U, kSeg>::kBatches], uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t lane)
-{
-    using S = Seg<U, kSeg>;
-#pragma unroll
-    for (int b = 0; b < S::kBatches; ++b) inc[b] = packed[b];
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         uint32_t u[S::kBatches];
@@ -357,47 +403,47 @@ __device__ __forceinline__ void segment_scan(const uint32_t (&packed)[Seg<U, kSe
         for (int b = 0; b < S::kBatches; ++b)
             if (lane >= static_cast<uint32_t>(o)) inc[b] += u[b];
     }
-}
-
-// (4) second pass: the segment is packed in place.  Every lane reads its vectors again and stores its kept
-// elements at its exclusive offset from the segment's start, with predicated instructions.  The loads of a batch
-// of steps are issued before the stores of the batch before it: a store of a batch lands below the batch's end
-// and a later batch reads at or above it, so they never meet.
-template <typename U, int kSeg>
-__device__ __forceinline__ void segment_pack(const uint32_t seg_addr, const uint32_t lane, const uint32_t (&m)[Seg<U, kSeg>::kSteps],
-                                             const uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t (&packed)[Seg<U, kSeg>::kBatches])
-{
-    using S        = Seg<U, kSeg>;
-    uint32_t out = seg_addr;                         // address of the step's first packed slot (warp-uniform)
-    uint4    q[S::kPack], qn[S::kPack];
-#pragma unroll
-    for (int p = 0; p < S::kPack; ++p) q[p] = lds_vec(seg_addr + (p * 32 + lane) * 16u);
+    uint32_t cnt = 0;
 #pragma unroll
     for (int b = 0; b < S::kBatches; ++b) {
-        if (b + 1 < S::kBatches) {
+        const uint32_t tot = __shfl_sync(kFull, inc[b], 31);
 #pragma unroll
-            for (int p = 0; p < S::kPack; ++p) qn[p] = lds_vec(seg_addr + (((b + 1) * S::kPack + p) * 32 + lane) * 16u);
-        }
+        for (int p = 0; p < S::kPack; ++p) cnt += (tot >> (p * S::kFB)) & S::kFieldMask;
+    }
+    return cnt;
+}
+
+// (4) every lane stores its kept elements at its exclusive offset behind `at0`, the shared-window address of the
+// segment's run in the ring of packed values [end - ring, end).  kWrap: the run crosses the ring's end.
+template <typename U, int kSeg, bool kWrap>
+__device__ __forceinline__ void segment_store(const uint4 (&q)[Seg<U, kSeg>::kSteps], const uint32_t (&m)[Seg<U, kSeg>::kSteps],
+                                              const uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t (&packed)[Seg<U, kSeg>::kBatches],
+                                              const uint32_t at0, const uint32_t end, const uint32_t ring)
+{
+    using S        = Seg<U, kSeg>;
+    uint32_t out = at0;                              // address of the step's first packed slot (warp-uniform)
+#pragma unroll
+    for (int b = 0; b < S::kBatches; ++b) {
         const uint32_t tot = __shfl_sync(kFull, inc[b], 31);
         const uint32_t exc = inc[b] - packed[b];
 #pragma unroll
         for (int p = 0; p < S::kPack; ++p) {
-            const uint4    &v  = q[p];
+            const uint4    &v  = q[b * S::kPack + p];
             const uint32_t  mm = m[b * S::kPack + p];
             uint32_t        at = out + S::kES * ((exc >> (p * S::kFB)) & S::kFieldMask);
+            wrap_addr<kWrap>(at, end, ring);
             if constexpr (sizeof(U) == 8) {
-                sts64_if<false>(at, v.x, v.y, mm & 1u, 0, 0), sts64_if<false>(at, v.z, v.w, mm & 2u, 0, 0);
+                sts64_if<kWrap>(at, v.x, v.y, mm & 1u, end, ring), sts64_if<kWrap>(at, v.z, v.w, mm & 2u, end, ring);
             } else if constexpr (sizeof(U) == 4) {
-                sts32_if<false>(at, v.x, mm & 1u, 0, 0), sts32_if<false>(at, v.y, mm & 2u, 0, 0);
-                sts32_if<false>(at, v.z, mm & 4u, 0, 0), sts32_if<false>(at, v.w, mm & 8u, 0, 0);
+                sts32_if<kWrap>(at, v.x, mm & 1u, end, ring), sts32_if<kWrap>(at, v.y, mm & 2u, end, ring);
+                sts32_if<kWrap>(at, v.z, mm & 4u, end, ring), sts32_if<kWrap>(at, v.w, mm & 8u, end, ring);
             } else {
-                sts16x2_if<false>(at, v.x, mm & 1u, mm & 2u, 0, 0), sts16x2_if<false>(at, v.y, mm & 4u, mm & 8u, 0, 0);
-                sts16x2_if<false>(at, v.z, mm & 16u, mm & 32u, 0, 0), sts16x2_if<false>(at, v.w, mm & 64u, mm & 128u, 0, 0);
+                sts16x2_if<kWrap>(at, v.x, mm & 1u, mm & 2u, end, ring), sts16x2_if<kWrap>(at, v.y, mm & 4u, mm & 8u, end, ring);
+                sts16x2_if<kWrap>(at, v.z, mm & 16u, mm & 32u, end, ring), sts16x2_if<kWrap>(at, v.w, mm & 64u, mm & 128u, end, ring);
             }
             out += S::kES * ((tot >> (p * S::kFB)) & S::kFieldMask);
+            wrap_addr<kWrap>(out, end, ring);
         }
-#pragma unroll
-        for (int p = 0; p < S::kPack; ++p) q[p] = qn[p];
     }
 }
 
@@ -517,321 +563,484 @@ __device__ __forceinline__ void copy_out_piece(const U *src, const uint32_t cnt,
     }
 }
 
-
 // ---------------------------------------------------------------------------------------------
-// A tile's descriptors: kLevels pairs of 64-bit words per tile in the workspace.  A pair holds one 64-bit sum:
-//   word 0 = (tag >> 32) << 32 | low half of the sum,   word 1 = (tag & 0xFFFFFFFF) << 32 | high half of the sum
-// Both words carry half of the launch's tag: a reader takes the pair only if both halves are those of its own
-// launch, so the two words may be written and read separately, and memory this library never wrote matches by
-// chance only (2^-64).  Pair 0 of tile t is the tile's own count.  Pair L (L >= 1) is written only by the last
-// tile of a group of 64^L tiles (t = 64^L - 1 mod 64^L, counted inside its tensor) and holds the count of that
-// whole group.
-struct TagHalves {
-    uint64_t w0, w1;
-    __device__ __forceinline__ explicit TagHalves(uint64_t tag) : w0(tag & 0xFFFFFFFF00000000ull), w1(tag << 32) {}
-    __device__ __forceinline__ bool valid(uint64_t d0, uint64_t d1) const { return ((d0 ^ w0) >> 32) == 0 && ((d1 ^ w1) >> 32) == 0; }
-    __device__ __forceinline__ static uint64_t value(uint64_t d0, uint64_t d1) { return (d0 & 0xFFFFFFFFull) | (d1 << 32); }
-    __device__ __forceinline__ void publish(uint64_t *pair, uint64_t sum) const { st_relaxed_2xu64(pair, w0 | (sum & 0xFFFFFFFFull), w1 | (sum >> 32)); }
+// The tiles of a launch in the order one CTA takes them: tensor after tensor; inside tensor k the tiles
+// v, v + G, v + 2G, ... with v = (cta - rot_k) mod G, the CTA's place in the deal of that tensor.
+struct Walk {
+    uint32_t k;       // tensor
+    uint32_t j;       // wave of the tensor; the tile is v + j * G
+    uint32_t v;       // this CTA's virtual index in the tensor
+    uint32_t tiles;   // tiles of the tensor
+    bool     valid;
+    __device__ __forceinline__ uint32_t tile(const uint32_t G) const { return v + j * G; }
 };
-constexpr int kLevels    = 4;                     // 64^4 tiles of 32 KB: more than a tensor can hold
-constexpr int kDescWords = 2 * kLevels;           // 64-bit words per tile
 
-// Raise the abort flag under this launch's tag, move the workspace's sequence number so that the next launch
-// cannot take this one's words for its own, and report the timeout in every tensor's status word.
 template <int kJobs>
-__device__ __noinline__ void raise_timeout(const CompressParams<kJobs> &p, const uint64_t tag)
+__device__ __forceinline__ void walk_seek(Walk &w, const CompressParams<kJobs> &p, const uint32_t cta, const uint32_t G)
 {
-    st_relaxed_u64(p.c.ws_header + kHdrAbort, tag);
-    red_add_u64(p.c.ws_header + kHdrSeq, 1ull << 32);
-    __threadfence();
-    for (uint32_t k = 0; k < p.c.jobs; ++k)
-        if (p.job[k].dev_status) *reinterpret_cast<volatile int32_t *>(p.job[k].dev_status) = BT_ERR_TIMEOUT;
+    while (w.k < p.c.jobs) {
+        const uint32_t rot = p.job[w.k].rot;
+        w.tiles            = p.job[w.k].tiles;
+        w.v                = cta >= rot ? cta - rot : cta + G - rot;
+        if (w.v < w.tiles) {
+            w.j     = 0;
+            w.valid = true;
+            return;
+        }
+        ++w.k;
+    }
+    w.valid = false;
+}
+template <int kJobs>
+__device__ __forceinline__ void walk_begin(Walk &w, const CompressParams<kJobs> &p, const uint32_t cta, const uint32_t G)
+{
+    w.k = 0, w.j = 0, w.v = 0, w.tiles = 0;
+    walk_seek(w, p, cta, G);
+}
+template <int kJobs>
+__device__ __forceinline__ void walk_next(Walk &w, const CompressParams<kJobs> &p, const uint32_t cta, const uint32_t G)
+{
+    ++w.j;
+    if (static_cast<uint64_t>(w.v) + static_cast<uint64_t>(w.j) * G >= w.tiles) {
+        ++w.k;
+        walk_seek(w, p, cta, G);
+    }
 }
 
-// Shape of a CTA: 8 warps, a tile of 32 KB whatever the element width (512 8-byte, 1024 4-byte or 2048 2-byte
-// elements per warp: one, two or four chunks of the prefix array per tile).  The look-back advances at most one
-// window of tiles per round trip to L2, so a tile must be worth that round trip's share of the memory bandwidth;
-// kMinBlocks CTAs per SM bound the registers (the loaded vectors of all resident CTAs are the bytes in flight).
-template <typename U>
-struct TileShape {
-    static constexpr int kWarps     = 8;
-    static constexpr int kSeg       = 4096 / sizeof(U);
-    static constexpr int kTile      = kWarps * kSeg;
-    static constexpr int kThreads   = kWarps * 32;
-    static constexpr int kMinBlocks = 6;
-};
+// A wave total: the count of all G tiles of a wave, published by the CTA that takes the wave's last tile (it reads
+// the counts of all the others for its own base anyway) as a tagged pair like a descriptor: word 0 = (tag >> 32) <<
+// 32 | low half of the sum, word 1 = (tag & 0xFFFFFFFF) << 32 | high half.
+__device__ __forceinline__ bool pair_valid(const uint64_t w0, const uint64_t w1, const uint64_t tag_w0, const uint64_t tag_w1)
+{
+    return ((w0 ^ tag_w0) >> 32) == 0 && ((w1 ^ tag_w1) >> 32) == 0;
+}
+
+constexpr int kScanWarps = 3;
 
 // U: uint64_t, uint32_t or uint16_t (the element's width).
 // FUSED: -1 for the plain compressor, else the number of the fused forward form (element type, + 4 for ReLU6).
-// CAST: 0, or the 16-bit type the packed binary32 values are narrowed to on their way out (1 binary16, 2 bfloat16).
+// CAST: 0, or the 16-bit type the copiers narrow the packed binary32 values to (1 binary16, 2 bfloat16).
 // kJobs: room for tensors in the kernel's parameters (1, or kMaxBatch for the batched forms).
-template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs>
-__global__ void __launch_bounds__(TileShape<U>::kThreads, TileShape<U>::kMinBlocks)
+// kWarps compactor warps, kSeg elements per warp, kStages ring slots, kCopiers copier warps.
+template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kWarps, int kSeg, int kStages, int kCopiers>
+__global__ void __launch_bounds__((kWarps + kCopiers + kScanWarps + 1) * 32)
 compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
 {
-    using T                      = TileShape<U>;
-    constexpr int kW             = T::kWarps;
-    constexpr int kSeg           = T::kSeg;
-    constexpr int kTile          = T::kTile;
-    constexpr int kChunksPerTile = kTile / BT_CHUNK_ELEMS;
-    constexpr int kWarpsPerChunk = BT_CHUNK_ELEMS / kSeg;
-    using S                      = Seg<U, kSeg>;
-    using V                      = Stored<CAST, U>;
+    using S                       = Seg<U, kSeg>;
+    constexpr int kTile           = kWarps * kSeg;
+    constexpr int kChunksPerTile  = kTile / BT_CHUNK_ELEMS;
+    constexpr int kWarpsPerChunk  = BT_CHUNK_ELEMS / kSeg;
+    constexpr int kCompactThreads = kWarps * 32;
+    // warp roles
+    constexpr int kFirstCopier   = kWarps;
+    constexpr int kScanWarp      = kWarps + kCopiers;       // ... kScanWarp + kScanWarps - 1
+    constexpr int kLoadWarp      = kWarps + kCopiers + kScanWarps;
+    constexpr int kSegsPerCopier = kWarps / kCopiers;
+    static_assert(kWarps % kCopiers == 0, "equal shares for the copier warps");
+    static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
+    static_assert(kTile % BT_CHUNK_ELEMS == 0, "a tile holds whole chunks");
+    static_assert(kWarps <= 32, "one lane per warp count");
+    static_assert(kStages >= 3, "loading, compacting, awaiting its base or being copied out");
 
-    __shared__ __align__(128) U            s_tile[kTile];              // the tile as it lands; packed in place, segment by segment
-    __shared__ __align__(16) unsigned char s_bits[kW][kSeg / 8];       // bitmap bytes of each warp's segment
-    __shared__ __align__(8) uint64_t       s_landed;                   // mbarrier: the bulk copy of the tile has landed
-    __shared__ uint32_t                    s_wcnt[kW];                 // kept elements of each warp's segment
-    __shared__ uint64_t                    s_tag;                      // the launch's tag
-    __shared__ uint64_t                    s_excl;                     // the tile's exclusive prefix
-    __shared__ uint64_t                    s_arena_c0;                 // arena forms: the cursor as this launch found it
-    __shared__ uint32_t                    s_failed;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    U *const tiles = reinterpret_cast<U *>(smem_raw);
+
+    __shared__ __align__(8) uint64_t s_full[kStages];      // the bulk copy has landed            (copy engine -> compactors)
+    __shared__ __align__(8) uint64_t s_counted[kStages];   // every compactor posted its count    (compactors -> scan warp)
+    __shared__ __align__(8) uint64_t s_ready[kStages];     // base and offsets are in shared      (scan warp -> copiers)
+    __shared__ __align__(8) uint64_t s_empty[kStages];     // every copier is done with the slot  (copiers -> load warp)
+    __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
+    __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
+    __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
+    __shared__ __align__(16) unsigned char s_bits[kWarps][kSeg / 8];   // bitmap bytes of the segment a warp is compacting
+    __shared__ volatile uint32_t s_abort;
+    __shared__ volatile uint64_t s_tag;                    // this launch's tag once the first scan warp has it, else 0
+    __shared__ uint64_t          s_arena_c0;               // arena forms: the cursor as this launch found it
 
     const uint32_t tid  = threadIdx.x;
     const uint32_t lane = tid & 31u;
-    const uint32_t warp = tid >> 5;
+    // broadcast from lane 0 so that the compiler knows the role branches below are warp-uniform
+    const uint32_t warp    = __shfl_sync(kFull, tid >> 5, 0);
+    const uint32_t G       = gridDim.x;
+    const uint32_t cta     = blockIdx.x;
+    const uint64_t wait_ns = p.c.wait_ns;
 
-    // which tile of which tensor: tiles are numbered tensor after tensor, in the order of the block index
-    uint32_t k = 0;
-    uint64_t t = blockIdx.x;
-    if constexpr (kJobs > 1) {
-        while (t >= p.job[k].tiles) t -= p.job[k].tiles, ++k;
-    }
-    const CompressJob &jb    = p.job[k];
-    const uint64_t     n     = jb.n;
-    const uint64_t     first = t * kTile;                               // the tile's first element
-    const uint32_t     have  = n - first < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(n - first) : static_cast<uint32_t>(kTile);
-    const uint64_t     e0    = first + warp * kSeg;                     // first element of this warp's segment
-    const uint32_t     valid = have > warp * kSeg ? (have - warp * kSeg < static_cast<uint32_t>(kSeg) ? have - warp * kSeg : static_cast<uint32_t>(kSeg)) : 0u;
-    uint64_t *const    desc  = p.c.ws_desc + kDescWords * static_cast<uint64_t>(blockIdx.x);
-    const U *const     src   = static_cast<const U *>(jb.src) + first;
-
-    // ---- the tile into shared memory: one bulk copy (whole 16-byte units; the few elements behind them and the
-    // zeros of a ragged last tile by ordinary stores).  The first thread also reads the workspace's sequence number
-    // (and the arena's cursor): every CTA does so before it publishes anything, and both change only after the last
-    // tile of the launch has seen a publication from every tile.
-    const uint32_t bytes = (have * static_cast<uint32_t>(sizeof(U))) & ~15u;
     if (tid == 0) {
-        mbar_init(&s_landed, 1);
+        // Read before the barrier below: the kernel's one update of the cursor follows the last tile's base,
+        // which needs a publication from every CTA, and a CTA publishes only after this barrier.
+        s_arena_c0 = p.c.arena_cursor ? *reinterpret_cast<const volatile uint64_t *>(p.c.arena_cursor) : 0;
+        s_abort    = 0;
+        s_tag      = 0;
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&s_full[s], 1);
+            mbar_init(&s_counted[s], kWarps);
+            mbar_init(&s_ready[s], 1);
+            mbar_init(&s_empty[s], kCopiers);
+        }
         fence_proxy_async();
-        mbar_arrive_expect_tx(&s_landed, bytes);
-        if (bytes) bulk_load(s_tile, src, bytes, &s_landed);
-        const uint64_t seq = ld_relaxed_u64(p.c.ws_header + kHdrSeq);
-        s_arena_c0         = p.c.arena_cursor ? ld_relaxed_u64(p.c.arena_cursor) : 0;
-        s_tag              = mix64(p.c.call_tag + seq * 0x9E3779B97F4A7C15ull) | 1ull;
-        s_failed           = 0;
     }
-    if (have < static_cast<uint32_t>(kTile)) {
-        for (uint32_t e = bytes / sizeof(U) + tid; e < static_cast<uint32_t>(kTile); e += T::kThreads) s_tile[e] = e < have ? src[e] : U(0);
-    }
-    __syncthreads();                                 // the barrier is initialised; the tail is in place
-    {
-        const uint64_t t0 = now_ns();
-        while (!mbar_try_wait(&s_landed, 0)) {
-            if (now_ns() - t0 > p.c.wait_ns) {       // cannot happen unless the copy engine is stuck: leave without touching the tile
-                if (tid == 0) raise_timeout(p, s_tag);
-                return;
-            }
-        }
-    }
-
-    // ---- (1) first pass: masks (and the fused forward form)
-    const uint32_t seg_addr = smem_addr(s_tile + warp * kSeg);
-    uint32_t       m[S::kSteps];
-    segment_masks<U, FUSED, WRITE_Y, kSeg>(seg_addr, valid, lane, m, WRITE_Y ? static_cast<U *>(jb.y) + e0 : nullptr, p.c.tau);
-
-    // ---- (3a) count, and out with the tile's count as early as possible: the tiles behind this one wait for it,
-    // and every microsecond it is out before they ask saves them a second round trip to L2
-    uint32_t       inc[S::kBatches], packed[S::kBatches];
-    const uint32_t cnt = segment_count<U, kSeg>(m, packed);
-    if (lane == 0) s_wcnt[warp] = cnt;
     __syncthreads();
-    // every warp: where its run goes in the tensor's packed values relative to the tile's, and the tile's count
-    uint32_t before = 0, total = 0;
-#pragma unroll
-    for (int j = 0; j < kW; ++j) {
-        const uint32_t c = s_wcnt[j];
-        before += j < static_cast<int>(warp) ? c : 0u;
-        total += c;
-    }
-    const TagHalves tag(s_tag);
-    if (tid == 0) tag.publish(desc, total);
 
-    // ---- (2) the bitmap
-    uint32_t word[S::kWordsPerLane];
-    segment_bitmap<U, kSeg>(m, smem_addr(&s_bits[warp][0]), lane, word);
-    if (lane * S::kWordsPerLane < static_cast<uint32_t>(S::kWords)) {
-        const uint64_t wd = t * (kTile / 32) + warp * S::kWords + lane * S::kWordsPerLane;
-#pragma unroll
-        for (int j = 0; j < S::kWordsPerLane; ++j)
-            if (wd + j < ((n + 31) >> 5)) jb.bitmap[wd + j] = word[j];
-    }
-
-    // ---- (3b) the lanes' offsets, (4) second pass: the segment packed in place
-    segment_scan<U, kSeg>(packed, inc, lane);
-    segment_pack<U, kSeg>(seg_addr, lane, m, inc, packed);
-
-    // ---- warp 0 gathers the tile's exclusive prefix.  With t = a + 64 b + 4096 c + 262144 d (digits of the tile's
-    // number inside its tensor) it is the counts of the a tiles before it in its group of 64, of the b groups of 64
-    // before that group in their group of 4096, of the c groups of 4096 before that one, and of the d groups of
-    // 262144 before that: at most 63 sums per level, two per lane, all read at once.  Nothing here waits for another
-    // tile's prefix -- only for counts, and for group counts that the last tile of a group forms from counts.
-    if (warp == 0) {
-        const uint64_t g0 = static_cast<uint64_t>(blockIdx.x) - t;               // the tensor's first tile
-        uint64_t       sum[kLevels];                                             // this lane's share of each level
-        bool           got[kLevels][2];
-        uint32_t       digit[kLevels];
-        {
-            uint64_t r = t;
-#pragma unroll
-            for (int L = 0; L < kLevels; ++L) digit[L] = static_cast<uint32_t>(r & 63u), r >>= 6, sum[L] = 0, got[L][0] = got[L][1] = false;
-        }
-        // group counts this tile closes: that of level L + 1 if its digits 0 .. L are all 63 -- it goes out as soon as
-        // the levels up to L are complete (it must not wait for the higher levels: they wait for other groups' counts,
-        // and a count that waits for counts is a chain again)
-        uint32_t closes = 0;
-#pragma unroll
-        for (int L = 0; L + 1 < kLevels; ++L) {
-            if (digit[L] != 63u) break;
-            closes = L + 1;
-        }
-        uint32_t published = 0;             // group counts of levels 1 .. published are out
-        bool     failed    = false;
-        uint32_t polls     = 0;
-        uint64_t t_start   = 0;
-        for (;;) {
-            uint32_t missing = 0;           // bit L: an entry of level L is not there yet
-            uint64_t span    = 1;           // tiles in an entry of the level: 64^L
-            uint64_t floor_t = t;           // the tile's number with the digits below the level cleared
-#pragma unroll
-            for (int L = 0; L < kLevels; ++L) {
-                floor_t -= static_cast<uint64_t>(digit[L]) * span;
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const uint32_t i = lane + 32u * j;                           // entry i of the level
-                    if (i < digit[L] && !got[L][j]) {
-                        // the group of 64^L tiles that starts at floor_t + i * span; its count sits with its last tile
-                        const uint64_t *d = p.c.ws_desc + kDescWords * (g0 + floor_t + (i + 1) * span - 1) + 2 * L;
-                        uint64_t        d0, d1;
-                        ld_relaxed_2xu64(d, d0, d1);
-                        if (tag.valid(d0, d1)) {
-                            got[L][j] = true;
-                            sum[L] += TagHalves::value(d0, d1);
-                        } else {
-                            missing |= 1u << L;
-                        }
-                    }
+    if (warp == kLoadWarp) {
+        // ------------------------------------------------------------ load warp (one lane)
+        if (lane == 0) {
+            bool     ok     = true;
+            uint32_t issued = 0;
+            Walk     w;
+            walk_begin(w, p, cta, G);
+            for (uint32_t it = 0; ok && w.valid; ++it, walk_next(w, p, cta, G)) {
+                if (it >= static_cast<uint32_t>(kStages)) {
+                    ok = mbar_wait(&s_empty[it % kStages], ((it / kStages) - 1) & 1u, &s_abort, wait_ns);
+                    if (!ok) break;
                 }
-                span <<= 6;
+                // Start-up pacing: at most two bulk copies outstanding per SM while the ring fills for the first
+                // time, as in steady state, where a copy is issued only as a slot frees.  Requesting the whole ring
+                // at once puts 33 MB in front of every other memory operation of the launch's first microseconds.
+                if (it >= 2u && it < static_cast<uint32_t>(kStages)) mbar_wait<false>(&s_full[(it - 2u) % kStages], 0, &s_abort, wait_ns);
+                // bulk copy of the tile into its ring slot
+                const uint32_t s     = it % kStages;
+                const U *const src   = static_cast<const U *>(p.job[w.k].src);
+                const uint64_t first = static_cast<uint64_t>(w.tile(G)) * kTile;
+                const uint64_t left  = p.job[w.k].n - first;
+                const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
+                const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
+                fence_proxy_async();                       // the copiers' and compactors' accesses to the slot come first
+                mbar_arrive_expect_tx(&s_full[s], bytes);  // bytes == 0 simply completes the phase
+                if (bytes) bulk_load(tiles + static_cast<size_t>(s) * kTile, src + first, bytes, &s_full[s]);
+                issued = it + 1;
             }
-            missing = __reduce_or_sync(kFull, missing);
-            if (published < closes) {
-                uint64_t upto = total;
+            // This lane stays until every bulk copy it issued has landed, whatever the other warps do (they may
+            // leave early once a bounded wait has run out somewhere): the CTA never retires with a copy into its
+            // shared memory in flight.  Only the last kStages copies can still be pending; each wait is bounded.
+            for (uint32_t it = issued > static_cast<uint32_t>(kStages) ? issued - kStages : 0; it < issued; ++it)
+                mbar_wait<false>(&s_full[it % kStages], (it / kStages) & 1u, &s_abort, 20000000ull);
+        }
+        return;
+    }
+
+    if (warp >= kScanWarp) {
+        // ------------------------------------------------------------ scan warps
+        // kScanWarps warps share the scan: warp q takes this CTA's tiles q, q + kScanWarps, ... (counted in the order
+        // the CTA takes them).  A warp's turn for a tile:
+        //   (a) wait until the compactors have counted the tile, publish the count;
+        //   (b) read, in ONE batch of independent loads, the descriptors of the virtual CTAs in front of this one in
+        //       the tile's wave and the totals of the waves since this warp's previous tile; repeat for what was not
+        //       there yet (CTAs do not run in step: a CTA that is ahead of the others waits here for them);
+        //   (c) base = the totals of the waves in front + the counts in front; hand the tile to the copiers; the CTA
+        //       that took the last tile of a wave publishes the wave's total.
+        // A turn is one round trip to L2 (one to three microseconds while the SM's bulk copies are in flight) and a
+        // tile takes about one, so three warps keep up.  While a warp waits in (b) it also looks out for its next
+        // tile's count and publishes it at once: other CTAs are waiting for it.
+        const uint32_t  q          = warp - kScanWarp;
+        uint64_t *const wave_total = p.c.ws_total;
+        uint64_t *const desc       = p.c.ws_desc;
+        bool            failed     = false;
+
+        // number of tiles this CTA takes
+        uint32_t my_tiles = 0;
+        for (uint32_t k = 0; k < p.c.jobs; ++k) {
+            const uint32_t rot = p.job[k].rot, t = p.job[k].tiles;
+            const uint32_t v   = cta >= rot ? cta - rot : cta + G - rot;
+            if (v < t) my_tiles += (t - v + G - 1) / G;
+        }
+
+        // The tag of this launch.  One warp reads the sequence number; it changes only once every CTA has published
+        // a count, which a CTA does after this read.
+        uint64_t tag = 0;
+        if (q == 0) {
+            if (lane == 0) {
+                const uint64_t seq = ld_relaxed_u64(p.c.ws_header + kHdrSeq);
+                tag                = mix64(p.c.call_tag + seq * 0x9E3779B97F4A7C15ull) | 1ull;
+                s_tag              = tag;
+            }
+        } else if (lane == 0) {
+            tag = wait_tag(&s_tag, &s_abort, wait_ns);
+        }
+        tag = __shfl_sync(kFull, tag, 0);
+        if (tag == 0) {
+            if (lane == 0) raise_timeout(p, &s_abort, 0);
+            return;
+        }
+        const uint64_t tag_w0 = tag & 0xFFFFFFFF00000000ull, tag_w1 = tag << 32;
+        auto valid = [&](const uint64_t w0, const uint64_t w1) {
+            return pair_valid(w0, w1, tag_w0, tag_w1) && static_cast<uint32_t>(w0) == static_cast<uint32_t>(w1);
+        };
+
+        // (a) for the tile `c` of flat index i: counts of the segments -> offsets, the tile's count published
+        struct Counted {
+            uint32_t off;      // lane l < kWarps: exclusive offset of segment l
+            uint32_t agg;      // the tile's count
+        };
+        auto publish = [&](const Walk &c, const uint32_t i) {
+            const uint32_t s   = i % kStages;
+            const uint32_t cn  = lane < kWarps ? s_cnt[s][lane] : 0u;
+            uint32_t       inc = cn;
 #pragma unroll
-                for (int L = 0; L + 1 < kLevels; ++L) {
-                    if (static_cast<uint32_t>(L) >= closes || (missing & ((2u << L) - 1u))) break;      // a level up to L is incomplete
-                    upto += warp_sum_u64(sum[L]);
-                    if (published == static_cast<uint32_t>(L)) {
-                        if (lane == 0) tag.publish(desc + 2 * (L + 1), upto);
-                        published = L + 1;
-                    }
-                }
+            for (int o = 1; o < kWarps; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(kFull, inc, o);
+                if (lane >= static_cast<uint32_t>(o)) inc += u;
             }
-            if (!missing) break;
-            __nanosleep(32);
-            if ((++polls & 63u) == 0 || p.c.wait_ns < 1000000ull) {
-                if (t_start == 0) t_start = now_ns();
-                if (__any_sync(kFull, now_ns() - t_start > p.c.wait_ns || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == s_tag)) {
+            Counted r;
+            r.agg = __shfl_sync(kFull, inc, kWarps - 1);
+            r.off = inc - cn;
+            if (lane == 0) st_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(p.job[c.k].desc0) + c.tile(G)), tag_w0 | r.agg, tag_w1 | r.agg);
+            if (lane < kWarps) s_off[s][lane] = r.off;
+            return r;
+        };
+
+        Walk cur;                                   // this warp's tile of the turn
+        walk_begin(cur, p, cta, G);
+        for (uint32_t k = 0; k < q; ++k) walk_next(cur, p, cta, G);
+        Walk     nxt = cur;                         // and its next one
+        for (int k = 0; k < kScanWarps; ++k) walk_next(nxt, p, cta, G);
+        bool     nxt_published = false;
+        Counted  nxt_counted{0, 0};
+        uint64_t waves_before = 0;                  // sum of the totals of the waves before this warp's previous tile ...
+        uint32_t waves_of     = 0xFFFFFFFFu;        // ... of this tensor
+
+        for (uint32_t i = q; !failed && i < my_tiles; i += kScanWarps) {
+            // ---- (a)
+            Counted me;
+            if (nxt_published) {
+                me = nxt_counted;
+            } else {
+                if (!mbar_wait(&s_counted[i % kStages], (i / kStages) & 1u, &s_abort, wait_ns)) {
                     failed = true;
                     break;
                 }
+                me = publish(cur, i);
             }
-        }
-        uint64_t excl = 0;
-        if (!failed) {
+            nxt_published         = false;
+            const uint32_t i_next = i + kScanWarps;
+            const bool     has_n  = i_next < my_tiles;
+
+            // ---- (b)
+            const CompressJob &jb      = p.job[cur.k];
+            const uint64_t     d_first = static_cast<uint64_t>(jb.desc0) + static_cast<uint64_t>(cur.j) * G;
+            const uint32_t     n_tot   = cur.j < static_cast<uint32_t>(kScanWarps) ? cur.j : static_cast<uint32_t>(kScanWarps);   // totals to read: waves cur.j - 1, cur.j - 2, ...
+            uint64_t           d0[kMaxWindows], d1[kMaxWindows], t0w = 0, t1w = 0;
+            bool               have[kMaxWindows], have_t = lane >= n_tot;
 #pragma unroll
-            for (int L = 0; L < kLevels; ++L) excl += warp_sum_u64(sum[L]);
-        }
-        if (lane == 0) {
-            if (failed) {
-                raise_timeout(p, s_tag);
-                s_failed = 1;
-            } else {
-                s_excl = excl;
+            for (int k = 0; k < kMaxWindows; ++k) {
+                have[k] = lane + 32u * k >= cur.v;                   // not in front of this CTA: a count of 0
+                d0[k] = d1[k] = 0;
             }
-        }
-        __syncwarp();
-        if (!failed) {
-            // exclusive count in front of each chunk of the tile
-            if (lane < static_cast<uint32_t>(kChunksPerTile)) {
-                const uint64_t ch = t * kChunksPerTile + lane;
-                uint64_t       at = excl;
-                for (uint32_t j = 0; j < lane * kWarpsPerChunk; ++j) at += s_wcnt[j];
-                if (ch < (n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = at;
+            uint32_t polls   = 0;
+            uint64_t t_start = 0;
+            for (;;) {
+                bool missing = false;
+#pragma unroll
+                for (int k = 0; k < kMaxWindows; ++k) {
+                    if (!have[k]) {
+                        ld_relaxed_2xu64(desc + 2 * (d_first + lane + 32u * k), d0[k], d1[k]);
+                        have[k] = valid(d0[k], d1[k]);
+                        missing |= !have[k];
+                    }
+                }
+                if (!have_t) {
+                    ld_relaxed_2xu64(wave_total + 2 * (static_cast<uint64_t>(jb.total0) + cur.j - 1 - lane), t0w, t1w);
+                    have_t = pair_valid(t0w, t1w, tag_w0, tag_w1);
+                    missing |= !have_t;
+                }
+                if (!__any_sync(kFull, missing)) break;
+                // meanwhile: the next tile's count, as soon as it is there
+                if (has_n && !nxt_published && mbar_try_wait(&s_counted[i_next % kStages], (i_next / kStages) & 1u, 0u)) {
+                    nxt_counted   = publish(nxt, i_next);
+                    nxt_published = true;
+                }
+                __nanosleep(200);
+                if ((++polls & 127u) == 0 || wait_ns < 1000000ull) {
+                    if (t_start == 0) t_start = now_ns();
+                    if (__any_sync(kFull, (now_ns() - t_start > wait_ns) || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)) {
+                        failed = true;
+                        break;
+                    }
+                }
             }
-            if (lane == 0 && t == jb.tiles - 1) {
-                // the tensor's last tile: the count of the tensor, the status word, the arena's cursor
-                const uint64_t incl = excl + total;
-                *jb.nnz_out         = incl;
-                uint64_t capacity   = jb.capacity;
-                bool     fits       = incl <= capacity;
+            if (failed) break;
+
+            // ---- (c)
+            uint64_t part = 0;
+#pragma unroll
+            for (int k = 0; k < kMaxWindows; ++k)
+                if (lane + 32u * k < cur.v) part += static_cast<uint32_t>(d0[k]);
+            const uint64_t in_front = warp_sum_u64(part);
+            const uint64_t totals   = warp_sum_u64(lane < n_tot ? ((t0w & 0xFFFFFFFFull) | (t1w << 32)) : 0ull);
+            waves_before            = (waves_of == cur.k ? waves_before : 0ull) + totals;
+            waves_of                = cur.k;
+            const uint64_t base     = waves_before + in_front;
+            const uint32_t s        = i % kStages;
+            const uint64_t tile     = cur.tile(G);
+            // the CTA of a wave's last tile has read the counts of all the others: the wave's total
+            if (cur.v == G - 1 && lane == 0) {
+                const uint64_t sum = in_front + me.agg;
+                st_relaxed_2xu64(wave_total + 2 * (static_cast<uint64_t>(jb.total0) + cur.j), tag_w0 | (sum & 0xFFFFFFFFull), tag_w1 | (sum >> 32));
+            }
+            // exclusive count in front of each chunk of that tile
+            if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
+                const uint64_t ch = tile * kChunksPerTile + lane / kWarpsPerChunk;
+                if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + me.off;
+            }
+            if (tile == jb.tiles - 1 && lane == 0) {
+                const uint64_t nnz = base + me.agg;
+                *jb.nnz_out        = nnz;
+                __threadfence();
+                const bool aborted  = ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag;
+                uint64_t   capacity = jb.capacity;
                 if (p.c.arena_cursor) {
-                    const uint64_t cur = s_arena_c0;
-                    capacity           = cur <= p.c.arena_bytes ? (p.c.arena_bytes - cur) / sizeof(V) : 0;
-                    fits               = incl <= capacity;
-                    if (fits) {
-                        *p.c.values_offset_out = cur;
-                        *p.c.arena_cursor      = cur + ((incl * sizeof(V) + 15) & ~15ull);
+                    // arena form: the room left behind the cursor; the cursor moves only when everything fitted
+                    const uint64_t c0 = s_arena_c0;
+                    capacity          = c0 <= p.c.arena_bytes ? (p.c.arena_bytes - c0) / sizeof(Stored<CAST, U>) : 0;
+                    if (!aborted && nnz <= capacity) {
+                        *p.c.values_offset_out = c0;
+                        *p.c.arena_cursor      = c0 + ((nnz * sizeof(Stored<CAST, U>) + 15) & ~15ull);
                     }
                 }
                 if (jb.dev_status) {
-                    *reinterpret_cast<volatile int32_t *>(jb.dev_status) = fits ? BT_OK : BT_ERR_CAPACITY;
+                    *reinterpret_cast<volatile int32_t *>(jb.dev_status) = aborted ? BT_ERR_TIMEOUT : (nnz > capacity ? BT_ERR_CAPACITY : BT_OK);
                     // a CTA that gives up from now on stores its BT_ERR_TIMEOUT after this word; one that gave
                     // up just before is seen here
                     __threadfence();
-                    if (ld_relaxed_u64(p.c.ws_header + kHdrAbort) == s_tag) *reinterpret_cast<volatile int32_t *>(jb.dev_status) = BT_ERR_TIMEOUT;
-                }
-                // Every tile of this tensor has published its count by now (the sums above cover them all).  The
-                // tensor's last tile says so in the header; the launch's last tile waits for the other tensors' words,
-                // after which every CTA has read the sequence number and the next launch gets another tag.
-                __threadfence();
-                st_relaxed_u64(p.c.ws_header + kHdrDone + k, s_tag);
-                if (k + 1 == p.c.jobs) {
-                    bool all = true;
-                    for (uint32_t kk = 0; all && kk + 1 < p.c.jobs; ++kk) {
-                        const uint64_t t0 = now_ns();
-                        while (ld_relaxed_u64(p.c.ws_header + kHdrDone + kk) != s_tag) {
-                            if (now_ns() - t0 > p.c.wait_ns) {
-                                all = false;
-                                break;
-                            }
-                            __nanosleep(100);
-                        }
-                    }
-                    red_add_u64(p.c.ws_header + kHdrSeq, all ? 1ull : 1ull << 32);
+                    if (!aborted && ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)
+                        *reinterpret_cast<volatile int32_t *>(jb.dev_status) = BT_ERR_TIMEOUT;
                 }
             }
+            if (lane == 0) {
+                s_base[s] = base;
+                mbar_arrive(&s_ready[s]);                       // the copiers may take the tile
+            }
+            if (cur.k + 1 == p.c.jobs && tile == jb.tiles - 1) {
+                // The launch's last tile.  The next launch on this workspace must get another tag, and the sequence
+                // number may move only once every CTA has read it, i.e. has published a count.  For one tensor the
+                // base above says so (it holds, through the totals, a count from every CTA).  In a batch the first G
+                // tiles of the launch are one per CTA: wait for their counts.
+                bool all = true;
+                if (p.c.jobs > 1) {
+                    bool seen[kMaxWindows];
+#pragma unroll
+                    for (int k = 0; k < kMaxWindows; ++k) seen[k] = lane + 32u * k >= G;
+                    const uint64_t t0 = now_ns();
+                    for (;;) {
+                        bool missing = false;
+#pragma unroll
+                        for (int k = 0; k < kMaxWindows; ++k) {
+                            if (!seen[k]) {
+                                uint64_t x0, x1;
+                                ld_relaxed_2xu64(desc + 2 * static_cast<uint64_t>(lane + 32u * k), x0, x1);
+                                seen[k] = valid(x0, x1);
+                                missing |= !seen[k];
+                            }
+                        }
+                        if (!__any_sync(kFull, missing)) break;
+                        if (__any_sync(kFull, now_ns() - t0 > wait_ns)) {
+                            all = false;
+                            break;
+                        }
+                        __nanosleep(200);
+                    }
+                }
+                if (lane == 0) red_add_u64(p.c.ws_header + kHdrSeq, all ? 1ull : 1ull << 32);
+            }
+            cur = nxt;
+            for (int k = 0; k < kScanWarps; ++k) walk_next(nxt, p, cta, G);
         }
+        if (failed && lane == 0) raise_timeout(p, &s_abort, tag);
+        return;
     }
-    __syncthreads();
-    if (s_failed) return;
 
-    // ---- the staged run to values[exclusive prefix ...]
-    V       *vals     = static_cast<V *>(jb.values);
-    uint64_t capacity = jb.capacity;
-    if (p.c.arena_cursor) {
-        const uint64_t cur = s_arena_c0;
-        vals               = reinterpret_cast<V *>(static_cast<unsigned char *>(jb.values) + cur);
-        capacity           = cur <= p.c.arena_bytes ? (p.c.arena_bytes - cur) / sizeof(V) : 0;
+    if (warp >= kFirstCopier) {
+        // ------------------------------------------------------------ copier warps
+        const uint32_t copier = warp - kFirstCopier;
+        using V               = Stored<CAST, U>;
+        Walk           w;
+        walk_begin(w, p, cta, G);
+        for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
+            const uint32_t s = it % kStages;
+            if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort, wait_ns)) break;
+            V       *vals     = static_cast<V *>(p.job[w.k].values);
+            uint64_t capacity = p.job[w.k].capacity;
+            if (p.c.arena_cursor) {
+                const uint64_t c0 = s_arena_c0;
+                vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(p.job[w.k].values) + c0);
+                capacity          = c0 <= p.c.arena_bytes ? (p.c.arena_bytes - c0) / sizeof(V) : 0;
+            }
+            const uint64_t base = s_base[s];
+#pragma unroll
+            for (int qq = 0; qq < kSegsPerCopier; ++qq) {
+                const uint32_t seg  = copier * kSegsPerCopier + qq;
+                const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
+                const uint32_t cnt  = s_cnt[s][seg];
+                const uint64_t dst  = base + s_off[s][seg];
+                if (dst + cnt <= capacity)
+                    copy_out_piece<U, CAST, 1, false>(pseg, cnt, vals + dst, 0, 0, lane);
+                else
+                    copy_out_piece<U, CAST, 1, true>(pseg, cnt, vals + dst, dst < capacity ? capacity - dst : 0, 0, lane);
+            }
+            __syncwarp();
+            asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
+            if (lane == 0) mbar_arrive(&s_empty[s]);
+        }
+        return;
     }
-    // every warp copies its own run, which starts its segment
-    __syncwarp();
-    const uint64_t base = s_excl + before;
-    const U *const run  = s_tile + warp * kSeg;
-    if (base + cnt <= capacity) {
-        copy_out_piece<U, CAST, 1, false>(run, cnt, vals + base, 0, 0, lane);
-    } else {
-        copy_out_piece<U, CAST, 1, true>(run, cnt, vals + base, base < capacity ? capacity - base : 0, 0, lane);
+
+    // ---------------------------------------------------------------- compactor warps
+    const uint32_t bm_addr = smem_addr(&s_bits[warp][0]);
+    Walk           w;
+    walk_begin(w, p, cta, G);
+    for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
+        const CompressJob &jb    = p.job[w.k];
+        const uint64_t     n     = jb.n;
+        const uint64_t     t64   = w.tile(G);
+        const uint32_t     s     = it % kStages;
+        U *const           tile  = tiles + static_cast<size_t>(s) * kTile;
+        const uint64_t     first = t64 * kTile;
+        if (!mbar_wait(&s_full[s], (it / kStages) & 1u, &s_abort, wait_ns)) {
+            if (lane == 0) raise_timeout(p, &s_abort, s_tag);
+            break;
+        }
+        if (n - first < static_cast<uint64_t>(kTile)) {
+            // ragged last tile: fetch what the 16-byte granular bulk copy left out, zero the rest
+            const U *const src     = static_cast<const U *>(jb.src);
+            const uint32_t have    = static_cast<uint32_t>(n - first);
+            const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
+            for (uint32_t e = by_bulk + tid; e < static_cast<uint32_t>(kTile); e += kCompactThreads)
+                tile[e] = (e < have) ? src[first + e] : U(0);
+            asm volatile("bar.sync %0, %1;" ::"n"(kBarWorkers), "n"(kCompactThreads) : "memory");
+        }
+
+        // ---- this warp's segment: into registers, counted, packed in place
+        const uint64_t e0     = first + warp * kSeg;                 // first element of the segment
+        uint32_t       yvalid = 0;
+        U             *y      = nullptr;
+        if constexpr (WRITE_Y) {
+            y      = static_cast<U *>(jb.y) + e0;
+            yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
+        }
+        const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
+        uint4          q[S::kSteps];
+        uint32_t       m[S::kSteps];
+        if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
+            segment_load<U, FUSED, WRITE_Y, false, kSeg>(seg_addr, lane, q, m, y, yvalid, p.c.tau);
+        else
+            segment_load<U, FUSED, WRITE_Y, true, kSeg>(seg_addr, lane, q, m, y, yvalid, p.c.tau);
+        uint32_t       inc[S::kBatches], packed[S::kBatches];
+        const uint32_t cnt = segment_scan<U, kSeg>(m, inc, packed, lane);
+        // the whole segment is in registers: the packed values may overwrite it from its start
+        segment_store<U, kSeg, false>(q, m, inc, packed, seg_addr, 0, 0);
+        __syncwarp();
+        if (lane == 0) {
+            s_cnt[s][warp] = cnt;
+            mbar_arrive(&s_counted[s]);                   // hand the count to the scan warps
+        }
+        // the bitmap, behind the count: nobody waits for it
+        uint32_t word[S::kWordsPerLane];
+        segment_bitmap<U, kSeg>(m, bm_addr, lane, word);
+        if (lane * S::kWordsPerLane < static_cast<uint32_t>(S::kWords)) {
+            const uint64_t wd = t64 * (kTile / 32) + warp * S::kWords + lane * S::kWordsPerLane;
+#pragma unroll
+            for (int k = 0; k < S::kWordsPerLane; ++k)
+                if (wd + k < ((n + 31) >> 5)) jb.bitmap[wd + k] = word[k];
+        }
     }
 }
 
@@ -845,47 +1054,125 @@ uint64_t next_call_tag()
     return counter.fetch_add(1, std::memory_order_relaxed);
 }
 
+// The calling thread's limit on the CTAs of one compress launch (0: none).  A cooperative launch needs all its
+// CTAs resident at once and a CTA of this kernel fills an SM, so two launches of more than half the SMs each run
+// one after the other even on different streams; a caller that keeps several launches in flight gives each a
+// share of the SMs.
+thread_local uint32_t t_max_ctas = 0;
+
 // The bound of the kernels' waits; only a test build can change it.
 std::atomic<uint64_t> g_wait_ns{kDefaultWaitNs};
 
-template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs>
-cudaError_t launch_sized(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, cudaStream_t stream)
+// Launch shape of one kernel instantiation on one device: the opt-in shared
+// memory size is set and the number of co-resident CTAs is looked up once.
+struct LaunchShape {
+    std::mutex lock;
+    int        grid_of_device[64] = {};
+    template <typename Kernel>
+    cudaError_t max_grid(Kernel kernel, int threads, size_t smem, int &grid)
+    {
+        int         dev = 0;
+        cudaError_t e   = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> g(lock);
+        if (grid_of_device[dev] == 0) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+            if (e != cudaSuccess) return e;
+            int sms = 0, per_sm = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return e;
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+            if (e != cudaSuccess) return e;
+            if (per_sm < 1 || sms < 1) return cudaErrorLaunchOutOfResources;
+            grid_of_device[dev] = sms * per_sm;
+        }
+        grid = grid_of_device[dev];
+        return cudaSuccess;
+    }
+};
+
+template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kWarps, int kSeg, int kStages, int kCopiers>
+cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, cudaStream_t stream)
 {
+    constexpr int    kTile    = kWarps * kSeg;
+    constexpr int    kThreads = (kWarps + kCopiers + kScanWarps + 1) * 32;
+    constexpr size_t kSmem    = static_cast<size_t>(kStages) * kTile * sizeof(U);
+    static LaunchShape shape;   // one per instantiation
+    auto kernel = compress_kernel<U, FUSED, WRITE_Y, CAST, kJobs, kWarps, kSeg, kStages, kCopiers>;
     if (count == 0 || count > static_cast<uint32_t>(kJobs)) return cudaErrorInvalidValue;
+
     CompressParams<kJobs> p;
-    p.c            = c;
-    uint64_t tiles = 0;
+    p.c             = c;
+    uint64_t tiles  = 0;
     for (uint32_t k = 0; k < count; ++k) {
-        p.job[k]         = jobs[k];
-        const uint64_t t = (jobs[k].n + TileShape<U>::kTile - 1) / TileShape<U>::kTile;
-        if (t == 0 || t > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-        p.job[k].tiles   = static_cast<uint32_t>(t);
+        p.job[k]            = jobs[k];
+        const uint64_t t    = (jobs[k].n + kTile - 1) / kTile;
+        if (t == 0 || t > 0xFFFFFFFFull) return cudaErrorInvalidValue;
+        p.job[k].tiles      = static_cast<uint32_t>(t);
         tiles += t;
     }
-    if (tiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;                 // one CTA per tile
+    if (tiles > 0xFFFFFFFFull) return cudaErrorInvalidValue;
     for (uint32_t k = count; k < static_cast<uint32_t>(kJobs); ++k) p.job[k] = CompressJob{};
+
+    int         max_grid = 0;
+    cudaError_t e        = shape.max_grid(kernel, kThreads, kSmem, max_grid);
+    if (e != cudaSuccess) return e;
+    if (max_grid > static_cast<int>(kMaxGrid)) max_grid = kMaxGrid;
+    if (t_max_ctas != 0 && static_cast<uint32_t>(max_grid) > t_max_ctas) max_grid = static_cast<int>(t_max_ctas);
+    const uint32_t grid = tiles < static_cast<uint64_t>(max_grid) ? static_cast<uint32_t>(tiles) : static_cast<uint32_t>(max_grid);
+
+    // the deal: tile t of tensor k goes to CTA (rot_k + t) mod grid; wave totals and descriptors tensor after tensor
+    uint64_t dealt = 0, totals = 0;
+    for (uint32_t k = 0; k < count; ++k) {
+        p.job[k].rot    = static_cast<uint32_t>(dealt % grid);
+        p.job[k].total0 = static_cast<uint32_t>(totals);
+        p.job[k].desc0  = static_cast<uint32_t>(dealt);
+        dealt += p.job[k].tiles;
+        totals += (p.job[k].tiles + grid - 1) / grid;
+    }
     p.c.jobs      = count;
+    p.c.ws_totals = static_cast<uint32_t>(2 * totals);              // a pair of words per wave
     p.c.ws_header = static_cast<uint64_t *>(workspace);
-    p.c.ws_desc   = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + kWsHeaderBytes);
+    p.c.ws_total  = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + kWsHeaderBytes);
+    p.c.ws_desc   = p.c.ws_total + p.c.ws_totals;
     p.c.call_tag  = next_call_tag();
     p.c.wait_ns   = g_wait_ns.load(std::memory_order_relaxed);
-    compress_kernel<U, FUSED, WRITE_Y, CAST, kJobs><<<static_cast<unsigned>(tiles), TileShape<U>::kThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    // cooperative launch: the runtime guarantees that all `grid` CTAs are resident together
+    void *params[] = {&p};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(kernel), dim3(grid), dim3(kThreads), params, kSmem, stream);
 }
 
 template <typename U, int FUSED, bool WRITE_Y, int CAST = 0>
 cudaError_t launch_typed(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, cudaStream_t stream)
 {
-    // batches (plain and ReLU forms only) run the instantiation with room for kMaxBatch tensors
+    // One CTA per SM, the ring takes nearly all of its shared memory.
+    //   8-byte elements: 8 compactor warps x 512 elements (32 KB tiles), 8 copiers, 7 stages;
+    //   4-byte elements: 8 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 7 stages;
+    //   2-byte elements: 16 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 6 stages.
+    // Batches (plain and ReLU forms only) run the instantiation with room for kMaxBatch tensors.
     constexpr bool kBatchable = CAST == 0 && FUSED < kFusedRelu6;
     if constexpr (kBatchable) {
-        if (count > 1) return launch_sized<U, FUSED, WRITE_Y, CAST, kMaxBatch>(c, jobs, count, workspace, stream);
+        if (count > 1) {
+            if constexpr (sizeof(U) == 8) return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 8, 512, 7, 8>(c, jobs, count, workspace, stream);
+            else if constexpr (sizeof(U) == 4) return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 8, 1024, 7, 8>(c, jobs, count, workspace, stream);
+            else return launch_shaped<U, FUSED, WRITE_Y, CAST, kMaxBatch, 16, 1024, 6, 8>(c, jobs, count, workspace, stream);
+        }
     }
     if (count != 1) return cudaErrorInvalidValue;
-    return launch_sized<U, FUSED, WRITE_Y, CAST, 1>(c, jobs, count, workspace, stream);
+    if constexpr (sizeof(U) == 8) return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 8, 512, 7, 8>(c, jobs, count, workspace, stream);
+    else if constexpr (sizeof(U) == 4) return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 8, 1024, 7, 8>(c, jobs, count, workspace, stream);
+    else return launch_shaped<U, FUSED, WRITE_Y, CAST, 1, 16, 1024, 6, 8>(c, jobs, count, workspace, stream);
 }
 
 }  // namespace
+
+uint32_t set_compress_max_ctas(uint32_t max_ctas)
+{
+    const uint32_t before = t_max_ctas;
+    t_max_ctas            = max_ctas;
+    return before;
+}
 
 uint64_t set_compress_wait_ns(uint64_t wait_ns) { return g_wait_ns.exchange(wait_ns, std::memory_order_relaxed); }
 

@@ -13,17 +13,20 @@ namespace bt {
 // ---------------------------------------------------------------- workspace layout
 // The workspace arrives with unspecified contents and is never cleared.  It holds, in 64-bit words,
 //   a header of kWsHeaderBytes: [0] seq, the launch sequence number of this workspace; [1] abort, equal to the
-//     launch's tag once a bounded wait of that launch ran out; [8 ..] one word per tensor of the launch, equal
-//     to the tag once all tiles of that tensor have published their counts;
-//   eight words per tile (32 KB of elements): four pairs of words, each pair one 64-bit sum with half of the
-//     launch's tag in each word (bt_compress.cu has the layout).  A reader takes a pair only if both halves are
-//     those of its own launch.
+//     launch's tag once a bounded wait of that launch ran out;
+//   one pair of words per wave of tiles of every tensor of the launch: the wave's total;
+//   one pair of words per tile: the tile's count.
+// Each word of a pair carries half of the launch's 64-bit tag, and a reader takes a pair only if both halves are
+// those of its own launch (bt_compress.cu has the layouts), so stale or never-written words are simply "not yet
+// published" and the two words may be written and read separately.
 // tag = mix64(call_tag + seq * odd) | 1: call_tag comes from the host (a process-wide counter: two calls never
-// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (its last
-// tile adds 1 once every tile has published, i.e. has read seq; a tile that gives up adds 2^32), so replays of
-// one captured launch -- same call_tag -- get different tags too.  Memory this library never wrote matches by
-// chance only: 2^-64 per pair.
-constexpr size_t   kWsHeaderBytes = 512;
+// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (the CTA of
+// its last tile adds 1 once every CTA has published a count, i.e. has read seq; a CTA that gives up adds 2^32),
+// so replays of one captured launch -- same call_tag -- get different tags too.  Memory this library never wrote
+// matches by chance only: 2^-64 per pair.
+// Sized for the smallest tile (4096 elements): 32 bytes per 4096 elements.
+constexpr uint32_t kMaxGrid       = 160;                       // CTAs of one compress launch (32 * 5 descriptor windows)
+constexpr size_t   kWsHeaderBytes = 256;
 constexpr uint32_t kMaxBatch      = 32;                        // tensors of one batched launch
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;             // bound of every in-kernel wait: 2 s
 
@@ -38,13 +41,19 @@ struct CompressJob {
     uint64_t   *nnz_out;
     int32_t    *dev_status;
     uint64_t    n;
-    uint32_t    tiles;      // number of tiles (4096 elements) of the tensor; set by launch_compress
+    // set by launch_compress:
+    uint32_t    tiles;      // number of tiles of the tensor
+    uint32_t    rot;        // the CTA that takes the tensor's tile 0 (tile t goes to CTA (rot + t) mod grid)
+    uint32_t    total0;     // index of the tensor's first wave-total word
+    uint32_t    desc0;      // index of the tensor's first tile descriptor
 };
 
 // What every tensor of a launch shares.
 struct CompressCommon {
-    uint64_t   *ws_header;  // (set by launch_compress)
+    uint64_t   *ws_header;
+    uint64_t   *ws_total;   // wave totals (set by launch_compress)
     uint64_t   *ws_desc;    // tile descriptors (set by launch_compress)
+    uint32_t    ws_totals;  // number of wave-total words (two per wave; set by launch_compress)
     uint32_t    jobs;       // number of tensors
     uint64_t    call_tag;   // unique to the call (set by launch_compress)
     uint64_t    wait_ns;    // bound of every in-kernel wait (set by launch_compress)
@@ -64,8 +73,9 @@ struct CompressCommon {
 cudaError_t launch_compress(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, int dtype,
                             int fused, cudaStream_t s);
 // bytes of workspace for tensors holding `chunks` 4096-element chunks in all
-// (64 bytes per tile, and a tile is at least one chunk)
-constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 64 * static_cast<size_t>(chunks); }
+constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 32 * static_cast<size_t>(chunks); }
+// the calling thread's limit on the CTAs of one compress launch (0: none); returns the limit it replaces
+uint32_t set_compress_max_ctas(uint32_t max_ctas);
 // the bound of the compress kernels' waits for later launches of the process; returns the one it replaces
 // (reachable only from a test build of the library)
 uint64_t set_compress_wait_ns(uint64_t wait_ns);
