@@ -63,7 +63,10 @@ constexpr uint32_t kFull       = 0xFFFFFFFFu;
 constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
 constexpr int      kMaxWindows = kMaxGrid / 32;       // descriptor windows of 32 CTAs
 constexpr int      kHdrSeq     = 0;                   // header words (64-bit): launch sequence number,
-constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out)
+constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out),
+constexpr int      kHdrGo      = 2;                   //   go word (== the launch's tag once every CTA has arrived at the meeting)
+constexpr int      kCountShift = 40;                  // wave total word: (tiles added << 40) | sum of counts
+constexpr uint32_t kDirect     = 4;                   // waves of a tensor whose bases come from descriptors alone
 
 template <int kJobs>
 struct CompressParams {
@@ -132,15 +135,22 @@ __device__ __noinline__ void raise_timeout(const CompressParams<kJobs> &p, volat
         if (p.job[k].dev_status) *reinterpret_cast<volatile int32_t *>(p.job[k].dev_status) = BT_ERR_TIMEOUT;
 }
 
-// Bounded wait on an mbarrier phase.  False once the limit passed or the CTA is aborting.
-template <bool kStopOnAbort = true>
+// Bounded wait on an mbarrier phase.  False once the limit passed or the CTA is aborting.  A warp that waits
+// sleeps kSleepNs between probes: a probe loop without it takes a third of the SM's issue slots from the warps
+// that work (the hardware holds a probing thread only for some tens of cycles), and the clock and the abort
+// flag are looked at every 64 probes only.
+template <bool kStopOnAbort = true, unsigned kSleepNs = 100>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *s_abort, const uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = now_ns();
-    for (;;) {
+    uint64_t t0 = 0;
+    for (uint32_t probes = 1;; ++probes) {
+        __nanosleep(kSleepNs);
         if (mbar_try_wait(bar, parity)) return true;
-        if ((kStopOnAbort && *s_abort) || now_ns() - t0 > limit_ns) return false;
+        if ((probes & 63u) == 0 || limit_ns < 1000000ull) {
+            if (t0 == 0) t0 = now_ns();
+            if ((kStopOnAbort && *s_abort) || now_ns() - t0 > limit_ns) return false;
+        }
     }
 }
 
@@ -247,41 +257,36 @@ __device__ __forceinline__ uint32_t vec_mask(const uint4 &q)
     return m;
 }
 
-// if (cond) { store the element at addr; addr += its size; } as predicated instructions (a branch per element
-// costs more than the element's other work); with kWrap, addr then wraps from `end` back by `ring` bytes
-template <bool kWrap>
-__device__ __forceinline__ void wrap_addr(uint32_t &addr, const uint32_t end, const uint32_t ring)
+// The kept elements of one 16-byte vector, stored one behind the other from `addr` on, which moves past them:
+// per element a test of its pattern, a predicated store and a predicated add (a branch per element costs more
+// than the element's other work).
+template <typename U>
+__device__ __forceinline__ void sts_kept(uint32_t &addr, const uint4 &v)
 {
-    if constexpr (kWrap) addr = addr >= end ? addr - ring : addr;
-}
-template <bool kWrap>
-__device__ __forceinline__ void sts32_if(uint32_t &addr, uint32_t x, uint32_t cond, const uint32_t end, const uint32_t ring)
-{
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t}" : "+r"(addr) : "r"(x), "r"(cond));
-    wrap_addr<kWrap>(addr, end, ring);
-}
-template <bool kWrap>
-__device__ __forceinline__ void sts64_if(uint32_t &addr, uint32_t lo, uint32_t hi, uint32_t cond, const uint32_t end, const uint32_t ring)
-{
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\t@p st.shared.v2.u32 [%0], {%1, %2};\n\t@p add.u32 %0, %0, 8;\n\t}" : "+r"(addr) : "r"(lo), "r"(hi), "r"(cond));
-    wrap_addr<kWrap>(addr, end, ring);
-}
-// the two 16-bit elements of a word, each under its own condition
-template <bool kWrap>
-__device__ __forceinline__ void sts16x2_if(uint32_t &addr, uint32_t x, uint32_t cond_lo, uint32_t cond_hi, const uint32_t end, const uint32_t ring)
-{
-    if constexpr (!kWrap) {
+    if constexpr (sizeof(U) == 8) {
         asm volatile(
-            "{\n\t.reg .pred p, q;\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\t"
-            "setp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], l;\n\t@p add.u32 %0, %0, 2;\n\t"
-            "setp.ne.u32 q, %3, 0;\n\t@q st.shared.u16 [%0], h;\n\t@q add.u32 %0, %0, 2;\n\t}"
+            "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+            "or.b32 t, %1, %2;\n\tsetp.ne.u32 p, t, 0;\n\t@p st.shared.v2.u32 [%0], {%1, %2};\n\t@p add.u32 %0, %0, 8;\n\t"
+            "or.b32 t, %3, %4;\n\tsetp.ne.u32 p, t, 0;\n\t@p st.shared.v2.u32 [%0], {%3, %4};\n\t@p add.u32 %0, %0, 8;\n\t}"
             : "+r"(addr)
-            : "r"(x), "r"(cond_lo), "r"(cond_hi));
+            : "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+    } else if constexpr (sizeof(U) == 4) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.u32 p, %1, 0;\n\t@p st.shared.u32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t"
+            "setp.ne.u32 p, %2, 0;\n\t@p st.shared.u32 [%0], %2;\n\t@p add.u32 %0, %0, 4;\n\t"
+            "setp.ne.u32 p, %3, 0;\n\t@p st.shared.u32 [%0], %3;\n\t@p add.u32 %0, %0, 4;\n\t"
+            "setp.ne.u32 p, %4, 0;\n\t@p st.shared.u32 [%0], %4;\n\t@p add.u32 %0, %0, 4;\n\t}"
+            : "+r"(addr)
+            : "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
     } else {
-        asm volatile("{\n\t.reg .pred p;\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], l;\n\t@p add.u32 %0, %0, 2;\n\t}" : "+r"(addr) : "r"(x), "r"(cond_lo));
-        wrap_addr<true>(addr, end, ring);
-        asm volatile("{\n\t.reg .pred p;\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tsetp.ne.u32 p, %2, 0;\n\t@p st.shared.u16 [%0], h;\n\t@p add.u32 %0, %0, 2;\n\t}" : "+r"(addr) : "r"(x), "r"(cond_hi));
-        wrap_addr<true>(addr, end, ring);
+#define BT_STS_HALVES(X)                                                                                                  \
+    "mov.b32 {l, h}, " X ";\n\tand.b32 t, " X ", 0xFFFF;\n\tsetp.ne.u32 p, t, 0;\n\t@p st.shared.u16 [%0], l;\n\t@p add.u32 %0, %0, 2;\n\t" \
+    "setp.gt.u32 p, " X ", 0xFFFF;\n\t@p st.shared.u16 [%0], h;\n\t@p add.u32 %0, %0, 2;\n\t"
+        asm volatile("{\n\t.reg .pred p;\n\t.reg .b16 l, h;\n\t.reg .b32 t;\n\t" BT_STS_HALVES("%1") BT_STS_HALVES("%2") BT_STS_HALVES("%3") BT_STS_HALVES("%4") "}"
+                     : "+r"(addr)
+                     : "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+#undef BT_STS_HALVES
     }
 }
 
@@ -413,12 +418,11 @@ __device__ __forceinline__ uint32_t segment_scan(const uint32_t (&m)[Seg<U, kSeg
     return cnt;
 }
 
-// (4) every lane stores its kept elements at its exclusive offset behind `at0`, the shared-window address of the
-// segment's run in the ring of packed values [end - ring, end).  kWrap: the run crosses the ring's end.
-template <typename U, int kSeg, bool kWrap>
-__device__ __forceinline__ void segment_store(const uint4 (&q)[Seg<U, kSeg>::kSteps], const uint32_t (&m)[Seg<U, kSeg>::kSteps],
-                                              const uint32_t (&inc)[Seg<U, kSeg>::kBatches], const uint32_t (&packed)[Seg<U, kSeg>::kBatches],
-                                              const uint32_t at0, const uint32_t end, const uint32_t ring)
+// (4) every lane stores its kept elements at its exclusive offset behind `at0`, the shared-window address where
+// the segment's packed run starts.
+template <typename U, int kSeg>
+__device__ __forceinline__ void segment_store(const uint4 (&q)[Seg<U, kSeg>::kSteps], const uint32_t (&inc)[Seg<U, kSeg>::kBatches],
+                                              const uint32_t (&packed)[Seg<U, kSeg>::kBatches], const uint32_t at0)
 {
     using S        = Seg<U, kSeg>;
     uint32_t out = at0;                              // address of the step's first packed slot (warp-uniform)
@@ -428,21 +432,9 @@ __device__ __forceinline__ void segment_store(const uint4 (&q)[Seg<U, kSeg>::kSt
         const uint32_t exc = inc[b] - packed[b];
 #pragma unroll
         for (int p = 0; p < S::kPack; ++p) {
-            const uint4    &v  = q[b * S::kPack + p];
-            const uint32_t  mm = m[b * S::kPack + p];
-            uint32_t        at = out + S::kES * ((exc >> (p * S::kFB)) & S::kFieldMask);
-            wrap_addr<kWrap>(at, end, ring);
-            if constexpr (sizeof(U) == 8) {
-                sts64_if<kWrap>(at, v.x, v.y, mm & 1u, end, ring), sts64_if<kWrap>(at, v.z, v.w, mm & 2u, end, ring);
-            } else if constexpr (sizeof(U) == 4) {
-                sts32_if<kWrap>(at, v.x, mm & 1u, end, ring), sts32_if<kWrap>(at, v.y, mm & 2u, end, ring);
-                sts32_if<kWrap>(at, v.z, mm & 4u, end, ring), sts32_if<kWrap>(at, v.w, mm & 8u, end, ring);
-            } else {
-                sts16x2_if<kWrap>(at, v.x, mm & 1u, mm & 2u, end, ring), sts16x2_if<kWrap>(at, v.y, mm & 4u, mm & 8u, end, ring);
-                sts16x2_if<kWrap>(at, v.z, mm & 16u, mm & 32u, end, ring), sts16x2_if<kWrap>(at, v.w, mm & 64u, mm & 128u, end, ring);
-            }
+            uint32_t at = out + S::kES * ((exc >> (p * S::kFB)) & S::kFieldMask);
+            sts_kept<U>(at, q[b * S::kPack + p]);
             out += S::kES * ((tot >> (p * S::kFB)) & S::kFieldMask);
-            wrap_addr<kWrap>(out, end, ring);
         }
     }
 }
@@ -579,8 +571,8 @@ template <int kJobs>
 __device__ __forceinline__ void walk_seek(Walk &w, const CompressParams<kJobs> &p, const uint32_t cta, const uint32_t G)
 {
     while (w.k < p.c.jobs) {
-        const uint32_t rot = p.job[w.k].rot;
-        w.tiles            = p.job[w.k].tiles;
+        const uint32_t rot = p.job[kJobs == 1 ? 0u : w.k].rot;
+        w.tiles            = p.job[kJobs == 1 ? 0u : w.k].tiles;
         w.v                = cta >= rot ? cta - rot : cta + G - rot;
         if (w.v < w.tiles) {
             w.j     = 0;
@@ -607,23 +599,13 @@ __device__ __forceinline__ void walk_next(Walk &w, const CompressParams<kJobs> &
     }
 }
 
-// A wave total: the count of all G tiles of a wave, published by the CTA that takes the wave's last tile (it reads
-// the counts of all the others for its own base anyway) as a tagged pair like a descriptor: word 0 = (tag >> 32) <<
-// 32 | low half of the sum, word 1 = (tag & 0xFFFFFFFF) << 32 | high half.
-__device__ __forceinline__ bool pair_valid(const uint64_t w0, const uint64_t w1, const uint64_t tag_w0, const uint64_t tag_w1)
-{
-    return ((w0 ^ tag_w0) >> 32) == 0 && ((w1 ^ tag_w1) >> 32) == 0;
-}
-
-constexpr int kScanWarps = 3;
-
 // U: uint64_t, uint32_t or uint16_t (the element's width).
 // FUSED: -1 for the plain compressor, else the number of the fused forward form (element type, + 4 for ReLU6).
 // CAST: 0, or the 16-bit type the copiers narrow the packed binary32 values to (1 binary16, 2 bfloat16).
 // kJobs: room for tensors in the kernel's parameters (1, or kMaxBatch for the batched forms).
 // kWarps compactor warps, kSeg elements per warp, kStages ring slots, kCopiers copier warps.
 template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kWarps, int kSeg, int kStages, int kCopiers>
-__global__ void __launch_bounds__((kWarps + kCopiers + kScanWarps + 1) * 32)
+__global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32)
 compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
 {
     using S                       = Seg<U, kSeg>;
@@ -633,14 +615,17 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     constexpr int kCompactThreads = kWarps * 32;
     // warp roles
     constexpr int kFirstCopier   = kWarps;
-    constexpr int kScanWarp      = kWarps + kCopiers;       // ... kScanWarp + kScanWarps - 1
-    constexpr int kLoadWarp      = kWarps + kCopiers + kScanWarps;
+    constexpr int kScanWarp      = kWarps + kCopiers;       // and kScanWarp + 1
+    constexpr int kLoadWarp      = kWarps + kCopiers + 2;
     constexpr int kSegsPerCopier = kWarps / kCopiers;
     static_assert(kWarps % kCopiers == 0, "equal shares for the copier warps");
     static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
     static_assert(kTile % BT_CHUNK_ELEMS == 0, "a tile holds whole chunks");
     static_assert(kWarps <= 32, "one lane per warp count");
-    static_assert(kStages >= 3, "loading, compacting, awaiting its base or being copied out");
+    // A scan warp makes tile i ready only in its turn for tile i + 2, after that tile has been counted, so
+    // tiles i, i + 1 and i + 2 must hold slots at once: three stages are the minimum that cannot deadlock,
+    // the fourth keeps the bulk copy of the next tile in flight.
+    static_assert(kStages >= 4, "loading, compacting, awaiting its base, copying out");
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     U *const tiles = reinterpret_cast<U *>(smem_raw);
@@ -652,9 +637,17 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
     __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
     __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
+    __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
     __shared__ __align__(16) unsigned char s_bits[kWarps][kSeg / 8];   // bitmap bytes of the segment a warp is compacting
     __shared__ volatile uint32_t s_abort;
     __shared__ volatile uint64_t s_tag;                    // this launch's tag once the first scan warp has it, else 0
+    __shared__ volatile uint32_t s_met;                    // the grid has met: wave totals may be added to and read
+    // Contributions to wave totals held back until then, and the total words they belong to.  This CTA's i-th tile
+    // can be counted before the meeting is over only while i <= kStages (tile kStages + 1 needs the slot of tile 1,
+    // whose base may need a total), so kStages + 1 slots, indexed by i modulo that, never collide.
+    constexpr uint32_t kHeld = kStages + 1;
+    __shared__ unsigned long long s_held[kHeld];
+    __shared__ uint32_t          s_held_word[kHeld];
     __shared__ uint64_t          s_arena_c0;               // arena forms: the cursor as this launch found it
 
     const uint32_t tid  = threadIdx.x;
@@ -664,6 +657,11 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     const uint32_t G       = gridDim.x;
     const uint32_t cta     = blockIdx.x;
     const uint64_t wait_ns = p.c.wait_ns;
+    // The first kDirect waves of a tensor take the counts of the waves before them straight from the descriptors, so
+    // totals (and with them the zeroing and the meeting) are needed only by tensors of more waves than that; and
+    // without totals the last tile's base of one tensor holds a count from every CTA: no meeting.
+    bool meet = p.c.jobs > 1;
+    for (uint32_t k = 0; k < p.c.jobs; ++k) meet = meet || p.job[k].tiles > kDirect * G;
 
     if (tid == 0) {
         // Read before the barrier below: the kernel's one update of the cursor follows the last tile's base,
@@ -671,6 +669,8 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         s_arena_c0 = p.c.arena_cursor ? *reinterpret_cast<const volatile uint64_t *>(p.c.arena_cursor) : 0;
         s_abort    = 0;
         s_tag      = 0;
+        s_met      = 0;
+        for (uint32_t k = 0; k < kHeld; ++k) s_held[k] = 0;
         for (int s = 0; s < kStages; ++s) {
             mbar_init(&s_full[s], 1);
             mbar_init(&s_counted[s], kWarps);
@@ -699,9 +699,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 if (it >= 2u && it < static_cast<uint32_t>(kStages)) mbar_wait<false>(&s_full[(it - 2u) % kStages], 0, &s_abort, wait_ns);
                 // bulk copy of the tile into its ring slot
                 const uint32_t s     = it % kStages;
-                const U *const src   = static_cast<const U *>(p.job[w.k].src);
+                const U *const src   = static_cast<const U *>(p.job[kJobs == 1 ? 0u : w.k].src);
                 const uint64_t first = static_cast<uint64_t>(w.tile(G)) * kTile;
-                const uint64_t left  = p.job[w.k].n - first;
+                const uint64_t left  = p.job[kJobs == 1 ? 0u : w.k].n - first;
                 const uint32_t valid = left < static_cast<uint64_t>(kTile) ? static_cast<uint32_t>(left) : kTile;
                 const uint32_t bytes = (valid * static_cast<uint32_t>(sizeof(U))) & ~15u;   // whole 16-byte units
                 fence_proxy_async();                       // the copiers' and compactors' accesses to the slot come first
@@ -718,19 +718,18 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         return;
     }
 
-    if (warp >= kScanWarp) {
+    if (warp == kScanWarp || warp == kScanWarp + 1) {
         // ------------------------------------------------------------ scan warps
-        // kScanWarps warps share the scan: warp q takes this CTA's tiles q, q + kScanWarps, ... (counted in the order
-        // the CTA takes them).  A warp's turn for a tile:
-        //   (a) wait until the compactors have counted the tile, publish the count;
-        //   (b) read, in ONE batch of independent loads, the descriptors of the virtual CTAs in front of this one in
-        //       the tile's wave and the totals of the waves since this warp's previous tile; repeat for what was not
-        //       there yet (CTAs do not run in step: a CTA that is ahead of the others waits here for them);
-        //   (c) base = the totals of the waves in front + the counts in front; hand the tile to the copiers; the CTA
-        //       that took the last tile of a wave publishes the wave's total.
-        // A turn is one round trip to L2 (one to three microseconds while the SM's bulk copies are in flight) and a
-        // tile takes about one, so three warps keep up.  While a warp waits in (b) it also looks out for its next
-        // tile's count and publishes it at once: other CTAs are waiting for it.
+        // Two warps share the scan: warp q takes this CTA's tiles q, q + 2, q + 4, ... (counted in the order the
+        // CTA takes them).  A warp's turn for tile i is
+        //   (a) wait until the compactors have counted tile i, publish the count,
+        //   (c) finish tile i - 2 (its own previous tile) from the loads of its previous turn and hand it
+        //       to the copiers,
+        //   (b) wait until tile i + 1 is counted -- about one tile later, when every CTA has published
+        //       the wave of tile i -- and issue, in ONE batch of independent loads, the reads of the descriptors
+        //       of that wave and of the totals of the two waves before it.
+        // The loads of (b) are used a whole tile later, in (c) of the next turn, so the round trip to L2
+        // (1.3 us under load, longer than one tile) never stalls a turn for long: a turn has two tiles' time.
         const uint32_t  q          = warp - kScanWarp;
         uint64_t *const wave_total = p.c.ws_total;
         uint64_t *const desc       = p.c.ws_desc;
@@ -743,9 +742,10 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             const uint32_t v   = cta >= rot ? cta - rot : cta + G - rot;
             if (v < t) my_tiles += (t - v + G - 1) / G;
         }
+        const uint32_t last_i = my_tiles - 1;       // every CTA has a tile: the grid is no larger than the tile count
 
-        // The tag of this launch.  One warp reads the sequence number; it changes only once every CTA has published
-        // a count, which a CTA does after this read.
+        // The tag of this launch.  One warp reads the sequence number; it changes only once every CTA has arrived
+        // at the meeting, which a CTA does after this read.
         uint64_t tag = 0;
         if (q == 0) {
             if (lane == 0) {
@@ -763,186 +763,204 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         }
         const uint64_t tag_w0 = tag & 0xFFFFFFFF00000000ull, tag_w1 = tag << 32;
         auto valid = [&](const uint64_t w0, const uint64_t w1) {
-            return pair_valid(w0, w1, tag_w0, tag_w1) && static_cast<uint32_t>(w0) == static_cast<uint32_t>(w1);
+            return ((w0 ^ tag_w0) >> 32) == 0 && ((w1 ^ tag_w1) >> 32) == 0 && static_cast<uint32_t>(w0) == static_cast<uint32_t>(w1);
         };
 
-        // (a) for the tile `c` of flat index i: counts of the segments -> offsets, the tile's count published
-        struct Counted {
-            uint32_t off;      // lane l < kWarps: exclusive offset of segment l
-            uint32_t agg;      // the tile's count
-        };
-        auto publish = [&](const Walk &c, const uint32_t i) {
-            const uint32_t s   = i % kStages;
-            const uint32_t cn  = lane < kWarps ? s_cnt[s][lane] : 0u;
-            uint32_t       inc = cn;
-#pragma unroll
-            for (int o = 1; o < kWarps; o <<= 1) {
-                const uint32_t u = __shfl_up_sync(kFull, inc, o);
-                if (lane >= static_cast<uint32_t>(o)) inc += u;
+        // Wave totals are sums made by reductions, so their words must be zero first, and the grid must have met
+        // after the zeroing before anyone adds or reads.  That meeting is a copier warp's job (below): until it is
+        // over, a scan warp parks its contribution in shared memory and goes on -- the tagged descriptors need no
+        // clearing, so counts are published and read without waiting for the meeting.
+        auto add_to_total = [&](const uint32_t i, const uint32_t word_index, const unsigned long long contribution) {   // lane 0 only
+            if (s_met) {
+                red_add_u64(wave_total + word_index, contribution);
+                return;
             }
-            Counted r;
-            r.agg = __shfl_sync(kFull, inc, kWarps - 1);
-            r.off = inc - cn;
-            if (lane == 0) st_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(p.job[c.k].desc0) + c.tile(G)), tag_w0 | r.agg, tag_w1 | r.agg);
-            if (lane < kWarps) s_off[s][lane] = r.off;
-            return r;
+            const uint32_t slot = i % kHeld;
+            s_held_word[slot]   = word_index;
+            __threadfence_block();
+            atomicExch(&s_held[slot], contribution);
+            __threadfence_block();
+            if (s_met) {
+                // the meeting ended meanwhile: whoever takes the parked value out adds it
+                const unsigned long long v = atomicExch(&s_held[slot], 0ull);
+                if (v) red_add_u64(wave_total + word_index, v);
+            }
         };
+
+        // d0[k], d1[k], lane l <-> descriptor of virtual CTA l + 32k of the wave of this warp's previous tile;
+        // w1, w2: total words of the one and the two waves before it (0: not read yet)
+        uint64_t d0[kMaxWindows], d1[kMaxWindows], w1 = 0, w2 = 0;
+#pragma unroll
+        for (int k = 0; k < kMaxWindows; ++k) d0[k] = tag_w0, d1[k] = tag_w1;
 
         Walk cur;                                   // this warp's tile of the turn
         walk_begin(cur, p, cta, G);
-        for (uint32_t k = 0; k < q; ++k) walk_next(cur, p, cta, G);
-        Walk     nxt = cur;                         // and its next one
-        for (int k = 0; k < kScanWarps; ++k) walk_next(nxt, p, cta, G);
-        bool     nxt_published = false;
-        Counted  nxt_counted{0, 0};
-        uint64_t waves_before = 0;                  // sum of the totals of the waves before this warp's previous tile ...
-        uint32_t waves_of     = 0xFFFFFFFFu;        // ... of this tensor
+        if (q == 1 && cur.valid) walk_next(cur, p, cta, G);
+        uint32_t pk = 0, pj = 0, pv = 0;            // this warp's previous tile: tensor, wave, virtual CTA
+        uint64_t p_direct = 0;                      //   and, for a wave < kDirect, the counts of all the waves before it
+        uint64_t waves_before = 0;                  // sum of the counts of the waves before the previous tile (of its tensor)
 
-        for (uint32_t i = q; !failed && i < my_tiles; i += kScanWarps) {
-            // ---- (a)
-            Counted me;
-            if (nxt_published) {
-                me = nxt_counted;
-            } else {
-                if (!mbar_wait(&s_counted[i % kStages], (i / kStages) & 1u, &s_abort, wait_ns)) {
+        for (uint32_t i = q; !failed && i <= last_i + 2; i += 2) {
+            const bool has = i <= last_i;
+            if (has) {
+                // ---- (a)
+                const uint32_t s = i % kStages;
+                if (!mbar_wait(&s_counted[s], (i / kStages) & 1u, &s_abort, wait_ns)) {
                     failed = true;
                     break;
                 }
-                me = publish(cur, i);
-            }
-            nxt_published         = false;
-            const uint32_t i_next = i + kScanWarps;
-            const bool     has_n  = i_next < my_tiles;
-
-            // ---- (b)
-            const CompressJob &jb      = p.job[cur.k];
-            const uint64_t     d_first = static_cast<uint64_t>(jb.desc0) + static_cast<uint64_t>(cur.j) * G;
-            const uint32_t     n_tot   = cur.j < static_cast<uint32_t>(kScanWarps) ? cur.j : static_cast<uint32_t>(kScanWarps);   // totals to read: waves cur.j - 1, cur.j - 2, ...
-            uint64_t           d0[kMaxWindows], d1[kMaxWindows], t0w = 0, t1w = 0;
-            bool               have[kMaxWindows], have_t = lane >= n_tot;
+                const uint32_t c   = lane < kWarps ? s_cnt[s][lane] : 0u;
+                uint32_t       inc = c;
 #pragma unroll
-            for (int k = 0; k < kMaxWindows; ++k) {
-                have[k] = lane + 32u * k >= cur.v;                   // not in front of this CTA: a count of 0
-                d0[k] = d1[k] = 0;
+                for (int o = 1; o < kWarps; o <<= 1) {
+                    const uint32_t u = __shfl_up_sync(kFull, inc, o);
+                    if (lane >= static_cast<uint32_t>(o)) inc += u;
+                }
+                const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
+                if (lane == 0) {
+                    st_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(p.job[kJobs == 1 ? 0u : cur.k].desc0) + cur.tile(G)), tag_w0 | agg, tag_w1 | agg);
+                    s_agg[s] = agg;
+                }
+                if (lane < kWarps) s_off[s][lane] = inc - c;
+                if (cur.tiles > kDirect * G && lane == 0) add_to_total(i, p.job[kJobs == 1 ? 0u : cur.k].total0 + cur.j, (1ull << kCountShift) + agg);
             }
-            uint32_t polls   = 0;
-            uint64_t t_start = 0;
-            for (;;) {
-                bool missing = false;
+            if (i >= 2) {
+                // ---- (c): this warp's previous tile, (pk, pj, pv)
+                const CompressJob &jb    = p.job[kJobs == 1 ? 0u : pk];
+                uint32_t           polls = 0;
+                uint64_t           t0    = 0;
+                for (;;) {
+                    bool missing = pj >= kDirect && ((w1 >> kCountShift) != G || (w2 >> kCountShift) != G);
 #pragma unroll
-                for (int k = 0; k < kMaxWindows; ++k) {
-                    if (!have[k]) {
-                        ld_relaxed_2xu64(desc + 2 * (d_first + lane + 32u * k), d0[k], d1[k]);
-                        have[k] = valid(d0[k], d1[k]);
-                        missing |= !have[k];
-                    }
-                }
-                if (!have_t) {
-                    ld_relaxed_2xu64(wave_total + 2 * (static_cast<uint64_t>(jb.total0) + cur.j - 1 - lane), t0w, t1w);
-                    have_t = pair_valid(t0w, t1w, tag_w0, tag_w1);
-                    missing |= !have_t;
-                }
-                if (!__any_sync(kFull, missing)) break;
-                // meanwhile: the next tile's count, as soon as it is there
-                if (has_n && !nxt_published && mbar_try_wait(&s_counted[i_next % kStages], (i_next / kStages) & 1u, 0u)) {
-                    nxt_counted   = publish(nxt, i_next);
-                    nxt_published = true;
-                }
-                __nanosleep(200);
-                if ((++polls & 127u) == 0 || wait_ns < 1000000ull) {
-                    if (t_start == 0) t_start = now_ns();
-                    if (__any_sync(kFull, (now_ns() - t_start > wait_ns) || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)) {
-                        failed = true;
-                        break;
-                    }
-                }
-            }
-            if (failed) break;
-
-            // ---- (c)
-            uint64_t part = 0;
-#pragma unroll
-            for (int k = 0; k < kMaxWindows; ++k)
-                if (lane + 32u * k < cur.v) part += static_cast<uint32_t>(d0[k]);
-            const uint64_t in_front = warp_sum_u64(part);
-            const uint64_t totals   = warp_sum_u64(lane < n_tot ? ((t0w & 0xFFFFFFFFull) | (t1w << 32)) : 0ull);
-            waves_before            = (waves_of == cur.k ? waves_before : 0ull) + totals;
-            waves_of                = cur.k;
-            const uint64_t base     = waves_before + in_front;
-            const uint32_t s        = i % kStages;
-            const uint64_t tile     = cur.tile(G);
-            // the CTA of a wave's last tile has read the counts of all the others: the wave's total
-            if (cur.v == G - 1 && lane == 0) {
-                const uint64_t sum = in_front + me.agg;
-                st_relaxed_2xu64(wave_total + 2 * (static_cast<uint64_t>(jb.total0) + cur.j), tag_w0 | (sum & 0xFFFFFFFFull), tag_w1 | (sum >> 32));
-            }
-            // exclusive count in front of each chunk of that tile
-            if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
-                const uint64_t ch = tile * kChunksPerTile + lane / kWarpsPerChunk;
-                if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + me.off;
-            }
-            if (tile == jb.tiles - 1 && lane == 0) {
-                const uint64_t nnz = base + me.agg;
-                *jb.nnz_out        = nnz;
-                __threadfence();
-                const bool aborted  = ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag;
-                uint64_t   capacity = jb.capacity;
-                if (p.c.arena_cursor) {
-                    // arena form: the room left behind the cursor; the cursor moves only when everything fitted
-                    const uint64_t c0 = s_arena_c0;
-                    capacity          = c0 <= p.c.arena_bytes ? (p.c.arena_bytes - c0) / sizeof(Stored<CAST, U>) : 0;
-                    if (!aborted && nnz <= capacity) {
-                        *p.c.values_offset_out = c0;
-                        *p.c.arena_cursor      = c0 + ((nnz * sizeof(Stored<CAST, U>) + 15) & ~15ull);
-                    }
-                }
-                if (jb.dev_status) {
-                    *reinterpret_cast<volatile int32_t *>(jb.dev_status) = aborted ? BT_ERR_TIMEOUT : (nnz > capacity ? BT_ERR_CAPACITY : BT_OK);
-                    // a CTA that gives up from now on stores its BT_ERR_TIMEOUT after this word; one that gave
-                    // up just before is seen here
-                    __threadfence();
-                    if (!aborted && ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)
-                        *reinterpret_cast<volatile int32_t *>(jb.dev_status) = BT_ERR_TIMEOUT;
-                }
-            }
-            if (lane == 0) {
-                s_base[s] = base;
-                mbar_arrive(&s_ready[s]);                       // the copiers may take the tile
-            }
-            if (cur.k + 1 == p.c.jobs && tile == jb.tiles - 1) {
-                // The launch's last tile.  The next launch on this workspace must get another tag, and the sequence
-                // number may move only once every CTA has read it, i.e. has published a count.  For one tensor the
-                // base above says so (it holds, through the totals, a count from every CTA).  In a batch the first G
-                // tiles of the launch are one per CTA: wait for their counts.
-                bool all = true;
-                if (p.c.jobs > 1) {
-                    bool seen[kMaxWindows];
-#pragma unroll
-                    for (int k = 0; k < kMaxWindows; ++k) seen[k] = lane + 32u * k >= G;
-                    const uint64_t t0 = now_ns();
-                    for (;;) {
-                        bool missing = false;
-#pragma unroll
-                        for (int k = 0; k < kMaxWindows; ++k) {
-                            if (!seen[k]) {
-                                uint64_t x0, x1;
-                                ld_relaxed_2xu64(desc + 2 * static_cast<uint64_t>(lane + 32u * k), x0, x1);
-                                seen[k] = valid(x0, x1);
-                                missing |= !seen[k];
-                            }
-                        }
-                        if (!__any_sync(kFull, missing)) break;
-                        if (__any_sync(kFull, now_ns() - t0 > wait_ns)) {
-                            all = false;
+                    for (int k = 0; k < kMaxWindows; ++k) missing |= !valid(d0[k], d1[k]);
+                    if (!__any_sync(kFull, missing)) break;
+                    __nanosleep(100);
+                    if ((++polls & 255u) == 0 || wait_ns < 1000000ull) {
+                        if (t0 == 0) t0 = now_ns();
+                        if (__any_sync(kFull, (now_ns() - t0 > wait_ns) || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)) {
+                            failed = true;
                             break;
                         }
-                        __nanosleep(200);
+                    }
+#pragma unroll
+                    for (int k = 0; k < kMaxWindows; ++k)
+                        if (!valid(d0[k], d1[k]))
+                            ld_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(jb.desc0) + static_cast<uint64_t>(pj) * G + lane + 32u * k), d0[k], d1[k]);
+                    if (s_met && pj >= kDirect) {        // a total counts only once every CTA has zeroed its share
+                        if ((w1 >> kCountShift) != G) w1 = ld_relaxed_u64(wave_total + jb.total0 + (pj - 1));
+                        if ((w2 >> kCountShift) != G) w2 = ld_relaxed_u64(wave_total + jb.total0 + (pj - 2));
                     }
                 }
-                if (lane == 0) red_add_u64(p.c.ws_header + kHdrSeq, all ? 1ull : 1ull << 32);
+                if (failed) break;
+                uint64_t part = 0;
+#pragma unroll
+                for (int k = 0; k < kMaxWindows; ++k) part += static_cast<uint32_t>(d0[k]);
+                // the waves in front of the tile: those in front of this warp's tile before it, if that was wave
+                // pj - 2 of the same tensor, and the one or two waves read for this turn
+                // (a wave < kDirect brings the sum with it; the tile of this warp before a wave >= kDirect is of the same tensor)
+                waves_before = pj < kDirect ? p_direct : waves_before + (w1 & ((1ull << kCountShift) - 1)) + (w2 & ((1ull << kCountShift) - 1));
+                const uint64_t base = waves_before + warp_sum_u64(part);
+                const uint32_t ps   = (i - 2) % kStages;
+                const uint64_t pt   = pv + static_cast<uint64_t>(pj) * G;
+                // exclusive count in front of each chunk of that tile
+                if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
+                    const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
+                    if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + s_off[ps][lane];
+                }
+                if (pt == jb.tiles - 1 && lane == 0) {
+                    const uint64_t nnz = base + s_agg[ps];
+                    *jb.nnz_out        = nnz;
+                    __threadfence();
+                    const bool aborted  = ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag;
+                    uint64_t   capacity = jb.capacity;
+                    if (p.c.arena_cursor) {
+                        // arena form: the room left behind the cursor; the cursor moves only when everything fitted
+                        const uint64_t c0 = s_arena_c0;
+                        capacity          = c0 <= p.c.arena_bytes ? (p.c.arena_bytes - c0) / sizeof(Stored<CAST, U>) : 0;
+                        if (!aborted && nnz <= capacity) {
+                            *p.c.values_offset_out = c0;
+                            *p.c.arena_cursor      = c0 + ((nnz * sizeof(Stored<CAST, U>) + 15) & ~15ull);
+                        }
+                    }
+                    // without a meeting: every CTA has published its count by now, so every CTA has read the sequence
+                    // number, and the next launch on this workspace gets another tag
+                    if (!meet) red_add_u64(p.c.ws_header + kHdrSeq, 1ull);
+                    if (jb.dev_status) {
+                        *reinterpret_cast<volatile int32_t *>(jb.dev_status) = aborted ? BT_ERR_TIMEOUT : (nnz > capacity ? BT_ERR_CAPACITY : BT_OK);
+                        // a CTA that gives up from now on stores its BT_ERR_TIMEOUT after this word; one that gave
+                        // up just before is seen here
+                        __threadfence();
+                        if (!aborted && ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)
+                            *reinterpret_cast<volatile int32_t *>(jb.dev_status) = BT_ERR_TIMEOUT;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    s_base[ps] = base;
+                    mbar_arrive(&s_ready[ps]);                       // the copiers may take the tile
+                }
             }
-            cur = nxt;
-            for (int k = 0; k < kScanWarps; ++k) walk_next(nxt, p, cta, G);
+            if (has) {
+                // ---- (b): a tile later (when the other scan warp's next tile is counted, if there is one)
+                if (i + 1 > last_i) {
+                    // This CTA's last tile: no next tile to wait for.  A short pause gives the other counts of the
+                    // wave time to land, so that the reads below usually succeed at once instead of costing a second
+                    // round trip.
+                    __nanosleep(300);
+                } else if (!mbar_wait(&s_counted[(i + 1) % kStages], ((i + 1) / kStages) & 1u, &s_abort, wait_ns)) {
+                    failed = true;
+                    break;
+                }
+                const uint64_t d_first = static_cast<uint64_t>(p.job[kJobs == 1 ? 0u : cur.k].desc0) + static_cast<uint64_t>(cur.j) * G;
+#pragma unroll
+                for (int k = 0; k < kMaxWindows; ++k) {
+                    const uint32_t b = lane + 32u * k;
+                    if (b < cur.v) ld_relaxed_2xu64(desc + 2 * (d_first + b), d0[k], d1[k]);
+                    else d0[k] = tag_w0, d1[k] = tag_w1;             // not in front of this CTA: a valid count of 0
+                }
+                const bool met = s_met != 0;
+                w1 = (cur.j >= kDirect && met) ? ld_relaxed_u64(wave_total + p.job[kJobs == 1 ? 0u : cur.k].total0 + (cur.j - 1)) : 0ull;
+                w2 = (cur.j >= kDirect && met) ? ld_relaxed_u64(wave_total + p.job[kJobs == 1 ? 0u : cur.k].total0 + (cur.j - 2)) : 0ull;
+                p_direct = 0;
+                if (cur.j > 0 && cur.j < kDirect) {
+                    // one of a tensor's first waves: the counts of all tiles of the waves before it, read here and now
+                    // (they were published a tile ago and more; what is not there yet is asked for again)
+                    const uint64_t t_first = static_cast<uint64_t>(p.job[kJobs == 1 ? 0u : cur.k].desc0);
+                    uint64_t       sum     = 0;
+                    for (uint32_t jj = 0; jj < cur.j && !failed; ++jj) {
+                        bool     got[kMaxWindows];
+#pragma unroll
+                        for (int k = 0; k < kMaxWindows; ++k) got[k] = lane + 32u * k >= G;
+                        uint32_t tries = 0;
+                        uint64_t t_start = 0;
+                        for (;;) {
+                            bool miss = false;
+#pragma unroll
+                            for (int k = 0; k < kMaxWindows; ++k) {
+                                if (!got[k]) {
+                                    uint64_t x0, x1;
+                                    ld_relaxed_2xu64(desc + 2 * (t_first + static_cast<uint64_t>(jj) * G + lane + 32u * k), x0, x1);
+                                    if (valid(x0, x1)) got[k] = true, sum += static_cast<uint32_t>(x0);
+                                    else miss = true;
+                                }
+                            }
+                            if (!__any_sync(kFull, miss)) break;
+                            __nanosleep(100);
+                            if ((++tries & 255u) == 0 || wait_ns < 1000000ull) {
+                                if (t_start == 0) t_start = now_ns();
+                                if (__any_sync(kFull, (now_ns() - t_start > wait_ns) || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)) {
+                                    failed = true;
+                                    break;
+                                }
+                            }
+                        }
+                    }
+                    p_direct = warp_sum_u64(sum);
+                }
+                pk = cur.k, pj = cur.j, pv = cur.v;
+                walk_next(cur, p, cta, G);
+                if (cur.valid) walk_next(cur, p, cta, G);
+            }
         }
         if (failed && lane == 0) raise_timeout(p, &s_abort, tag);
         return;
@@ -952,16 +970,87 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         // ------------------------------------------------------------ copier warps
         const uint32_t copier = warp - kFirstCopier;
         using V               = Stored<CAST, U>;
-        Walk           w;
+        if (copier == kCopiers - 1 && meet) {
+            // The meeting: this warp has nothing to copy for the first microseconds.  It zeroes this CTA's share of
+            // the wave totals and writes the launch's tag into this CTA's arrival word.  CTA 0 waits (bounded) until
+            // all G arrival words carry the tag -- every CTA has then zeroed its share, and has read the sequence
+            // number, which CTA 0 now moves on -- and writes the tag into the "go" word; the others wait for that
+            // word (one poller and one word per CTA: every CTA polling every arrival word makes a hot spot in L2
+            // that takes microseconds to cool).  Then the warp adds what the scan warps have parked meanwhile.
+            uint64_t *const wave_total = p.c.ws_total;
+            uint64_t *const arrive     = p.c.ws_header + kWsArriveWord;
+            uint64_t        tag        = 0;
+            if (lane == 0) tag = wait_tag(&s_tag, &s_abort, wait_ns);
+            tag     = __shfl_sync(kFull, tag, 0);
+            bool ok = tag != 0;
+            if (ok) {
+                for (uint32_t i = cta * 32 + lane; i < p.c.ws_totals; i += G * 32) wave_total[i] = 0;
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    st_release_u64(arrive + cta, tag);
+                }
+                const uint64_t t0 = now_ns();
+                if (cta == 0) {
+                    bool here[kMaxWindows];
+#pragma unroll
+                    for (int k = 0; k < kMaxWindows; ++k) here[k] = lane + 32u * k >= G;
+                    for (;;) {
+                        bool missing = false;
+#pragma unroll
+                        for (int k = 0; k < kMaxWindows; ++k) {
+                            if (!here[k]) here[k] = ld_acquire_u64(arrive + lane + 32u * k) == tag;
+                            missing |= !here[k];
+                        }
+                        if (!__any_sync(kFull, missing)) break;
+                        if (__any_sync(kFull, s_abort != 0 || now_ns() - t0 > wait_ns)) {
+                            ok = false;
+                            break;
+                        }
+                    }
+                    if (ok && lane == 0) {
+                        __threadfence();
+                        st_release_u64(p.c.ws_header + kHdrGo, tag);
+                        red_add_u64(p.c.ws_header + kHdrSeq, 1ull);      // every CTA has read it: the next launch gets another tag
+                    }
+                } else {
+                    if (lane == 0) {
+                        while (ld_acquire_u64(p.c.ws_header + kHdrGo) != tag) {
+                            if (s_abort != 0 || now_ns() - t0 > wait_ns) {
+                                ok = false;
+                                break;
+                            }
+                            __nanosleep(64);
+                        }
+                    }
+                    ok = __shfl_sync(kFull, ok ? 1 : 0, 0) != 0;
+                }
+            }
+            if (lane == 0) {
+                if (ok) {
+                    __threadfence();
+                    s_met = 1;
+                    __threadfence_block();
+                    for (uint32_t k = 0; k < kHeld; ++k) {
+                        const unsigned long long v = atomicExch(&s_held[k], 0ull);
+                        if (v) red_add_u64(wave_total + s_held_word[k], v);
+                    }
+                } else {
+                    raise_timeout(p, &s_abort, tag);
+                }
+            }
+            __syncwarp();
+        }
+        Walk w;
         walk_begin(w, p, cta, G);
         for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
             const uint32_t s = it % kStages;
             if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort, wait_ns)) break;
-            V       *vals     = static_cast<V *>(p.job[w.k].values);
-            uint64_t capacity = p.job[w.k].capacity;
+            V       *vals     = static_cast<V *>(p.job[kJobs == 1 ? 0u : w.k].values);
+            uint64_t capacity = p.job[kJobs == 1 ? 0u : w.k].capacity;
             if (p.c.arena_cursor) {
                 const uint64_t c0 = s_arena_c0;
-                vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(p.job[w.k].values) + c0);
+                vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(p.job[kJobs == 1 ? 0u : w.k].values) + c0);
                 capacity          = c0 <= p.c.arena_bytes ? (p.c.arena_bytes - c0) / sizeof(V) : 0;
             }
             const uint64_t base = s_base[s];
@@ -988,7 +1077,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     Walk           w;
     walk_begin(w, p, cta, G);
     for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
-        const CompressJob &jb    = p.job[w.k];
+        const CompressJob &jb    = p.job[kJobs == 1 ? 0u : w.k];
         const uint64_t     n     = jb.n;
         const uint64_t     t64   = w.tile(G);
         const uint32_t     s     = it % kStages;
@@ -1026,11 +1115,11 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         uint32_t       inc[S::kBatches], packed[S::kBatches];
         const uint32_t cnt = segment_scan<U, kSeg>(m, inc, packed, lane);
         // the whole segment is in registers: the packed values may overwrite it from its start
-        segment_store<U, kSeg, false>(q, m, inc, packed, seg_addr, 0, 0);
+        segment_store<U, kSeg>(q, inc, packed, seg_addr);
         __syncwarp();
         if (lane == 0) {
             s_cnt[s][warp] = cnt;
-            mbar_arrive(&s_counted[s]);                   // hand the count to the scan warps
+            mbar_arrive(&s_counted[s]);                   // hand the count to the scan warp
         }
         // the bitmap, behind the count: nobody waits for it
         uint32_t word[S::kWordsPerLane];
@@ -1096,7 +1185,7 @@ template <typename U, int FUSED, bool WRITE_Y, int CAST, int kJobs, int kWarps, 
 cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, cudaStream_t stream)
 {
     constexpr int    kTile    = kWarps * kSeg;
-    constexpr int    kThreads = (kWarps + kCopiers + kScanWarps + 1) * 32;
+    constexpr int    kThreads = (kWarps + kCopiers + 3) * 32;
     constexpr size_t kSmem    = static_cast<size_t>(kStages) * kTile * sizeof(U);
     static LaunchShape shape;   // one per instantiation
     auto kernel = compress_kernel<U, FUSED, WRITE_Y, CAST, kJobs, kWarps, kSeg, kStages, kCopiers>;
@@ -1132,7 +1221,7 @@ cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint
         totals += (p.job[k].tiles + grid - 1) / grid;
     }
     p.c.jobs      = count;
-    p.c.ws_totals = static_cast<uint32_t>(2 * totals);              // a pair of words per wave
+    p.c.ws_totals = static_cast<uint32_t>((totals + 1) & ~1ull);     // an even number of total words keeps the descriptors 16-byte aligned
     p.c.ws_header = static_cast<uint64_t *>(workspace);
     p.c.ws_total  = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + kWsHeaderBytes);
     p.c.ws_desc   = p.c.ws_total + p.c.ws_totals;

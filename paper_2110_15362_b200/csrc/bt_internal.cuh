@@ -11,22 +11,25 @@
 namespace bt {
 
 // ---------------------------------------------------------------- workspace layout
-// The workspace arrives with unspecified contents and is never cleared.  It holds, in 64-bit words,
+// The workspace arrives with unspecified contents and is never cleared as a whole.  It holds, in 64-bit words,
 //   a header of kWsHeaderBytes: [0] seq, the launch sequence number of this workspace; [1] abort, equal to the
-//     launch's tag once a bounded wait of that launch ran out;
-//   one pair of words per wave of tiles of every tensor of the launch: the wave's total;
-//   one pair of words per tile: the tile's count.
-// Each word of a pair carries half of the launch's 64-bit tag, and a reader takes a pair only if both halves are
-// those of its own launch (bt_compress.cu has the layouts), so stale or never-written words are simply "not yet
-// published" and the two words may be written and read separately.
+//     launch's tag once a bounded wait of that launch ran out; from kWsArriveWord on, one arrival word per CTA
+//     (the launch's tag once that CTA has zeroed its share of the wave totals: the grid's one meeting);
+//   one total per wave of tiles of every tensor of the launch (an even number of words), zeroed by the launch
+//     itself before use and read only after the meeting;
+//   one 16-byte descriptor per tile, never cleared: word 0 = (tag >> 32) << 32 | count, word 1 = (tag & 0xFFFFFFFF)
+//     << 32 | count.  A reader takes a descriptor only if both halves carry its own launch's tag and agree on
+//     the count (the two halves may be written and read separately).
 // tag = mix64(call_tag + seq * odd) | 1: call_tag comes from the host (a process-wide counter: two calls never
-// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (the CTA of
-// its last tile adds 1 once every CTA has published a count, i.e. has read seq; a CTA that gives up adds 2^32),
-// so replays of one captured launch -- same call_tag -- get different tags too.  Memory this library never wrote
-// matches by chance only: 2^-64 per pair.
-// Sized for the smallest tile (4096 elements): 32 bytes per 4096 elements.
+// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (CTA 0 adds 1
+// once every CTA has arrived at the meeting, i.e. has read seq; a CTA that gives up adds 2^32), so replays of
+// one captured launch -- same call_tag -- get different tags too.  Memory this library never wrote matches by
+// chance only: 2^-64 per word for the tag, and the repeated count on top.
+// Sized for the smallest tile: 24 bytes per 4096 elements.
 constexpr uint32_t kMaxGrid       = 160;                       // CTAs of one compress launch (32 * 5 descriptor windows)
-constexpr size_t   kWsHeaderBytes = 256;
+constexpr uint32_t kWsArriveWord  = 32;                        // first arrival word
+constexpr size_t   kWsHeaderBytes = 8 * (kWsArriveWord + kMaxGrid);
+constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;
 constexpr uint32_t kMaxBatch      = 32;                        // tensors of one batched launch
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;             // bound of every in-kernel wait: 2 s
 
@@ -53,7 +56,7 @@ struct CompressCommon {
     uint64_t   *ws_header;
     uint64_t   *ws_total;   // wave totals (set by launch_compress)
     uint64_t   *ws_desc;    // tile descriptors (set by launch_compress)
-    uint32_t    ws_totals;  // number of wave-total words (two per wave; set by launch_compress)
+    uint32_t    ws_totals;  // number of wave-total words (even; set by launch_compress)
     uint32_t    jobs;       // number of tensors
     uint64_t    call_tag;   // unique to the call (set by launch_compress)
     uint64_t    wait_ns;    // bound of every in-kernel wait (set by launch_compress)
@@ -73,7 +76,7 @@ struct CompressCommon {
 cudaError_t launch_compress(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, int dtype,
                             int fused, cudaStream_t s);
 // bytes of workspace for tensors holding `chunks` 4096-element chunks in all
-constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 32 * static_cast<size_t>(chunks); }
+constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 16 + 24 * static_cast<size_t>(chunks); }
 // the calling thread's limit on the CTAs of one compress launch (0: none); returns the limit it replaces
 uint32_t set_compress_max_ctas(uint32_t max_ctas);
 // the bound of the compress kernels' waits for later launches of the process; returns the one it replaces
@@ -122,7 +125,7 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
 
 // One probe of an mbarrier phase.  The hardware may hold the thread for up to `hint_ns` while the phase is not
 // complete (a suspended thread takes no issue slots from the warps that work), so a wait loop needs few probes.
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, uint32_t hint_ns = 1000u)
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, uint32_t hint_ns = 2000u)
 {
     uint32_t ok;
     asm volatile(
