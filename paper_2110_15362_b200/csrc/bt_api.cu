@@ -51,23 +51,24 @@ int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau
         return BT_ERR_ALIGN;
     if (workspace_bytes < bt_workspace_bytes(n)) return BT_ERR_WORKSPACE;
 
-    bt::CompressJob j{};
-    j.src        = src;
-    j.y          = y;
-    j.bitmap     = bitmap;
-    j.values     = values;
-    j.capacity   = values_capacity;
-    j.prefix     = chunk_prefix;
-    j.nnz_out    = nnz_out;
-    j.dev_status = dev_status;
-    j.n          = n;
-    bt::CompressCommon c{};
-    c.cast              = cast;
-    c.tau               = tau;
-    c.arena_cursor      = arena.cursor;
-    c.values_offset_out = arena.offset_out;
-    c.arena_bytes       = arena.bytes;
-    return bt::launch_compress(c, &j, 1, workspace, dtype, fused, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+    bt::CompressArgs a{};
+    a.src        = src;
+    a.y          = y;
+    a.bitmap     = bitmap;
+    a.values     = values;
+    a.capacity   = values_capacity;
+    a.prefix     = chunk_prefix;
+    a.nnz_out    = nnz_out;
+    a.dev_status = dev_status;
+    a.ws_header  = static_cast<uint64_t *>(workspace);
+    a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + bt::kWsHeaderBytes);
+    a.cast       = cast;
+    a.tau        = tau;
+    a.arena_cursor      = arena.cursor;
+    a.values_offset_out = arena.offset_out;
+    a.arena_bytes       = arena.bytes;
+    a.n          = n;
+    return bt::launch_compress(a, dtype, fused, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
 
 // The batched forms: every tensor is checked before anything is launched; empty tensors get their nnz and status
@@ -102,9 +103,8 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
     if (any && !aligned(workspace, 16)) return BT_ERR_ALIGN;
     if (any && workspace_bytes < bt::compress_workspace_bytes(chunks)) return BT_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    bt::CompressJob    jobs[bt::kMaxBatch];
-    uint32_t           m = 0;
-    bt::CompressCommon c{};
+    bt::CompressJob jobs[bt::kMaxBatch];
+    uint32_t        m = 0;
     for (uint32_t k = 0; k < count; ++k) {
         const bt_batch_item &it = items[k];
         if (it.n == 0) {
@@ -124,7 +124,7 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
             j.n                = it.n;
         }
         if (m == bt::kMaxBatch || (k + 1 == count && m > 0)) {
-            if (bt::launch_compress(c, jobs, m, workspace, dtype, fused, s) != cudaSuccess) return BT_ERR_CUDA;
+            if (bt::launch_compress_batch(jobs, m, 0.0f, workspace, dtype, fused, s) != cudaSuccess) return BT_ERR_CUDA;
             m = 0;
         }
     }

@@ -1,0 +1,243 @@
+// What the single-tensor and the batched compress kernels share: constants of the workspace protocol, small PTX
+// wrappers, the bounded mbarrier wait, the in-place compaction of one segment by one warp, the copy-out of a
+// packed segment, and the host-side launch shape.
+#pragma once
+
+#include <mutex>
+#include <type_traits>
+
+#include "bt_internal.cuh"
+
+namespace bt {
+
+// A value no other call of this process gets (bt_compress.cu).
+uint64_t next_call_tag();
+// The calling thread's limit on the CTAs of one compress launch, 0: none (bt_compress.cu).
+uint32_t compress_max_ctas();
+// The bound of the kernels' waits in nanoseconds; only a test build can change it (bt_compress.cu).
+uint64_t compress_wait_ns();
+
+namespace cmp {
+
+constexpr uint32_t kFull       = 0xFFFFFFFFu;
+constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
+constexpr int      kMaxWindows = 5;                   // the grid never exceeds 32 * kMaxWindows CTAs
+constexpr int      kHdrSeq     = 0;                   // header words (64-bit): launch sequence number,
+constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out)
+constexpr int      kCountShift = 40;                  // wave total word: (tiles added << 40) | sum of counts
+
+
+__device__ __forceinline__ uint64_t now_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__device__ __forceinline__ void red_add_u64(uint64_t *p, uint64_t v)
+{
+    asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// A bijective mixer of 64-bit words (the finaliser of splitmix64).
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t x)
+{
+    x ^= x >> 30;
+    x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27;
+    x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return x;
+}
+
+// Raise the abort flag (shared, and global under this launch's tag if a scan warp got as far as reading it),
+// move the workspace's sequence number so that the next launch cannot take this one's words for its own, and
+// report the timeout.
+static __device__ __noinline__ void raise_timeout(uint64_t *ws_header, int32_t *dev_status, volatile uint32_t *s_abort,
+                                           const uint64_t tag)
+{
+    *s_abort = 1u;
+    if (tag) st_relaxed_u64(ws_header + kHdrAbort, tag);
+    red_add_u64(ws_header + kHdrSeq, 1ull << 32);
+    __threadfence();
+    if (dev_status) *reinterpret_cast<volatile int32_t *>(dev_status) = BT_ERR_TIMEOUT;
+}
+
+// Bounded wait on an mbarrier phase.  False once the limit passed or the CTA is aborting.
+template <bool kStopOnAbort = true>
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *s_abort, const uint64_t limit_ns)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = now_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if ((kStopOnAbort && *s_abort) || now_ns() - t0 > limit_ns) return false;
+    }
+}
+
+// shared-memory accesses by 32-bit shared address, kept in program order among themselves
+// register type that holds one element: 64 bits for 8-byte elements, 32 bits otherwise
+template <typename U>
+using Reg = std::conditional_t<sizeof(U) == 8, uint64_t, uint32_t>;
+
+template <typename U>
+__device__ __forceinline__ Reg<U> lds_elem(uint32_t addr)
+{
+    Reg<U> v;
+    if constexpr (sizeof(U) == 8) asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr));
+    else if constexpr (sizeof(U) == 4) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    else asm volatile("ld.shared.s16 %0, [%1];" : "=r"(v) : "r"(addr));   // sign-extended
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One warp compacts its segment of kSteps * 32 elements in place.  Returns the number of packed
+// values; lane k leaves with the ballot of step k, which is bitmap word k of the segment, in `word`
+// (kept in registers through a tree of selects: a store to shared memory per step costs more).
+// `y` (fused form with dense output) points at the segment's first element of the dense ReLU
+// output, `yvalid` is how many of them exist.  seg_addr is a shared-window address.
+//
+// The loads of a batch of 8 steps are issued before the stores of the batch before it: a store of
+// step k lands below element 32(k+1) and a later batch reads at or above it, so they never meet.
+template <typename U, int RELU_DT, bool WRITE_Y, bool kGuardY, int kSteps>
+__device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uint32_t &word, const uint32_t lane,
+                                                    const uint32_t lt, U *y, const uint32_t yvalid, const float tau)
+{
+    constexpr int      kBatch = 8;
+    static_assert(kSteps % kBatch == 0 && kSteps <= 32, "whole batches; one bitmap word per lane");
+    constexpr uint32_t kES    = sizeof(U);
+    const uint32_t     in0    = seg_addr + lane * kES;
+    uint32_t           out    = seg_addr;               // address of the next free packed slot
+    Reg<U>             v[kBatch], vn[kBatch];
+    uint32_t           bb[kBatch];
+    const bool l0 = lane & 1u, l1 = lane & 2u, l2 = lane & 4u;
+    word = 0;
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) v[j] = lds_elem<U>(in0 + j * 32 * kES);
+#pragma unroll
+    for (int kb = 0; kb < kSteps; kb += kBatch) {
+        if (kb + kBatch < kSteps) {
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) vn[j] = lds_elem<U>(in0 + (kb + kBatch + j) * 32 * kES);
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+            Reg<U> x = v[j];
+            if constexpr (RELU_DT >= 0) {
+                x = fused_forward<RELU_DT>(x, tau);
+                if constexpr (WRITE_Y) {
+                    const uint32_t e = (kb + j) * 32 + lane;
+                    if (!kGuardY || e < yvalid) y[e] = static_cast<U>(x);
+                }
+            }
+            const uint32_t b = __ballot_sync(kFull, x != Reg<U>(0));
+            bb[j] = b;
+            if (x != Reg<U>(0)) {
+                const uint32_t at = out + kES * __popc(b & lt);
+                if constexpr (kES == 8) asm volatile("st.shared.u64 [%0], %1;" ::"r"(at), "l"(x));
+                else if constexpr (kES == 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"(x));
+                else asm volatile("st.shared.u16 [%0], %1;" ::"r"(at), "h"(static_cast<uint16_t>(x)));
+            }
+            out += kES * __popc(b);
+        }
+        {
+            // lane kb + j keeps ballot j of this batch: a binary tree of selects over the low lane bits
+            static_assert(kBatch == 8, "the select tree is written for batches of 8 ballots");
+            const uint32_t t0 = l0 ? bb[1] : bb[0], t1 = l0 ? bb[3] : bb[2], t2 = l0 ? bb[5] : bb[4], t3 = l0 ? bb[7] : bb[6];
+            const uint32_t u0 = l1 ? t1 : t0, u1 = l1 ? t3 : t2;
+            const uint32_t w  = l2 ? u1 : u0;
+            word = (lane >> 3) == static_cast<uint32_t>(kb / 8) ? w : word;
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) v[j] = vn[j];
+    }
+    return (out - seg_addr) / kES;
+}
+
+// Down-cast on stash: a binary32 pattern narrowed to binary16 (CAST 1) or bfloat16 (CAST 2), round to nearest
+// even by the hardware conversion, every NaN to the one quiet NaN 0x7FFF.  CAST 0 passes the element through.
+template <int CAST, typename U>
+__device__ __forceinline__ auto narrowed(const U v)
+{
+    if constexpr (CAST == 0) {
+        return v;
+    } else {
+        static_assert(sizeof(U) == 4, "the narrowing forms take binary32 tensors");
+        const float f = __uint_as_float(v);
+        uint16_t    h;
+        if constexpr (CAST == 1) asm("cvt.rn.f16.f32 %0, %1;" : "=h"(h) : "f"(f));
+        else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(f));
+        return (v & 0x7FFFFFFFu) > 0x7F800000u ? static_cast<uint16_t>(0x7FFFu) : h;
+    }
+}
+template <int CAST, typename U>
+using Stored = std::conditional_t<CAST == 0, U, uint16_t>;
+
+// One warp copies the `cnt` packed slots of its segment to out[0..cnt): contiguous, coalesced.
+template <typename U, int CAST, bool kGuard>
+__device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, const uint32_t lane, const uint32_t cnt,
+                                                 Stored<CAST, U> *__restrict__ out, const uint64_t room)
+{
+    // (Pairing narrowed values into 4-byte stores was measured and is no faster: at half zeros the narrowing
+    // forms run at the speed of the compaction, not of the copy-out.)
+    uint32_t j = lane;
+    for (; j + 96 < cnt; j += 128) {
+        const auto v0 = narrowed<CAST>(seg[j]), v1 = narrowed<CAST>(seg[j + 32]), v2 = narrowed<CAST>(seg[j + 64]),
+                   v3 = narrowed<CAST>(seg[j + 96]);
+        if (!kGuard || j < room) out[j] = v0;
+        if (!kGuard || j + 32 < room) out[j + 32] = v1;
+        if (!kGuard || j + 64 < room) out[j + 64] = v2;
+        if (!kGuard || j + 96 < room) out[j + 96] = v3;
+    }
+    for (; j < cnt; j += 32) {
+        const auto v = narrowed<CAST>(seg[j]);
+        if (!kGuard || j < room) out[j] = v;
+    }
+}
+
+// Launch shape of one kernel instantiation on one device: the opt-in shared
+// memory size is set and the number of co-resident CTAs is looked up once.
+struct LaunchShape {
+    std::mutex lock;
+    int        grid_of_device[64] = {};
+    template <typename Kernel>
+    cudaError_t max_grid(Kernel kernel, int threads, size_t smem, int &grid)
+    {
+        int         dev = 0;
+        cudaError_t e   = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        std::lock_guard<std::mutex> g(lock);
+        if (grid_of_device[dev] == 0) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+            if (e != cudaSuccess) return e;
+            int sms = 0, per_sm = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return e;
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+            if (e != cudaSuccess) return e;
+            if (per_sm < 1 || sms < 1) return cudaErrorLaunchOutOfResources;
+            grid_of_device[dev] = sms * per_sm;
+        }
+        grid = grid_of_device[dev];
+        return cudaSuccess;
+    }
+};
+
+
+}  // namespace cmp
+}  // namespace bt

@@ -11,32 +11,58 @@
 namespace bt {
 
 // ---------------------------------------------------------------- workspace layout
-// The workspace arrives with unspecified contents and is never cleared as a whole.  It holds, in 64-bit words,
-//   a header of kWsHeaderBytes: [0] seq, the launch sequence number of this workspace; [1] abort, equal to the
-//     launch's tag once a bounded wait of that launch ran out; from kWsArriveWord on, one arrival word per CTA
-//     (the launch's tag once that CTA has zeroed its share of the wave totals: the grid's one meeting);
-//   one total per wave of tiles of every tensor of the launch (an even number of words), zeroed by the launch
-//     itself before use and read only after the meeting;
+// The workspace arrives with unspecified contents.  It holds
+//   a 256-byte header, 64-bit words: [0] seq, the launch sequence number of this workspace; [1] abort, equal to
+//     the launch's tag once a bounded wait of that launch ran out;
+//   one 64-bit total per wave of tiles of every tensor of the launch (an even number of words): sums made by
+//     reductions, zeroed by the launch itself before the grid's one meeting, used only by tensors of more than
+//     one wave;
 //   one 16-byte descriptor per tile, never cleared: word 0 = (tag >> 32) << 32 | count, word 1 = (tag & 0xFFFFFFFF)
 //     << 32 | count.  A reader takes a descriptor only if both halves carry its own launch's tag and agree on
 //     the count (the two halves may be written and read separately).
 // tag = mix64(call_tag + seq * odd) | 1: call_tag comes from the host (a process-wide counter: two calls never
-// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (CTA 0 adds 1
-// once every CTA has arrived at the meeting, i.e. has read seq; a CTA that gives up adds 2^32), so replays of
-// one captured launch -- same call_tag -- get different tags too.  Memory this library never wrote matches by
-// chance only: 2^-64 per word for the tag, and the repeated count on top.
+// share one), seq is header word 0 as the launch found it.  Every launch changes seq before it ends (the CTA of
+// the last tile adds 1 once all counts are in; a CTA that gives up adds 2^32), so replays of one captured launch
+// -- same call_tag -- get different tags too.  Memory this library never wrote matches by chance only: 2^-64
+// per word for the tag, and the repeated count on top.
 // Sized for the smallest tile: 24 bytes per 4096 elements.
-constexpr uint32_t kMaxGrid       = 160;                       // CTAs of one compress launch (32 * 5 descriptor windows)
-constexpr uint32_t kWsArriveWord  = 32;                        // first arrival word
-constexpr size_t   kWsHeaderBytes = 8 * (kWsArriveWord + kMaxGrid);
+constexpr size_t   kWsHeaderBytes = 256;
 constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;
 constexpr uint32_t kMaxBatch      = 32;                        // tensors of one batched launch
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;             // bound of every in-kernel wait: 2 s
+// bytes of workspace for tensors holding `chunks` 4096-element chunks in all
+constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 16 + 24 * static_cast<size_t>(chunks); }
 
-// One tensor of a compress launch.
+// One tensor, one launch.
+struct CompressArgs {
+    const void *src;        // dense input (pre-activation for the fused form)
+    void       *y;          // optional dense ReLU output
+    uint32_t   *bitmap;
+    void       *values;
+    uint64_t    capacity;   // in elements
+    uint64_t   *prefix;
+    uint64_t   *nnz_out;
+    int32_t    *dev_status;
+    uint64_t   *ws_header;
+    uint64_t   *ws_desc;    // wave totals, then tile descriptors
+    uint32_t    ws_waves;   // number of wave-total words (even; set by launch_compress)
+    uint64_t    call_tag;   // unique to the call (set by launch_compress)
+    uint64_t    wait_ns;    // bound of every in-kernel wait (set by launch_compress)
+    int         cast;       // 0, or the 16-bit type (BT_F16 / BT_BF16) the stashed values of a binary32 tensor are narrowed to
+    float       tau;        // fused forms: elements <= tau become +0 (0 for plain ReLU)
+    // arena forms: `values` is the arena's base, the packed values go to values + *arena_cursor (bytes);
+    // on success the kernel stores the old cursor in *values_offset_out and advances the cursor past the
+    // values (rounded up to 16 bytes).  All three are NULL / 0 for the plain forms.
+    uint64_t   *arena_cursor;
+    uint64_t   *values_offset_out;
+    uint64_t    arena_bytes;
+    uint64_t    n;
+};
+
+// One tensor of a batched launch.
 struct CompressJob {
-    const void *src;        // dense input (pre-activation for the fused forms)
-    void       *y;          // optional dense output of the fused forms
+    const void *src;        // dense input (pre-activation for the fused form)
+    void       *y;          // optional dense output of the fused form
     uint32_t   *bitmap;
     void       *values;
     uint64_t    capacity;   // in elements
@@ -44,39 +70,31 @@ struct CompressJob {
     uint64_t   *nnz_out;
     int32_t    *dev_status;
     uint64_t    n;
-    // set by launch_compress:
+    // set by launch_compress_batch:
     uint32_t    tiles;      // number of tiles of the tensor
     uint32_t    rot;        // the CTA that takes the tensor's tile 0 (tile t goes to CTA (rot + t) mod grid)
     uint32_t    total0;     // index of the tensor's first wave-total word
     uint32_t    desc0;      // index of the tensor's first tile descriptor
 };
 
-// What every tensor of a launch shares.
+// What the tensors of a batched launch share (all set by launch_compress_batch but tau).
 struct CompressCommon {
     uint64_t   *ws_header;
-    uint64_t   *ws_total;   // wave totals (set by launch_compress)
-    uint64_t   *ws_desc;    // tile descriptors (set by launch_compress)
-    uint32_t    ws_totals;  // number of wave-total words (even; set by launch_compress)
+    uint64_t   *ws_total;   // wave totals
+    uint64_t   *ws_desc;    // tile descriptors
+    uint32_t    ws_totals;  // number of wave-total words (even)
     uint32_t    jobs;       // number of tensors
-    uint64_t    call_tag;   // unique to the call (set by launch_compress)
-    uint64_t    wait_ns;    // bound of every in-kernel wait (set by launch_compress)
-    int         cast;       // 0, or the 16-bit type (BT_F16 / BT_BF16) the stashed values of a binary32 tensor are narrowed to
-    float       tau;        // fused forms: elements <= tau become +0 (0 for plain ReLU)
-    // arena forms (one tensor): `values` is the arena's base, the packed values go to values + *arena_cursor
-    // (bytes); on success the kernel stores the old cursor in *values_offset_out and advances the cursor past the
-    // values (rounded up to 16 bytes).  All three are NULL / 0 for the plain forms.
-    uint64_t   *arena_cursor;
-    uint64_t   *values_offset_out;
-    uint64_t    arena_bytes;
+    uint64_t    call_tag;   // unique to the call
+    uint64_t    wait_ns;    // bound of every in-kernel wait
+    float       tau;        // fused form: elements <= tau become +0 (0 for plain ReLU)
 };
 
 // fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0), 2 ReLU6
-// `jobs` (count of them: 1 .. kMaxBatch, every n > 0) are the tensors of one launch; `workspace` is at least
-// compress_workspace_bytes() of them
-cudaError_t launch_compress(const CompressCommon &c, const CompressJob *jobs, uint32_t count, void *workspace, int dtype,
-                            int fused, cudaStream_t s);
-// bytes of workspace for tensors holding `chunks` 4096-element chunks in all
-constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 16 + 24 * static_cast<size_t>(chunks); }
+cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStream_t s);
+// `jobs` (count of them: 1 .. kMaxBatch, every n > 0) are the tensors of one launch; `workspace` holds at least
+// compress_workspace_bytes() of their chunks; fused: 0 plain compressor, 1 threshold form
+cudaError_t launch_compress_batch(const CompressJob *jobs, uint32_t count, float tau, void *workspace, int dtype, int fused,
+                                  cudaStream_t s);
 // the calling thread's limit on the CTAs of one compress launch (0: none); returns the limit it replaces
 uint32_t set_compress_max_ctas(uint32_t max_ctas);
 // the bound of the compress kernels' waits for later launches of the process; returns the one it replaces
@@ -123,17 +141,15 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
                  : "memory");
 }
 
-// One probe of an mbarrier phase.  The hardware may hold the thread for up to `hint_ns` while the phase is not
-// complete (a suspended thread takes no issue slots from the warps that work), so a wait loop needs few probes.
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, uint32_t hint_ns = 2000u)
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_addr(bar)), "r"(parity), "r"(hint_ns)
+        : "r"(smem_addr(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }

@@ -65,16 +65,17 @@ extern "C" int bt_compress_noalloc(const void *dense, uint64_t n, int dtype, uin
     const int rc      = scratch_for_current_device(&scratch);   // first call on a device: looks the address up
     if (rc != BT_OK) return rc;
 
-    bt::CompressJob j{};
-    j.src        = dense;
-    j.bitmap     = bitmap;
-    j.values     = values;
-    j.capacity   = values_capacity;
-    j.prefix     = chunk_prefix;
-    j.nnz_out    = nnz_out;
-    j.dev_status = dev_status;
-    j.n          = n;
-    bt::CompressCommon c{};
+    bt::CompressArgs a{};
+    a.src        = dense;
+    a.bitmap     = bitmap;
+    a.values     = values;
+    a.capacity   = values_capacity;
+    a.prefix     = chunk_prefix;
+    a.nnz_out    = nnz_out;
+    a.dev_status = dev_status;
+    a.ws_header  = static_cast<uint64_t *>(scratch);
+    a.ws_desc    = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(scratch) + bt::kWsHeaderBytes);
+    a.n          = n;
     // nothing in the scratch is cleared between calls: the kernel tells this call's words by their tag
-    return bt::launch_compress(c, &j, 1, scratch, dtype, 0, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
+    return bt::launch_compress(a, dtype, 0, s) == cudaSuccess ? BT_OK : BT_ERR_CUDA;
 }
