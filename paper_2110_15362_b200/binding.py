@@ -31,7 +31,18 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_decompress_arena", "bt_relu6_fwd_compress", "bt_relu6_bwd_from_stash", "bt_compress_narrow",
            "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd",
            "bt_compress_narrow_arena", "bt_prune_fwd_compress_narrow_arena", "bt_decompress_widen_arena",
-           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked", "bt_set_max_ctas")
+           "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked", "bt_set_max_ctas",
+           "bt_batch_workspace_bytes", "bt_compress_batch", "bt_relu_fwd_compress_batch")
+
+MAX_BATCH_PER_LAUNCH = 32
+
+
+class BatchItem(ctypes.Structure):
+    """bt_batch_item of the C ABI: one tensor of a batched call (device pointers as integers)."""
+    _fields_ = [("dense", ctypes.c_void_p), ("y_out", ctypes.c_void_p), ("bitmap", ctypes.c_void_p),
+                ("values", ctypes.c_void_p), ("values_capacity", ctypes.c_uint64), ("chunk_prefix", ctypes.c_void_p),
+                ("nnz_out", ctypes.c_void_p), ("dev_status", ctypes.c_void_p), ("n", ctypes.c_uint64)]
+
 
 _lib: Optional[ctypes.CDLL] = None
 
@@ -65,6 +76,11 @@ def lib() -> ctypes.CDLL:
         L.bt_workspace_bytes.argtypes = [u64]
         L.bt_compress.restype = i32
         L.bt_compress.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+        L.bt_batch_workspace_bytes.restype = sz
+        L.bt_batch_workspace_bytes.argtypes = [ctypes.POINTER(u64), ctypes.c_uint32]
+        for name in ("bt_compress_batch", "bt_relu_fwd_compress_batch"):
+            getattr(L, name).restype = i32
+            getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp, sz, vp]
         L.bt_decompress.restype = i32
         L.bt_decompress.argtypes = [vp, vp, vp, u64, i32, vp, vp]
         L.bt_relu_fwd_compress.restype = i32
@@ -159,6 +175,36 @@ def bt_compress(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor,
                            _ptr(chunk_prefix), _ptr(nnz_out), _ptr(workspace),
                            workspace.numel() * workspace.element_size(), _ptr(dev_status), _stream(stream))
     return _check("bt_compress", st, check)
+
+
+def bt_batch_workspace_bytes(ns) -> int:
+    """Bytes of workspace a batched call over tensors of these element counts needs."""
+    arr = (ctypes.c_uint64 * len(ns))(*[int(v) for v in ns])
+    return int(lib().bt_batch_workspace_bytes(arr, len(ns)))
+
+
+def batch_items(dense, stashes, y_out=None) -> "ctypes.Array":
+    """The host array of bt_batch_item for tensors `dense[k]` stashed into `stashes[k]` (Stash objects), with the
+    dense outputs `y_out[k]` if given.  Marshalling only: built once, it can be passed to many calls."""
+    items = (BatchItem * len(dense))()
+    for k, (x, st) in enumerate(zip(dense, stashes)):
+        items[k] = BatchItem(_ptr(x), _ptr(y_out[k]) if y_out is not None else None, _ptr(st.bitmap), _ptr(st.values),
+                             st.values.numel(), _ptr(st.chunk_prefix), _ptr(st.nnz_out), _ptr(st.dev_status), x.numel())
+    return items
+
+
+def bt_compress_batch(items, dtype: torch.dtype, workspace: torch.Tensor, *, stream=None, check: bool = True) -> int:
+    """bt_compress of every tensor of `items` (from batch_items) in one pass."""
+    st = lib().bt_compress_batch(items, len(items), DTYPE_CODE[dtype], _ptr(workspace), _nbytes(workspace), _stream(stream))
+    return _check("bt_compress_batch", st, check)
+
+
+def bt_relu_fwd_compress_batch(items, dtype: torch.dtype, workspace: torch.Tensor, *, stream=None,
+                               check: bool = True) -> int:
+    """bt_relu_fwd_compress of every tensor of `items` (from batch_items) in one pass."""
+    st = lib().bt_relu_fwd_compress_batch(items, len(items), DTYPE_CODE[dtype], _ptr(workspace), _nbytes(workspace),
+                                          _stream(stream))
+    return _check("bt_relu_fwd_compress_batch", st, check)
 
 
 def bt_compress_noalloc(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,

@@ -336,6 +336,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
                     if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + s_off[ps][lane];
                 }
+                bool bump = false;              // lane 0: this is the launch's last tile
                 if (pt == jb.tiles - 1 && lane == 0) {
                     const uint64_t nnz = base + s_agg[ps];
                     *jb.nnz_out        = nnz;
@@ -344,7 +345,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     const uint64_t capacity = jb.capacity;
                     // without a meeting: every CTA has published its count by now, so every CTA has read the sequence
                     // number, and the next launch on this workspace gets another tag
-                    if (pk + 1 == p.c.jobs) red_add_u64(p.c.ws_header + kHdrSeq, 1ull);
+                    bump = pk + 1 == p.c.jobs;
                     if (jb.dev_status) {
                         *reinterpret_cast<volatile int32_t *>(jb.dev_status) = aborted ? BT_ERR_TIMEOUT : (nnz > capacity ? BT_ERR_CAPACITY : BT_OK);
                         // a CTA that gives up from now on stores its BT_ERR_TIMEOUT after this word; one that gave
@@ -355,6 +356,35 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     }
                 }
                 __syncwarp();
+                if (__shfl_sync(kFull, bump ? 1 : 0, 0)) {
+                    // The launch's last tile.  The next launch on this workspace must get another tag, and the sequence
+                    // number may move only once every CTA has read it, i.e. has published a count.  The first G tiles
+                    // of the launch are one per CTA: wait for their counts (they have been out for a long time).
+                    bool seen[kMaxWindows];
+#pragma unroll
+                    for (int k = 0; k < kMaxWindows; ++k) seen[k] = lane + 32u * k >= G;
+                    bool           all = true;
+                    const uint64_t ts  = now_ns();
+                    for (;;) {
+                        bool miss = false;
+#pragma unroll
+                        for (int k = 0; k < kMaxWindows; ++k) {
+                            if (!seen[k]) {
+                                uint64_t x0, x1;
+                                ld_relaxed_2xu64(desc + 2 * static_cast<uint64_t>(lane + 32u * k), x0, x1);
+                                seen[k] = valid(x0, x1);
+                                miss |= !seen[k];
+                            }
+                        }
+                        if (!__any_sync(kFull, miss)) break;
+                        if (__any_sync(kFull, now_ns() - ts > wait_ns)) {
+                            all = false;
+                            break;
+                        }
+                        __nanosleep(200);
+                    }
+                    if (lane == 0) red_add_u64(p.c.ws_header + kHdrSeq, all ? 1ull : 1ull << 32);
+                }
                 if (lane == 0) {
                     s_base[ps] = base;
                     mbar_arrive(&s_ready[ps]);                       // the copiers may take the tile

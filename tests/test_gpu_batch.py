@@ -1,0 +1,93 @@
+"""The batched forms (bt_compress_batch, bt_relu_fwd_compress_batch): every tensor of a batch must get exactly what
+the oracle computes for that tensor alone -- the prefix restarts at each tensor -- whatever the mix of sizes (tensors
+of a fraction of a tile, of several waves of tiles, ragged, empty), whatever the number of tensors (more than one
+launch holds) and on a workspace that the batch before it left full of its own words."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2110_15362_b200 import binding as B
+from paper_2110_15362_b200 import workloads as W
+from tests.gpu_util import TDT, from_raw
+
+pytestmark = pytest.mark.gpu
+
+SIZES = [5, 4096, 0, 8192 * 3 + 17, 33, 16384 * 9, 1, 8192 * 160 + 4097, 4095, 8192 * 40, 65536 + 31]
+
+
+def run_batch(kind, sizes, seed, fused, want_y, ws=None, zeros=0.5):
+    dt = TDT[kind]
+    raws = [W.random_patterns(n, kind, zeros, seed=seed + 7 * k) for k, n in enumerate(sizes)]
+    xs = [from_raw(r, kind) if r.size else torch.empty(0, dtype=dt, device="cuda") for r in raws]
+    sts = [B.Stash(max(n, 1), dt)for n in sizes]
+    ys = [torch.empty_like(x) for x in xs] if want_y else None
+    items = B.batch_items(xs, sts, ys)
+    for k, n in enumerate(sizes):                                   # Stash(max(n, 1)) keeps pointers non-NULL; the count is n
+        items[k].n = n
+    if ws is None:
+        ws = torch.empty(B.bt_batch_workspace_bytes(sizes), dtype=torch.uint8, device="cuda")
+        ws.random_(0, 255)
+    (B.bt_relu_fwd_compress_batch if fused else B.bt_compress_batch)(items, dt, ws)
+    torch.cuda.synchronize()
+    return raws, sts, ys, ws
+
+
+def check_batch(oracle, kind, raws, sts, ys, fused):
+    for k, raw in enumerate(raws):
+        n = raw.size
+        st = sts[k]
+        assert st.status == B.BT_OK, (k, n)
+        if fused:
+            y_ref, c = oracle.relu_fwd_compress(raw, kind)
+        else:
+            y_ref, c = None, oracle.compress(raw)
+        assert st.nnz == c.nnz, (k, n)
+        if n == 0:
+            continue
+        assert np.array_equal(W.raw_numpy(st.bitmap)[:(n + 31) // 32].view(np.uint32), c.bitmap), (k, n)
+        assert np.array_equal(W.raw_numpy(st.chunk_prefix)[:(n + 4095) // 4096].view(np.uint64), c.prefix), (k, n)
+        assert np.array_equal(W.raw_numpy(st.values[:c.nnz]), c.values), (k, n)
+        if ys is not None:
+            assert np.array_equal(W.raw_numpy(ys[k]), y_ref), (k, n)
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16", "f16", "f64"])
+@pytest.mark.parametrize("fused,want_y", [(False, False), (True, False), (True, True)])
+def test_batch_equals_the_oracle_tensor_by_tensor(oracle, kind, fused, want_y):
+    raws, sts, ys, ws = run_batch(kind, SIZES, 4100, fused, want_y)
+    check_batch(oracle, kind, raws, sts, ys, fused)
+    # the same workspace again, other data, other sizes: nothing of the first batch may be taken for the second's
+    raws, sts, ys, _ = run_batch(kind, SIZES[::-1], 977, fused, want_y, ws=ws, zeros=0.8)
+    check_batch(oracle, kind, raws, sts, ys, fused)
+
+
+def test_more_tensors_than_one_launch_holds(oracle):
+    sizes = [4096 * (1 + k % 5) + k for k in range(2 * B.MAX_BATCH_PER_LAUNCH + 3)]
+    raws, sts, ys, _ = run_batch("f32", sizes, 31, False, False)
+    check_batch(oracle, "f32", raws, sts, ys, False)
+
+
+def test_batch_under_a_cta_limit(oracle):
+    B.bt_set_max_ctas(3)
+    try:
+        raws, sts, ys, _ = run_batch("bf16", SIZES, 555, True, True)
+    finally:
+        B.bt_set_max_ctas(0)
+    check_batch(oracle, "bf16", raws, sts, ys, True)
+
+
+def test_batch_argument_checks():
+    L = B.lib()
+    x = torch.zeros(64, device="cuda")
+    st = B.Stash(64, torch.float32)
+    ws = torch.empty(B.bt_batch_workspace_bytes([64, 64]), dtype=torch.uint8, device="cuda")
+    items = B.batch_items([x, x], [st, st], [x, x])
+    assert B.bt_compress_batch(items, torch.float32, ws, check=False) == B.BT_ERR_SHAPE          # the plain form has no y
+    items[1].y_out = None
+    assert B.bt_relu_fwd_compress_batch(items, torch.float32, ws, check=False) == B.BT_ERR_SHAPE  # y for all or none
+    items[0].y_out = None
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    assert B.bt_compress_batch(items, torch.float32, small, check=False) == B.BT_ERR_WORKSPACE
+    items[1].bitmap = None
+    assert B.bt_compress_batch(items, torch.float32, ws, check=False) == B.BT_ERR_NULL
+    assert L.bt_compress_batch(None, 0, B.BT_F32, None, 0, None) == B.BT_OK
