@@ -22,14 +22,20 @@
  *
  * General rules for every call below
  *   - All tensor pointers are DEVICE pointers unless a parameter says "host".
- *     The caller owns every buffer; the library allocates nothing, keeps no
- *     state between calls, and neither synchronises nor prints.
+ *     The caller owns every buffer; the library allocates nothing and neither
+ *     synchronises nor prints.  Nothing about a tensor or a call outlives the
+ *     call.  What the library does keep, all of it on the host: the calling
+ *     thread's CTA limit (bt_set_max_ctas, off by default), a process-wide
+ *     counter from which every compress launch draws its 64-bit tag, and, per
+ *     device, the address of bt_compress_noalloc's built-in scratch array.
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL
  *     for the default stream) on the current device.
  *   - Tensors are flat contiguous arrays of n elements (Algorithm 1 flattens
  *     the tensor first; the shape is the caller's metadata).
- *   - dense / values / y / gradient pointers and the bitmap pointer must be
- *     16-byte aligned, chunk_prefix and nnz_out 8-byte aligned.
+ *   - dense / values / y / gradient pointers must be 16-byte aligned, the
+ *     bitmap 4-byte aligned (a 16-byte aligned bitmap is read with wider
+ *     loads), chunk_prefix, nnz_out and the arena words 8-byte aligned, a
+ *     workspace 16-byte aligned.
  *   - The return value reports what the host can see: BT_OK, an argument
  *     error (nothing was launched), or BT_ERR_CUDA if the launch itself
  *     failed.  Conditions only the device can see are written to *dev_status
@@ -68,6 +74,11 @@ enum {
     BT_ERR_SHAPE = 9       /* a dimension the call cannot take (bt_maxpool2x2_*: odd or zero) */
 };
 
+/* ======================================================================================
+ * The codec proper: the size query, Algorithm 1, Algorithm 2, the fused ReLU forward and
+ * the ReLU backward from the bitmap (plus the workspace query the two compressors need).
+ * ====================================================================================== */
+
 /*
  * Size in bytes of the compressed form: 4*ceil(n/32) + nnz*sizeof(dtype) +
  * 8*ceil(n/4096).  This is M_b of section 3.2 (element bytes times the
@@ -79,14 +90,76 @@ size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype);
 
 /*
  * Bytes of device scratch bt_compress / bt_relu_fwd_compress need for n
- * elements (the tile descriptors of the single-pass scan plus a small header).
- * The contents need no initialisation and are unspecified after a call: a
- * word counts as written by the running call only if it carries that call's
- * 64-bit tag, which no other call shares.  Two
- * calls that run concurrently must not share a workspace.  No counterpart in
- * the paper (its scan is sequential).
+ * elements: the tile descriptors and per-wave totals of the single-pass scan
+ * plus a small header.  The contents need no initialisation and are
+ * unspecified after a call: a tile descriptor counts as written by the running
+ * call only if it carries that call's 64-bit tag, which no other call shares,
+ * and the per-wave totals are cleared by the running launch itself, before a
+ * grid-wide meeting that precedes the first addition to them.  Two calls that
+ * run concurrently must not share a workspace; calls ordered on the device
+ * (one stream, or events) may.  No counterpart in the paper (its scan is
+ * sequential).
  */
 size_t bt_workspace_bytes(uint64_t n);
+
+/*
+ * Algorithm 1 (dense -> bitmap).  Reads dense[0..n), writes bitmap
+ * (ceil(n/32) words), values[0..nnz), chunk_prefix (ceil(n/4096) entries) and
+ * *nnz_out.  values_capacity is the number of ELEMENTS the values buffer can
+ * hold; n always suffices.  If nnz exceeds it, stores past the capacity are
+ * suppressed, bitmap, chunk_prefix and *nnz_out are still complete and
+ * correct, and *dev_status = BT_ERR_CAPACITY, so the caller can run again with
+ * a buffer of nnz elements.  values[nnz..capacity) is left untouched or
+ * unspecified.  *dev_status = BT_ERR_TIMEOUT means an internal bounded wait
+ * gave up (two seconds without the data it waits for; every CTA then leaves
+ * the kernel) and every output is undefined; the workspace and the context
+ * stay usable and the next call runs normally.  The kernel is launched
+ * cooperatively (all its CTAs resident at once, one per SM at most).
+ */
+int bt_compress(const void *dense, uint64_t n, int dtype,
+                uint32_t *bitmap, void *values, uint64_t values_capacity,
+                uint64_t *chunk_prefix, uint64_t *nnz_out,
+                void *workspace, size_t workspace_bytes,
+                int32_t *dev_status, void *stream);
+
+/*
+ * Algorithm 2 (bitmap -> dense).  dense_out[i] = bit i set ? the next value :
+ * all-zero bits.  Chunks are decoded independently from chunk_prefix; values
+ * must hold at least the nnz elements the bitmap calls for.
+ */
+int bt_decompress(const uint32_t *bitmap, const void *values,
+                  const uint64_t *chunk_prefix, uint64_t n, int dtype,
+                  void *dense_out, void *stream);
+
+/*
+ * ReLU forward fused with Algorithm 1: y[i] = (x[i] <= 0) ? +0 : x[i] under
+ * IEEE comparison (so -0, negatives and -inf give +0 and a NaN passes through
+ * with its payload), and y is stashed in compressed form in the same pass
+ * (ReLU is the source of the sparsity, section 3.1; the activation is saved in
+ * the forward pass, section 3.2).  y_out may be NULL (only the stash is
+ * written) and may alias pre_act (in-place ReLU).  Other parameters as
+ * bt_compress.
+ */
+int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out,
+                         uint32_t *bitmap, void *values, uint64_t values_capacity,
+                         uint64_t *chunk_prefix, uint64_t *nnz_out,
+                         void *workspace, size_t workspace_bytes,
+                         int32_t *dev_status, void *stream);
+
+/*
+ * ReLU backward from the stash: grad_in[i] = bit i set ? grad_out[i] : +0.
+ * The backward pass restores activations to form gradients (section 3.2); for
+ * ReLU itself only the bitmap is needed.  A select, not a multiply: masked
+ * lanes are +0 even where grad_out is negative, infinite or NaN.  grad_in may
+ * alias grad_out.
+ */
+int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
+                            uint64_t n, int dtype, void *grad_in, void *stream);
+
+/* ======================================================================================
+ * Everything below is an extension around the six calls above: batched, fused, narrowing,
+ * pooling, arena and host-buffer forms.  Each says what in the paper it serves.
+ * ====================================================================================== */
 
 /*
  * Batched forms of bt_compress and bt_relu_fwd_compress: `count` tensors of one element type in ONE
@@ -137,47 +210,6 @@ int bt_relu_fwd_compress_batch(const bt_batch_item *items /* host */, uint32_t c
  * No counterpart in the paper.
  */
 int bt_set_max_ctas(int max_ctas);
-
-/*
- * Algorithm 1 (dense -> bitmap).  Reads dense[0..n), writes bitmap
- * (ceil(n/32) words), values[0..nnz), chunk_prefix (ceil(n/4096) entries) and
- * *nnz_out.  values_capacity is the number of ELEMENTS the values buffer can
- * hold; n always suffices.  If nnz exceeds it, stores past the capacity are
- * suppressed, bitmap, chunk_prefix and *nnz_out are still complete and
- * correct, and *dev_status = BT_ERR_CAPACITY, so the caller can run again with
- * a buffer of nnz elements.  values[nnz..capacity) is left untouched or
- * unspecified.  *dev_status = BT_ERR_TIMEOUT means an internal bounded wait
- * gave up and every output is undefined.
- */
-int bt_compress(const void *dense, uint64_t n, int dtype,
-                uint32_t *bitmap, void *values, uint64_t values_capacity,
-                uint64_t *chunk_prefix, uint64_t *nnz_out,
-                void *workspace, size_t workspace_bytes,
-                int32_t *dev_status, void *stream);
-
-/*
- * Algorithm 2 (bitmap -> dense).  dense_out[i] = bit i set ? the next value :
- * all-zero bits.  Chunks are decoded independently from chunk_prefix; values
- * must hold at least the nnz elements the bitmap calls for.
- */
-int bt_decompress(const uint32_t *bitmap, const void *values,
-                  const uint64_t *chunk_prefix, uint64_t n, int dtype,
-                  void *dense_out, void *stream);
-
-/*
- * ReLU forward fused with Algorithm 1: y[i] = (x[i] <= 0) ? +0 : x[i] under
- * IEEE comparison (so -0, negatives and -inf give +0 and a NaN passes through
- * with its payload), and y is stashed in compressed form in the same pass
- * (ReLU is the source of the sparsity, section 3.1; the activation is saved in
- * the forward pass, section 3.2).  y_out may be NULL (only the stash is
- * written) and may alias pre_act (in-place ReLU).  Other parameters as
- * bt_compress.
- */
-int bt_relu_fwd_compress(const void *pre_act, uint64_t n, int dtype, void *y_out,
-                         uint32_t *bitmap, void *values, uint64_t values_capacity,
-                         uint64_t *chunk_prefix, uint64_t *nnz_out,
-                         void *workspace, size_t workspace_bytes,
-                         int32_t *dev_status, void *stream);
 
 /*
  * Activation pruning fused with Algorithm 1 (section 4, "Combining BitTrain
@@ -248,7 +280,7 @@ int bt_prune_fwd_compress_narrow(const void *x, uint64_t n, int to_dtype, float 
  * activation).  bt_maxpool2x2_bwd needs only the codes: grad_in (planes x
  * height x width) gets grad_out[o] at the coded position of window o and +0
  * at the other three; every element of grad_in is written.  x / y and
- * grad_out / grad_in must not overlap.  Pointers 16-byte aligned.
+ * grad_out / grad_in must not overlap.  Tensors 16-byte aligned, codes and bitmaps 4-byte.
  */
 int bt_maxpool2x2_fwd(const void *x, uint64_t planes, uint64_t height, uint64_t width, int dtype,
                       void *y, uint32_t *codes, void *stream);
@@ -317,16 +349,6 @@ int bt_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values, const ui
 int bt_mask_compress(const void *x, uint64_t n, int dtype,
                      const uint32_t *mask_bitmap, const uint64_t *mask_chunk_prefix,
                      void *y_out, void *values, uint64_t values_capacity, void *stream);
-
-/*
- * ReLU backward from the stash: grad_in[i] = bit i set ? grad_out[i] : +0.
- * The backward pass restores activations to form gradients (section 3.2); for
- * ReLU itself only the bitmap is needed.  A select, not a multiply: masked
- * lanes are +0 even where grad_out is negative, infinite or NaN.  grad_in may
- * alias grad_out.
- */
-int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out,
-                            uint64_t n, int dtype, void *grad_in, void *stream);
 
 /*
  * bt_compress for callers that cannot allocate device memory.  (The paper has
@@ -430,9 +452,14 @@ int bt_relu6_bwd_from_stash_arena(const uint32_t *bitmap, const void *arena, con
  * bt_host_staging_bytes(n, dtype) bytes, 256-byte aligned, owned by the caller
  * and free for reuse after the call.  Each call copies its inputs to the
  * staging area, runs the same kernels as the device forms, copies the results
- * back and SYNCHRONISES the stream before it returns (the packed values can be
- * copied only once nnz is known), so device-side conditions (BT_ERR_CAPACITY,
- * BT_ERR_TIMEOUT) arrive in the return value.  host_values_capacity counts
+ * back and SYNCHRONISES the stream before it returns, so device-side conditions
+ * (BT_ERR_CAPACITY, BT_ERR_TIMEOUT) arrive in the return value.  The packed
+ * values are nnz elements, a number only the device knows: into a page-locked
+ * host_values buffer (16-byte aligned) the device writes exactly that many
+ * itself and the call synchronises once, at its end; for pageable memory the
+ * call synchronises a first time to learn nnz, then copies.  On any error
+ * after the first copy was enqueued the stream is synchronised before the call
+ * returns: nothing of a finished call is still pending on the caller's memory.  host_values_capacity counts
  * elements; if nnz exceeds it the first host_values_capacity values are
  * copied, *host_nnz holds the true count and BT_ERR_CAPACITY is returned.
  * Otherwise arguments mean what they mean in the device forms.

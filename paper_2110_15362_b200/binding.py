@@ -62,82 +62,86 @@ def lib() -> ctypes.CDLL:
     """Load libbittrain.so (built in-tree by build.build_library()).  No fallback."""
     global _lib
     if _lib is None:
-        path = library_path()
-        if not os.path.exists(path):
-            raise ImportError(f"{path} is missing: build it with "
-                              "`python -m paper_2110_15362_b200.build` (needs nvcc); there is no CPU fallback")
-        L = ctypes.CDLL(path)
-        u64, vp, i32, sz = ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
-        L.bt_compressed_bytes.restype = sz
-        L.bt_compressed_bytes.argtypes = [u64, u64, i32]
-        L.bt_set_max_ctas.restype = i32
-        L.bt_set_max_ctas.argtypes = [i32]
-        L.bt_workspace_bytes.restype = sz
-        L.bt_workspace_bytes.argtypes = [u64]
-        L.bt_compress.restype = i32
-        L.bt_compress.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
-        L.bt_batch_workspace_bytes.restype = sz
-        L.bt_batch_workspace_bytes.argtypes = [ctypes.POINTER(u64), ctypes.c_uint32]
-        for name in ("bt_compress_batch", "bt_relu_fwd_compress_batch"):
-            getattr(L, name).restype = i32
-            getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp, sz, vp]
-        L.bt_decompress.restype = i32
-        L.bt_decompress.argtypes = [vp, vp, vp, u64, i32, vp, vp]
-        L.bt_relu_fwd_compress.restype = i32
-        L.bt_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
-        L.bt_relu_bwd_from_bitmap.restype = i32
-        L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
-        L.bt_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
-        L.bt_prune_fwd_compress.restype = i32
-        L.bt_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp, u64, vp]
-        L.bt_mask_compress.restype = i32
-        L.bt_compress_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.bt_compress_arena.restype = i32
-        L.bt_prune_fwd_compress_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.bt_prune_fwd_compress_arena.restype = i32
-        L.bt_decompress_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
-        L.bt_decompress_arena.restype = i32
-        L.bt_relu6_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
-        L.bt_relu6_fwd_compress.restype = i32
-        L.bt_relu6_bwd_from_stash.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
-        L.bt_relu6_bwd_from_stash.restype = i32
-        L.bt_compress_narrow.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
-        L.bt_compress_narrow.restype = i32
-        L.bt_prune_fwd_compress_narrow.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
-        L.bt_prune_fwd_compress_narrow.restype = i32
-        L.bt_decompress_widen.argtypes = [vp, vp, vp, u64, i32, vp, vp]
-        L.bt_decompress_widen.restype = i32
-        L.bt_maxpool2x2_fwd.argtypes = [vp, u64, u64, u64, i32, vp, vp, vp]
-        L.bt_maxpool2x2_fwd.restype = i32
-        L.bt_maxpool2x2_bwd.argtypes = [vp, vp, u64, u64, u64, i32, vp, vp]
-        L.bt_maxpool2x2_bwd.restype = i32
-        L.bt_maxpool2x2_bwd_masked.argtypes = [vp, vp, vp, u64, u64, u64, i32, vp, vp]
-        L.bt_maxpool2x2_bwd_masked.restype = i32
-        L.bt_compress_narrow_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.bt_compress_narrow_arena.restype = i32
-        L.bt_prune_fwd_compress_narrow_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz,
-                                                         vp, vp]
-        L.bt_prune_fwd_compress_narrow_arena.restype = i32
-        L.bt_decompress_widen_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
-        L.bt_decompress_widen_arena.restype = i32
-        L.bt_relu6_fwd_compress_arena.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
-        L.bt_relu6_fwd_compress_arena.restype = i32
-        L.bt_relu6_bwd_from_stash_arena.argtypes = [vp, vp, vp, vp, vp, u64, i32, vp, vp]
-        L.bt_relu6_bwd_from_stash_arena.restype = i32
-        L.bt_compress_noalloc.restype = i32
-        L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
-        L.bt_host_staging_bytes.restype = sz
-        L.bt_host_staging_bytes.argtypes = [u64, i32]
-        L.bt_compress_host.restype = i32
-        L.bt_compress_host.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp]
-        L.bt_decompress_host.restype = i32
-        L.bt_decompress_host.argtypes = [vp, vp, vp, u64, u64, i32, vp, vp, sz, vp]
-        L.bt_relu_fwd_compress_host.restype = i32
-        L.bt_relu_fwd_compress_host.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp]
-        L.bt_relu_bwd_from_bitmap_host.restype = i32
-        L.bt_relu_bwd_from_bitmap_host.argtypes = [vp, vp, u64, i32, vp, vp, sz, vp]
-        _lib = L
+        _lib = load_library(library_path())
     return _lib
+
+
+def load_library(path: str) -> ctypes.CDLL:
+    """Open a build of the library and declare the C ABI's signatures on it."""
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with "
+                          "`python -m paper_2110_15362_b200.build` (needs nvcc); there is no CPU fallback")
+    L = ctypes.CDLL(path)
+    u64, vp, i32, sz = ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    L.bt_compressed_bytes.restype = sz
+    L.bt_compressed_bytes.argtypes = [u64, u64, i32]
+    L.bt_set_max_ctas.restype = i32
+    L.bt_set_max_ctas.argtypes = [i32]
+    L.bt_workspace_bytes.restype = sz
+    L.bt_workspace_bytes.argtypes = [u64]
+    L.bt_compress.restype = i32
+    L.bt_compress.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+    L.bt_batch_workspace_bytes.restype = sz
+    L.bt_batch_workspace_bytes.argtypes = [ctypes.POINTER(u64), ctypes.c_uint32]
+    for name in ("bt_compress_batch", "bt_relu_fwd_compress_batch"):
+        getattr(L, name).restype = i32
+        getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp, sz, vp]
+    L.bt_decompress.restype = i32
+    L.bt_decompress.argtypes = [vp, vp, vp, u64, i32, vp, vp]
+    L.bt_relu_fwd_compress.restype = i32
+    L.bt_relu_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+    L.bt_relu_bwd_from_bitmap.restype = i32
+    L.bt_relu_bwd_from_bitmap.argtypes = [vp, vp, u64, i32, vp, vp]
+    L.bt_prune_fwd_compress.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+    L.bt_prune_fwd_compress.restype = i32
+    L.bt_mask_compress.argtypes = [vp, u64, i32, vp, vp, vp, vp, u64, vp]
+    L.bt_mask_compress.restype = i32
+    L.bt_compress_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.bt_compress_arena.restype = i32
+    L.bt_prune_fwd_compress_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.bt_prune_fwd_compress_arena.restype = i32
+    L.bt_decompress_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
+    L.bt_decompress_arena.restype = i32
+    L.bt_relu6_fwd_compress.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+    L.bt_relu6_fwd_compress.restype = i32
+    L.bt_relu6_bwd_from_stash.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
+    L.bt_relu6_bwd_from_stash.restype = i32
+    L.bt_compress_narrow.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+    L.bt_compress_narrow.restype = i32
+    L.bt_prune_fwd_compress_narrow.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, sz, vp, vp]
+    L.bt_prune_fwd_compress_narrow.restype = i32
+    L.bt_decompress_widen.argtypes = [vp, vp, vp, u64, i32, vp, vp]
+    L.bt_decompress_widen.restype = i32
+    L.bt_maxpool2x2_fwd.argtypes = [vp, u64, u64, u64, i32, vp, vp, vp]
+    L.bt_maxpool2x2_fwd.restype = i32
+    L.bt_maxpool2x2_bwd.argtypes = [vp, vp, u64, u64, u64, i32, vp, vp]
+    L.bt_maxpool2x2_bwd.restype = i32
+    L.bt_maxpool2x2_bwd_masked.argtypes = [vp, vp, vp, u64, u64, u64, i32, vp, vp]
+    L.bt_maxpool2x2_bwd_masked.restype = i32
+    L.bt_compress_narrow_arena.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.bt_compress_narrow_arena.restype = i32
+    L.bt_prune_fwd_compress_narrow_arena.argtypes = [vp, u64, i32, ctypes.c_float, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz,
+                                                     vp, vp]
+    L.bt_prune_fwd_compress_narrow_arena.restype = i32
+    L.bt_decompress_widen_arena.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp]
+    L.bt_decompress_widen_arena.restype = i32
+    L.bt_relu6_fwd_compress_arena.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, vp, vp, sz, vp, vp]
+    L.bt_relu6_fwd_compress_arena.restype = i32
+    L.bt_relu6_bwd_from_stash_arena.argtypes = [vp, vp, vp, vp, vp, u64, i32, vp, vp]
+    L.bt_relu6_bwd_from_stash_arena.restype = i32
+    L.bt_compress_noalloc.restype = i32
+    L.bt_compress_noalloc.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, vp]
+    L.bt_host_staging_bytes.restype = sz
+    L.bt_host_staging_bytes.argtypes = [u64, i32]
+    L.bt_compress_host.restype = i32
+    L.bt_compress_host.argtypes = [vp, u64, i32, vp, vp, u64, vp, vp, vp, sz, vp]
+    L.bt_decompress_host.restype = i32
+    L.bt_decompress_host.argtypes = [vp, vp, vp, u64, u64, i32, vp, vp, sz, vp]
+    L.bt_relu_fwd_compress_host.restype = i32
+    L.bt_relu_fwd_compress_host.argtypes = [vp, u64, i32, vp, vp, vp, u64, vp, vp, vp, sz, vp]
+    L.bt_relu_bwd_from_bitmap_host.restype = i32
+    L.bt_relu_bwd_from_bitmap_host.argtypes = [vp, vp, u64, i32, vp, vp, sz, vp]
+    return L
 
 
 def _ptr(t: Optional[torch.Tensor]):

@@ -133,6 +133,12 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
 
 }  // namespace
 
+#ifdef BT_BOUNDS_CHECK
+namespace bt {
+__device__ unsigned long long g_bounds_violations = 0;
+}
+#endif
+
 extern "C" {
 
 size_t bt_compressed_bytes(uint64_t n, uint64_t nnz, int dtype)
@@ -147,6 +153,21 @@ int bt_set_max_ctas(int max_ctas)
     if (max_ctas < 0) return -1;
     return static_cast<int>(bt::set_compress_max_ctas(static_cast<uint32_t>(max_ctas)));
 }
+
+#ifdef BT_BOUNDS_CHECK
+// Checking build only: the number of stores the kernels skipped because they fell outside their buffer, since
+// the last reset.  Synchronises the device.  Returns a negative number if the runtime refuses the copy.
+long long bt_test_bounds_violations(int reset)
+{
+    unsigned long long v = 0;
+    if (cudaMemcpyFromSymbol(&v, bt::g_bounds_violations, sizeof(v)) != cudaSuccess) return -1;
+    if (reset) {
+        const unsigned long long zero = 0;
+        if (cudaMemcpyToSymbol(bt::g_bounds_violations, &zero, sizeof(zero)) != cudaSuccess) return -1;
+    }
+    return static_cast<long long>(v);
+}
+#endif
 
 #ifdef BT_TEST_HOOKS
 // Test builds only (never the product library): the bound of every wait inside the compress kernels, so that a
@@ -235,7 +256,7 @@ int bt_relu6_bwd_from_stash(const uint32_t *bitmap, const void *values, const ui
     if (es == 0) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !chunk_prefix || !grad_out || !grad_in) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(grad_out, 16) ||
+    if (!aligned(bitmap, 4) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(grad_out, 16) ||
         !aligned(grad_in, 16))
         return BT_ERR_ALIGN;
     return bt::launch_relu6_bwd(bitmap, values, nullptr, chunk_prefix, grad_out, n, dtype, grad_in,
@@ -274,7 +295,7 @@ int bt_decompress_arena(const uint32_t *bitmap, const void *arena, const uint64_
     if (es == 0) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !chunk_prefix || !dense_out || !arena || !values_offset) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
+    if (!aligned(bitmap, 4) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
         !aligned(dense_out, 16))
         return BT_ERR_ALIGN;
     return bt::launch_decompress(bitmap, arena, values_offset, chunk_prefix, n, es, dense_out,
@@ -327,7 +348,7 @@ int bt_decompress_widen_arena(const uint32_t *bitmap, const void *arena, const u
     if (from_dtype != BT_F16 && from_dtype != BT_BF16) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !chunk_prefix || !dense_out || !arena || !values_offset) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
+    if (!aligned(bitmap, 4) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
         !aligned(dense_out, 16))
         return BT_ERR_ALIGN;
     return bt::launch_decompress_widen(bitmap, arena, values_offset, chunk_prefix, n, from_dtype, dense_out,
@@ -344,7 +365,7 @@ int bt_relu6_bwd_from_stash_arena(const uint32_t *bitmap, const void *arena, con
     if (es == 0) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !chunk_prefix || !grad_out || !grad_in || !arena || !values_offset) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
+    if (!aligned(bitmap, 4) || !aligned(arena, 16) || !aligned(values_offset, 8) || !aligned(chunk_prefix, 8) ||
         !aligned(grad_out, 16) || !aligned(grad_in, 16))
         return BT_ERR_ALIGN;
     return bt::launch_relu6_bwd(bitmap, arena, values_offset, chunk_prefix, grad_out, n, dtype, grad_in,
@@ -360,7 +381,7 @@ int bt_decompress(const uint32_t *bitmap, const void *values, const uint64_t *ch
     if (es == 0) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !chunk_prefix || !dense_out) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
+    if (!aligned(bitmap, 4) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
         return BT_ERR_ALIGN;
     // values may be NULL only when the bitmap has no set bit; the kernel then never reads it
     return bt::launch_decompress(bitmap, values, nullptr, chunk_prefix, n, es, dense_out, static_cast<cudaStream_t>(stream)) ==
@@ -375,7 +396,7 @@ int bt_decompress_widen(const uint32_t *bitmap, const void *values, const uint64
     if (from_dtype != BT_F16 && from_dtype != BT_BF16) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !chunk_prefix || !dense_out) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
+    if (!aligned(bitmap, 4) || !aligned(values, 16) || !aligned(chunk_prefix, 8) || !aligned(dense_out, 16))
         return BT_ERR_ALIGN;
     return bt::launch_decompress_widen(bitmap, values, nullptr, chunk_prefix, n, from_dtype, dense_out,
                                        static_cast<cudaStream_t>(stream)) == cudaSuccess
@@ -391,7 +412,7 @@ int bt_mask_compress(const void *x, uint64_t n, int dtype, const uint32_t *mask_
     if (n == 0) return BT_OK;
     if (!x || !mask_bitmap || !mask_chunk_prefix) return BT_ERR_NULL;
     if (!values && values_capacity != 0) return BT_ERR_NULL;
-    if (!aligned(x, 16) || !aligned(y_out, 16) || !aligned(mask_bitmap, 16) || !aligned(values, 16) ||
+    if (!aligned(x, 16) || !aligned(y_out, 16) || !aligned(mask_bitmap, 4) || !aligned(values, 16) ||
         !aligned(mask_chunk_prefix, 8))
         return BT_ERR_ALIGN;
     return bt::launch_mask_gather(x, mask_bitmap, mask_chunk_prefix, n, es, y_out, values, values_capacity,
@@ -452,7 +473,7 @@ int bt_relu_bwd_from_bitmap(const uint32_t *bitmap, const void *grad_out, uint64
     if (es == 0) return BT_ERR_DTYPE;
     if (n == 0) return BT_OK;
     if (!bitmap || !grad_out || !grad_in) return BT_ERR_NULL;
-    if (!aligned(bitmap, 16) || !aligned(grad_out, 16) || !aligned(grad_in, 16)) return BT_ERR_ALIGN;
+    if (!aligned(bitmap, 4) || !aligned(grad_out, 16) || !aligned(grad_in, 16)) return BT_ERR_ALIGN;
     return bt::launch_relu_bwd(bitmap, grad_out, n, es, grad_in, static_cast<cudaStream_t>(stream)) == cudaSuccess
                ? BT_OK
                : BT_ERR_CUDA;

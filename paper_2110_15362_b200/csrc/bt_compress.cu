@@ -76,7 +76,6 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     constexpr int kSteps         = kSeg / 32;
     constexpr int kChunksPerTile = kTile / BT_CHUNK_ELEMS;
     constexpr int kWarpsPerChunk = BT_CHUNK_ELEMS / kSeg;
-    constexpr int kCompactThreads = kWarps * 32;
     // warp roles
     constexpr int kFirstCopier = kWarps;
     constexpr int kScanWarp    = kWarps + kCopiers;       // and kScanWarp + 1
@@ -152,12 +151,15 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     // count is added.  Every CTA zeroes a share and the grid meets once, here, before any warp takes up its role;
     // the first two bulk copies are on their way meanwhile, so the meeting costs a launch next to nothing.
     const bool     multi  = num_tiles > G;
+    // the part of the workspace behind its header, as large as the size query promises the caller
+    const Extent   wsx    = extent_of(a.ws_desc, compress_workspace_bytes((n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) - kWsHeaderBytes);
     uint32_t       it_pre = 0;                    // bulk copies issued before the meeting
     if (multi) {
         if (warp == kLoadWarp && lane == 0) {
             for (; it_pre < 2u && tile_of(it_pre) < num_tiles; ++it_pre) issue_load(it_pre);
         }
-        for (uint32_t i = cta * blockDim.x + tid; i < a.ws_waves; i += G * blockDim.x) a.ws_desc[i] = 0;
+        for (uint32_t i = cta * blockDim.x + tid; i < a.ws_waves; i += G * blockDim.x)
+            if (wsx.holds(a.ws_desc + i, 8)) a.ws_desc[i] = 0;
         cooperative_groups::this_grid().sync();
     }
 
@@ -247,11 +249,11 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 }
                 const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
                 if (lane == 0) {
-                    st_relaxed_2xu64(desc + 2 * tile_of(j), tag_w0 | agg, tag_w1 | agg);
+                    if (wsx.holds(desc + 2 * tile_of(j), 16)) st_relaxed_2xu64(desc + 2 * tile_of(j), tag_w0 | agg, tag_w1 | agg);
                     s_agg[s] = agg;
                 }
                 if (lane < kWarps) s_off[s][lane] = inc - c;
-                if (multi && lane == 0) red_add_u64(wave_total + j, (1ull << kCountShift) + agg);
+                if (multi && lane == 0 && wsx.holds(wave_total + j, 8)) red_add_u64(wave_total + j, (1ull << kCountShift) + agg);
             }
             if (j >= 2) {
                 // ---- (c): tile j - 2 <= last_it
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                     for (int k = 0; k < kMaxWindows; ++k) missing |= !valid(d0[k], d1[k]);
                     if (!__any_sync(kFull, missing)) break;
                     __nanosleep(100);
-                    if ((++polls & 255u) == 0) {
+                    if ((++polls & 255u) == 0 || (kTestHooks && wait_ns < kStrictLimitNs)) {
                         if (t0 == 0) t0 = now_ns();
                         if (__any_sync(kFull, (now_ns() - t0 > wait_ns) || ld_relaxed_u64(a.ws_header + kHdrAbort) == tag)) {
                             failed = true;
@@ -290,7 +292,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 // exclusive count in front of each chunk of that tile
                 if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
                     const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
-                    if (ch < chunks_total) a.prefix[ch] = base + s_off[ps][lane];
+                    if (ch < chunks_total && extent_of(a.prefix, 8 * chunks_total).holds(a.prefix + ch, 8)) a.prefix[ch] = base + s_off[ps][lane];
                 }
                 if (pt == num_tiles - 1 && lane == 0) {
                     const uint64_t nnz = base + s_agg[ps];
@@ -355,6 +357,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(a.values) + c0);
             capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(V) : 0;
         }
+        const Extent vx = extent_of(vals, capacity * sizeof(V));
         for (uint32_t it = 0;; ++it) {
             if (tile_of(it) >= num_tiles) break;
             const uint32_t s = it % kStages;
@@ -367,9 +370,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
                 const uint32_t cnt  = s_cnt[s][seg];
                 const uint64_t dst  = base + s_off[s][seg];
                 if (dst + cnt <= capacity)
-                    copy_out_segment<U, CAST, false>(pseg, lane, cnt, vals + dst, 0);
+                    copy_out_segment<U, CAST, false>(pseg, lane, cnt, vals + dst, 0, vx);
                 else
-                    copy_out_segment<U, CAST, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
+                    copy_out_segment<U, CAST, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0, vx);
             }
             __syncwarp();
             asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
@@ -381,6 +384,8 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     // ---------------------------------------------------------------- compactor warps
     const uint32_t lt          = lanemask_lt();
     const uint64_t words_total = (n + 31) >> 5;
+    const Extent   bx          = extent_of(a.bitmap, 4 * words_total);
+    const Extent   yx          = extent_of(a.y, n * sizeof(U));
     for (uint32_t it = 0;; ++it) {
         const uint64_t t64 = tile_of(it);
         if (t64 >= num_tiles) break;
@@ -393,12 +398,15 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             break;
         }
         if (n - first < static_cast<uint64_t>(kTile)) {
-            // ragged last tile: fetch what the 16-byte granular bulk copy left out, zero the rest
+            // Ragged last tile: each warp completes its own segment -- what the 16-byte granular bulk copy left out,
+            // zeros behind the end of the tensor -- and meets no other warp over it.  (A barrier among the compactor
+            // warps here would never open if one of them had left the kernel because its wait ran out.)
             const uint32_t have    = static_cast<uint32_t>(n - first);
             const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
-            for (uint32_t e = by_bulk + tid; e < static_cast<uint32_t>(kTile); e += kCompactThreads)
+            const uint32_t seg0    = warp * kSeg;
+            for (uint32_t e = (by_bulk > seg0 ? by_bulk : seg0) + lane; e < seg0 + kSeg; e += 32)
                 tile[e] = (e < have) ? src[first + e] : U(0);
-            asm volatile("bar.sync %0, %1;" ::"n"(kBarWorkers), "n"(kCompactThreads) : "memory");
+            __syncwarp();
         }
 
         // ---- in-place compaction of this warp's segment
@@ -412,12 +420,12 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
         const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
         uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau);
+            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau, yx);
         else
-            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau);
+            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau, yx);
         if (lane < kSteps) {
             const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * kSteps + lane;
-            if (w < words_total) a.bitmap[w] = word;
+            if (w < words_total && bx.holds(a.bitmap + w, 4)) a.bitmap[w] = word;
         }
         __syncwarp();
         if (lane == 0) {

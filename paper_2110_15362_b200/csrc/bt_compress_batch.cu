@@ -111,7 +111,6 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     constexpr int kTile           = kWarps * kSeg;
     constexpr int kChunksPerTile  = kTile / BT_CHUNK_ELEMS;
     constexpr int kWarpsPerChunk  = BT_CHUNK_ELEMS / kSeg;
-    constexpr int kCompactThreads = kWarps * 32;
     // warp roles
     constexpr int kFirstCopier   = kWarps;
     constexpr int kScanWarp      = kWarps + kCopiers;       // and kScanWarp + 1
@@ -168,8 +167,10 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     // Tensors of more than one wave use wave totals: sums made by reductions, whose words must be zero before the
     // first count is added.  Every CTA zeroes a share and the grid meets once, here, before any warp takes up its
     // role; the first two bulk copies are on their way meanwhile.
+    const Extent wsx = extent_of(p.c.ws_total, 8 * p.c.ws_words);
     if (meet) {
-        for (uint32_t i = cta * blockDim.x + tid; i < p.c.ws_totals; i += G * blockDim.x) p.c.ws_total[i] = 0;
+        for (uint32_t i = cta * blockDim.x + tid; i < p.c.ws_totals; i += G * blockDim.x)
+            if (wsx.holds(p.c.ws_total + i, 8)) p.c.ws_total[i] = 0;
         cooperative_groups::this_grid().sync();
     }
 
@@ -289,11 +290,13 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 }
                 const uint32_t agg = __shfl_sync(kFull, inc, kWarps - 1);
                 if (lane == 0) {
-                    st_relaxed_2xu64(desc + 2 * (static_cast<uint64_t>(p.job[cur.k].desc0) + cur.tile(G)), tag_w0 | agg, tag_w1 | agg);
+                    uint64_t *const d = desc + 2 * (static_cast<uint64_t>(p.job[cur.k].desc0) + cur.tile(G));
+                    if (wsx.holds(d, 16)) st_relaxed_2xu64(d, tag_w0 | agg, tag_w1 | agg);
                     s_agg[s] = agg;
                 }
                 if (lane < kWarps) s_off[s][lane] = inc - c;
-                if (cur.tiles > G && lane == 0) red_add_u64(wave_total + p.job[cur.k].total0 + cur.j, (1ull << kCountShift) + agg);
+                if (cur.tiles > G && lane == 0 && wsx.holds(wave_total + p.job[cur.k].total0 + cur.j, 8))
+                    red_add_u64(wave_total + p.job[cur.k].total0 + cur.j, (1ull << kCountShift) + agg);
             }
             if (i >= 2) {
                 // ---- (c): this warp's previous tile, (pk, pj, pv)
@@ -306,7 +309,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     for (int k = 0; k < kMaxWindows; ++k) missing |= !valid(d0[k], d1[k]);
                     if (!__any_sync(kFull, missing)) break;
                     __nanosleep(100);
-                    if ((++polls & 255u) == 0 || wait_ns < 1000000ull) {
+                    if ((++polls & 255u) == 0 || (kTestHooks && wait_ns < kStrictLimitNs)) {
                         if (t0 == 0) t0 = now_ns();
                         if (__any_sync(kFull, (now_ns() - t0 > wait_ns) || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag)) {
                             failed = true;
@@ -334,7 +337,8 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 // exclusive count in front of each chunk of that tile
                 if (lane < kWarps && (lane % kWarpsPerChunk) == 0) {
                     const uint64_t ch = pt * kChunksPerTile + lane / kWarpsPerChunk;
-                    if (ch < (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS) jb.prefix[ch] = base + s_off[ps][lane];
+                    const uint64_t chunks_total = (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
+                    if (ch < chunks_total && extent_of(jb.prefix, 8 * chunks_total).holds(jb.prefix + ch, 8)) jb.prefix[ch] = base + s_off[ps][lane];
                 }
                 bool bump = false;              // lane 0: this is the launch's last tile
                 if (pt == jb.tiles - 1 && lane == 0) {
@@ -430,7 +434,8 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort, wait_ns)) break;
             V *const       vals     = static_cast<V *>(p.job[w.k].values);
             const uint64_t capacity = p.job[w.k].capacity;
-            const uint64_t base = s_base[s];
+            const Extent   vx       = extent_of(vals, capacity * sizeof(V));
+            const uint64_t base     = s_base[s];
 #pragma unroll
             for (int qq = 0; qq < kSegsPerCopier; ++qq) {
                 const uint32_t seg  = copier * kSegsPerCopier + qq;
@@ -438,9 +443,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 const uint32_t cnt  = s_cnt[s][seg];
                 const uint64_t dst  = base + s_off[s][seg];
                 if (dst + cnt <= capacity)
-                    copy_out_segment<U, 0, false>(pseg, lane, cnt, vals + dst, 0);
+                    copy_out_segment<U, 0, false>(pseg, lane, cnt, vals + dst, 0, vx);
                 else
-                    copy_out_segment<U, 0, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0);
+                    copy_out_segment<U, 0, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0, vx);
             }
             __syncwarp();
             asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
@@ -465,13 +470,16 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             break;
         }
         if (n - first < static_cast<uint64_t>(kTile)) {
-            // ragged last tile: fetch what the 16-byte granular bulk copy left out, zero the rest
+            // Ragged last tile: each warp completes its own segment -- what the 16-byte granular bulk copy left out,
+            // zeros behind the end of the tensor -- and meets no other warp over it.  (A barrier among the compactor
+            // warps here would never open if one of them had left the kernel because its wait ran out.)
             const U *const src     = static_cast<const U *>(jb.src);
             const uint32_t have    = static_cast<uint32_t>(n - first);
             const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
-            for (uint32_t e = by_bulk + tid; e < static_cast<uint32_t>(kTile); e += kCompactThreads)
+            const uint32_t seg0    = warp * kSeg;
+            for (uint32_t e = (by_bulk > seg0 ? by_bulk : seg0) + lane; e < seg0 + kSeg; e += 32)
                 tile[e] = (e < have) ? src[first + e] : U(0);
-            asm volatile("bar.sync %0, %1;" ::"n"(kBarWorkers), "n"(kCompactThreads) : "memory");
+            __syncwarp();
         }
 
         // ---- in-place compaction of this warp's segment
@@ -482,15 +490,16 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
             y      = static_cast<U *>(jb.y) + e0;
             yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
         }
+        const Extent   yx       = extent_of(jb.y, n * sizeof(U));
         const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
         uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, FUSED, WRITE_Y, false, kSeg / 32>(seg_addr, word, lane, lanemask_lt(), y, yvalid, p.c.tau);
+            run = compact_segment<U, FUSED, WRITE_Y, false, kSeg / 32>(seg_addr, word, lane, lanemask_lt(), y, yvalid, p.c.tau, yx);
         else
-            run = compact_segment<U, FUSED, WRITE_Y, true, kSeg / 32>(seg_addr, word, lane, lanemask_lt(), y, yvalid, p.c.tau);
+            run = compact_segment<U, FUSED, WRITE_Y, true, kSeg / 32>(seg_addr, word, lane, lanemask_lt(), y, yvalid, p.c.tau, yx);
         if (lane < static_cast<uint32_t>(kSeg / 32)) {
             const uint64_t wd = t64 * (kTile / 32) + warp * (kSeg / 32) + lane;
-            if (wd < ((n + 31) >> 5)) jb.bitmap[wd] = word;
+            if (wd < ((n + 31) >> 5) && extent_of(jb.bitmap, 4 * ((n + 31) >> 5)).holds(jb.bitmap + wd, 4)) jb.bitmap[wd] = word;
         }
         __syncwarp();
         if (lane == 0) {
@@ -512,13 +521,14 @@ cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint
 
     CompressParams<kJobs> p;
     p.c             = c;
-    uint64_t tiles  = 0;
+    uint64_t tiles  = 0, chunks = 0;
     for (uint32_t k = 0; k < count; ++k) {
         p.job[k]            = jobs[k];
         const uint64_t t    = (jobs[k].n + kTile - 1) / kTile;
         if (t == 0 || t > 0xFFFFFFFFull) return cudaErrorInvalidValue;
         p.job[k].tiles      = static_cast<uint32_t>(t);
         tiles += t;
+        chunks += (jobs[k].n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
     }
     if (tiles > 0xFFFFFFFFull) return cudaErrorInvalidValue;
     for (uint32_t k = count; k < static_cast<uint32_t>(kJobs); ++k) p.job[k] = CompressJob{};
@@ -544,6 +554,7 @@ cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint
     p.c.ws_header = static_cast<uint64_t *>(workspace);
     p.c.ws_total  = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + kWsHeaderBytes);
     p.c.ws_desc   = p.c.ws_total + p.c.ws_totals;
+    p.c.ws_words  = (compress_workspace_bytes(chunks) - kWsHeaderBytes) / 8;
     p.c.call_tag  = next_call_tag();
     p.c.wait_ns   = compress_wait_ns();
     // cooperative launch: the runtime guarantees that all `grid` CTAs are resident together

@@ -20,7 +20,6 @@ uint64_t compress_wait_ns();
 namespace cmp {
 
 constexpr uint32_t kFull       = 0xFFFFFFFFu;
-constexpr int      kBarWorkers = 1;                   // named barrier of the worker warps (ragged tile only)
 constexpr int      kMaxWindows = 5;                   // the grid never exceeds 32 * kMaxWindows CTAs
 constexpr int      kHdrSeq     = 0;                   // header words (64-bit): launch sequence number,
 constexpr int      kHdrAbort   = 1;                   //   abort word (== the launch's tag once a wait ran out)
@@ -75,10 +74,42 @@ static __device__ __noinline__ void raise_timeout(uint64_t *ws_header, int32_t *
     if (dev_status) *reinterpret_cast<volatile int32_t *>(dev_status) = BT_ERR_TIMEOUT;
 }
 
-// Bounded wait on an mbarrier phase.  False once the limit passed or the CTA is aborting.
+// A limit below this is kept to the nanosecond (see mbar_wait_strict).  Only the test build of the library
+// (-DBT_TEST_HOOKS) can set such a limit, and only that build carries the code for it: the product's waits
+// are the same instructions with or without it.
+constexpr uint64_t kStrictLimitNs = 1000;
+#ifdef BT_TEST_HOOKS
+constexpr bool kTestHooks = true;
+#else
+constexpr bool kTestHooks = false;
+#endif
+
+// The wait under a limit of less than a microsecond, which only a test build of the library can set: probes that
+// return at once (a try_wait may itself suspend the thread for longer than such a limit), the clock read after
+// every probe.  A phase that is not complete at the first probe and does not complete within the limit fails.
+static __device__ __noinline__ bool mbar_wait_strict(uint64_t *bar, const uint32_t parity, const uint64_t limit_ns)
+{
+    const uint64_t t0 = now_ns();
+    for (;;) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(smem_addr(bar)), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (now_ns() - t0 > limit_ns) return false;
+    }
+}
+
+// Bounded wait on an mbarrier phase.  False once the limit passed or the CTA is aborting.  The limit is checked
+// every 32 probes, each of which may suspend the thread for a while: exact enough for the product's two seconds.
 template <bool kStopOnAbort = true>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *s_abort, const uint64_t limit_ns)
 {
+    if (kTestHooks && limit_ns < kStrictLimitNs) return mbar_wait_strict(bar, parity, limit_ns);
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = now_ns();
     for (;;) {
@@ -115,7 +146,8 @@ __device__ __forceinline__ Reg<U> lds_elem(uint32_t addr)
 // step k lands below element 32(k+1) and a later batch reads at or above it, so they never meet.
 template <typename U, int RELU_DT, bool WRITE_Y, bool kGuardY, int kSteps>
 __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uint32_t &word, const uint32_t lane,
-                                                    const uint32_t lt, U *y, const uint32_t yvalid, const float tau)
+                                                    const uint32_t lt, U *y, const uint32_t yvalid, const float tau,
+                                                    const Extent yx)
 {
     constexpr int      kBatch = 8;
     static_assert(kSteps % kBatch == 0 && kSteps <= 32, "whole batches; one bitmap word per lane");
@@ -141,7 +173,7 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
                 x = fused_forward<RELU_DT>(x, tau);
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
-                    if (!kGuardY || e < yvalid) y[e] = static_cast<U>(x);
+                    if ((!kGuardY || e < yvalid) && yx.holds(y + e, sizeof(U))) y[e] = static_cast<U>(x);
                 }
             }
             const uint32_t b = __ballot_sync(kFull, x != Reg<U>(0));
@@ -190,7 +222,7 @@ using Stored = std::conditional_t<CAST == 0, U, uint16_t>;
 // One warp copies the `cnt` packed slots of its segment to out[0..cnt): contiguous, coalesced.
 template <typename U, int CAST, bool kGuard>
 __device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, const uint32_t lane, const uint32_t cnt,
-                                                 Stored<CAST, U> *__restrict__ out, const uint64_t room)
+                                                 Stored<CAST, U> *__restrict__ out, const uint64_t room, const Extent vx)
 {
     // (Pairing narrowed values into 4-byte stores was measured and is no faster: at half zeros the narrowing
     // forms run at the speed of the compaction, not of the copy-out.)
@@ -198,14 +230,14 @@ __device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, cons
     for (; j + 96 < cnt; j += 128) {
         const auto v0 = narrowed<CAST>(seg[j]), v1 = narrowed<CAST>(seg[j + 32]), v2 = narrowed<CAST>(seg[j + 64]),
                    v3 = narrowed<CAST>(seg[j + 96]);
-        if (!kGuard || j < room) out[j] = v0;
-        if (!kGuard || j + 32 < room) out[j + 32] = v1;
-        if (!kGuard || j + 64 < room) out[j + 64] = v2;
-        if (!kGuard || j + 96 < room) out[j + 96] = v3;
+        if ((!kGuard || j < room) && vx.holds(out + j, sizeof(*out))) out[j] = v0;
+        if ((!kGuard || j + 32 < room) && vx.holds(out + j + 32, sizeof(*out))) out[j + 32] = v1;
+        if ((!kGuard || j + 64 < room) && vx.holds(out + j + 64, sizeof(*out))) out[j + 64] = v2;
+        if ((!kGuard || j + 96 < room) && vx.holds(out + j + 96, sizeof(*out))) out[j + 96] = v3;
     }
     for (; j < cnt; j += 32) {
         const auto v = narrowed<CAST>(seg[j]);
-        if (!kGuard || j < room) out[j] = v;
+        if ((!kGuard || j < room) && vx.holds(out + j, sizeof(*out))) out[j] = v;
     }
 }
 

@@ -63,14 +63,7 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<
     const uint64_t w0          = chunk * 128 + 4 * lane;   // this lane's four words of the chunk
 
     // the chunk's 128 words (zero past the end of the bitmap) and its prefix entry: independent loads
-    uint4 w4 = make_uint4(0, 0, 0, 0);
-    if (w0 + 3 < words_total) {
-        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
-    } else {
-        if (w0 < words_total) w4.x = bitmap[w0];
-        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
-        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
-    }
+    const uint4 w4 = load_words4(bitmap, w0, words_total);
     const uint64_t chunk_base = prefix[chunk];
     // arena form: the packed values start *values_offset bytes into `values`
     using V = std::conditional_t<WIDEN != 0, uint16_t, U>;   // type of a stashed value
@@ -98,6 +91,7 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<
 
     const uint64_t e0    = warp_global << 10;               // first element of the quarter
     const uint32_t shift = (lane % kLanesPerWord) * kE;     // which kE-bit group of the word
+    const Extent   ox    = extent_of(out, n * sizeof(U));
     // the gathers of kGrp steps are issued before their stores, so that a lane has kGrp * kE independent loads
     // in flight.  All 32 of the quarter (kGrp = kSteps) is the setting used: smaller groups raise the occupancy
     // and are 2 % faster on a 1 GiB tensor, but 10 % slower on the few-MB layers of a ResNet, whose cold
@@ -141,11 +135,11 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<
                     pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
                                       ev[4] | (uint32_t(ev[5]) << 16), ev[6] | (uint32_t(ev[7]) << 16));
                 }
-                *reinterpret_cast<uint4 *>(out + at) = pack;
+                if (ox.holds(out + at, 16)) *reinterpret_cast<uint4 *>(out + at) = pack;
             } else {
 #pragma unroll
                 for (int j = 0; j < kVec; ++j)
-                    if (at + j < n) out[at + j] = ev[j];
+                    if (at + j < n && ox.holds(out + at + j, sizeof(U))) out[at + j] = ev[j];
             }
         }
     }
@@ -259,6 +253,7 @@ decompress16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values,
     // 0.131 ms instead of 0.126 on 205 M elements; with 2 per lane the shuffles and stores double: 0.153 ms.)
     const uint64_t e0    = warp_global << 10;
     const bool     whole = e0 + 1024 <= n;
+    const Extent   ox    = extent_of(out, n * sizeof(uint16_t));
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         const int      from = k * 4 + (lane >> 3);
@@ -269,12 +264,12 @@ decompress16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values,
         const uint2    v    = expand4_u16(stage + shift + 2u * off, w >> sh);
         const uint64_t at   = e0 + static_cast<uint64_t>(k) * 128 + lane * 4;
         if (whole || at + 4 <= n) {
-            *reinterpret_cast<uint2 *>(out + at) = v;
+            if (ox.holds(out + at, 8)) *reinterpret_cast<uint2 *>(out + at) = v;
         } else {
             const uint32_t h[2] = {v.x, v.y};
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (at + j < n) out[at + j] = static_cast<uint16_t>(h[j >> 1] >> (16 * (j & 1)));
+                if (at + j < n && ox.holds(out + at + j, 2)) out[at + j] = static_cast<uint16_t>(h[j >> 1] >> (16 * (j & 1)));
         }
     }
 }

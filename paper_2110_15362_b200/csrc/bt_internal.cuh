@@ -31,7 +31,7 @@ constexpr uint32_t kMinTileElems  = BT_CHUNK_ELEMS;
 constexpr uint32_t kMaxBatch      = 32;                        // tensors of one batched launch
 constexpr uint64_t kDefaultWaitNs = 2000000000ull;             // bound of every in-kernel wait: 2 s
 // bytes of workspace for tensors holding `chunks` 4096-element chunks in all
-constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 16 + 24 * static_cast<size_t>(chunks); }
+__host__ __device__ constexpr size_t compress_workspace_bytes(uint64_t chunks) { return kWsHeaderBytes + 16 + 24 * static_cast<size_t>(chunks); }
 
 // One tensor, one launch.
 struct CompressArgs {
@@ -83,6 +83,7 @@ struct CompressCommon {
     uint64_t   *ws_total;   // wave totals
     uint64_t   *ws_desc;    // tile descriptors
     uint32_t    ws_totals;  // number of wave-total words (even)
+    uint64_t    ws_words;   // 8-byte words of the workspace behind its header (what the size query promises)
     uint32_t    jobs;       // number of tensors
     uint64_t    call_tag;   // unique to the call
     uint64_t    wait_ns;    // bound of every in-kernel wait
@@ -139,6 +140,52 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
                  : "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// Checking build (-DBT_BOUNDS_CHECK, a library of its own that only the tests load): every store to
+// global memory is tested against the extent of the buffer it belongs to.  A store that would fall
+// outside is skipped and counted in a device word the test reads back; nothing traps.  In the
+// product build an Extent is empty and `holds` is the constant true, so the checks cost nothing.
+#ifdef BT_BOUNDS_CHECK
+extern __device__ unsigned long long g_bounds_violations;   // one word for the library: relocatable device code
+struct Extent {
+    uintptr_t lo, hi;   // [lo, hi) in bytes
+    __device__ __forceinline__ bool holds(const void *p, const size_t bytes) const
+    {
+        const uintptr_t a  = reinterpret_cast<uintptr_t>(p);
+        const bool      ok = a >= lo && a + bytes <= hi;
+        if (!ok) atomicAdd(&g_bounds_violations, 1ull);
+        return ok;
+    }
+};
+__device__ __forceinline__ Extent extent_of(const void *base, const uint64_t bytes)
+{
+    return Extent{reinterpret_cast<uintptr_t>(base), reinterpret_cast<uintptr_t>(base) + bytes};
+}
+#else
+struct Extent {
+    __device__ __forceinline__ bool holds(const void *, const size_t) const { return true; }
+};
+__device__ __forceinline__ Extent extent_of(const void *, const uint64_t) { return Extent{}; }
+#endif
+
+// A lane's four consecutive words of a chunk's bitmap, w0 a multiple of four; words past the end of the
+// bitmap read as zero.  One 16-byte load where the bitmap's base address allows it (the format only
+// asks for 4-byte alignment), four word loads otherwise.
+__device__ __forceinline__ uint4 load_words4(const uint32_t *__restrict__ bitmap, const uint64_t w0,
+                                             const uint64_t words_total)
+{
+    uint4 w4 = make_uint4(0, 0, 0, 0);
+    if (w0 + 3 < words_total && (reinterpret_cast<uintptr_t>(bitmap) & 15u) == 0) {
+        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
+    } else {
+        if (w0 < words_total) w4.x = bitmap[w0];
+        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
+        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
+        if (w0 + 3 < words_total) w4.w = bitmap[w0 + 3];
+    }
+    return w4;
 }
 
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)

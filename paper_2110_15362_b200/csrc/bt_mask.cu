@@ -81,14 +81,7 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
     }
 
     // the chunk's 128 words (zero past the end of the bitmap) and its prefix entry
-    uint4 w4 = make_uint4(0, 0, 0, 0);
-    if (w0 + 3 < words_total) {
-        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
-    } else {
-        if (w0 < words_total) w4.x = bitmap[w0];
-        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
-        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
-    }
+    const uint4 w4 = load_words4(bitmap, w0, words_total);
     const uint64_t chunk_base = prefix[chunk];
 
     uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
@@ -121,6 +114,8 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
     const uint32_t total = __shfl_sync(kFull, incl, 31);          // set bits of the quarter
 
     const uint32_t shift = (lane % kLanesPerWord) * kE;     // which kE-bit group of the word
+    const Extent   yx    = extent_of(y, n * sizeof(U));
+    const Extent   vx    = extent_of(values, capacity * sizeof(U));
 #pragma unroll
     for (int k = 0; k < kSteps; ++k) {
         const int      from = k * kWordsPerStep + lane / kLanesPerWord;
@@ -152,11 +147,11 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
                         pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
                                           ev[4] | (uint32_t(ev[5]) << 16), ev[6] | (uint32_t(ev[7]) << 16));
                     }
-                    *reinterpret_cast<uint4 *>(y + at) = pack;
+                    if (yx.holds(y + at, 16)) *reinterpret_cast<uint4 *>(y + at) = pack;
                 } else {
 #pragma unroll
                     for (int j = 0; j < kVec; ++j)
-                        if (at + j < n) y[at + j] = ev[j];
+                        if (at + j < n && yx.holds(y + at + j, sizeof(U))) y[at + j] = ev[j];
                 }
             }
         }
@@ -171,11 +166,11 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
         const uint32_t lo = v * kVec, hi = lo + kVec;
         const uint64_t g  = gbase + lo;
         if (lo >= skew && hi <= end && g + kVec <= capacity) {
-            *reinterpret_cast<uint4 *>(values + g) = *reinterpret_cast<const uint4 *>(stage + lo);
+            if (vx.holds(values + g, 16)) *reinterpret_cast<uint4 *>(values + g) = *reinterpret_cast<const uint4 *>(stage + lo);
         } else {
 #pragma unroll
             for (int j = 0; j < kVec; ++j)
-                if (lo + j >= skew && lo + j < end && g + j < capacity) values[g + j] = stage[lo + j];
+                if (lo + j >= skew && lo + j < end && g + j < capacity && vx.holds(values + g + j, sizeof(U))) values[g + j] = stage[lo + j];
         }
     }
 }

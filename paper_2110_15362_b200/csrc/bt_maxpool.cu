@@ -73,13 +73,13 @@ maxpool2x2_fwd_kernel(const U *__restrict__ x, const uint64_t outputs, const I w
             bestv           = take ? v : bestv;
             code            = take ? k : code;
         }
-        y[o64] = best;
+        if (extent_of(y, outputs * sizeof(U)).holds(y + o64, sizeof(U))) y[o64] = best;
     }
     if (codes) {
         uint32_t word = code << (2u * (lane & 15u));
 #pragma unroll
         for (int d = 8; d > 0; d >>= 1) word |= __shfl_xor_sync(kFull, word, d);
-        if (live && (lane & 15u) == 0) codes[o64 >> 4] = word;
+        if (live && (lane & 15u) == 0 && extent_of(codes, 4 * ((outputs + 15) >> 4)).holds(codes + (o64 >> 4), 4)) codes[o64 >> 4] = word;
     }
 }
 
@@ -99,8 +99,10 @@ maxpool2x2_bwd_kernel(const uint32_t *__restrict__ codes, const uint32_t *__rest
     const uint32_t k    = (codes[o64 >> 4] >> (2u * (static_cast<uint32_t>(o64) & 15u))) & 3u;
     U              g    = gout[o64];
     if (mask != nullptr && ((mask[o64 >> 5] >> (static_cast<uint32_t>(o64) & 31u)) & 1u) == 0) g = U(0);
-    *reinterpret_cast<typename P::T *>(gin + at)         = P::make(k == 0 ? g : U(0), k == 1 ? g : U(0));
-    *reinterpret_cast<typename P::T *>(gin + at + width) = P::make(k == 2 ? g : U(0), k == 3 ? g : U(0));
+    const Extent gx = extent_of(gin, 4 * outputs * sizeof(U));
+    if (gx.holds(gin + at, 2 * sizeof(U))) *reinterpret_cast<typename P::T *>(gin + at) = P::make(k == 0 ? g : U(0), k == 1 ? g : U(0));
+    if (gx.holds(gin + at + width, 2 * sizeof(U)))
+        *reinterpret_cast<typename P::T *>(gin + at + width) = P::make(k == 2 ? g : U(0), k == 3 ? g : U(0));
 }
 
 // Vector form for 2- and 4-byte elements whose rows hold whole 16-byte vectors of window pairs (width a multiple of
@@ -161,15 +163,17 @@ maxpool2x2_fwd_vec_kernel(const U *__restrict__ x, const uint64_t groups, const 
             win[j] = best;
             bits |= code << (2 * j);
         }
-        if constexpr (sizeof(U) == 4) *reinterpret_cast<uint2 *>(y + g64 * kOut) = make_uint2(win[0], win[1]);
-        else
-            *reinterpret_cast<uint2 *>(y + g64 * kOut) = make_uint2(win[0] | (uint32_t(win[1]) << 16), win[2] | (uint32_t(win[3]) << 16));
+        uint2 pack;
+        if constexpr (sizeof(U) == 4) pack = make_uint2(win[0], win[1]);
+        else pack = make_uint2(win[0] | (uint32_t(win[1]) << 16), win[2] | (uint32_t(win[3]) << 16));
+        if (extent_of(y, groups * kOut * sizeof(U)).holds(y + g64 * kOut, 8)) *reinterpret_cast<uint2 *>(y + g64 * kOut) = pack;
     }
     if (codes) {
         uint32_t word = bits << (2u * kOut * (lane % kLanesPerWord));
 #pragma unroll
         for (int d = kLanesPerWord / 2; d > 0; d >>= 1) word |= __shfl_xor_sync(kFull, word, d);
-        if (live && (lane % kLanesPerWord) == 0) codes[(g64 * kOut) >> 4] = word;
+        if (live && (lane % kLanesPerWord) == 0 && extent_of(codes, 4 * ((groups * kOut + 15) >> 4)).holds(codes + ((g64 * kOut) >> 4), 4))
+            codes[(g64 * kOut) >> 4] = word;
     }
 }
 
@@ -205,8 +209,9 @@ maxpool2x2_bwd_vec_kernel(const uint32_t *__restrict__ codes, const uint32_t *__
         bot[2 * j]       = k == 2 ? gr[j] : U(0);
         bot[2 * j + 1]   = k == 3 ? gr[j] : U(0);
     }
-    *reinterpret_cast<uint4 *>(gin + at)         = pack16<U>(top);
-    *reinterpret_cast<uint4 *>(gin + at + width) = pack16<U>(bot);
+    const Extent gx = extent_of(gin, 4 * groups * kOut * sizeof(U));
+    if (gx.holds(gin + at, 16)) *reinterpret_cast<uint4 *>(gin + at) = pack16<U>(top);
+    if (gx.holds(gin + at + width, 16)) *reinterpret_cast<uint4 *>(gin + at + width) = pack16<U>(bot);
 }
 
 template <typename U, int DT>

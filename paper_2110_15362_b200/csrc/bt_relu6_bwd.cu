@@ -77,14 +77,7 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     };
     fetch(0);
 
-    uint4 w4 = make_uint4(0, 0, 0, 0);
-    if (w0 + 3 < words_total) {
-        w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
-    } else {
-        if (w0 < words_total) w4.x = bitmap[w0];
-        if (w0 + 1 < words_total) w4.y = bitmap[w0 + 1];
-        if (w0 + 2 < words_total) w4.z = bitmap[w0 + 2];
-    }
+    const uint4 w4 = load_words4(bitmap, w0, words_total);
     const uint64_t chunk_base = prefix[chunk];
 
     uint32_t before = lane < 8 * q ? __popc(w4.x) + __popc(w4.y) + __popc(w4.z) + __popc(w4.w) : 0u;
@@ -110,6 +103,7 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     const U *const vp   = values + (chunk_base + before);
 
     const uint32_t shift = (lane % kLanesPerWord) * kE;
+    const Extent   ox    = extent_of(gin, n * sizeof(U));
 #pragma unroll
     for (int kk = 0; kk < kSteps; ++kk) {
         const int k = kk % kBlk;                              // row of g
@@ -144,11 +138,11 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
                     pack = make_uint4(gv[0] | (uint32_t(gv[1]) << 16), gv[2] | (uint32_t(gv[3]) << 16),
                                       gv[4] | (uint32_t(gv[5]) << 16), gv[6] | (uint32_t(gv[7]) << 16));
                 }
-                *reinterpret_cast<uint4 *>(gin + at) = pack;
+                if (ox.holds(gin + at, 16)) *reinterpret_cast<uint4 *>(gin + at) = pack;
             } else {
 #pragma unroll
                 for (int j = 0; j < kVec; ++j)
-                    if (at + j < n) gin[at + j] = gv[j];
+                    if (at + j < n && ox.holds(gin + at + j, sizeof(U))) gin[at + j] = gv[j];
             }
         }
     }

@@ -56,6 +56,7 @@ relu_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *gout, const uint64
     const uint64_t vecs      = n / kVec;                       // whole 16-byte vectors
     const uint64_t block0    = static_cast<uint64_t>(blockIdx.x) * (kThreads * kUnroll);
 
+    const Extent ox = extent_of(gin, n * sizeof(U));
     uint4    g[kUnroll];
     uint32_t w[kUnroll];
 #pragma unroll
@@ -71,14 +72,14 @@ relu_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *gout, const uint64
         const uint64_t v = block0 + u * kThreads + threadIdx.x;
         if (v < vecs) {
             const uint32_t bits = (w[u] >> ((v * kVec) & 31u)) & kMask;
-            reinterpret_cast<uint4 *>(gin)[v] = select_vec<U>(g[u], bits);
+            if (ox.holds(reinterpret_cast<uint4 *>(gin) + v, 16)) reinterpret_cast<uint4 *>(gin)[v] = select_vec<U>(g[u], bits);
         }
     }
     // the last n % kVec elements, one by one
     if (blockIdx.x == 0 && threadIdx.x < n - vecs * kVec) {
         const uint64_t i = vecs * kVec + threadIdx.x;
         const bool set   = (bitmap[i >> 5] >> (i & 31u)) & 1u;
-        gin[i]           = set ? gout[i] : U(0);
+        if (ox.holds(gin + i, sizeof(U))) gin[i] = set ? gout[i] : U(0);
     }
 }
 

@@ -131,6 +131,39 @@ def test_later_entry_points_check_their_arguments_before_any_launch(L):
     assert L.bt_relu6_bwd_from_stash_arena(None, None, None, None, None, 0, B.BT_F32, None, None) == B.BT_OK
 
 
+def test_bitmap_needs_four_byte_alignment_only(L):
+    """The bitmap is an array of 32-bit words: 4-byte alignment is all the format asks for, in the compressors and
+    in every consumer.  A 2-byte offset is refused; a 4-byte offset passes the alignment check (shown here by the
+    check that comes after it; the GPU tests run such bitmaps through every kernel)."""
+    A = 0x10000
+    ws = L.bt_workspace_bytes(8192)
+    for off, expect in ((2, B.BT_ERR_ALIGN), (4, B.BT_ERR_WORKSPACE), (8, B.BT_ERR_WORKSPACE), (12, B.BT_ERR_WORKSPACE)):
+        assert L.bt_compress(A, 8192, B.BT_F32, A + off, A, 8192, A, A, A, ws - 1, A, None) == expect
+        assert L.bt_relu_fwd_compress(A, 8192, B.BT_BF16, None, A + off, A, 8192, A, A, A, ws - 1, A, None) == expect
+    assert L.bt_compress_noalloc(A, 16, B.BT_F32, A + 2, A, 16, A, A, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_decompress(A + 2, A, A, 10, B.BT_F32, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_decompress_widen(A + 2, A, A, 10, B.BT_F16, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_relu_bwd_from_bitmap(A + 2, A, 10, B.BT_F32, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_relu6_bwd_from_stash(A + 2, A, A, A, 10, B.BT_F32, A, None) == B.BT_ERR_ALIGN
+    assert L.bt_mask_compress(A, 10, B.BT_F32, A + 2, A, None, A, 10, None) == B.BT_ERR_ALIGN
+    # a 4-byte offset and a second, real fault: the second one is what gets reported
+    assert L.bt_decompress(A + 4, A, A, 10, B.BT_F32, A + 2, None) == B.BT_ERR_ALIGN
+    assert L.bt_decompress(A + 4, A, A + 4, 10, B.BT_F32, A, None) == B.BT_ERR_ALIGN
+
+
+def test_header_puts_the_codec_proper_first_and_states_what_the_library_keeps():
+    import os
+    import re
+    text = open(os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "bittrain.h")).read()
+    names = re.findall(r"^(?:int|size_t|long long)\s+(bt_\w+)\s*\(", text, flags=re.M)
+    assert names[:6] == ["bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decompress",
+                         "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap"]
+    head = text[:text.index("#ifndef BITTRAIN_H")]
+    assert "bitmap 4-byte aligned" in head
+    assert "bt_set_max_ctas" in head and "counter" in head          # the host-side state is named, not denied
+    assert "keeps no" not in head
+
+
 def test_cta_limit_is_per_thread_host_state(L):
     import threading
     assert L.bt_set_max_ctas(0) == 0

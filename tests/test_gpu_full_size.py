@@ -1,17 +1,23 @@
 """Parity at the full sizes of the five workload configurations, in the launch configuration the
-benchmark times (the library's own launch shapes, one stream).  A tensor of up to a gigabyte is too
-much for the single-threaded oracle, so each one is checked three ways: (1) the oracle on randomly
-sampled 4096-element chunks (bitmap words, packed values, prefix entry, restored elements), (2) torch
-routines on the GPU over the whole tensor (boolean indexing, packed bits, chunk counts, relu, where) as
-an independent full-size check, (3) properties that hold at any size (nnz == popcount(bitmap), the
-round trip is the identity bit for bit, bytes formula).  The small layers of configuration 2 go through
-the oracle whole."""
+benchmark times (the library's own launch shapes, one stream).
+
+Whole tensors against the CPU oracle, every output compared element by element, outputs in guarded
+buffers: the 1 GiB tensor of configuration 3 (i.i.d. at half zeros, clustered at 90 % zeros), the largest
+tensor of configuration 4 in bfloat16 and binary16 (fused forward with the dense output, and the backward
+pass), one layer of configuration 5, and every layer of configuration 2.
+
+The rest of the sweep (every sparsity, every distinct shape, the forward-then-reverse trace) is checked
+three ways per tensor: (1) the oracle on randomly sampled 4096-element chunks (bitmap words, packed values,
+prefix entry, restored elements), (2) torch routines on the GPU over the whole tensor (boolean indexing,
+packed bits, chunk counts, relu, where) as an independent full-size check, (3) properties that hold at any
+size (nnz == popcount(bitmap), the round trip is the identity bit for bit, bytes formula)."""
 import numpy as np
 import pytest
 import torch
 
 from paper_2110_15362_b200 import binding as B
 from paper_2110_15362_b200 import workloads as W
+from tests.gpu_util import Guarded
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -97,22 +103,109 @@ def decompress(st, like):
     return out
 
 
+class GuardedStash:
+    """The buffers of one stash, each between canary regions."""
+
+    def __init__(self, n, dtype):
+        self.bitmap = Guarded((n + 31) // 32, torch.int32)
+        self.values = Guarded(n, dtype)
+        self.prefix = Guarded((n + 4095) // 4096, torch.int64)
+        self.nnz = Guarded(1, torch.int64)
+        self.status = Guarded(1, torch.int32)
+
+    def args(self):
+        return self.bitmap.inner, self.values.inner, self.prefix.inner, self.nnz.inner
+
+    def intact(self):
+        return all(g.guards_intact() for g in (self.bitmap, self.values, self.prefix, self.nnz, self.status))
+
+    def equals(self, c):
+        nnz = int(self.nnz.inner.item())
+        assert int(self.status.inner.item()) == B.BT_OK and nnz == c.nnz
+        assert np.array_equal(self.bitmap.raw().view(np.uint32), c.bitmap)
+        assert np.array_equal(self.prefix.raw().view(np.uint64), c.prefix)
+        assert np.array_equal(W.raw_numpy(self.values.inner[:nnz]), c.values)
+        assert self.intact()
+
+
+def whole_tensor_round_trip(oracle, x):
+    """bt_compress, bt_decompress and bt_relu_bwd_from_bitmap of one tensor, every output against the oracle."""
+    n = x.numel()
+    raw = W.raw_numpy(x)
+    st = GuardedStash(n, x.dtype)
+    B.bt_compress(x, *st.args(), B.new_workspace(n, DEV), st.status.inner)
+    c = oracle.compress(raw)
+    st.equals(c)
+    back = Guarded(n, x.dtype)
+    B.bt_decompress(st.bitmap.inner, st.values.inner, st.prefix.inner, back.inner)
+    assert np.array_equal(back.raw(), oracle.decompress(c)) and back.guards_intact()
+    assert np.array_equal(back.raw(), raw)
+    del back
+    g = torch.randn(n, generator=torch.Generator(device=DEV).manual_seed(n % 1000003), device=DEV, dtype=torch.float32).to(x.dtype)
+    gin = Guarded(n, x.dtype)
+    B.bt_relu_bwd_from_bitmap(st.bitmap.inner, g, gin.inner)
+    assert np.array_equal(gin.raw(), oracle.relu_bwd_from_bitmap(c.bitmap, W.raw_numpy(g))) and gin.guards_intact()
+    return c
+
+
+def test_cfg3_one_gibibyte_iid_half_zeros_whole_tensor_against_the_oracle(oracle):
+    x = W.cfg3_iid(1 << 28, 0.5, W.SPARSITY_SWEEP.index(0.5), DEV)
+    c = whole_tensor_round_trip(oracle, x)
+    assert abs(c.nnz / x.numel() - 0.5) < 0.01
+
+
+def test_cfg3_one_gibibyte_clustered_ninety_percent_zeros_whole_tensor_against_the_oracle(oracle):
+    x = W.cfg3_clustered(1 << 28, 0.9, W.SPARSITY_SWEEP.index(0.9), DEV)
+    c = whole_tensor_round_trip(oracle, x)
+    assert abs(c.nnz / x.numel() - 0.1) < 0.02
+
+
+@pytest.mark.parametrize("kind", ["bf16", "f16"])
+def test_cfg4_largest_tensor_fused_pair_whole_tensor_against_the_oracle(oracle, kind):
+    shapes = W.vgg16_shapes(64)
+    i = max(range(len(shapes)), key=lambda k: W.numel(shapes[k]))
+    n = W.numel(shapes[i])
+    assert n == 205520896
+    pre = W.cfg4_preact(i, shapes[i], kind, DEV).reshape(-1)
+    g = W.cfg4_grad(i, shapes[i], kind, DEV).reshape(-1)
+    y_ref, c = oracle.relu_fwd_compress(W.raw_numpy(pre), kind)
+    ws = B.new_workspace(n, DEV)
+    st = GuardedStash(n, pre.dtype)
+    y = Guarded(n, pre.dtype)
+    B.bt_relu_fwd_compress(pre, y.inner, *st.args(), ws, st.status.inner)
+    st.equals(c)
+    assert np.array_equal(y.raw(), y_ref) and y.guards_intact()
+    st2 = GuardedStash(n, pre.dtype)                         # the form without the dense output
+    B.bt_relu_fwd_compress(pre, None, *st2.args(), ws, st2.status.inner)
+    st2.equals(c)
+    del st2, y
+    gin = Guarded(n, pre.dtype)
+    B.bt_relu_bwd_from_bitmap(st.bitmap.inner, g, gin.inner)
+    assert np.array_equal(gin.raw(), oracle.relu_bwd_from_bitmap(c.bitmap, W.raw_numpy(g))) and gin.guards_intact()
+    back = Guarded(n, pre.dtype)
+    B.bt_decompress(st.bitmap.inner, st.values.inner, st.prefix.inner, back.inner)
+    assert np.array_equal(back.raw(), y_ref) and back.guards_intact()
+
+
+def test_cfg5_one_layer_whole_tensor_against_the_oracle(oracle):
+    shapes = W.mobilenetv2_shapes(128)
+    fractions = W.cfg5_zero_fractions(len(shapes))
+    i = max(range(len(shapes)), key=lambda k: W.numel(shapes[k]))       # the largest layer of the trace
+    x = W.cfg5_layer(i, shapes[i], fractions[i], DEV).reshape(-1)
+    c = whole_tensor_round_trip(oracle, x)
+    assert abs((1 - c.nnz / x.numel()) - fractions[i]) < 0.02
+
+
 def test_cfg2_resnet18_batch32_every_layer_against_the_oracle(oracle):
     for i, shape, n in W.iter_layers(W.resnet18_shapes(32)):
         x = W.cfg2_layer(i, shape, DEV).reshape(-1)
-        st = compress(x)
-        back = decompress(st, x)
+        st = GuardedStash(n, x.dtype)
+        B.bt_compress(x, *st.args(), B.new_workspace(n, DEV), st.status.inner)
+        back = Guarded(n, x.dtype)
+        B.bt_decompress(st.bitmap.inner, st.values.inner, st.prefix.inner, back.inner)
         torch.cuda.synchronize()
-        if n <= 8_000_000:                                   # small enough for the oracle, whole
-            ref = oracle.compress(W.raw_numpy(x))
-            assert st.nnz == ref.nnz and st.status == B.BT_OK
-            assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), ref.bitmap)
-            assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), ref.prefix)
-            assert np.array_equal(W.raw_numpy(st.values[:ref.nnz]), ref.values)
-        else:
-            check_against_torch(st, x)
-            check_sampled_chunks(oracle, st, x, back, seed=i)
-        assert torch.equal(bits_of(back), bits_of(x))
+        st.equals(oracle.compress(W.raw_numpy(x)))            # every layer whole
+        assert np.array_equal(back.raw(), W.raw_numpy(x)) and back.guards_intact()
 
 
 @pytest.mark.parametrize("variant", ["iid", "clustered"])

@@ -76,3 +76,35 @@ def test_host_capacity_and_argument_errors(oracle):
                                     h_prefix.data_ptr(), h_nnz.data_ptr(), staging.data_ptr(), 1024, None) == B.BT_ERR_WORKSPACE
     assert B.lib().bt_decompress_host(h_bitmap.data_ptr(), small.data_ptr(), h_prefix.data_ptr(), 1, n, 9,
                                       h_x.data_ptr(), staging.data_ptr(), staging.numel(), None) == B.BT_ERR_DTYPE
+
+
+@pytest.mark.parametrize("where", ["pageable", "pinned_unaligned", "pinned_odd_capacity"])
+def test_host_value_buffers_of_every_kind(oracle, where):
+    """The packed values reach the host by two routes: a page-locked, 16-byte aligned buffer is written by the
+    device itself (exactly nnz values, one synchronisation), any other buffer by a sized copy after a first
+    synchronisation.  Same results either way; nothing behind the values is touched."""
+    kind, dt, n = "bf16", torch.bfloat16, 8192 * 7 + 4097 + 3
+    x = W.random_patterns(n, kind, 0.5, seed=77)
+    c = oracle.compress(x)
+    assert c.nnz % 8 != 0                                                  # the last 16-byte vector is partial
+    staging = torch.empty(B.bt_host_staging_bytes(n, dt), dtype=torch.uint8, device="cuda")
+    h_x = host_tensor(x, kind)
+    h_bitmap = torch.empty((n + 31) // 32, dtype=torch.int32).pin_memory()
+    h_prefix = torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory()
+    h_nnz = torch.zeros(1, dtype=torch.int64).pin_memory()
+    room = torch.full((n + 64,), 3.0, dtype=dt)
+    if where == "pageable":
+        buf, cap = room[:n], n
+    elif where == "pinned_unaligned":
+        room = room.pin_memory()
+        buf, cap = room[1:n + 1], n                                       # 2 bytes off a 16-byte boundary
+    else:
+        room = room.pin_memory()
+        buf, cap = room[:n], c.nnz + 5                                    # capacity just above nnz
+    st = B.lib().bt_compress_host(h_x.data_ptr(), n, B.BT_BF16, h_bitmap.data_ptr(), buf.data_ptr(), cap,
+                                  h_prefix.data_ptr(), h_nnz.data_ptr(), staging.data_ptr(), staging.numel(), None)
+    assert st == B.BT_OK and int(h_nnz.item()) == c.nnz
+    assert np.array_equal(W.raw_numpy(buf[:c.nnz]), c.values)
+    assert (buf[c.nnz:] == 3.0).all()                                      # exactly nnz values were written
+    assert np.array_equal(W.raw_numpy(h_bitmap).view(np.uint32), c.bitmap)
+    assert np.array_equal(W.raw_numpy(h_prefix).view(np.uint64), c.prefix)

@@ -142,3 +142,28 @@ def test_argument_checks(G):
     assert L.bt_compress_narrow(x.data_ptr(), n, B.BT_F16, *args) == B.BT_OK
     torch.cuda.synchronize()
     assert st.status == B.BT_OK and st.nnz == 0
+
+
+@pytest.mark.parametrize("from_kind", TO)
+def test_widen_every_nan_and_infinity_stash(G, oracle, from_kind):
+    """bt_decompress_widen on stashes that hold every 16-bit NaN and infinity of the type, both signs, quiet and
+    signalling, scattered among zeros and ordinary values over several chunks: the oracle's patterns bit for bit
+    (a signalling NaN stays signalling; sign and payload are kept)."""
+    if from_kind == "f16":
+        mant = np.arange(0, 1024, dtype=np.uint16)
+        specials = np.concatenate([0x7C00 | mant, 0xFC00 | mant]).astype(np.uint16)
+    else:
+        specials = np.concatenate([np.arange(0x7F80, 0x8000), np.arange(0xFF80, 0x10000)]).astype(np.uint16)
+    n = 4096 * 5 + 777
+    x = W.random_patterns(n, from_kind, 0.5, seed=7)
+    rng = np.random.default_rng(11)
+    where = rng.choice(n, size=specials.size, replace=False)
+    x[where] = specials
+    c = oracle.compress(x)                                   # the 16-bit stash, patterns untouched
+    want = oracle.widen_decompress(c, from_kind)
+    assert np.isnan(want.view(np.float32)).sum() >= specials.size - 2
+    got = widen_on_gpu(G, c, n, from_kind)
+    assert np.array_equal(got, want)
+    # and the same stash restored in its own type, then cast by torch: NaN for NaN, equal elsewhere
+    plain, ok = G.gpu_decompress(c.bitmap, c.values, c.prefix, n, from_kind)
+    assert ok and np.array_equal(plain, x)

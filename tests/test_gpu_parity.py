@@ -139,3 +139,55 @@ def test_workspace_is_reusable_without_clearing(G, oracle):
         assert st.nnz == c.nnz and st.status == B.BT_OK
         assert np.array_equal(W.raw_numpy(st.values[:c.nnz]), c.values)
         assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), c.prefix)
+
+
+@pytest.mark.parametrize("kind", KINDS)
+@pytest.mark.parametrize("offset_words", [1, 2, 3])
+def test_bitmap_at_any_four_byte_boundary(G, oracle, kind, offset_words):
+    """A bitmap that starts 4, 8 or 12 bytes off a 16-byte boundary (a slice of a larger buffer) goes through every
+    kernel that writes or reads one: compress, fused forward, decompress, bitmap backward, masked gather, ReLU6
+    backward, the batched form."""
+    n = 8192 * 21 + 4097 + 9
+    dt = G.TDT[kind]
+    raw = W.random_patterns(n, kind, 0.5, seed=600 + offset_words)
+    x = G.from_raw(raw, kind)
+    c = oracle.compress(raw)
+    words = (n + 31) // 32
+    room = torch.full((words + 8,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    bitmap = room[offset_words:offset_words + words]
+    assert bitmap.data_ptr() % 16 == 4 * offset_words
+    st = B.Stash(n, dt)
+    ws = B.new_workspace(n)
+    B.bt_compress(x, bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+    torch.cuda.synchronize()
+    assert st.status == B.BT_OK and st.nnz == c.nnz
+    assert np.array_equal(W.raw_numpy(bitmap).view(np.uint32), c.bitmap)
+    assert (room[:offset_words] == 0x5A5A5A5A).all() and (room[offset_words + words:] == 0x5A5A5A5A).all()
+    assert np.array_equal(W.raw_numpy(st.values[:c.nnz]), c.values)
+    # readers
+    back = torch.empty_like(x)
+    B.bt_decompress(bitmap, st.values, st.chunk_prefix, back)
+    assert np.array_equal(W.raw_numpy(back), raw)
+    g_raw = W.random_patterns(n, kind, 0.1, seed=601)
+    g = G.from_raw(g_raw, kind)
+    gin = torch.empty_like(g)
+    B.bt_relu_bwd_from_bitmap(bitmap, g, gin)
+    assert np.array_equal(W.raw_numpy(gin), oracle.relu_bwd_from_bitmap(c.bitmap, g_raw))
+    vals2 = torch.empty(max(c.nnz, 1), dtype=dt, device="cuda")
+    y2 = torch.empty_like(x)
+    B.bt_mask_compress(g, bitmap, st.chunk_prefix, y2, vals2)
+    y_ref, v_ref = oracle.mask_compress(g_raw, c.bitmap)
+    assert np.array_equal(W.raw_numpy(vals2[:c.nnz]), v_ref) and np.array_equal(W.raw_numpy(y2), y_ref)
+    B.bt_relu6_bwd_from_stash(bitmap, st.values, st.chunk_prefix, g, gin)
+    assert np.array_equal(W.raw_numpy(gin), oracle.relu6_bwd_from_stash(c, kind, g_raw))
+    # fused forward and the batched form writing the same unaligned bitmap
+    y_ref, cr = oracle.relu_fwd_compress(raw, kind)
+    B.bt_relu_fwd_compress(x, None, bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+    torch.cuda.synchronize()
+    assert st.nnz == cr.nnz and np.array_equal(W.raw_numpy(bitmap).view(np.uint32), cr.bitmap)
+    st.bitmap = bitmap
+    items = B.batch_items([x], [st])
+    B.bt_compress_batch(items, dt, torch.empty(B.bt_batch_workspace_bytes([n]), dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert st.nnz == c.nnz and np.array_equal(W.raw_numpy(bitmap).view(np.uint32), c.bitmap)
+    assert (room[:offset_words] == 0x5A5A5A5A).all() and (room[offset_words + words:] == 0x5A5A5A5A).all()

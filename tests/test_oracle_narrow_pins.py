@@ -134,3 +134,54 @@ def test_widening_restore_matches_library_casts(oracle, to_kind):
     _, again = oracle.narrow_compress(back, to_kind)                 # idempotent on what survives as non-zero
     keep = c.values != 0                                             # an underflow to +0 drops out; -0 keeps its bit
     assert np.array_equal(again.values, c.values[keep])
+
+
+def _hand_made_stash(oracle, values16):
+    """A stash whose values are exactly `values16` (every bit set): what bt_compress gives for a 16-bit tensor
+    without zeros, built with the plain compressor so that no narrowing step touches the patterns."""
+    c = oracle.compress(values16)
+    assert c.nnz == values16.size
+    return c
+
+
+def test_widening_every_half_nan_keeps_sign_and_payload(oracle):
+    """All 2046 binary16 NaNs (both signs, quiet and signalling) through the widening restore.
+
+    Reading pinned here: the restore moves the 10 mantissa bits into the top of the binary32 mantissa and
+    the sign into bit 31, and does nothing else -- a signalling NaN stays signalling (quiet bit clear),
+    where a hardware conversion would set the quiet bit.  Against numpy and against torch, whose casts may
+    quiet: equal on sign and payload for every NaN, equal on every bit for the quiet ones, and for a
+    signalling one the library result is the oracle's with at most the quiet bit added."""
+    mant = np.arange(1, 1024, dtype=np.uint16)
+    h = np.concatenate([0x7C00 | mant, 0xFC00 | mant]).astype(np.uint16)
+    got = oracle.widen_decompress(_hand_made_stash(oracle, h), "f16")
+    want = ((h.astype(np.uint32) & 0x8000) << 16) | 0x7F800000 | ((h.astype(np.uint32) & 0x3FF) << 13)
+    assert np.array_equal(got, want)                                   # written out from the formats' layouts
+    quiet = (h & 0x0200) != 0
+    by_numpy = h.view(np.float16).astype(np.float32).view(np.uint32)
+    by_torch = torch.from_numpy(h.view(np.int16).copy()).view(torch.float16).to(torch.float32).view(torch.int32).numpy().view(np.uint32)
+    # numpy's cast keeps every NaN as it is; torch's sets the quiet bit, and gives the elements of an array's
+    # unvectorised tail the one pattern 0x7FFFFFFF (those pin only that the result is a NaN)
+    assert np.array_equal(by_numpy, got)
+    kept = by_torch != 0x7FFFFFFF
+    assert kept.sum() >= h.size - 16 and np.isnan(by_torch.view(np.float32)).all()
+    for lib_bits, sel in ((by_numpy, np.ones(h.size, bool)), (by_torch, kept)):
+        assert np.array_equal(lib_bits[quiet & sel], got[quiet & sel])
+        assert np.array_equal(lib_bits[sel] | 0x00400000, got[sel] | 0x00400000)          # sign, exponent, payload
+        assert np.isin(lib_bits[~quiet & sel] ^ got[~quiet & sel], (0, 0x00400000)).all()   # only the quiet bit may differ
+    assert np.isnan(got.view(np.float32)).all()
+    # a signalling NaN whose payload would vanish if the shift were wrong by one either way
+    assert got[0] == 0x7F802000 and got[mant.size] == 0xFF802000
+    # the scalar entry point agrees on the quiet ones (a float returned through Python is quieted on the way)
+    for hh in (0x7E00, 0xFE00, 0x7FFF, 0xFE01):
+        assert np.float32(oracle.half_to_float(hh)).view(np.uint32) == want[np.flatnonzero(h == hh)[0]]
+
+
+def test_widening_every_bfloat16_nan_and_infinity(oracle):
+    h = np.concatenate([np.arange(0x7F80, 0x8000), np.arange(0xFF80, 0x10000)]).astype(np.uint16)
+    got = oracle.widen_decompress(_hand_made_stash(oracle, h), "bf16")
+    assert np.array_equal(got, h.astype(np.uint32) << 16)
+    by_torch = torch.from_numpy(h.view(np.int16).copy()).view(torch.bfloat16).to(torch.float32).view(torch.int32).numpy().view(np.uint32)
+    assert np.array_equal(by_torch | 0x00400000, got | 0x00400000)
+    quiet = (h & 0x0040) != 0
+    assert np.array_equal(by_torch[quiet], got[quiet])
