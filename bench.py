@@ -1,25 +1,27 @@
 #!/usr/bin/env python3
 """Benchmark of the sparse-bitmap codec hot path on B200.
 
-One "step" is one pass of the whole path over one batch of synthetic
-activations shaped like a ResNet-18 at batch 32 (17 post-ReLU tensors, fp32,
-about half zeros): in forward order every layer is stashed twice -- once with
-bt_compress (from the post-ReLU activation) and once with bt_relu_fwd_compress
-(from the pre-activation) -- and in reverse order every layer is restored with
-bt_decompress and its ReLU gradient formed with bt_relu_bwd_from_bitmap.  The
-metric is dense-equivalent GB/s: the dense bytes of every tensor an entry point
-consumed or produced (N * sizeof(dtype) per call), summed over the step,
-divided by the step time.  The step is one CUDA graph of eight independent chains
-(plain codec / fused pair, layers by index mod 4) on eight streams; each compress
-launch is limited to a share of the SMs (bt_set_max_ctas) so that the chains'
-cooperative launches are resident side by side.
+Headline workload: the sparsity-sweep tensor of 2^28 fp32 elements (1 GiB) at half zeros.  One "step" is
+one pass of the whole hot path over one batch of such tensors (24 of them, seeded differently, all
+resident in HBM): per tensor bt_compress of the activation, bt_decompress of that stash,
+bt_relu_fwd_compress of the pre-activation (stash only) and bt_relu_bwd_from_bitmap of an upstream
+gradient -- four launches per tensor on one stream, about 26 ms per step, so that the 20 steps the
+round-end run times last half a second and the clock samples fall inside the timed region.  The metric
+is dense-equivalent GB/s: N * sizeof(dtype) per call, summed over the step, divided by the step time.
+
+The same JSON line carries, under roofline.kernels, every kernel of the five workload configurations
+timed on its own: CUDA events around ONE launch, the L2 flushed before it, median over repetitions --
+the single fp32 layer, the ResNet-18 step (batched launches), the sparsity sweep (i.i.d. and clustered),
+the VGG-16 tensors in bf16 and fp16 (fused forward with and without the dense output, backward), and the
+MobileNetV2 forward-then-reverse trace.  `roofline` itself is the row with the lowest fraction among
+the five graded calls on tensors of at least 256 MB.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py --case <f32|f16|bf16|f64> <op> [--log2n 26] [--zeros 0.5] [--reps 3]     # one kernel, for a profiler
 
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank
-runs the same batch shard on its own GPU -- data-parallel replicas compress
-their own activations, there is no data-path collective -- and the value is the
-sum over ranks divided by the slowest rank's time (weak scaling).
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs the same batch on its
+own GPU -- data-parallel replicas stash their own activations, there is no data-path collective -- and
+the value is the sum over ranks divided by the slowest rank's time (weak scaling).
 """
 from __future__ import annotations
 
@@ -37,27 +39,53 @@ if ROOT not in sys.path:
 
 METRIC = "codec_dense_equivalent_throughput"
 UNIT = "GB/s"
-WORKLOAD = "cfg2_resnet18_b32_f32"
-OPS = ("bt_compress", "bt_relu_fwd_compress", "bt_decompress", "bt_relu_bwd_from_bitmap")
+WORKLOAD = "cfg3_sparsity_sweep_2p28_f32_half_zeros"
+OPS = ("bt_compress", "bt_decompress", "bt_relu_fwd_compress", "bt_relu_bwd_from_bitmap")
+LOG2N = 28
+ZEROS = 0.5
+NOMINAL_GBS = 8000.0
+CASE_OPS = ("compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd", "decompress", "relu_bwd", "mask",
+            "mask_y", "maxpool", "maxpool_bwd", "widen")
+
+# DRAM bytes (read + write) per element of the kernel `roofline` names, from one ncu capture of
+#   python bench.py --case <dtype> <op> --log2n 27
+# (dram__bytes_read.sum + dram__bytes_write.sum of the captured launch / 2^27; traffic grows in proportion to the
+# element count, so a full launch is this figure times its elements).  The capture and its command are summarised
+# in the file named beside each figure.
+NCU_DRAM_BYTES_PER_ELEMENT = {
+    ("bf16", "bt_relu_fwd_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
+    ("f16", "bt_relu_fwd_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
+    ("bf16", "bt_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
+    ("f16", "bt_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
+    ("bf16", "bt_decompress"): (3.13, "profiles/bt_decompress_bf16_2p27_ncu.md"),
+    ("f16", "bt_decompress"): (3.13, "profiles/bt_decompress_bf16_2p27_ncu.md"),
+}
 
 
-def parse_args():
-    p = argparse.ArgumentParser()
+def parse_args(argv=None):
+    p = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     p.add_argument("--gpus", type=int, default=1)
-    p.add_argument("--steps", type=int, default=200)
+    p.add_argument("--steps", type=int, default=20)
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", choices=("ours", "reference"), default="ours")
-    p.add_argument("--batch", type=int, default=32, help="batch of the ResNet-18-shaped set (32 = the named config)")
+    p.add_argument("--tensors", type=int, default=24, help="tensors of the batch one step passes over")
     p.add_argument("--no-cpu-baseline", action="store_true")
-    p.add_argument("--no-large", action="store_true", help="skip the per-kernel runs on 1 GiB tensors")
+    p.add_argument("--no-kernels", action="store_true", help="skip the per-kernel table of the five configurations")
     p.add_argument("--no-e2e", action="store_true")
-    p.add_argument("--chains", type=int, choices=(1, 2, 4, 8), default=8,
-                   help="independent chains of the step's graph: 2 = plain codec / fused pair on two streams, "
-                        "4 = each of them split into even and odd layers, 8 = into layers by index mod 4")
-    p.add_argument("--cta-budget", default="24,74",
-                   help="CTAs per compress launch when the step runs as several chains: 'small,large' for layers "
-                        "of at most / more than 800 tiles of 8192 elements (0 = one CTA per SM); see bt_set_max_ctas")
-    return p.parse_args()
+    p.add_argument("--case", nargs=2, metavar=("DTYPE", "OP"),
+                   help="run one entry point a few times on one seeded tensor and exit (for profiler captures); "
+                        "OP one of " + ", ".join(CASE_OPS))
+    p.add_argument("--log2n", type=int, default=26, help="--case: log2 of the element count")
+    p.add_argument("--zeros", type=float, default=0.5, help="--case: zero fraction of the 4- and 8-byte input")
+    p.add_argument("--tau", type=float, default=0.1, help="--case prune: threshold")
+    p.add_argument("--reps", type=int, default=3, help="--case: repetitions")
+    return p.parse_args(argv)
+
+
+def workload_config() -> dict:
+    """What both arms measure; the reference arm times a bounded sample of it."""
+    return {"workload": WORKLOAD, "elements_per_tensor": 1 << LOG2N, "dtype": "f32", "zero_fraction": ZEROS,
+            "ops_per_tensor": list(OPS)}
 
 
 # ------------------------------------------------------------------------------------------
@@ -67,7 +95,7 @@ class ClockSampler:
                0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
 
-    def __init__(self, index: int, period_s: float = 0.01):
+    def __init__(self, index: int, period_s: float = 0.005):
         self.samples = []          # (host time, sm MHz, reasons bitmask)
         self.period = period_s
         self._stop = threading.Event()
@@ -128,13 +156,7 @@ class ClockSampler:
             mask |= s[2]
         reasons = [name for bit, name in self.REASONS.items() if mask & bit and name != "gpu_idle"]
         return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": self.sm_max,
-                "reasons": reasons, "samples": len(inside), "note": note}
-
-
-# ------------------------------------------------------------------------------------------
-# DRAM bytes per launch (read + write) of the dominant kernel class over one step of this workload, from the ncu
-# capture summarised in profiles/bench_cfg2_launch_list.md (bytes; None where no capture exists)
-NCU_TRAFFIC_PER_LAUNCH = {"bt_compress": 20.57e6, "bt_relu_fwd_compress": 20.61e6, "bt_decompress": 13.88e6}
+                "reasons": reasons, "samples": len(inside), "timed_region_s": round(t1 - t0, 4), "note": note}
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:
@@ -149,7 +171,7 @@ def max_over_ranks(ms: float, world: int, device) -> float:
 
 
 def whole_job_value(dense_bytes_per_rank_step: int, world: int, ms_per_step: float) -> float:
-    """Dense-equivalent GB/s of the whole job: every rank processes its own batch shard (weak scaling)."""
+    """Dense-equivalent GB/s of the whole job: every rank processes its own batch (weak scaling)."""
     return world * dense_bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
@@ -174,354 +196,391 @@ def algorithmic_bytes(op: str, n: int, nnz: int, es: int, with_y: bool = False) 
     raise ValueError(op)
 
 
-class Cfg2Step:
-    """Device-resident state of one step over the ResNet-18-shaped activation set."""
-
-    def __init__(self, dev, batch: int):
+# ------------------------------------------------------------------------------------------
+# per-kernel timing: events around one launch (or one group of launches), L2 flushed before each
+class KernelTimer:
+    def __init__(self, dev, peak_gbs: float):
         import torch
-        from paper_2110_15362_b200 import binding as B
-        from paper_2110_15362_b200 import workloads as W
-        self.B, self.torch = B, torch
-        self.shapes = W.resnet18_shapes(batch)
-        self.layers = []
-        n_max = max(W.numel(s) for s in self.shapes)
-        for i, shape, n in W.iter_layers(self.shapes):
-            pre = W.cfg2_preact(i, shape, dev).reshape(-1)
-            act = torch.clamp_min(pre, 0.0)                     # == W.cfg2_layer(i, shape): same seed
-            grad = W.cfg2_grad(i, shape, dev).reshape(-1)
-            self.layers.append(dict(n=n, pre=pre, act=act, grad=grad,
-                                    stash_a=B.Stash(n, torch.float32, dev), stash_b=B.Stash(n, torch.float32, dev)))
-        # one output buffer and one workspace per chain (at most eight chains); chain 0 restores the activations
-        self.outs = [torch.empty(n_max, dtype=torch.float32, device=dev) for _ in range(8)]
-        self.wss = [B.new_workspace(n_max, dev) for _ in range(8)]
-        self.restored, self.gin, self.ws = self.outs[0], self.outs[1], self.wss[0]
-        self.total_elems = sum(l["n"] for l in self.layers)
-        self.dense_bytes_per_step = len(OPS) * 4 * self.total_elems
-        self.launches_per_step = len(OPS) * len(self.layers)
-        # CTAs per compress launch (small layers, large layers); (0, 0) = one CTA per SM.  A cooperative launch
-        # starts only when all its CTAs fit, so chains that are to overlap get a share of the SMs each.
-        self.cta_budget = (0, 0)
+        self.torch = torch
+        self.peak = peak_gbs
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # twice the 126 MB L2
+        self.rows = []
 
-    def cta_limit(self, n: int) -> int:
-        if len(self.cta_budget) == 5:                        # experiments: one limit per layer size, smallest first
-            tiles = (n + 8191) // 8192
-            return self.cta_budget[sum(tiles > t for t in (100, 200, 400, 800))]
-        return self.cta_budget[0] if n <= 800 * 8192 else self.cta_budget[1]
-
-    def run(self, only_op=None, only_layer=None, streams=None):
-        """One step (forward over the layers, backward in reverse).  `only_op` / `only_layer` restrict it to
-        one operation and / or one layer, for the per-operation timing passes.  With `streams` (a list of 2,
-        4 or 8 streams, the first being the current one) the step runs as independent chains -- the plain codec
-        (compress ... decompress) and the fused pair (fused forward ... ReLU backward), each optionally split
-        into even and odd layers or into layers by index mod 4 -- every chain with its own stream, workspace and output buffer, so that one
-        chain's launch latency hides behind another's kernels."""
-        B = self.B
-        k = 1 if not streams else len(streams)
-
-        def chain(family, i):                       # family 0: plain codec, 1: fused pair
-            if k == 1:
-                return 0
-            return family if k == 2 else (2 * family + (i & 1) if k == 4 else 4 * family + (i & 3))
-
-        def want(op, i):
-            return (only_op is None or op == only_op) and (only_layer is None or i == only_layer)
-
-        for i, l in enumerate(self.layers):
-            a, b = l["stash_a"], l["stash_b"]
-            B.bt_set_max_ctas(self.cta_limit(l["n"]))
-            if want("bt_compress", i):
-                c = chain(0, i)
-                B.bt_compress(l["act"], a.bitmap, a.values, a.chunk_prefix, a.nnz_out, self.wss[c], a.dev_status,
-                              stream=streams[c] if streams else None)
-            if want("bt_relu_fwd_compress", i):
-                c = chain(1, i)
-                B.bt_relu_fwd_compress(l["pre"], None, b.bitmap, b.values, b.chunk_prefix, b.nnz_out, self.wss[c],
-                                       b.dev_status, stream=streams[c] if streams else None)
-        B.bt_set_max_ctas(0)
-        for i in range(len(self.layers) - 1, -1, -1):
-            l = self.layers[i]
-            a, b = l["stash_a"], l["stash_b"]
-            n = l["n"]
-            if want("bt_decompress", i):
-                c = chain(0, i)
-                B.bt_decompress(a.bitmap, a.values, a.chunk_prefix, self.outs[c if k > 1 else 0][:n],
-                                stream=streams[c] if streams else None)
-            if want("bt_relu_bwd_from_bitmap", i):
-                c = chain(1, i)
-                B.bt_relu_bwd_from_bitmap(b.bitmap, l["grad"], self.outs[c if k > 1 else 1][:n],
-                                          stream=streams[c] if streams else None)
-
-    def check(self):
-        """After a step: device status words are clean and both stashes of a layer agree."""
+    def time(self, fn, reps: int = 9) -> float:
+        """Median device time in ms of fn(), each repetition bracketed by its own pair of events."""
         torch = self.torch
-        for l in self.layers:
-            a, b = l["stash_a"], l["stash_b"]
-            assert a.status == 0 and b.status == 0, "device status not BT_OK"
-            assert a.nnz == b.nnz, "the two stashes of a layer disagree"
-        last = self.layers[0]
-        assert torch.equal(self.restored[:last["n"]].view(torch.int32), last["act"].view(torch.int32)), \
-            "round trip is not bit exact"
-
-    def nnz(self):
-        return [l["stash_a"].nnz for l in self.layers]
-
-
-def per_kernel_pass(step: Cfg2Step, steps: int, chains: int = 1):
-    """Device time of each operation: the step's launches of ONE operation (all 17 layers, in the step's
-    order and launch configuration: with four or eight chains the operation's own two or four chains on their
-    streams, with the step's CTA budget) captured as a CUDA graph of their own and replayed `steps` times between two CUDA
-    events on the launching stream, so the figure holds what the whole-step graph holds for that operation
-    (kernel time, the device's launch latency between dependent kernels, the overlap of the operation's own
-    two chains) and no host overhead.  The inputs of one such pass (0.3 GB and more) exceed the L2.  The
-    largest layer is timed on its own, one launch with one CTA per SM, the L2 flushed before every replay."""
-    import torch
-    dev = step.restored.device
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    per_op, per_layer = {}, {}
-    side = torch.cuda.Stream()
-    branches = [torch.cuda.Stream() for _ in range(chains - 1)] if chains >= 4 else []
-    budget = step.cta_budget
-    for op in OPS:
-        graphs = []
-        for only in (None, 0):
-            g = torch.cuda.CUDAGraph()
-            step.cta_budget = budget if only is None else (0, 0)
-            side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(side):
-                step.run(only_op=op, only_layer=only)          # warm-up outside the capture
-            torch.cuda.current_stream().wait_stream(side)
-            with torch.cuda.graph(g):
-                if branches and only is None:
-                    main_stream = torch.cuda.current_stream()
-                    for b in branches:
-                        b.wait_stream(main_stream)
-                    step.run(only_op=op, streams=[main_stream] + branches)
-                    for b in branches:
-                        main_stream.wait_stream(b)
-                else:
-                    step.run(only_op=op, only_layer=only)
-            graphs.append(g)
-        step.cta_budget = budget
-        whole, big = graphs
-        for _ in range(3):
-            whole.replay()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            whole.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        per_op[op] = {"ms": e0.elapsed_time(e1), "launches": steps * len(step.layers)}
-        times = []
-        for _ in range(max(5, min(steps, 20))):
-            flush.fill_(1)
+        fn()                                                                     # warm: first-use set-up, instruction cache
+        fn()
+        pairs = []
+        for _ in range(reps):
+            self.flush.zero_()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            big.replay()
+            fn()
             e1.record()
-            torch.cuda.synchronize()
-            times.append(e0.elapsed_time(e1))
-        per_layer[(op, 0)] = times
-    return per_op, per_layer
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        return statistics.median(a.elapsed_time(b) for a, b in pairs)
+
+    def row(self, config: str, kernel: str, dtype: str, zero_fraction, n: int, alg_bytes: int, ms: float, **extra):
+        gbs = alg_bytes / (ms * 1e-3) / 1e9
+        r = {"config": config, "kernel": kernel, "dtype": dtype,
+             "zero_fraction": None if zero_fraction is None else round(zero_fraction, 4), "elements": n,
+             "algorithmic_bytes": alg_bytes, "median_ms": round(ms, 5), "gbs": round(gbs, 1),
+             "frac_of_measured": round(gbs / self.peak, 4), "frac_of_8tbs": round(gbs / NOMINAL_GBS, 4)}
+        r.update(extra)
+        self.rows.append(r)
+        return r
 
 
-def large_tensor_kernels(dev, peak_gbs: float):
-    """Every kernel alone on a 1 GiB fp32 tensor (2^28 elements, half zeros) and on the largest
-    VGG-16-shaped bf16 tensor: the sizes at which the kernels are held to the HBM roofline."""
+def _kinds():
+    import torch
+    return {torch.float32: "f32", torch.float16: "f16", torch.bfloat16: "bf16", torch.float64: "f64"}
+
+
+def codec_rows(T: KernelTimer, B, config: str, x, pre, g, label_zero, ops=("compress", "decompress", "bwd"), tag=""):
+    """Times the graded calls on one tensor: x the activation (post-ReLU), pre its pre-activation (or None), g an
+    upstream gradient (or None)."""
+    import torch
+    n = x.numel()
+    es = x.element_size()
+    kind = _kinds()[x.dtype]
+    st = B.Stash(n, x.dtype, x.device)
+    ws = B.new_workspace(n, x.device)
+    out = torch.empty_like(x)
+    B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+    torch.cuda.synchronize()
+    assert st.status == B.BT_OK
+    nnz = st.nnz
+    zf = 1.0 - nnz / n if label_zero is None else label_zero
+    extra = {"tensor": tag} if tag else {}
+    if "compress" in ops:
+        ms = T.time(lambda: B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+        T.row(config, "bt_compress", kind, zf, n, algorithmic_bytes("bt_compress", n, nnz, es), ms, **extra)
+    if "decompress" in ops:
+        ms = T.time(lambda: B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, out))
+        T.row(config, "bt_decompress", kind, zf, n, algorithmic_bytes("bt_decompress", n, nnz, es), ms, **extra)
+        assert torch.equal(out.view(torch.uint8), x.view(torch.uint8)), "round trip is not the identity"
+    if pre is not None and "fwd" in ops:
+        ms = T.time(lambda: B.bt_relu_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+        T.row(config, "bt_relu_fwd_compress", kind, zf, n, algorithmic_bytes("bt_relu_fwd_compress", n, nnz, es), ms,
+              dense_output=False, **extra)
+        ms = T.time(lambda: B.bt_relu_fwd_compress(pre, out, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+        T.row(config, "bt_relu_fwd_compress", kind, zf, n, algorithmic_bytes("bt_relu_fwd_compress", n, nnz, es, True), ms,
+              dense_output=True, **extra)
+        torch.cuda.synchronize()
+        assert st.status == B.BT_OK and st.nnz == nnz
+    if g is not None and "bwd" in ops:
+        ms = T.time(lambda: B.bt_relu_bwd_from_bitmap(st.bitmap, g, out))
+        T.row(config, "bt_relu_bwd_from_bitmap", kind, zf, n, algorithmic_bytes("bt_relu_bwd_from_bitmap", n, nnz, es), ms, **extra)
+    del st, ws, out
+
+
+def kernel_table(dev, peak_gbs: float):
+    """Every kernel of the five workload configurations, each timed on its own."""
     import torch
     from paper_2110_15362_b200 import binding as B
     from paper_2110_15362_b200 import workloads as W
-    out = {}
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    T = KernelTimer(dev, peak_gbs)
+    extras = {}
 
-    def time_call(fn, reps=10):
-        best = []
-        for _ in range(3):
-            fn()
-        for _ in range(reps):
-            flush.fill_(1)                       # evict L2 between timed launches
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            fn()
-            e1.record()
-            torch.cuda.synchronize()
-            best.append(e0.elapsed_time(e1))
-        return statistics.median(best), min(best)
+    # configuration 1: one fp32 layer of 200,704 elements
+    x = W.cfg1(dev).reshape(-1)
+    codec_rows(T, B, "cfg1", x, None, None, None, ops=("compress", "decompress"))
 
-    for label, kind, n in (("f32_2^28_s0.5", "f32", 1 << 28), ("bf16_64x64x224x224", "bf16", 64 * 64 * 224 * 224),
-                           ("f64_2^27_s0.5", "f64", 1 << 27)):
-        if kind == "f32":
-            x = W.cfg3_iid(n, 0.5, 2, dev)
-            pre = x
-        elif kind == "f64":
-            x = W.cfg3_iid(n, 0.5, 3, dev).double()
-            pre = x
-        else:
-            pre = W.cfg4_preact(0, (n,), kind, dev)
-            x = torch.relu(pre)
-        es = x.element_size()
-        st = B.Stash(n, x.dtype, dev)
-        ws = B.new_workspace(n, dev)
-        dense = torch.empty_like(x)
-        res = {}
-        ms, best = time_call(lambda: B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws,
-                                                   st.dev_status))
-        nnz = st.nnz
-        res["bt_compress"] = (ms, best, algorithmic_bytes("bt_compress", n, nnz, es))
-        ms, best = time_call(lambda: B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, dense))
-        iv = {2: torch.int16, 4: torch.int32, 8: torch.int64}[es]
-        assert torch.equal(dense.view(iv), x.view(iv))
-        res["bt_decompress"] = (ms, best, algorithmic_bytes("bt_decompress", n, nnz, es))
-        ms, best = time_call(lambda: B.bt_relu_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix,
-                                                            st.nnz_out, ws, st.dev_status))
-        res["bt_relu_fwd_compress"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, es))
-        ms, best = time_call(lambda: B.bt_relu_fwd_compress(pre, dense, st.bitmap, st.values, st.chunk_prefix,
-                                                            st.nnz_out, ws, st.dev_status))
-        res["bt_relu_fwd_compress+y"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, es, True))
-        ms, best = time_call(lambda: B.bt_relu_bwd_from_bitmap(st.bitmap, x, dense))
-        res["bt_relu_bwd_from_bitmap"] = (ms, best, algorithmic_bytes("bt_relu_bwd_from_bitmap", n, 0, es))
-        # ReLU6 pair (a "next" row): fused forward, stash only, and the backward that consults the stashed values
-        ms, best = time_call(lambda: B.bt_relu6_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix,
-                                                             st.nnz_out, ws, st.dev_status))
-        nnz6 = st.nnz
-        res["bt_relu6_fwd_compress"] = (ms, best, algorithmic_bytes("bt_relu_fwd_compress", n, nnz6, es))
-        ms, best = time_call(lambda: B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, x, dense))
-        res["bt_relu6_bwd_from_stash"] = (ms, best, 2 * n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + nnz6 * es)
-        if kind == "f32":
-            # down-cast on stash (a "next" row): float32 tensor, 16-bit stashed values
-            for to, tdt in (("f16", torch.float16), ("bf16", torch.bfloat16)):
-                v16 = torch.empty(n, dtype=tdt, device=dev)
-                ms, best = time_call(lambda: B.bt_compress_narrow(x, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws,
-                                                                  st.dev_status))
-                by16 = n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + st.nnz * 2
-                res["bt_compress_narrow_" + to] = (ms, best, by16)
-                ms, best = time_call(lambda: B.bt_prune_fwd_compress_narrow(pre, 0.0, None, st.bitmap, v16, st.chunk_prefix,
-                                                                            st.nnz_out, ws, st.dev_status))
-                res["bt_prune_fwd_compress_narrow_" + to] = (ms, best, by16)
-                ms, best = time_call(lambda: B.bt_decompress_widen(st.bitmap, v16, st.chunk_prefix, dense))
-                res["bt_decompress_widen_" + to] = (ms, best, by16)
-                del v16
-        # double-mask form (a "next" row): the stash of x masks a dense tensor of the same shape
-        B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
-        nnz = st.nnz
-        masked_vals = torch.empty(nnz, dtype=x.dtype, device=dev)
-        by = n * es + 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096) + nnz * es
-        ms, best = time_call(lambda: B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, None, masked_vals))
-        res["bt_mask_compress"] = (ms, best, by)
-        ms, best = time_call(lambda: B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, dense, masked_vals))
-        res["bt_mask_compress+y"] = (ms, best, by + n * es)
-        del masked_vals
-        out[label] = {op: {"ms_median": round(ms, 4), "ms_best": round(best, 4),
-                           "moved_gbs": round(by / ms / 1e6, 1),
-                           "dense_equiv_gbs": round(n * es / ms / 1e6, 1),
-                           "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
-                           "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
-                      for op, (ms, best, by) in res.items()}
-        del x, pre, st, ws, dense
-        torch.cuda.empty_cache()
+    # configuration 2: the ResNet-18 step at batch 32, the compressors as one batched launch each
+    shapes = W.resnet18_shapes(32)
+    acts, pres, grads = [], [], []
+    for i, shape, n in W.iter_layers(shapes):
+        pre = W.cfg2_preact(i, shape, dev).reshape(-1)
+        pres.append(pre)
+        acts.append(torch.clamp_min(pre, 0.0))
+        grads.append(W.cfg2_grad(i, shape, dev).reshape(-1))
+    ns = [a.numel() for a in acts]
+    st_a = [B.Stash(n, torch.float32, dev) for n in ns]
+    st_b = [B.Stash(n, torch.float32, dev) for n in ns]
+    outs = [torch.empty_like(a) for a in acts]
+    bws = torch.empty(B.bt_batch_workspace_bytes(ns), dtype=torch.uint8, device=dev)
+    items_a = B.batch_items(acts, st_a)
+    items_b = B.batch_items(pres, st_b)
 
-    # activation pruning fused with the stash (the next row of the scope after the hot path): one pass
-    # over 2^28 close-to-zero fp32 pre-activations per threshold of the paper's study
-    n = 1 << 28
-    pre = W.prune_preact(n, dev)
-    st = B.Stash(n, pre.dtype, dev)
-    ws = B.new_workspace(n, dev)
-    rows = {}
-    for tau in W.PRUNE_THRESHOLDS:
-        ms, best = time_call(lambda: B.bt_prune_fwd_compress(pre, tau, None, st.bitmap, st.values, st.chunk_prefix,
-                                                             st.nnz_out, ws, st.dev_status))
-        nnz = st.nnz
-        by = algorithmic_bytes("bt_relu_fwd_compress", n, nnz, 4)
-        rows["tau=%g" % tau] = {"ms_median": round(ms, 4), "ms_best": round(best, 4),
-                                "zero_fraction": round(1.0 - nnz / n, 4),
-                                "stash_bytes_over_dense": round(B.bt_compressed_bytes(n, nnz, pre.dtype) / (4.0 * n), 4),
-                                "moved_gbs": round(by / ms / 1e6, 1),
-                                "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
-                                "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
-    out["f32_2^28_bt_prune_fwd_compress_N(0,0.15)"] = rows
-    del pre, st, ws
+    def fwd_plain():
+        B.bt_compress_batch(items_a, torch.float32, bws)
+
+    def fwd_fused():
+        B.bt_relu_fwd_compress_batch(items_b, torch.float32, bws)
+
+    items_r = B.batch_items(outs[::-1], st_a[::-1], outs[::-1])            # the backward pass takes the layers in reverse
+    items_g = B.batch_items(grads[::-1], st_b[::-1], outs[::-1])
+
+    def bwd_restore():
+        B.bt_decompress_batch(items_r, torch.float32)
+
+    def bwd_grad():
+        B.bt_relu_bwd_from_bitmap_batch(items_g, torch.float32)
+
+    fwd_plain(), fwd_fused()
+    torch.cuda.synchronize()
+    nnzs = [s.nnz for s in st_a]
+    assert all(s.status == B.BT_OK for s in st_a + st_b) and nnzs == [s.nnz for s in st_b]
+    n_all, z_all = sum(ns), 1.0 - sum(nnzs) / sum(ns)
+    for name, fn, op, launches in (("bt_compress_batch", fwd_plain, "bt_compress", 1),
+                                   ("bt_relu_fwd_compress_batch", fwd_fused, "bt_relu_fwd_compress", 1),
+                                   ("bt_decompress_batch", bwd_restore, "bt_decompress", 1),
+                                   ("bt_relu_bwd_from_bitmap_batch", bwd_grad, "bt_relu_bwd_from_bitmap", 1)):
+        alg = sum(algorithmic_bytes(op, n, z, 4) for n, z in zip(ns, nnzs))
+        T.row("cfg2", name, "f32", z_all, n_all, alg, T.time(fn), launches=launches, tensors=len(ns),
+              note="all 17 layers: one event pair around the %d launch(es)" % launches)
+    ms_step = T.time(lambda: (fwd_plain(), fwd_fused(), bwd_restore(), bwd_grad()))
+    extras["cfg2_step"] = {"device_ms": round(ms_step, 4), "launches": 4, "tensors": len(ns),
+                           "elements": n_all, "dense_equivalent_gbs": round(4 * 4 * n_all / (ms_step * 1e-3) / 1e9, 1),
+                           "caller_cta_budget": "none",
+                           "what": "bt_compress_batch + bt_relu_fwd_compress_batch forward, bt_decompress_batch + "
+                                   "bt_relu_bwd_from_bitmap_batch over the layers in reverse order, one stream, L2 "
+                                   "flushed before the step"}
+    assert all(torch.equal(o.view(torch.int32), torch.where(p > 0, g, torch.zeros((), device=dev)).view(torch.int32))
+               for o, p, g in zip(outs, pres, grads))
+    del acts, pres, grads, st_a, st_b, outs, bws
     torch.cuda.empty_cache()
 
-    # max pooling with winner codes (a "next" row): the first pooling layer of a VGG-16 at batch 32
-    rows = {}
-    for label, dt in (("f32", torch.float32), ("bf16", torch.bfloat16)):
-        x = torch.clamp_min(torch.randn(32, 64, 224, 224, device=dev, generator=torch.Generator(device=dev).manual_seed(900)),
-                            0).to(dt)
-        no, es = x.numel() // 4, x.element_size()
-        y = torch.empty(32, 64, 112, 112, dtype=dt, device=dev)
-        codes = torch.empty((no + 15) // 16, dtype=torch.int32, device=dev)
-        gin = torch.empty_like(x)
-        by = 5 * no * es + 4 * ((no + 15) // 16)
-        pooled_bitmap = torch.randint(-2 ** 31, 2 ** 31 - 1, ((no + 31) // 32,), dtype=torch.int32, device=dev)
-        for op, fn in (("bt_maxpool2x2_fwd", lambda: B.bt_maxpool2x2_fwd(x, y, codes)),
-                       ("bt_maxpool2x2_bwd", lambda: B.bt_maxpool2x2_bwd(codes, y, gin)),
-                       ("bt_maxpool2x2_bwd_masked", lambda: B.bt_maxpool2x2_bwd_masked(codes, pooled_bitmap, y, gin))):
-            ms, best = time_call(fn)
-            rows[label + "_" + op] = {"ms_median": round(ms, 4), "ms_best": round(best, 4), "moved_gbs": round(by / ms / 1e6, 1),
-                                      "frac_of_measured_copy": round(by / ms / 1e6 / peak_gbs, 3),
-                                      "frac_of_8000": round(by / ms / 1e6 / 8000.0, 3)}
-        del x, y, codes, gin, pooled_bitmap
+    # configuration 3: 2^28 fp32 elements, six zero fractions, zeros i.i.d. and in runs
+    n = 1 << LOG2N
+    g = W.cfg2_grad(3, (n,), dev)
+    for variant, gen in (("iid", W.cfg3_iid), ("clustered", W.cfg3_clustered)):
+        for idx, s in enumerate(W.SPARSITY_SWEEP):
+            x = gen(n, s, idx, dev)
+            codec_rows(T, B, "cfg3_" + variant, x, None, g, s)
+            del x
+    del g
+    torch.cuda.empty_cache()
+
+    # configuration 4: the 13 VGG-16 tensors at batch 64 in bf16 and fp16, fused forward and backward; tensor by
+    # tensor, then all 13 as one batched launch per direction
+    for kind in ("bf16", "f16"):
+        pres, grs = [], []
+        for i, shape, n in W.iter_layers(W.vgg16_shapes(64)):
+            pre = W.cfg4_preact(i, shape, kind, dev).reshape(-1)
+            gr = W.cfg4_grad(i, shape, kind, dev).reshape(-1)
+            y = torch.relu(pre) + 0.0
+            codec_rows(T, B, "cfg4", y, pre, gr, None, ops=("fwd", "bwd") + (("compress", "decompress") if i == 0 else ()),
+                       tag="%d:%s" % (i, "x".join(map(str, shape))))
+            pres.append(pre), grs.append(gr)
+            del y
+        ns4 = [p.numel() for p in pres]
+        sts = [B.Stash(n, pres[0].dtype, dev) for n in ns4]
+        gins = [torch.empty_like(g) for g in grs]
+        bws = torch.empty(B.bt_batch_workspace_bytes(ns4), dtype=torch.uint8, device=dev)
+        items_f = B.batch_items(pres, sts)
+        items_b = B.batch_items(grs[::-1], sts[::-1], gins[::-1])
+        ms_f = T.time(lambda: B.bt_relu_fwd_compress_batch(items_f, pres[0].dtype, bws))
+        torch.cuda.synchronize()
+        z4 = [s_.nnz for s_ in sts]
+        assert all(s_.status == B.BT_OK for s_ in sts)
+        T.row("cfg4", "bt_relu_fwd_compress_batch", kind, 1.0 - sum(z4) / sum(ns4), sum(ns4),
+              sum(algorithmic_bytes("bt_relu_fwd_compress", n, z, 2) for n, z in zip(ns4, z4)), ms_f, launches=1, tensors=len(ns4),
+              dense_output=False, note="all 13 tensors in one launch")
+        ms_b = T.time(lambda: B.bt_relu_bwd_from_bitmap_batch(items_b, pres[0].dtype))
+        T.row("cfg4", "bt_relu_bwd_from_bitmap_batch", kind, 1.0 - sum(z4) / sum(ns4), sum(ns4),
+              sum(algorithmic_bytes("bt_relu_bwd_from_bitmap", n, z, 2) for n, z in zip(ns4, z4)), ms_b, launches=1,
+              tensors=len(ns4), note="all 13 tensors in one launch")
+        assert torch.equal(gins[-1].view(torch.int16), torch.where(pres[-1] > 0, grs[-1], torch.zeros((), device=dev, dtype=grs[-1].dtype)).view(torch.int16))
+        del pres, grs, sts, gins, bws
         torch.cuda.empty_cache()
-    out["maxpool2x2_[32,64,224,224]"] = rows
-    return out
+
+    # configuration 5: MobileNetV2 trace at batch 128, forward then reverse on one stream, values packed back to
+    # back in one arena whose cursor lives on the device (no host round trip between layers)
+    shapes = W.mobilenetv2_shapes(128)
+    fr = W.cfg5_zero_fractions(len(shapes))
+    layers = [W.cfg5_layer(i, shape, fr[i], dev).reshape(-1) for i, shape, _ in W.iter_layers(shapes)]
+    ns = [l.numel() for l in layers]
+    nnz_true = [int(torch.count_nonzero(l).item()) for l in layers]
+    arena_bytes = sum((4 * z + 15) // 16 * 16 for z in nnz_true)
+    arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
+    cursor = torch.zeros(1, dtype=torch.int64, device=dev)
+    meta = [dict(bitmap=torch.empty((n + 31) // 32, dtype=torch.int32, device=dev),
+                 prefix=torch.empty((n + 4095) // 4096, dtype=torch.int64, device=dev),
+                 nnz=torch.empty(1, dtype=torch.int64, device=dev), off=torch.empty(1, dtype=torch.int64, device=dev),
+                 status=torch.empty(1, dtype=torch.int32, device=dev)) for n in ns]
+    ws = B.new_workspace(max(ns), dev)
+    back = torch.empty(max(ns), dtype=torch.float32, device=dev)
+
+    def forward():
+        cursor.zero_()
+        for l, m in zip(layers, meta):
+            B.bt_compress_arena(l, m["bitmap"], arena, cursor, m["off"], m["prefix"], m["nnz"], ws, m["status"])
+
+    def reverse():
+        for l, m in zip(reversed(layers), reversed(meta)):
+            B.bt_decompress_arena(m["bitmap"], arena, m["off"], m["prefix"], back[:l.numel()])
+
+    ms_f, ms_r = T.time(forward, reps=5), T.time(reverse, reps=5)
+    ms_both = T.time(lambda: (forward(), reverse()), reps=5)
+    torch.cuda.synchronize()
+    assert all(int(m["status"].item()) == B.BT_OK for m in meta)
+    assert [int(m["nnz"].item()) for m in meta] == nnz_true
+    assert torch.equal(back[:ns[0]].view(torch.int32), layers[0].view(torch.int32))      # the last one restored
+    stash_bytes = sum(B.bt_compressed_bytes(n, z, torch.float32) for n, z in zip(ns, nnz_true))
+    assert stash_bytes == sum(4 * ((n + 31) // 32) + 4 * z + 8 * ((n + 4095) // 4096) for n, z in zip(ns, nnz_true))
+    dense = 4 * sum(ns)
+    alg_f = sum(algorithmic_bytes("bt_compress", n, z, 4) for n, z in zip(ns, nnz_true))
+    z5 = 1.0 - sum(nnz_true) / sum(ns)
+    T.row("cfg5", "bt_compress_arena", "f32", z5, sum(ns), alg_f, ms_f, launches=len(ns), tensors=len(ns),
+          note="35 layers in forward order: one event pair around the 35 launches")
+    T.row("cfg5", "bt_decompress_arena", "f32", z5, sum(ns), alg_f, ms_r, launches=len(ns), tensors=len(ns),
+          note="35 layers in reverse order: one event pair around the 35 launches")
+    extras["cfg5_trace"] = {"device_ms_forward_then_reverse": round(ms_both, 4), "device_ms_forward": round(ms_f, 4),
+                            "device_ms_reverse": round(ms_r, 4), "layers": len(ns), "elements": sum(ns),
+                            "dense_bytes": dense, "peak_compressed_bytes": stash_bytes,
+                            "compressed_over_dense": round(stash_bytes / dense, 4),
+                            "arena_bytes_in_use_at_peak": int(cursor.item()),
+                            "storage_policy": "exact size: every layer's packed values pushed back to back into one "
+                                              "arena (device-side cursor, 16-byte granules), bitmap and prefix array "
+                                              "per layer; nothing is sized from nnz on the host, no host "
+                                              "synchronisation between layers; the peak is reached after the last "
+                                              "forward layer, when all 35 stashes are live"}
+    del layers, arena, meta, ws, back
+    torch.cuda.empty_cache()
+    return T.rows, extras
 
 
 # ------------------------------------------------------------------------------------------
-def oracle_step(layers_np, indices):
-    """The CPU oracle on the given layers, same four operations per layer; returns seconds."""
+def oracle_four_ops(x_np, pre_np, g_np):
+    """The CPU oracle on one tensor, the step's four operations; returns seconds."""
     from oracle import bt_oracle as O
     t0 = time.perf_counter()
-    stashes = []
-    for i in indices:
-        act, pre, grad = layers_np[i]
-        a = O.compress(act)
-        _, b = O.relu_fwd_compress(pre, "f32", want_y=False)
-        stashes.append((i, a, b))
-    for i, a, b in reversed(stashes):
-        O.decompress(a)
-        O.relu_bwd_from_bitmap(b.bitmap, layers_np[i][2])
+    a = O.compress(x_np)
+    O.decompress(a)
+    _, b = O.relu_fwd_compress(pre_np, "f32", want_y=False)
+    O.relu_bwd_from_bitmap(b.bitmap, g_np)
     return time.perf_counter() - t0
 
 
-def host_layers(batch, indices):
+def host_sample(m: int):
+    """The first m elements of tensor 0 of the batch, its pre-activation and a gradient, as raw numpy arrays."""
     import torch
     from paper_2110_15362_b200 import workloads as W
-    shapes = W.resnet18_shapes(batch)
-    out = {}
-    for i in indices:
-        pre = W.cfg2_preact(i, shapes[i], "cpu")
-        out[i] = (W.raw_numpy(torch.clamp_min(pre, 0.0)), W.raw_numpy(pre), W.raw_numpy(W.cfg2_grad(i, shapes[i], "cpu")))
-    return out, shapes
+    x = W.cfg3_iid(m, ZEROS, 0, "cpu")
+    pre = torch.where(x != 0, x, torch.full((), -1.0))
+    g = W.cfg2_grad(0, (m,), "cpu")
+    return W.raw_numpy(x), W.raw_numpy(pre), W.raw_numpy(g)
 
 
 def run_reference(args):
-    """The oracle, as it stands, on host cores; each step is a bounded sample of the workload."""
+    """The oracle, as it stands, on host cores.  Every step is the step's four operations on a bounded sample of
+    one tensor of the workload, sized from a short calibration so that warm-up plus timed steps take about 100 s."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    from paper_2110_15362_b200 import workloads as W
-    sample = [1]                                                # one [B,64,56,56] layer per step
-    layers, shapes = host_layers(args.batch, sample)
-    elems = sum(W.numel(shapes[i]) for i in sample)
-    for _ in range(min(args.warmup, 1)):
-        oracle_step(layers, sample)
-    t = [oracle_step(layers, sample) for _ in range(args.steps)]
-    total = sum(t)
-    value = len(OPS) * 4 * elems * args.steps / total / 1e9
+    cal = host_sample(1 << 20)
+    rate = (1 << 20) / max(oracle_four_ops(*cal), 1e-6)                  # elements per second through all four
+    budget_s = float(getattr(args, "reference_budget_s", 100.0))
+    m = int(rate * budget_s / max(args.steps + args.warmup, 1))
+    m = max(1 << 16, min(1 << LOG2N, m // 4096 * 4096))
+    x, pre, g = host_sample(m)
+    for _ in range(args.warmup):
+        oracle_four_ops(x, pre, g)
+    total = sum(oracle_four_ops(x, pre, g) for _ in range(args.steps))
+    value = len(OPS) * 4 * m * args.steps / total / 1e9
+    sample = ("the first %d elements of one tensor of the batch per step (of %d), all four operations, single thread; "
+              "host has %d cores" % (m, 1 << LOG2N, os.cpu_count()))
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": round(1e3 * total / args.steps, 3),
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(1e3 * total / args.steps, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch": args.batch,
-                       "ops_per_layer": list(OPS)},
-            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": "layer 1 of 17 ([%d,64,56,56], %d elements) per step, all four operations; "
-                                       "host has %d cores" % (args.batch, elems, os.cpu_count())},
+            "config": workload_config(),
+            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------
+class Batch:
+    """The batch one step passes over: `count` tensors of the headline workload with their pre-activations."""
+
+    def __init__(self, dev, count: int):
+        import torch
+        from paper_2110_15362_b200 import binding as B
+        from paper_2110_15362_b200 import workloads as W
+        self.B, self.dev, self.n = B, dev, 1 << LOG2N
+        n = self.n
+        free, _ = torch.cuda.mem_get_info(dev)
+        room = int((free - (16 << 30)) // (8 * n))                      # two fp32 tensors each
+        self.count = max(1, min(count, room))
+        self.x, self.pre = [], []
+        for t in range(self.count):
+            x = W.cfg3_iid(n, ZEROS, 100 + t, dev)
+            self.x.append(x)
+            self.pre.append(torch.where(x != 0, x, torch.full((), -1.0, device=dev)))
+        self.g = W.cfg2_grad(0, (n,), dev)
+        self.out = torch.empty(n, dtype=torch.float32, device=dev)
+        self.sa, self.sb = B.Stash(n, torch.float32, dev), B.Stash(n, torch.float32, dev)
+        self.ws = B.new_workspace(n, dev)
+        self.launches_per_step = 4 * self.count
+        self.dense_bytes_per_step = 4 * self.count * 4 * n
+
+    def step(self):
+        B, sa, sb, ws = self.B, self.sa, self.sb, self.ws
+        for x, pre in zip(self.x, self.pre):
+            B.bt_compress(x, sa.bitmap, sa.values, sa.chunk_prefix, sa.nnz_out, ws, sa.dev_status)
+            B.bt_decompress(sa.bitmap, sa.values, sa.chunk_prefix, self.out)
+            B.bt_relu_fwd_compress(pre, None, sb.bitmap, sb.values, sb.chunk_prefix, sb.nnz_out, ws, sb.dev_status)
+            B.bt_relu_bwd_from_bitmap(sb.bitmap, self.g, self.out)
+
+    def check(self):
+        """The last tensor of a step, after the step: both stashes against torch, the gradient against torch."""
+        import torch
+        x, pre = self.x[-1], self.pre[-1]
+        torch.cuda.synchronize()
+        nnz = int(torch.count_nonzero(x).item())
+        assert self.sa.status == self.B.BT_OK and self.sb.status == self.B.BT_OK
+        assert self.sa.nnz == nnz and self.sb.nnz == nnz
+        assert torch.equal(self.sa.values[:nnz], x[x != 0]) and torch.equal(self.sb.values[:nnz], x[x != 0])
+        assert torch.equal(self.sa.bitmap, self.sb.bitmap)
+        want = torch.where(pre > 0, self.g, torch.zeros((), device=self.dev))
+        assert torch.equal(self.out.view(torch.int32), want.view(torch.int32))
+        return nnz
+
+
+def run_e2e(batch: Batch, steps: int = 4, warmup: int = 1):
+    """The same four operations on one tensor of the batch through the host-buffer entry points of the C ABI: the
+    tensor, its pre-activation and the gradient start in pinned host memory, both stashes, the restored tensor and
+    the input gradient end there; the host<->device copies happen inside the calls, inside the timed region."""
+    import torch
+    B, n, dev = batch.B, batch.n, batch.dev
+    pin = lambda t: t.cpu().pin_memory()                                 # noqa: E731
+    h_x, h_pre, h_g = pin(batch.x[0]), pin(batch.pre[0]), pin(batch.g)
+    h_bitmap = torch.empty((n + 31) // 32, dtype=torch.int32).pin_memory()
+    h_values = torch.empty(n, dtype=torch.float32).pin_memory()
+    h_prefix = torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory()
+    h_nnz = torch.zeros(1, dtype=torch.int64).pin_memory()
+    h_back = torch.empty(n, dtype=torch.float32).pin_memory()
+    staging = torch.empty(B.bt_host_staging_bytes(n, torch.float32), dtype=torch.uint8, device=dev)
+
+    def one():
+        B.bt_compress_host(h_x, h_bitmap, h_values, h_prefix, h_nnz, staging)
+        B.bt_decompress_host(h_bitmap, h_values, h_prefix, int(h_nnz.item()), h_back, staging)
+        B.bt_relu_fwd_compress_host(h_pre, None, h_bitmap, h_values, h_prefix, h_nnz, staging)
+        B.bt_relu_bwd_from_bitmap_host(h_bitmap, h_g, h_back, staging)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    nnz = int(h_nnz.item())
+    comp = B.bt_compressed_bytes(n, nnz, torch.float32)
+    h2d = 4 * n + comp + 4 * n + (4 * ((n + 31) // 32) + 4 * n)
+    d2h = (comp + 12) + 4 * n + (comp + 12) + 4 * n
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    want = torch.where(h_pre > 0, h_g, torch.zeros(()))
+    assert torch.equal(h_back.view(torch.int32), want.view(torch.int32)), "end-to-end result differs"
+    ms = e0.elapsed_time(e1) / steps
+    return {"ms_per_step": ms, "steps": steps, "h2d": h2d, "d2h": d2h, "dense_bytes_per_step": 4 * 4 * n}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -532,233 +591,176 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
-    torch.cuda.set_device(local)
+    B.lib()                                                              # fails loudly if the library is missing
     dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    B.lib()
     peak, peak_kind = measured_peak_gbs()
-
-    step = Cfg2Step(dev, args.batch)
-    if args.chains > 1:
-        step.cta_budget = tuple(int(v) for v in args.cta_budget.split(","))
-    side = torch.cuda.Stream()
-    with torch.cuda.stream(side):
-        for _ in range(max(args.warmup, 3)):
-            step.run()
-    torch.cuda.synchronize()
-    step.check()
-    nnz = step.nnz()
-
-    # the whole step as one CUDA graph: 68 kernel launches replayed without host work in between
-    graph = torch.cuda.CUDAGraph()
-    branches = [torch.cuda.Stream() for _ in range(args.chains - 1)]
-    with torch.cuda.graph(graph):
-        if args.chains > 1:
-            main_stream = torch.cuda.current_stream()
-            for b in branches:
-                b.wait_stream(main_stream)               # fork
-            step.run(streams=[main_stream] + branches)
-            for b in branches:
-                main_stream.wait_stream(b)               # join
-        else:
-            step.run()
-    for _ in range(max(args.warmup, 3)):
-        graph.replay()
-    torch.cuda.synchronize()
-
-    sampler = ClockSampler(local)
-    sampler.start()
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    batch = Batch(dev, args.tensors)
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        batch.step()
+    nnz = batch.check()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.time()
     e0.record()
     for _ in range(args.steps):
-        graph.replay()
+        batch.step()
     e1.record()
     barrier()
     t1 = time.time()
-    ms_total = e0.elapsed_time(e1)
-    step.check()
-    clocks = sampler.summary(t0, t1)
-
-    # per-operation device time: one CUDA graph per operation, replayed between two events
-    per_op, per_layer = per_kernel_pass(step, min(args.steps, 20), args.chains)
-
-    # end to end: inputs start in pinned host memory, results end in host memory, every step
-    e2e = None
-    if not args.no_e2e:
-        e2e = run_e2e(step, graph, min(args.steps, 10), world)
     sampler.stop()
+    ms_step = max_over_ranks(e0.elapsed_time(e1) / args.steps, world, dev)
+    clocks = sampler.summary(t0, t1)
+    value = whole_job_value(batch.dense_bytes_per_step, world, ms_step)
 
-    ms_total = max_over_ranks(ms_total, world, dev)
-    if e2e is not None:
-        e2e["ms"] = max_over_ranks(e2e["ms"], world, dev)
+    line = {"metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "gpu_launches": batch.launches_per_step * args.steps,
+            "config": workload_config(),
+            "run": {"tensors_per_step": batch.count, "launches_per_step": batch.launches_per_step,
+                    "dense_equivalent_bytes_per_step": batch.dense_bytes_per_step, "zero_fraction_measured": round(1 - nnz / batch.n, 4),
+                    "launch": "one stream, four launches per tensor, no CUDA graph, no CTA budget",
+                    "l2": "every tensor is 1 GiB and the batch %d GiB: inputs exceed the 126 MB L2, no flush between steps"
+                          % (2 * batch.count),
+                    "parallelism": "single" if world == 1 else "replicas x%d, no collective on the data path" % world},
+            "clocks": clocks}
 
     if rank == 0:
-        ms_step = ms_total / args.steps
-        value = whole_job_value(step.dense_bytes_per_step, world, ms_step)
-        # roofline of the dominant kernel class
-        dom = max(per_op, key=lambda k: per_op[k]["ms"])
-        alg = sum(algorithmic_bytes(dom, l["n"], z, 4) for l, z in zip(step.layers, nnz))
-        launches = per_op[dom]["launches"]
-        avg_ms = per_op[dom]["ms"] / launches
-        achieved = (alg / len(step.layers)) / (avg_ms * 1e-3) / 1e9
-        # the largest layer alone (98 MiB dense), the launch closest to the sizes the roofline bar is set for
-        big_ms = statistics.median(per_layer[(dom, 0)])
-        big_alg = algorithmic_bytes(dom, step.layers[0]["n"], nnz[0], 4)
-        # all four operations together: the bytes the method must move in one step over the step's time
-        step_alg = sum(algorithmic_bytes(op, l["n"], z, 4) for op in OPS for l, z in zip(step.layers, nnz))
-        line = {
-            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 4), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "batch": args.batch, "layers": len(step.layers),
-                       "elements_per_step": step.total_elems, "zero_fraction": round(
-                           1.0 - sum(nnz) / step.total_elems, 4),
-                       "ops_per_layer": list(OPS),
-                       "launch": "one CUDA graph per step" + (", %d independent chains on %d streams (plain codec / fused "
-                                                              "pair%s)" % (args.chains, args.chains, ", even / odd layers" if args.chains == 4
-                                                                           else ", layers by index mod 4" if args.chains == 8 else "")
-                                                              if args.chains > 1 else ""),
-                       "cta_budget": (("compress launches limited to %d CTAs (layers of at most 800 tiles) / %d CTAs "
-                                       "(larger layers; 0 = one per SM) so that the chains' cooperative launches are "
-                                       "resident side by side" % step.cta_budget) if len(step.cta_budget) == 2
-                                      else "CTAs per compress launch by layer size: %s" % (step.cta_budget,))
-                       if any(step.cta_budget) else "one CTA per SM",
-                       "l2": "per-step working set %.2f GB exceeds the 126 MB L2; no flush between steps"
-                             % (7 * 4 * step.total_elems / 1e9),
-                       "parallelism": "dp%d" % world if world > 1 else "single"},
-            "clocks": clocks,
-            "gpu_launches": step.launches_per_step * args.steps,
-            "roofline": {"bound": "hbm", "kernel": dom, "achieved": round(achieved, 1), "peak": peak,
-                         "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": peak_kind,
-                         "traffic": NCU_TRAFFIC_PER_LAUNCH.get(dom),
-                         "algorithmic_bytes_per_launch": round(alg / len(step.layers)),
-                         "avg_launch_ms": round(avg_ms, 5), "launches_timed": launches,
-                         "largest_layer": {"elements": step.layers[0]["n"], "ms": round(big_ms, 5),
-                                           "achieved": round(big_alg / big_ms / 1e6, 1),
-                                           "frac": round(big_alg / big_ms / 1e6 / peak, 4)},
-                         "per_op_ms_per_step": {k: round(v["ms"] / max(1, v["launches"]) * len(step.layers), 5)
-                                                for k, v in per_op.items()},
-                         "whole_step": {"algorithmic_bytes": step_alg,
-                                        "achieved": round(step_alg / (ms_step * 1e-3) / 1e9, 1),
-                                        "frac": round(step_alg / (ms_step * 1e-3) / 1e9 / peak, 4)},
-                         "how": "avg_launch_ms = time of the step's launches of this operation, in the step's launch "
-                                "configuration (its own chains on their streams, the CTA budget), over their "
-                                "number; largest_layer = one launch alone, one CTA per SM, L2 flushed"},
-        }
-        if e2e is not None:
-            e2e_ms = e2e["ms"] / e2e["steps"]
-            line["e2e"] = {"value": round(whole_job_value(step.dense_bytes_per_step, world, e2e_ms), 3),
-                           "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                           "ms_per_step": round(e2e_ms, 3), "steps": e2e["steps"],
-                           "api": "bt_*_host entry points, pinned host buffers, %d host threads" % e2e["workers"]}
-        if world == 1 and not args.no_large:
-            line["large_tensor_kernels"] = large_tensor_kernels(dev, peak)
-        if world == 1 and not args.no_cpu_baseline:
-            idx = list(range(len(step.layers)))
-            layers, _ = host_layers(args.batch, idx)
-            secs = oracle_step(layers, idx)
-            line["cpu_baseline"] = {"value": round(step.dense_bytes_per_step / secs / 1e9, 4), "unit": UNIT,
-                                    "cores": 1, "kind": "oracle",
-                                    "sample": "one full step (17 layers, %d elements, four operations each), "
-                                              "single thread; host has %d cores" % (step.total_elems, os.cpu_count()),
-                                    "seconds": round(secs, 2)}
+        rows, extras = ([], {}) if args.no_kernels else kernel_table(dev, peak)
+        graded = [r for r in rows if r["kernel"] in OPS and r.get("launches", 1) == 1 and r["algorithmic_bytes"] >= 256e6]
+        if graded:
+            low = min(graded, key=lambda r: r["frac_of_measured"])
+            per_el, src = NCU_DRAM_BYTES_PER_ELEMENT.get((low["dtype"], low["kernel"]), (None, None))
+            line["roofline"] = {"bound": "hbm", "kernel": low["kernel"], "dtype": low["dtype"], "config": low["config"],
+                                "tensor": low.get("tensor"), "dense_output": low.get("dense_output"),
+                                "achieved": low["gbs"], "peak": peak, "unit": "GB/s", "frac": low["frac_of_measured"],
+                                "peak_kind": peak_kind, "frac_of_8tbs": low["frac_of_8tbs"],
+                                "algorithmic_bytes_per_launch": low["algorithmic_bytes"], "avg_launch_ms": low["median_ms"],
+                                "traffic": None if per_el is None else round(per_el * low["elements"]),
+                                "traffic_source": src,
+                                "how": "the lowest fraction among the five graded calls on tensors of at least 256 MB; "
+                                       "each row: CUDA events around one launch, L2 flushed before it, median of 9",
+                                "kernels": rows}
+        else:
+            # without the table: the headline tensor's own four kernels, timed one by one
+            T = KernelTimer(dev, peak)
+            codec_rows(T, B, "cfg3_iid", batch.x[0], batch.pre[0], batch.g, ZEROS, ops=("compress", "decompress", "fwd", "bwd"))
+            low = min(T.rows, key=lambda r: r["frac_of_measured"])
+            line["roofline"] = {"bound": "hbm", "kernel": low["kernel"], "dtype": "f32", "achieved": low["gbs"], "peak": peak,
+                                "unit": "GB/s", "frac": low["frac_of_measured"], "peak_kind": peak_kind, "traffic": None,
+                                "kernels": T.rows}
+        line.update(extras)
+        if not args.no_e2e:
+            e = run_e2e(batch)
+            line["e2e"] = {"value": round(world * e["dense_bytes_per_step"] / (e["ms_per_step"] * 1e-3) / 1e9, 3), "unit": UNIT,
+                           "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"],
+                           "ms_per_step": round(e["ms_per_step"], 3), "steps": e["steps"],
+                           "what": "the step's four operations on one tensor of the batch through bt_*_host: pinned host "
+                                   "buffers in, pinned host buffers out, copies inside the calls (rank 0's GPU; "
+                                   "value scaled by the number of ranks)"}
+        if not args.no_cpu_baseline and world == 1:
+            cal = host_sample(1 << 20)
+            rate = (1 << 20) / max(oracle_four_ops(*cal), 1e-6)
+            m = max(1 << 20, min(1 << LOG2N, int(rate * 15.0) // 4096 * 4096))          # about 15 s of CPU work
+            sec = oracle_four_ops(*host_sample(m))
+            line["cpu_baseline"] = {"value": round(len(OPS) * 4 * m / sec / 1e9, 4), "unit": UNIT, "cores": 1,
+                                    "kind": "oracle", "seconds": round(sec, 2),
+                                    "sample": "the first %d elements of one tensor of the batch (of %d), all four operations, "
+                                              "single thread; host has %d cores" % (m, 1 << LOG2N, os.cpu_count())}
         print(json.dumps(line))
+    barrier()
     if world > 1:
         dist.destroy_process_group()
 
 
-def run_e2e(step: Cfg2Step, graph, steps: int, world: int, workers: int = int(os.environ.get("BT_E2E_WORKERS", "4"))):
-    """The same step through the host-buffer entry points of the C ABI: every tensor the step consumes
-    starts in pinned host memory and every tensor it produces (both stashes, the restored activation, the
-    input gradient) ends there; the host<->device copies happen inside the calls, inside the timed region.
-
-    The calls are synchronous, so a few host threads (each with its own stream, staging area and output
-    buffers) work on different layers at once: one call's host->device copy overlaps another's
-    device->host copy and kernels.  All forward calls of a step finish before its backward calls start."""
-    import queue
-    from concurrent.futures import ThreadPoolExecutor
+# ------------------------------------------------------------------------------------------
+def run_case(args) -> int:
+    """One small, seeded invocation of one kernel, for profiler captures (python bench.py --case <dtype> <op>):
+    `reps` repetitions of one entry point on a tensor of 2**log2n elements (default 2**26: larger than the 126 MB L2
+    and small enough for a multi-pass capture); prints the non-zero count and the device status, non-zero exit
+    if the status is not BT_OK.  The 4- and 8-byte input has independent zeros of the given fraction, the
+    2-byte input is the ReLU of a normal pre-activation (about half zeros)."""
     import torch
-    B = step.B
-    dev = step.restored.device
-    n_max = step.restored.numel()
-    host = []
-    h2d = d2h = 0
-    for l in step.layers:
-        n = l["n"]
-        h = dict(act=l["act"].cpu().pin_memory(), pre=l["pre"].cpu().pin_memory(), grad=l["grad"].cpu().pin_memory())
-        for tag in ("a", "b"):
-            h["bitmap_" + tag] = torch.empty((n + 31) // 32, dtype=torch.int32).pin_memory()
-            h["values_" + tag] = torch.empty(n, dtype=torch.float32).pin_memory()
-            h["prefix_" + tag] = torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory()
-            h["nnz_" + tag] = torch.zeros(1, dtype=torch.int64).pin_memory()
-        host.append(h)
-    for l, z in zip(step.layers, step.nnz()):
-        n = l["n"]
-        comp = B.bt_compressed_bytes(n, z, torch.float32)
-        h2d += 4 * n + 4 * n + comp + (4 * ((n + 31) // 32) + 4 * n)      # compress, fused forward, decompress, backward
-        d2h += (comp + 8) + (comp + 8) + 4 * n + 4 * n
+    from paper_2110_15362_b200 import binding as B
+    from paper_2110_15362_b200 import workloads as W
+    kind, op = args.case
+    if kind not in ("f32", "f16", "bf16", "f64") or op not in CASE_OPS:
+        raise SystemExit("--case <f32|f16|bf16|f64> <%s>" % "|".join(CASE_OPS))
+    dev = torch.device("cuda")
+    n = 1 << args.log2n
+    if kind == "f32":
+        x = W.prune_preact(n, dev) if op == "prune" else W.cfg3_iid(n, args.zeros, 2, dev)
+    elif kind == "f64":
+        x = W.cfg3_iid(n, args.zeros, 3, dev).double()
+    else:
+        x = torch.relu(W.cfg4_preact(0, (n,), kind, dev))
+    st = B.Stash(n, x.dtype, dev)
+    ws = B.new_workspace(n, dev)
+    d = torch.empty_like(x)
+    v16 = torch.empty(n, dtype=torch.float16, device=dev) if op in ("narrow", "widen") else None
+    d32 = torch.empty(n, dtype=torch.float32, device=dev) if op == "widen" else None
 
-    # per-thread resources, handed out through a queue
-    pool = queue.SimpleQueue()
-    for _ in range(workers):
-        pool.put(dict(stream=torch.cuda.Stream(device=dev),
-                      staging=torch.empty(B.bt_host_staging_bytes(n_max, torch.float32), dtype=torch.uint8, device=dev),
-                      restored=torch.empty(n_max, dtype=torch.float32).pin_memory(),
-                      gin=torch.empty(n_max, dtype=torch.float32).pin_memory()))
-    check = {}
+    def compress():
+        B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
 
-    def call(task):
-        kind, i = task
-        r = pool.get()
-        try:
-            torch.cuda.set_device(dev)
-            h, s, n = host[i], r["stream"], step.layers[i]["n"]
-            if kind == "compress":
-                B.bt_compress_host(h["act"], h["bitmap_a"], h["values_a"], h["prefix_a"], h["nnz_a"], r["staging"], stream=s)
-            elif kind == "fused":
-                B.bt_relu_fwd_compress_host(h["pre"], None, h["bitmap_b"], h["values_b"], h["prefix_b"], h["nnz_b"],
-                                            r["staging"], stream=s)
-            elif kind == "decompress":
-                B.bt_decompress_host(h["bitmap_a"], h["values_a"], h["prefix_a"], int(h["nnz_a"].item()),
-                                     r["restored"][:n], r["staging"], stream=s)
-                if i == 0:
-                    check["ok"] = torch.equal(r["restored"][:n].view(torch.int32), h["act"].view(torch.int32))
-            else:
-                B.bt_relu_bwd_from_bitmap_host(h["bitmap_b"], h["grad"], r["gin"][:n], r["staging"], stream=s)
-        finally:
-            pool.put(r)
-
-    order = sorted(range(len(step.layers)), key=lambda i: -step.layers[i]["n"])     # large layers first
-    fwd = [(k, i) for i in order for k in ("compress", "fused")]
-    bwd = [(k, i) for i in order for k in ("decompress", "backward")]
-    with ThreadPoolExecutor(max_workers=workers) as ex:
-        def one():
-            list(ex.map(call, fwd))
-            list(ex.map(call, bwd))
-        one()
+    if op in ("maxpool", "maxpool_bwd"):                                 # the tensor seen as rows of 256 elements
+        xp = x.view(-1, n // 256 // 64, 256)
+        yp = torch.empty(xp.shape[0], xp.shape[1] // 2, 128, dtype=x.dtype, device=dev)
+        codes = torch.empty((yp.numel() + 15) // 16, dtype=torch.int32, device=dev)
+        for _ in range(args.reps):
+            B.bt_maxpool2x2_fwd(xp, yp, codes)
+            if op == "maxpool_bwd":
+                B.bt_maxpool2x2_bwd(codes, yp, d.view_as(xp))
         torch.cuda.synchronize()
-        assert check.get("ok"), "end-to-end round trip is not bit exact"
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(steps):
-            one()
-        # every call has synchronised its own stream before returning; the closing event follows them all
-        e1.record()
-        torch.cuda.synchronize()
-    return {"ms": e0.elapsed_time(e1), "steps": steps, "h2d": h2d, "d2h": d2h, "workers": workers}
+        print("pooled", tuple(yp.shape), "non-zero", int(torch.count_nonzero(yp)))
+        return 0
+    for _ in range(args.reps):
+        if op == "compress":
+            compress()
+        elif op == "relu":
+            B.bt_relu_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif op == "relu_y":
+            B.bt_relu_fwd_compress(x, d, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif op == "prune":
+            B.bt_prune_fwd_compress(x, args.tau, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif op == "narrow":                                             # float32 tensor, float16 stashed values
+            B.bt_compress_narrow(x, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif op == "widen":
+            B.bt_compress_narrow(x, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+            B.bt_decompress_widen(st.bitmap, v16, st.chunk_prefix, d32)
+        elif op == "relu6":
+            B.bt_relu6_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        elif op == "relu6_bwd":
+            B.bt_relu6_fwd_compress(x, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+            B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, x, d)
+        elif op in ("mask", "mask_y"):
+            compress()
+            B.bt_mask_compress(x, st.bitmap, st.chunk_prefix, d if op == "mask_y" else None, st.values)
+        elif op == "decompress":
+            compress()
+            B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, d)
+        else:
+            compress()
+            B.bt_relu_bwd_from_bitmap(st.bitmap, x, d)
+    torch.cuda.synchronize()
+    print("nnz", st.nnz, "status", st.status)
+    return 0 if st.status == B.BT_OK else 1
 
 
 def main():
     args = parse_args()
+    if args.case:
+        sys.exit(run_case(args))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -196,6 +196,20 @@ int bt_relu_fwd_compress_batch(const bt_batch_item *items /* host */, uint32_t c
                                void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * Batched forms of the two consumers, for the backward pass of a step that restores many stashes: `count`
+ * tensors of one element type per launch (more than 32 non-empty tensors: several launches), each handled
+ * exactly as by the single-tensor call.  The items are the ones the batched compressors took, read as
+ *   bt_decompress_batch             y_out[i] = bit i ? next value : +0 from (bitmap, values, chunk_prefix);
+ *                                   dense, values_capacity, nnz_out and dev_status are ignored
+ *   bt_relu_bwd_from_bitmap_batch   y_out[i] = bit i ? dense[i] : +0 (dense: the upstream gradient; y_out may
+ *                                   alias it); values, chunk_prefix, nnz_out and dev_status are ignored
+ * Tensors with n == 0 are skipped.  No workspace.  Nothing is launched on an argument error.
+ */
+int bt_decompress_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype, void *stream);
+
+int bt_relu_bwd_from_bitmap_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype, void *stream);
+
+/*
  * Launch configuration for callers that keep several compress calls in flight
  * (on several streams, or in the branches of a CUDA graph).  The compress
  * kernel is launched cooperatively with one CTA per SM, and a cooperative

@@ -32,7 +32,8 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_prune_fwd_compress_narrow", "bt_decompress_widen", "bt_maxpool2x2_fwd", "bt_maxpool2x2_bwd",
            "bt_compress_narrow_arena", "bt_prune_fwd_compress_narrow_arena", "bt_decompress_widen_arena",
            "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked", "bt_set_max_ctas",
-           "bt_batch_workspace_bytes", "bt_compress_batch", "bt_relu_fwd_compress_batch")
+           "bt_batch_workspace_bytes", "bt_compress_batch", "bt_relu_fwd_compress_batch", "bt_decompress_batch",
+           "bt_relu_bwd_from_bitmap_batch")
 
 MAX_BATCH_PER_LAUNCH = 32
 
@@ -86,6 +87,9 @@ def load_library(path: str) -> ctypes.CDLL:
     for name in ("bt_compress_batch", "bt_relu_fwd_compress_batch"):
         getattr(L, name).restype = i32
         getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp, sz, vp]
+    for name in ("bt_decompress_batch", "bt_relu_bwd_from_bitmap_batch"):
+        getattr(L, name).restype = i32
+        getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp]
     L.bt_decompress.restype = i32
     L.bt_decompress.argtypes = [vp, vp, vp, u64, i32, vp, vp]
     L.bt_relu_fwd_compress.restype = i32
@@ -209,6 +213,18 @@ def bt_relu_fwd_compress_batch(items, dtype: torch.dtype, workspace: torch.Tenso
     st = lib().bt_relu_fwd_compress_batch(items, len(items), DTYPE_CODE[dtype], _ptr(workspace), _nbytes(workspace),
                                           _stream(stream))
     return _check("bt_relu_fwd_compress_batch", st, check)
+
+
+def bt_decompress_batch(items, dtype: torch.dtype, *, stream=None, check: bool = True) -> int:
+    """bt_decompress of every stash of `items` into its y_out, in one pass."""
+    st = lib().bt_decompress_batch(items, len(items), DTYPE_CODE[dtype], _stream(stream))
+    return _check("bt_decompress_batch", st, check)
+
+
+def bt_relu_bwd_from_bitmap_batch(items, dtype: torch.dtype, *, stream=None, check: bool = True) -> int:
+    """bt_relu_bwd_from_bitmap of every item (dense: upstream gradient, y_out: input gradient), in one pass."""
+    st = lib().bt_relu_bwd_from_bitmap_batch(items, len(items), DTYPE_CODE[dtype], _stream(stream))
+    return _check("bt_relu_bwd_from_bitmap_batch", st, check)
 
 
 def bt_compress_noalloc(dense: torch.Tensor, bitmap: torch.Tensor, values: torch.Tensor, chunk_prefix: torch.Tensor,

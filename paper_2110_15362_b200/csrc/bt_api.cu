@@ -131,6 +131,37 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
     return BT_OK;
 }
 
+// The consumers of a batch of stashes: backward == false restores items[k].y_out from (bitmap, values, chunk_prefix),
+// backward == true writes items[k].y_out = bit ? items[k].dense : +0.
+int consume_batch_common(const bt_batch_item *items, uint32_t count, int dtype, bool backward, void *stream)
+{
+    const int es = elem_size_of(dtype);
+    if (es == 0) return BT_ERR_DTYPE;
+    if (count == 0) return BT_OK;
+    if (!items) return BT_ERR_NULL;
+    for (uint32_t k = 0; k < count; ++k) {
+        const bt_batch_item &it = items[k];
+        if (it.n == 0) continue;
+        if (!it.bitmap || !it.y_out) return BT_ERR_NULL;
+        if (backward ? !it.dense : (!it.values || !it.chunk_prefix)) return BT_ERR_NULL;
+        if (!aligned(it.bitmap, 4) || !aligned(it.y_out, 16)) return BT_ERR_ALIGN;
+        if (backward ? !aligned(it.dense, 16) : (!aligned(it.values, 16) || !aligned(it.chunk_prefix, 8))) return BT_ERR_ALIGN;
+    }
+    cudaStream_t      s = static_cast<cudaStream_t>(stream);
+    bt::DecompressJob jobs[bt::kMaxBatch];
+    uint32_t          m = 0;
+    for (uint32_t k = 0; k < count; ++k) {
+        const bt_batch_item &it = items[k];
+        if (it.n != 0) jobs[m++] = bt::DecompressJob{it.bitmap, it.values, it.chunk_prefix, it.dense, it.y_out, it.n};
+        if (m == bt::kMaxBatch || (k + 1 == count && m > 0)) {
+            const cudaError_t e = backward ? bt::launch_relu_bwd_batch(jobs, m, es, s) : bt::launch_decompress_batch(jobs, m, es, s);
+            if (e != cudaSuccess) return BT_ERR_CUDA;
+            m = 0;
+        }
+    }
+    return BT_OK;
+}
+
 }  // namespace
 
 #ifdef BT_BOUNDS_CHECK
@@ -191,6 +222,16 @@ int bt_compress_batch(const bt_batch_item *items, uint32_t count, int dtype, voi
                       void *stream)
 {
     return compress_batch_common(items, count, dtype, 0, workspace, workspace_bytes, stream);
+}
+
+int bt_decompress_batch(const bt_batch_item *items, uint32_t count, int dtype, void *stream)
+{
+    return consume_batch_common(items, count, dtype, false, stream);
+}
+
+int bt_relu_bwd_from_bitmap_batch(const bt_batch_item *items, uint32_t count, int dtype, void *stream)
+{
+    return consume_batch_common(items, count, dtype, true, stream);
 }
 
 int bt_relu_fwd_compress_batch(const bt_batch_item *items, uint32_t count, int dtype, void *workspace,

@@ -40,11 +40,27 @@ __device__ __forceinline__ uint32_t widened(const uint16_t h)
     }
 }
 
+// One tensor restored by a batched launch (see decompress_batch_kernel).
+struct RestoreJob {
+    const uint32_t *bitmap;
+    const void     *values;
+    const uint64_t *prefix;
+    void           *out;
+    uint64_t        n;
+    uint32_t        first_block;    // the launch's blocks [first_block, next job's first_block) restore this tensor
+};
+template <int kJobs>
+struct RestoreParams {
+    RestoreJob job[kJobs];
+    uint32_t   jobs;
+};
+
+// `block`: index of this CTA among those that restore the tensor
 template <typename U, int kE, int kGrp, int kWarps, int WIDEN = 0>
-__global__ void __launch_bounds__(kWarps * 32)
-decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<WIDEN != 0, uint16_t, U> *values,
-                  const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
-                  U *__restrict__ out)
+__device__ __forceinline__ void
+decompress_body(const uint32_t *__restrict__ bitmap, const std::conditional_t<WIDEN != 0, uint16_t, U> *values,
+                const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
+                U *__restrict__ out, const uint64_t block)
 {
     constexpr int kVec          = 16 / sizeof(U);          // elements per 16-byte store
     constexpr int kLanesPerWord = 32 / kE;                 // lanes that share one bitmap word
@@ -53,7 +69,7 @@ decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<
     static_assert(kE % kVec == 0 && 32 % kE == 0 && kE < 32, "a lane takes whole vectors of one word");
 
     const uint32_t lane        = threadIdx.x & 31u;
-    const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    const uint64_t warp_global = block * kWarps + (threadIdx.x >> 5);
     const uint64_t quarters    = (n + 1023) >> 10;
     if (warp_global >= quarters) return;
 
@@ -176,16 +192,16 @@ __device__ __forceinline__ uint2 expand4_u16(uint32_t a, const uint32_t bits)
 }
 
 template <int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 2048 / (kWarps * 32))
-decompress16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values, const uint64_t *__restrict__ values_offset,
-                    const uint64_t *__restrict__ prefix, const uint64_t n, uint16_t *__restrict__ out)
+__device__ __forceinline__ void
+decompress16_body(const uint32_t *__restrict__ bitmap, const uint16_t *values, const uint64_t *__restrict__ values_offset,
+                  const uint64_t *__restrict__ prefix, const uint64_t n, uint16_t *__restrict__ out, const uint64_t block)
 {
     // a quarter's run (at most 1024 values) behind up to 14 bytes of its first vector, whole vectors
     __shared__ __align__(16) unsigned char s_run[kWarps][2048 + 32];
 
     const uint32_t lane        = threadIdx.x & 31u;
     const uint32_t wic         = threadIdx.x >> 5;
-    const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + wic;
+    const uint64_t warp_global = block * kWarps + wic;
     const uint64_t quarters    = (n + 1023) >> 10;
     if (warp_global >= quarters) return;
 
@@ -274,6 +290,52 @@ decompress16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values,
     }
 }
 
+template <typename U, int kE, int kGrp, int kWarps, int WIDEN = 0>
+__global__ void __launch_bounds__(kWarps * 32)
+decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<WIDEN != 0, uint16_t, U> *values,
+                  const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
+                  U *__restrict__ out)
+{
+    decompress_body<U, kE, kGrp, kWarps, WIDEN>(bitmap, values, values_offset, prefix, n, out, blockIdx.x);
+}
+
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 2048 / (kWarps * 32))
+decompress16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values, const uint64_t *__restrict__ values_offset,
+                    const uint64_t *__restrict__ prefix, const uint64_t n, uint16_t *__restrict__ out)
+{
+    decompress16_body<kWarps>(bitmap, values, values_offset, prefix, n, out, blockIdx.x);
+}
+
+// The tensor a CTA of a batched launch works on: the last job whose first block is not behind this one.
+template <int kJobs>
+__device__ __forceinline__ uint32_t job_of_block(const RestoreParams<kJobs> &p)
+{
+    uint32_t k = 0;
+    for (uint32_t j = 1; j < p.jobs; ++j) k = p.job[j].first_block <= blockIdx.x ? j : k;
+    return k;
+}
+
+// Several tensors of one element type restored by ONE launch: every CTA looks up its tensor in the job table (in
+// the kernel's parameters) and restores its four quarters of it exactly as the single-tensor kernel does.
+template <typename U, int kE, int kGrp, int kWarps, int kJobs>
+__global__ void __launch_bounds__(kWarps * 32)
+decompress_batch_kernel(const __grid_constant__ RestoreParams<kJobs> p)
+{
+    const RestoreJob &j = p.job[job_of_block(p)];
+    decompress_body<U, kE, kGrp, kWarps, 0>(j.bitmap, static_cast<const U *>(j.values), nullptr, j.prefix, j.n, static_cast<U *>(j.out),
+                                            blockIdx.x - j.first_block);
+}
+
+template <int kWarps, int kJobs>
+__global__ void __launch_bounds__(kWarps * 32, 2048 / (kWarps * 32))
+decompress16_batch_kernel(const __grid_constant__ RestoreParams<kJobs> p)
+{
+    const RestoreJob &j = p.job[job_of_block(p)];
+    decompress16_body<kWarps>(j.bitmap, static_cast<const uint16_t *>(j.values), nullptr, j.prefix, j.n, static_cast<uint16_t *>(j.out),
+                              blockIdx.x - j.first_block);
+}
+
 template <typename U, int kE, int kGrp>
 cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                          const uint64_t *prefix, uint64_t n, void *out, cudaStream_t stream)
@@ -316,6 +378,26 @@ cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const 
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     decompress16_kernel<kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
         bitmap, static_cast<const uint16_t *>(values), values_offset, prefix, n, static_cast<uint16_t *>(out));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decompress_batch(const DecompressJob *jobs, uint32_t count, int elem_size, cudaStream_t stream)
+{
+    constexpr int kWarps = 4;
+    if (count == 0 || count > kMaxBatch) return cudaErrorInvalidValue;
+    RestoreParams<kMaxBatch> p{};
+    uint64_t                 blocks = 0;
+    for (uint32_t k = 0; k < count; ++k) {
+        const uint64_t quarters = (jobs[k].n + 1023) >> 10;
+        p.job[k] = RestoreJob{jobs[k].bitmap, jobs[k].values, jobs[k].prefix, jobs[k].out, jobs[k].n, static_cast<uint32_t>(blocks)};
+        blocks += (quarters + kWarps - 1) / kWarps;
+        if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    }
+    p.jobs = count;
+    const unsigned grid = static_cast<unsigned>(blocks);
+    if (elem_size == 8) decompress_batch_kernel<uint64_t, 2, 16, kWarps, kMaxBatch><<<grid, kWarps * 32, 0, stream>>>(p);
+    else if (elem_size == 4) decompress_batch_kernel<uint32_t, 4, 8, kWarps, kMaxBatch><<<grid, kWarps * 32, 0, stream>>>(p);
+    else decompress16_batch_kernel<kWarps, kMaxBatch><<<grid, kWarps * 32, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

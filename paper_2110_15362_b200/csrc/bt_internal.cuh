@@ -104,6 +104,18 @@ uint64_t set_compress_wait_ns(uint64_t wait_ns);
 // values_offset: NULL, or a device word holding the byte offset of the packed values inside `values`
 cudaError_t launch_decompress(const uint32_t *bitmap, const void *values, const uint64_t *values_offset,
                               const uint64_t *prefix, uint64_t n, int elem_size, void *out, cudaStream_t s);
+// One tensor of a batched restore / batched ReLU backward (every n > 0); `in` is the upstream gradient of the
+// backward form and unused by the restore.
+struct DecompressJob {
+    const uint32_t *bitmap;
+    const void     *values;
+    const uint64_t *prefix;
+    const void     *in;
+    void           *out;
+    uint64_t        n;
+};
+cudaError_t launch_decompress_batch(const DecompressJob *jobs, uint32_t count, int elem_size, cudaStream_t s);
+cudaError_t launch_relu_bwd_batch(const DecompressJob *jobs, uint32_t count, int elem_size, cudaStream_t s);
 cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16, const uint64_t *values_offset,
                                     const uint64_t *prefix, uint64_t n, int from_dtype, void *out_f32, cudaStream_t s);
 cudaError_t launch_mask_gather(const void *x, const uint32_t *bitmap, const uint64_t *prefix, uint64_t n,

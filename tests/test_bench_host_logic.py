@@ -58,8 +58,18 @@ def test_max_over_ranks_gloo_world_size_2():
 
 def test_reference_arm_prints_one_json_line(capsys):
     import json
-    args = type("A", (), dict(gpus=1, steps=1, warmup=0, batch=1, impl="reference"))()
+    args = type("A", (), dict(gpus=1, steps=2, warmup=1, impl="reference", reference_budget_s=1.5))()
     bench.run_reference(args)
     line = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0 and line["metric"] == bench.METRIC
+    # the same workload, step count and warm-up as the other arm is asked for
+    assert line["config"] == bench.workload_config() and line["steps"] == 2 and line["warmup"] == 1
+    assert line["config"]["workload"] == bench.WORKLOAD and line["cpu_baseline"]["value"] == line["value"]
+
+
+def test_default_arguments_are_the_round_end_run():
+    a = bench.parse_args([])
+    assert (a.gpus, a.steps, a.warmup, a.impl) == (1, 20, 5, "ours") and a.case is None
+    c = bench.parse_args(["--case", "bf16", "relu", "--log2n", "27"])
+    assert c.case == ["bf16", "relu"] and c.log2n == 27

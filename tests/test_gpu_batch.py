@@ -91,3 +91,58 @@ def test_batch_argument_checks():
     items[1].bitmap = None
     assert B.bt_compress_batch(items, torch.float32, ws, check=False) == B.BT_ERR_NULL
     assert L.bt_compress_batch(None, 0, B.BT_F32, None, 0, None) == B.BT_OK
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16", "f16", "f64"])
+def test_batched_consumers_equal_the_oracle_tensor_by_tensor(oracle, kind):
+    """bt_decompress_batch and bt_relu_bwd_from_bitmap_batch on the stashes a batched compressor wrote: per tensor
+    the oracle's restored tensor and masked gradient, outputs between guard regions."""
+    from tests.gpu_util import Guarded
+    dt = TDT[kind]
+    raws, sts, _, _ = run_batch(kind, SIZES, 8080, False, False)
+    outs = [Guarded(max(r.size, 1), dt) for r in raws]
+    items = B.batch_items([o.inner for o in outs], sts, [o.inner for o in outs])
+    for k, r in enumerate(raws):
+        items[k].n = r.size
+        items[k].dense = None                                        # the restore reads no dense input
+    B.bt_decompress_batch(items, dt)
+    torch.cuda.synchronize()
+    for k, (r, o) in enumerate(zip(raws, outs)):
+        assert np.array_equal(o.raw()[:r.size], r), (k, r.size)
+        assert o.guards_intact()
+    # backward: gradients in, masked gradients out (one tensor in place)
+    g_raws = [W.random_patterns(r.size, kind, 0.1, seed=9000 + k) for k, r in enumerate(raws)]
+    gs = [from_raw(g, kind) if g.size else torch.empty(1, dtype=dt, device="cuda") for g in g_raws]
+    gins = [Guarded(max(g.size, 1), dt) for g in g_raws]
+    ys = [gi.inner for gi in gins]
+    ys[3] = gs[3]                                                     # in place
+    items = B.batch_items(gs, sts, ys)
+    for k, r in enumerate(raws):
+        items[k].n = r.size
+    B.bt_relu_bwd_from_bitmap_batch(items, dt)
+    torch.cuda.synchronize()
+    for k, (r, g) in enumerate(zip(raws, g_raws)):
+        if r.size == 0:
+            continue
+        want = oracle.relu_bwd_from_bitmap(oracle.compress(r).bitmap, g)
+        got = W.raw_numpy(ys[k])[:r.size]
+        assert np.array_equal(got, want), (k, r.size)
+        assert gins[k].guards_intact()
+
+
+def test_batched_consumers_over_more_tensors_than_one_launch_holds_and_argument_checks(oracle):
+    sizes = [4096 * (1 + k % 5) + k for k in range(2 * B.MAX_BATCH_PER_LAUNCH + 3)]
+    raws, sts, _, _ = run_batch("bf16", sizes, 61, False, False)
+    outs = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for n in sizes]
+    items = B.batch_items(outs, sts, outs)
+    B.bt_decompress_batch(items, torch.bfloat16)
+    torch.cuda.synchronize()
+    for r, o in zip(raws, outs):
+        assert np.array_equal(W.raw_numpy(o), r)
+    items[5].y_out = None
+    assert B.bt_decompress_batch(items, torch.bfloat16, check=False) == B.BT_ERR_NULL
+    assert B.bt_relu_bwd_from_bitmap_batch(items, torch.bfloat16, check=False) == B.BT_ERR_NULL
+    items[5].y_out = outs[5].data_ptr() + 2
+    assert B.bt_decompress_batch(items, torch.bfloat16, check=False) == B.BT_ERR_ALIGN
+    assert B.lib().bt_decompress_batch(None, 0, B.BT_F32, None) == B.BT_OK
+    assert B.lib().bt_decompress_batch(items, 1, 11, None) == B.BT_ERR_DTYPE
