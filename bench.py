@@ -47,18 +47,23 @@ NOMINAL_GBS = 8000.0
 CASE_OPS = ("compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd", "decompress", "relu_bwd", "mask",
             "mask_y", "maxpool", "maxpool_bwd", "widen")
 
-# DRAM bytes (read + write) per element of the kernel `roofline` names, from one ncu capture of
-#   python bench.py --case <dtype> <op> --log2n 27
-# (dram__bytes_read.sum + dram__bytes_write.sum of the captured launch / 2^27; traffic grows in proportion to the
-# element count, so a full launch is this figure times its elements).  The capture and its command are summarised
-# in the file named beside each figure.
+# DRAM bytes (read + write) per element of a kernel, from one ncu capture of
+#   python bench.py --case <dtype> <op> --log2n <26 for 4-byte, 27 for 2-byte elements>
+# (dram__bytes_read.sum + dram__bytes_write.sum of the captured launch / its elements, at half zeros).  Traffic
+# grows in proportion to the element count, so a full launch is this figure times its elements; the figure sits a
+# little below the algorithmic bytes because the tail of what a launch writes is still in the L2 when it ends.
+# The capture and its command are summarised in the file named beside each figure.
 NCU_DRAM_BYTES_PER_ELEMENT = {
-    ("bf16", "bt_relu_fwd_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
-    ("f16", "bt_relu_fwd_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
-    ("bf16", "bt_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
-    ("f16", "bt_compress"): (3.13, "profiles/bt_compress_bf16_2p27_ncu.md"),
-    ("bf16", "bt_decompress"): (3.13, "profiles/bt_decompress_bf16_2p27_ncu.md"),
-    ("f16", "bt_decompress"): (3.13, "profiles/bt_decompress_bf16_2p27_ncu.md"),
+    ("bf16", "bt_relu_fwd_compress"): (2.835, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
+    ("f16", "bt_relu_fwd_compress"): (2.835, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("bf16", "bt_compress"): (2.831, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
+    ("f16", "bt_compress"): (2.831, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("bf16", "bt_decompress"): (2.779, "profiles/bt_decompress_bf16_2p27_ncu_full.md"),
+    ("f16", "bt_decompress"): (2.779, "profiles/bt_decompress_bf16_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("f32", "bt_compress"): (5.562, "profiles/bt_codec_f32_2p26_ncu_full.md"),
+    ("f32", "bt_relu_fwd_compress"): (5.562, "profiles/bt_codec_f32_2p26_ncu_full.md (plain compressor; same kernel body)"),
+    ("f32", "bt_decompress"): (5.308, "profiles/bt_codec_f32_2p26_ncu_full.md"),
+    ("f32", "bt_relu_bwd_from_bitmap"): (7.382, "profiles/bt_codec_f32_2p26_ncu_full.md"),
 }
 
 
