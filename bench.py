@@ -5,8 +5,8 @@ Headline workload: the sparsity-sweep tensor of 2^28 fp32 elements (1 GiB) at ha
 one pass of the whole hot path over one batch of such tensors (24 of them, seeded differently, all
 resident in HBM): per tensor bt_compress of the activation, bt_decompress of that stash,
 bt_relu_fwd_compress of the pre-activation (stash only) and bt_relu_bwd_from_bitmap of an upstream
-gradient -- four launches per tensor on one stream, about 26 ms per step, so that the 20 steps the
-round-end run times last half a second and the clock samples fall inside the timed region.  The metric
+gradient -- four launches per tensor on one stream, about 27 ms per step, so that the default 20 steps
+last half a second and the clock samples fall inside the timed region.  The metric
 is dense-equivalent GB/s: N * sizeof(dtype) per call, summed over the step, divided by the step time.
 
 The same JSON line carries, under roofline.kernels, every kernel of the five workload configurations

@@ -68,7 +68,7 @@ def test_reference_arm_prints_one_json_line(capsys):
     assert line["config"]["workload"] == bench.WORKLOAD and line["cpu_baseline"]["value"] == line["value"]
 
 
-def test_default_arguments_are_the_round_end_run():
+def test_default_arguments():
     a = bench.parse_args([])
     assert (a.gpus, a.steps, a.warmup, a.impl) == (1, 20, 5, "ours") and a.case is None
     c = bench.parse_args(["--case", "bf16", "relu", "--log2n", "27"])
