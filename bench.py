@@ -472,13 +472,13 @@ def host_sample(m: int):
 
 def run_reference(args):
     """The oracle, as it stands, on host cores.  Every step is the step's four operations on a bounded sample of
-    one tensor of the workload, sized from a short calibration so that warm-up plus timed steps take about 100 s."""
+    one tensor of the workload, sized from a short calibration so that warm-up plus timed steps take a minute or two."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     cal = host_sample(1 << 20)
     rate = (1 << 20) / max(oracle_four_ops(*cal), 1e-6)                  # elements per second through all four
-    budget_s = float(getattr(args, "reference_budget_s", 100.0))
+    budget_s = float(getattr(args, "reference_budget_s", 60.0))
     m = int(rate * budget_s / max(args.steps + args.warmup, 1))
     m = max(1 << 16, min(1 << LOG2N, m // 4096 * 4096))
     x, pre, g = host_sample(m)

@@ -541,6 +541,13 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStr
                      : launch_typed<uint16_t, k6 + BT_BF16, false>(a, stream);
         }
     }
+    if (y && a.tau == 0.0f && (dtype == BT_F16 || dtype == BT_BF16)) {
+        // The ReLU itself on a 2-byte type, with the dense output: decided on the bit pattern (0.182 -> 0.178 ms on
+        // the 392 MiB tensor).  Without the dense output the same test measured slower than the float compare
+        // (0.169 against 0.162 ms), so that form keeps the compare.
+        constexpr int kb = kFusedReluBits;
+        return dtype == BT_F16 ? launch_typed<uint16_t, kb + BT_F16, true>(a, stream) : launch_typed<uint16_t, kb + BT_BF16, true>(a, stream);
+    }
     switch (dtype) {
     case BT_F64:
         return y ? launch_typed<uint64_t, BT_F64, true>(a, stream) : launch_typed<uint64_t, BT_F64, false>(a, stream);

@@ -589,6 +589,12 @@ cudaError_t launch_compress_batch(const CompressJob *jobs, uint32_t count, float
                : dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(c, jobs, count, workspace, stream)
                                  : launch_typed<uint16_t, -1, false>(c, jobs, count, workspace, stream);
     }
+    if (y && tau == 0.0f && (dtype == BT_F16 || dtype == BT_BF16)) {
+        // the ReLU itself on a 2-byte type, with the dense output: decided on the bit pattern (as in the single-tensor kernel)
+        constexpr int kb = kFusedReluBits;
+        return dtype == BT_F16 ? launch_typed<uint16_t, kb + BT_F16, true>(c, jobs, count, workspace, stream)
+                               : launch_typed<uint16_t, kb + BT_BF16, true>(c, jobs, count, workspace, stream);
+    }
     switch (dtype) {
     case BT_F64:
         return y ? launch_typed<uint64_t, BT_F64, true>(c, jobs, count, workspace, stream)

@@ -169,16 +169,26 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
             Reg<U> x = v[j];
-            if constexpr (RELU_DT >= 0) {
-                x = fused_forward<RELU_DT>(x, tau);
+            bool   nz;
+            if constexpr (RELU_DT >= kFusedReluBits) {
+                nz = relu_keeps_bits<RELU_DT & 3>(x);        // a kept element is never the zero pattern
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
-                    if ((!kGuardY || e < yvalid) && yx.holds(y + e, sizeof(U))) y[e] = static_cast<U>(x);
+                    if ((!kGuardY || e < yvalid) && yx.holds(y + e, sizeof(U))) y[e] = nz ? static_cast<U>(x) : U(0);
                 }
+            } else {
+                if constexpr (RELU_DT >= 0) {
+                    x = fused_forward<RELU_DT>(x, tau);
+                    if constexpr (WRITE_Y) {
+                        const uint32_t e = (kb + j) * 32 + lane;
+                        if ((!kGuardY || e < yvalid) && yx.holds(y + e, sizeof(U))) y[e] = static_cast<U>(x);
+                    }
+                }
+                nz = x != Reg<U>(0);
             }
-            const uint32_t b = __ballot_sync(kFull, x != Reg<U>(0));
+            const uint32_t b = __ballot_sync(kFull, nz);
             bb[j] = b;
-            if (x != Reg<U>(0)) {
+            if (nz) {
                 const uint32_t at = out + kES * __popc(b & lt);
                 if constexpr (kES == 8) asm volatile("st.shared.u64 [%0], %1;" ::"r"(at), "l"(x));
                 else if constexpr (kES == 4) asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"(x));

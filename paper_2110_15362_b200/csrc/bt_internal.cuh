@@ -349,8 +349,22 @@ __device__ __forceinline__ uint32_t greater_or_nan(double v, double b)
 }
 
 // The fused forward forms are numbered by one template argument: -1 none (plain compressor), DT (0..3) keep
-// what exceeds the threshold (tau = 0: ReLU), 4 + DT ReLU6.
-constexpr int kFusedRelu6 = 4;
+// what exceeds the threshold (tau = 0: ReLU), 4 + DT ReLU6, 8 + DT (2-byte types only) the ReLU decided on the
+// bit pattern.
+constexpr int kFusedRelu6    = 4;
+constexpr int kFusedReluBits = 8;
+
+// ReLU of a 2-byte element without widening it: x, the element's pattern sign-extended to 32 bits, is kept iff
+// it is a positive number, +inf or a NaN of either sign -- exactly the elements for which x <= 0 is false under
+// IEEE comparison.  Positive patterns are the positive signed integers; a negative NaN lies above -inf's pattern.
+// Two integer compares instead of a conversion, a float compare, a select and the zero test.
+template <int DT>
+__device__ __forceinline__ bool relu_keeps_bits(const uint32_t x)
+{
+    static_assert(DT == BT_F16 || DT == BT_BF16, "2-byte element types");
+    constexpr uint32_t kMinusInf = DT == BT_F16 ? 0xFFFFFC00u : 0xFFFFFF80u;
+    return (static_cast<int32_t>(x) > 0) | (x > kMinusInf);      // no short circuit: two compares, no branch
+}
 
 // y = (x <= tau) ? +0 : x, and for ReLU6 additionally 6 where x >= 6; IEEE comparisons, so a NaN is kept.
 template <int FUSED, typename R>

@@ -363,53 +363,27 @@ def test_more_than_two_to_the_32_elements(oracle):
     torch.cuda.empty_cache()
 
 
-def test_cfg2_step_in_the_launch_configuration_the_benchmark_times(oracle):
-    """The benchmark's own step object, captured as it is timed (one CUDA graph, eight chains on eight streams, 24
-    / 74 CTAs per compress launch) and replayed: both stashes of every layer against the oracle (the largest
-    layer against torch routines and on sampled chunks), the restored activations and the ReLU gradients."""
+def test_the_benchmarks_own_step_against_the_oracle(oracle):
+    """The benchmark's batch object in the configuration it is timed in (one stream, four launches per tensor, no
+    graph, no CTA limit): after two steps over a batch of two tensors, the batch's own check, and both stashes of
+    the last tensor, the restored tensor and the masked gradient whole against the oracle."""
     import bench
-    step = bench.Cfg2Step(DEV, 32)
-    step.cta_budget = (24, 74)
-    side = torch.cuda.Stream()
-    with torch.cuda.stream(side):
-        step.run()
-    torch.cuda.synchronize()
-    for l in step.layers:                                    # forget what the warm-up wrote
-        for st in (l["stash_a"], l["stash_b"]):
-            st.bitmap.zero_(), st.values.zero_(), st.chunk_prefix.zero_(), st.nnz_out.zero_()
-    graph = torch.cuda.CUDAGraph()
-    branches = [torch.cuda.Stream() for _ in range(7)]
-    with torch.cuda.graph(graph):
-        main = torch.cuda.current_stream()
-        for b in branches:
-            b.wait_stream(main)
-        step.run(streams=[main] + branches)
-        for b in branches:
-            main.wait_stream(b)
-    assert B.bt_set_max_ctas(0) == 0                         # the step leaves no limit behind
-    for _ in range(3):
-        graph.replay()
-    torch.cuda.synchronize()
-    step.check()
-    for i, l in enumerate(step.layers):
-        x, n = l["act"], l["n"]
-        for st in (l["stash_a"], l["stash_b"]):
-            if n <= 8_000_000:
-                ref = oracle.compress(W.raw_numpy(x))
-                assert st.nnz == ref.nnz and st.status == B.BT_OK
-                assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), ref.bitmap)
-                assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), ref.prefix)
-                assert np.array_equal(W.raw_numpy(st.values[:ref.nnz]), ref.values)
-            else:
-                check_against_torch(st, x)
-                check_sampled_chunks(oracle, st, x, decompress(st, x), seed=i)
-    # the last layer each chain restored / differentiated is still in that chain's output buffer
-    for c in range(8):
-        fam, r = divmod(c, 4)
-        i = min(j for j in range(len(step.layers)) if j % 4 == r)         # backward runs in reverse: lowest index last
-        l = step.layers[i]
-        out = step.outs[c][:l["n"]]
-        if fam == 0:
-            assert torch.equal(bits_of(out), bits_of(l["act"]))
-        else:
-            assert torch.equal(bits_of(out), bits_of(torch.where(l["act"] != 0, l["grad"], torch.zeros_like(l["grad"]))))
+    batch = bench.Batch(torch.device(DEV), 2)
+    assert batch.count == 2 and batch.n == 1 << 28
+    batch.step()
+    batch.step()
+    nnz = batch.check()
+    x, pre = batch.x[-1], batch.pre[-1]
+    c = oracle.compress(W.raw_numpy(x))
+    y_ref, cr = oracle.relu_fwd_compress(W.raw_numpy(pre), "f32")
+    assert np.array_equal(y_ref, W.raw_numpy(x))                        # the pre-activation's ReLU is the activation
+    for st, ref in ((batch.sa, c), (batch.sb, cr)):
+        assert st.status == B.BT_OK and st.nnz == ref.nnz == nnz
+        assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), ref.bitmap)
+        assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), ref.prefix)
+        assert np.array_equal(W.raw_numpy(st.values[:ref.nnz]), ref.values)
+    # the step's last launch left the masked gradient in the output buffer; the restore is repeated here
+    assert np.array_equal(W.raw_numpy(batch.out), oracle.relu_bwd_from_bitmap(cr.bitmap, W.raw_numpy(batch.g)))
+    B.bt_decompress(batch.sa.bitmap, batch.sa.values, batch.sa.chunk_prefix, batch.out)
+    assert np.array_equal(W.raw_numpy(batch.out), oracle.decompress(c))
+    assert B.bt_set_max_ctas(0) == 0                                    # the benchmark sets no CTA limit
