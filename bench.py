@@ -402,48 +402,67 @@ def kernel_table(dev, peak_gbs: float):
     arena_bytes = sum((4 * z + 15) // 16 * 16 for z in nnz_true)
     arena = torch.empty(arena_bytes, dtype=torch.uint8, device=dev)
     cursor = torch.zeros(1, dtype=torch.int64, device=dev)
-    meta = [dict(bitmap=torch.empty((n + 31) // 32, dtype=torch.int32, device=dev),
-                 prefix=torch.empty((n + 4095) // 4096, dtype=torch.int64, device=dev),
-                 nnz=torch.empty(1, dtype=torch.int64, device=dev), off=torch.empty(1, dtype=torch.int64, device=dev),
-                 status=torch.empty(1, dtype=torch.int32, device=dev)) for n in ns]
-    ws = B.new_workspace(max(ns), dev)
-    back = torch.empty(max(ns), dtype=torch.float32, device=dev)
+    stashes = [B.Stash(n, torch.float32, dev, values_capacity=1) for n in ns]     # bitmap, prefix, nnz, status; values in the arena
+    offsets = torch.zeros(len(ns), dtype=torch.int64, device=dev)
+    backs = [torch.empty(n, dtype=torch.float32, device=dev) for n in ns]
+    ws = torch.empty(B.bt_batch_workspace_bytes(ns), dtype=torch.uint8, device=dev)
+    items_f = B.batch_items(layers, stashes)
+    items_r = B.batch_items(backs[::-1], stashes[::-1], backs[::-1])
+    offsets_r = torch.empty_like(offsets)
 
     def forward():
         cursor.zero_()
-        for l, m in zip(layers, meta):
-            B.bt_compress_arena(l, m["bitmap"], arena, cursor, m["off"], m["prefix"], m["nnz"], ws, m["status"])
+        B.bt_compress_arena_batch(items_f, torch.float32, arena, cursor, offsets, ws)
 
     def reverse():
-        for l, m in zip(reversed(layers), reversed(meta)):
-            B.bt_decompress_arena(m["bitmap"], arena, m["off"], m["prefix"], back[:l.numel()])
+        offsets_r.copy_(offsets.flip(0))
+        B.bt_decompress_arena_batch(items_r, torch.float32, arena, offsets_r)
 
     ms_f, ms_r = T.time(forward, reps=5), T.time(reverse, reps=5)
     ms_both = T.time(lambda: (forward(), reverse()), reps=5)
     torch.cuda.synchronize()
-    assert all(int(m["status"].item()) == B.BT_OK for m in meta)
-    assert [int(m["nnz"].item()) for m in meta] == nnz_true
-    assert torch.equal(back[:ns[0]].view(torch.int32), layers[0].view(torch.int32))      # the last one restored
+    assert all(st.status == B.BT_OK for st in stashes)
+    assert [st.nnz for st in stashes] == nnz_true
+    assert all(torch.equal(b.view(torch.int32), l.view(torch.int32)) for b, l in zip(backs, layers))
+    # the same trace as one launch per layer, for comparison
+    ws1 = B.new_workspace(max(ns), dev)
+    offs1 = [torch.zeros(1, dtype=torch.int64, device=dev) for _ in ns]
+
+    def forward_single():
+        cursor.zero_()
+        for l, st, o in zip(layers, stashes, offs1):
+            B.bt_compress_arena(l, st.bitmap, arena, cursor, o, st.chunk_prefix, st.nnz_out, ws1, st.dev_status)
+
+    def reverse_single():
+        for b, st, o in zip(reversed(backs), reversed(stashes), reversed(offs1)):
+            B.bt_decompress_arena(st.bitmap, arena, o, st.chunk_prefix, b)
+
+    ms_f1, ms_r1 = T.time(forward_single, reps=5), T.time(reverse_single, reps=5)
+    launches_f = (len(ns) + B.MAX_BATCH_PER_LAUNCH - 1) // B.MAX_BATCH_PER_LAUNCH
     stash_bytes = sum(B.bt_compressed_bytes(n, z, torch.float32) for n, z in zip(ns, nnz_true))
     assert stash_bytes == sum(4 * ((n + 31) // 32) + 4 * z + 8 * ((n + 4095) // 4096) for n, z in zip(ns, nnz_true))
     dense = 4 * sum(ns)
     alg_f = sum(algorithmic_bytes("bt_compress", n, z, 4) for n, z in zip(ns, nnz_true))
     z5 = 1.0 - sum(nnz_true) / sum(ns)
-    T.row("cfg5", "bt_compress_arena", "f32", z5, sum(ns), alg_f, ms_f, launches=len(ns), tensors=len(ns),
-          note="35 layers in forward order: one event pair around the 35 launches")
-    T.row("cfg5", "bt_decompress_arena", "f32", z5, sum(ns), alg_f, ms_r, launches=len(ns), tensors=len(ns),
-          note="35 layers in reverse order: one event pair around the 35 launches")
+    T.row("cfg5", "bt_compress_arena_batch", "f32", z5, sum(ns), alg_f, ms_f, launches=launches_f, tensors=len(ns),
+          note="35 layers in forward order, 32 per launch: one event pair around the %d launches" % launches_f)
+    T.row("cfg5", "bt_decompress_arena_batch", "f32", z5, sum(ns), alg_f, ms_r, launches=launches_f, tensors=len(ns),
+          note="35 layers in reverse order, 32 per launch: one event pair around the %d launches" % launches_f)
+    T.row("cfg5", "bt_compress_arena", "f32", z5, sum(ns), alg_f, ms_f1, launches=len(ns), tensors=len(ns),
+          note="the same forward pass as one launch per layer: one event pair around the 35 launches")
+    T.row("cfg5", "bt_decompress_arena", "f32", z5, sum(ns), alg_f, ms_r1, launches=len(ns), tensors=len(ns),
+          note="the same reverse pass as one launch per layer: one event pair around the 35 launches")
     extras["cfg5_trace"] = {"device_ms_forward_then_reverse": round(ms_both, 4), "device_ms_forward": round(ms_f, 4),
-                            "device_ms_reverse": round(ms_r, 4), "layers": len(ns), "elements": sum(ns),
+                            "device_ms_reverse": round(ms_r, 4), "launches": 2 * launches_f, "layers": len(ns), "elements": sum(ns),
                             "dense_bytes": dense, "peak_compressed_bytes": stash_bytes,
                             "compressed_over_dense": round(stash_bytes / dense, 4),
                             "arena_bytes_in_use_at_peak": int(cursor.item()),
                             "storage_policy": "exact size: every layer's packed values pushed back to back into one "
-                                              "arena (device-side cursor, 16-byte granules), bitmap and prefix array "
-                                              "per layer; nothing is sized from nnz on the host, no host "
-                                              "synchronisation between layers; the peak is reached after the last "
-                                              "forward layer, when all 35 stashes are live"}
-    del layers, arena, meta, ws, back
+                                              "arena (device-side cursor, 16-byte granules) by the batched arena calls, "
+                                              "32 layers per launch, bitmap and prefix array per layer; nothing is "
+                                              "sized from nnz on the host, no host synchronisation between layers; the "
+                                              "peak is reached after the last forward layer, when all 35 stashes are live"}
+    del layers, arena, stashes, ws, ws1, backs
     torch.cuda.empty_cache()
     return T.rows, extras
 

@@ -426,6 +426,29 @@ int bt_decompress_arena(const uint32_t *bitmap, const void *arena, const uint64_
                         const uint64_t *chunk_prefix, uint64_t n, int dtype, void *dense_out, void *stream);
 
 /*
+ * Batched arena forms: the tensors of a step pushed into the arena, or restored from it, by one launch per 32
+ * tensors.  bt_compress_arena_batch / bt_relu_fwd_compress_arena_batch: what `count` calls of bt_compress_arena /
+ * bt_prune_fwd_compress_arena (tau = 0) in the items' order would do -- tensor k's values start where tensor k-1's
+ * ended, each rounded up to 16 bytes, and values_offsets_out[k] (a DEVICE array of `count` words) receives the byte
+ * offset of tensor k's values; a tensor that does not fit reports BT_ERR_CAPACITY in its *dev_status, leaves its
+ * offset word and the cursor where they were, and the next tensor starts at the same place.  The items' values and
+ * values_capacity are ignored; a tensor with n == 0 gets *nnz_out = 0, *dev_status = BT_OK and offset 0.
+ * workspace_bytes >= bt_batch_workspace_bytes(n of every item).  bt_decompress_arena_batch restores every item's
+ * y_out from (bitmap, arena + values_offsets[k], chunk_prefix).  Calls that share an arena must be ordered on the
+ * device, as for the single-tensor forms.
+ */
+int bt_compress_arena_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype, void *arena,
+                            uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offsets_out,
+                            void *workspace, size_t workspace_bytes, void *stream);
+
+int bt_relu_fwd_compress_arena_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype, void *arena,
+                                     uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offsets_out,
+                                     void *workspace, size_t workspace_bytes, void *stream);
+
+int bt_decompress_arena_batch(const bt_batch_item *items /* host */, uint32_t count, int dtype, const void *arena,
+                              const uint64_t *values_offsets, void *stream);
+
+/*
  * Arena forms of the later calls.  The narrowing compressors push 16-bit values: the cursor advances by
  * 2 * nnz bytes rounded up to 16, and the room behind the cursor is counted in 16-bit elements;
  * bt_decompress_widen_arena (or bt_decompress_arena with the 16-bit type) reads them back.  The ReLU6

@@ -33,7 +33,8 @@ EXPORTS = ("bt_compressed_bytes", "bt_workspace_bytes", "bt_compress", "bt_decom
            "bt_compress_narrow_arena", "bt_prune_fwd_compress_narrow_arena", "bt_decompress_widen_arena",
            "bt_relu6_fwd_compress_arena", "bt_relu6_bwd_from_stash_arena", "bt_maxpool2x2_bwd_masked", "bt_set_max_ctas",
            "bt_batch_workspace_bytes", "bt_compress_batch", "bt_relu_fwd_compress_batch", "bt_decompress_batch",
-           "bt_relu_bwd_from_bitmap_batch")
+           "bt_relu_bwd_from_bitmap_batch", "bt_compress_arena_batch", "bt_relu_fwd_compress_arena_batch",
+           "bt_decompress_arena_batch")
 
 MAX_BATCH_PER_LAUNCH = 32
 
@@ -90,6 +91,11 @@ def load_library(path: str) -> ctypes.CDLL:
     for name in ("bt_decompress_batch", "bt_relu_bwd_from_bitmap_batch"):
         getattr(L, name).restype = i32
         getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp]
+    for name in ("bt_compress_arena_batch", "bt_relu_fwd_compress_arena_batch"):
+        getattr(L, name).restype = i32
+        getattr(L, name).argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp, u64, vp, vp, vp, sz, vp]
+    L.bt_decompress_arena_batch.restype = i32
+    L.bt_decompress_arena_batch.argtypes = [ctypes.POINTER(BatchItem), ctypes.c_uint32, i32, vp, vp, vp]
     L.bt_decompress.restype = i32
     L.bt_decompress.argtypes = [vp, vp, vp, u64, i32, vp, vp]
     L.bt_relu_fwd_compress.restype = i32
@@ -213,6 +219,24 @@ def bt_relu_fwd_compress_batch(items, dtype: torch.dtype, workspace: torch.Tenso
     st = lib().bt_relu_fwd_compress_batch(items, len(items), DTYPE_CODE[dtype], _ptr(workspace), _nbytes(workspace),
                                           _stream(stream))
     return _check("bt_relu_fwd_compress_batch", st, check)
+
+
+def bt_compress_arena_batch(items, dtype: torch.dtype, arena: torch.Tensor, arena_cursor: torch.Tensor,
+                            values_offsets_out: torch.Tensor, workspace: torch.Tensor, *, fused: bool = False, stream=None,
+                            check: bool = True) -> int:
+    """The tensors of `items` pushed into the arena back to back by one pass (fused: ReLU forward first);
+    values_offsets_out is a device int64 tensor with one word per item."""
+    fn = lib().bt_relu_fwd_compress_arena_batch if fused else lib().bt_compress_arena_batch
+    st = fn(items, len(items), DTYPE_CODE[dtype], _ptr(arena), _nbytes(arena), _ptr(arena_cursor), _ptr(values_offsets_out),
+            _ptr(workspace), _nbytes(workspace), _stream(stream))
+    return _check("bt_compress_arena_batch", st, check)
+
+
+def bt_decompress_arena_batch(items, dtype: torch.dtype, arena: torch.Tensor, values_offsets: torch.Tensor, *, stream=None,
+                              check: bool = True) -> int:
+    """Every item's y_out restored from (bitmap, arena + values_offsets[k], chunk_prefix) in one pass."""
+    st = lib().bt_decompress_arena_batch(items, len(items), DTYPE_CODE[dtype], _ptr(arena), _ptr(values_offsets), _stream(stream))
+    return _check("bt_decompress_arena_batch", st, check)
 
 
 def bt_decompress_batch(items, dtype: torch.dtype, *, stream=None, check: bool = True) -> int:

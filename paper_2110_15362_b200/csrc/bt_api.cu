@@ -75,11 +75,16 @@ int compress_common(const void *src, uint64_t n, int dtype, int fused, float tau
 // words and take no part in the launches; the others go out kMaxBatch at a time, one launch after the other on
 // the stream, all through the same workspace.
 int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype, int fused, void *workspace,
-                          size_t workspace_bytes, void *stream)
+                          size_t workspace_bytes, void *stream, const bt::BatchArena *arena = nullptr,
+                          uint64_t *offsets_out = nullptr)
 {
     if (elem_size_of(dtype) == 0) return BT_ERR_DTYPE;
     if (count == 0) return BT_OK;
     if (!items) return BT_ERR_NULL;
+    if (arena) {
+        if (!arena->arena || !arena->arena_cursor || !offsets_out) return BT_ERR_NULL;
+        if (!aligned(arena->arena, 16) || !aligned(arena->arena_cursor, 8) || !aligned(offsets_out, 8)) return BT_ERR_ALIGN;
+    }
     uint64_t chunks = 0;
     bool     any_y = false, all_y = true, any = false;
     for (uint32_t k = 0; k < count; ++k) {
@@ -88,8 +93,8 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
         if (!aligned(it.nnz_out, 8) || !aligned(it.dev_status, 4)) return BT_ERR_ALIGN;
         if (it.n == 0) continue;
         if (!it.dense || !it.bitmap || !it.chunk_prefix) return BT_ERR_NULL;
-        if (!it.values && it.values_capacity != 0) return BT_ERR_NULL;
-        if (!aligned(it.dense, 16) || !aligned(it.y_out, 16) || !aligned(it.bitmap, 4) || !aligned(it.values, 16) ||
+        if (!arena && !it.values && it.values_capacity != 0) return BT_ERR_NULL;
+        if (!aligned(it.dense, 16) || !aligned(it.y_out, 16) || !aligned(it.bitmap, 4) || (!arena && !aligned(it.values, 16)) ||
             !aligned(it.chunk_prefix, 8))
             return BT_ERR_ALIGN;
         any = true;
@@ -101,7 +106,7 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
     if (any_y && !all_y) return BT_ERR_SHAPE;                // a dense output for every tensor of a batch or for none
     if (any && !workspace) return BT_ERR_NULL;
     if (any && !aligned(workspace, 16)) return BT_ERR_ALIGN;
-    if (any && workspace_bytes < bt::compress_workspace_bytes(chunks)) return BT_ERR_WORKSPACE;
+    if (any && workspace_bytes < bt::batch_workspace_bytes(chunks, count)) return BT_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     bt::CompressJob jobs[bt::kMaxBatch];
     uint32_t        m = 0;
@@ -110,21 +115,23 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
         if (it.n == 0) {
             if (cudaMemsetAsync(it.nnz_out, 0, sizeof(uint64_t), s) != cudaSuccess) return BT_ERR_CUDA;
             if (it.dev_status && cudaMemsetAsync(it.dev_status, 0, sizeof(int32_t), s) != cudaSuccess) return BT_ERR_CUDA;
+            if (arena && cudaMemsetAsync(offsets_out + k, 0, sizeof(uint64_t), s) != cudaSuccess) return BT_ERR_CUDA;
         } else {
             bt::CompressJob &j = jobs[m++];
             j                  = bt::CompressJob{};
             j.src              = it.dense;
             j.y                = fused ? it.y_out : nullptr;
             j.bitmap           = it.bitmap;
-            j.values           = it.values;
-            j.capacity         = it.values_capacity;
+            j.values           = arena ? nullptr : it.values;
+            j.capacity         = arena ? 0 : it.values_capacity;
             j.prefix           = it.chunk_prefix;
             j.nnz_out          = it.nnz_out;
             j.dev_status       = it.dev_status;
             j.n                = it.n;
+            j.offset_out       = arena ? offsets_out + k : nullptr;
         }
         if (m == bt::kMaxBatch || (k + 1 == count && m > 0)) {
-            if (bt::launch_compress_batch(jobs, m, 0.0f, workspace, dtype, fused, s) != cudaSuccess) return BT_ERR_CUDA;
+            if (bt::launch_compress_batch(jobs, m, 0.0f, workspace, dtype, fused, arena, s) != cudaSuccess) return BT_ERR_CUDA;
             m = 0;
         }
     }
@@ -133,7 +140,8 @@ int compress_batch_common(const bt_batch_item *items, uint32_t count, int dtype,
 
 // The consumers of a batch of stashes: backward == false restores items[k].y_out from (bitmap, values, chunk_prefix),
 // backward == true writes items[k].y_out = bit ? items[k].dense : +0.
-int consume_batch_common(const bt_batch_item *items, uint32_t count, int dtype, bool backward, void *stream)
+int consume_batch_common(const bt_batch_item *items, uint32_t count, int dtype, bool backward, void *stream,
+                         const void *arena = nullptr, const uint64_t *offsets = nullptr)
 {
     const int es = elem_size_of(dtype);
     if (es == 0) return BT_ERR_DTYPE;
@@ -143,16 +151,18 @@ int consume_batch_common(const bt_batch_item *items, uint32_t count, int dtype, 
         const bt_batch_item &it = items[k];
         if (it.n == 0) continue;
         if (!it.bitmap || !it.y_out) return BT_ERR_NULL;
-        if (backward ? !it.dense : (!it.values || !it.chunk_prefix)) return BT_ERR_NULL;
+        if (backward ? !it.dense : ((!arena && !it.values) || !it.chunk_prefix)) return BT_ERR_NULL;
         if (!aligned(it.bitmap, 4) || !aligned(it.y_out, 16)) return BT_ERR_ALIGN;
-        if (backward ? !aligned(it.dense, 16) : (!aligned(it.values, 16) || !aligned(it.chunk_prefix, 8))) return BT_ERR_ALIGN;
+        if (backward ? !aligned(it.dense, 16) : ((!arena && !aligned(it.values, 16)) || !aligned(it.chunk_prefix, 8))) return BT_ERR_ALIGN;
     }
     cudaStream_t      s = static_cast<cudaStream_t>(stream);
     bt::DecompressJob jobs[bt::kMaxBatch];
     uint32_t          m = 0;
     for (uint32_t k = 0; k < count; ++k) {
         const bt_batch_item &it = items[k];
-        if (it.n != 0) jobs[m++] = bt::DecompressJob{it.bitmap, it.values, it.chunk_prefix, it.dense, it.y_out, it.n};
+        if (it.n != 0)
+            jobs[m++] = bt::DecompressJob{it.bitmap, arena ? arena : it.values, it.chunk_prefix, it.dense, it.y_out, it.n,
+                                          arena ? offsets + k : nullptr};
         if (m == bt::kMaxBatch || (k + 1 == count && m > 0)) {
             const cudaError_t e = backward ? bt::launch_relu_bwd_batch(jobs, m, es, s) : bt::launch_decompress_batch(jobs, m, es, s);
             if (e != cudaSuccess) return BT_ERR_CUDA;
@@ -215,7 +225,7 @@ size_t bt_batch_workspace_bytes(const uint64_t *n, uint32_t count)
 {
     uint64_t chunks = 0;
     for (uint32_t k = 0; n && k < count; ++k) chunks += ceil_div(n[k], BT_CHUNK_ELEMS);
-    return bt::compress_workspace_bytes(chunks);
+    return bt::batch_workspace_bytes(chunks, count);
 }
 
 int bt_compress_batch(const bt_batch_item *items, uint32_t count, int dtype, void *workspace, size_t workspace_bytes,
@@ -224,9 +234,33 @@ int bt_compress_batch(const bt_batch_item *items, uint32_t count, int dtype, voi
     return compress_batch_common(items, count, dtype, 0, workspace, workspace_bytes, stream);
 }
 
+int bt_compress_arena_batch(const bt_batch_item *items, uint32_t count, int dtype, void *arena, uint64_t arena_bytes,
+                            uint64_t *arena_cursor, uint64_t *values_offsets_out, void *workspace, size_t workspace_bytes,
+                            void *stream)
+{
+    const bt::BatchArena a{arena, arena_bytes, arena_cursor};
+    return compress_batch_common(items, count, dtype, 0, workspace, workspace_bytes, stream, &a, values_offsets_out);
+}
+
+int bt_relu_fwd_compress_arena_batch(const bt_batch_item *items, uint32_t count, int dtype, void *arena,
+                                     uint64_t arena_bytes, uint64_t *arena_cursor, uint64_t *values_offsets_out,
+                                     void *workspace, size_t workspace_bytes, void *stream)
+{
+    const bt::BatchArena a{arena, arena_bytes, arena_cursor};
+    return compress_batch_common(items, count, dtype, 1, workspace, workspace_bytes, stream, &a, values_offsets_out);
+}
+
 int bt_decompress_batch(const bt_batch_item *items, uint32_t count, int dtype, void *stream)
 {
     return consume_batch_common(items, count, dtype, false, stream);
+}
+
+int bt_decompress_arena_batch(const bt_batch_item *items, uint32_t count, int dtype, const void *arena,
+                              const uint64_t *values_offsets, void *stream)
+{
+    if (count != 0 && (!arena || !values_offsets)) return BT_ERR_NULL;
+    if (!aligned(arena, 16) || !aligned(values_offsets, 8)) return BT_ERR_ALIGN;
+    return consume_batch_common(items, count, dtype, false, stream, arena, values_offsets);
 }
 
 int bt_relu_bwd_from_bitmap_batch(const bt_batch_item *items, uint32_t count, int dtype, void *stream)

@@ -133,6 +133,8 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     __shared__ __align__(8) uint64_t s_ready[kStages];     // base and offsets are in shared      (scan warp -> copiers)
     __shared__ __align__(8) uint64_t s_empty[kStages];     // every copier is done with the slot  (copiers -> load warp)
     __shared__ uint64_t          s_base[kStages];          // exclusive base of the tile in the slot
+    __shared__ uint64_t          s_dst[kStages];           // arena form: byte offset of the tile's tensor in the arena
+    __shared__ uint64_t          s_arena_c0;               // arena form: the cursor as the launch found it
     __shared__ uint32_t          s_cnt[kStages][kWarps];   // packed count of each segment
     __shared__ uint32_t          s_off[kStages][kWarps];   // exclusive offset of each segment in the tile
     __shared__ uint32_t          s_agg[kStages];           // packed count of the tile
@@ -151,7 +153,11 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
     bool meet = false;
     for (uint32_t k = 0; k < p.c.jobs; ++k) meet = meet || p.job[k].tiles > G;
 
+    const bool in_arena = p.c.arena != nullptr;
     if (tid == 0) {
+        // read before the barrier below: the launch's first update of the cursor follows a tensor's last base,
+        // which needs a publication from every CTA, and a CTA publishes only after this barrier
+        s_arena_c0 = in_arena ? *reinterpret_cast<const volatile uint64_t *>(p.c.arena_cursor) : 0;
         s_abort    = 0;
         s_tag      = 0;
         for (int s = 0; s < kStages; ++s) {
@@ -271,6 +277,8 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         uint32_t pk = 0, pj = 0, pv = 0;            // this warp's previous tile: tensor, wave, virtual CTA
         uint64_t waves_before = 0;                  // sum of the totals of the waves before the previous tile ...
         uint32_t waves_of     = 0xFFFFFFFFu;        // ... of this tensor
+        uint64_t arena_at     = 0;                  // arena form: byte offset of the values of tensor arena_of ...
+        uint32_t arena_of     = 0xFFFFFFFFu;        // ... (none yet)
 
         for (uint32_t i = q; !failed && i <= last_i + 2; i += 2) {
             const bool has = i <= last_i;
@@ -340,13 +348,46 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                     const uint64_t chunks_total = (jb.n + BT_CHUNK_ELEMS - 1) / BT_CHUNK_ELEMS;
                     if (ch < chunks_total && extent_of(jb.prefix, 8 * chunks_total).holds(jb.prefix + ch, 8)) jb.prefix[ch] = base + s_off[ps][lane];
                 }
+                // Arena form: the tensor's values start where the tensor before it ended.  That cursor is published,
+                // under the launch's tag, by whoever finishes that tensor's last tile; tensor 0 starts at the cursor
+                // the launch found.  Read once per tensor and warp (bounded, like every wait here).
+                if (in_arena && arena_of != pk) {
+                    uint64_t at = s_arena_c0;
+                    if (pk > 0) {
+                        const uint64_t *const w = p.c.ws_arena + 2 * (pk - 1);
+                        uint64_t       a0 = 0, a1 = 0;
+                        const uint64_t ta = now_ns();
+                        for (;;) {
+                            ld_relaxed_2xu64(w, a0, a1);
+                            if (((a0 ^ tag_w0) >> 32) == 0 && ((a1 ^ tag_w1) >> 32) == 0) break;
+                            if (now_ns() - ta > wait_ns || ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag) {
+                                failed = true;
+                                break;
+                            }
+                            __nanosleep(100);
+                        }
+                        if (failed) break;
+                        at = (a0 & 0xFFFFFFFFull) | (a1 << 32);
+                    }
+                    arena_at = at, arena_of = pk;
+                }
                 bool bump = false;              // lane 0: this is the launch's last tile
                 if (pt == jb.tiles - 1 && lane == 0) {
                     const uint64_t nnz = base + s_agg[ps];
                     *jb.nnz_out        = nnz;
                     __threadfence();
                     const bool aborted  = ld_relaxed_u64(p.c.ws_header + kHdrAbort) == tag;
-                    const uint64_t capacity = jb.capacity;
+                    uint64_t   capacity = jb.capacity;
+                    if (in_arena) {
+                        // the room behind the tensor's start; the cursor moves past it only when everything fitted
+                        capacity            = arena_at <= p.c.arena_bytes ? (p.c.arena_bytes - arena_at) / sizeof(U) : 0;
+                        const bool     fits = !aborted && nnz <= capacity;
+                        const uint64_t end  = fits ? arena_at + ((nnz * sizeof(U) + 15) & ~15ull) : arena_at;
+                        if (fits) *jb.offset_out = arena_at;
+                        if (pk + 1 == p.c.jobs) *p.c.arena_cursor = end;
+                        if (wsx.holds(p.c.ws_arena + 2 * pk, 16))
+                            st_relaxed_2xu64(p.c.ws_arena + 2 * pk, tag_w0 | (end & 0xFFFFFFFFull), tag_w1 | (end >> 32));
+                    }
                     // without a meeting: every CTA has published its count by now, so every CTA has read the sequence
                     // number, and the next launch on this workspace gets another tag
                     bump = pk + 1 == p.c.jobs;
@@ -391,6 +432,7 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 }
                 if (lane == 0) {
                     s_base[ps] = base;
+                    s_dst[ps]  = arena_at;
                     mbar_arrive(&s_ready[ps]);                       // the copiers may take the tile
                 }
             }
@@ -432,8 +474,13 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         for (uint32_t it = 0; w.valid; ++it, walk_next(w, p, cta, G)) {
             const uint32_t s = it % kStages;
             if (!mbar_wait(&s_ready[s], (it / kStages) & 1u, &s_abort, wait_ns)) break;
-            V *const       vals     = static_cast<V *>(p.job[w.k].values);
-            const uint64_t capacity = p.job[w.k].capacity;
+            V             *vals     = static_cast<V *>(p.job[w.k].values);
+            uint64_t       capacity = p.job[w.k].capacity;
+            if (in_arena) {
+                const uint64_t at = s_dst[s];
+                vals              = reinterpret_cast<V *>(static_cast<unsigned char *>(p.c.arena) + at);
+                capacity          = at <= p.c.arena_bytes ? (p.c.arena_bytes - at) / sizeof(V) : 0;
+            }
             const Extent   vx       = extent_of(vals, capacity * sizeof(V));
             const uint64_t base     = s_base[s];
 #pragma unroll
@@ -554,7 +601,8 @@ cudaError_t launch_shaped(const CompressCommon &c, const CompressJob *jobs, uint
     p.c.ws_header = static_cast<uint64_t *>(workspace);
     p.c.ws_total  = reinterpret_cast<uint64_t *>(static_cast<unsigned char *>(workspace) + kWsHeaderBytes);
     p.c.ws_desc   = p.c.ws_total + p.c.ws_totals;
-    p.c.ws_words  = (compress_workspace_bytes(chunks) - kWsHeaderBytes) / 8;
+    p.c.ws_words  = (batch_workspace_bytes(chunks, count) - kWsHeaderBytes) / 8;
+    p.c.ws_arena  = p.c.ws_desc + 2 * dealt;                          // behind the descriptors: 16-byte aligned like them
     p.c.call_tag  = next_call_tag();
     p.c.wait_ns   = compress_wait_ns();
     // cooperative launch: the runtime guarantees that all `grid` CTAs are resident together
@@ -574,7 +622,7 @@ cudaError_t launch_typed(const CompressCommon &c, const CompressJob *jobs, uint3
 }  // namespace
 
 cudaError_t launch_compress_batch(const CompressJob *jobs, uint32_t count, float tau, void *workspace, int dtype, int fused,
-                                  cudaStream_t stream)
+                                  const BatchArena *arena, cudaStream_t stream)
 {
     // fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0)
     // the dense output is written for all tensors of a launch or for none
@@ -584,6 +632,11 @@ cudaError_t launch_compress_batch(const CompressJob *jobs, uint32_t count, float
         if ((jobs[k].y != nullptr) != y) return cudaErrorInvalidValue;
     CompressCommon c{};
     c.tau = tau;
+    if (arena) {
+        c.arena        = arena->arena;
+        c.arena_bytes  = arena->arena_bytes;
+        c.arena_cursor = arena->arena_cursor;
+    }
     if (fused == 0) {
         return dtype == BT_F64   ? launch_typed<uint64_t, -1, false>(c, jobs, count, workspace, stream)
                : dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(c, jobs, count, workspace, stream)

@@ -44,6 +44,7 @@ __device__ __forceinline__ uint32_t widened(const uint16_t h)
 struct RestoreJob {
     const uint32_t *bitmap;
     const void     *values;
+    const uint64_t *values_offset;  // NULL, or the device word holding the byte offset of the values inside `values`
     const uint64_t *prefix;
     void           *out;
     uint64_t        n;
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(kWarps * 32)
 decompress_batch_kernel(const __grid_constant__ RestoreParams<kJobs> p)
 {
     const RestoreJob &j = p.job[job_of_block(p)];
-    decompress_body<U, kE, kGrp, kWarps, 0>(j.bitmap, static_cast<const U *>(j.values), nullptr, j.prefix, j.n, static_cast<U *>(j.out),
+    decompress_body<U, kE, kGrp, kWarps, 0>(j.bitmap, static_cast<const U *>(j.values), j.values_offset, j.prefix, j.n, static_cast<U *>(j.out),
                                             blockIdx.x - j.first_block);
 }
 
@@ -332,7 +333,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2048 / (kWarps * 32))
 decompress16_batch_kernel(const __grid_constant__ RestoreParams<kJobs> p)
 {
     const RestoreJob &j = p.job[job_of_block(p)];
-    decompress16_body<kWarps>(j.bitmap, static_cast<const uint16_t *>(j.values), nullptr, j.prefix, j.n, static_cast<uint16_t *>(j.out),
+    decompress16_body<kWarps>(j.bitmap, static_cast<const uint16_t *>(j.values), j.values_offset, j.prefix, j.n, static_cast<uint16_t *>(j.out),
                               blockIdx.x - j.first_block);
 }
 
@@ -389,7 +390,7 @@ cudaError_t launch_decompress_batch(const DecompressJob *jobs, uint32_t count, i
     uint64_t                 blocks = 0;
     for (uint32_t k = 0; k < count; ++k) {
         const uint64_t quarters = (jobs[k].n + 1023) >> 10;
-        p.job[k] = RestoreJob{jobs[k].bitmap, jobs[k].values, jobs[k].prefix, jobs[k].out, jobs[k].n, static_cast<uint32_t>(blocks)};
+        p.job[k] = RestoreJob{jobs[k].bitmap, jobs[k].values, jobs[k].values_offset, jobs[k].prefix, jobs[k].out, jobs[k].n, static_cast<uint32_t>(blocks)};
         blocks += (quarters + kWarps - 1) / kWarps;
         if (blocks > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     }

@@ -70,6 +70,7 @@ struct CompressJob {
     uint64_t   *nnz_out;
     int32_t    *dev_status;
     uint64_t    n;
+    uint64_t   *offset_out; // arena form: where the byte offset of the tensor's values in the arena goes
     // set by launch_compress_batch:
     uint32_t    tiles;      // number of tiles of the tensor
     uint32_t    rot;        // the CTA that takes the tensor's tile 0 (tile t goes to CTA (rot + t) mod grid)
@@ -88,14 +89,34 @@ struct CompressCommon {
     uint64_t    call_tag;   // unique to the call
     uint64_t    wait_ns;    // bound of every in-kernel wait
     float       tau;        // fused form: elements <= tau become +0 (0 for plain ReLU)
+    // arena form (arena != nullptr): the tensors' values go back to back behind *arena_cursor
+    void       *arena;
+    uint64_t    arena_bytes;
+    uint64_t   *arena_cursor;
+    uint64_t   *ws_arena;   // two tagged words per tensor: the cursor behind that tensor (set by launch_compress_batch)
 };
+
+// What the caller of launch_compress_batch gives for the arena form.
+struct BatchArena {
+    void     *arena;
+    uint64_t  arena_bytes;
+    uint64_t *arena_cursor;
+};
+
+// bytes of workspace for a batched launch: the tensors' descriptors and totals, and two words per tensor for the
+// arena form's chain of cursors
+__host__ __device__ constexpr size_t batch_workspace_bytes(uint64_t chunks, uint32_t count)
+{
+    return compress_workspace_bytes(chunks) + 16 * static_cast<size_t>(count);
+}
 
 // fused: 0 plain compressor, 1 threshold form (ReLU at tau = 0), 2 ReLU6
 cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStream_t s);
 // `jobs` (count of them: 1 .. kMaxBatch, every n > 0) are the tensors of one launch; `workspace` holds at least
-// compress_workspace_bytes() of their chunks; fused: 0 plain compressor, 1 threshold form
+// batch_workspace_bytes() of their chunks; fused: 0 plain compressor, 1 threshold form; arena: nullptr, or the arena
+// the values go to (the jobs' values / capacity are then ignored and their offset_out must be set)
 cudaError_t launch_compress_batch(const CompressJob *jobs, uint32_t count, float tau, void *workspace, int dtype, int fused,
-                                  cudaStream_t s);
+                                  const BatchArena *arena, cudaStream_t s);
 // the calling thread's limit on the CTAs of one compress launch (0: none); returns the limit it replaces
 uint32_t set_compress_max_ctas(uint32_t max_ctas);
 // the bound of the compress kernels' waits for later launches of the process; returns the one it replaces
@@ -113,6 +134,7 @@ struct DecompressJob {
     const void     *in;
     void           *out;
     uint64_t        n;
+    const uint64_t *values_offset;   // restore only: NULL, or a device word with the byte offset of the values inside `values`
 };
 cudaError_t launch_decompress_batch(const DecompressJob *jobs, uint32_t count, int elem_size, cudaStream_t s);
 cudaError_t launch_relu_bwd_batch(const DecompressJob *jobs, uint32_t count, int elem_size, cudaStream_t s);

@@ -146,3 +146,88 @@ def test_batched_consumers_over_more_tensors_than_one_launch_holds_and_argument_
     assert B.bt_decompress_batch(items, torch.bfloat16, check=False) == B.BT_ERR_ALIGN
     assert B.lib().bt_decompress_batch(None, 0, B.BT_F32, None) == B.BT_OK
     assert B.lib().bt_decompress_batch(items, 1, 11, None) == B.BT_ERR_DTYPE
+
+
+def _arena_batch(kind, sizes, seed, fused, arena_bytes, cursor0=0, zeros=0.5):
+    dt = TDT[kind]
+    raws = [W.random_patterns(n, kind, zeros, seed=seed + 7 * k) for k, n in enumerate(sizes)]
+    xs = [from_raw(r, kind) if r.size else torch.empty(0, dtype=dt, device="cuda") for r in raws]
+    sts = [B.Stash(max(n, 1), dt, values_capacity=1) for n in sizes]          # the values go to the arena, not here
+    items = B.batch_items(xs, sts)
+    for k, n in enumerate(sizes):
+        items[k].n = n
+        items[k].values = None
+        items[k].values_capacity = 0
+    arena = torch.full((arena_bytes + 4096,), 0x5A, dtype=torch.uint8, device="cuda")
+    cursor = torch.full((1,), cursor0, dtype=torch.int64, device="cuda")
+    offsets = torch.full((len(sizes),), -7, dtype=torch.int64, device="cuda")
+    ws = torch.empty(B.bt_batch_workspace_bytes(sizes), dtype=torch.uint8, device="cuda")
+    ws.random_(0, 255)
+    B.bt_compress_arena_batch(items, dt, arena[:arena_bytes], cursor, offsets, ws, fused=fused)
+    torch.cuda.synchronize()
+    return raws, sts, items, arena, cursor, offsets
+
+
+@pytest.mark.parametrize("kind", ["f32", "bf16", "f16", "f64"])
+@pytest.mark.parametrize("fused", [False, True])
+def test_arena_batch_is_the_sequence_of_single_arena_pushes(oracle, kind, fused):
+    """Values of all tensors back to back behind the cursor, 16-byte granules, exactly as one bt_compress_arena call
+    per tensor would leave them; offsets, cursor, bitmaps, prefix arrays and counts against the oracle; nothing
+    written beyond the final cursor; then the whole batch restored from the arena by one call."""
+    es = np.dtype(W.random_patterns(1, kind, 0.0, seed=0).dtype).itemsize
+    raws, sts, items, arena, cursor, offsets = _arena_batch(kind, SIZES, 321, fused, 64 << 20, cursor0=4096)
+    at = 4096
+    for k, raw in enumerate(raws):
+        c = oracle.relu_fwd_compress(raw, kind)[1] if fused else oracle.compress(raw)
+        assert sts[k].status == B.BT_OK and sts[k].nnz == c.nnz, k
+        if raw.size == 0:
+            assert int(offsets[k].item()) == 0
+            continue
+        assert int(offsets[k].item()) == at, k
+        got = arena[at:at + c.nnz * es].cpu().numpy().view(raw.dtype)
+        assert np.array_equal(got, c.values), k
+        assert np.array_equal(W.raw_numpy(sts[k].bitmap)[:(raw.size + 31) // 32].view(np.uint32), c.bitmap), k
+        assert np.array_equal(W.raw_numpy(sts[k].chunk_prefix)[:(raw.size + 4095) // 4096].view(np.uint64), c.prefix), k
+        at += (c.nnz * es + 15) // 16 * 16
+    assert int(cursor.item()) == at
+    assert bool((arena[:4096] == 0x5A).all().item()) and bool((arena[at:] == 0x5A).all().item())
+    # restore all of them with one call
+    dt = TDT[kind]
+    outs = [torch.empty(max(r.size, 1), dtype=dt, device="cuda") for r in raws]
+    ritems = B.batch_items(outs, sts, outs)
+    for k, r in enumerate(raws):
+        ritems[k].n = r.size
+        ritems[k].values = None
+    B.bt_decompress_arena_batch(ritems, dt, arena, offsets)
+    torch.cuda.synchronize()
+    for k, raw in enumerate(raws):
+        want = oracle.relu_fwd_compress(raw, kind)[0] if fused else raw
+        assert np.array_equal(W.raw_numpy(outs[k])[:raw.size], want), k
+
+
+def test_arena_batch_over_several_launches_and_an_arena_that_runs_full(oracle):
+    sizes = [4096 * (1 + k % 5) + k for k in range(2 * B.MAX_BATCH_PER_LAUNCH + 3)]
+    raws, sts, items, arena, cursor, offsets = _arena_batch("f32", sizes, 77, False, 16 << 20)
+    at = 0
+    for k, raw in enumerate(raws):                               # the cursor runs on from launch to launch
+        c = oracle.compress(raw)
+        assert sts[k].status == B.BT_OK and int(offsets[k].item()) == at
+        assert np.array_equal(arena[at:at + 4 * c.nnz].cpu().numpy().view(np.uint32), c.values)
+        at += (4 * c.nnz + 15) // 16 * 16
+    assert int(cursor.item()) == at
+    # an arena with room for the first two tensors only: the others report BT_ERR_CAPACITY, the cursor stays behind
+    # the second, their counts, bitmaps and prefix arrays are still complete
+    sizes = [8192 * 3 + 5, 4096, 8192 * 30 + 1, 100, 8192 * 2]
+    counts = [oracle.compress(W.random_patterns(n, "f32", 0.5, seed=500 + 7 * k)).nnz for k, n in enumerate(sizes)]
+    room = sum((4 * z + 15) // 16 * 16 for z in counts[:2]) + 16
+    raws, sts, items, arena, cursor, offsets = _arena_batch("f32", sizes, 500, False, room)
+    end2 = room - 16
+    assert [st.status for st in sts] == [B.BT_OK, B.BT_OK, B.BT_ERR_CAPACITY, B.BT_ERR_CAPACITY, B.BT_ERR_CAPACITY]
+    assert int(cursor.item()) == end2 and [int(o) for o in offsets[:2].tolist()] == [0, (4 * counts[0] + 15) // 16 * 16]
+    assert [int(o) for o in offsets[2:].tolist()] == [-7, -7, -7]
+    for k, raw in enumerate(raws):
+        c = oracle.compress(raw)
+        assert sts[k].nnz == c.nnz
+        assert np.array_equal(W.raw_numpy(sts[k].bitmap)[:(raw.size + 31) // 32].view(np.uint32), c.bitmap)
+        assert np.array_equal(W.raw_numpy(sts[k].chunk_prefix)[:(raw.size + 4095) // 4096].view(np.uint64), c.prefix)
+    assert bool((arena[room:] == 0x5A).all().item())           # nothing beyond the arena, whatever did not fit

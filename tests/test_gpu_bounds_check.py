@@ -97,6 +97,12 @@ def test_arena_forms(checked, oracle):
 def test_batched_forms(checked, oracle, kind):
     test_gpu_batch.test_batch_equals_the_oracle_tensor_by_tensor(oracle, kind, False, False)
     test_gpu_batch.test_batch_equals_the_oracle_tensor_by_tensor(oracle, kind, True, True)
+    test_gpu_batch.test_batched_consumers_equal_the_oracle_tensor_by_tensor(oracle, kind)
+    test_gpu_batch.test_arena_batch_is_the_sequence_of_single_arena_pushes(oracle, kind, True)
+
+
+def test_arena_batch_that_runs_full(checked, oracle):
+    test_gpu_batch.test_arena_batch_over_several_launches_and_an_arena_that_runs_full(oracle)
 
 
 def test_host_forms(checked, oracle):
