@@ -31,7 +31,11 @@ def build_all(force: bool = False) -> None:
 
 def _load(path: str) -> ctypes.CDLL:
     if path not in _loaded:
-        _build.build_library(out=path, extra_flags=_FLAGS[path])
+        try:
+            _build.build_library(out=path, extra_flags=_FLAGS[path])      # a no-op when the library is up to date
+        except Exception:
+            if not os.path.exists(path):                                   # no compiler here and nothing built: give up
+                raise
         _loaded[path] = B.load_library(path)
     return _loaded[path]
 
