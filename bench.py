@@ -464,7 +464,99 @@ def kernel_table(dev, peak_gbs: float):
                                               "peak is reached after the last forward layer, when all 35 stashes are live"}
     del layers, arena, stashes, ws, ws1, backs
     torch.cuda.empty_cache()
+
+    next_rows(T, B, W, dev)
     return T.rows, extras
+
+
+def next_rows(T: KernelTimer, B, W, dev):
+    """The calls built after the hot path (pruning threshold, double mask, ReLU6 pair, down-cast on stash, 8-byte
+    elements, max pooling), each alone on the 1 GiB fp32 tensor, the 392 MiB bf16 tensor or the 1 GiB fp64 tensor."""
+    import torch
+    for kind, n in (("f32", 1 << 28), ("bf16", 64 * 64 * 224 * 224), ("f64", 1 << 27)):
+        if kind == "f32":
+            x = W.cfg3_iid(n, 0.5, 2, dev)
+            pre = x
+        elif kind == "f64":
+            x = W.cfg3_iid(n, 0.5, 3, dev).double()
+            pre = x
+        else:
+            pre = W.cfg4_preact(0, (n,), kind, dev)
+            x = torch.relu(pre) + 0.0
+        es = x.element_size()
+        st = B.Stash(n, x.dtype, dev)
+        ws = B.new_workspace(n, dev)
+        dense = torch.empty_like(x)
+        meta = 4 * ((n + 31) // 32) + 8 * ((n + 4095) // 4096)
+
+        def add(kernel, ms, alg, **extra):
+            T.row("next", kernel, kind, 1.0 - st.nnz / n, n, alg, ms, **extra)
+
+        if kind == "f64":                                    # 8-byte elements through the graded calls
+            ms = T.time(lambda: B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+            add("bt_compress", ms, algorithmic_bytes("bt_compress", n, st.nnz, es))
+            ms = T.time(lambda: B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, dense))
+            add("bt_decompress", ms, algorithmic_bytes("bt_decompress", n, st.nnz, es))
+            ms = T.time(lambda: B.bt_relu_bwd_from_bitmap(st.bitmap, x, dense))
+            add("bt_relu_bwd_from_bitmap", ms, algorithmic_bytes("bt_relu_bwd_from_bitmap", n, 0, es))
+        ms = T.time(lambda: B.bt_relu6_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+        torch.cuda.synchronize()
+        nnz6 = st.nnz
+        add("bt_relu6_fwd_compress", ms, n * es + meta + nnz6 * es, dense_output=False)
+        ms = T.time(lambda: B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, x, dense))
+        add("bt_relu6_bwd_from_stash", ms, 2 * n * es + meta + nnz6 * es)
+        if kind == "f32":
+            for to, tdt in (("f16", torch.float16), ("bf16", torch.bfloat16)):
+                v16 = torch.empty(n, dtype=tdt, device=dev)
+                ms = T.time(lambda: B.bt_compress_narrow(x, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+                torch.cuda.synchronize()
+                by16 = n * es + meta + st.nnz * 2
+                add("bt_compress_narrow", ms, by16, values=to)
+                ms = T.time(lambda: B.bt_prune_fwd_compress_narrow(pre, 0.0, None, st.bitmap, v16, st.chunk_prefix, st.nnz_out, ws,
+                                                                    st.dev_status))
+                add("bt_prune_fwd_compress_narrow", ms, by16, values=to, tau=0.0)
+                ms = T.time(lambda: B.bt_decompress_widen(st.bitmap, v16, st.chunk_prefix, dense))
+                add("bt_decompress_widen", ms, by16, values=to)
+                del v16
+        B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
+        torch.cuda.synchronize()
+        nnz = st.nnz
+        masked = torch.empty(nnz, dtype=x.dtype, device=dev)
+        ms = T.time(lambda: B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, None, masked))
+        add("bt_mask_compress", ms, n * es + meta + nnz * es, dense_output=False)
+        ms = T.time(lambda: B.bt_mask_compress(pre, st.bitmap, st.chunk_prefix, dense, masked))
+        add("bt_mask_compress", ms, 2 * n * es + meta + nnz * es, dense_output=True)
+        del x, pre, st, ws, dense, masked
+        torch.cuda.empty_cache()
+
+    # the pruning thresholds of the paper's study on 2^28 close-to-zero fp32 pre-activations
+    n = 1 << 28
+    pre = W.prune_preact(n, dev)
+    st = B.Stash(n, pre.dtype, dev)
+    ws = B.new_workspace(n, dev)
+    for tau in W.PRUNE_THRESHOLDS:
+        ms = T.time(lambda: B.bt_prune_fwd_compress(pre, tau, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status))
+        torch.cuda.synchronize()
+        T.row("next", "bt_prune_fwd_compress", "f32", 1.0 - st.nnz / n, n, algorithmic_bytes("bt_relu_fwd_compress", n, st.nnz, 4), ms,
+              tau=tau, stash_bytes_over_dense=round(B.bt_compressed_bytes(n, st.nnz, pre.dtype) / (4.0 * n), 4), dense_output=False)
+    del pre, st, ws
+    torch.cuda.empty_cache()
+
+    # max pooling with winner codes: the first pooling layer of a VGG-16 at batch 32
+    for kind, dt in (("f32", torch.float32), ("bf16", torch.bfloat16)):
+        x = torch.clamp_min(torch.randn(32, 64, 224, 224, device=dev, generator=torch.Generator(device=dev).manual_seed(900)), 0).to(dt)
+        no, es = x.numel() // 4, x.element_size()
+        y = torch.empty(32, 64, 112, 112, dtype=dt, device=dev)
+        codes = torch.empty((no + 15) // 16, dtype=torch.int32, device=dev)
+        gin = torch.empty_like(x)
+        by = 5 * no * es + 4 * ((no + 15) // 16)
+        pooled_bitmap = torch.randint(-2 ** 31, 2 ** 31 - 1, ((no + 31) // 32,), dtype=torch.int32, device=dev)
+        for op, fn in (("bt_maxpool2x2_fwd", lambda: B.bt_maxpool2x2_fwd(x, y, codes)),
+                       ("bt_maxpool2x2_bwd", lambda: B.bt_maxpool2x2_bwd(codes, y, gin)),
+                       ("bt_maxpool2x2_bwd_masked", lambda: B.bt_maxpool2x2_bwd_masked(codes, pooled_bitmap, y, gin))):
+            T.row("next", op, kind, None, x.numel(), by, T.time(fn), tensor="32x64x224x224")
+        del x, y, codes, gin, pooled_bitmap
+        torch.cuda.empty_cache()
 
 
 # ------------------------------------------------------------------------------------------
