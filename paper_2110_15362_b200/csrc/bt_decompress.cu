@@ -16,6 +16,7 @@
 #include <type_traits>
 
 #include "bt_internal.cuh"
+#include "bt_quarter16.cuh"
 
 namespace bt {
 namespace {
@@ -57,9 +58,9 @@ struct RestoreParams {
 };
 
 // `block`: index of this CTA among those that restore the tensor
-template <typename U, int kE, int kGrp, int kWarps, int WIDEN = 0>
+template <typename U, int kE, int kGrp, int kWarps>
 __device__ __forceinline__ void
-decompress_body(const uint32_t *__restrict__ bitmap, const std::conditional_t<WIDEN != 0, uint16_t, U> *values,
+decompress_body(const uint32_t *__restrict__ bitmap, const U *values,
                 const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
                 U *__restrict__ out, const uint64_t block)
 {
@@ -83,7 +84,7 @@ decompress_body(const uint32_t *__restrict__ bitmap, const std::conditional_t<WI
     const uint4 w4 = load_words4(bitmap, w0, words_total);
     const uint64_t chunk_base = prefix[chunk];
     // arena form: the packed values start *values_offset bytes into `values`
-    using V = std::conditional_t<WIDEN != 0, uint16_t, U>;   // type of a stashed value
+    using V = U;
     if (values_offset) values = reinterpret_cast<const V *>(reinterpret_cast<const unsigned char *>(values) + *values_offset);
 
     // non-zeros of the chunk in front of this quarter
@@ -128,8 +129,7 @@ decompress_body(const uint32_t *__restrict__ bitmap, const std::conditional_t<WI
 #pragma unroll
         for (int j = 0; j < kE; ++j) {
             const bool set = (bits >> j) & 1u;
-            if constexpr (WIDEN != 0) e[kk][j] = set ? widened<WIDEN>(vp[off]) : 0u;
-            else e[kk][j] = set ? vp[off] : U(0);
+            e[kk][j] = set ? vp[off] : U(0);
             off += set;
         }
     }
@@ -164,148 +164,76 @@ decompress_body(const uint32_t *__restrict__ bitmap, const std::conditional_t<WI
 }
 
 // ---------------------------------------------------------------------------------------------
-// The decompressor for 2-byte elements.  The gather of the kernel above issues one global load and a 64-bit
-// address computation per element, which makes a 2-byte element cost as many instructions as a 4-byte one: on a
-// tensor of 2-byte elements that kernel is bound by the integer pipes at 0.74 of the copy bandwidth.  Here the
-// warp first brings its quarter's packed run into shared memory with 16-byte loads (the run starts wherever its
-// rank puts it: the 16-byte vectors that cover it are copied whole, the last one element by element so that
-// nothing behind the caller's values is read), and the gather reads shared memory: a test of the element's bit,
-// a 2-byte shared load, a select, a predicated 32-bit add.
-__device__ __forceinline__ uint4 ldg_vec_stream(const uint4 *p)
-{
-    uint4 v;
-    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-}
-
-// Four consecutive elements under the four low bits of `bits`: for every set bit the next 2-byte value at shared
-// address `a` (which moves on), +0 for a clear bit; packed two to a word.
-__device__ __forceinline__ uint2 expand4_u16(uint32_t a, const uint32_t bits)
-{
-    uint2 r;
-#define BT_PAIR(OUT, B0, B1)                                                                                         \
-    "and.b32 t, %3, " #B0 ";\n\tsetp.ne.u32 p, t, 0;\n\tld.shared.u16 lo, [%2];\n\tselp.b32 lo, lo, 0, p;\n\t@p add.u32 %2, %2, 2;\n\t" \
-    "and.b32 t, %3, " #B1 ";\n\tsetp.ne.u32 p, t, 0;\n\tld.shared.u16 hi, [%2];\n\tselp.b32 hi, hi, 0, p;\n\t@p add.u32 %2, %2, 2;\n\t" \
-    "prmt.b32 " OUT ", lo, hi, 0x5410;\n\t"
-    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 t, lo, hi;\n\t" BT_PAIR("%0", 1, 2) BT_PAIR("%1", 4, 8) "}" : "=r"(r.x), "=r"(r.y), "+r"(a) : "r"(bits));
-#undef BT_PAIR
-    return r;
-}
-
-template <int kWarps>
+// The decompressor for 2-byte elements: the quarter's packed run staged in shared memory, expanded from there
+// (bt_quarter16.cuh).  WIDEN: 0 restores 2-byte elements; 1 (binary16) / 2 (bfloat16) widens every restored value
+// to binary32 on its way out.
+template <int kWarps, int WIDEN = 0>
 __device__ __forceinline__ void
 decompress16_body(const uint32_t *__restrict__ bitmap, const uint16_t *values, const uint64_t *__restrict__ values_offset,
-                  const uint64_t *__restrict__ prefix, const uint64_t n, uint16_t *__restrict__ out, const uint64_t block)
+                  const uint64_t *__restrict__ prefix, const uint64_t n,
+                  std::conditional_t<WIDEN != 0, uint32_t, uint16_t> *__restrict__ out, const uint64_t block)
 {
-    // a quarter's run (at most 1024 values) behind up to 14 bytes of its first vector, whole vectors
-    __shared__ __align__(16) unsigned char s_run[kWarps][2048 + 32];
-
-    const uint32_t lane        = threadIdx.x & 31u;
-    const uint32_t wic         = threadIdx.x >> 5;
-    const uint64_t warp_global = block * kWarps + wic;
-    const uint64_t quarters    = (n + 1023) >> 10;
-    if (warp_global >= quarters) return;
-
-    const uint64_t chunk       = warp_global >> 2;
-    const uint32_t q           = static_cast<uint32_t>(warp_global & 3u);
-    const uint64_t words_total = (n + 31) >> 5;
-    const uint64_t w0          = chunk * 128 + 4 * lane;   // this lane's four words of the chunk
-
-    // the chunk's 128 words (zero past the end of the bitmap) and its prefix entry: independent loads
-    uint32_t c4[4] = {0, 0, 0, 0};
-    if (w0 + 3 < words_total && (reinterpret_cast<uintptr_t>(bitmap) & 15u) == 0) {
-        const uint4 w4 = *reinterpret_cast<const uint4 *>(bitmap + w0);
-        c4[0] = w4.x, c4[1] = w4.y, c4[2] = w4.z, c4[3] = w4.w;
-    } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (w0 + j < words_total) c4[j] = bitmap[w0 + j];
-    }
-    const uint64_t chunk_base = prefix[chunk];
-    if (values_offset) values = reinterpret_cast<const uint16_t *>(reinterpret_cast<const unsigned char *>(values) + *values_offset);
-
-    // non-zeros of the chunk in front of this quarter
-    uint32_t before = lane < 8 * q ? __popc(c4[0]) + __popc(c4[1]) + __popc(c4[2]) + __popc(c4[3]) : 0u;
-    before          = __reduce_add_sync(kFull, before);
-    // lane l takes word l of its own quarter: component l & 3 of lane 8q + (l >> 2)
-    const int      from_lane = 8 * q + (lane >> 2);
-    const uint32_t x0 = __shfl_sync(kFull, c4[0], from_lane), x1 = __shfl_sync(kFull, c4[1], from_lane);
-    const uint32_t x2 = __shfl_sync(kFull, c4[2], from_lane), x3 = __shfl_sync(kFull, c4[3], from_lane);
-    const uint32_t word = (lane & 2u) ? ((lane & 1u) ? x3 : x2) : ((lane & 1u) ? x1 : x0);
-    uint32_t       incl = __popc(word);
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t u = __shfl_up_sync(kFull, incl, o);
-        if (lane >= static_cast<uint32_t>(o)) incl += u;
-    }
-    const uint32_t excl = incl - __popc(word);
-    const uint32_t cnt  = __shfl_sync(kFull, incl, 31);      // values of this quarter
-
-    // ---- the run into shared memory
-    const uint16_t *const src   = values + (chunk_base + before);
-    const uint32_t        shift = static_cast<uint32_t>(reinterpret_cast<uintptr_t>(src) & 15u);         // bytes
-    const uint32_t        bytes = shift + 2u * cnt;                                                      // of the staging area in use
-    const uint32_t        stage = smem_addr(&s_run[wic][0]);
-    if (cnt) {
-        const uint4 *const gv   = reinterpret_cast<const uint4 *>(reinterpret_cast<const unsigned char *>(src) - shift);
-        const uint32_t     full = bytes >> 4;                                                            // whole vectors
-        // all loads first (at most five vectors per lane), then the stores: one round trip, not one per vector
-        uint4 v[5];
-#pragma unroll
-        for (int k = 0; k < 5; ++k)
-            if (lane + 32u * k < full) v[k] = ldg_vec_stream(gv + lane + 32u * k);
-#pragma unroll
-        for (int k = 0; k < 5; ++k)
-            if (lane + 32u * k < full)
-                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(stage + 16u * (lane + 32u * k)), "r"(v[k].x), "r"(v[k].y), "r"(v[k].z), "r"(v[k].w) : "memory");
-        // the elements of the last, partial vector one by one
-        const uint32_t tail0 = full * 16u > shift ? full * 16u : shift;
-        for (uint32_t b = tail0 + 2u * lane; b < bytes; b += 64u)
-            s_run[wic][b] = reinterpret_cast<const unsigned char *>(gv)[b], s_run[wic][b + 1] = reinterpret_cast<const unsigned char *>(gv)[b + 1];
-    }
-    __syncwarp();
-
-    // ---- expand: a lane owns 4 consecutive elements, i.e. 4 consecutive bits of one word, per step.  (With 8 per
-    // lane the 32 lanes of one shared load reach over 256 bytes of the run and every load takes two passes:
-    // 0.131 ms instead of 0.126 on 205 M elements; with 2 per lane the shuffles and stores double: 0.153 ms.)
-    const uint64_t e0    = warp_global << 10;
-    const bool     whole = e0 + 1024 <= n;
-    const Extent   ox    = extent_of(out, n * sizeof(uint16_t));
+    q16::Quarter qt;
+    if (!q16::stage_quarter<kWarps>(bitmap, values, values_offset, prefix, n, block, qt)) return;
+    const uint32_t lane = threadIdx.x & 31u;
+    const Extent   ox   = extent_of(out, n * sizeof(*out));
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const int      from = k * 4 + (lane >> 3);
-        const uint32_t w    = __shfl_sync(kFull, word, from);
-        const uint32_t wex  = __shfl_sync(kFull, excl, from);
-        const uint32_t sh   = (lane & 7u) * 4u;
-        const uint32_t off  = wex + __popc(w & ((1u << sh) - 1u));
-        const uint2    v    = expand4_u16(stage + shift + 2u * off, w >> sh);
-        const uint64_t at   = e0 + static_cast<uint64_t>(k) * 128 + lane * 4;
-        if (whole || at + 4 <= n) {
-            if (ox.holds(out + at, 8)) *reinterpret_cast<uint2 *>(out + at) = v;
-        } else {
-            const uint32_t h[2] = {v.x, v.y};
+        uint32_t       bits;
+        const uint2    v  = q16::expand_step(qt, k, lane, bits);
+        const uint64_t at = qt.e0 + static_cast<uint64_t>(k) * 128 + lane * 4;
+        if constexpr (WIDEN == 0) {
+            if (qt.whole || at + 4 <= n) {
+                if (ox.holds(out + at, 8)) *reinterpret_cast<uint2 *>(out + at) = v;
+            } else {
+                const uint32_t h[2] = {v.x, v.y};
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (at + j < n && ox.holds(out + at + j, 2)) out[at + j] = static_cast<uint16_t>(h[j >> 1] >> (16 * (j & 1)));
+                for (int j = 0; j < 4; ++j)
+                    if (at + j < n && ox.holds(out + at + j, 2)) out[at + j] = static_cast<uint16_t>(h[j >> 1] >> (16 * (j & 1)));
+            }
+        } else {
+            // a clear bit gave the pattern 0, which widens to +0
+            uint32_t f[4];
+            if constexpr (WIDEN == 2) {
+                f[0] = v.x << 16, f[1] = v.x & 0xFFFF0000u, f[2] = v.y << 16, f[3] = v.y & 0xFFFF0000u;
+            } else {
+                f[0] = widened<WIDEN>(static_cast<uint16_t>(v.x)), f[1] = widened<WIDEN>(static_cast<uint16_t>(v.x >> 16));
+                f[2] = widened<WIDEN>(static_cast<uint16_t>(v.y)), f[3] = widened<WIDEN>(static_cast<uint16_t>(v.y >> 16));
+            }
+            if (qt.whole || at + 4 <= n) {
+                if (ox.holds(out + at, 16)) *reinterpret_cast<uint4 *>(out + at) = make_uint4(f[0], f[1], f[2], f[3]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (at + j < n && ox.holds(out + at + j, 4)) out[at + j] = f[j];
+            }
         }
     }
 }
 
-template <typename U, int kE, int kGrp, int kWarps, int WIDEN = 0>
+template <typename U, int kE, int kGrp, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32)
-decompress_kernel(const uint32_t *__restrict__ bitmap, const std::conditional_t<WIDEN != 0, uint16_t, U> *values,
+decompress_kernel(const uint32_t *__restrict__ bitmap, const U *values,
                   const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint64_t n,
                   U *__restrict__ out)
 {
-    decompress_body<U, kE, kGrp, kWarps, WIDEN>(bitmap, values, values_offset, prefix, n, out, blockIdx.x);
+    decompress_body<U, kE, kGrp, kWarps>(bitmap, values, values_offset, prefix, n, out, blockIdx.x);
 }
 
 template <int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 2048 / (kWarps * 32))
+__global__ void __launch_bounds__(kWarps * 32, 1536 / (kWarps * 32))
 decompress16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values, const uint64_t *__restrict__ values_offset,
                     const uint64_t *__restrict__ prefix, const uint64_t n, uint16_t *__restrict__ out)
 {
     decompress16_body<kWarps>(bitmap, values, values_offset, prefix, n, out, blockIdx.x);
+}
+
+template <int kWarps, int WIDEN>
+__global__ void __launch_bounds__(kWarps * 32, 1536 / (kWarps * 32))
+decompress16_widen_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *values, const uint64_t *__restrict__ values_offset,
+                          const uint64_t *__restrict__ prefix, const uint64_t n, uint32_t *__restrict__ out)
+{
+    decompress16_body<kWarps, WIDEN>(bitmap, values, values_offset, prefix, n, out, blockIdx.x);
 }
 
 // The tensor a CTA of a batched launch works on: the last job whose first block is not behind this one.
@@ -324,12 +252,12 @@ __global__ void __launch_bounds__(kWarps * 32)
 decompress_batch_kernel(const __grid_constant__ RestoreParams<kJobs> p)
 {
     const RestoreJob &j = p.job[job_of_block(p)];
-    decompress_body<U, kE, kGrp, kWarps, 0>(j.bitmap, static_cast<const U *>(j.values), j.values_offset, j.prefix, j.n, static_cast<U *>(j.out),
+    decompress_body<U, kE, kGrp, kWarps>(j.bitmap, static_cast<const U *>(j.values), j.values_offset, j.prefix, j.n, static_cast<U *>(j.out),
                                             blockIdx.x - j.first_block);
 }
 
 template <int kWarps, int kJobs>
-__global__ void __launch_bounds__(kWarps * 32, 2048 / (kWarps * 32))
+__global__ void __launch_bounds__(kWarps * 32, 1536 / (kWarps * 32))
 decompress16_batch_kernel(const __grid_constant__ RestoreParams<kJobs> p)
 {
     const RestoreJob &j = p.job[job_of_block(p)];
@@ -361,10 +289,9 @@ cudaError_t launch_decompress_widen(const uint32_t *bitmap, const void *values16
     if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     const auto *v = static_cast<const uint16_t *>(values16);
     auto       *o = static_cast<uint32_t *>(out_f32);
-    if (from_dtype == BT_F16)
-        decompress_kernel<uint32_t, 4, 8, kWarps, 1><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, values_offset, prefix, n, o);
-    else
-        decompress_kernel<uint32_t, 4, 8, kWarps, 2><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, values_offset, prefix, n, o);
+    // the 2-byte decompressor (packed run staged in shared memory) with the widening in its store path
+    if (from_dtype == BT_F16) decompress16_widen_kernel<kWarps, 1><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, values_offset, prefix, n, o);
+    else decompress16_widen_kernel<kWarps, 2><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(bitmap, v, values_offset, prefix, n, o);
     return cudaGetLastError();
 }
 

@@ -13,6 +13,7 @@
 // costs registers and with them occupancy: measured 20 to 45 % slower), all four
 // for 2-byte elements (measured faster than two).
 #include "bt_internal.cuh"
+#include "bt_quarter16.cuh"
 
 namespace bt {
 namespace {
@@ -148,6 +149,74 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     }
 }
 
+// 2-byte elements: the quarter's packed run staged in shared memory and gathered from there (bt_quarter16.cuh)
+// instead of one global gather per value.  The quarter's gradient -- eight 8-byte loads per lane that do not
+// depend on the stash -- is requested first, so that it arrives while the run is staged.
+template <int DT, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1024 / (kWarps * 32))
+relu6_bwd16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ values,
+                   const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint16_t *gout,
+                   const uint64_t n, uint16_t *gin)   // gin may alias gout
+{
+    const uint32_t lane        = threadIdx.x & 31u;
+    const uint64_t warp_global = static_cast<uint64_t>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    if (warp_global >= ((n + 1023) >> 10)) return;
+    const uint64_t e0 = warp_global << 10;
+    uint2          g[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const uint64_t at = e0 + static_cast<uint64_t>(k) * 128 + lane * 4;
+        if (at + 4 <= n) {
+            g[k] = *reinterpret_cast<const uint2 *>(gout + at);
+        } else {
+            uint32_t h[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) h[j] = at + j < n ? gout[at + j] : 0u;
+            g[k] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+        }
+    }
+    q16::Quarter qt;
+    if (!q16::stage_quarter<kWarps>(bitmap, values, values_offset, prefix, n, blockIdx.x, qt)) return;
+    const Extent ox = extent_of(gin, n * sizeof(uint16_t));
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        uint32_t    bits;
+        const uint2 v = q16::expand_step(qt, k, lane, bits);
+        // the gradient passes where the bit is set and the stashed value is below 6 (false for a stored 6 and for a NaN)
+        const uint32_t h[4] = {v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16};
+        uint32_t       keep[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bool pass = ((bits >> j) & 1u) && Elem<DT>::widen(h[j]) < 6.0f;
+            keep[j]         = pass ? 0xFFFFu : 0u;
+        }
+        const uint2    r  = make_uint2(g[k].x & (keep[0] | (keep[1] << 16)), g[k].y & (keep[2] | (keep[3] << 16)));
+        const uint64_t at = e0 + static_cast<uint64_t>(k) * 128 + lane * 4;
+        if (qt.whole || at + 4 <= n) {
+            if (ox.holds(gin + at, 8)) *reinterpret_cast<uint2 *>(gin + at) = r;
+        } else {
+            const uint32_t o[2] = {r.x, r.y};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (at + j < n && ox.holds(gin + at + j, 2)) gin[at + j] = static_cast<uint16_t>(o[j >> 1] >> (16 * (j & 1)));
+        }
+    }
+}
+
+template <int DT>
+cudaError_t launch_16(const uint32_t *bitmap, const void *values, const uint64_t *values_offset, const uint64_t *prefix,
+                      const void *gout, uint64_t n, void *gin, cudaStream_t stream)
+{
+    constexpr int  kWarps   = 4;
+    const uint64_t quarters = (n + 1023) >> 10;
+    const uint64_t grid     = (quarters + kWarps - 1) / kWarps;
+    if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    relu6_bwd16_kernel<DT, kWarps><<<static_cast<unsigned>(grid), kWarps * 32, 0, stream>>>(
+        bitmap, static_cast<const uint16_t *>(values), values_offset, prefix, static_cast<const uint16_t *>(gout), n,
+        static_cast<uint16_t *>(gin));
+    return cudaGetLastError();
+}
+
 template <typename U, int DT, int kE, int kBlk>
 cudaError_t launch_typed(const uint32_t *bitmap, const void *values, const uint64_t *values_offset, const uint64_t *prefix,
                          const void *gout, uint64_t n, void *gin, cudaStream_t stream)
@@ -170,8 +239,8 @@ cudaError_t launch_relu6_bwd(const uint32_t *bitmap, const void *values, const u
     switch (dtype) {
     case BT_F64: return launch_typed<uint64_t, BT_F64, 2, 2>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
     case BT_F32: return launch_typed<uint32_t, BT_F32, 4, 2>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
-    case BT_F16: return launch_typed<uint16_t, BT_F16, 8, 4>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
-    default: return launch_typed<uint16_t, BT_BF16, 8, 4>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
+    case BT_F16: return launch_16<BT_F16>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
+    default: return launch_16<BT_BF16>(bitmap, values, values_offset, prefix, gout, n, gin, stream);
     }
 }
 
