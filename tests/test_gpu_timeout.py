@@ -95,3 +95,38 @@ def test_fused_and_batched_forms_time_out_cleanly(hooks, oracle):
         assert np.array_equal(W.raw_numpy(st.chunk_prefix).view(np.uint64), c.prefix)
         assert np.array_equal(W.raw_numpy(st.values[:c.nnz]), c.values)
         assert np.array_equal(y.raw(), y_ref) and y.guards_intact()
+
+
+def test_batched_arena_form_times_out_cleanly(hooks, oracle):
+    """The batched arena form has one more wait (a tensor's place in the arena comes from the tensor before it):
+    under a limit of a few nanoseconds the launch gives up by itself, and the next ordinary launch on the same
+    workspace and arena is the oracle's."""
+    sizes = [8192 * 200 + 5, 8192 * 150, 4097, 8192 * 170 + 1]
+    raws = [W.random_patterns(n, "f32", 0.5, seed=90 + i) for i, n in enumerate(sizes)]
+    xs = [from_raw(r, "f32") for r in raws]
+    stashes = [B.Stash(n, torch.float32, "cuda", values_capacity=1) for n in sizes]
+    items = B.batch_items(xs, stashes)
+    arena = Guarded(sum(sizes), torch.float32)
+    cursor = torch.zeros(1, dtype=torch.int64, device="cuda")
+    offsets = torch.zeros(len(sizes), dtype=torch.int64, device="cuda")
+    ws = torch.empty(B.bt_batch_workspace_bytes(sizes), dtype=torch.uint8, device="cuda")
+
+    hooks.bt_test_set_wait_ns(30)
+    t0 = time.perf_counter()
+    rc = B.bt_compress_arena_batch(items, torch.float32, arena.inner.view(torch.uint8), cursor, offsets, ws, check=False)
+    torch.cuda.synchronize()
+    assert rc == B.BT_OK and time.perf_counter() - t0 < 1.0
+    assert stashes[0].status == B.BT_ERR_TIMEOUT and arena.guards_intact()
+
+    hooks.bt_test_set_wait_ns(2_000_000_000)
+    cursor.zero_()
+    B.bt_compress_arena_batch(items, torch.float32, arena.inner.view(torch.uint8), cursor, offsets, ws)
+    torch.cuda.synchronize()
+    at = 0
+    raw_arena = arena.inner.view(torch.uint8)
+    for k, raw in enumerate(raws):
+        c = oracle.compress(raw)
+        assert stashes[k].status == B.BT_OK and stashes[k].nnz == c.nnz and int(offsets[k].item()) == at
+        assert np.array_equal(raw_arena[at:at + 4 * c.nnz].cpu().numpy().view(np.uint32), c.values)
+        at += (4 * c.nnz + 15) // 16 * 16
+    assert int(cursor.item()) == at and arena.guards_intact()
