@@ -57,6 +57,7 @@ def check_against_torch(st: B.Stash, y: torch.Tensor):
     mask = bits_of(y) != 0
     nnz = int(mask.sum().item())
     assert st.status == B.BT_OK and st.nnz == nnz
+    assert not hasattr(st, "intact") or st.intact()          # nothing written outside the stash's buffers
     assert torch.equal(st.bitmap, torch_bitmap(mask))
     assert torch.equal(st.chunk_prefix, torch_prefix(mask))
     assert torch.equal(bits_of(st.values[:nnz]), bits_of(y)[mask])
@@ -91,7 +92,7 @@ def check_sampled_chunks(oracle, st: B.Stash, y: torch.Tensor, restored, seed: i
 
 def compress(x, ws=None):
     n = x.numel()
-    st = B.Stash(n, x.dtype, DEV)
+    st = GStash(n, x.dtype, DEV)
     B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws if ws is not None else B.new_workspace(n, DEV),
                   st.dev_status)
     return st
@@ -101,6 +102,20 @@ def decompress(st, like):
     out = torch.empty_like(like)
     B.bt_decompress(st.bitmap, st.values, st.chunk_prefix, out)
     return out
+
+
+class GStash(B.Stash):
+    """B.Stash with every buffer between canary regions (same attributes, plus intact())."""
+
+    def __init__(self, n, dtype, device=DEV, values_capacity=None):
+        self.n, self.dtype = n, dtype
+        cap = n if values_capacity is None else values_capacity
+        self._g = [Guarded((n + 31) // 32, torch.int32), Guarded(cap, dtype), Guarded((n + 4095) // 4096, torch.int64),
+                   Guarded(1, torch.int64), Guarded(1, torch.int32)]
+        self.bitmap, self.values, self.chunk_prefix, self.nnz_out, self.dev_status = (g.inner for g in self._g)
+
+    def intact(self):
+        return all(g.guards_intact() for g in self._g)
 
 
 class GuardedStash:
@@ -242,12 +257,12 @@ def test_cfg4_vgg16_batch64_fused_relu_pair(oracle, kind):
         y_ref = (torch.relu(pre) + 0.0).to(pre.dtype)        # +0.0: torch.relu keeps the sign of -0.0
         ws = B.new_workspace(n, DEV)
         # stash only
-        st = B.Stash(n, pre.dtype, DEV)
+        st = GStash(n, pre.dtype, DEV)
         B.bt_relu_fwd_compress(pre, None, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
         check_against_torch(st, y_ref)
         check_sampled_chunks(oracle, st, y_ref, None, seed=40 + i, samples=12)
         # with the dense output
-        st2 = B.Stash(n, pre.dtype, DEV)
+        st2 = GStash(n, pre.dtype, DEV)
         y = torch.empty_like(pre)
         B.bt_relu_fwd_compress(pre, y, st2.bitmap, st2.values, st2.chunk_prefix, st2.nnz_out, ws, st2.dev_status)
         assert torch.equal(bits_of(y), bits_of(y_ref))
@@ -270,10 +285,10 @@ def test_cfg5_mobilenetv2_batch128_forward_then_reverse(oracle):
     stashes, nnzs, total_bytes = [], [], 0
     for i, shape, n in W.iter_layers(shapes):                 # forward order, one stream
         x = W.cfg5_layer(i, shape, fractions[i], DEV).reshape(-1)
-        st = B.Stash(n, x.dtype, DEV, values_capacity=n)
+        st = GStash(n, x.dtype, DEV, values_capacity=n)
         B.bt_compress(x, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
         nnz = int((bits_of(x) != 0).sum().item())
-        assert st.nnz == nnz and st.status == B.BT_OK
+        assert st.nnz == nnz and st.status == B.BT_OK and st.intact()
         assert abs((1 - nnz / n) - fractions[i]) < 0.02
         if i % 6 == 0:
             check_sampled_chunks(oracle, st, x, None, seed=70 + i, samples=8)
@@ -308,12 +323,12 @@ def test_more_than_two_to_the_32_elements(oracle):
         m = min(step, n - lo)
         pre[lo:lo + m] = torch.randn(m, generator=torch.Generator(device=DEV).manual_seed(9000 + k), device=DEV,
                                      dtype=torch.float32).to(torch.bfloat16)
-    st = B.Stash(n, pre.dtype, DEV)
+    st = GStash(n, pre.dtype, DEV)
     ws = B.new_workspace(n, DEV)
     y = torch.empty_like(pre)
     B.bt_relu_fwd_compress(pre, y, st.bitmap, st.values, st.chunk_prefix, st.nnz_out, ws, st.dev_status)
     torch.cuda.synchronize()
-    assert st.status == B.BT_OK
+    assert st.status == B.BT_OK and st.intact()
     nnz = st.nnz
     # whole tensor, slice by slice: the dense output, the bitmap, the prefix array and the packed values
     total = 0
@@ -340,7 +355,7 @@ def test_more_than_two_to_the_32_elements(oracle):
         assert np.array_equal(W.raw_numpy(st.bitmap[lo // 32:(hi + 31) // 32]).view(np.uint32), ref.bitmap)
         assert np.array_equal(W.raw_numpy(st.values[start:start + ref.nnz]), ref.values)
     # the plain compressor on y gives the same stash
-    st2 = B.Stash(n, pre.dtype, DEV)
+    st2 = GStash(n, pre.dtype, DEV)
     B.bt_compress(y, st2.bitmap, st2.values, st2.chunk_prefix, st2.nnz_out, ws, st2.dev_status)
     assert st2.status == B.BT_OK and st2.nnz == nnz
     assert torch.equal(st2.bitmap, st.bitmap) and torch.equal(st2.chunk_prefix, st.chunk_prefix)
