@@ -45,7 +45,7 @@ LOG2N = 28
 ZEROS = 0.5
 NOMINAL_GBS = 8000.0
 CASE_OPS = ("compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd", "decompress", "relu_bwd", "mask",
-            "mask_y", "maxpool", "maxpool_bwd", "widen")
+            "mask_y", "maxpool", "maxpool_bwd", "widen", "batch", "batch_restore")
 
 # DRAM bytes (read + write) per element of a kernel, from one ncu capture of
 #   python bench.py --case <dtype> <op> --log2n <26 for 4-byte, 27 for 2-byte elements>
@@ -813,6 +813,21 @@ def run_case(args) -> int:
     if kind not in ("f32", "f16", "bf16", "f64") or op not in CASE_OPS:
         raise SystemExit("--case <f32|f16|bf16|f64> <%s>" % "|".join(CASE_OPS))
     dev = torch.device("cuda")
+    if op in ("batch", "batch_restore"):                                 # the 17 ResNet-18 layers at batch 32, one launch
+        tdt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16, "f64": torch.float64}[kind]
+        acts = [torch.clamp_min(W.cfg2_preact(i, shape, dev), 0.0).reshape(-1).to(tdt) for i, shape, _ in W.iter_layers(W.resnet18_shapes(32))]
+        sts = [B.Stash(a.numel(), tdt, dev) for a in acts]
+        outs = [torch.empty_like(a) for a in acts]
+        ws = torch.empty(B.bt_batch_workspace_bytes([a.numel() for a in acts]), dtype=torch.uint8, device=dev)
+        items, ritems = B.batch_items(acts, sts), B.batch_items(outs[::-1], sts[::-1], outs[::-1])
+        for _ in range(args.reps):
+            B.bt_compress_batch(items, tdt, ws)
+            if op == "batch_restore":
+                B.bt_decompress_batch(ritems, tdt)
+        torch.cuda.synchronize()
+        ok = all(st.status == B.BT_OK for st in sts) and (op == "batch" or all(torch.equal(o, a) for o, a in zip(outs, acts)))
+        print("tensors", len(acts), "nnz", sum(st.nnz for st in sts), "ok", ok)
+        return 0 if ok else 1
     n = 1 << args.log2n
     if kind == "f32":
         x = W.prune_preact(n, dev) if op == "prune" else W.cfg3_iid(n, args.zeros, 2, dev)
