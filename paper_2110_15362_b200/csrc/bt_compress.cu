@@ -534,10 +534,12 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStr
             return y ? launch_typed<uint64_t, k6 + BT_F64, true>(a, stream) : launch_typed<uint64_t, k6 + BT_F64, false>(a, stream);
         case BT_F32:
             return y ? launch_typed<uint32_t, k6 + BT_F32, true>(a, stream) : launch_typed<uint32_t, k6 + BT_F32, false>(a, stream);
+        // 2-byte types: with the dense output the decisions are taken on the bit pattern (0.1925 -> 0.1864 ms on the
+        // 392 MiB tensor); without it the float compares measured faster (0.182 against 0.192 ms), as for the ReLU
         case BT_F16:
-            return y ? launch_typed<uint16_t, k6 + BT_F16, true>(a, stream) : launch_typed<uint16_t, k6 + BT_F16, false>(a, stream);
+            return y ? launch_typed<uint16_t, kFusedRelu6Bits + BT_F16, true>(a, stream) : launch_typed<uint16_t, k6 + BT_F16, false>(a, stream);
         default:
-            return y ? launch_typed<uint16_t, k6 + BT_BF16, true>(a, stream)
+            return y ? launch_typed<uint16_t, kFusedRelu6Bits + BT_BF16, true>(a, stream)
                      : launch_typed<uint16_t, k6 + BT_BF16, false>(a, stream);
         }
     }

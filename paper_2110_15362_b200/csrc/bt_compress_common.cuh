@@ -172,6 +172,7 @@ __device__ __forceinline__ uint32_t compact_segment(const uint32_t seg_addr, uin
             bool   nz;
             if constexpr (RELU_DT >= kFusedReluBits) {
                 nz = relu_keeps_bits<RELU_DT & 3>(x);        // a kept element is never the zero pattern
+                if constexpr (RELU_DT >= kFusedRelu6Bits) x = relu6_saturates_bits<RELU_DT & 3>(x) ? Elem<RELU_DT & 3>::kSix : x;
                 if constexpr (WRITE_Y) {
                     const uint32_t e = (kb + j) * 32 + lane;
                     if ((!kGuardY || e < yvalid) && yx.holds(y + e, sizeof(U))) y[e] = nz ? static_cast<U>(x) : U(0);

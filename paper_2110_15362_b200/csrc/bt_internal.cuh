@@ -373,8 +373,9 @@ __device__ __forceinline__ uint32_t greater_or_nan(double v, double b)
 // The fused forward forms are numbered by one template argument: -1 none (plain compressor), DT (0..3) keep
 // what exceeds the threshold (tau = 0: ReLU), 4 + DT ReLU6, 8 + DT (2-byte types only) the ReLU decided on the
 // bit pattern.
-constexpr int kFusedRelu6    = 4;
-constexpr int kFusedReluBits = 8;
+constexpr int kFusedRelu6     = 4;
+constexpr int kFusedReluBits  = 8;
+constexpr int kFusedRelu6Bits = 12;    // 12 + DT: ReLU6 of a 2-byte type decided on the bit pattern
 
 // ReLU of a 2-byte element without widening it: x, the element's pattern sign-extended to 32 bits, is kept iff
 // it is a positive number, +inf or a NaN of either sign -- exactly the elements for which x <= 0 is false under
@@ -386,6 +387,16 @@ __device__ __forceinline__ bool relu_keeps_bits(const uint32_t x)
     static_assert(DT == BT_F16 || DT == BT_BF16, "2-byte element types");
     constexpr uint32_t kMinusInf = DT == BT_F16 ? 0xFFFFFC00u : 0xFFFFFF80u;
     return (static_cast<int32_t>(x) > 0) | (x > kMinusInf);      // no short circuit: two compares, no branch
+}
+
+// x >= 6 for the same sign-extended pattern: the positive numbers from 6 up to +inf are the integers from 6's
+// pattern to +inf's (a positive NaN lies above +inf's pattern, a negative pattern is a negative integer).
+template <int DT>
+__device__ __forceinline__ bool relu6_saturates_bits(const uint32_t x)
+{
+    static_assert(DT == BT_F16 || DT == BT_BF16, "2-byte element types");
+    constexpr int32_t kInf = DT == BT_F16 ? 0x7C00 : 0x7F80;
+    return (static_cast<int32_t>(x) >= static_cast<int32_t>(Elem<DT>::kSix)) & (static_cast<int32_t>(x) <= kInf);
 }
 
 // y = (x <= tau) ? +0 : x, and for ReLU6 additionally 6 where x >= 6; IEEE comparisons, so a NaN is kept.
