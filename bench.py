@@ -657,44 +657,55 @@ class Batch:
         return nnz
 
 
-def run_e2e(batch: Batch, steps: int = 4, warmup: int = 1):
-    """The same four operations on one tensor of the batch through the host-buffer entry points of the C ABI: the
-    tensor, its pre-activation and the gradient start in pinned host memory, both stashes, the restored tensor and
-    the input gradient end there; the host<->device copies happen inside the calls, inside the timed region."""
+def run_e2e(batch: Batch, steps: int = 3, warmup: int = 1, workers: int = 4):
+    """The same four operations through the host-buffer entry points of the C ABI: a tensor, its pre-activation and
+    the gradient start in pinned host memory, both stashes, the restored tensor and the input gradient end there;
+    the host<->device copies happen inside the calls, inside the timed region.
+
+    The calls are synchronous (each returns with its results on the host), so `workers` host threads, each with its
+    own stream, staging area and output buffers, work on one tensor each at the same time: one call's upload
+    overlaps another's download.  A step is `workers` tensors through the four operations."""
+    from concurrent.futures import ThreadPoolExecutor
     import torch
     B, n, dev = batch.B, batch.n, batch.dev
     pin = lambda t: t.cpu().pin_memory()                                 # noqa: E731
-    h_x, h_pre, h_g = pin(batch.x[0]), pin(batch.pre[0]), pin(batch.g)
-    h_bitmap = torch.empty((n + 31) // 32, dtype=torch.int32).pin_memory()
-    h_values = torch.empty(n, dtype=torch.float32).pin_memory()
-    h_prefix = torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory()
-    h_nnz = torch.zeros(1, dtype=torch.int64).pin_memory()
-    h_back = torch.empty(n, dtype=torch.float32).pin_memory()
-    staging = torch.empty(B.bt_host_staging_bytes(n, torch.float32), dtype=torch.uint8, device=dev)
+    h_x, h_pre, h_g = pin(batch.x[0]), pin(batch.pre[0]), pin(batch.g)   # read-only inputs, shared by the workers
+    res = []
+    for _ in range(workers):
+        res.append(dict(stream=torch.cuda.Stream(device=dev),
+                        staging=torch.empty(B.bt_host_staging_bytes(n, torch.float32), dtype=torch.uint8, device=dev),
+                        bitmap=torch.empty((n + 31) // 32, dtype=torch.int32).pin_memory(),
+                        values=torch.empty(n, dtype=torch.float32).pin_memory(),
+                        prefix=torch.empty((n + 4095) // 4096, dtype=torch.int64).pin_memory(),
+                        nnz=torch.zeros(1, dtype=torch.int64).pin_memory(),
+                        back=torch.empty(n, dtype=torch.float32).pin_memory()))
 
-    def one():
-        B.bt_compress_host(h_x, h_bitmap, h_values, h_prefix, h_nnz, staging)
-        B.bt_decompress_host(h_bitmap, h_values, h_prefix, int(h_nnz.item()), h_back, staging)
-        B.bt_relu_fwd_compress_host(h_pre, None, h_bitmap, h_values, h_prefix, h_nnz, staging)
-        B.bt_relu_bwd_from_bitmap_host(h_bitmap, h_g, h_back, staging)
+    def one(r):
+        torch.cuda.set_device(dev)
+        s = r["stream"]
+        B.bt_compress_host(h_x, r["bitmap"], r["values"], r["prefix"], r["nnz"], r["staging"], stream=s)
+        B.bt_decompress_host(r["bitmap"], r["values"], r["prefix"], int(r["nnz"].item()), r["back"], r["staging"], stream=s)
+        B.bt_relu_fwd_compress_host(h_pre, None, r["bitmap"], r["values"], r["prefix"], r["nnz"], r["staging"], stream=s)
+        B.bt_relu_bwd_from_bitmap_host(r["bitmap"], h_g, r["back"], r["staging"], stream=s)
 
-    for _ in range(warmup):
-        one()
-    torch.cuda.synchronize()
-    nnz = int(h_nnz.item())
-    comp = B.bt_compressed_bytes(n, nnz, torch.float32)
-    h2d = 4 * n + comp + 4 * n + (4 * ((n + 31) // 32) + 4 * n)
-    d2h = (comp + 12) + 4 * n + (comp + 12) + 4 * n
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        one()
-    e1.record()
-    torch.cuda.synchronize()
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        for _ in range(warmup):
+            list(ex.map(one, res))
+        torch.cuda.synchronize()
+        nnz = int(res[0]["nnz"].item())
+        comp = B.bt_compressed_bytes(n, nnz, torch.float32)
+        h2d = workers * (4 * n + comp + 4 * n + (4 * ((n + 31) // 32) + 4 * n))
+        d2h = workers * ((comp + 12) + 4 * n + (comp + 12) + 4 * n)
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            list(ex.map(one, res))                                       # every call has synchronised its stream
+        torch.cuda.synchronize()
+        ms = (time.perf_counter() - t0) * 1e3 / steps
     want = torch.where(h_pre > 0, h_g, torch.zeros(()))
-    assert torch.equal(h_back.view(torch.int32), want.view(torch.int32)), "end-to-end result differs"
-    ms = e0.elapsed_time(e1) / steps
-    return {"ms_per_step": ms, "steps": steps, "h2d": h2d, "d2h": d2h, "dense_bytes_per_step": 4 * 4 * n}
+    for r in res:
+        assert torch.equal(r["back"].view(torch.int32), want.view(torch.int32)), "end-to-end result differs"
+    return {"ms_per_step": ms, "steps": steps, "h2d": h2d, "d2h": d2h, "dense_bytes_per_step": workers * 4 * 4 * n,
+            "workers": workers}
 
 
 def run_ours(args):
@@ -780,10 +791,11 @@ def run_ours(args):
             e = run_e2e(batch)
             line["e2e"] = {"value": round(world * e["dense_bytes_per_step"] / (e["ms_per_step"] * 1e-3) / 1e9, 3), "unit": UNIT,
                            "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"],
-                           "ms_per_step": round(e["ms_per_step"], 3), "steps": e["steps"],
-                           "what": "the step's four operations on one tensor of the batch through bt_*_host: pinned host "
-                                   "buffers in, pinned host buffers out, copies inside the calls (rank 0's GPU; "
-                                   "value scaled by the number of ranks)"}
+                           "ms_per_step": round(e["ms_per_step"], 3), "steps": e["steps"], "tensors_per_step": e["workers"],
+                           "what": "the step's four operations through bt_*_host on %d tensors at a time, one host thread, "
+                                   "stream and staging area each: pinned host buffers in, pinned host buffers out, copies "
+                                   "inside the calls, timed on the host around the synchronous calls (rank 0's GPU; value "
+                                   "scaled by the number of ranks)" % e["workers"]}
         if not args.no_cpu_baseline and world == 1:
             cal = host_sample(1 << 20)
             rate = (1 << 20) / max(oracle_four_ops(*cal), 1e-6)
