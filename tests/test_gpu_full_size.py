@@ -402,3 +402,14 @@ def test_the_benchmarks_own_step_against_the_oracle(oracle):
     B.bt_decompress(batch.sa.bitmap, batch.sa.values, batch.sa.chunk_prefix, batch.out)
     assert np.array_equal(W.raw_numpy(batch.out), oracle.decompress(c))
     assert B.bt_set_max_ctas(0) == 0                                    # the benchmark sets no CTA limit
+
+
+@pytest.mark.parametrize("kind,op", [("f32", "compress"), ("bf16", "relu"), ("bf16", "relu_y"), ("f16", "decompress"), ("f32", "relu_bwd"),
+                                     ("f32", "prune"), ("f32", "narrow"), ("f32", "widen"), ("bf16", "relu6_bwd"), ("f32", "mask_y"),
+                                     ("bf16", "maxpool_bwd"), ("f64", "compress"), ("f32", "batch_restore")])
+def test_the_profiling_cases_of_the_benchmark_run(kind, op):
+    """`python bench.py --case <dtype> <op>` is the command every summary under profiles/ names: each case runs to
+    the end and reports BT_OK (here on 2^20 elements)."""
+    import bench
+    args = bench.parse_args(["--case", kind, op, "--log2n", "20", "--reps", "2"])
+    assert bench.run_case(args) == 0
