@@ -181,3 +181,18 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "library_path", lambda: str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         B.lib()
+
+
+def test_test_hooks_exist_only_in_the_checking_builds(L):
+    """The product library exports no test hook; the two checking builds (tests/lib/, loaded by tests only) export
+    every symbol of the header plus their hook."""
+    import ctypes
+    from tests import checking_libs as C
+    for hook in ("bt_test_set_wait_ns", "bt_test_bounds_violations"):
+        assert not hasattr(L, hook), hook
+    for path, hook in ((C.HOOKS_PATH, "bt_test_set_wait_ns"), (C.BOUNDS_PATH, "bt_test_bounds_violations")):
+        C._build.build_library(out=path, extra_flags=C._FLAGS[path])      # a no-op when up to date
+        T = ctypes.CDLL(path)
+        assert hasattr(T, hook)
+        for name in B.EXPORTS:
+            assert hasattr(T, name), (path, name)
