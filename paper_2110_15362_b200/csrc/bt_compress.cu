@@ -48,11 +48,10 @@
 // descriptor carries the launch's 64-bit tag in both of its halves, and a reader
 // takes only descriptors with its own launch's tag; so counts are published and
 // read from the first tile on.  Only the wave totals, being sums, need zeroed
-// words: the last copier warp of every CTA zeroes a share of them and the grid
-// meets once at the barrier word of the cooperative launch; until that meeting
-// is over the scan warps park their contributions to totals in shared memory,
-// and the copier warp adds them afterwards.  A launch of one wave has no totals
-// and no meeting.
+// words: in the prologue every CTA zeroes a share of them and the grid meets
+// once (cooperative_groups::this_grid().sync()), the first two bulk copies
+// already on their way; nothing reads or adds to a total before that meeting.
+// A launch of one wave has no totals and no meeting.
 #include <cooperative_groups.h>
 
 #include <atomic>
@@ -68,18 +67,20 @@ using namespace cmp;
 // U: uint32_t (4-byte elements) or uint16_t (2-byte elements).
 // RELU_DT: -1 for the plain compressor, else the number of the fused forward form (element type, + 4 for ReLU6).
 // CAST: 0, or the 16-bit type the copiers narrow the packed binary32 values to (1 binary16, 2 bfloat16).
-// kWarps compactor warps and as many copier warps, kSeg elements per warp, kStages ring slots.
-template <typename U, int RELU_DT, bool WRITE_Y, int CAST, int kWarps, int kSeg, int kStages, int kCopiers>
-__global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
+// A tile is kWarps segments of kSeg elements; kCompactors compactor warps take the CTA's segments in turn
+// (segment g of the CTA's stream of tiles goes to warp g mod kCompactors; with kCompactors == kWarps warp w
+// simply owns segment w of every tile), kCopiers copier warps, kStages ring slots.
+template <typename U, int RELU_DT, bool WRITE_Y, int CAST, int kWarps, int kSeg, int kStages, int kCopiers, int kCompactors = kWarps>
+__global__ void __launch_bounds__((kCompactors + kCopiers + 3) * 32) compress_kernel(const CompressArgs a, const uint32_t num_tiles)
 {
     constexpr int kTile          = kWarps * kSeg;
     constexpr int kSteps         = kSeg / 32;
     constexpr int kChunksPerTile = kTile / BT_CHUNK_ELEMS;
     constexpr int kWarpsPerChunk = BT_CHUNK_ELEMS / kSeg;
     // warp roles
-    constexpr int kFirstCopier = kWarps;
-    constexpr int kScanWarp    = kWarps + kCopiers;       // and kScanWarp + 1
-    constexpr int kLoadWarp    = kWarps + kCopiers + 2;
+    constexpr int kFirstCopier = kCompactors;
+    constexpr int kScanWarp    = kCompactors + kCopiers;  // and kScanWarp + 1
+    constexpr int kLoadWarp    = kCompactors + kCopiers + 2;
     constexpr int kSegsPerCopier = kWarps / kCopiers;
     static_assert(kWarps % kCopiers == 0, "equal shares for the copier warps");
     static_assert(kSeg % 32 == 0 && kSeg <= 1024 && BT_CHUNK_ELEMS % kSeg == 0, "segments tile a chunk");
@@ -358,6 +359,7 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             capacity          = c0 <= a.arena_bytes ? (a.arena_bytes - c0) / sizeof(V) : 0;
         }
         const Extent vx = extent_of(vals, capacity * sizeof(V));
+        constexpr bool kBulk = kBulkCopyOut16 && sizeof(U) == 2 && CAST == 0;   // 2-byte runs leave through the copy engine
         for (uint32_t it = 0;; ++it) {
             if (tile_of(it) >= num_tiles) break;
             const uint32_t s = it % kStages;
@@ -366,13 +368,18 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
 #pragma unroll
             for (int q = 0; q < kSegsPerCopier; ++q) {
                 const uint32_t seg  = copier * kSegsPerCopier + q;
-                const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
+                U *const       pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
                 const uint32_t cnt  = s_cnt[s][seg];
                 const uint64_t dst  = base + s_off[s][seg];
-                if (dst + cnt <= capacity)
-                    copy_out_segment<U, CAST, false>(pseg, lane, cnt, vals + dst, 0, vx);
-                else
+                if (dst + cnt <= capacity) {
+                    if constexpr (kBulk) copy_out_run16(pseg, lane, cnt, vals + dst, vx);
+                    else copy_out_segment<U, CAST, false>(pseg, lane, cnt, vals + dst, 0, vx);
+                } else {
                     copy_out_segment<U, CAST, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0, vx);
+                }
+            }
+            if constexpr (kBulk) {
+                if (lane == 0) bulk_store_wait_read();            // the copy engine has read the segments
             }
             __syncwarp();
             asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
@@ -386,7 +393,9 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
     const uint64_t words_total = (n + 31) >> 5;
     const Extent   bx          = extent_of(a.bitmap, 4 * words_total);
     const Extent   yx          = extent_of(a.y, n * sizeof(U));
-    for (uint32_t it = 0;; ++it) {
+    for (uint32_t g = warp;; g += kCompactors) {
+        const uint32_t it  = g / kWarps;              // iteration (tile of this CTA) and segment of it
+        const uint32_t seg = g % kWarps;
         const uint64_t t64 = tile_of(it);
         if (t64 >= num_tiles) break;
         const uint32_t s     = it % kStages;
@@ -403,33 +412,33 @@ __global__ void __launch_bounds__((kWarps + kCopiers + 3) * 32) compress_kernel(
             // warps here would never open if one of them had left the kernel because its wait ran out.)
             const uint32_t have    = static_cast<uint32_t>(n - first);
             const uint32_t by_bulk = ((have * static_cast<uint32_t>(sizeof(U))) & ~15u) / sizeof(U);
-            const uint32_t seg0    = warp * kSeg;
+            const uint32_t seg0    = seg * kSeg;
             for (uint32_t e = (by_bulk > seg0 ? by_bulk : seg0) + lane; e < seg0 + kSeg; e += 32)
                 tile[e] = (e < have) ? src[first + e] : U(0);
             __syncwarp();
         }
 
         // ---- in-place compaction of this warp's segment
-        const uint64_t e0     = first + warp * kSeg;                 // first element of the segment
+        const uint64_t e0     = first + seg * kSeg;                 // first element of the segment
         uint32_t       yvalid = 0;
         U             *y      = nullptr;
         if constexpr (WRITE_Y) {
             y      = static_cast<U *>(a.y) + e0;
             yvalid = e0 + kSeg <= n ? static_cast<uint32_t>(kSeg) : (e0 < n ? static_cast<uint32_t>(n - e0) : 0u);
         }
-        const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
+        const uint32_t seg_addr = smem_addr(tile + seg * kSeg);
         uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
             run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau, yx);
         else
             run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau, yx);
         if (lane < kSteps) {
-            const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + warp * kSteps + lane;
+            const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + seg * kSteps + lane;
             if (w < words_total && bx.holds(a.bitmap + w, 4)) a.bitmap[w] = word;
         }
         __syncwarp();
         if (lane == 0) {
-            s_cnt[s][warp] = run;
+            s_cnt[s][seg] = run;
             mbar_arrive(&s_counted[s]);                   // hand the count to the scan warp
         }
     }
@@ -467,14 +476,14 @@ uint64_t set_compress_wait_ns(uint64_t wait_ns) { return g_wait_ns.exchange(wait
 
 namespace {
 
-template <typename U, int RELU_DT, bool WRITE_Y, int CAST, int kWarps, int kSeg, int kStages, int kCopiers>
+template <typename U, int RELU_DT, bool WRITE_Y, int CAST, int kWarps, int kSeg, int kStages, int kCopiers, int kCompactors = kWarps>
 cudaError_t launch_shaped(const CompressArgs &a, cudaStream_t stream)
 {
     constexpr int kTile    = kWarps * kSeg;
-    constexpr int kThreads = (kWarps + kCopiers + 3) * 32;
+    constexpr int kThreads = (kCompactors + kCopiers + 3) * 32;
     constexpr size_t kSmem = static_cast<size_t>(kStages) * kTile * sizeof(U);
     static LaunchShape shape;   // one per instantiation
-    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, CAST, kWarps, kSeg, kStages, kCopiers>;
+    auto kernel = compress_kernel<U, RELU_DT, WRITE_Y, CAST, kWarps, kSeg, kStages, kCopiers, kCompactors>;
 
     const uint32_t num_tiles = static_cast<uint32_t>((a.n + kTile - 1) / kTile);
     int            max_grid  = 0;
@@ -501,11 +510,14 @@ cudaError_t launch_typed(const CompressArgs &a, cudaStream_t stream)
     // One CTA per SM, the ring takes nearly all of its shared memory.
     //   8-byte elements: 8 compactor warps x 512 elements (32 KB tiles), 8 copiers, 7 stages;
     //   4-byte elements: 8 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 7 stages;
-    //   2-byte elements: 16 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 6 stages --
+    //   2-byte elements: 16 compactor warps x 1024 elements (32 KB tiles), 8 copiers, 7 stages --
     //   a 2-byte tile takes as many compaction steps per byte again, so it gets twice the warps.
+    //   (More compactor warps than segments, taking segments in turn -- 18, 20, 21 or 24 with 8 or 4 copiers --
+    //   measured slower on the 392 MiB bf16 tensor: 0.151-0.161 ms against 0.1485; with fewer than 8 copiers the
+    //   copy-out falls behind: 0.19 ms with 4, 0.29 with 2.)
     if constexpr (sizeof(U) == 8) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 512, 7, 8>(a, stream);
     else if constexpr (sizeof(U) == 4) return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 8, 1024, 7, 8>(a, stream);
-    else return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 16, 1024, 6, 8>(a, stream);
+    else return launch_shaped<U, RELU_DT, WRITE_Y, CAST, 16, 1024, 7, 8>(a, stream);
 }
 
 }  // namespace

@@ -482,17 +482,23 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
                 capacity          = at <= p.c.arena_bytes ? (p.c.arena_bytes - at) / sizeof(V) : 0;
             }
             const Extent   vx       = extent_of(vals, capacity * sizeof(V));
+            constexpr bool kBulk    = kBulkCopyOut16 && sizeof(U) == 2;             // 2-byte runs leave through the copy engine
             const uint64_t base     = s_base[s];
 #pragma unroll
             for (int qq = 0; qq < kSegsPerCopier; ++qq) {
                 const uint32_t seg  = copier * kSegsPerCopier + qq;
-                const U *const pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
+                U *const       pseg = tiles + static_cast<size_t>(s) * kTile + seg * kSeg;
                 const uint32_t cnt  = s_cnt[s][seg];
                 const uint64_t dst  = base + s_off[s][seg];
-                if (dst + cnt <= capacity)
-                    copy_out_segment<U, 0, false>(pseg, lane, cnt, vals + dst, 0, vx);
-                else
+                if (dst + cnt <= capacity) {
+                    if constexpr (kBulk) copy_out_run16(pseg, lane, cnt, vals + dst, vx);
+                    else copy_out_segment<U, 0, false>(pseg, lane, cnt, vals + dst, 0, vx);
+                } else {
                     copy_out_segment<U, 0, true>(pseg, lane, cnt, vals + dst, dst < capacity ? capacity - dst : 0, vx);
+                }
+            }
+            if constexpr (kBulk) {
+                if (lane == 0) bulk_store_wait_read();            // the copy engine has read the segments
             }
             __syncwarp();
             asm volatile("" ::: "memory");        // the copy-out stays above the release of the slot
@@ -616,7 +622,7 @@ cudaError_t launch_typed(const CompressCommon &c, const CompressJob *jobs, uint3
     // the shapes of the single-tensor kernel
     if constexpr (sizeof(U) == 8) return launch_shaped<U, FUSED, WRITE_Y, kMaxBatch, 8, 512, 7, 8>(c, jobs, count, workspace, stream);
     else if constexpr (sizeof(U) == 4) return launch_shaped<U, FUSED, WRITE_Y, kMaxBatch, 8, 1024, 7, 8>(c, jobs, count, workspace, stream);
-    else return launch_shaped<U, FUSED, WRITE_Y, kMaxBatch, 16, 1024, 6, 8>(c, jobs, count, workspace, stream);
+    else return launch_shaped<U, FUSED, WRITE_Y, kMaxBatch, 16, 1024, 7, 8>(c, jobs, count, workspace, stream);
 }
 
 }  // namespace

@@ -252,6 +252,70 @@ __device__ __forceinline__ void copy_out_segment(const U *__restrict__ seg, cons
     }
 }
 
+// The copy-out of a packed run of 2-byte values through the copy engine.  A lane-by-lane copy costs a shared load
+// and a 2-byte global store per survivor on the port the compactors' votes, counts and stores also queue at; a
+// bulk copy reads shared memory by itself.  It wants source and destination on 16-byte boundaries, and the
+// destination is wherever the run's rank puts it: so the up to 7 values in front of the destination's first
+// boundary and the up to 7 behind its last one leave as single elements, and the rest is first moved down inside
+// the segment by that many elements (two 16-byte loads, four funnel shifts, one 16-byte store per 8 values;
+// loads of a round before its stores, rounds in rising order, so nothing is overwritten before it is read).
+// The caller waits for the copy engine's reads (bulk_store_wait_read) before it releases the slot.
+constexpr bool kBulkCopyOut16 = true;
+
+__device__ __forceinline__ void bulk_store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
+__device__ __forceinline__ void copy_out_run16(uint16_t *seg, const uint32_t lane, const uint32_t cnt, uint16_t *out,
+                                               const Extent vx)
+{
+    const uint32_t sa = smem_addr(seg);
+    uint32_t       h  = (static_cast<uint32_t>(16u - (reinterpret_cast<uintptr_t>(out) & 15u)) & 15u) >> 1;
+    h                 = h < cnt ? h : cnt;                       // values in front of the first boundary
+    const uint32_t vecs = (cnt - h) >> 3;                        // whole 16-byte units behind them
+    const uint32_t tail = h + 8u * vecs;                         // first of the values behind the last unit
+    // the ragged ends: lanes 0..6 the head, lanes 8..14 the tail; read now, the move below overwrites the head
+    const bool     is_head = lane < h, is_tail = lane >= 8u && tail + (lane - 8u) < cnt;
+    const uint32_t ei      = is_head ? lane : tail + (lane - 8u);
+    uint16_t       edge    = 0;
+    if (is_head || is_tail) edge = seg[ei];
+    if (vecs) {
+        if (h) {
+            __syncwarp();
+            const uint32_t sh = (h & 1u) * 16u;
+            for (uint32_t v0 = 0; v0 < vecs; v0 += 32) {
+                const uint32_t v  = v0 + lane;
+                const uint32_t at = sa + 16u * v;
+                uint32_t       w0 = 0, w1 = 0, w2 = 0, w3 = 0, w4 = 0, w5 = 0, w6 = 0, w7 = 0;
+                if (v < vecs) {
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w0), "=r"(w1), "=r"(w2), "=r"(w3) : "r"(at));
+                    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w4), "=r"(w5), "=r"(w6), "=r"(w7) : "r"(at + 16u));
+                }
+                __syncwarp();
+                if (v < vecs) {
+                    uint32_t o0, o1, o2, o3;
+                    switch (h >> 1) {                              // the same for the whole warp
+                    case 0: o0 = __funnelshift_r(w0, w1, sh), o1 = __funnelshift_r(w1, w2, sh), o2 = __funnelshift_r(w2, w3, sh), o3 = __funnelshift_r(w3, w4, sh); break;
+                    case 1: o0 = __funnelshift_r(w1, w2, sh), o1 = __funnelshift_r(w2, w3, sh), o2 = __funnelshift_r(w3, w4, sh), o3 = __funnelshift_r(w4, w5, sh); break;
+                    case 2: o0 = __funnelshift_r(w2, w3, sh), o1 = __funnelshift_r(w3, w4, sh), o2 = __funnelshift_r(w4, w5, sh), o3 = __funnelshift_r(w5, w6, sh); break;
+                    default: o0 = __funnelshift_r(w3, w4, sh), o1 = __funnelshift_r(w4, w5, sh), o2 = __funnelshift_r(w5, w6, sh), o3 = __funnelshift_r(w6, w7, sh); break;
+                    }
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(at), "r"(o0), "r"(o1), "r"(o2), "r"(o3) : "memory");
+                }
+            }
+            fence_proxy_async();                                  // the moved values, before the copy engine reads them
+        }
+        __syncwarp();
+        if (lane == 0 && vx.holds(out + h, 16u * vecs)) {
+            fence_proxy_async();                                  // the compactors' stores (ordered before this by the mbarriers)
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(out + h), "r"(sa), "r"(16u * vecs) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+    }
+    if ((is_head || is_tail) && vx.holds(out + ei, 2)) out[ei] = edge;
+}
+
 // Launch shape of one kernel instantiation on one device: the opt-in shared
 // memory size is set and the number of co-resident CTAs is looked up once.
 struct LaunchShape {

@@ -231,3 +231,18 @@ def test_arena_batch_over_several_launches_and_an_arena_that_runs_full(oracle):
         assert np.array_equal(W.raw_numpy(sts[k].bitmap)[:(raw.size + 31) // 32].view(np.uint32), c.bitmap)
         assert np.array_equal(W.raw_numpy(sts[k].chunk_prefix)[:(raw.size + 4095) // 4096].view(np.uint64), c.prefix)
     assert bool((arena[room:] == 0x5A).all().item())           # nothing beyond the arena, whatever did not fit
+
+
+@pytest.mark.parametrize("kind", ["bf16", "f16"])
+def test_batch_of_two_byte_runs_at_every_offset_from_a_16_byte_boundary(oracle, kind):
+    """The batched kernel's copy-out of 2-byte runs (16-byte units, single values at the ragged ends) on tensors
+    whose runs start at each of the eight positions relative to a unit."""
+    from tests.test_gpu_parity import _runs_at_offset
+    dt = TDT[kind]
+    raws = [_runs_at_offset(kind, lead, 7100 + lead) for lead in range(8)]
+    xs = [from_raw(r, kind) for r in raws]
+    sts = [B.Stash(r.size, dt) for r in raws]
+    ws = torch.empty(B.bt_batch_workspace_bytes([r.size for r in raws]), dtype=torch.uint8, device="cuda")
+    B.bt_compress_batch(B.batch_items(xs, sts, None), dt, ws)
+    torch.cuda.synchronize()
+    check_batch(oracle, kind, raws, sts, None, False)

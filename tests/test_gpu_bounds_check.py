@@ -41,6 +41,11 @@ def test_compress_and_decompress(checked, oracle, kind):
     test_gpu_parity.test_compress_decompress_sparsity_levels(gpu_util, oracle, kind, 0.99)
 
 
+@pytest.mark.parametrize("kind", ["bf16", "f16"])
+def test_two_byte_runs_in_16_byte_units(checked, oracle, kind):
+    test_gpu_parity.test_two_byte_runs_at_every_offset_from_a_16_byte_boundary(gpu_util, oracle, kind, 5)
+
+
 def test_capacity_overflow(checked, oracle):
     test_gpu_parity.test_capacity_overflow_reports_and_stays_in_bounds(gpu_util, oracle)
 

@@ -191,3 +191,37 @@ def test_bitmap_at_any_four_byte_boundary(G, oracle, kind, offset_words):
     torch.cuda.synchronize()
     assert st.nnz == c.nnz and np.array_equal(W.raw_numpy(bitmap).view(np.uint32), c.bitmap)
     assert (room[:offset_words] == 0x5A5A5A5A).all() and (room[offset_words + words:] == 0x5A5A5A5A).all()
+
+
+def _runs_at_offset(kind, lead, seed):
+    """2-byte patterns whose packed runs start `lead` values past a 16-byte boundary of values[]: segment 0
+    (1024 elements) keeps exactly `lead` non-zeros, then come full segments (runs of 1024 values), segments
+    with 1..15 survivors (runs shorter than one 16-byte unit, or one unit and ragged ends), an empty segment
+    and a ragged tail."""
+    n = 16384 * 5 + 1024 * 3 + 777
+    x = W.random_patterns(n, kind, 0.0, seed=seed)
+    rng = np.random.default_rng(seed)
+    dense = x[:1024 * 6]
+    dense[(dense & 0x7FFF) == 0] = 0x3F80                           # five runs of exactly 1024 values
+    x[lead:1024] = 0
+    for seg, keep in zip(range(20, 36), range(0, 16)):              # segments of the second tile: 0..15 survivors
+        lo = 1024 * seg
+        kill = np.ones(1024, dtype=bool)
+        kill[rng.choice(1024, size=keep, replace=False)] = False
+        x[lo:lo + 1024][kill] = 0
+    return x
+
+
+@pytest.mark.parametrize("kind", ["bf16", "f16"])
+@pytest.mark.parametrize("lead", range(8))
+def test_two_byte_runs_at_every_offset_from_a_16_byte_boundary(G, oracle, kind, lead):
+    """The packed runs of 2-byte values leave in 16-byte units with single values at their ragged ends: every
+    position of a run's start relative to the unit, full-length runs, runs of fewer values than a unit."""
+    x = _runs_at_offset(kind, lead, 7000 + lead)
+    c = oracle.compress(x)
+    g = G.gpu_compress(G.from_raw(x, kind))
+    assert_same_compressed(g, c)
+    y_ref, cr = oracle.relu_fwd_compress(x, kind)
+    g = G.gpu_compress(G.from_raw(x, kind), relu=True, want_y=True)
+    assert_same_compressed(g, cr)
+    assert np.array_equal(g.y, y_ref)
