@@ -12,7 +12,7 @@
 //
 //   step k:  lane l reads element 32k+l (conflict-free shared load);
 //            ballot(non-zero) IS bitmap word k (LSB first), kept by lane k;
-//            popc(ballot & lanemask_lt) is the lane's rank;
+//            the number of ballot bits below the lane is the lane's rank;
 //            non-zero lanes store the element at [run + rank] of the same
 //            segment -- in place: the write position never passes the read
 //            position, and a batch's loads are issued before the previous
@@ -389,7 +389,6 @@ __global__ void __launch_bounds__((kCompactors + kCopiers + 3) * 32) compress_ke
     }
 
     // ---------------------------------------------------------------- compactor warps
-    const uint32_t lt          = lanemask_lt();
     const uint64_t words_total = (n + 31) >> 5;
     const Extent   bx          = extent_of(a.bitmap, 4 * words_total);
     const Extent   yx          = extent_of(a.y, n * sizeof(U));
@@ -429,9 +428,9 @@ __global__ void __launch_bounds__((kCompactors + kCopiers + 3) * 32) compress_ke
         const uint32_t seg_addr = smem_addr(tile + seg * kSeg);
         uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau, yx);
+            run = compact_segment<U, RELU_DT, WRITE_Y, false, kSteps>(seg_addr, word, lane, y, yvalid, a.tau, yx);
         else
-            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, lt, y, yvalid, a.tau, yx);
+            run = compact_segment<U, RELU_DT, WRITE_Y, true, kSteps>(seg_addr, word, lane, y, yvalid, a.tau, yx);
         if (lane < kSteps) {
             const uint64_t w = static_cast<uint64_t>(t) * (kTile / 32) + seg * kSteps + lane;
             if (w < words_total && bx.holds(a.bitmap + w, 4)) a.bitmap[w] = word;
@@ -546,21 +545,20 @@ cudaError_t launch_compress(const CompressArgs &a, int dtype, int fused, cudaStr
             return y ? launch_typed<uint64_t, k6 + BT_F64, true>(a, stream) : launch_typed<uint64_t, k6 + BT_F64, false>(a, stream);
         case BT_F32:
             return y ? launch_typed<uint32_t, k6 + BT_F32, true>(a, stream) : launch_typed<uint32_t, k6 + BT_F32, false>(a, stream);
-        // 2-byte types: with the dense output the decisions are taken on the bit pattern (0.1925 -> 0.1864 ms on the
-        // 392 MiB tensor); without it the float compares measured faster (0.182 against 0.192 ms), as for the ReLU
+        // 2-byte types: the decisions by compares in the element's own type
         case BT_F16:
-            return y ? launch_typed<uint16_t, kFusedRelu6Bits + BT_F16, true>(a, stream) : launch_typed<uint16_t, k6 + BT_F16, false>(a, stream);
+            return y ? launch_typed<uint16_t, kFusedRelu6Half + BT_F16, true>(a, stream) : launch_typed<uint16_t, kFusedRelu6Half + BT_F16, false>(a, stream);
         default:
-            return y ? launch_typed<uint16_t, kFusedRelu6Bits + BT_BF16, true>(a, stream)
-                     : launch_typed<uint16_t, k6 + BT_BF16, false>(a, stream);
+            return y ? launch_typed<uint16_t, kFusedRelu6Half + BT_BF16, true>(a, stream)
+                     : launch_typed<uint16_t, kFusedRelu6Half + BT_BF16, false>(a, stream);
         }
     }
-    if (y && a.tau == 0.0f && (dtype == BT_F16 || dtype == BT_BF16)) {
-        // The ReLU itself on a 2-byte type, with the dense output: decided on the bit pattern (0.182 -> 0.178 ms on
-        // the 392 MiB tensor).  Without the dense output the same test measured slower than the float compare
-        // (0.169 against 0.162 ms), so that form keeps the compare.
-        constexpr int kb = kFusedReluBits;
-        return dtype == BT_F16 ? launch_typed<uint16_t, kb + BT_F16, true>(a, stream) : launch_typed<uint16_t, kb + BT_BF16, true>(a, stream);
+    if (a.tau == 0.0f && (dtype == BT_F16 || dtype == BT_BF16)) {
+        // The ReLU itself on a 2-byte type: decided by one compare in the element's own type (on the 392 MiB tensor
+        // 0.165 -> 0.138 ms without the dense output, together with the multiply-add forms of the compaction step).
+        constexpr int kh = kFusedReluHalf;
+        if (dtype == BT_F16) return y ? launch_typed<uint16_t, kh + BT_F16, true>(a, stream) : launch_typed<uint16_t, kh + BT_F16, false>(a, stream);
+        return y ? launch_typed<uint16_t, kh + BT_BF16, true>(a, stream) : launch_typed<uint16_t, kh + BT_BF16, false>(a, stream);
     }
     switch (dtype) {
     case BT_F64:

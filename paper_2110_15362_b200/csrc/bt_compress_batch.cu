@@ -547,9 +547,9 @@ compress_kernel(const __grid_constant__ CompressParams<kJobs> p)
         const uint32_t seg_addr = smem_addr(tile + warp * kSeg);
         uint32_t       run, word;
         if (!WRITE_Y || yvalid == static_cast<uint32_t>(kSeg))   // all but a ragged last tile: no bounds checks on y
-            run = compact_segment<U, FUSED, WRITE_Y, false, kSeg / 32>(seg_addr, word, lane, lanemask_lt(), y, yvalid, p.c.tau, yx);
+            run = compact_segment<U, FUSED, WRITE_Y, false, kSeg / 32>(seg_addr, word, lane, y, yvalid, p.c.tau, yx);
         else
-            run = compact_segment<U, FUSED, WRITE_Y, true, kSeg / 32>(seg_addr, word, lane, lanemask_lt(), y, yvalid, p.c.tau, yx);
+            run = compact_segment<U, FUSED, WRITE_Y, true, kSeg / 32>(seg_addr, word, lane, y, yvalid, p.c.tau, yx);
         if (lane < static_cast<uint32_t>(kSeg / 32)) {
             const uint64_t wd = t64 * (kTile / 32) + warp * (kSeg / 32) + lane;
             if (wd < ((n + 31) >> 5) && extent_of(jb.bitmap, 4 * ((n + 31) >> 5)).holds(jb.bitmap + wd, 4)) jb.bitmap[wd] = word;
@@ -648,11 +648,14 @@ cudaError_t launch_compress_batch(const CompressJob *jobs, uint32_t count, float
                : dtype == BT_F32 ? launch_typed<uint32_t, -1, false>(c, jobs, count, workspace, stream)
                                  : launch_typed<uint16_t, -1, false>(c, jobs, count, workspace, stream);
     }
-    if (y && tau == 0.0f && (dtype == BT_F16 || dtype == BT_BF16)) {
-        // the ReLU itself on a 2-byte type, with the dense output: decided on the bit pattern (as in the single-tensor kernel)
-        constexpr int kb = kFusedReluBits;
-        return dtype == BT_F16 ? launch_typed<uint16_t, kb + BT_F16, true>(c, jobs, count, workspace, stream)
-                               : launch_typed<uint16_t, kb + BT_BF16, true>(c, jobs, count, workspace, stream);
+    if (tau == 0.0f && (dtype == BT_F16 || dtype == BT_BF16)) {
+        // the ReLU itself on a 2-byte type: decided by one compare in the element's own type (as in the single-tensor kernel)
+        constexpr int kh = kFusedReluHalf;
+        if (dtype == BT_F16)
+            return y ? launch_typed<uint16_t, kh + BT_F16, true>(c, jobs, count, workspace, stream)
+                     : launch_typed<uint16_t, kh + BT_F16, false>(c, jobs, count, workspace, stream);
+        return y ? launch_typed<uint16_t, kh + BT_BF16, true>(c, jobs, count, workspace, stream)
+                 : launch_typed<uint16_t, kh + BT_BF16, false>(c, jobs, count, workspace, stream);
     }
     switch (dtype) {
     case BT_F64:

@@ -371,32 +371,39 @@ __device__ __forceinline__ uint32_t greater_or_nan(double v, double b)
 }
 
 // The fused forward forms are numbered by one template argument: -1 none (plain compressor), DT (0..3) keep
-// what exceeds the threshold (tau = 0: ReLU), 4 + DT ReLU6, 8 + DT (2-byte types only) the ReLU decided on the
-// bit pattern.
+// what exceeds the threshold (tau = 0: ReLU), 4 + DT ReLU6, and for the 2-byte types 8 + DT the ReLU and 12 + DT
+// the ReLU6 decided by compares in the element's own type.
 constexpr int kFusedRelu6     = 4;
-constexpr int kFusedReluBits  = 8;
-constexpr int kFusedRelu6Bits = 12;    // 12 + DT: ReLU6 of a 2-byte type decided on the bit pattern
+constexpr int kFusedReluHalf  = 8;
+constexpr int kFusedRelu6Half = 12;
 
-// ReLU of a 2-byte element without widening it: x, the element's pattern sign-extended to 32 bits, is kept iff
-// it is a positive number, +inf or a NaN of either sign -- exactly the elements for which x <= 0 is false under
-// IEEE comparison.  Positive patterns are the positive signed integers; a negative NaN lies above -inf's pattern.
-// Two integer compares instead of a conversion, a float compare, a select and the zero test.
+// ReLU and ReLU6 of a 2-byte element (x: its pattern, possibly sign-extended) without widening it, by binary16 /
+// bfloat16 compare instructions: kept iff x > 0 or x is a NaN -- exactly the elements for which x <= 0 is false
+// under IEEE comparison --, saturated iff x >= 6 (false for a NaN).  One instruction per decision instead of a
+// conversion, a float compare, a select and the zero test, and not on the integer pipe that the rest of the
+// compaction step loads (integer compares of the bit pattern, two per decision, measured slower than the float
+// form without the dense output; these are faster than both, with and without it).
 template <int DT>
-__device__ __forceinline__ bool relu_keeps_bits(const uint32_t x)
+__device__ __forceinline__ bool relu_keeps_half(const uint32_t x)
 {
     static_assert(DT == BT_F16 || DT == BT_BF16, "2-byte element types");
-    constexpr uint32_t kMinusInf = DT == BT_F16 ? 0xFFFFFC00u : 0xFFFFFF80u;
-    return (static_cast<int32_t>(x) > 0) | (x > kMinusInf);      // no short circuit: two compares, no branch
+    uint32_t r;
+    if constexpr (DT == BT_F16)
+        asm("{\n\t.reg .pred p;\n\t.reg .b16 h, z;\n\tcvt.u16.u32 h, %1;\n\tmov.b16 z, 0;\n\tsetp.gtu.f16 p, h, z;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"(x));
+    else
+        asm("{\n\t.reg .pred p;\n\t.reg .b16 h, z;\n\tcvt.u16.u32 h, %1;\n\tmov.b16 z, 0;\n\tsetp.gtu.bf16 p, h, z;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"(x));
+    return r != 0;
 }
-
-// x >= 6 for the same sign-extended pattern: the positive numbers from 6 up to +inf are the integers from 6's
-// pattern to +inf's (a positive NaN lies above +inf's pattern, a negative pattern is a negative integer).
 template <int DT>
-__device__ __forceinline__ bool relu6_saturates_bits(const uint32_t x)
+__device__ __forceinline__ bool relu6_saturates_half(const uint32_t x)
 {
     static_assert(DT == BT_F16 || DT == BT_BF16, "2-byte element types");
-    constexpr int32_t kInf = DT == BT_F16 ? 0x7C00 : 0x7F80;
-    return (static_cast<int32_t>(x) >= static_cast<int32_t>(Elem<DT>::kSix)) & (static_cast<int32_t>(x) <= kInf);
+    uint32_t r;
+    if constexpr (DT == BT_F16)
+        asm("{\n\t.reg .pred p;\n\t.reg .b16 h, z;\n\tcvt.u16.u32 h, %1;\n\tmov.b16 z, 0x4600;\n\tsetp.ge.f16 p, h, z;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"(x));
+    else
+        asm("{\n\t.reg .pred p;\n\t.reg .b16 h, z;\n\tcvt.u16.u32 h, %1;\n\tmov.b16 z, 0x40C0;\n\tsetp.ge.bf16 p, h, z;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r) : "r"(x));
+    return r != 0;
 }
 
 // y = (x <= tau) ? +0 : x, and for ReLU6 additionally 6 where x >= 6; IEEE comparisons, so a NaN is kept.
