@@ -114,6 +114,8 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
     const uint32_t total = __shfl_sync(kFull, incl, 31);          // set bits of the quarter
 
     const uint32_t shift = (lane % kLanesPerWord) * kE;     // which kE-bit group of the word
+    uint32_t       one, two;                                 // registers the compiler cannot see through
+    asm volatile("mov.u32 %0, 1;\n\tmov.u32 %1, 2;" : "=r"(one), "=r"(two));
     const Extent   yx    = extent_of(y, n * sizeof(U));
     const Extent   vx    = extent_of(values, capacity * sizeof(U));
 #pragma unroll
@@ -123,12 +125,30 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
         const uint32_t wex  = __shfl_sync(kFull, excl, from);
         const uint32_t bits = (w >> shift) & ((1u << kE) - 1u);
         uint32_t       off  = skew + wex + __popc(w & ((1u << shift) - 1u));
+        if constexpr (sizeof(U) == 2) {
+            // 2-byte elements: this loop is bound by the integer pipe, so the running position advances by a
+            // predicated multiply-add (FMA pipe) and the staged address is a byte address kept in one register
+            uint32_t at = smem_addr(stage) + 2u * off;
 #pragma unroll
-        for (int j = 0; j < kE; ++j) {
-            const bool set = (bits >> j) & 1u;
-            if (set) stage[off] = e[k][j];
-            off += set;
-            if constexpr (WRITE_Y) e[k][j] = set ? e[k][j] : U(0);
+            for (int j = 0; j < kE; ++j) {
+                asm volatile(
+                    "{\n\t.reg .pred p;\n\t.reg .b32 t;\n\t"
+                    "and.b32 t, %1, %2;\n\tsetp.ne.u32 p, t, 0;\n\t"
+                    "@p st.shared.u16 [%0], %3;\n\t"
+                    "@p mad.lo.u32 %0, %4, %5, %0;\n\t}"
+                    : "+r"(at)
+                    : "r"(bits), "r"(1u << j), "h"(e[k][j]), "r"(one), "r"(two)
+                    : "memory");
+                if constexpr (WRITE_Y) e[k][j] = ((bits >> j) & 1u) ? e[k][j] : U(0);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kE; ++j) {
+                const bool set = (bits >> j) & 1u;
+                if (set) stage[off] = e[k][j];
+                off += set;
+                if constexpr (WRITE_Y) e[k][j] = set ? e[k][j] : U(0);
+            }
         }
         if constexpr (WRITE_Y) {
             const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
