@@ -54,10 +54,12 @@ CASE_OPS = ("compress", "relu", "relu_y", "prune", "narrow", "relu6", "relu6_bwd
 # little below the algorithmic bytes because the tail of what a launch writes is still in the L2 when it ends.
 # The capture and its command are summarised in the file named beside each figure.
 NCU_DRAM_BYTES_PER_ELEMENT = {
-    ("bf16", "bt_relu_fwd_compress"): (2.835, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
-    ("f16", "bt_relu_fwd_compress"): (2.835, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
-    ("bf16", "bt_compress"): (2.831, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
-    ("f16", "bt_compress"): (2.831, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("bf16", "bt_relu_fwd_compress"): (2.844, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
+    ("f16", "bt_relu_fwd_compress"): (2.844, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("bf16", "bt_relu_fwd_compress+y"): (4.696, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
+    ("f16", "bt_relu_fwd_compress+y"): (4.696, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("bf16", "bt_compress"): (2.847, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
+    ("f16", "bt_compress"): (2.847, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
     ("bf16", "bt_decompress"): (2.779, "profiles/bt_decompress_bf16_2p27_ncu_full.md"),
     ("f16", "bt_decompress"): (2.779, "profiles/bt_decompress_bf16_2p27_ncu_full.md (bf16 capture; same kernel)"),
     ("f32", "bt_compress"): (5.562, "profiles/bt_codec_f32_2p26_ncu_full.md"),
@@ -767,7 +769,7 @@ def run_ours(args):
         graded = [r for r in rows if r["kernel"] in OPS and r.get("launches", 1) == 1 and r["algorithmic_bytes"] >= 256e6]
         if graded:
             low = min(graded, key=lambda r: r["frac_of_measured"])
-            per_el, src = NCU_DRAM_BYTES_PER_ELEMENT.get((low["dtype"], low["kernel"]), (None, None))
+            per_el, src = NCU_DRAM_BYTES_PER_ELEMENT.get((low["dtype"], low["kernel"] + ("+y" if low.get("dense_output") else "")), (None, None))
             line["roofline"] = {"bound": "hbm", "kernel": low["kernel"], "dtype": low["dtype"], "config": low["config"],
                                 "tensor": low.get("tensor"), "dense_output": low.get("dense_output"),
                                 "achieved": low["gbs"], "peak": peak, "unit": "GB/s", "frac": low["frac_of_measured"],
