@@ -29,6 +29,35 @@ namespace {
 
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 
+// A 16-byte vector of elements to and from its elements (element 0 at the lowest address).
+template <typename U>
+__device__ __forceinline__ void unpack_vec(const uint4 pack, U *ev)
+{
+    if constexpr (sizeof(U) == 8) {
+        ev[0] = pack.x | (static_cast<uint64_t>(pack.y) << 32);
+        ev[1] = pack.z | (static_cast<uint64_t>(pack.w) << 32);
+    } else if constexpr (sizeof(U) == 4) {
+        ev[0] = pack.x, ev[1] = pack.y, ev[2] = pack.z, ev[3] = pack.w;
+    } else {
+        ev[0] = static_cast<U>(pack.x), ev[1] = static_cast<U>(pack.x >> 16);
+        ev[2] = static_cast<U>(pack.y), ev[3] = static_cast<U>(pack.y >> 16);
+        ev[4] = static_cast<U>(pack.z), ev[5] = static_cast<U>(pack.z >> 16);
+        ev[6] = static_cast<U>(pack.w), ev[7] = static_cast<U>(pack.w >> 16);
+    }
+}
+template <typename U>
+__device__ __forceinline__ uint4 pack_vec(const U *ev)
+{
+    if constexpr (sizeof(U) == 8)
+        return make_uint4(static_cast<uint32_t>(ev[0]), static_cast<uint32_t>(ev[0] >> 32), static_cast<uint32_t>(ev[1]),
+                          static_cast<uint32_t>(ev[1] >> 32));
+    else if constexpr (sizeof(U) == 4)
+        return make_uint4(ev[0], ev[1], ev[2], ev[3]);
+    else
+        return make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16), ev[4] | (uint32_t(ev[5]) << 16),
+                          ev[6] | (uint32_t(ev[7]) << 16));
+}
+
 template <typename U, int kE, int kWarps, bool WRITE_Y>
 __global__ void __launch_bounds__(kWarps * 32)
 mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64_t *__restrict__ prefix,
@@ -51,31 +80,22 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
     const uint64_t w0          = chunk * 128 + 4 * lane;   // this lane's four words of the chunk
     const uint64_t e0          = warp_global << 10;        // first element of the quarter
 
-    // the quarter of x first: these loads do not depend on the bitmap
-    U e[kSteps][kE];
+    // the quarter of x first: these loads do not depend on the bitmap.  The 16-byte vectors stay packed until their
+    // step comes (unpacked at once, a quarter of 2-byte elements holds 32 registers per lane and costs occupancy).
+    uint4 xv[kSteps][kE / kVec];
 #pragma unroll
     for (int k = 0; k < kSteps; ++k) {
         const uint64_t eo = e0 + static_cast<uint64_t>(k) * (32 * kE) + lane * kE;
 #pragma unroll
         for (int v = 0; v < kE / kVec; ++v) {
             const uint64_t at = eo + v * kVec;
-            U             *ev = e[k] + v * kVec;
             if (at + kVec <= n) {
-                const uint4 pack = *reinterpret_cast<const uint4 *>(x + at);
-                if constexpr (kVec == 2) {
-                    ev[0] = pack.x | (static_cast<uint64_t>(pack.y) << 32);
-                    ev[1] = pack.z | (static_cast<uint64_t>(pack.w) << 32);
-                } else if constexpr (kVec == 4) {
-                    ev[0] = pack.x, ev[1] = pack.y, ev[2] = pack.z, ev[3] = pack.w;
-                } else {
-                    ev[0] = static_cast<U>(pack.x), ev[1] = static_cast<U>(pack.x >> 16);
-                    ev[2] = static_cast<U>(pack.y), ev[3] = static_cast<U>(pack.y >> 16);
-                    ev[4] = static_cast<U>(pack.z), ev[5] = static_cast<U>(pack.z >> 16);
-                    ev[6] = static_cast<U>(pack.w), ev[7] = static_cast<U>(pack.w >> 16);
-                }
+                xv[k][v] = *reinterpret_cast<const uint4 *>(x + at);
             } else {
+                U t[kVec];
 #pragma unroll
-                for (int j = 0; j < kVec; ++j) ev[j] = at + j < n ? x[at + j] : U(0);
+                for (int j = 0; j < kVec; ++j) t[j] = at + j < n ? x[at + j] : U(0);
+                xv[k][v] = pack_vec<U>(t);
             }
         }
     }
@@ -120,6 +140,9 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
     const Extent   vx    = extent_of(values, capacity * sizeof(U));
 #pragma unroll
     for (int k = 0; k < kSteps; ++k) {
+        U e[1][kE];                                            // this step's elements (indexed e[0][j] below)
+#pragma unroll
+        for (int v = 0; v < kE / kVec; ++v) unpack_vec<U>(xv[k][v], e[0] + v * kVec);
         const int      from = k * kWordsPerStep + lane / kLanesPerWord;
         const uint32_t w    = __shfl_sync(kFull, word, from);
         const uint32_t wex  = __shfl_sync(kFull, excl, from);
@@ -137,17 +160,17 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
                     "@p st.shared.u16 [%0], %3;\n\t"
                     "@p mad.lo.u32 %0, %4, %5, %0;\n\t}"
                     : "+r"(at)
-                    : "r"(bits), "r"(1u << j), "h"(e[k][j]), "r"(one), "r"(two)
+                    : "r"(bits), "r"(1u << j), "h"(e[0][j]), "r"(one), "r"(two)
                     : "memory");
-                if constexpr (WRITE_Y) e[k][j] = ((bits >> j) & 1u) ? e[k][j] : U(0);
+                if constexpr (WRITE_Y) e[0][j] = ((bits >> j) & 1u) ? e[0][j] : U(0);
             }
         } else {
 #pragma unroll
             for (int j = 0; j < kE; ++j) {
                 const bool set = (bits >> j) & 1u;
-                if (set) stage[off] = e[k][j];
+                if (set) stage[off] = e[0][j];
                 off += set;
-                if constexpr (WRITE_Y) e[k][j] = set ? e[k][j] : U(0);
+                if constexpr (WRITE_Y) e[0][j] = set ? e[0][j] : U(0);
             }
         }
         if constexpr (WRITE_Y) {
@@ -155,18 +178,9 @@ mask_gather_kernel(const U *x, const uint32_t *__restrict__ bitmap, const uint64
 #pragma unroll
             for (int v = 0; v < kE / kVec; ++v) {
                 const uint64_t at = eo + v * kVec;
-                const U       *ev = e[k] + v * kVec;
+                const U       *ev = e[0] + v * kVec;
                 if (at + kVec <= n) {
-                    uint4 pack;
-                    if constexpr (kVec == 2) {
-                        pack = make_uint4(static_cast<uint32_t>(ev[0]), static_cast<uint32_t>(ev[0] >> 32),
-                                          static_cast<uint32_t>(ev[1]), static_cast<uint32_t>(ev[1] >> 32));
-                    } else if constexpr (kVec == 4) {
-                        pack = make_uint4(ev[0], ev[1], ev[2], ev[3]);
-                    } else {
-                        pack = make_uint4(ev[0] | (uint32_t(ev[1]) << 16), ev[2] | (uint32_t(ev[3]) << 16),
-                                          ev[4] | (uint32_t(ev[5]) << 16), ev[6] | (uint32_t(ev[7]) << 16));
-                    }
+                    const uint4 pack = pack_vec<U>(ev);
                     if (yx.holds(y + at, 16)) *reinterpret_cast<uint4 *>(y + at) = pack;
                 } else {
 #pragma unroll

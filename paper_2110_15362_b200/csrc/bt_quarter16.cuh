@@ -24,15 +24,16 @@ __device__ __forceinline__ uint4 ldg_vec_stream(const uint4 *p)
 }
 
 // Four consecutive elements under the four low bits of `bits`: for every set bit the next 2-byte value at shared
-// address `a` (which moves on), +0 for a clear bit; packed two to a word.
+// address `a` (which moves on), kFill for a clear bit; packed two to a word.
+template <uint32_t kFill = 0>
 __device__ __forceinline__ uint2 expand4_u16(uint32_t a, const uint32_t bits)
 {
     uint2 r;
 #define BT_PAIR(OUT, B0, B1)                                                                                         \
-    "and.b32 t, %3, " #B0 ";\n\tsetp.ne.u32 p, t, 0;\n\tld.shared.u16 lo, [%2];\n\tselp.b32 lo, lo, 0, p;\n\t@p add.u32 %2, %2, 2;\n\t" \
-    "and.b32 t, %3, " #B1 ";\n\tsetp.ne.u32 p, t, 0;\n\tld.shared.u16 hi, [%2];\n\tselp.b32 hi, hi, 0, p;\n\t@p add.u32 %2, %2, 2;\n\t" \
+    "and.b32 t, %3, " #B0 ";\n\tsetp.ne.u32 p, t, 0;\n\tld.shared.u16 lo, [%2];\n\tselp.b32 lo, lo, %4, p;\n\t@p add.u32 %2, %2, 2;\n\t" \
+    "and.b32 t, %3, " #B1 ";\n\tsetp.ne.u32 p, t, 0;\n\tld.shared.u16 hi, [%2];\n\tselp.b32 hi, hi, %4, p;\n\t@p add.u32 %2, %2, 2;\n\t" \
     "prmt.b32 " OUT ", lo, hi, 0x5410;\n\t"
-    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 t, lo, hi;\n\t" BT_PAIR("%0", 1, 2) BT_PAIR("%1", 4, 8) "}" : "=r"(r.x), "=r"(r.y), "+r"(a) : "r"(bits));
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 t, lo, hi;\n\t" BT_PAIR("%0", 1, 2) BT_PAIR("%1", 4, 8) "}" : "=r"(r.x), "=r"(r.y), "+r"(a) : "r"(bits), "n"(kFill));
 #undef BT_PAIR
     return r;
 }
@@ -148,9 +149,10 @@ __device__ __forceinline__ bool stage_quarter(const uint32_t *__restrict__ bitma
 }
 
 // Step k (0..7) of the expansion: the lane's four consecutive elements e0 + 128k + 4 lane .. + 3, packed two to a
-// word, +0 where the bit is clear; `bits` receives the four bits (low nibble).  (With 8 elements per lane the 32
+// word, kFill (+0 unless the caller asks otherwise) where the bit is clear; `bits` receives the four bits (low nibble).  (With 8 elements per lane the 32
 // lanes of one shared load reach over 256 bytes of the run and every load takes two passes: 0.131 ms instead of
 // 0.126 on 205 M elements; with 2 per lane the shuffles and stores double: 0.153 ms.)
+template <uint32_t kFill = 0>
 __device__ __forceinline__ uint2 expand_step(const Quarter &qt, const int k, const uint32_t lane, uint32_t &bits)
 {
     const int      from = k * 4 + (lane >> 3);
@@ -159,7 +161,7 @@ __device__ __forceinline__ uint2 expand_step(const Quarter &qt, const int k, con
     const uint32_t sh   = (lane & 7u) * 4u;
     const uint32_t off  = wex + __popc(w & ((1u << sh) - 1u));
     bits                = w >> sh;
-    return expand4_u16(qt.run + 2u * off, bits);
+    return expand4_u16<kFill>(qt.run + 2u * off, bits);
 }
 
 }  // namespace q16

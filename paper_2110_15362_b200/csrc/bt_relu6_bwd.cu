@@ -149,11 +149,22 @@ relu6_bwd_kernel(const uint32_t *__restrict__ bitmap, const U *__restrict__ valu
     }
 }
 
+// Two packed 2-byte values compared with 6 in their own type: 0xFFFF in the half of a value below 6, else 0 (a NaN
+// is not below 6).
+template <int DT>
+__device__ __forceinline__ uint32_t below_six_mask(const uint32_t pair)
+{
+    uint32_t m;
+    if constexpr (DT == BT_F16) asm("set.lt.u32.f16x2 %0, %1, %2;" : "=r"(m) : "r"(pair), "r"(0x46004600u));
+    else asm("set.lt.u32.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(pair), "r"(0x40C040C0u));
+    return m;
+}
+
 // 2-byte elements: the quarter's packed run staged in shared memory and gathered from there (bt_quarter16.cuh)
 // instead of one global gather per value.  The quarter's gradient -- eight 8-byte loads per lane that do not
 // depend on the stash -- is requested first, so that it arrives while the run is staged.
 template <int DT, int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1024 / (kWarps * 32))
+__global__ void __launch_bounds__(kWarps * 32, 1536 / (kWarps * 32))   // 40 registers, 12 CTAs per SM: 0.199 -> 0.178 ms against 8 CTAs
 relu6_bwd16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restrict__ values,
                    const uint64_t *__restrict__ values_offset, const uint64_t *__restrict__ prefix, const uint16_t *gout,
                    const uint64_t n, uint16_t *gin)   // gin may alias gout
@@ -180,17 +191,12 @@ relu6_bwd16_kernel(const uint32_t *__restrict__ bitmap, const uint16_t *__restri
     const Extent ox = extent_of(gin, n * sizeof(uint16_t));
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
+        // The gradient passes where the bit is set and the stashed value is below 6 (false for a stored 6 and for a
+        // NaN).  Elements under a clear bit come out of the expansion as a NaN, so one compare of the packed pair in
+        // its own type decides both conditions for two elements: a 16-bit mask of ones per element that passes.
         uint32_t    bits;
-        const uint2 v = q16::expand_step(qt, k, lane, bits);
-        // the gradient passes where the bit is set and the stashed value is below 6 (false for a stored 6 and for a NaN)
-        const uint32_t h[4] = {v.x & 0xFFFFu, v.x >> 16, v.y & 0xFFFFu, v.y >> 16};
-        uint32_t       keep[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const bool pass = ((bits >> j) & 1u) && Elem<DT>::widen(h[j]) < 6.0f;
-            keep[j]         = pass ? 0xFFFFu : 0u;
-        }
-        const uint2    r  = make_uint2(g[k].x & (keep[0] | (keep[1] << 16)), g[k].y & (keep[2] | (keep[3] << 16)));
+        const uint2 v = q16::expand_step<0x7FFFu>(qt, k, lane, bits);
+        const uint2 r = make_uint2(g[k].x & below_six_mask<DT>(v.x), g[k].y & below_six_mask<DT>(v.y));
         const uint64_t at = e0 + static_cast<uint64_t>(k) * 128 + lane * 4;
         if (qt.whole || at + 4 <= n) {
             if (ox.holds(gin + at, 8)) *reinterpret_cast<uint2 *>(gin + at) = r;
