@@ -60,8 +60,8 @@ NCU_DRAM_BYTES_PER_ELEMENT = {
     ("f16", "bt_relu_fwd_compress+y"): (4.696, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
     ("bf16", "bt_compress"): (2.847, "profiles/bt_compress_16bit_2p27_ncu_full.md"),
     ("f16", "bt_compress"): (2.847, "profiles/bt_compress_16bit_2p27_ncu_full.md (bf16 capture; same kernel)"),
-    ("bf16", "bt_decompress"): (2.779, "profiles/bt_decompress_bf16_2p27_ncu_full.md"),
-    ("f16", "bt_decompress"): (2.779, "profiles/bt_decompress_bf16_2p27_ncu_full.md (bf16 capture; same kernel)"),
+    ("bf16", "bt_decompress"): (2.710, "profiles/bt_decompress_bf16_2p27_ncu_full.md"),
+    ("f16", "bt_decompress"): (2.710, "profiles/bt_decompress_bf16_2p27_ncu_full.md (bf16 capture; same kernel)"),
     ("f32", "bt_compress"): (5.562, "profiles/bt_codec_f32_2p26_ncu_full.md"),
     ("f32", "bt_relu_fwd_compress"): (5.562, "profiles/bt_codec_f32_2p26_ncu_full.md (plain compressor; same kernel body)"),
     ("f32", "bt_decompress"): (5.308, "profiles/bt_codec_f32_2p26_ncu_full.md"),
