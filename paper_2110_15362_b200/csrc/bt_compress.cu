@@ -39,8 +39,9 @@
 //   counted[s]  every compactor has posted its count         (compactors  -> scan warps)
 //   ready[s]    base and segment offsets are in shared       (scan warp   -> copiers)
 //   empty[s]    every copier has copied its segments out     (copiers     -> load warp)
-// Copier warp c copies its segments' packed values to values[base + offset ...].
-// With a ring of 6 or 7 tiles the load warp runs several tiles ahead of the
+// Copier warp c copies its segments' packed values to values[base + offset ...]
+// (2-byte values through the copy engine, in 16-byte units: copy_out_run16).
+// With a ring of 7 tiles the load warp runs several tiles ahead of the
 // compactors and the compactors several tiles ahead of the copiers, so nobody
 // waits for a round trip to L2 or to HBM.
 //
