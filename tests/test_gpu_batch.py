@@ -246,3 +246,20 @@ def test_batch_of_two_byte_runs_at_every_offset_from_a_16_byte_boundary(oracle, 
     B.bt_compress_batch(B.batch_items(xs, sts, None), dt, ws)
     torch.cuda.synchronize()
     check_batch(oracle, kind, raws, sts, None, False)
+
+
+@pytest.mark.parametrize("kind", ["bf16", "f16"])
+@pytest.mark.parametrize("want_y", [False, True])
+def test_fused_batch_on_every_two_byte_pattern(oracle, kind, want_y):
+    """The batched fused ReLU decides in the element's own type like the single-tensor kernel: all 65536 patterns of
+    the type (shuffled, as two tensors of one batch) against the oracle."""
+    rng = np.random.default_rng(4242)
+    raws = [rng.permutation(np.arange(65536, dtype=np.uint16)), rng.permutation(np.arange(65536, dtype=np.uint16))[:40001]]
+    dt = TDT[kind]
+    xs = [from_raw(r, kind) for r in raws]
+    sts = [B.Stash(r.size, dt) for r in raws]
+    ys = [torch.empty_like(x) for x in xs] if want_y else None
+    ws = torch.empty(B.bt_batch_workspace_bytes([r.size for r in raws]), dtype=torch.uint8, device="cuda")
+    B.bt_relu_fwd_compress_batch(B.batch_items(xs, sts, ys), dt, ws)
+    torch.cuda.synchronize()
+    check_batch(oracle, kind, raws, sts, ys, True)

@@ -99,3 +99,37 @@ def test_full_size_mobilenet_layer_against_torch(G, oracle):
         _, c = oracle.relu6_fwd_compress(raw[lo:lo + 4096], "f32")
         assert np.array_equal(bmp[lo // 32:lo // 32 + 128], c.bitmap)
         assert np.array_equal(vals[int(pfx[ch]):int(pfx[ch]) + c.nnz], c.values)
+
+
+@pytest.mark.parametrize("kind", ["f16", "bf16"])
+@pytest.mark.parametrize("mode", ["stash_only", "with_y"])
+def test_every_two_byte_pattern_through_relu_and_relu6(G, oracle, kind, mode):
+    """All 65536 patterns of a 2-byte type, shuffled, through the fused ReLU, the fused ReLU6 and the ReLU6
+    backward: the decisions these take in the element's own type (kept iff greater than 0 or a NaN, saturated iff
+    at least 6, the gradient passes iff the stashed value is below 6) must agree with the oracle's comparisons of
+    the exactly widened values on every pattern -- both zeros, subnormals, 6 and its neighbours, the infinities
+    and every NaN of either sign."""
+    rng = np.random.default_rng(65536)
+    x = rng.permutation(np.arange(65536, dtype=np.uint16))
+    g = rng.permutation(np.arange(65536, dtype=np.uint16))
+    xt = G.from_raw(x, kind)
+    # ReLU
+    y_ref, c = oracle.relu_fwd_compress(x, kind)
+    r = G.gpu_compress(xt, relu=True, want_y=(mode == "with_y"))
+    assert r.guards_ok and r.status == B.BT_OK and r.nnz == c.nnz
+    assert np.array_equal(r.bitmap, c.bitmap) and np.array_equal(r.prefix, c.prefix) and np.array_equal(r.values, c.values)
+    if mode == "with_y":
+        assert np.array_equal(r.y, y_ref)
+    # ReLU6 and its backward
+    y6_ref, c6 = oracle.relu6_fwd_compress(x, kind)
+    st, y6, ok = run_fwd(G, xt, mode)
+    assert ok and st.status == B.BT_OK and st.nnz == c6.nnz
+    assert np.array_equal(W.raw_numpy(st.bitmap).view(np.uint32), c6.bitmap)
+    assert np.array_equal(W.raw_numpy(st.values[:c6.nnz]), c6.values)
+    if mode == "with_y":
+        assert np.array_equal(y6, y6_ref)
+    gt = G.from_raw(g, kind)
+    gin = G.Guarded(x.size, gt.dtype)
+    B.bt_relu6_bwd_from_stash(st.bitmap, st.values, st.chunk_prefix, gt, gin.inner)
+    torch.cuda.synchronize()
+    assert np.array_equal(gin.raw(), oracle.relu6_bwd_from_stash(c6, kind, g)) and gin.guards_intact()
